@@ -1,0 +1,427 @@
+"""Pins for the CPU oracle: each test checks it against something other than itself — a library
+routine, an independent Llama implementation, brute force, a closed form, or an invariant the
+paper fixes (Section 2.1 losslessness, Section 2.2 tree attention, metric definition of tau)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+import hf_ref
+import pyoracle as po
+from paper_2503_01840_b200 import synth
+
+C1 = synth.C1
+TOL = 2e-5
+
+
+@pytest.fixture(scope="module")
+def c1():
+    tw = synth.make_target_weights(C1)
+    dw = synth.make_draft_weights(C1)
+    ids = synth.make_prompts(C1)[0].numpy()
+    return tw, dw, ids
+
+
+def _mk(cfg, tw, dw, max_ctx=256):
+    return po.Oracle(cfg, tw, dw, max_ctx)
+
+
+# ----------------------------------------------------------------------------- building blocks
+def test_linear_vs_matmul_fp64():
+    g = torch.Generator().manual_seed(0)
+    W = torch.randn(37, 129, generator=g)
+    x = torch.randn(5, 129, generator=g)
+    ref = (x.double() @ W.double().T).numpy()
+    assert np.abs(po.linear(W, x.numpy()) - ref).max() < 1e-4
+    Wb = W.to(torch.bfloat16)
+    refb = (x.double() @ Wb.double().T).numpy()
+    assert np.abs(po.linear(Wb, x.numpy()) - refb).max() < 1e-4
+    # a transposed operand or swapped index would not survive a non-square W
+    assert po.linear(W, x.numpy()).shape == (5, 37)
+
+
+def test_linear_rows_are_independent():
+    g = torch.Generator().manual_seed(1)
+    W = torch.randn(50, 300, generator=g)
+    x = torch.randn(70, 300, generator=g).numpy()
+    full = po.linear(W, x)
+    for m in (0, 13, 69):
+        assert np.array_equal(full[m], po.linear(W, x[m:m + 1])[0])
+
+
+def test_rmsnorm_vs_torch():
+    g = torch.Generator().manual_seed(2)
+    x = torch.randn(4, 256, generator=g) * 3
+    gain = 1 + 0.1 * torch.randn(256, generator=g)
+    ref = F.rms_norm(x, (256,), gain, 1e-5).numpy()
+    assert np.abs(po.rmsnorm(gain, x.numpy(), 1e-5) - ref).max() < TOL
+
+
+def test_rope_vs_transformers():
+    from transformers.models.llama.modeling_llama import LlamaRotaryEmbedding, apply_rotary_pos_emb
+    cfg = hf_ref._cfg(C1, 1, 16)
+    rot = LlamaRotaryEmbedding(cfg)
+    g = torch.Generator().manual_seed(3)
+    H, hd = 4, 64
+    x = torch.randn(1, H, 3, hd, generator=g)
+    pos = torch.tensor([[0, 17, 1234]])
+    cos, sin = rot(x, pos)
+    ref, _ = apply_rotary_pos_emb(x, x, cos, sin)
+    for t, p in enumerate(pos[0].tolist()):
+        mine = po.rope(x[0, :, t].reshape(-1).numpy(), H, hd, p, C1.rope_theta).reshape(H, hd)
+        assert np.abs(mine - ref[0, :, t].numpy()).max() < (2e-4 if p > 1000 else 1e-5), p
+    assert np.array_equal(po.rope(x[0, :, 0].reshape(-1).numpy(), H, hd, 0, 1e4), x[0, :, 0].reshape(-1).numpy())
+
+
+def test_swiglu_vs_torch():
+    g = torch.Generator().manual_seed(4)
+    a, b = torch.randn(1000, generator=g) * 4, torch.randn(1000, generator=g)
+    assert np.abs(po.swiglu(a.numpy(), b.numpy()) - (F.silu(a) * b).numpy()).max() < TOL
+
+
+def test_attend_vs_sdpa():
+    g = torch.Generator().manual_seed(5)
+    q, K, V = torch.randn(64, generator=g), torch.randn(37, 64, generator=g), torch.randn(37, 64, generator=g)
+    ref = F.scaled_dot_product_attention(q[None, None, None], K[None, None], V[None, None])[0, 0, 0].numpy()
+    assert np.abs(po.attend(q.numpy(), K.numpy(), V.numpy()) - ref).max() < TOL
+    # a single key returns its value exactly
+    assert np.allclose(po.attend(q.numpy(), K[:1].numpy(), V[:1].numpy()), V[0].numpy())
+
+
+def test_log_softmax_topk_argmax():
+    g = torch.Generator().manual_seed(6)
+    z = torch.randn(1024, generator=g) * 2
+    lp = po.log_softmax(z.numpy())
+    assert np.abs(lp - torch.log_softmax(z, 0).numpy()).max() < TOL
+    assert abs(np.exp(lp.astype(np.float64)).sum() - 1) < 1e-5
+    idx, val, nxt = po.topk(z.numpy(), 5)
+    tv, ti = torch.topk(z, 6)
+    assert idx.tolist() == ti[:5].tolist() and np.array_equal(val, tv[:5].numpy()) and nxt == tv[5].item()
+    # ties: lowest index first
+    t = np.array([1, 3, 3, 2, 3, 0], np.float32)
+    assert po.topk(t, 3)[0].tolist() == [1, 2, 4]
+    assert po.argmax(t) == (1, 0.0)
+    assert po.argmax(np.array([0, 5, 2], np.float32)) == (1, 3.0)
+
+
+# ----------------------------------------------------------------------------- the target model
+def test_target_forward_vs_independent_llama(c1):
+    tw, dw, ids = c1
+    hf = hf_ref.target_model(C1, tw)
+    logits, blocks = hf_ref.forward(hf, torch.from_numpy(ids))
+    o = _mk(C1, tw, dw)
+    first = o.prefill(ids)
+    assert first == int(logits[-1].argmax())
+    for pos in (0, 1, 31, 63):
+        taps = o.taps(pos).reshape(3, C1.hidden)
+        for s, layer in enumerate(C1.fuse_layers):
+            assert np.abs(taps[s] - blocks[layer][pos].numpy()).max() < 1e-4, (pos, s)
+
+
+def test_greedy_vs_independent_llama(c1):
+    tw, dw, ids = c1
+    hf = hf_ref.target_model(C1, tw)
+    gen = hf.generate(torch.from_numpy(ids)[None].long(), do_sample=False, max_new_tokens=12,
+                      pad_token_id=0, eos_token_id=None)[0, len(ids):].tolist()
+    o = _mk(C1, tw, dw)
+    first = o.prefill(ids)
+    mine = [first] + o.greedy(11).tolist()
+    assert mine == gen
+
+
+def test_tree_forward_vs_independent_llama_with_4d_mask(c1):
+    """Tree attention (Section 2.2): node i sees the context and its ancestors only."""
+    tw, dw, ids = c1
+    hf = hf_ref.target_model(C1, tw)
+    o = _mk(C1, tw, dw)
+    o.prefill(ids)
+    o.step()
+    o.step()
+    # state before the last step: n0 committed; reconstruct it from the inspection arrays
+    tok, depth, mask = o.get(po.TREE_TOK), o.get(po.TREE_DEPTH), o.get(po.TREE_MASK)
+    nn = tok.size
+    n0 = o.n - len(o.get(po.PATH))
+    ctx = o.ids[:n0]
+    allids = torch.from_numpy(np.concatenate([ctx, tok]).astype(np.int64))
+    T = n0 + nn
+    vis = torch.zeros(T, T, dtype=torch.bool)
+    vis[:n0, :n0] = torch.tril(torch.ones(n0, n0, dtype=torch.bool))
+    for i in range(nn):
+        vis[n0 + i, :n0] = True
+        for j in range(nn):
+            if (int(mask[i]) >> j) & 1:
+                vis[n0 + i, n0 + j] = True
+    posid = torch.cat([torch.arange(n0), n0 + torch.from_numpy(depth.astype(np.int64))])
+    logits, blocks = hf_ref.forward(hf, allids, position_ids=posid, mask_bool=vis)
+    mine = o.get(po.TARGET_LOGITS).reshape(nn, C1.vocab)
+    assert np.abs(mine - logits[n0:].numpy()).max() < 2e-4
+    taps = o.get(po.NODE_TAPS).reshape(nn, 3, C1.hidden)
+    for s, layer in enumerate(C1.fuse_layers):
+        assert np.abs(taps[:, s] - blocks[layer][n0:].numpy()).max() < 1e-4
+
+
+# ----------------------------------------------------------------------------- the draft head
+def test_draft_passes_vs_independent_llama_layer(c1):
+    """Section 3.1: g = FC3[l;m;h]; x = FC2[g or a ; e(tok)]; decoder layer -> a; LM head.  The
+    decoder layer, norm and head come from the independent implementation; every processed tree
+    node is re-run as an ordinary causal sequence over its own ancestor path."""
+    tw, dw, ids = c1
+    hfd = hf_ref.draft_model(C1, dw)
+    o = _mk(C1, tw, dw)
+    o.prefill(ids)
+    o.step()
+    n = o.n
+    P = o.pending
+    committed = o.ids                          # [n+1], last = root
+    o.step()
+    k, K, D, Vd = C1.hidden, C1.tree_topk, C1.tree_depth, C1.draft_vocab
+    fc3, fc2, E = dw["fc3"].double(), dw["fc2"].double(), tw["embed"].double()
+    o_taps = po.Oracle(C1, tw, dw, 256)        # fresh oracle just to read taps of the committed prefix
+    o_taps.prefill(committed[:n])
+    taps = torch.from_numpy(np.stack([o_taps.taps(p) for p in range(n)])).double()
+    gfeat = taps @ fc3.T                                                # [n][k]
+    gp = o.get(po.G_PENDING).reshape(P, k)
+    assert np.abs(gp - gfeat[n - P:].numpy()).max() < 1e-4
+    x_ctx = torch.cat([gfeat, E[torch.from_numpy(committed[1:n + 1].astype(np.int64))]], 1) @ fc2.T   # entries 0..n-1
+    logits_ctx, blocks = hf_ref.forward(hfd, embeds=x_ctx.float())
+    dl = o.get(po.DRAFT_LOGITS).reshape(D, K, Vd)
+    da = o.get(po.DRAFT_A).reshape(D, K, k)
+    assert np.abs(dl[0, 0] - logits_ctx[-1].numpy()).max() < 2e-4
+    assert np.abs(da[0, 0] - blocks[0][-1].numpy()).max() < 2e-4
+    # tree passes: node u at depth d-1 fed with (a of its parent, e(tok_u)) after the context
+    front = o.get(po.FRONTIER).reshape(D, K)
+    ptok, ppar = o.get(po.POOL_TOK), o.get(po.POOL_PARENT)
+    a_of = {0: torch.from_numpy(da[0, 0]).double()}
+    for d in range(1, D):
+        for r in range(K):
+            a_of[int(front[d, r])] = torch.from_numpy(da[d, r]).double()
+    checked = 0
+    for d in range(1, D):
+        for r in range(K):
+            u = int(front[d, r])
+            chain = []
+            v = u
+            while v != 0:
+                chain.append(v)
+                v = int(ppar[v])
+            chain.reverse()
+            rows = [torch.cat([a_of[int(ppar[v])], E[int(ptok[v])]]) @ fc2.T for v in chain]
+            x = torch.cat([x_ctx, torch.stack(rows)], 0)
+            lg, bl = hf_ref.forward(hfd, embeds=x.float())
+            assert np.abs(dl[d, r] - lg[-1].numpy()).max() < 3e-4, (d, r)
+            assert np.abs(da[d, r] - bl[0][-1].numpy()).max() < 3e-4
+            checked += 1
+    assert checked == (D - 1) * K
+
+
+# ----------------------------------------------------------------------------- tree construction
+def _check_tree(o, cfg):
+    K, D, N = cfg.tree_topk, cfg.tree_depth, cfg.tree_nodes
+    tok, par, dep, mask = (o.get(w) for w in (po.TREE_TOK, po.TREE_PARENT, po.TREE_DEPTH, po.TREE_MASK))
+    pidx, sc = o.get(po.TREE_POOLIDX), o.get(po.TREE_SCORE)
+    pscore, ppar, ptok = o.get(po.POOL_SCORE), o.get(po.POOL_PARENT), o.get(po.POOL_TOK)
+    pool = cfg.pool
+    nn = tok.size
+    assert nn == min(N - 1, pool) + 1
+    # masks == brute-force ancestor sets
+    for i in range(nn):
+        anc, v = set(), i
+        while v != -1:
+            anc.add(v)
+            v = int(par[v])
+        assert int(mask[i]) == sum(1 << a for a in anc)
+        assert bin(int(mask[i])).count("1") == dep[i] + 1
+        assert int(mask[i]) < (1 << (i + 1)) and (int(mask[i]) >> i) & 1
+        if i:
+            assert par[i] < i and dep[i] == dep[par[i]] + 1
+            assert sc[i] <= sc[par[i]]
+    # selection == stable sort of the pool by (-score, index); ancestor-closed by construction of that order
+    order = sorted(range(1, pool + 1), key=lambda i: (-float(pscore[i]), i))
+    chosen = sorted(order[: nn - 1])
+    assert pidx[1:].tolist() == chosen
+    sel = set(chosen) | {0}
+    assert all(int(ppar[i]) in sel for i in chosen)
+    if 0 < nn - 1 < pool:
+        assert min(float(pscore[i]) for i in chosen) >= max(float(pscore[i]) for i in range(1, pool + 1) if i not in sel)
+    # siblings carry distinct tokens (d2t is injective), so the accepted path is unique
+    for p in range(nn):
+        kids = [int(tok[c]) for c in range(1, nn) if par[c] == p]
+        assert len(kids) == len(set(kids))
+    # frontier of pass d = K best children of level d (score desc, pool index asc), all children of the previous frontier
+    front = o.get(po.FRONTIER).reshape(D, K)
+    assert front[0, 0] == 0
+    if D > 1:
+        assert front[1].tolist() == list(range(1, K + 1))
+    for d in range(2, D):
+        base = K + (d - 2) * K * K
+        kids = list(range(base + 1, base + K * K + 1))
+        best = sorted(kids, key=lambda i: (-float(pscore[i]), i))[:K]
+        assert front[d].tolist() == best
+        assert all(int(ppar[i]) in set(front[d - 1].tolist()) for i in best)
+    # pool layout: children of frontier rank r of pass d
+    for d in range(2, D + 1):
+        base = K + (d - 2) * K * K
+        for r in range(K):
+            u = int(front[d - 1, r])
+            for c in range(K):
+                ci = base + r * K + c + 1
+                assert ppar[ci] == u
+                if c:
+                    assert pscore[ci] <= pscore[ci - 1]
+    return nn
+
+
+@pytest.mark.parametrize("K,D,N", [(4, 3, 16), (1, 3, 4), (2, 4, 9), (3, 2, 64), (4, 1, 16), (5, 3, 1)])
+def test_tree_invariants_and_losslessness(c1, K, D, N):
+    """Section 2.1 / 'Metrics': strict acceptance leaves the output unchanged, so at temperature 0
+    the emitted tokens equal plain greedy decoding, whatever tree was drafted."""
+    tw, dw, ids = c1
+    cfg = C1.replace(tree_topk=K, tree_depth=D, tree_nodes=N)
+    o = _mk(cfg, tw, dw)
+    first = o.prefill(ids)
+    out = []
+    for _ in range(12):
+        n_before = o.n
+        r = o.step()
+        assert 1 <= len(r) <= D + 1                       # tau counts the bonus token
+        assert o.n == n_before + len(r) and o.pending == len(r)
+        nn = _check_tree(o, cfg)
+        if K == 1:
+            assert nn == min(N, D + 1)
+            assert o.get(po.TREE_PARENT).tolist() == list(range(-1, nn - 1))   # a chain
+        out += r.tolist()
+    ref = _mk(cfg, tw, dw)
+    assert ref.prefill(ids) == first
+    assert ref.greedy(len(out)).tolist() == out
+
+
+def test_output_invariant_to_draft_weights(c1):
+    tw, dw, ids = c1
+    dw2 = synth.make_draft_weights(C1, seed=123)
+    outs = []
+    for d in (dw, dw2):
+        o = _mk(C1, tw, d)
+        o.prefill(ids)
+        acc = []
+        while len(acc) < 16:
+            acc += o.step().tolist()
+        outs.append(acc[:16])
+    assert outs[0] == outs[1]
+
+
+def test_tree_forward_equals_per_path_sequential_bitwise(c1):
+    """Tree attention == running each root-to-node path as an ordinary causal sequence."""
+    tw, dw, ids = c1
+    o = _mk(C1, tw, dw)
+    o.prefill(ids)
+    o.step()
+    base_ids, n0 = o.ids, o.n
+    o.step()
+    tok, par = o.get(po.TREE_TOK), o.get(po.TREE_PARENT)
+    dep, y = o.get(po.TREE_DEPTH), o.get(po.Y)
+    taps = o.get(po.NODE_TAPS).reshape(tok.size, -1)
+    for i in range(tok.size):
+        chain, v = [], i
+        while v != -1:
+            chain.append(int(tok[v]))
+            v = int(par[v])
+        chain.reverse()                                   # root .. node i
+        seq = np.concatenate([base_ids[:n0], np.array(chain, np.int32)])
+        s = _mk(C1, tw, dw)
+        nxt = s.prefill(seq)
+        assert nxt == y[i]
+        assert np.array_equal(s.taps(n0 + dep[i]), taps[i])          # bit-identical
+
+
+def test_commit_equals_fresh_prefill(c1):
+    tw, dw, ids = c1
+    tws, dws, pi, pi2 = synth.make_structured(C1, 0.8, residual_scale=0.05)
+    prompt = synth.structured_prompt(C1, dws["d2t"], 40).numpy()
+    for (t, d, p) in ((tw, dw, ids), (tws, dws, prompt)):
+        o = _mk(C1, t, d)
+        o.prefill(p)
+        for _ in range(5):
+            o.step()
+        f = _mk(C1, t, d)
+        f.prefill(o.ids[: o.n])
+        assert f.ids[o.n] == o.ids[o.n]
+        for pos in range(o.n):
+            assert np.array_equal(o.taps(pos), f.taps(pos))
+            for l in range(C1.n_layers):
+                ka, va = o.target_kv(l, pos); kb, vb = f.target_kv(l, pos)
+                assert np.array_equal(ka, kb) and np.array_equal(va, vb)
+        for pos in range(o.n - o.pending):
+            ka, va = o.draft_kv(pos); kb, vb = f.draft_kv(pos)
+            assert np.array_equal(ka, kb) and np.array_equal(va, vb)
+
+
+def test_force_state_matches_stepping(c1):
+    tw, dw, ids = c1
+    a = _mk(C1, tw, dw)
+    a.prefill(ids)
+    for _ in range(3):
+        a.step()
+    b = _mk(C1, tw, dw)
+    b.prefill(ids[:20])
+    b.step()
+    b.force_state(a.ids, a.n, a.pending)
+    assert a.step().tolist() == b.step().tolist()
+    for w in (po.TREE_TOK, po.TREE_PARENT, po.TREE_MASK, po.TARGET_LOGITS, po.DRAFT_LOGITS):
+        assert np.array_equal(a.get(w), b.get(w))
+
+
+# ----------------------------------------------------------------------------- acceptance > 0, closed form
+@pytest.mark.parametrize("p_agree", [1.0, 0.8, 0.5])
+def test_structured_weights_closed_form_counts(p_agree):
+    """With zero W_o / W_down the target emits the pi-orbit of the root and the draft proposes pi2
+    of every token, so count = 1 + (run of pi == pi2 along the orbit, capped at D)."""
+    cfg = C1
+    tw, dw, pi, pi2 = synth.make_structured(cfg, p_agree, residual_scale=0.0)
+    prompt = synth.structured_prompt(cfg, dw["d2t"], 24, seed=int(p_agree * 10)).numpy()
+    o = _mk(cfg, tw, dw)
+    root = o.prefill(prompt)
+    assert root == int(pi[int(prompt[-1])])
+    seen_multi = False
+    for _ in range(10):
+        cur, run = root, 0
+        while run < cfg.tree_depth and int(pi[cur]) == int(pi2[cur]):
+            cur = int(pi[cur]); run += 1
+        expect, cur = [], root
+        for _ in range(run + 1):
+            cur = int(pi[cur]); expect.append(cur)
+        got = o.step().tolist()
+        assert got == expect
+        seen_multi |= len(got) > 1
+        root = got[-1]
+    assert seen_multi
+
+
+def test_accept_walk_unit():
+    #        0
+    #      1   2
+    #     3 4   5
+    tok = [7, 10, 11, 20, 21, 30]
+    par = [-1, 0, 0, 1, 1, 2]
+    cnt, path, out = po.accept(tok, par, [10, 21, 0, 0, 99, 0])
+    assert (cnt, path.tolist(), out.tolist()) == (3, [0, 1, 4], [10, 21, 99])
+    cnt, path, out = po.accept(tok, par, [12, 0, 0, 0, 0, 0])
+    assert (cnt, path.tolist(), out.tolist()) == (1, [0], [12])
+    cnt, path, out = po.accept(tok, par, [11, 0, 30, 0, 0, 5])
+    assert (cnt, path.tolist(), out.tolist()) == (3, [0, 2, 5], [11, 30, 5])
+
+
+def test_rerank_unit_ties_and_closure():
+    # pool: 1,2 children of root; 3,4 children of 1; 5,6 children of 2; log-prob 0 children tie with parents
+    score = np.array([0, -0.5, -1.0, -0.5, -2.0, -1.0, -1.0], np.float32)
+    parent = np.array([-1, 0, 0, 1, 1, 2, 2], np.int32)
+    tok = np.arange(100, 107, dtype=np.int32)
+    depth = np.array([0, 1, 1, 2, 2, 2, 2], np.int32)
+    r = po.rerank(score, parent, tok, depth, 5, 100)
+    assert r["poolidx"].tolist() == [0, 1, 2, 3, 5]      # ties resolved toward the lower index (parent first)
+    assert r["parent"].tolist() == [-1, 0, 0, 1, 2]
+    assert r["mask"].tolist() == [1, 3, 5, 11, 21]
+    assert r["cut_margin"] == 0.0
+    r = po.rerank(score, parent, tok, depth, 64, 100)
+    assert r["n"] == 7 and math.isinf(r["cut_margin"])
