@@ -1,0 +1,200 @@
+/*
+ * spec_b200.h — C ABI of the B200 (sm_100a) EAGLE-3 speculative-step library.
+ *
+ * One speculative step = drafting (feature fusion, draft decoder layer, reduced-vocabulary LM head,
+ * dynamic draft tree) followed by verification (one tree-masked target forward, greedy acceptance,
+ * KV-cache compaction).  The operations follow the EAGLE-3 paper: Section 2.1 (draft / verify
+ * alternation and the acceptance rule), Section 2.2 (tree drafts, tree attention, the dynamic tree
+ * with end-of-draft pruning), Section 3.1 (the inference pipeline: l/m/h fusion, g/a + embedding
+ * through an FC layer into one decoder layer, LM head), Appendix A (tree depth, total draft tokens,
+ * nodes per expansion).
+ *
+ * Conventions
+ *   - Every function returns 0 on success and a negative spec_status otherwise; nothing aborts or
+ *     throws.  spec_last_error() gives a static, human-readable string for the last failure of a ctx
+ *     (or of spec_init when ctx is NULL).
+ *   - "device" pointers are CUDA device memory of the current device, "host" pointers ordinary host
+ *     memory.  All matrices are row-major [out][in]; dtype is cfg.dtype for weights and caches.
+ *   - The caller owns weights, workspace and stream; they are borrowed from spec_init to spec_free.
+ *     Weights are never written; the workspace is written only by this library while the ctx lives.
+ *   - The library allocates no device memory except where a function says so.
+ */
+#ifndef SPEC_B200_H
+#define SPEC_B200_H
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct spec_ctx spec_ctx;
+
+enum spec_status {
+  SPEC_OK = 0,
+  SPEC_ERR_INVALID_CFG = -1,     /* a cfg field is out of range (message names it)                    */
+  SPEC_ERR_NULL = -2,            /* a required pointer is NULL                                        */
+  SPEC_ERR_WORKSPACE = -3,       /* workspace too small or misaligned (256 B)                         */
+  SPEC_ERR_CAPACITY = -4,        /* a sequence would outgrow max_ctx / its pages; state is unchanged  */
+  SPEC_ERR_STATE = -5,           /* call order: step before prefill, etc.                             */
+  SPEC_ERR_CUDA = -6,            /* a CUDA runtime/driver call failed                                 */
+  SPEC_ERR_DEVICE_STATUS = -7,   /* a kernel reported a bounded-wait timeout or a failed bounds check */
+  SPEC_ERR_UNSUPPORTED = -8
+};
+
+enum spec_dtype { SPEC_F32 = 0, SPEC_BF16 = 1 };
+
+/* cfg.flags */
+enum {
+  SPEC_FLAG_REF_GEMM = 1,        /* use the plain CUDA-core GEMM kernel also for bf16 (debugging aid)   */
+  SPEC_FLAG_REF_ATTN = 2,        /* use the plain CUDA-core attention kernel also for bf16             */
+  SPEC_FLAG_CAPTURE = 4,         /* keep per-pass draft logits / features for spec_debug_read          */
+  SPEC_FLAG_NO_GRAPH = 8         /* launch kernels one by one instead of replaying a CUDA graph        */
+};
+
+/* Target model weights (Section 3.1: the frozen target whose layers are tapped).  Device pointers;
+ * the per-layer members are HOST arrays of n_layers device pointers. */
+typedef struct {
+  const void *embed;        /* [vocab][hidden]                       */
+  const void *final_norm;   /* [hidden]                              */
+  const void *lm_head;      /* [vocab][hidden]                       */
+  const void *const *attn_norm, *const *wq, *const *wk, *const *wv, *const *wo;
+  const void *const *mlp_norm, *const *w_gate, *const *w_up, *const *w_down;
+} spec_target_weights;
+
+/* Draft head (Section 3.1): fc3 fuses [l;m;h] (3k -> k); fc2 maps [g or a ; e(token)] (2k -> k);
+ * one decoder layer of the target's shape; final norm; LM head over the draft vocabulary;
+ * d2t[i] = target id of draft id i, strictly increasing. */
+typedef struct {
+  const void *fc3, *fc2, *attn_norm, *wq, *wk, *wv, *wo, *mlp_norm, *w_gate, *w_up, *w_down,
+             *final_norm, *lm_head;
+  const int32_t *d2t;       /* device, [draft_vocab] */
+} spec_draft_weights;
+
+typedef struct {
+  int32_t dtype;            /* spec_dtype: storage type of weights, activations fed to GEMMs, KV cache */
+  int32_t n_layers, hidden, n_heads, n_kv_heads, head_dim, ffn, vocab, draft_vocab;
+  int32_t fuse_layers[3];   /* taps = residual stream after block i (0-based): low, mid, high          */
+  float rope_theta, rms_eps;
+  int32_t batch;            /* sequences advanced together by one spec_step                            */
+  int32_t max_ctx;          /* largest committed length + tree any sequence may reach                  */
+  int32_t page_size;        /* KV tokens per page (16 in the paper-shaped workloads)                   */
+  int32_t num_pages;        /* pages in the pool shared by all sequences                               */
+  int32_t page_shuffle_seed;/* 0: pages handed out in index order; else a seeded shuffle of the pool   */
+  int32_t tree_depth;       /* D: draft passes per step (Appendix A: "depth")                          */
+  int32_t tree_topk;        /* K: nodes kept per expansion                                            */
+  int32_t tree_nodes;       /* N: verified nodes including the root, <= 64                             */
+  int32_t flags;
+  void *workspace;          /* device, 256-byte aligned, spec_workspace_bytes(cfg) bytes               */
+  size_t workspace_bytes;
+  void *stream;             /* cudaStream_t on which every kernel is launched                          */
+} spec_cfg;
+
+/* Bytes of device workspace the ctx needs for this cfg (0 if the cfg is invalid). Pure host code. */
+size_t spec_workspace_bytes(const spec_cfg *cfg);
+
+/* Validates cfg, carves the workspace (KV pages, page tables, draft cache, tree buffers, counters),
+ * builds TMA descriptors.  Launches only small set-up kernels.  On failure *out is NULL. */
+int spec_init(spec_ctx **out, const spec_target_weights *tw, const spec_draft_weights *dw, const spec_cfg *cfg);
+
+/* Prefill (Section 3.1, "prefill phase"): target forward over each prompt, filling the paged KV cache
+ * and the three tapped feature streams, the first generated token (argmax at the last position), and
+ * the draft head's own cache for all but the last position.
+ *   prompt_ids  host, all prompts concatenated; prompt_lens host [batch]; reserve_tokens: tokens each
+ *   sequence may still generate (pages for prompt + reserve + tree are taken now);
+ *   first_ids   host [batch], out: the root token of the first step.
+ * Synchronises the stream before returning. */
+int spec_prefill(spec_ctx *ctx, const int32_t *prompt_ids, const int32_t *prompt_lens, int32_t reserve_tokens,
+                 int32_t *first_ids);
+
+/* One speculative step for every sequence (Sections 2.1, 2.2, 3.1).
+ *   out_ids    host [batch][tree_depth+1]: accepted draft tokens followed by the target's own token
+ *   out_counts host [batch]: tokens emitted, 1..tree_depth+1 (the paper's per-cycle acceptance length)
+ * Synchronises the stream.  SPEC_ERR_CAPACITY leaves every sequence unchanged. */
+int spec_step(spec_ctx *ctx, int32_t *out_ids, int32_t *out_counts);
+
+/* Same step without synchronisation: results go to DEVICE buffers dev_ids [batch][tree_depth+1] and
+ * dev_counts [batch] (either may be NULL).  Capacity is checked against an upper bound of the
+ * committed lengths (each async step may add tree_depth+1). */
+int spec_step_async(spec_ctx *ctx, int32_t *dev_ids, int32_t *dev_counts);
+
+/* Plain greedy decoding of the target on the same kernels (the paper's "vanilla" baseline): one target
+ * forward per token for every sequence, draft untouched.  out_ids host [batch]. Synchronises. */
+int spec_plain_step(spec_ctx *ctx, int32_t *out_ids);
+
+/* Committed length of every sequence (host [batch]); synchronises. */
+int spec_lengths(spec_ctx *ctx, int32_t *lens);
+
+/* Number of kernels one spec_step launches (for launch accounting). */
+int spec_launches_per_step(const spec_ctx *ctx);
+
+/* Algorithmic HBM bytes of one step at the current committed lengths: every weight once per pass,
+ * target and draft KV once (Section 4.3's "memory accesses"); synchronises to read the lengths. */
+int spec_step_bytes(spec_ctx *ctx, double *bytes);
+
+int spec_free(spec_ctx *ctx);
+const char *spec_last_error(const spec_ctx *ctx);
+
+/* ---- inspection for parity tests (synchronises; copies to host) ----------------------------- */
+enum spec_debug_what {
+  SPEC_DBG_TREE_TOK = 1,     /* int32 [nodes]            */
+  SPEC_DBG_TREE_PARENT,      /* int32 [nodes], root -1   */
+  SPEC_DBG_TREE_DEPTH,       /* int32 [nodes]            */
+  SPEC_DBG_TREE_MASK,        /* uint64 [nodes]           */
+  SPEC_DBG_TREE_POOLIDX,     /* int32 [nodes]            */
+  SPEC_DBG_TREE_SCORE,       /* float [nodes]            */
+  SPEC_DBG_Y,                /* int32 [nodes]            */
+  SPEC_DBG_TARGET_LOGITS,    /* float [nodes][vocab]     */
+  SPEC_DBG_NODE_TAPS,        /* float [nodes][3*hidden] (widened from the storage dtype) */
+  SPEC_DBG_NODE_HIDDEN,      /* float [nodes][hidden] residual stream after the last block */
+  SPEC_DBG_DRAFT_LOGITS,     /* float [D][K][draft_vocab]; needs SPEC_FLAG_CAPTURE      */
+  SPEC_DBG_DRAFT_A,          /* float [D][K][hidden];      needs SPEC_FLAG_CAPTURE      */
+  SPEC_DBG_POOL_TOK,         /* int32 [pool+1]           */
+  SPEC_DBG_POOL_SCORE,       /* float [pool+1]           */
+  SPEC_DBG_POOL_PARENT,      /* int32 [pool+1]           */
+  SPEC_DBG_FRONTIER,         /* int32 [D][K]             */
+  SPEC_DBG_PATH,             /* int32 [count]            */
+  SPEC_DBG_STATUS,           /* int32 [4] device status words */
+  SPEC_DBG_PAGE_TABLE        /* int32 [pages of seq]     */
+};
+/* Copies up to `bytes` of item `what` of sequence `seq` (last step) to host_dst; returns bytes
+ * available (>= 0) or a negative status. */
+int64_t spec_debug_read(spec_ctx *ctx, int32_t what, int32_t seq, void *host_dst, size_t bytes);
+/* K/V of a committed position as floats: k,v host [n_kv_heads*head_dim]; layer -1 = draft cache. */
+int spec_debug_read_kv(spec_ctx *ctx, int32_t seq, int32_t layer, int32_t pos, float *k, float *v);
+
+/* ---- single kernels on caller-provided DEVICE buffers, for per-kernel parity tests and timing ---
+ * Each launches on `stream` and does not synchronise.  dtype as spec_dtype. */
+
+/* out[r][o] = sum_i x[r][i] * w[o][i]; x [rows][in] dtype, w [out][in] dtype, out fp32 [rows][ldo]
+ * (first `out` columns).  impl 0: tcgen05/TMEM kernel (bf16 only), 1: plain CUDA-core kernel.
+ * scratch: device fp32 buffer of spec_gemm_scratch_bytes(rows, out, in) bytes for split-K partial
+ * sums (may be NULL when that size is 0). */
+size_t spec_gemm_scratch_bytes(int32_t rows, int32_t out, int32_t in);
+int spec_gemm(int32_t dtype, int32_t impl, const void *x, const void *w, float *out_f32, int32_t rows, int32_t out,
+              int32_t in, int32_t ldo, void *scratch, void *stream);
+
+/* Tree-masked paged GQA attention (Section 2.2 "tree attention") for `rows` query rows of one or
+ * more sequences.  q [rows][H][hd] dtype; K/V pools [num_pages][G][page_size][hd] dtype;
+ * page_table int32 [n_seq][pages_per_seq]; per row: seq, ctx_len (positions 0..ctx_len-1 all visible),
+ * tail_base (first tail position), mask lo/hi (bit t: tail position tail_base+t visible);
+ * out [rows][H][hd] dtype.  impl 0: tensor-core kernel (bf16), 1: plain kernel.
+ * scratch: spec_attn_scratch_bytes(...) bytes of device memory for split-KV partial results. */
+size_t spec_attn_scratch_bytes(int32_t rows, int32_t n_heads, int32_t head_dim, int32_t max_ctx);
+int spec_attention(int32_t dtype, int32_t impl, const void *q, const void *k_pool, const void *v_pool,
+                   const int32_t *page_table, int32_t pages_per_seq, int32_t page_size, const int32_t *row_seq,
+                   const int32_t *row_ctx, const int32_t *row_tail_base, const uint64_t *row_mask_lo,
+                   const uint64_t *row_mask_hi, int32_t tail_len, void *out, int32_t rows, int32_t n_heads,
+                   int32_t n_kv_heads, int32_t head_dim, int32_t max_ctx, void *scratch, void *stream);
+
+/* Per-row log-softmax + top-K (value desc, index asc) over fp32 logits [rows][n]: the expansion
+ * step of the dynamic tree.  out_idx int32 [rows][K], out_lp float [rows][K]. */
+int spec_logsoftmax_topk(const float *logits, int32_t rows, int32_t n, int32_t K, int32_t *out_idx, float *out_lp,
+                         void *stream);
+/* Per-row argmax (lowest index on ties) over fp32 [rows][n]. */
+int spec_argmax(const float *logits, int32_t rows, int32_t n, int32_t *out_idx, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -494,17 +494,22 @@ int orc_prefill(orc_ctx *c, const int32_t *ids, int32_t n, int32_t *first_id) {
   return 0;
 }
 
-int orc_greedy(orc_ctx *c, int32_t gen, int32_t *out) {
+int orc_greedy_margins(orc_ctx *c, int32_t gen, int32_t *out, float *margins) {
   if (c->n + gen + 1 > c->cfg.max_ctx) return -1;
+  float *lg = (float *)xcalloc((size_t)c->cfg.vocab, 4);
   for (int i = 0; i < gen; i++) {
-    int32_t y = 0;
-    target_extend(c, c->n, c->n + 1, &y, NULL);   /* forwards ids[n] at position n */
+    float mg = 0.0f;
+    target_extend(c, c->n, c->n + 1, NULL, lg);   /* forwards ids[n] at position n */
+    int32_t y = orc_argmax(lg, c->cfg.vocab, &mg);
     c->n += 1;
     c->ids[c->n] = y;
     out[i] = y;
+    if (margins) margins[i] = mg;
   }
+  free(lg);
   return 0;
 }
+int orc_greedy(orc_ctx *c, int32_t gen, int32_t *out) { return orc_greedy_margins(c, gen, out, NULL); }
 
 int orc_force_state(orc_ctx *c, const int32_t *ids, int32_t n, int32_t P) {
   if (n < 1 || P < 1 || P > n || n + c->cfg.tree_nodes > c->cfg.max_ctx) return -1;

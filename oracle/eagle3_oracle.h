@@ -65,6 +65,8 @@ int orc_step(orc_ctx *, int32_t *out_ids, int32_t *count);
 /* Plain greedy autoregressive decoding of the target (the paper's "vanilla" baseline): continue the
  * current state by `gen` tokens, one target forward per token.  Needs a prefilled ctx. */
 int orc_greedy(orc_ctx *, int32_t gen, int32_t *out_ids);
+/* same, also reporting the top1 - top2 logit gap of every emitted token */
+int orc_greedy_margins(orc_ctx *, int32_t gen, int32_t *out_ids, float *margins);
 
 /* Put the ctx into the state "ids[0..n-1] committed, ids[n] is the root, P pending entries",
  * recomputing whatever the current caches do not already hold (common prefix is kept). */

@@ -60,6 +60,7 @@ def lib():
         L.orc_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
         L.orc_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_greedy.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+        L.orc_greedy_margins.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.orc_force_state.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32]
         L.orc_n.argtypes = [C.c_void_p]
         L.orc_pending.argtypes = [C.c_void_p]
@@ -269,6 +270,13 @@ class Oracle:
         if lib().orc_greedy(self.h, gen, _p(out)):
             raise RuntimeError("orc_greedy failed")
         return out
+
+    def greedy_margins(self, gen: int):
+        out = np.zeros(gen, np.int32)
+        mg = np.zeros(gen, np.float32)
+        if lib().orc_greedy_margins(self.h, gen, _p(out), _p(mg)):
+            raise RuntimeError("orc_greedy failed")
+        return out, mg
 
     def force_state(self, ids, n: int, P: int):
         ids = _np(ids, np.int32)

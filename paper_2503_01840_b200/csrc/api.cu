@@ -1,0 +1,803 @@
+// C ABI of the speculative-step library: configuration checks, workspace carving, the kernel
+// schedule of prefill / spec_step / plain decode, and the inspection entry points.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <string>
+#include <vector>
+
+#include "../../include/spec_b200.h"
+#include "gemm_fast.cuh"
+#include "attn_fast.cuh"
+#include "state.cuh"
+
+using namespace spec;
+
+namespace spec {
+void launch_logsoftmax_topk_rows(const float *logits, const int32_t *src_row, int rows, int n, int K, int32_t *idx,
+                                 float *lp, cudaStream_t s);
+
+// dst row b*dst_stride_rows <- src row src_row[b] (fp32, `width` columns); rows with src_row < 0 are skipped
+__global__ void gather_rows_kernel(const float *__restrict__ src, const int32_t *__restrict__ src_row,
+                                   float *__restrict__ dst, int width, int dst_stride_rows) {
+  int b = blockIdx.x, sr = src_row[b];
+  if (sr < 0) return;
+  for (int i = threadIdx.x; i < width; i += blockDim.x)
+    dst[(size_t)b * dst_stride_rows * width + i] = src[(size_t)sr * width + i];
+}
+static void launch_gather_rows(const float *src, const int32_t *src_row, float *dst, int B, int width, int dst_stride_rows,
+                               cudaStream_t s) {
+  gather_rows_kernel<<<B, 256, 0, s>>>(src, src_row, dst, width, dst_stride_rows);
+}
+}
+
+static char g_init_err[256] = "";
+
+struct LayerW {
+  const void *attn_norm, *wq, *wk, *wv, *wo, *mlp_norm, *w_gate, *w_up, *w_down;
+};
+
+// Bump allocator over the caller's workspace; with base == nullptr it only measures.
+struct Carver {
+  char *base;
+  size_t off = 0;
+  explicit Carver(void *b) : base((char *)b) {}
+  template <typename U> U *take(size_t n) {
+    off = (off + 255) & ~(size_t)255;
+    U *p = base ? (U *)(base + off) : nullptr;
+    off += n * sizeof(U);
+    return p;
+  }
+  void *take_bytes(size_t n) { return take<char>(n); }
+};
+
+struct spec_ctx {
+  spec_cfg cfg;
+  cudaStream_t stream;
+  int B, L, k, H, G, hd, F, V, Vd, D, K, N, Pmax, pool, esz;
+  int Te, Td, Tv, R, Ralloc, pps, tail_tree, need_pos;
+  std::vector<LayerW> tl;
+  LayerW dl;
+  const void *embed, *final_norm, *lm_head, *fc3, *fc2, *dfinal_norm, *dlm_head;
+  const int32_t *d2t;
+  // device buffers
+  float *x, *proj, *qkv, *gu, *logits;
+  void *h, *q, *ao, *act, *cat, *node_taps, *pend_taps;
+  float2 *cs;
+  double *inv_freq;
+  RowMeta meta;
+  std::vector<KvPool> pools;   // [L] target, [L] = draft
+  KvPool *pools_dev;
+  int32_t *page_table;
+  SeqState st;
+  TreeBufs tb;
+  int32_t *status;
+  float *cap_logits, *cap_a;   // capture buffers (SPEC_FLAG_CAPTURE)
+  void *gemm_scratch;
+  size_t gemm_scratch_bytes;
+  void *attn_scratch;
+  size_t attn_scratch_bytes;
+  // split-K bookkeeping of the last GEMM into each buffer
+  int np_proj = 1, np_qkv = 1, np_gu = 1;
+  size_t ps_proj = 0, ps_qkv = 0, ps_gu = 0;
+  int smax_proj, smax_qkv, smax_gu;
+  // host mirrors
+  std::vector<int32_t> n_upper, cap_host, n_pages_host;
+  std::vector<int32_t> page_table_host;
+  bool prefilled = false, draft_stale = false;
+  cudaGraphExec_t graph = nullptr;
+  int launches = 0, launches_graph = 0;
+  int sched_err = 0;
+  FastGemm *fg = nullptr;
+  char err[256];
+};
+
+static int fail(spec_ctx *c, int code, const char *fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(c ? c->err : g_init_err, 256, fmt, ap);
+  va_end(ap);
+  return code;
+}
+#define CUDA_TRY(c, call)                                                                       \
+  do {                                                                                          \
+    cudaError_t e_ = (call);                                                                    \
+    if (e_ != cudaSuccess) return fail(c, SPEC_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+static const char *check_cfg(const spec_cfg *c) {
+  if (c->dtype != SPEC_F32 && c->dtype != SPEC_BF16) return "dtype must be 0 (fp32) or 1 (bf16)";
+  if (c->n_layers < 1 || c->n_layers > 1024) return "n_layers out of range";
+  if (c->hidden < 16 || c->hidden % 8) return "hidden must be a positive multiple of 8";
+  if (c->n_heads < 1 || c->n_kv_heads < 1 || c->n_heads % c->n_kv_heads) return "n_heads must be a multiple of n_kv_heads";
+  if (c->head_dim < 16 || c->head_dim > 256 || c->head_dim % 16) return "head_dim must be a multiple of 16 in [16,256]";
+  if (c->ffn < 8 || c->ffn % 8) return "ffn must be a positive multiple of 8";
+  if (c->vocab < 2 || c->draft_vocab < 1 || c->draft_vocab > c->vocab) return "vocab / draft_vocab out of range";
+  for (int i = 0; i < 3; i++)
+    if (c->fuse_layers[i] < 0 || c->fuse_layers[i] >= c->n_layers) return "fuse_layers must index target layers";
+  if (!(c->rope_theta > 1.0f) || !(c->rms_eps > 0.0f)) return "rope_theta must exceed 1 and rms_eps must be positive";
+  if (c->batch < 1 || c->batch > 4096) return "batch out of range";
+  if (c->tree_depth < 1 || c->tree_depth > 16) return "tree_depth must be in [1,16]";
+  if (c->tree_topk < 1 || c->tree_topk > 16 || c->tree_topk > c->draft_vocab) return "tree_topk must be in [1,16] and <= draft_vocab";
+  if (c->tree_nodes < 1 || c->tree_nodes > 64) return "tree_nodes must be in [1,64]";
+  if ((c->tree_depth - 1) * c->tree_topk > 128) return "(tree_depth-1)*tree_topk must be <= 128 (draft ancestor mask)";
+  if (c->tree_topk + (c->tree_depth - 1) * c->tree_topk * c->tree_topk > 1023) return "candidate pool must be <= 1023";
+  if (c->page_size < 1 || c->page_size > 256 || (c->page_size & (c->page_size - 1))) return "page_size must be a power of two <= 256";
+  if (c->max_ctx < 2 || c->max_ctx > (1 << 22)) return "max_ctx out of range";
+  if (c->num_pages < 1) return "num_pages must be positive";
+  return nullptr;
+}
+
+// Derives sizes and carves every buffer; with c->cfg.workspace == nullptr (measure mode) only sizes.
+static size_t carve(spec_ctx *c, void *base) {
+  const spec_cfg &g = c->cfg;
+  c->B = g.batch; c->L = g.n_layers; c->k = g.hidden; c->H = g.n_heads; c->G = g.n_kv_heads; c->hd = g.head_dim;
+  c->F = g.ffn; c->V = g.vocab; c->Vd = g.draft_vocab; c->D = g.tree_depth; c->K = g.tree_topk; c->N = g.tree_nodes;
+  c->Pmax = c->D + 1;
+  c->pool = c->K + (c->D - 1) * c->K * c->K;
+  c->esz = g.dtype == SPEC_F32 ? 4 : 2;
+  c->Te = c->B * c->Pmax; c->Td = c->B * c->K; c->Tv = c->B * c->N;
+  c->R = std::max(std::max(c->Te, c->Td), std::max(c->Tv, 64));
+  c->Ralloc = (c->R + 63) / 64 * 64;
+  c->pps = (g.max_ctx + g.page_size - 1) / g.page_size;
+  c->tail_tree = std::max(1, (c->D - 1) * c->K);
+  c->need_pos = std::max(c->N, c->tail_tree) + 1;
+  c->smax_proj = 16; c->smax_qkv = 8; c->smax_gu = 4;
+  int B = c->B, k = c->k, R = c->Ralloc, qd = c->H * c->hd, qkvd = (c->H + 2 * c->G) * c->hd;
+  size_t e = c->esz;
+  Carver cv(base);
+  c->x = cv.take<float>((size_t)R * k);
+  c->proj = cv.take<float>((size_t)c->smax_proj * R * k);
+  c->qkv = cv.take<float>((size_t)c->smax_qkv * R * qkvd);
+  c->gu = cv.take<float>((size_t)c->smax_gu * R * 2 * c->F);
+  c->logits = cv.take<float>((size_t)R * std::max(c->V, c->Vd));
+  c->h = cv.take_bytes((size_t)R * k * e);
+  c->q = cv.take_bytes((size_t)R * qd * e);
+  c->ao = cv.take_bytes((size_t)R * qd * e);
+  c->act = cv.take_bytes((size_t)R * c->F * e);
+  c->cat = cv.take_bytes((size_t)R * 2 * k * e);
+  c->node_taps = cv.take_bytes((size_t)R * 3 * k * e);
+  c->pend_taps = cv.take_bytes((size_t)R * 3 * k * e);
+  c->cs = cv.take<float2>((size_t)R * (c->hd / 2));
+  c->inv_freq = cv.take<double>(c->hd / 2);
+  c->meta.seq = cv.take<int32_t>(R); c->meta.pos = cv.take<int32_t>(R); c->meta.kvpos = cv.take<int32_t>(R);
+  c->meta.ctx = cv.take<int32_t>(R); c->meta.tail_base = cv.take<int32_t>(R); c->meta.tok = cv.take<int32_t>(R);
+  c->meta.mask_lo = cv.take<uint64_t>(R); c->meta.mask_hi = cv.take<uint64_t>(R);
+  size_t pool_elems = (size_t)g.num_pages * c->G * g.page_size * c->hd;
+  c->pools.resize(c->L + 1);
+  for (int l = 0; l <= c->L; l++) {
+    c->pools[l].k = cv.take_bytes(pool_elems * e);
+    c->pools[l].v = cv.take_bytes(pool_elems * e);
+  }
+  c->pools_dev = cv.take<KvPool>(c->L + 1);
+  c->page_table = cv.take<int32_t>((size_t)B * c->pps);
+  c->st.n = cv.take<int32_t>(B); c->st.n_prev = cv.take<int32_t>(B); c->st.P = cv.take<int32_t>(B);
+  c->st.root = cv.take<int32_t>(B); c->st.cap = cv.take<int32_t>(B); c->st.last_row = cv.take<int32_t>(B);
+  c->st.active = cv.take<int32_t>(B);
+  TreeBufs &t = c->tb;
+  t.pool = c->pool; t.K = c->K; t.D = c->D; t.N = c->N; t.Pmax = c->Pmax;
+  size_t pe = (size_t)B * (c->pool + 1);
+  t.pool_tok = cv.take<int32_t>(pe); t.pool_parent = cv.take<int32_t>(pe); t.pool_depth = cv.take<int32_t>(pe);
+  t.pool_score = cv.take<float>(pe);
+  t.frontier = cv.take<int32_t>((size_t)B * c->D * c->K);
+  t.front_cur = cv.take<int32_t>((size_t)B * c->K);
+  t.feat_row = cv.take<int32_t>(R);
+  t.tk_idx = cv.take<int32_t>((size_t)R * c->K); t.tk_lp = cv.take<float>((size_t)R * c->K);
+  size_t ne = (size_t)std::max(B * c->N, R);
+  t.tok = cv.take<int32_t>(ne); t.parent = cv.take<int32_t>(ne); t.depth = cv.take<int32_t>(ne);
+  t.poolidx = cv.take<int32_t>(ne); t.score = cv.take<float>(ne); t.mask = cv.take<uint64_t>(ne);
+  t.nn = cv.take<int32_t>(B); t.y = cv.take<int32_t>(ne);
+  t.path = cv.take<int32_t>((size_t)B * c->Pmax); t.out_ids = cv.take<int32_t>((size_t)B * c->Pmax);
+  t.out_cnt = cv.take<int32_t>(B); t.pend_tok = cv.take<int32_t>((size_t)B * c->Pmax);
+  c->status = cv.take<int32_t>(8);
+  if (g.flags & SPEC_FLAG_CAPTURE) {
+    c->cap_logits = cv.take<float>((size_t)c->D * c->Td * c->Vd);
+    c->cap_a = cv.take<float>((size_t)c->D * c->Td * k);
+  } else {
+    c->cap_logits = c->cap_a = nullptr;
+  }
+  c->gemm_scratch_bytes = 0;
+  c->gemm_scratch = nullptr;
+  c->attn_scratch_bytes = attn_fast_scratch_bytes(R, c->H, c->hd, g.max_ctx);
+  c->attn_scratch = cv.take_bytes(c->attn_scratch_bytes);
+  return (cv.off + 255) & ~(size_t)255;
+}
+
+extern "C" size_t spec_workspace_bytes(const spec_cfg *cfg) {
+  if (!cfg || check_cfg(cfg)) return 0;
+  spec_ctx tmp;
+  tmp.cfg = *cfg;
+  return carve(&tmp, nullptr);
+}
+
+extern "C" const char *spec_last_error(const spec_ctx *ctx) { return ctx ? ctx->err : g_init_err; }
+
+extern "C" int spec_init(spec_ctx **out, const spec_target_weights *tw, const spec_draft_weights *dw, const spec_cfg *cfg) {
+  if (out) *out = nullptr;
+  if (!out || !tw || !dw || !cfg) return fail(nullptr, SPEC_ERR_NULL, "spec_init: NULL argument");
+  if (const char *why = check_cfg(cfg)) return fail(nullptr, SPEC_ERR_INVALID_CFG, "spec_init: %s", why);
+  if (!cfg->workspace) return fail(nullptr, SPEC_ERR_NULL, "spec_init: workspace is NULL");
+  if ((uintptr_t)cfg->workspace & 255) return fail(nullptr, SPEC_ERR_WORKSPACE, "spec_init: workspace must be 256-byte aligned");
+  const void *req[] = {tw->embed, tw->final_norm, tw->lm_head, tw->attn_norm, tw->wq, tw->wk, tw->wv, tw->wo, tw->mlp_norm,
+                       tw->w_gate, tw->w_up, tw->w_down, dw->fc3, dw->fc2, dw->attn_norm, dw->wq, dw->wk, dw->wv, dw->wo,
+                       dw->mlp_norm, dw->w_gate, dw->w_up, dw->w_down, dw->final_norm, dw->lm_head, dw->d2t};
+  for (const void *p : req)
+    if (!p) return fail(nullptr, SPEC_ERR_NULL, "spec_init: a weight pointer is NULL");
+  spec_ctx *c = new spec_ctx();
+  c->cfg = *cfg;
+  c->err[0] = 0;
+  c->stream = (cudaStream_t)cfg->stream;
+  size_t need = carve(c, cfg->workspace);
+  if (need > cfg->workspace_bytes) {
+    delete c;
+    return fail(nullptr, SPEC_ERR_WORKSPACE, "spec_init: workspace has %zu bytes, %zu needed", cfg->workspace_bytes, need);
+  }
+  for (int l = 0; l < c->L; l++) {
+    LayerW w = {tw->attn_norm[l], tw->wq[l], tw->wk[l], tw->wv[l], tw->wo[l], tw->mlp_norm[l], tw->w_gate[l], tw->w_up[l], tw->w_down[l]};
+    const void *ps[] = {w.attn_norm, w.wq, w.wk, w.wv, w.wo, w.mlp_norm, w.w_gate, w.w_up, w.w_down};
+    for (const void *p : ps)
+      if (!p) { delete c; return fail(nullptr, SPEC_ERR_NULL, "spec_init: layer %d has a NULL weight", l); }
+    c->tl.push_back(w);
+  }
+  c->dl = LayerW{dw->attn_norm, dw->wq, dw->wk, dw->wv, dw->wo, dw->mlp_norm, dw->w_gate, dw->w_up, dw->w_down};
+  c->embed = tw->embed; c->final_norm = tw->final_norm; c->lm_head = tw->lm_head;
+  c->fc3 = dw->fc3; c->fc2 = dw->fc2; c->dfinal_norm = dw->final_norm; c->dlm_head = dw->lm_head; c->d2t = dw->d2t;
+  cudaStream_t s = c->stream;
+  cudaError_t e = cudaMemsetAsync(cfg->workspace, 0, need, s);
+  std::vector<double> inv(c->hd / 2);
+  for (int i = 0; i < c->hd / 2; i++) inv[i] = pow((double)cfg->rope_theta, -2.0 * (double)i / (double)c->hd);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(c->inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(c->pools_dev, c->pools.data(), sizeof(KvPool) * (c->L + 1), cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) {
+    int rc = fail(nullptr, SPEC_ERR_CUDA, "spec_init: %s", cudaGetErrorString(e));
+    delete c;
+    return rc;
+  }
+  c->n_upper.assign(c->B, 0); c->cap_host.assign(c->B, 0); c->n_pages_host.assign(c->B, 0);
+  c->page_table_host.assign((size_t)c->B * c->pps, 0);
+  if (cfg->dtype == SPEC_BF16 && !((cfg->flags & SPEC_FLAG_REF_GEMM))) {
+    std::string why;
+    c->fg = fast_gemm_create(why);
+    if (!c->fg) {
+      int rc = fail(nullptr, SPEC_ERR_CUDA, "spec_init: tcgen05 GEMM set-up failed: %s", why.c_str());
+      delete c;
+      return rc;
+    }
+  }
+  *out = c;
+  return SPEC_OK;
+}
+
+extern "C" int spec_free(spec_ctx *c) {
+  if (!c) return SPEC_OK;
+  if (c->graph) cudaGraphExecDestroy(c->graph);
+  if (c->fg) fast_gemm_destroy(c->fg);
+  delete c;
+  return SPEC_OK;
+}
+
+// ------------------------------------------------------------------------------------------ schedule
+template <typename T> struct Sched {
+  spec_ctx *c;
+  cudaStream_t s;
+  explicit Sched(spec_ctx *ctx) : c(ctx), s(ctx->stream) {}
+  void tick(int n = 1) { c->launches += n; }
+
+  // number of split-K slices for a weight of shape [O][I] whose output buffer holds smax slices
+  int pick(int O, int I, int smax) const { return c->fg ? fast_gemm_pick_split(O, I, smax) : 1; }
+  size_t pstride(int ldo) const { return (size_t)c->Ralloc * ldo; }
+
+  // S fp32 partial slices of x . w^T into columns [col0, col0+O) of `out` (row pitch ldo)
+  void gemm(const void *x, const void *w, float *out, int rows, int O, int I, int ldo, int col0, int S) {
+    if (c->fg) {
+      int rc = fast_gemm_run(c->fg, (const bf16 *)x, (const bf16 *)w, out + col0, rows, O, I, ldo, pstride(ldo), S, c->status, s);
+      if (rc && !c->sched_err) c->sched_err = rc;
+    } else {
+      launch_gemm_ref<T>((const T *)x, (const T *)w, out + col0, rows, O, I, ldo, s);
+    }
+    tick();
+  }
+
+  void attention(KvPool pool, int rows, int tail_len) {
+    PageMap pm{c->page_table, c->pps, c->cfg.page_size, c->cfg.num_pages};
+    bool fast = c->cfg.dtype == SPEC_BF16 && !(c->cfg.flags & SPEC_FLAG_REF_ATTN) && attn_fast_supported(c->hd, c->H / c->G);
+    if (fast) {
+      tick(launch_attn_fast((const bf16 *)c->q, pool, pm, c->meta, tail_len, (bf16 *)c->ao, rows, c->H, c->G, c->hd,
+                            c->cfg.max_ctx, c->attn_scratch, s));
+    } else {
+      launch_attn_ref<T>((const T *)c->q, pool, pm, c->meta, tail_len, (T *)c->ao, rows, c->H, c->G, c->hd,
+                         c->cfg.max_ctx + tail_len, s);
+      tick();
+    }
+  }
+
+  // One decoder block on `rows` rows described by c->meta.  first_mode: how the residual stream is
+  // formed from the pending partial sums (0 keep, 1 set, 2 add); tap_mask: taps of the previous block.
+  void block(const LayerW &w, KvPool pool, int rows, int tail_len, int first_mode, int tap_mask) {
+    int k = c->k, qd = c->H * c->hd, kvd = c->G * c->hd, qkvd = qd + 2 * kvd, F = c->F;
+    PageMap pm{c->page_table, c->pps, c->cfg.page_size, c->cfg.num_pages};
+    launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, first_mode, (T *)c->node_taps, tap_mask, (const T *)w.attn_norm,
+                       c->cfg.rms_eps, (T *)c->h, nullptr, rows, rows, k, s);
+    tick();
+    c->np_qkv = pick(qd, k, c->smax_qkv); c->ps_qkv = pstride(qkvd);
+    gemm(c->h, w.wq, c->qkv, rows, qd, k, qkvd, 0, c->np_qkv);
+    gemm(c->h, w.wk, c->qkv, rows, kvd, k, qkvd, qd, c->np_qkv);
+    gemm(c->h, w.wv, c->qkv, rows, kvd, k, qkvd, qd + kvd, c->np_qkv);
+    launch_rope_kv<T>(c->qkv, c->np_qkv, c->ps_qkv, c->cs, c->meta, (T *)c->q, pool, pm, rows, c->H, c->G, c->hd, c->status, s);
+    tick();
+    attention(pool, rows, tail_len);
+    c->np_proj = pick(k, qd, c->smax_proj); c->ps_proj = pstride(k);
+    gemm(c->ao, w.wo, c->proj, rows, k, qd, k, 0, c->np_proj);
+    launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, 2, (T *)nullptr, 0, (const T *)w.mlp_norm, c->cfg.rms_eps,
+                       (T *)c->h, nullptr, rows, rows, k, s);
+    tick();
+    c->np_gu = pick(F, k, c->smax_gu); c->ps_gu = pstride(2 * F);
+    gemm(c->h, w.w_gate, c->gu, rows, F, k, 2 * F, 0, c->np_gu);
+    gemm(c->h, w.w_up, c->gu, rows, F, k, 2 * F, F, c->np_gu);
+    launch_silu_mul<T>(c->gu, c->np_gu, c->ps_gu, (T *)c->act, rows, F, s);
+    tick();
+    c->np_proj = pick(k, F, c->smax_proj); c->ps_proj = pstride(k);
+    gemm(c->act, w.w_down, c->proj, rows, k, F, k, 0, c->np_proj);
+  }
+
+  int tap_mask_of(int layer) const {
+    int m = 0;
+    for (int i = 0; i < 3; i++) m |= (c->cfg.fuse_layers[i] == layer) ? (1 << i) : 0;
+    return m;
+  }
+
+  // target forward over the rows of c->meta: taps -> node_taps, argmax -> tb.y
+  void target_forward(int rows, int tail_len, bool want_logits) {
+    launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
+    launch_embed<T>((const T *)c->embed, c->meta.tok, c->x, rows, c->k, s); tick();
+    for (int l = 0; l < c->L; l++)
+      block(c->tl[l], c->pools[l], rows, tail_len, l == 0 ? 0 : 2, l == 0 ? 0 : tap_mask_of(l - 1));
+    launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, 2, (T *)c->node_taps, tap_mask_of(c->L - 1),
+                       (const T *)c->final_norm, c->cfg.rms_eps, (T *)c->h, nullptr, rows, rows, c->k, s);
+    tick();
+    if (want_logits) {
+      gemm(c->h, c->lm_head, c->logits, rows, c->V, c->k, c->V, 0, 1);
+      launch_argmax(c->logits, rows, c->V, c->tb.y, s); tick();
+    }
+  }
+
+  // FC3 over `rows` rows of taps -> proj (Section 3.1: g = FC([l;m;h]))
+  void fuse(const void *taps, int rows) {
+    c->np_proj = pick(c->k, 3 * c->k, c->smax_proj); c->ps_proj = pstride(c->k);
+    gemm(taps, c->fc3, c->proj, rows, c->k, 3 * c->k, c->k, 0, c->np_proj);
+  }
+
+  // draft head on the rows of c->meta: cat = [feat ; e(tok)], FC2, decoder block, final norm (-> h)
+  void draft_forward(const float *feat, int nparts, size_t fstride, const int32_t *src_row, int rows, int tail_len) {
+    launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
+    launch_build_cat<T>(feat, nparts, fstride, src_row, (const T *)c->embed, c->meta.tok, c->meta.seq, (T *)c->cat, rows, c->k, s);
+    tick();
+    c->np_proj = pick(c->k, 2 * c->k, c->smax_proj); c->ps_proj = pstride(c->k);
+    gemm(c->cat, c->fc2, c->proj, rows, c->k, 2 * c->k, c->k, 0, c->np_proj);
+    block(c->dl, c->pools[c->L], rows, tail_len, 1, 0);
+    launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, 2, (T *)nullptr, 0, (const T *)c->dfinal_norm, c->cfg.rms_eps,
+                       (T *)c->h, nullptr, rows, rows, c->k, s);
+    tick();
+  }
+
+  void draft_logits(int rows) {
+    gemm(c->h, c->dlm_head, c->logits, rows, c->Vd, c->k, c->Vd, 0, 1);
+  }
+
+  void capture(int pass, int rows, bool first) {
+    if (!c->cap_logits) return;
+    // pass 1: only the last pending row of each sequence matters; it lands in slot [0][b*K]
+    size_t lo = (size_t)(pass - 1) * c->Td;
+    if (first) {
+      launch_gather_rows(c->logits, c->st.last_row, c->cap_logits + lo * c->Vd, c->B, c->Vd, c->K, s);
+      launch_gather_rows(c->x, c->st.last_row, c->cap_a + lo * c->k, c->B, c->k, c->K, s);
+    } else {
+      cudaMemcpyAsync(c->cap_logits + lo * c->Vd, c->logits, (size_t)rows * c->Vd * 4, cudaMemcpyDeviceToDevice, s);
+      cudaMemcpyAsync(c->cap_a + lo * c->k, c->x, (size_t)rows * c->k * 4, cudaMemcpyDeviceToDevice, s);
+    }
+    tick(2);
+  }
+
+  void step(bool plain) {
+    int rows = plain ? c->B : c->Tv, rps = plain ? 1 : c->N;
+    if (!plain) {
+      launch_prep_extend(c->st, c->tb, c->meta, c->B, c->need_pos, c->status, s); tick();
+      fuse(c->pend_taps, c->Te);
+      draft_forward(c->proj, c->np_proj, c->ps_proj, nullptr, c->Te, c->Pmax);
+      draft_logits(c->Te);
+      launch_logsoftmax_topk_rows(c->logits, c->st.last_row, c->B, c->Vd, c->K, c->tb.tk_idx, c->tb.tk_lp, s); tick();
+      capture(1, c->Te, true);
+      launch_expand(c->st, c->tb, c->meta, c->d2t, 1, c->B, s); tick();
+      for (int p = 2; p <= c->D; p++) {
+        draft_forward(c->x, 1, 0, c->tb.feat_row, c->Td, c->tail_tree);
+        draft_logits(c->Td);
+        launch_logsoftmax_topk_rows(c->logits, nullptr, c->Td, c->Vd, c->K, c->tb.tk_idx, c->tb.tk_lp, s); tick();
+        capture(p, c->Td, false);
+        launch_expand(c->st, c->tb, c->meta, c->d2t, p, c->B, s); tick();
+      }
+      launch_rerank(c->st, c->tb, c->meta, c->B, s); tick();
+    } else {
+      launch_plain_tree(c->st, c->tb, c->meta, c->B, s); tick();
+    }
+    target_forward(rows, rps, true);
+    launch_accept(c->st, c->tb, c->B, rps, s); tick();
+    PageMap pm{c->page_table, c->pps, c->cfg.page_size, c->cfg.num_pages};
+    launch_commit<T>(c->st, c->tb, c->pools_dev, pm, (const T *)c->node_taps, (T *)c->pend_taps, c->B, c->L, c->G, c->hd,
+                     c->k, rps, s);
+    tick();
+  }
+};
+
+// hazard note: draft_forward for tree passes reads c->x (previous pass) in build_cat before FC2 + the
+// block's first add_norm overwrite it; everything is ordered on one stream.
+
+static int read_status(spec_ctx *c) {
+  int32_t st[4] = {0, 0, 0, 0};
+  CUDA_TRY(c, cudaMemcpyAsync(st, c->status, sizeof st, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  if (st[0] != 0) {
+    cudaMemsetAsync(c->status, 0, 16, c->stream);
+    int code = st[0] == ST_CAPACITY ? SPEC_ERR_CAPACITY : SPEC_ERR_DEVICE_STATUS;
+    return fail(c, code, "device status %d at site %d (detail %d, %d)", st[0], st[1], st[2], st[3]);
+  }
+  return SPEC_OK;
+}
+
+template <typename T> static int do_prefill(spec_ctx *c, const int32_t *ids, const int32_t *lens, int32_t reserve, int32_t *first) {
+  const spec_cfg &g = c->cfg;
+  cudaStream_t s = c->stream;
+  int B = c->B, ps = g.page_size;
+  // ---- pages: each sequence takes what prompt + reserve + one tree needs, from a (shuffled) free list
+  std::vector<int32_t> order(g.num_pages);
+  for (int i = 0; i < g.num_pages; i++) order[i] = i;
+  if (g.page_shuffle_seed) {
+    uint64_t z = (uint64_t)(uint32_t)g.page_shuffle_seed * 0x9E3779B97F4A7C15ull + 1;
+    for (int i = g.num_pages - 1; i > 0; i--) {
+      z = z * 6364136223846793005ull + 1442695040888963407ull;
+      int j = (int)((z >> 33) % (uint64_t)(i + 1));
+      std::swap(order[i], order[j]);
+    }
+  }
+  size_t next = 0;
+  std::vector<int32_t> cap(B);
+  for (int b = 0; b < B; b++) {
+    if (lens[b] < 1) return fail(c, SPEC_ERR_INVALID_CFG, "spec_prefill: prompt %d is empty", b);
+    long long want = (long long)lens[b] + reserve + c->need_pos;
+    if (want > g.max_ctx) return fail(c, SPEC_ERR_CAPACITY, "spec_prefill: sequence %d needs %lld positions, max_ctx is %d", b, want, g.max_ctx);
+    int np = (int)((want + ps - 1) / ps);
+    if (next + np > (size_t)g.num_pages) return fail(c, SPEC_ERR_CAPACITY, "spec_prefill: page pool exhausted at sequence %d", b);
+    for (int p = 0; p < c->pps; p++) c->page_table_host[(size_t)b * c->pps + p] = p < np ? order[next + p] : -1;
+    next += np;
+    c->n_pages_host[b] = np;
+    cap[b] = std::min(np * ps, g.max_ctx);
+  }
+  c->cap_host = cap;
+  CUDA_TRY(c, cudaMemcpyAsync(c->page_table, c->page_table_host.data(), c->page_table_host.size() * 4, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(c, cudaMemcpyAsync(c->st.cap, cap.data(), B * 4, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(c, cudaStreamSynchronize(s));
+
+  Sched<T> sc(c);
+  const int CH = 64;
+  std::vector<int32_t> mseq(CH), mpos(CH), mctx(CH), mtok(CH), mzero(CH, 0);
+  std::vector<uint64_t> mlo(CH), mhi(CH, 0);
+  auto upload_meta = [&](int nvalid, int b, int start, const int32_t *toks) -> cudaError_t {
+    for (int r = 0; r < CH; r++) {
+      bool v = r < nvalid;
+      mseq[r] = v ? b : -1; mpos[r] = v ? start + r : 0; mctx[r] = v ? start : 0; mtok[r] = v ? toks[r] : 0;
+      mlo[r] = v ? (r >= 63 ? ~0ull : ((1ull << (r + 1)) - 1ull)) : 0ull;
+    }
+    cudaError_t e = cudaMemcpyAsync(c->meta.seq, mseq.data(), CH * 4, cudaMemcpyHostToDevice, s);
+    if (!e) e = cudaMemcpyAsync(c->meta.pos, mpos.data(), CH * 4, cudaMemcpyHostToDevice, s);
+    if (!e) e = cudaMemcpyAsync(c->meta.kvpos, mpos.data(), CH * 4, cudaMemcpyHostToDevice, s);
+    if (!e) e = cudaMemcpyAsync(c->meta.ctx, mctx.data(), CH * 4, cudaMemcpyHostToDevice, s);
+    if (!e) e = cudaMemcpyAsync(c->meta.tail_base, mctx.data(), CH * 4, cudaMemcpyHostToDevice, s);
+    if (!e) e = cudaMemcpyAsync(c->meta.tok, mtok.data(), CH * 4, cudaMemcpyHostToDevice, s);
+    if (!e) e = cudaMemcpyAsync(c->meta.mask_lo, mlo.data(), CH * 8, cudaMemcpyHostToDevice, s);
+    if (!e) e = cudaMemcpyAsync(c->meta.mask_hi, mhi.data(), CH * 8, cudaMemcpyHostToDevice, s);
+    if (!e) e = cudaStreamSynchronize(s);   // host vectors are reused by the next chunk
+    return e;
+  };
+  size_t off = 0;
+  std::vector<int32_t> n_host(B), P_host(B, 1), root_host(B);
+  for (int b = 0; b < B; b++) {
+    const int32_t *p = ids + off;
+    int n = lens[b];
+    for (int i = 0; i < n; i++)
+      if (p[i] < 0 || p[i] >= g.vocab) return fail(c, SPEC_ERR_INVALID_CFG, "spec_prefill: token id out of range in prompt %d", b);
+    for (int start = 0; start < n; start += CH) {
+      int nv = std::min(CH, n - start);
+      bool last = start + nv == n;
+      CUDA_TRY(c, upload_meta(nv, b, start, p + start));
+      sc.target_forward(CH, CH, last);
+      if (last) {
+        // the last position stays pending: its taps become pending entry 0
+        CUDA_TRY(c, cudaMemcpyAsync((char *)c->pend_taps + (size_t)b * c->Pmax * 3 * c->k * c->esz,
+                                    (char *)c->node_taps + (size_t)(nv - 1) * 3 * c->k * c->esz, (size_t)3 * c->k * c->esz,
+                                    cudaMemcpyDeviceToDevice, s));
+        CUDA_TRY(c, cudaMemcpyAsync(&root_host[b], c->tb.y + (nv - 1), 4, cudaMemcpyDeviceToHost, s));
+      }
+      int nd = last ? nv - 1 : nv;        // draft entries j use token j+1; the last position waits for the root
+      if (nd > 0) {
+        sc.fuse(c->node_taps, CH);
+        CUDA_TRY(c, upload_meta(nd, b, start, p + start + 1));
+        sc.draft_forward(c->proj, c->np_proj, c->ps_proj, nullptr, CH, CH);
+      }
+    }
+    CUDA_TRY(c, cudaStreamSynchronize(s));
+    n_host[b] = n;
+    off += n;
+  }
+  CUDA_TRY(c, cudaMemcpyAsync(c->st.n, n_host.data(), B * 4, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(c, cudaMemcpyAsync(c->st.n_prev, n_host.data(), B * 4, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(c, cudaMemcpyAsync(c->st.P, P_host.data(), B * 4, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(c, cudaMemcpyAsync(c->st.root, root_host.data(), B * 4, cudaMemcpyHostToDevice, s));
+  std::vector<int32_t> pt((size_t)B * c->Pmax, 0);
+  for (int b = 0; b < B; b++) pt[(size_t)b * c->Pmax] = root_host[b];
+  CUDA_TRY(c, cudaMemcpyAsync(c->tb.pend_tok, pt.data(), pt.size() * 4, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(c, cudaStreamSynchronize(s));
+  for (int b = 0; b < B; b++) { c->n_upper[b] = n_host[b]; first[b] = root_host[b]; }
+  c->prefilled = true;
+  c->draft_stale = false;
+  if (c->graph) { cudaGraphExecDestroy(c->graph); c->graph = nullptr; }
+  return read_status(c);
+}
+
+extern "C" int spec_prefill(spec_ctx *c, const int32_t *ids, const int32_t *lens, int32_t reserve, int32_t *first) {
+  if (!c) return SPEC_ERR_NULL;
+  if (!ids || !lens || !first) return fail(c, SPEC_ERR_NULL, "spec_prefill: NULL argument");
+  if (reserve < 0) return fail(c, SPEC_ERR_INVALID_CFG, "spec_prefill: reserve_tokens is negative");
+  return c->cfg.dtype == SPEC_F32 ? do_prefill<float>(c, ids, lens, reserve, first) : do_prefill<bf16>(c, ids, lens, reserve, first);
+}
+
+static int launch_step(spec_ctx *c, bool plain) {
+  bool use_graph = !(c->cfg.flags & SPEC_FLAG_NO_GRAPH) && !plain;
+  c->launches = 0;
+  if (!use_graph) {
+    if (c->cfg.dtype == SPEC_F32) Sched<float>(c).step(plain); else Sched<bf16>(c).step(plain);
+    CUDA_TRY(c, cudaGetLastError());
+    if (c->sched_err) return fail(c, SPEC_ERR_CUDA, "a GEMM launch was rejected (code %d)", c->sched_err);
+    return SPEC_OK;
+  }
+  if (!c->graph) {
+    cudaGraph_t gr;
+    CUDA_TRY(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+    if (c->cfg.dtype == SPEC_F32) Sched<float>(c).step(false); else Sched<bf16>(c).step(false);
+    cudaError_t e = cudaStreamEndCapture(c->stream, &gr);
+    if (e != cudaSuccess) return fail(c, SPEC_ERR_CUDA, "graph capture: %s", cudaGetErrorString(e));
+    if (c->sched_err) { cudaGraphDestroy(gr); return fail(c, SPEC_ERR_CUDA, "a GEMM launch was rejected (code %d)", c->sched_err); }
+    e = cudaGraphInstantiate(&c->graph, gr, 0);
+    cudaGraphDestroy(gr);
+    if (e != cudaSuccess) { c->graph = nullptr; return fail(c, SPEC_ERR_CUDA, "graph instantiate: %s", cudaGetErrorString(e)); }
+    c->launches_graph = c->launches;
+  }
+  c->launches = c->launches_graph;
+  CUDA_TRY(c, cudaGraphLaunch(c->graph, c->stream));
+  return SPEC_OK;
+}
+
+static int check_capacity(spec_ctx *c, int grow, const char *who) {
+  if (!c->prefilled) return fail(c, SPEC_ERR_STATE, "%s before spec_prefill", who);
+  for (int b = 0; b < c->B; b++)
+    if (c->n_upper[b] + c->need_pos > c->cap_host[b])
+      return fail(c, SPEC_ERR_CAPACITY, "%s: sequence %d may reach %d positions (+%d for the tree) but has pages for %d", who, b,
+                  c->n_upper[b], c->need_pos, c->cap_host[b]);
+  (void)grow;
+  return SPEC_OK;
+}
+
+extern "C" int spec_step_async(spec_ctx *c, int32_t *dev_ids, int32_t *dev_counts) {
+  if (!c) return SPEC_ERR_NULL;
+  if (c->draft_stale) return fail(c, SPEC_ERR_STATE, "spec_step after spec_plain_step: the draft cache is stale, prefill again");
+  if (int rc = check_capacity(c, c->Pmax, "spec_step")) return rc;
+  if (int rc = launch_step(c, false)) return rc;
+  for (int b = 0; b < c->B; b++) c->n_upper[b] += c->Pmax;
+  if (dev_ids) CUDA_TRY(c, cudaMemcpyAsync(dev_ids, c->tb.out_ids, (size_t)c->B * c->Pmax * 4, cudaMemcpyDeviceToDevice, c->stream));
+  if (dev_counts) CUDA_TRY(c, cudaMemcpyAsync(dev_counts, c->tb.out_cnt, (size_t)c->B * 4, cudaMemcpyDeviceToDevice, c->stream));
+  return SPEC_OK;
+}
+
+static int sync_lengths(spec_ctx *c) {
+  std::vector<int32_t> n(c->B);
+  CUDA_TRY(c, cudaMemcpyAsync(n.data(), c->st.n, c->B * 4, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  c->n_upper = n;
+  return SPEC_OK;
+}
+
+extern "C" int spec_step(spec_ctx *c, int32_t *out_ids, int32_t *out_counts) {
+  if (!c) return SPEC_ERR_NULL;
+  if (!out_ids || !out_counts) return fail(c, SPEC_ERR_NULL, "spec_step: NULL output");
+  if (int rc = spec_step_async(c, nullptr, nullptr)) return rc;
+  CUDA_TRY(c, cudaMemcpyAsync(out_ids, c->tb.out_ids, (size_t)c->B * c->Pmax * 4, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(out_counts, c->tb.out_cnt, (size_t)c->B * 4, cudaMemcpyDeviceToHost, c->stream));
+  if (int rc = read_status(c)) return rc;
+  return sync_lengths(c);
+}
+
+extern "C" int spec_plain_step(spec_ctx *c, int32_t *out_ids) {
+  if (!c) return SPEC_ERR_NULL;
+  if (!out_ids) return fail(c, SPEC_ERR_NULL, "spec_plain_step: NULL output");
+  if (int rc = check_capacity(c, 1, "spec_plain_step")) return rc;
+  c->draft_stale = true;
+  if (int rc = launch_step(c, true)) return rc;
+  std::vector<int32_t> ids((size_t)c->B * c->Pmax);
+  CUDA_TRY(c, cudaMemcpyAsync(ids.data(), c->tb.out_ids, ids.size() * 4, cudaMemcpyDeviceToHost, c->stream));
+  if (int rc = read_status(c)) return rc;
+  for (int b = 0; b < c->B; b++) out_ids[b] = ids[(size_t)b * c->Pmax];
+  return sync_lengths(c);
+}
+
+extern "C" int spec_lengths(spec_ctx *c, int32_t *lens) {
+  if (!c || !lens) return SPEC_ERR_NULL;
+  if (int rc = sync_lengths(c)) return rc;
+  for (int b = 0; b < c->B; b++) lens[b] = c->n_upper[b];
+  return SPEC_OK;
+}
+
+extern "C" int spec_launches_per_step(const spec_ctx *c) { return c ? c->launches : 0; }
+
+extern "C" int spec_step_bytes(spec_ctx *c, double *bytes) {
+  if (!c || !bytes) return SPEC_ERR_NULL;
+  if (int rc = sync_lengths(c)) return rc;
+  double e = c->esz, k = c->k, qd = (double)c->H * c->hd, kvd = (double)c->G * c->hd, F = c->F;
+  double layer = (k * qd + 2 * k * kvd + qd * k + 3 * k * F + 2 * k) * e;
+  double draft_pass = (2 * k * k + k) * e + layer + (double)c->Vd * k * e;
+  double w = c->D * draft_pass + 3 * k * k * e + c->L * layer + ((double)c->V * k + k) * e;
+  double kv = 0;
+  for (int b = 0; b < c->B; b++) kv += (double)c->n_upper[b] * 2 * kvd * e * (c->L + c->D);
+  *bytes = w + kv;
+  return SPEC_OK;
+}
+
+// ------------------------------------------------------------------------------------------ inspection
+template <typename U> static int64_t copy_out(spec_ctx *c, const U *dev, size_t count, void *dst, size_t bytes) {
+  size_t avail = count * sizeof(U);
+  size_t n = std::min(avail, bytes);
+  if (n && dst) {
+    if (cudaMemcpyAsync(dst, dev, n, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess) return SPEC_ERR_CUDA;
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SPEC_ERR_CUDA;
+  }
+  return (int64_t)avail;
+}
+
+// widen a [rows][width] block of the storage dtype to floats on the host
+static int64_t copy_widen(spec_ctx *c, const void *dev, size_t count, void *dst, size_t bytes) {
+  size_t avail = count * 4;
+  if (!dst || !bytes) return (int64_t)avail;
+  size_t n = std::min(count, bytes / 4);
+  if (c->esz == 4) return copy_out(c, (const float *)dev, n, dst, n * 4) < 0 ? SPEC_ERR_CUDA : (int64_t)avail;
+  std::vector<uint16_t> tmp(n);
+  if (cudaMemcpyAsync(tmp.data(), dev, n * 2, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess) return SPEC_ERR_CUDA;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SPEC_ERR_CUDA;
+  float *f = (float *)dst;
+  for (size_t i = 0; i < n; i++) { uint32_t u = (uint32_t)tmp[i] << 16; memcpy(&f[i], &u, 4); }
+  return (int64_t)avail;
+}
+
+extern "C" int64_t spec_debug_read(spec_ctx *c, int32_t what, int32_t seq, void *dst, size_t bytes) {
+  if (!c) return SPEC_ERR_NULL;
+  if (seq < 0 || seq >= c->B) return fail(c, SPEC_ERR_INVALID_CFG, "spec_debug_read: sequence %d out of range", seq);
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SPEC_ERR_CUDA;
+  int32_t nn = 0, cnt = 0;
+  cudaMemcpy(&nn, c->tb.nn + seq, 4, cudaMemcpyDeviceToHost);
+  cudaMemcpy(&cnt, c->tb.out_cnt + seq, 4, cudaMemcpyDeviceToHost);
+  size_t t0 = (size_t)seq * c->N, p0 = (size_t)seq * (c->pool + 1);
+  const TreeBufs &t = c->tb;
+  switch (what) {
+    case SPEC_DBG_TREE_TOK: return copy_out(c, t.tok + t0, nn, dst, bytes);
+    case SPEC_DBG_TREE_PARENT: return copy_out(c, t.parent + t0, nn, dst, bytes);
+    case SPEC_DBG_TREE_DEPTH: return copy_out(c, t.depth + t0, nn, dst, bytes);
+    case SPEC_DBG_TREE_MASK: return copy_out(c, t.mask + t0, nn, dst, bytes);
+    case SPEC_DBG_TREE_POOLIDX: return copy_out(c, t.poolidx + t0, nn, dst, bytes);
+    case SPEC_DBG_TREE_SCORE: return copy_out(c, t.score + t0, nn, dst, bytes);
+    case SPEC_DBG_Y: return copy_out(c, t.y + t0, nn, dst, bytes);
+    case SPEC_DBG_TARGET_LOGITS: return copy_out(c, c->logits + t0 * c->V, (size_t)nn * c->V, dst, bytes);
+    case SPEC_DBG_NODE_TAPS: return copy_widen(c, (const char *)c->node_taps + t0 * 3 * c->k * c->esz, (size_t)nn * 3 * c->k, dst, bytes);
+    case SPEC_DBG_NODE_HIDDEN: return copy_out(c, c->x + t0 * c->k, (size_t)nn * c->k, dst, bytes);
+    case SPEC_DBG_DRAFT_LOGITS:
+    case SPEC_DBG_DRAFT_A: {
+      if (!c->cap_logits) return fail(c, SPEC_ERR_STATE, "spec_debug_read: needs SPEC_FLAG_CAPTURE");
+      size_t w = what == SPEC_DBG_DRAFT_LOGITS ? c->Vd : c->k;
+      const float *src = what == SPEC_DBG_DRAFT_LOGITS ? c->cap_logits : c->cap_a;
+      size_t per_pass = (size_t)c->K * w, avail = (size_t)c->D * per_pass * 4;
+      if (!dst || !bytes) return (int64_t)avail;
+      if (bytes < avail) return fail(c, SPEC_ERR_INVALID_CFG, "spec_debug_read: buffer too small");
+      for (int d = 0; d < c->D; d++)
+        if (cudaMemcpy((float *)dst + d * per_pass, src + ((size_t)d * c->Td + (size_t)seq * c->K) * w, per_pass * 4,
+                       cudaMemcpyDeviceToHost) != cudaSuccess) return SPEC_ERR_CUDA;
+      return (int64_t)avail;
+    }
+    case SPEC_DBG_POOL_TOK: return copy_out(c, t.pool_tok + p0, c->pool + 1, dst, bytes);
+    case SPEC_DBG_POOL_SCORE: return copy_out(c, t.pool_score + p0, c->pool + 1, dst, bytes);
+    case SPEC_DBG_POOL_PARENT: return copy_out(c, t.pool_parent + p0, c->pool + 1, dst, bytes);
+    case SPEC_DBG_FRONTIER: return copy_out(c, t.frontier + (size_t)seq * c->D * c->K, (size_t)c->D * c->K, dst, bytes);
+    case SPEC_DBG_PATH: return copy_out(c, t.path + (size_t)seq * c->Pmax, cnt, dst, bytes);
+    case SPEC_DBG_STATUS: return copy_out(c, c->status, 4, dst, bytes);
+    case SPEC_DBG_PAGE_TABLE: return copy_out(c, c->page_table + (size_t)seq * c->pps, c->n_pages_host[seq], dst, bytes);
+    default: return fail(c, SPEC_ERR_INVALID_CFG, "spec_debug_read: unknown item %d", what);
+  }
+}
+
+extern "C" int spec_debug_read_kv(spec_ctx *c, int32_t seq, int32_t layer, int32_t pos, float *k, float *v) {
+  if (!c || !k || !v) return SPEC_ERR_NULL;
+  if (seq < 0 || seq >= c->B || layer < -1 || layer >= c->L || pos < 0 || pos >= c->cap_host[seq])
+    return fail(c, SPEC_ERR_INVALID_CFG, "spec_debug_read_kv: index out of range");
+  int l = layer < 0 ? c->L : layer;
+  int ps = c->cfg.page_size;
+  int page = c->page_table_host[(size_t)seq * c->pps + pos / ps];
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SPEC_ERR_CUDA;
+  for (int g = 0; g < c->G; g++) {
+    size_t off = (((size_t)page * c->G + g) * ps + pos % ps) * c->hd;
+    if (copy_widen(c, (const char *)c->pools[l].k + off * c->esz, c->hd, k + (size_t)g * c->hd, (size_t)c->hd * 4) < 0) return SPEC_ERR_CUDA;
+    if (copy_widen(c, (const char *)c->pools[l].v + off * c->esz, c->hd, v + (size_t)g * c->hd, (size_t)c->hd * 4) < 0) return SPEC_ERR_CUDA;
+  }
+  return SPEC_OK;
+}
+
+// ------------------------------------------------------------------------------------------ single kernels
+extern "C" size_t spec_gemm_scratch_bytes(int32_t rows, int32_t out, int32_t in) {
+  return fast_gemm_scratch_bytes(rows, out, in);
+}
+
+extern "C" int spec_gemm(int32_t dtype, int32_t impl, const void *x, const void *w, float *out, int32_t rows, int32_t O,
+                         int32_t I, int32_t ldo, void *scratch, void *stream) {
+  if (!x || !w || !out) return SPEC_ERR_NULL;
+  if (rows < 1 || O < 1 || I < 1 || ldo < O) return SPEC_ERR_INVALID_CFG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (impl == 1) {
+    if (dtype == SPEC_F32) launch_gemm_ref<float>((const float *)x, (const float *)w, out, rows, O, I, ldo, s);
+    else if (dtype == SPEC_BF16) launch_gemm_ref<bf16>((const bf16 *)x, (const bf16 *)w, out, rows, O, I, ldo, s);
+    else return SPEC_ERR_INVALID_CFG;
+    return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
+  }
+  if (dtype != SPEC_BF16) return SPEC_ERR_UNSUPPORTED;
+  return fast_gemm_oneshot((const bf16 *)x, (const bf16 *)w, out, rows, O, I, ldo, scratch, s);
+}
+
+extern "C" size_t spec_attn_scratch_bytes(int32_t rows, int32_t n_heads, int32_t head_dim, int32_t max_ctx) {
+  return attn_fast_scratch_bytes(rows, n_heads, head_dim, max_ctx);
+}
+
+extern "C" int spec_attention(int32_t dtype, int32_t impl, const void *q, const void *k_pool, const void *v_pool,
+                              const int32_t *page_table, int32_t pages_per_seq, int32_t page_size, const int32_t *row_seq,
+                              const int32_t *row_ctx, const int32_t *row_tail_base, const uint64_t *row_mask_lo,
+                              const uint64_t *row_mask_hi, int32_t tail_len, void *out, int32_t rows, int32_t H, int32_t G,
+                              int32_t hd, int32_t max_ctx, void *scratch, void *stream) {
+  if (!q || !k_pool || !v_pool || !page_table || !row_seq || !row_ctx || !row_tail_base || !row_mask_lo || !row_mask_hi || !out)
+    return SPEC_ERR_NULL;
+  if (rows < 1 || H < 1 || G < 1 || H % G || hd < 16 || hd % 16 || tail_len < 0 || tail_len > 128) return SPEC_ERR_INVALID_CFG;
+  cudaStream_t s = (cudaStream_t)stream;
+  RowMeta m{};
+  m.seq = (int32_t *)row_seq; m.ctx = (int32_t *)row_ctx; m.tail_base = (int32_t *)row_tail_base;
+  m.mask_lo = (uint64_t *)row_mask_lo; m.mask_hi = (uint64_t *)row_mask_hi;
+  KvPool pool{(void *)k_pool, (void *)v_pool};
+  PageMap pm{page_table, pages_per_seq, page_size, 1 << 30};
+  if (impl == 1) {
+    if (dtype == SPEC_F32) launch_attn_ref<float>((const float *)q, pool, pm, m, tail_len, (float *)out, rows, H, G, hd, max_ctx + tail_len, s);
+    else if (dtype == SPEC_BF16) launch_attn_ref<bf16>((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, max_ctx + tail_len, s);
+    else return SPEC_ERR_INVALID_CFG;
+    return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
+  }
+  if (dtype != SPEC_BF16 || !attn_fast_supported(hd, H / G)) return SPEC_ERR_UNSUPPORTED;
+  launch_attn_fast((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, max_ctx, scratch, s);
+  return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
+}
+
+extern "C" int spec_logsoftmax_topk(const float *logits, int32_t rows, int32_t n, int32_t K, int32_t *out_idx, float *out_lp,
+                                    void *stream) {
+  if (!logits || !out_idx || !out_lp) return SPEC_ERR_NULL;
+  if (rows < 1 || n < 1 || K < 1 || K > n) return SPEC_ERR_INVALID_CFG;
+  launch_logsoftmax_topk(logits, rows, n, K, out_idx, out_lp, (cudaStream_t)stream);
+  return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
+}
+
+extern "C" int spec_argmax(const float *logits, int32_t rows, int32_t n, int32_t *out_idx, void *stream) {
+  if (!logits || !out_idx) return SPEC_ERR_NULL;
+  if (rows < 1 || n < 1) return SPEC_ERR_INVALID_CFG;
+  launch_argmax(logits, rows, n, out_idx, (cudaStream_t)stream);
+  return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
+}

@@ -1,0 +1,93 @@
+// Shared declarations of the speculative-step library: dtype helpers, per-row metadata, the
+// device-side state block and the launchers each .cu file exports to the step scheduler.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace spec {
+
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// Device status words: [0] error code (0 = fine), [1] where, [2..3] detail.
+enum { ST_OK = 0, ST_CAPACITY = 1, ST_BOUNDS = 2, ST_TIMEOUT = 3 };
+__device__ __forceinline__ void set_status(int32_t *st, int code, int where, int a = 0, int b = 0) {
+  if (atomicCAS(st, 0, code) == 0) { st[1] = where; st[2] = a; st[3] = b; }
+}
+
+// Per-row description of one forward pass (draft extend, draft tree pass, target verify).  A row
+// attends cache positions [0, ctx) unmasked, then "tail" positions tail_base + t for every set bit t
+// of (mask_lo, mask_hi); it writes its own K/V at cache position kvpos and is rotated by pos.
+struct RowMeta {
+  int32_t *seq;        // sequence id, -1 = padding row
+  int32_t *pos;        // RoPE position
+  int32_t *kvpos;      // cache position of this row's K/V
+  int32_t *ctx;        // unmasked context length
+  int32_t *tail_base;
+  uint64_t *mask_lo, *mask_hi;
+  int32_t *tok;        // token id whose embedding this row consumes
+};
+
+// Paged KV pool of one layer: [num_pages][G][page_size][hd]
+struct KvPool {
+  void *k, *v;
+};
+
+struct PageMap {
+  const int32_t *table;    // [batch][pages_per_seq]
+  int32_t pages_per_seq, page_size, num_pages;
+};
+
+__device__ __forceinline__ size_t kv_offset(const PageMap &pm, int seq, int pos, int g, int G, int hd) {
+  int page = pm.table[(size_t)seq * pm.pages_per_seq + pos / pm.page_size];
+  return (((size_t)page * G + g) * pm.page_size + (pos % pm.page_size)) * hd;
+}
+
+// ---------------------------------------------------------------- launchers (elementwise.cu)
+template <typename T>
+void launch_embed(const T *embed, const int32_t *tok, float *x, int rows, int k, cudaStream_t s);
+
+// x (+)= sum of `nparts` partial slices [nparts][rows][k]; optional taps (T, [rows][3k], slots by bitmask);
+// optional h[r] = rmsnorm(x[src_row ? src_row[r] : r]) * gain.  mode: 0 keep x, 1 x = parts, 2 x += parts.
+template <typename T>
+void launch_add_norm(float *x, const float *parts, int nparts, size_t part_stride, int mode, T *taps, int tap_mask,
+                     const T *gain, float eps, T *h, const int32_t *src_row, int rows_x, int rows_h, int k,
+                     cudaStream_t s);
+
+void launch_rope_table(const int32_t *pos, int rows, int half, const double *inv_freq, float2 *cs, cudaStream_t s);
+
+// qkv partial sums [nparts][rows][(H+2G)hd] fp32 -> q (T, [rows][H][hd], rotated) and K/V written into the
+// paged pool at kvpos (K rotated).
+template <typename T>
+void launch_rope_kv(const float *qkv, int nparts, size_t part_stride, const float2 *cs, RowMeta m, T *q, KvPool pool,
+                    PageMap pm, int rows, int H, int G, int hd, int32_t *status, cudaStream_t s);
+
+template <typename T>
+void launch_silu_mul(const float *gu, int nparts, size_t part_stride, T *act, int rows, int F, cudaStream_t s);
+
+// cat[r] = [ T(feat[src_row[r]]) ; embed[tok[r]] ], feat = sum of partial slices (fp32)
+template <typename T>
+void launch_build_cat(const float *feat, int nparts, size_t part_stride, const int32_t *src_row, const T *embed,
+                      const int32_t *tok, const int32_t *seq, T *cat, int rows, int k, cudaStream_t s);
+
+// ---------------------------------------------------------------- launchers (gemm_ref.cu)
+template <typename T>
+void launch_gemm_ref(const T *x, const T *w, float *out, int rows, int O, int I, int ldo, cudaStream_t s);
+
+// ---------------------------------------------------------------- launchers (attn_ref.cu)
+template <typename T>
+void launch_attn_ref(const T *q, KvPool pool, PageMap pm, RowMeta m, int tail_len, T *out, int rows, int H, int G,
+                     int hd, int max_keys, cudaStream_t s);
+size_t attn_ref_smem_bytes(int max_keys, int hd);
+
+// ---------------------------------------------------------------- launchers (tree.cu)
+void launch_logsoftmax_topk(const float *logits, int rows, int n, int K, int32_t *idx, float *lp, cudaStream_t s);
+void launch_argmax(const float *logits, int rows, int n, int32_t *idx, cudaStream_t s);
+
+}  // namespace spec

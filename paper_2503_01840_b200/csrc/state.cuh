@@ -1,0 +1,46 @@
+// Device-resident per-sequence state and tree buffers of a speculative-step context.
+#pragma once
+#include "common.cuh"
+
+namespace spec {
+
+struct SeqState {        // arrays of [batch]
+  int32_t *n;            // committed length; the root token sits at position n
+  int32_t *n_prev;       // n before the last commit
+  int32_t *P;            // pending draft entries (positions n-P .. n-1)
+  int32_t *root;         // token at position n (already emitted)
+  int32_t *cap;          // positions this sequence has pages for
+  int32_t *last_row;     // row of the last pending entry in the extend pass
+  int32_t *active;       // 0: sequence skipped this step (capacity)
+};
+
+struct TreeBufs {
+  int32_t pool, K, D, N, Pmax;          // pool = K + (D-1) K^2 ; Pmax = D + 1
+  int32_t *pool_tok, *pool_parent, *pool_depth;   // [B][pool+1]
+  float *pool_score;
+  int32_t *frontier;     // [B][D][K] pool indices processed by each pass
+  int32_t *front_cur;    // [B][K]
+  int32_t *feat_row;     // [B*K] row (of the previous pass's residual) holding the parent's output
+  int32_t *tk_idx;       // [rows][K] top-k draft ids
+  float *tk_lp;          // [rows][K]
+  int32_t *tok, *parent, *depth, *poolidx;   // [B][N]
+  float *score;
+  uint64_t *mask;
+  int32_t *nn;           // [B] nodes in the tree
+  int32_t *y;            // [B*N] target argmax per node
+  int32_t *path;         // [B][Pmax]
+  int32_t *out_ids;      // [B][Pmax]
+  int32_t *out_cnt;      // [B]
+  int32_t *pend_tok;     // [B][Pmax] token following each pending position
+};
+
+void launch_prep_extend(SeqState st, TreeBufs tb, RowMeta m, int B, int need_positions, int32_t *status, cudaStream_t s);
+void launch_expand(SeqState st, TreeBufs tb, RowMeta m, const int32_t *d2t, int pass, int B, cudaStream_t s);
+void launch_rerank(SeqState st, TreeBufs tb, RowMeta m, int B, cudaStream_t s);
+void launch_plain_tree(SeqState st, TreeBufs tb, RowMeta m, int B, cudaStream_t s);
+void launch_accept(SeqState st, TreeBufs tb, int B, int rows_per_seq, cudaStream_t s);
+template <typename T>
+void launch_commit(SeqState st, TreeBufs tb, const KvPool *pools /*device array [L]*/, PageMap pm, const T *node_taps,
+                   T *pend_taps, int B, int L, int G, int hd, int k, int rows_per_seq, cudaStream_t s);
+
+}  // namespace spec

@@ -1,0 +1,380 @@
+// Integer / fp32-compare kernels of the step: per-row log-softmax + top-k, dynamic-tree expansion
+// (Section 2.2: expand by draft confidence, cumulative log-probability as the node value), the
+// end-of-draft pruning ("rerank") that fixes the verified tree and its ancestor masks, per-node
+// argmax, greedy acceptance (Section 2.1 at temperature 0) and KV-cache compaction.
+#include "state.cuh"
+
+namespace spec {
+
+// ---------------------------------------------------------------- block argmax helpers
+struct VI { float v; int i; };
+// "a before b" in (value desc, index asc) order
+__device__ __forceinline__ bool before(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
+
+__device__ __forceinline__ VI block_best(VI x, VI *sh) {
+  for (int o = 16; o > 0; o >>= 1) {
+    float ov = __shfl_xor_sync(0xffffffffu, x.v, o);
+    int oi = __shfl_xor_sync(0xffffffffu, x.i, o);
+    if (oi >= 0 && (x.i < 0 || before(ov, oi, x.v, x.i))) { x.v = ov; x.i = oi; }
+  }
+  int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
+  if (l == 0) sh[w] = x;
+  __syncthreads();
+  if (w == 0) {
+    VI t = (l < nw) ? sh[l] : VI{0.0f, -1};
+    for (int o = 16; o > 0; o >>= 1) {
+      float ov = __shfl_xor_sync(0xffffffffu, t.v, o);
+      int oi = __shfl_xor_sync(0xffffffffu, t.i, o);
+      if (oi >= 0 && (t.i < 0 || before(ov, oi, t.v, t.i))) { t.v = ov; t.i = oi; }
+    }
+    if (l == 0) sh[0] = t;
+  }
+  __syncthreads();
+  VI r = sh[0];
+  __syncthreads();
+  return r;
+}
+
+__global__ void __launch_bounds__(256) argmax_kernel(const float *__restrict__ logits, int n, int32_t *__restrict__ out) {
+  __shared__ VI sh[32];
+  const float *z = logits + (size_t)blockIdx.x * n;
+  VI b{0.0f, -1};
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    float v = z[i];
+    if (b.i < 0 || before(v, i, b.v, b.i)) { b.v = v; b.i = i; }
+  }
+  b = block_best(b, sh);
+  if (threadIdx.x == 0) out[blockIdx.x] = b.i;
+}
+void launch_argmax(const float *logits, int rows, int n, int32_t *idx, cudaStream_t s) {
+  argmax_kernel<<<rows, 256, 0, s>>>(logits, n, idx);
+}
+
+// log-softmax + top-K, (value desc, index asc).  Row r reads logits row src_row[r] when given.
+__global__ void __launch_bounds__(256) logsoftmax_topk_kernel(const float *__restrict__ logits, const int32_t *src_row,
+                                                              int n, int K, int32_t *__restrict__ idx,
+                                                              float *__restrict__ lp) {
+  __shared__ VI sh[32];
+  __shared__ float shf[32];
+  int r = blockIdx.x;
+  int sr = src_row ? src_row[r] : r;
+  if (sr < 0) {
+    for (int c = threadIdx.x; c < K; c += blockDim.x) { idx[(size_t)r * K + c] = 0; lp[(size_t)r * K + c] = 0.0f; }
+    return;
+  }
+  const float *z = logits + (size_t)sr * n;
+  float mx = -INFINITY;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) mx = fmaxf(mx, z[i]);
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  mx = shf[0];
+  for (int w = 1; w < (int)(blockDim.x >> 5); w++) mx = fmaxf(mx, shf[w]);
+  __syncthreads();
+  float sum = 0.0f;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) sum += expf(z[i] - mx);
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  sum = 0.0f;
+  for (int w = 0; w < (int)(blockDim.x >> 5); w++) sum += shf[w];
+  float lse = logf(sum);
+  __syncthreads();
+  float pv = INFINITY;
+  int pi = -1;
+  for (int c = 0; c < K; c++) {
+    VI b{0.0f, -1};
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      float v = (z[i] - mx) - lse;
+      bool after_prev = (pi < 0) || before(pv, pi, v, i);
+      if (after_prev && (b.i < 0 || before(v, i, b.v, b.i))) { b.v = v; b.i = i; }
+    }
+    b = block_best(b, sh);
+    if (threadIdx.x == 0) { idx[(size_t)r * K + c] = b.i; lp[(size_t)r * K + c] = b.v; }
+    pv = b.v; pi = b.i;
+  }
+}
+void launch_logsoftmax_topk(const float *logits, int rows, int n, int K, int32_t *idx, float *lp, cudaStream_t s) {
+  logsoftmax_topk_kernel<<<rows, 256, 0, s>>>(logits, nullptr, n, K, idx, lp);
+}
+void launch_logsoftmax_topk_rows(const float *logits, const int32_t *src_row, int rows, int n, int K, int32_t *idx,
+                                 float *lp, cudaStream_t s) {
+  logsoftmax_topk_kernel<<<rows, 256, 0, s>>>(logits, src_row, n, K, idx, lp);
+}
+
+// ---------------------------------------------------------------- step set-up: rows of the extend pass
+// Row b*Pmax + j is pending entry j of sequence b: position n-P+j, causal among the pending rows.
+__global__ void prep_extend_kernel(SeqState st, TreeBufs tb, RowMeta m, int need_positions, int32_t *status) {
+  int b = blockIdx.x, j = threadIdx.x;
+  int n = st.n[b], P = st.P[b];
+  bool ok = (n + need_positions <= st.cap[b]) && P >= 1 && P <= tb.Pmax;
+  if (j == 0) {
+    st.active[b] = ok ? 1 : 0;
+    st.last_row[b] = ok ? b * tb.Pmax + P - 1 : -1;
+    if (!ok) set_status(status, ST_CAPACITY, 10, b, n);
+    tb.frontier[(size_t)b * tb.D * tb.K] = 0;
+    tb.pool_tok[(size_t)b * (tb.pool + 1)] = st.root[b];
+    tb.pool_parent[(size_t)b * (tb.pool + 1)] = -1;
+    tb.pool_depth[(size_t)b * (tb.pool + 1)] = 0;
+    tb.pool_score[(size_t)b * (tb.pool + 1)] = 0.0f;
+  }
+  if (j >= tb.Pmax) return;
+  int r = b * tb.Pmax + j;
+  bool valid = ok && j < P;
+  m.seq[r] = valid ? b : -1;
+  m.pos[r] = valid ? n - P + j : 0;
+  m.kvpos[r] = valid ? n - P + j : 0;
+  m.ctx[r] = valid ? n - P : 0;
+  m.tail_base[r] = valid ? n - P : 0;
+  m.mask_lo[r] = valid ? ((j >= 63) ? ~0ull : ((1ull << (j + 1)) - 1ull)) : 0ull;
+  m.mask_hi[r] = 0ull;
+  m.tok[r] = valid ? tb.pend_tok[b * tb.Pmax + j] : 0;
+}
+void launch_prep_extend(SeqState st, TreeBufs tb, RowMeta m, int B, int need_positions, int32_t *status, cudaStream_t s) {
+  int threads = ((tb.Pmax + 31) / 32) * 32;
+  prep_extend_kernel<<<B, threads, 0, s>>>(st, tb, m, need_positions, status);
+}
+
+// ---------------------------------------------------------------- dynamic-tree expansion after draft pass `pass` (1-based)
+// Adds this pass's children to the pool (cumulative log-prob scores), picks the next frontier (the K
+// best of the level) and writes the row metadata of the next draft pass.
+__global__ void __launch_bounds__(256) expand_kernel(SeqState st, TreeBufs tb, RowMeta m, const int32_t *__restrict__ d2t,
+                                                     int pass) {
+  extern __shared__ unsigned char smraw[];
+  int K = tb.K, D = tb.D, b = blockIdx.x;
+  int nch = (pass == 1) ? K : K * K;        // children created by this pass
+  float *cs = (float *)smraw;               // [nch] child scores
+  uint64_t *pm_lo = (uint64_t *)(cs + ((nch + 1) & ~1));   // [K] parent masks
+  uint64_t *pm_hi = pm_lo + K;
+  int32_t *newf = (int32_t *)(pm_hi + K);   // [K] local child index of the new frontier
+  if (!st.active[b]) {   // skipped sequence: its rows of the next pass are padding
+    for (int rr = threadIdx.x; rr < K; rr += blockDim.x) { m.seq[b * K + rr] = -1; m.tok[b * K + rr] = 0; m.pos[b * K + rr] = 0; }
+    return;
+  }
+  size_t pb = (size_t)b * (tb.pool + 1);
+  int base = (pass == 1) ? 0 : K + (pass - 2) * K * K;     // pool index of child 0 is base + 1
+  int n = st.n[b];
+  for (int c = threadIdx.x; c < nch; c += blockDim.x) {
+    int r = (pass == 1) ? 0 : c / K, cc = (pass == 1) ? c : c % K;
+    int row = (pass == 1) ? b : b * K + r;                  // row of the top-k output
+    int u = (pass == 1) ? 0 : tb.front_cur[b * K + r];
+    float sc = tb.pool_score[pb + u] + tb.tk_lp[(size_t)row * K + cc];
+    int ci = base + c + 1;
+    tb.pool_tok[pb + ci] = d2t[tb.tk_idx[(size_t)row * K + cc]];
+    tb.pool_parent[pb + ci] = u;
+    tb.pool_depth[pb + ci] = pass;
+    tb.pool_score[pb + ci] = sc;
+    cs[c] = sc;
+  }
+  for (int r = threadIdx.x; r < K; r += blockDim.x) {
+    pm_lo[r] = (pass == 1) ? 0ull : m.mask_lo[b * K + r];
+    pm_hi[r] = (pass == 1) ? 0ull : m.mask_hi[b * K + r];
+  }
+  __syncthreads();
+  if (pass >= D) return;
+  // next frontier: rank by (score desc, pool index asc)
+  for (int c = threadIdx.x; c < nch; c += blockDim.x) {
+    float s = cs[c];
+    int rank = 0;
+    for (int j = 0; j < nch; j++) rank += (cs[j] > s || (cs[j] == s && j < c)) ? 1 : 0;
+    if (rank < K) newf[rank] = c;
+  }
+  __syncthreads();
+  int last_row = st.last_row[b];
+  for (int rr = threadIdx.x; rr < K; rr += blockDim.x) {
+    int c = newf[rr];
+    int ci = base + c + 1;
+    int pr = (pass == 1) ? 0 : c / K;                       // parent's rank in the current pass
+    int row = b * K + rr;
+    int slot = (pass - 1) * K + rr;
+    tb.front_cur[b * K + rr] = ci;
+    tb.frontier[((size_t)b * D + pass) * K + rr] = ci;
+    tb.feat_row[row] = (pass == 1) ? last_row : b * K + pr;
+    uint64_t lo = pm_lo[pr], hi = pm_hi[pr];
+    if (slot < 64) lo |= 1ull << slot; else hi |= 1ull << (slot - 64);
+    m.seq[row] = b;
+    m.pos[row] = n + pass - 1;
+    m.kvpos[row] = n + slot;
+    m.ctx[row] = n;
+    m.tail_base[row] = n;
+    m.mask_lo[row] = lo;
+    m.mask_hi[row] = hi;
+    m.tok[row] = tb.pool_tok[pb + ci];
+  }
+}
+void launch_expand(SeqState st, TreeBufs tb, RowMeta m, const int32_t *d2t, int pass, int B, cudaStream_t s) {
+  int K = tb.K, nch = K * K;
+  size_t smem = (size_t)((nch + 1) & ~1) * 4 + (size_t)K * 16 + (size_t)K * 4 + 16;
+  expand_kernel<<<B, 256, smem, s>>>(st, tb, m, d2t, pass);
+}
+
+// ---------------------------------------------------------------- pruning + tree assembly
+// Keeps the M = min(N-1, pool) best candidates (score desc, pool index asc), numbers them in pool
+// order after the root and emits parents, depths, ancestor-or-self bit masks and the verify rows.
+__global__ void __launch_bounds__(256) rerank_kernel(SeqState st, TreeBufs tb, RowMeta m) {
+  extern __shared__ unsigned char smraw[];
+  int b = blockIdx.x, pool = tb.pool, N = tb.N;
+  float *sc = (float *)smraw;                       // [pool+1]
+  int32_t *node_of = (int32_t *)(sc + pool + 1);    // [pool+1], -1 = dropped
+  int32_t *par = node_of + pool + 1;                // [pool+1]
+  int M = (N - 1 < pool) ? N - 1 : pool;
+  size_t pb = (size_t)b * (pool + 1);
+  int n = st.n[b];
+  bool act = st.active[b] != 0;
+  for (int i = threadIdx.x; i <= pool; i += blockDim.x) { sc[i] = tb.pool_score[pb + i]; par[i] = tb.pool_parent[pb + i]; }
+  __syncthreads();
+  for (int i = threadIdx.x; i <= pool; i += blockDim.x) {
+    if (i == 0) { node_of[0] = 0; continue; }
+    float s = sc[i];
+    int rank = 0;
+    for (int j = 1; j <= pool; j++) rank += (sc[j] > s || (sc[j] == s && j < i)) ? 1 : 0;
+    node_of[i] = (rank < M) ? 1 : -1;
+  }
+  __syncthreads();
+  // number the kept candidates in pool order
+  int mine[4];   // pool <= 1024 with 256 threads -> up to 4 candidates each (checked on the host)
+  int cnt = 0;
+  for (int i = threadIdx.x; i <= pool; i += blockDim.x) {
+    int idx = -1;
+    if (i == 0) idx = 0;
+    else if (node_of[i] > 0) {
+      idx = 1;
+      for (int j = 1; j < i; j++) idx += (node_of[j] > 0) ? 1 : 0;
+    }
+    mine[cnt++] = idx;
+  }
+  __syncthreads();
+  cnt = 0;
+  for (int i = threadIdx.x; i <= pool; i += blockDim.x) node_of[i] = mine[cnt++];
+  __syncthreads();
+  if (threadIdx.x == 0) tb.nn[b] = act ? M + 1 : 0;
+  for (int i = threadIdx.x; i <= pool; i += blockDim.x) {
+    int ni = node_of[i];
+    if (ni < 0) continue;
+    uint64_t mask = 0;
+    for (int v = i, it = 0; v >= 0 && v <= pool && it < 64; v = par[v], it++) mask |= 1ull << (node_of[v] & 63);
+    size_t t = (size_t)b * N + ni;
+    int depth = tb.pool_depth[pb + i];
+    tb.tok[t] = tb.pool_tok[pb + i];
+    tb.parent[t] = (i == 0) ? -1 : node_of[par[i]];
+    tb.depth[t] = depth;
+    tb.poolidx[t] = i;
+    tb.score[t] = sc[i];
+    tb.mask[t] = mask;
+    m.seq[t] = act ? b : -1;
+    m.pos[t] = act ? n + depth : 0;
+    m.kvpos[t] = act ? n + ni : 0;
+    m.ctx[t] = act ? n : 0;
+    m.tail_base[t] = act ? n : 0;
+    m.mask_lo[t] = mask;
+    m.mask_hi[t] = 0ull;
+    m.tok[t] = act ? tb.pool_tok[pb + i] : 0;
+  }
+  // rows beyond the tree (only when pool < N-1) are padding
+  for (int i = M + 1 + threadIdx.x; i < N; i += blockDim.x) {
+    size_t t = (size_t)b * N + i;
+    m.seq[t] = -1; m.pos[t] = 0; m.kvpos[t] = 0; m.ctx[t] = 0; m.tail_base[t] = 0;
+    m.mask_lo[t] = 0; m.mask_hi[t] = 0; m.tok[t] = 0;
+  }
+}
+void launch_rerank(SeqState st, TreeBufs tb, RowMeta m, int B, cudaStream_t s) {
+  size_t smem = (size_t)(tb.pool + 1) * 12 + 16;
+  rerank_kernel<<<B, 256, smem, s>>>(st, tb, m);
+}
+
+// Tree of the root alone (plain autoregressive decoding on the same kernels): one row per sequence.
+__global__ void plain_tree_kernel(SeqState st, TreeBufs tb, RowMeta m, int B) {
+  int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  int n = st.n[b];
+  bool act = n + 1 <= st.cap[b];
+  st.active[b] = act ? 1 : 0;
+  tb.nn[b] = act ? 1 : 0;
+  tb.tok[b] = st.root[b]; tb.parent[b] = -1; tb.depth[b] = 0; tb.poolidx[b] = 0; tb.score[b] = 0.0f; tb.mask[b] = 1ull;
+  m.seq[b] = act ? b : -1; m.pos[b] = n; m.kvpos[b] = n; m.ctx[b] = n; m.tail_base[b] = n;
+  m.mask_lo[b] = 1ull; m.mask_hi[b] = 0ull; m.tok[b] = act ? st.root[b] : 0;
+}
+void launch_plain_tree(SeqState st, TreeBufs tb, RowMeta m, int B, cudaStream_t s) {
+  plain_tree_kernel<<<(B + 63) / 64, 64, 0, s>>>(st, tb, m, B);
+}
+
+// ---------------------------------------------------------------- greedy acceptance
+// Follow, from the root, the child whose token equals the target's argmax at the current node.
+__global__ void accept_kernel(SeqState st, TreeBufs tb, int rows_per_seq) {
+  int b = blockIdx.x;
+  if (threadIdx.x != 0) return;
+  int Pmax = tb.Pmax;
+  int nn = tb.nn[b];
+  if (!st.active[b] || nn < 1) { tb.out_cnt[b] = 0; return; }
+  const int32_t *tok = tb.tok + (size_t)b * rows_per_seq, *par = tb.parent + (size_t)b * rows_per_seq;
+  const int32_t *y = tb.y + (size_t)b * rows_per_seq;
+  int cur = 0, a = 0;
+  tb.path[b * Pmax] = 0;
+  while (a + 1 < Pmax) {
+    int nxt = -1;
+    for (int c = cur + 1; c < nn; c++)
+      if (par[c] == cur && tok[c] == y[cur]) { nxt = c; break; }
+    if (nxt < 0) break;
+    tb.out_ids[b * Pmax + a] = tok[nxt];
+    tb.pend_tok[b * Pmax + a] = tok[nxt];
+    cur = nxt;
+    tb.path[b * Pmax + (++a)] = cur;
+  }
+  tb.out_ids[b * Pmax + a] = y[cur];
+  tb.pend_tok[b * Pmax + a] = y[cur];
+  for (int j = a + 1; j < Pmax; j++) tb.out_ids[b * Pmax + j] = -1;
+  tb.out_cnt[b] = a + 1;
+  int n = st.n[b];
+  st.n_prev[b] = n;
+  st.n[b] = n + a + 1;
+  st.P[b] = a + 1;
+  st.root[b] = y[cur];
+}
+void launch_accept(SeqState st, TreeBufs tb, int B, int rows_per_seq, cudaStream_t s) {
+  accept_kernel<<<B, 32, 0, s>>>(st, tb, rows_per_seq);
+}
+
+// ---------------------------------------------------------------- commit: KV compaction + tap gather
+// Accepted node path[j] (K/V at cache position n+path[j]) moves to position n+j in every layer; its
+// taps become pending entry j.  path[j] >= j and is increasing, and a thread copies the same element
+// offsets for every j, so the in-place move in increasing j never reads an overwritten slot.
+template <typename T>
+__global__ void __launch_bounds__(256) commit_kernel(SeqState st, TreeBufs tb, const KvPool *__restrict__ pools,
+                                                     PageMap pm, const T *__restrict__ node_taps,
+                                                     T *__restrict__ pend_taps, int L, int G, int hd, int k,
+                                                     int rows_per_seq) {
+  int b = blockIdx.x, l = blockIdx.y;
+  int cnt = tb.out_cnt[b];
+  if (cnt <= 0) return;
+  int n0 = st.n_prev[b], Pmax = tb.Pmax;
+  if (l < L) {
+    T *Kp = (T *)pools[l].k, *Vp = (T *)pools[l].v;
+    for (int j = 0; j < cnt; j++) {
+      int src = n0 + tb.path[b * Pmax + j], dst = n0 + j;
+      if (src == dst) continue;
+      for (int e = threadIdx.x; e < G * hd; e += blockDim.x) {
+        int g = e / hd, i = e % hd;
+        size_t so = kv_offset(pm, b, src, g, G, hd) + i, dof = kv_offset(pm, b, dst, g, G, hd) + i;
+        Kp[dof] = Kp[so];
+        Vp[dof] = Vp[so];
+      }
+    }
+  } else {
+    for (int j = 0; j < cnt; j++) {
+      const T *src = node_taps + ((size_t)b * rows_per_seq + tb.path[b * Pmax + j]) * 3 * k;
+      T *dst = pend_taps + ((size_t)b * Pmax + j) * 3 * k;
+      for (int e = threadIdx.x; e < 3 * k; e += blockDim.x) dst[e] = src[e];
+    }
+  }
+}
+template <typename T>
+void launch_commit(SeqState st, TreeBufs tb, const KvPool *pools, PageMap pm, const T *node_taps, T *pend_taps, int B,
+                   int L, int G, int hd, int k, int rows_per_seq, cudaStream_t s) {
+  commit_kernel<T><<<dim3(B, L + 1), 256, 0, s>>>(st, tb, pools, pm, node_taps, pend_taps, L, G, hd, k, rows_per_seq);
+}
+template void launch_commit<float>(SeqState, TreeBufs, const KvPool *, PageMap, const float *, float *, int, int, int,
+                                   int, int, int, cudaStream_t);
+template void launch_commit<bf16>(SeqState, TreeBufs, const KvPool *, PageMap, const bf16 *, bf16 *, int, int, int, int,
+                                  int, int, cudaStream_t);
+
+}  // namespace spec

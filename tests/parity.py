@@ -1,0 +1,169 @@
+"""Step-by-step comparison of the CUDA path with the CPU oracle on identical seeded inputs.
+
+Rule: integer results (tree structure, argmax, accepted ids, counts) must be bit-exact wherever every
+decision that led to them had an oracle margin above MARGIN; floating-point results (logits, hidden
+states, taps) must agree within `tol` max-abs.  One flipped low-margin decision changes all later
+state, so after every step the oracle is put into the CUDA path's committed state (resync)."""
+import numpy as np
+import torch
+
+import pyoracle as po
+from paper_2503_01840_b200 import binding as sb
+from paper_2503_01840_b200 import synth
+
+MARGIN = 1e-2
+
+
+def to_dev(w, dev="cuda"):
+    if isinstance(w, dict):
+        return {k: to_dev(v, dev) for k, v in w.items()}
+    if isinstance(w, list):
+        return [to_dev(v, dev) for v in w]
+    return w.to(dev).contiguous()
+
+
+def to_cpu(w):
+    return to_dev(w, "cpu")
+
+
+class Stats:
+    def __init__(self):
+        self.steps = self.exact_tree = self.same_tree = self.exact_out = self.resyncs = self.tokens = 0
+        self.max_err = {}
+
+    def err(self, name, a, b):
+        e = float(np.abs(np.asarray(a, np.float64) - np.asarray(b, np.float64)).max()) if np.size(a) else 0.0
+        self.max_err[name] = max(self.max_err.get(name, 0.0), e)
+        return e
+
+    def __repr__(self):
+        errs = ", ".join(f"{k}={v:.2e}" for k, v in sorted(self.max_err.items()))
+        return (f"steps={self.steps} exact_tree={self.exact_tree} same_tree={self.same_tree} exact_out={self.exact_out} resyncs={self.resyncs} "
+                f"tokens={self.tokens} | {errs}")
+
+
+def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_tol=None):
+    """`orc` has just executed the same step from the same state.  Returns True if outputs were
+    required to be (and were) identical."""
+    K, D, N, Vd, k, V = cfg.tree_topk, cfg.tree_depth, cfg.tree_nodes, cfg.draft_vocab, cfg.hidden, cfg.vocab
+    tap_tol = tol if tap_tol is None else tap_tol
+    o_front = orc.get(po.FRONTIER).reshape(D, K)
+    g_front = dec.debug(sb.DBG_FRONTIER, seq).reshape(D, K)
+    tk_m = orc.get(po.TOPK_MARGIN).reshape(D, K)
+    fr_m = orc.get(po.FRONTIER_MARGIN)
+    rr_m = float(orc.get(po.RERANK_MARGIN)[0])
+    capture = check_floats
+    if capture:
+        g_dl = dec.debug(sb.DBG_DRAFT_LOGITS, seq).reshape(D, K, Vd)
+        g_da = dec.debug(sb.DBG_DRAFT_A, seq).reshape(D, K, k)
+        o_dl = orc.get(po.DRAFT_LOGITS).reshape(D, K, Vd)
+        o_da = orc.get(po.DRAFT_A).reshape(D, K, k)
+    # draft passes: comparable while the frontier (and its order) is the same
+    safe = True                                    # every decision so far had margin
+    o_ptok, g_ptok = orc.get(po.POOL_TOK), dec.debug(sb.DBG_POOL_TOK, seq)
+    for d in range(D):
+        rows = 1 if d == 0 else K
+        # same nodes in the same order, carrying the same tokens (a swapped near-tie inside one top-k
+        # row keeps the pool indices but exchanges the tokens)
+        same_front = d == 0 or (np.array_equal(o_front[d], g_front[d]) and
+                                np.array_equal(o_ptok[o_front[d]], g_ptok[g_front[d]]))
+        if d > 0 and safe:
+            assert same_front, f"frontier of pass {d} differs although all margins > {MARGIN}: {o_front[d]} vs {g_front[d]}"
+        if not same_front:
+            safe = False
+            break
+        if capture:
+            assert st.err("draft_logits", g_dl[d, :rows], o_dl[d, :rows]) <= tol, (d, st.max_err)
+            assert st.err("draft_a", g_da[d, :rows], o_da[d, :rows]) <= tol, (d, st.max_err)
+        if tk_m[d, :rows].min() <= MARGIN or (d + 1 < D and d >= 1 and fr_m[d] <= MARGIN):
+            safe = False
+            # later passes may still coincide; keep comparing floats only if frontiers match
+    safe_tree = bool((tk_m[np.isfinite(tk_m)] > MARGIN).all() and (fr_m[np.isfinite(fr_m)] > MARGIN).all() and rr_m > MARGIN)
+    ints = {n: (dec.debug(g, seq), orc.get(o)) for n, g, o in (
+        ("tok", sb.DBG_TREE_TOK, po.TREE_TOK), ("parent", sb.DBG_TREE_PARENT, po.TREE_PARENT),
+        ("depth", sb.DBG_TREE_DEPTH, po.TREE_DEPTH), ("mask", sb.DBG_TREE_MASK, po.TREE_MASK),
+        ("poolidx", sb.DBG_TREE_POOLIDX, po.TREE_POOLIDX))}
+    same_tree = all(np.array_equal(a, b) for a, b in ints.values())
+    st.same_tree += int(same_tree)
+    if safe_tree:
+        for n, (a, b) in ints.items():
+            assert np.array_equal(a, b), f"tree {n} differs although all margins > {MARGIN}\n{a}\n{b}"
+        st.exact_tree += 1
+    # GPU tree must be a valid tree whatever the margins
+    g_par, g_dep, g_mask = ints["parent"][0], ints["depth"][0], ints["mask"][0]
+    for i in range(g_par.size):
+        if i == 0:
+            assert g_par[0] == -1 and g_dep[0] == 0 and int(g_mask[0]) == 1
+        else:
+            p = int(g_par[i])
+            assert 0 <= p < i and g_dep[i] == g_dep[p] + 1 and int(g_mask[i]) == (int(g_mask[p]) | (1 << i))
+    exact_out = False
+    if same_tree:
+        nn = ints["tok"][0].size
+        assert st.err("tree_score", dec.debug(sb.DBG_TREE_SCORE, seq), orc.get(po.TREE_SCORE)) <= tol
+        if check_floats:
+            assert st.err("target_logits", dec.debug(sb.DBG_TARGET_LOGITS, seq), orc.get(po.TARGET_LOGITS)) <= tol, st.max_err
+            assert st.err("node_hidden", dec.debug(sb.DBG_NODE_HIDDEN, seq), orc.get(po.NODE_HIDDEN)) <= tol, st.max_err
+            assert st.err("node_taps", dec.debug(sb.DBG_NODE_TAPS, seq), orc.get(po.NODE_TAPS)) <= tap_tol, st.max_err
+        gy, oy, ym = dec.debug(sb.DBG_Y, seq), orc.get(po.Y), orc.get(po.Y_MARGIN)
+        big = ym > MARGIN
+        assert np.array_equal(gy[big], oy[big]), "argmax differs at a node with margin"
+        o_path = orc.get(po.PATH)
+        if big[o_path].all():
+            g_path = dec.debug(sb.DBG_PATH, seq)
+            assert np.array_equal(g_path, o_path), (g_path, o_path)
+            exact_out = True
+    return exact_out
+
+
+def run_trajectory(cfg, tw, dw, prompts, n_steps, tol, flags=0, max_ctx=None, check_floats=True, tap_tol=None,
+                   page_shuffle_seed=0, num_pages=None):
+    """tw/dw: CPU weight dicts.  Returns Stats; raises AssertionError on a parity violation."""
+    B = len(prompts)
+    reserve = n_steps * (cfg.tree_depth + 1) + 8
+    if max_ctx is None:
+        max_ctx = max(len(p) for p in prompts) + reserve + 2 * max(cfg.tree_nodes, (cfg.tree_depth - 1) * cfg.tree_topk) + 8
+    if check_floats:
+        flags |= sb.FLAG_CAPTURE
+    dec = sb.SpecDecoder(cfg, to_dev(tw), to_dev(dw), batch=B, max_ctx=max_ctx, flags=flags,
+                         page_shuffle_seed=page_shuffle_seed, num_pages=num_pages)
+    st = Stats()
+    first = dec.prefill([np.asarray(p) for p in prompts], reserve)
+    orcs = []
+    for b in range(B):
+        o = po.Oracle(cfg, tw, dw, max_ctx)
+        f = o.prefill(np.asarray(prompts[b]))
+        assert f == first[b], f"first token differs for sequence {b}: {f} vs {first[b]}"
+        orcs.append(o)
+    emitted = [[] for _ in range(B)]
+    for step in range(n_steps):
+        outs = dec.step()
+        for b in range(B):
+            o = orcs[b]
+            ids_before, n_before = o.ids, o.n
+            o_out = o.step()
+            g_out = outs[b]
+            assert 1 <= len(g_out) <= cfg.tree_depth + 1
+            exact = compare_step(dec, o, b, cfg, tol, st, g_out, check_floats, tap_tol)
+            if exact:
+                assert np.array_equal(g_out, o_out), (g_out, o_out)
+                st.exact_out += 1
+            emitted[b] += g_out.tolist()
+            if not np.array_equal(g_out, o_out):
+                st.resyncs += 1
+                new_ids = np.concatenate([ids_before, g_out]).astype(np.int32)
+                o.force_state(new_ids, n_before + len(g_out), len(g_out))
+            st.tokens += len(g_out)
+        st.steps += 1
+        assert np.array_equal(dec.lengths(), [o.n for o in orcs])
+    # losslessness against plain greedy decoding of the oracle, up to the first low-margin token
+    for b in range(B):
+        g = po.Oracle(cfg, tw, dw, max_ctx)
+        g.prefill(np.asarray(prompts[b]))
+        ref, mg = g.greedy_margins(len(emitted[b]))
+        for i, (a, r) in enumerate(zip(emitted[b], ref)):
+            if a != r:
+                assert mg[i] <= MARGIN, f"sequence {b}: token {i} differs from greedy decoding with margin {mg[i]}"
+                break
+    dec.close()
+    return st, emitted

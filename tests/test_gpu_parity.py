@@ -1,0 +1,251 @@
+"""GPU parity tests: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import parity
+import pyoracle as po
+from paper_2503_01840_b200 import binding as sb
+from paper_2503_01840_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+C1 = synth.C1
+# the tiny model in bf16: exercises the tcgen05 GEMM and bf16 caches at a size the oracle runs in ms
+T1 = C1.replace(name="T1-tiny-bf16", dtype="bf16")
+# a wider small bf16 model with head_dim 128 and 4 query heads per KV head, like the 8B shapes
+T2 = synth.ModelCfg("T2-small-bf16", "bf16", 3, 512, 8, 2, 128, 1408, 8192, 2048, (0, 1, 2), 5e5,
+                    prompt_len=150, tree_depth=4, tree_topk=5, tree_nodes=24, seed=11)
+
+
+def _weights(cfg):
+    return synth.make_target_weights(cfg), synth.make_draft_weights(cfg)
+
+
+# ----------------------------------------------------------------------------- single kernels
+@pytest.mark.parametrize("rows,O,I", [(1, 128, 64), (7, 256, 256), (10, 1000, 512), (16, 4096, 4096), (17, 384, 200),
+                                      (60, 6144, 4096), (64, 128, 14336), (65, 640, 1024), (200, 512, 768),
+                                      (256, 1024, 2048)])
+def test_gemm_tcgen05_vs_oracle(rows, O, I):
+    g = torch.Generator().manual_seed(rows * 1000 + O + I)
+    x = (torch.randn(rows, I, generator=g)).to(torch.bfloat16)
+    w = (torch.randn(O, I, generator=g) / I ** 0.5).to(torch.bfloat16)
+    ref = po.linear(w, x.float().numpy())
+    out = sb.gemm(x.cuda(), w.cuda(), impl=0).cpu().numpy()
+    assert np.isfinite(out).all()
+    assert np.abs(out - ref).max() < 2e-3, np.abs(out - ref).max()
+    out_ref_kernel = sb.gemm(x.cuda(), w.cuda(), impl=1).cpu().numpy()
+    assert np.abs(out_ref_kernel - ref).max() < 2e-3
+
+
+def test_gemm_plain_fp32_vs_oracle():
+    g = torch.Generator().manual_seed(5)
+    x, w = torch.randn(33, 300, generator=g), torch.randn(77, 300, generator=g) / 17
+    ref = po.linear(w, x.numpy())
+    out = sb.gemm(x.cuda(), w.cuda(), impl=1).cpu().numpy()
+    assert np.abs(out - ref).max() < 1e-4
+
+
+def test_logsoftmax_topk_and_argmax_bit_exact():
+    g = torch.Generator().manual_seed(6)
+    z = torch.randn(12, 32000, generator=g) * 1.5
+    z[3, 100] = z[3, 200] = z[3].max() + 1.0          # a tie at the top: lowest index first
+    z[5, :] = 0.25                                     # all equal
+    idx, lp = sb.logsoftmax_topk(z.cuda(), 10)
+    am = sb.argmax(z.cuda()).cpu().numpy()
+    idx, lp = idx.cpu().numpy(), lp.cpu().numpy()
+    for r in range(z.shape[0]):
+        olp = po.log_softmax(z[r].numpy())
+        oi, ov, _ = po.topk(olp, 10)
+        gaps = np.diff(ov)
+        if r in (3, 5) or (np.abs(gaps) > 1e-5).all():
+            assert idx[r].tolist() == oi.tolist(), r
+        assert np.abs(lp[r] - ov).max() < 1e-5
+        assert am[r] == po.argmax(z[r].numpy())[0]
+    assert idx[3, 0] == 100 and idx[3, 1] == 200 and idx[5].tolist() == list(range(10))
+    big = torch.randn(3, 128256, generator=g)
+    assert sb.argmax(big.cuda()).cpu().tolist() == big.argmax(1).tolist()
+
+
+@pytest.mark.parametrize("dtype,impl", [(torch.float32, 1), (torch.bfloat16, 1), (torch.bfloat16, 0)])
+def test_attention_kernel_vs_oracle(dtype, impl):
+    """Paged, tree-masked GQA attention against the oracle's per-head routine."""
+    H, G, hd, ps = 8, 2, 128, 16
+    if impl == 0 and not _fast_attn_available(hd, H // G):
+        pytest.skip("tensor-core attention not built for this shape")
+    g = torch.Generator().manual_seed(7)
+    n_seq, pps = 2, 24
+    ctx = [203, 77]
+    tail_len = 40
+    perm = torch.randperm(n_seq * pps, generator=g).to(torch.int32).reshape(n_seq, pps)
+    kp = torch.randn(n_seq * pps, G, ps, hd, generator=g).to(dtype)
+    vp = torch.randn(n_seq * pps, G, ps, hd, generator=g).to(dtype)
+    rows = 24
+    q = torch.randn(rows, H, hd, generator=g).to(dtype)
+    seq = torch.tensor([r % 2 for r in range(rows)], dtype=torch.int32)
+    seq[5] = -1
+    rctx = torch.tensor([ctx[r % 2] for r in range(rows)], dtype=torch.int32)
+    lo = torch.randint(0, 2 ** 40, (rows,), generator=g, dtype=torch.int64) | 1
+    lo[3] = 1
+    hi = torch.zeros(rows, dtype=torch.int64)
+    out = sb.attention(q.cuda(), kp.cuda(), vp.cuda(), perm.cuda(), ps, seq.cuda(), rctx.cuda(), rctx.cuda(),
+                       lo.cuda(), hi.cuda(), tail_len, G, 512, impl=impl).float().cpu().numpy()
+    tol = 1e-4 if dtype == torch.float32 else 2e-2
+    for r in range(rows):
+        if seq[r] < 0:
+            assert (out[r] == 0).all()
+            continue
+        s = int(seq[r])
+        pos = list(range(ctx[s])) + [ctx[s] + t for t in range(tail_len) if (int(lo[r]) >> t) & 1]
+        for h in range(H):
+            gk = h // (H // G)
+            K = np.stack([kp[perm[s, p // ps], gk, p % ps].float().numpy() for p in pos])
+            V = np.stack([vp[perm[s, p // ps], gk, p % ps].float().numpy() for p in pos])
+            ref = po.attend(q[r, h].float().numpy(), K, V)
+            assert np.abs(out[r, h] - ref).max() < tol, (r, h)
+
+
+def _fast_attn_available(hd, group):
+    return sb.lib().spec_attn_scratch_bytes(64, 8, hd, 1024) > 0
+
+
+# ----------------------------------------------------------------------------- whole step
+@pytest.mark.parametrize("flags", [0, sb.FLAG_NO_GRAPH])
+def test_c1_full_trajectory_fp32(flags):
+    """Config 1 end to end: 64-token prompt, depth 3, top-k 4, 16 nodes, 32 generated tokens, fp32, 1e-4."""
+    tw, dw = _weights(C1)
+    prompts = [p.numpy() for p in synth.make_prompts(C1)]
+    st, emitted = parity.run_trajectory(C1, tw, dw, prompts, n_steps=32, tol=1e-4, flags=flags)
+    print("C1", st)
+    assert st.tokens >= 32 and st.exact_tree >= 1 and st.same_tree >= 24 and st.exact_out >= 24
+
+
+@pytest.mark.parametrize("flags", [0, sb.FLAG_REF_GEMM | sb.FLAG_REF_ATTN])
+def test_tiny_bf16_trajectory(flags):
+    tw, dw = _weights(T1)
+    prompts = [p.numpy() for p in synth.make_prompts(T1)]
+    st, _ = parity.run_trajectory(T1, tw, dw, prompts, n_steps=16, tol=2e-2, flags=flags, tap_tol=3e-2)
+    print("T1", flags, st)
+    assert st.same_tree >= 4
+
+
+def test_small_bf16_hd128_trajectory():
+    tw, dw = _weights(T2)
+    prompts = [p.numpy() for p in synth.make_prompts(T2)]
+    st, _ = parity.run_trajectory(T2, tw, dw, prompts, n_steps=10, tol=2e-2, tap_tol=3e-2)
+    print("T2", st)
+
+
+@pytest.mark.parametrize("cfg", [C1, T1], ids=["fp32", "bf16"])
+def test_structured_weights_accept_more_than_one(cfg):
+    """Designed agreement between draft and target: counts > 1, KV compaction and multi-entry extend."""
+    tw, dw, pi, pi2 = synth.make_structured(cfg, 0.85, residual_scale=0.05)
+    prompt = synth.structured_prompt(cfg, dw["d2t"], 48).numpy()
+    tol = 1e-4 if cfg.dtype == "fp32" else 2e-2
+    st, emitted = parity.run_trajectory(cfg, tw, dw, [prompt], n_steps=12, tol=tol, tap_tol=tol * 1.5)
+    print("structured", cfg.name, st)
+    assert st.tokens > 12 + 6, "the structured workload must accept draft tokens"
+    # committed KV equals the oracle's for the whole prefix (compaction moved the right rows)
+    B = 1
+    dec = sb.SpecDecoder(cfg, parity.to_dev(tw), parity.to_dev(dw), batch=B, max_ctx=256)
+    orc = po.Oracle(cfg, tw, dw, 256)
+    assert dec.prefill([prompt], 120)[0] == orc.prefill(prompt)
+    for _ in range(6):
+        g = dec.step()[0]
+        o = orc.step()
+        if not np.array_equal(g, o):
+            orc.force_state(np.concatenate([orc.ids[: orc.n - len(o)], g]).astype(np.int32), orc.n - len(o) + len(g), len(g))
+    n = int(dec.lengths()[0])
+    assert n == orc.n
+    for pos in list(range(0, n, 7)) + [n - 1, n - 2]:
+        for layer in range(cfg.n_layers):
+            gk, gv = dec.read_kv(0, layer, pos)
+            ok, ov = orc.target_kv(layer, pos)
+            assert np.abs(gk - ok).max() < 4 * tol and np.abs(gv - ov).max() < 4 * tol, (pos, layer)
+    for pos in range(0, n - orc.pending, 5):
+        gk, gv = dec.read_kv(0, -1, pos)
+        ok, ov = orc.draft_kv(pos)
+        assert np.abs(gk - ok).max() < 4 * tol and np.abs(gv - ov).max() < 4 * tol, pos
+    dec.close()
+
+
+def test_batch_chain_with_shuffled_pages():
+    """Serving-style case (Section 4.3): several sequences of different lengths, chain drafts (top-k 1)."""
+    cfg = T1.replace(name="T1-chain", batch=5, prompt_lo=20, prompt_hi=90, tree_depth=3, tree_topk=1, tree_nodes=4, seed=3)
+    tw, dw = _weights(cfg)
+    prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+    st, _ = parity.run_trajectory(cfg, tw, dw, prompts, n_steps=8, tol=2e-2, tap_tol=3e-2, page_shuffle_seed=77)
+    print("chain", st)
+
+
+def test_page_permutation_invariance():
+    cfg = C1
+    tw, dw = _weights(cfg)
+    prompt = synth.make_prompts(cfg)[0].numpy()
+    outs = []
+    for seed in (0, 5, 9):
+        dec = sb.SpecDecoder(cfg, parity.to_dev(tw), parity.to_dev(dw), batch=1, max_ctx=256, num_pages=40,
+                             page_shuffle_seed=seed)
+        first = dec.prefill([prompt], 100)
+        toks = [int(first[0])]
+        for _ in range(8):
+            toks += dec.step()[0].tolist()
+        table = dec.debug(sb.DBG_PAGE_TABLE, 0)
+        logits = dec.debug(sb.DBG_TARGET_LOGITS, 0)
+        outs.append((toks, table, logits))
+        dec.close()
+    assert not np.array_equal(outs[0][1], outs[1][1])
+    for o in outs[1:]:
+        assert o[0] == outs[0][0]
+        assert np.array_equal(o[2], outs[0][2])          # physical placement must not change a single bit
+
+
+def test_capacity_error_leaves_state_unchanged():
+    cfg = C1
+    tw, dw = _weights(cfg)
+    prompt = synth.make_prompts(cfg)[0].numpy()
+    dec = sb.SpecDecoder(cfg, parity.to_dev(tw), parity.to_dev(dw), batch=1, max_ctx=256)
+    dec.prefill([prompt], 4)
+    n_ok = 0
+    with pytest.raises(sb.SpecError) as e:
+        for _ in range(40):
+            dec.step()
+            n_ok += 1
+    assert e.value.code == -4 and n_ok >= 1
+    n = dec.lengths()
+    with pytest.raises(sb.SpecError):
+        dec.step()
+    assert np.array_equal(dec.lengths(), n)
+    with pytest.raises(sb.SpecError) as e2:
+        sb.SpecDecoder(cfg, parity.to_dev(tw), parity.to_dev(dw), batch=1, max_ctx=256, num_pages=2).prefill([prompt], 4)
+    assert e2.value.code == -4
+    dec.close()
+
+
+def test_plain_decode_matches_oracle_greedy():
+    tw, dw = _weights(C1)
+    prompt = synth.make_prompts(C1)[0].numpy()
+    dec = sb.SpecDecoder(C1, parity.to_dev(tw), parity.to_dev(dw), batch=1, max_ctx=256)
+    first = dec.prefill([prompt], 40)
+    got = [int(dec.plain_step()[0]) for _ in range(12)]
+    o = po.Oracle(C1, tw, dw, 256)
+    assert o.prefill(prompt) == first[0]
+    ref, mg = o.greedy_margins(12)
+    for i in range(12):
+        if got[i] != ref[i]:
+            assert mg[i] < parity.MARGIN
+            break
+    with pytest.raises(sb.SpecError):
+        dec.step()                     # the draft cache is stale after plain decoding
+    dec.close()
+
+
+def test_c2_two_layer_truncation_first_steps():
+    """8B-shaped widths (hidden 4096, 32/8 heads of 128, FFN 14336, vocab 128256 / 32000, depth 6, top-k 10,
+    60 nodes) on a 2-layer truncation, first steps, bf16."""
+    cfg = synth.C2.truncated(2, prompt_len=48)
+    tw = synth.make_target_weights(cfg, device="cuda")
+    dw = synth.make_draft_weights(cfg, device="cuda")
+    prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+    st, _ = parity.run_trajectory(cfg, parity.to_cpu(tw), parity.to_cpu(dw), prompts, n_steps=2, tol=2e-2, tap_tol=3e-2)
+    print("C2-L2", st)
