@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Benchmark of one EAGLE-3 speculative step (draft + verify) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--impl ours|reference]
+
+A "step" is one full pass of the hot path (fuse pending taps, D draft passes with tree expansion,
+rerank, one tree-masked target forward, greedy acceptance, KV compaction) for every sequence of the
+batch.  Metric: accepted tokens per second (sum of per-step counts / time); ms_per_step is the
+`spec_step ms` of the same run.  The workload at N=1 is the 8B-shaped batch-1 configuration (32
+layers, hidden 4096, 32/8 heads of 128, FFN 14336, vocab 128256 / 32000, prompt 512, depth 6,
+top-k 10, 60 verified nodes) on seeded random-init weights and random prompt ids; with N>1 every rank
+runs an independent replica (the path has no collective), so the value is the sum over ranks.
+
+Prints ONE JSON line on rank 0.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2503_01840_b200 import synth  # noqa: E402
+
+METRIC = "spec_step accepted tok/s"
+UNIT = "tok/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMM kernel from the ncu capture
+# summarised in profiles/ (None until a capture exists for that workload)
+NCU_TRAFFIC_PER_LAUNCH = {}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def workload_cfg(name: str):
+    base, _, mod = name.partition(":")
+    cfg = synth.CONFIGS[base]
+    if mod.startswith("L="):
+        cfg = cfg.truncated(int(mod[2:]))
+    return cfg
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                       "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            busy = [s for s in sm if s > 0]
+            out.update(sm_mhz=statistics.median(busy), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def weight_bytes_per_step(cfg) -> float:
+    """Algorithmic weight bytes of one step: every weight once per pass (D draft passes + FC3 + L layers + LM head)."""
+    e = 4 if cfg.dtype == "fp32" else 2
+    k, qd, kvd, F = cfg.hidden, cfg.n_heads * cfg.head_dim, cfg.n_kv_heads * cfg.head_dim, cfg.ffn
+    layer = (k * qd + 2 * k * kvd + qd * k + 3 * k * F) * e
+    draft_pass = 2 * k * k * e + layer + cfg.draft_vocab * k * e
+    return cfg.tree_depth * draft_pass + 3 * k * k * e + cfg.n_layers * layer + cfg.vocab * k * e
+
+
+# ----------------------------------------------------------------------------------------------- CPU oracle legs
+def oracle_step_seconds(cfg, layers, prompt_len=64, steps=1):
+    """Median wall time of the CPU oracle's step on an `layers`-layer truncation (full widths)."""
+    sys.path.insert(0, os.path.join(ROOT, "oracle"))
+    import pyoracle as po
+    c = cfg.truncated(layers, prompt_len=prompt_len, batch=1)
+    dev = "cuda" if torch.cuda.is_available() else "cpu"      # the seeded generator runs on either device
+    tw = synth.make_target_weights(c, device=dev)
+    dw = synth.make_draft_weights(c, device=dev)
+    cpu = lambda w: {k: ([cpu(x) for x in v] if isinstance(v, list) else v.to("cpu")) for k, v in w.items()}
+    tw, dw = cpu(tw), cpu(dw)
+    o = po.Oracle(c, tw, dw, prompt_len + 64 * (steps + 2))
+    o.prefill(synth.make_prompts(c)[0].numpy())
+    ts, toks = [], 0
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        toks += len(o.step())
+        ts.append(time.perf_counter() - t0)
+    o.close()
+    return statistics.median(ts), toks / max(1, steps)
+
+
+def cpu_baseline(cfg):
+    """Oracle as it stands on the host cores, on a bounded sample: one step each on 1- and 2-layer truncations
+    at full width and a short context; a full step is extrapolated linearly in the layer count."""
+    cores = os.cpu_count() or 1      # the oracle's OpenMP loops use every host core
+    t1, tau = oracle_step_seconds(cfg, 1)
+    t2, _ = oracle_step_seconds(cfg, 2)
+    per_layer = max(t2 - t1, 1e-9)
+    full = t1 + (cfg.n_layers - 1) * per_layer
+    return {"value": cfg.batch * tau / full, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": (f"oracle spec_step timed on 1- and 2-layer truncations of {cfg.name} at full widths "
+                       f"(prompt 64, batch 1): {t1:.2f}s and {t2:.2f}s; extrapolated linearly to {cfg.n_layers} layers "
+                       f"= {full:.1f}s per step per sequence")}
+
+
+def run_reference(args, cfg):
+    """`--impl reference`: the CPU oracle (there is no other implementation of the paper here)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = os.cpu_count() or 1
+    t1, _ = oracle_step_seconds(cfg, 1)
+    per_step, tau = [], 1.0
+    sys.path.insert(0, os.path.join(ROOT, "oracle"))
+    import pyoracle as po
+    c = cfg.truncated(2, prompt_len=64, batch=1)
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    tw, dw = synth.make_target_weights(c, device=dev), synth.make_draft_weights(c, device=dev)
+    cpu = lambda w: {k: ([cpu(x) for x in v] if isinstance(v, list) else v.to("cpu")) for k, v in w.items()}
+    tw, dw = cpu(tw), cpu(dw)
+    o = po.Oracle(c, tw, dw, 64 + 64 * (args.steps + args.warmup + 2))
+    o.prefill(synth.make_prompts(c)[0].numpy())
+    toks = 0
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        n = len(o.step())
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            per_step.append(t1 + (cfg.n_layers - 1) * max(dt - t1, 1e-9))
+            toks += n
+    total = sum(per_step)
+    value = cfg.batch * toks / total
+    sample = (f"each step = one oracle spec_step on a 2-layer truncation of {cfg.name} at full widths (prompt 64, batch 1), "
+              f"scaled to {cfg.n_layers} layers with the 1-layer step time {t1:.2f}s as the layer-independent part")
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * total / max(1, len(per_step)), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "impl": "reference",
+            "config": {"workload": cfg.name, "batch": cfg.batch, "tree": f"D{cfg.tree_depth} K{cfg.tree_topk} N{cfg.tree_nodes}"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------- the CUDA arm
+def timed_steps(dec, n_steps, counts_dev):
+    """n_steps x spec_step_async between two events on the decoder's stream; returns (ms, tokens)."""
+    stream = dec.stream
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for i in range(n_steps):
+        dec.step_async(None, counts_dev[i])
+    e1.record(stream)
+    e1.synchronize()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1), int(counts_dev[:n_steps].sum().item())
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C2", help="C1..C5, optionally ':L=<layers>' for a truncation")
+    ap.add_argument("--no-extras", action="store_true", help="skip plain-decode / structured-acceptance / CPU legs")
+    ap.add_argument("--flags", type=int, default=0)
+    args = ap.parse_args()
+    cfg = workload_cfg(args.workload)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the speculative step has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2503_01840_b200 import binding as sb
+
+    B, D = cfg.batch, cfg.tree_depth
+    prof_steps = 3
+    total_steps = args.warmup + args.steps + prof_steps + 40
+    reserve = total_steps * (D + 1) + 64
+    prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+    max_ctx = max(len(p) for p in prompts) + reserve + 192
+    t0 = time.time()
+    tw = synth.make_target_weights(cfg, device=dev)
+    dw = synth.make_draft_weights(cfg, device=dev)
+    torch.cuda.synchronize()
+    t_gen = time.time() - t0
+    dec = sb.SpecDecoder(cfg, tw, dw, batch=B, max_ctx=max_ctx, flags=args.flags, page_shuffle_seed=cfg.seed)
+    t0 = time.time()
+    dec.prefill(prompts, reserve)
+    t_prefill = time.time() - t0
+
+    counts = torch.zeros(max(args.steps, args.warmup), B, dtype=torch.int32, device=dev)
+    timed_steps(dec, args.warmup, counts)
+    n_mid = dec.lengths().astype(np.float64)
+    bytes_step = dec.step_bytes()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms, toks = timed_steps(dec, args.steps, counts)
+    clocks = sampler.stop() if sampler else None
+    launches = dec.launches_per_step()
+    if world > 1:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        k = torch.tensor([toks], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(k, op=dist.ReduceOp.SUM)
+        ms, toks = float(t.item()), int(k.item())
+    ms_per_step = ms / args.steps
+    value = toks / (ms * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (sync + device->host copy every step)
+    e2e_steps = min(args.steps, 50)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    e2e_toks = 0
+    for _ in range(e2e_steps):
+        e2e_toks += sum(len(o) for o in dec.step())
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    e2e_val = e2e_toks / e2e_s
+    if world > 1:
+        v = torch.tensor([e2e_val], device=dev, dtype=torch.float64)
+        dist.all_reduce(v, op=dist.ReduceOp.SUM)
+        e2e_val = float(v.item())
+    d2h = B * (D + 1) * 4 + B * 4 + 16 + B * 4
+
+    # ---- dominant kernel (the tcgen05 GEMM) timed with an event before every launch
+    peak, peak_kind = peaks()
+    gemm_ms = gemm_n = 0.0
+    breakdown = {}
+    for _ in range(prof_steps):
+        pr = dec.profile_step()
+        for c, (m_, n_) in pr.items():
+            a = breakdown.setdefault(c, [0.0, 0])
+            a[0] += m_ / prof_steps
+            a[1] = n_
+    gemm_ms, gemm_n = breakdown["gemm"]
+    wbytes = weight_bytes_per_step(cfg)
+    achieved = wbytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
+    traffic = NCU_TRAFFIC_PER_LAUNCH.get(cfg.name)
+    roofline = {"bound": "hbm", "kernel": "gemm_tcgen05_kernel (all weight GEMMs of the step)", "achieved": achieved,
+                "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                "bytes_per_launch": wbytes / max(1, gemm_n), "avg_launch_us": 1e3 * gemm_ms / max(1, gemm_n),
+                "launches_per_step": gemm_n, "traffic": traffic,
+                "step": {"algorithmic_bytes": bytes_step, "achieved": bytes_step / (ms_per_step * 1e-3) / 1e9,
+                         "frac_of_measured_copy": bytes_step / (ms_per_step * 1e-3) / 1e9 / peak,
+                         "frac_of_8TBs": bytes_step / (ms_per_step * 1e-3) / 1e9 / 8000.0},
+                "class_ms_per_step": {c: round(v[0], 4) for c, v in breakdown.items()}}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": cfg.name, "batch": B, "context_mid_run": float(n_mid.mean()),
+                       "tree": f"D{D} K{cfg.tree_topk} N{cfg.tree_nodes}", "page_size": cfg.page_size,
+                       "parallelism": "replicas" if world > 1 else "single GPU",
+                       "l2": "inputs (weights + KV) far larger than L2, no flush", "tau": toks / (args.steps * B * world)},
+            "clocks": clocks, "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": d2h,
+                                      "note": "spec_step with host outputs, synchronised every step; a step has no host input"},
+            "gpu_launches": launches * args.steps, "roofline": roofline,
+            "setup_s": {"weights": round(t_gen, 2), "prefill": round(t_prefill, 2)}}
+
+    if rank == 0 and world == 1 and not args.no_extras:
+        extras = {}
+        # plain greedy decoding on the same kernels (the paper's vanilla baseline), synchronised per token
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(20):
+            dec.plain_step()
+        torch.cuda.synchronize()
+        extras["plain_decode_tok_s"] = 20 * B / (time.perf_counter() - t0)
+        dec.close()
+        del dec
+        if cfg.batch == 1 and cfg.tree_depth >= 2:
+            # designed draft/target agreement: same shapes and bytes, acceptance length near the paper's
+            tw2, dw2, _, _ = synth.make_structured(cfg, 0.96, device=dev)
+            pr = synth.structured_prompt(cfg, dw2["d2t"].cpu(), len(prompts[0])).numpy()
+            dec2 = sb.SpecDecoder(cfg, tw2, dw2, batch=1, max_ctx=len(pr) + 60 * (D + 1) + 256, page_shuffle_seed=cfg.seed)
+            dec2.prefill([pr], 60 * (D + 1))
+            c2 = torch.zeros(40, 1, dtype=torch.int32, device=dev)
+            timed_steps(dec2, 5, c2)
+            ms2, tk2 = timed_steps(dec2, 40, c2)
+            extras["structured_agreement"] = {"p_agree": 0.96, "tau": tk2 / 40, "ms_per_step": ms2 / 40,
+                                              "accepted_tok_s": tk2 / (ms2 * 1e-3)}
+            dec2.close()
+            del dec2, tw2, dw2
+        extras["projection_at_paper_tau"] = {"tau": 6.23, "tok_s": 6.23 * B / (ms_per_step * 1e-3),
+                                            "note": "paper's mean acceptance length for the 8B target (Table 1) / measured step time"}
+        line["extras"] = extras
+        del tw, dw
+        torch.cuda.empty_cache()
+        line["cpu_baseline"] = cpu_baseline(cfg)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

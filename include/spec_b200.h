@@ -125,6 +125,15 @@ int spec_plain_step(spec_ctx *ctx, int32_t *out_ids);
 /* Committed length of every sequence (host [batch]); synchronises. */
 int spec_lengths(spec_ctx *ctx, int32_t *lens);
 
+/* One speculative step launched kernel by kernel with a CUDA event in front of every launch; reports,
+ * per kernel class, the summed time to the next launch (ms) and the number of launches.  Arrays of
+ * SPEC_PROF_CLASSES entries.  State advances exactly as in spec_step; synchronises.  Timing aid only. */
+enum spec_prof_class {
+  SPEC_PROF_GEMM = 0, SPEC_PROF_ATTN, SPEC_PROF_NORM, SPEC_PROF_ROPE_KV, SPEC_PROF_ACT, SPEC_PROF_MISC,
+  SPEC_PROF_TOPK, SPEC_PROF_TREE, SPEC_PROF_ARGMAX, SPEC_PROF_COMMIT, SPEC_PROF_CLASSES
+};
+int spec_profile_step(spec_ctx *ctx, float *class_ms, int32_t *class_launches);
+
 /* Number of kernels one spec_step launches (for launch accounting). */
 int spec_launches_per_step(const spec_ctx *ctx);
 

@@ -55,7 +55,7 @@ class _Cfg(C.Structure):
 
 
 EXPORTS = ("spec_workspace_bytes", "spec_init", "spec_prefill", "spec_step", "spec_step_async", "spec_plain_step",
-           "spec_lengths", "spec_launches_per_step", "spec_step_bytes", "spec_free", "spec_last_error",
+           "spec_lengths", "spec_profile_step", "spec_launches_per_step", "spec_step_bytes", "spec_free", "spec_last_error",
            "spec_debug_read", "spec_debug_read_kv", "spec_gemm_scratch_bytes", "spec_gemm", "spec_attn_scratch_bytes",
            "spec_attention", "spec_logsoftmax_topk", "spec_argmax")
 
@@ -81,6 +81,7 @@ def lib():
     L.spec_plain_step.argtypes = [vp, vp]
     L.spec_lengths.argtypes = [vp, vp]
     L.spec_launches_per_step.argtypes = [vp]
+    L.spec_profile_step.argtypes = [vp, vp, vp]
     L.spec_step_bytes.argtypes = [vp, C.POINTER(C.c_double)]
     L.spec_free.argtypes = [vp]
     L.spec_last_error.argtypes = [vp]
@@ -234,6 +235,15 @@ class SpecDecoder:
         out = np.zeros(self.batch, np.int32)
         self._check(lib().spec_lengths(self.h, out.ctypes.data))
         return out
+
+    PROF_CLASSES = ("gemm", "attention", "add_norm", "rope_kv", "silu_mul", "misc", "topk", "tree", "argmax", "commit")
+
+    def profile_step(self):
+        """One step with an event before every launch: {class: (ms, launches)}."""
+        ms = np.zeros(len(self.PROF_CLASSES), np.float32)
+        n = np.zeros(len(self.PROF_CLASSES), np.int32)
+        self._check(lib().spec_profile_step(self.h, ms.ctypes.data, n.ctypes.data))
+        return {c: (float(ms[i]), int(n[i])) for i, c in enumerate(self.PROF_CLASSES)}
 
     def launches_per_step(self) -> int:
         return lib().spec_launches_per_step(self.h)

@@ -91,6 +91,11 @@ struct spec_ctx {
   cudaGraphExec_t graph = nullptr;
   int launches = 0, launches_graph = 0;
   int sched_err = 0;
+  int cur_rps = 1;             // rows per sequence of the pass being scheduled
+  bool prof = false;
+  std::vector<cudaEvent_t> prof_ev;
+  std::vector<int> prof_cls;
+  int prof_n = 0;
   FastGemm *fg = nullptr;
   char err[256];
 };
@@ -276,6 +281,7 @@ extern "C" int spec_free(spec_ctx *c) {
   if (!c) return SPEC_OK;
   if (c->graph) cudaGraphExecDestroy(c->graph);
   if (c->fg) fast_gemm_destroy(c->fg);
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   delete c;
   return SPEC_OK;
 }
@@ -286,6 +292,19 @@ template <typename T> struct Sched {
   cudaStream_t s;
   explicit Sched(spec_ctx *ctx) : c(ctx), s(ctx->stream) {}
   void tick(int n = 1) { c->launches += n; }
+  // profiling: one event at the start of every launch; the interval to the next event is charged to `cls`
+  void mark(int cls) {
+    if (!c->prof) return;
+    if (c->prof_n >= (int)c->prof_ev.size()) {
+      cudaEvent_t e;
+      cudaEventCreate(&e);
+      c->prof_ev.push_back(e);
+      c->prof_cls.push_back(0);
+    }
+    cudaEventRecord(c->prof_ev[c->prof_n], s);
+    c->prof_cls[c->prof_n] = cls;
+    c->prof_n++;
+  }
 
   // number of split-K slices for a weight of shape [O][I] whose output buffer holds smax slices
   int pick(int O, int I, int smax) const { return c->fg ? fast_gemm_pick_split(O, I, smax) : 1; }
@@ -293,6 +312,7 @@ template <typename T> struct Sched {
 
   // S fp32 partial slices of x . w^T into columns [col0, col0+O) of `out` (row pitch ldo)
   void gemm(const void *x, const void *w, float *out, int rows, int O, int I, int ldo, int col0, int S) {
+    mark(SPEC_PROF_GEMM);
     if (c->fg) {
       int rc = fast_gemm_run(c->fg, (const bf16 *)x, (const bf16 *)w, out + col0, rows, O, I, ldo, pstride(ldo), S, c->status, s);
       if (rc && !c->sched_err) c->sched_err = rc;
@@ -303,11 +323,14 @@ template <typename T> struct Sched {
   }
 
   void attention(KvPool pool, int rows, int tail_len) {
+    mark(SPEC_PROF_ATTN);
     PageMap pm{c->page_table, c->pps, c->cfg.page_size, c->cfg.num_pages};
     bool fast = c->cfg.dtype == SPEC_BF16 && !(c->cfg.flags & SPEC_FLAG_REF_ATTN) && attn_fast_supported(c->hd, c->H / c->G);
     if (fast) {
+      int hint = 0;
+      for (int b = 0; b < c->B; b++) hint = std::max(hint, c->n_upper[b]);
       tick(launch_attn_fast((const bf16 *)c->q, pool, pm, c->meta, tail_len, (bf16 *)c->ao, rows, c->H, c->G, c->hd,
-                            c->cfg.max_ctx, c->attn_scratch, s));
+                            c->cur_rps, hint, c->attn_scratch, s));
     } else {
       launch_attn_ref<T>((const T *)c->q, pool, pm, c->meta, tail_len, (T *)c->ao, rows, c->H, c->G, c->hd,
                          c->cfg.max_ctx + tail_len, s);
@@ -320,25 +343,25 @@ template <typename T> struct Sched {
   void block(const LayerW &w, KvPool pool, int rows, int tail_len, int first_mode, int tap_mask) {
     int k = c->k, qd = c->H * c->hd, kvd = c->G * c->hd, qkvd = qd + 2 * kvd, F = c->F;
     PageMap pm{c->page_table, c->pps, c->cfg.page_size, c->cfg.num_pages};
-    launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, first_mode, (T *)c->node_taps, tap_mask, (const T *)w.attn_norm,
+    mark(SPEC_PROF_NORM); launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, first_mode, (T *)c->node_taps, tap_mask, (const T *)w.attn_norm,
                        c->cfg.rms_eps, (T *)c->h, nullptr, rows, rows, k, s);
     tick();
     c->np_qkv = pick(qd, k, c->smax_qkv); c->ps_qkv = pstride(qkvd);
     gemm(c->h, w.wq, c->qkv, rows, qd, k, qkvd, 0, c->np_qkv);
     gemm(c->h, w.wk, c->qkv, rows, kvd, k, qkvd, qd, c->np_qkv);
     gemm(c->h, w.wv, c->qkv, rows, kvd, k, qkvd, qd + kvd, c->np_qkv);
-    launch_rope_kv<T>(c->qkv, c->np_qkv, c->ps_qkv, c->cs, c->meta, (T *)c->q, pool, pm, rows, c->H, c->G, c->hd, c->status, s);
+    mark(SPEC_PROF_ROPE_KV); launch_rope_kv<T>(c->qkv, c->np_qkv, c->ps_qkv, c->cs, c->meta, (T *)c->q, pool, pm, rows, c->H, c->G, c->hd, c->status, s);
     tick();
     attention(pool, rows, tail_len);
     c->np_proj = pick(k, qd, c->smax_proj); c->ps_proj = pstride(k);
     gemm(c->ao, w.wo, c->proj, rows, k, qd, k, 0, c->np_proj);
-    launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, 2, (T *)nullptr, 0, (const T *)w.mlp_norm, c->cfg.rms_eps,
+    mark(SPEC_PROF_NORM); launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, 2, (T *)nullptr, 0, (const T *)w.mlp_norm, c->cfg.rms_eps,
                        (T *)c->h, nullptr, rows, rows, k, s);
     tick();
     c->np_gu = pick(F, k, c->smax_gu); c->ps_gu = pstride(2 * F);
     gemm(c->h, w.w_gate, c->gu, rows, F, k, 2 * F, 0, c->np_gu);
     gemm(c->h, w.w_up, c->gu, rows, F, k, 2 * F, F, c->np_gu);
-    launch_silu_mul<T>(c->gu, c->np_gu, c->ps_gu, (T *)c->act, rows, F, s);
+    mark(SPEC_PROF_ACT); launch_silu_mul<T>(c->gu, c->np_gu, c->ps_gu, (T *)c->act, rows, F, s);
     tick();
     c->np_proj = pick(k, F, c->smax_proj); c->ps_proj = pstride(k);
     gemm(c->act, w.w_down, c->proj, rows, k, F, k, 0, c->np_proj);
@@ -352,16 +375,16 @@ template <typename T> struct Sched {
 
   // target forward over the rows of c->meta: taps -> node_taps, argmax -> tb.y
   void target_forward(int rows, int tail_len, bool want_logits) {
-    launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
-    launch_embed<T>((const T *)c->embed, c->meta.tok, c->x, rows, c->k, s); tick();
+    mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
+    mark(SPEC_PROF_MISC); launch_embed<T>((const T *)c->embed, c->meta.tok, c->x, rows, c->k, s); tick();
     for (int l = 0; l < c->L; l++)
       block(c->tl[l], c->pools[l], rows, tail_len, l == 0 ? 0 : 2, l == 0 ? 0 : tap_mask_of(l - 1));
-    launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, 2, (T *)c->node_taps, tap_mask_of(c->L - 1),
+    mark(SPEC_PROF_NORM); launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, 2, (T *)c->node_taps, tap_mask_of(c->L - 1),
                        (const T *)c->final_norm, c->cfg.rms_eps, (T *)c->h, nullptr, rows, rows, c->k, s);
     tick();
     if (want_logits) {
       gemm(c->h, c->lm_head, c->logits, rows, c->V, c->k, c->V, 0, 1);
-      launch_argmax(c->logits, rows, c->V, c->tb.y, s); tick();
+      mark(SPEC_PROF_ARGMAX); launch_argmax(c->logits, rows, c->V, c->tb.y, s); tick();
     }
   }
 
@@ -373,13 +396,13 @@ template <typename T> struct Sched {
 
   // draft head on the rows of c->meta: cat = [feat ; e(tok)], FC2, decoder block, final norm (-> h)
   void draft_forward(const float *feat, int nparts, size_t fstride, const int32_t *src_row, int rows, int tail_len) {
-    launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
-    launch_build_cat<T>(feat, nparts, fstride, src_row, (const T *)c->embed, c->meta.tok, c->meta.seq, (T *)c->cat, rows, c->k, s);
+    mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
+    mark(SPEC_PROF_MISC); launch_build_cat<T>(feat, nparts, fstride, src_row, (const T *)c->embed, c->meta.tok, c->meta.seq, (T *)c->cat, rows, c->k, s);
     tick();
     c->np_proj = pick(c->k, 2 * c->k, c->smax_proj); c->ps_proj = pstride(c->k);
     gemm(c->cat, c->fc2, c->proj, rows, c->k, 2 * c->k, c->k, 0, c->np_proj);
     block(c->dl, c->pools[c->L], rows, tail_len, 1, 0);
-    launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, 2, (T *)nullptr, 0, (const T *)c->dfinal_norm, c->cfg.rms_eps,
+    mark(SPEC_PROF_NORM); launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, 2, (T *)nullptr, 0, (const T *)c->dfinal_norm, c->cfg.rms_eps,
                        (T *)c->h, nullptr, rows, rows, c->k, s);
     tick();
   }
@@ -392,6 +415,7 @@ template <typename T> struct Sched {
     if (!c->cap_logits) return;
     // pass 1: only the last pending row of each sequence matters; it lands in slot [0][b*K]
     size_t lo = (size_t)(pass - 1) * c->Td;
+    mark(SPEC_PROF_MISC);
     if (first) {
       launch_gather_rows(c->logits, c->st.last_row, c->cap_logits + lo * c->Vd, c->B, c->Vd, c->K, s);
       launch_gather_rows(c->x, c->st.last_row, c->cap_a + lo * c->k, c->B, c->k, c->K, s);
@@ -405,30 +429,34 @@ template <typename T> struct Sched {
   void step(bool plain) {
     int rows = plain ? c->B : c->Tv, rps = plain ? 1 : c->N;
     if (!plain) {
-      launch_prep_extend(c->st, c->tb, c->meta, c->B, c->need_pos, c->status, s); tick();
+      mark(SPEC_PROF_TREE); launch_prep_extend(c->st, c->tb, c->meta, c->B, c->need_pos, c->status, s); tick();
+      c->cur_rps = c->Pmax;
       fuse(c->pend_taps, c->Te);
       draft_forward(c->proj, c->np_proj, c->ps_proj, nullptr, c->Te, c->Pmax);
       draft_logits(c->Te);
-      launch_logsoftmax_topk_rows(c->logits, c->st.last_row, c->B, c->Vd, c->K, c->tb.tk_idx, c->tb.tk_lp, s); tick();
+      mark(SPEC_PROF_TOPK); launch_logsoftmax_topk_rows(c->logits, c->st.last_row, c->B, c->Vd, c->K, c->tb.tk_idx, c->tb.tk_lp, s); tick();
       capture(1, c->Te, true);
-      launch_expand(c->st, c->tb, c->meta, c->d2t, 1, c->B, s); tick();
+      mark(SPEC_PROF_TREE); launch_expand(c->st, c->tb, c->meta, c->d2t, 1, c->B, s); tick();
       for (int p = 2; p <= c->D; p++) {
+        c->cur_rps = c->K;
         draft_forward(c->x, 1, 0, c->tb.feat_row, c->Td, c->tail_tree);
         draft_logits(c->Td);
-        launch_logsoftmax_topk_rows(c->logits, nullptr, c->Td, c->Vd, c->K, c->tb.tk_idx, c->tb.tk_lp, s); tick();
+        mark(SPEC_PROF_TOPK); launch_logsoftmax_topk_rows(c->logits, nullptr, c->Td, c->Vd, c->K, c->tb.tk_idx, c->tb.tk_lp, s); tick();
         capture(p, c->Td, false);
-        launch_expand(c->st, c->tb, c->meta, c->d2t, p, c->B, s); tick();
+        mark(SPEC_PROF_TREE); launch_expand(c->st, c->tb, c->meta, c->d2t, p, c->B, s); tick();
       }
-      launch_rerank(c->st, c->tb, c->meta, c->B, s); tick();
+      mark(SPEC_PROF_TREE); launch_rerank(c->st, c->tb, c->meta, c->B, s); tick();
     } else {
-      launch_plain_tree(c->st, c->tb, c->meta, c->B, s); tick();
+      mark(SPEC_PROF_TREE); launch_plain_tree(c->st, c->tb, c->meta, c->B, s); tick();
     }
+    c->cur_rps = rps;
     target_forward(rows, rps, true);
-    launch_accept(c->st, c->tb, c->B, rps, s); tick();
+    mark(SPEC_PROF_TREE); launch_accept(c->st, c->tb, c->B, rps, s); tick();
     PageMap pm{c->page_table, c->pps, c->cfg.page_size, c->cfg.num_pages};
-    launch_commit<T>(c->st, c->tb, c->pools_dev, pm, (const T *)c->node_taps, (T *)c->pend_taps, c->B, c->L, c->G, c->hd,
+    mark(SPEC_PROF_COMMIT); launch_commit<T>(c->st, c->tb, c->pools_dev, pm, (const T *)c->node_taps, (T *)c->pend_taps, c->B, c->L, c->G, c->hd,
                      c->k, rps, s);
     tick();
+    mark(-1);
   }
 };
 
@@ -512,6 +540,7 @@ template <typename T> static int do_prefill(spec_ctx *c, const int32_t *ids, con
       int nv = std::min(CH, n - start);
       bool last = start + nv == n;
       CUDA_TRY(c, upload_meta(nv, b, start, p + start));
+      c->cur_rps = CH;
       sc.target_forward(CH, CH, last);
       if (last) {
         // the last position stays pending: its taps become pending entry 0
@@ -636,6 +665,28 @@ extern "C" int spec_lengths(spec_ctx *c, int32_t *lens) {
   if (int rc = sync_lengths(c)) return rc;
   for (int b = 0; b < c->B; b++) lens[b] = c->n_upper[b];
   return SPEC_OK;
+}
+
+extern "C" int spec_profile_step(spec_ctx *c, float *class_ms, int32_t *class_launches) {
+  if (!c || !class_ms || !class_launches) return SPEC_ERR_NULL;
+  if (c->draft_stale) return fail(c, SPEC_ERR_STATE, "spec_profile_step after spec_plain_step");
+  if (int rc = check_capacity(c, c->Pmax, "spec_profile_step")) return rc;
+  for (int i = 0; i < SPEC_PROF_CLASSES; i++) { class_ms[i] = 0.0f; class_launches[i] = 0; }
+  c->prof = true;
+  c->prof_n = 0;
+  c->launches = 0;
+  if (c->cfg.dtype == SPEC_F32) Sched<float>(c).step(false); else Sched<bf16>(c).step(false);
+  c->prof = false;
+  for (int b = 0; b < c->B; b++) c->n_upper[b] += c->Pmax;
+  CUDA_TRY(c, cudaGetLastError());
+  if (int rc = read_status(c)) return rc;
+  for (int i = 0; i + 1 < c->prof_n; i++) {
+    float ms = 0.0f;
+    CUDA_TRY(c, cudaEventElapsedTime(&ms, c->prof_ev[i], c->prof_ev[i + 1]));
+    int cls = c->prof_cls[i];
+    if (cls >= 0 && cls < SPEC_PROF_CLASSES) { class_ms[cls] += ms; class_launches[cls] += 1; }
+  }
+  return sync_lengths(c);
 }
 
 extern "C" int spec_launches_per_step(const spec_ctx *c) { return c ? c->launches : 0; }
@@ -783,7 +834,7 @@ extern "C" int spec_attention(int32_t dtype, int32_t impl, const void *q, const 
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
   }
   if (dtype != SPEC_BF16 || !attn_fast_supported(hd, H / G)) return SPEC_ERR_UNSUPPORTED;
-  launch_attn_fast((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, max_ctx, scratch, s);
+  launch_attn_fast((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, 1, max_ctx, scratch, s);
   return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }
 

@@ -1,13 +1,299 @@
-// Tensor-core tree-masked paged GQA attention (bf16).
+// Tree-masked paged GQA attention on tensor cores (Section 2.2 "tree attention"), bf16.
+//
+// One CTA owns up to 128 query rows of one (sequence, KV head): the rows are (tree node, query head of
+// the GQA group) pairs, so every K/V tile fetched from the paged cache is shared by all nodes and all
+// heads of the group.  Keys are split across CTAs (flash-decoding style); each CTA streams 64-key
+// tiles through a two-stage cp.async pipeline, computes S = Q K^T and O += P V with mma.sync
+// m16n8k16, keeps the softmax statistics in registers (quad shuffles), applies the bit-packed
+// ancestor mask to the tail keys, and writes either the final output (one split) or an unnormalised
+// partial (several splits) that a small combine kernel merges.
 #include "attn_fast.cuh"
 
 namespace spec {
 
-bool attn_fast_supported(int head_dim, int group) { (void)head_dim; (void)group; return false; }
-size_t attn_fast_scratch_bytes(int rows, int n_heads, int head_dim, int max_ctx) { return 0; }
+namespace {
+
+constexpr int KT = 64;          // keys per tile
+constexpr int MT = 128;         // query rows per CTA (8 warps x 16)
+constexpr int MAX_SPLITS = 32;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid) {
+  int sz = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *(uint32_t *)&v;
+}
+// byte offset of 16-byte chunk `c` of row `row` in a tile with ROWB bytes per row, XOR-swizzled
+template <int ROWB> __device__ __forceinline__ uint32_t swz(int row, int c) { return (uint32_t)(row * ROWB + ((c ^ (row & 7)) << 4)); }
+
+struct AttnParams {
+  const bf16 *q;
+  const bf16 *kpool, *vpool;
+  PageMap pm;
+  RowMeta m;
+  int tail_len, rows, H, G, rps, nsplit;
+  bf16 *out;
+  float *part_o;    // [nsplit][rows*H][hd]
+  float *part_ml;   // [nsplit][rows*H][2]
+};
+
+template <int HD>
+__global__ void __launch_bounds__(256) attn_mma_kernel(AttnParams p) {
+  constexpr int ROWB = HD * 2, CPR = HD / 8;          // bytes / 16-byte chunks per row
+  constexpr int NKS = HD / 16;                        // k-steps of Q K^T
+  extern __shared__ __align__(128) unsigned char sm[];
+  unsigned char *sK[2] = {sm, sm + 2 * KT * ROWB};
+  unsigned char *sV[2] = {sm + KT * ROWB, sm + 3 * KT * ROWB};
+  unsigned char *sQ = sm;                              // the Q tile borrows the stage memory before the main loop
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int grp = p.H / p.G;
+  const int b = blockIdx.z / p.G, g = blockIdx.z % p.G;
+  const int M = p.rps * grp;                           // query rows of this (sequence, KV head)
+  const int m0 = blockIdx.x * MT;
+  const int row0 = b * p.rps;
+  // sequence-level quantities from the first row of the sequence (all rows of a sequence share them)
+  int seq = -1, ctx = 0, tb = 0;
+  for (int i = 0; i < p.rps; i++) {
+    int s = p.m.seq[row0 + i];
+    if (s >= 0) { seq = s; ctx = p.m.ctx[row0 + i]; tb = p.m.tail_base[row0 + i]; break; }
+  }
+  const int nkeys = (seq >= 0) ? ctx + p.tail_len : 0;
+  const int ntiles = (nkeys + KT - 1) / KT;
+  const int t_begin = (int)(((long long)blockIdx.y * ntiles) / p.nsplit);
+  const int t_end = (int)(((long long)(blockIdx.y + 1) * ntiles) / p.nsplit);
+
+  // ---- Q tile -> shared (swizzled) -> A fragments
+  for (int id = threadIdx.x; id < MT * CPR; id += 256) {
+    int lr = id / CPR, c = id % CPR, mrow = m0 + lr;
+    bool v = mrow < M;
+    int i = v ? mrow / grp : 0, hq = v ? mrow % grp : 0;
+    v = v && p.m.seq[row0 + i] >= 0;
+    const bf16 *src = p.q + ((size_t)(row0 + i) * p.H + g * grp + hq) * HD + c * 8;
+    cp_async16(smem_u32(sQ + swz<ROWB>(lr, c)), src, v);
+  }
+  cp_async_commit();
+  cp_async_wait<0>();
+  __syncthreads();
+  uint32_t qf[NKS][4];
+#pragma unroll
+  for (int ks = 0; ks < NKS; ks++) {
+    int r = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = ks * 2 + (lane >> 4);
+    ldsm_x4(smem_u32(sQ + swz<ROWB>(r, c)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+  }
+  __syncthreads();
+
+  // rows owned by this thread: rA = quad row, rB = rA + 8 (within the warp's 16 rows)
+  const int mA = m0 + warp * 16 + (lane >> 2), mB = mA + 8;
+  uint64_t loA = 0, hiA = 0, loB = 0, hiB = 0;
+  bool vA = false, vB = false;
+  if (mA < M) { int r = row0 + mA / grp; vA = p.m.seq[r] >= 0; if (vA) { loA = p.m.mask_lo[r]; hiA = p.m.mask_hi[r]; } }
+  if (mB < M) { int r = row0 + mB / grp; vB = p.m.seq[r] >= 0; if (vB) { loB = p.m.mask_lo[r]; hiB = p.m.mask_hi[r]; } }
+
+  float o[HD / 8][4];
+#pragma unroll
+  for (int n = 0; n < HD / 8; n++) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.0f; }
+  float mxA = -INFINITY, mxB = -INFINITY, lA = 0.0f, lB = 0.0f;
+  const float sc = rsqrtf((float)HD) * 1.4426950408889634f;    // softmax scale folded into exp2
+
+  auto load_tile = [&](int t, int st) {
+    int k0 = t * KT;
+    for (int id = threadIdx.x; id < KT * CPR; id += 256) {
+      int kr = id / CPR, c = id % CPR, key = k0 + kr;
+      bool v = key < nkeys;
+      int pos = key < ctx ? key : tb + (key - ctx);
+      size_t off = 0;
+      if (v) {
+        int pidx = pos / p.pm.page_size;
+        v = pidx < p.pm.pages_per_seq;
+        if (v) {
+          int page = p.pm.table[(size_t)seq * p.pm.pages_per_seq + pidx];
+          v = page >= 0 && page < p.pm.num_pages;
+          off = (((size_t)page * p.G + g) * p.pm.page_size + (pos % p.pm.page_size)) * HD + c * 8;
+        }
+      }
+      if (!v) off = 0;
+      cp_async16(smem_u32(sK[st] + swz<ROWB>(kr, c)), p.kpool + off, v);
+      cp_async16(smem_u32(sV[st] + swz<ROWB>(kr, c)), p.vpool + off, v);
+    }
+    cp_async_commit();
+  };
+
+  if (t_begin < t_end) load_tile(t_begin, 0);
+  for (int t = t_begin; t < t_end; t++) {
+    int st = (t - t_begin) & 1;
+    if (t + 1 < t_end) { load_tile(t + 1, st ^ 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
+    __syncthreads();
+    // ---- S = Q K^T for 64 keys: 8 n-tiles of 8 keys
+    float s[KT / 8][4];
+#pragma unroll
+    for (int n = 0; n < KT / 8; n++) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.0f; }
+#pragma unroll
+    for (int ks = 0; ks < NKS; ks++) {
+#pragma unroll
+      for (int n2 = 0; n2 < KT / 16; n2++) {
+        uint32_t b0, b1, b2, b3;
+        int kr = n2 * 16 + (lane & 7) + (lane >> 4) * 8, c = ks * 2 + ((lane >> 3) & 1);
+        ldsm_x4(smem_u32(sK[st] + swz<ROWB>(kr, c)), b0, b1, b2, b3);
+        mma_bf16(s[2 * n2], qf[ks], b0, b1);
+        mma_bf16(s[2 * n2 + 1], qf[ks], b2, b3);
+      }
+    }
+    // ---- mask + online softmax (two rows per thread, reductions across the quad)
+    float tmA = -INFINITY, tmB = -INFINITY;
+#pragma unroll
+    for (int n = 0; n < KT / 8; n++) {
+#pragma unroll
+      for (int e = 0; e < 2; e++) {
+        int key = t * KT + n * 8 + (lane & 3) * 2 + e;
+        bool in_ctx = key < ctx;
+        int tt = key - ctx;
+        bool in_tail = !in_ctx && tt < p.tail_len;
+        bool okA = vA && (in_ctx || (in_tail && ((tt < 64 ? (loA >> tt) : (hiA >> (tt - 64))) & 1ull)));
+        bool okB = vB && (in_ctx || (in_tail && ((tt < 64 ? (loB >> tt) : (hiB >> (tt - 64))) & 1ull)));
+        s[n][e] = okA ? s[n][e] : -INFINITY;
+        s[n][2 + e] = okB ? s[n][2 + e] : -INFINITY;
+        tmA = fmaxf(tmA, s[n][e]);
+        tmB = fmaxf(tmB, s[n][2 + e]);
+      }
+    }
+    tmA = fmaxf(tmA, __shfl_xor_sync(0xffffffffu, tmA, 1)); tmA = fmaxf(tmA, __shfl_xor_sync(0xffffffffu, tmA, 2));
+    tmB = fmaxf(tmB, __shfl_xor_sync(0xffffffffu, tmB, 1)); tmB = fmaxf(tmB, __shfl_xor_sync(0xffffffffu, tmB, 2));
+    float nmA = fmaxf(mxA, tmA), nmB = fmaxf(mxB, tmB);
+    float fA = (nmA == -INFINITY) ? 1.0f : exp2f((mxA - nmA) * sc), fB = (nmB == -INFINITY) ? 1.0f : exp2f((mxB - nmB) * sc);
+    float baseA = (nmA == -INFINITY) ? 0.0f : nmA, baseB = (nmB == -INFINITY) ? 0.0f : nmB;
+    float rsA = 0.0f, rsB = 0.0f;
+    uint32_t pf[KT / 16][4];
+#pragma unroll
+    for (int n = 0; n < KT / 8; n++) {
+      float p0 = exp2f((s[n][0] - baseA) * sc), p1 = exp2f((s[n][1] - baseA) * sc);
+      float p2 = exp2f((s[n][2] - baseB) * sc), p3 = exp2f((s[n][3] - baseB) * sc);
+      rsA += p0 + p1; rsB += p2 + p3;
+      pf[n >> 1][(n & 1) * 2] = pack_bf16(p0, p1);
+      pf[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
+    }
+    rsA += __shfl_xor_sync(0xffffffffu, rsA, 1); rsA += __shfl_xor_sync(0xffffffffu, rsA, 2);
+    rsB += __shfl_xor_sync(0xffffffffu, rsB, 1); rsB += __shfl_xor_sync(0xffffffffu, rsB, 2);
+    lA = lA * fA + rsA; lB = lB * fB + rsB;
+    mxA = nmA; mxB = nmB;
+#pragma unroll
+    for (int n = 0; n < HD / 8; n++) { o[n][0] *= fA; o[n][1] *= fA; o[n][2] *= fB; o[n][3] *= fB; }
+    // ---- O += P V
+#pragma unroll
+    for (int kk = 0; kk < KT / 16; kk++) {
+#pragma unroll
+      for (int d2 = 0; d2 < HD / 16; d2++) {
+        uint32_t b0, b1, b2, b3;
+        int kr = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = d2 * 2 + (lane >> 4);
+        ldsm_x4_t(smem_u32(sV[st] + swz<ROWB>(kr, c)), b0, b1, b2, b3);
+        mma_bf16(o[2 * d2], pf[kk], b0, b1);
+        mma_bf16(o[2 * d2 + 1], pf[kk], b2, b3);
+      }
+    }
+    __syncthreads();      // all warps done with this stage before it is refilled
+  }
+
+  // ---- write: final (one split) or partial
+  const int qcol = (lane & 3) * 2;
+#pragma unroll
+  for (int half = 0; half < 2; half++) {
+    int mrow = half ? mB : mA;
+    if (mrow >= M) continue;
+    int r = row0 + mrow / grp, h = g * grp + mrow % grp;
+    float l = half ? lB : lA, mx = half ? mxB : mxA;
+    if (p.nsplit == 1) {
+      float inv = l > 0.0f ? 1.0f / l : 0.0f;
+      bf16 *dst = p.out + ((size_t)r * p.H + h) * HD;
+#pragma unroll
+      for (int n = 0; n < HD / 8; n++)
+        *(uint32_t *)(dst + n * 8 + qcol) = pack_bf16(o[n][half * 2] * inv, o[n][half * 2 + 1] * inv);
+    } else {
+      size_t idx = (size_t)blockIdx.y * p.rows * p.H + (size_t)r * p.H + h;
+      float *dst = p.part_o + idx * HD;
+#pragma unroll
+      for (int n = 0; n < HD / 8; n++) *(float2 *)(dst + n * 8 + qcol) = make_float2(o[n][half * 2], o[n][half * 2 + 1]);
+      if ((lane & 3) == 0) { p.part_ml[idx * 2] = mx; p.part_ml[idx * 2 + 1] = l; }
+    }
+  }
+}
+
+// merge the splits: out = sum_s 2^((m_s - M) c) O_s / sum_s 2^((m_s - M) c) l_s
+template <int HD>
+__global__ void attn_combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, int nsplit, int nrh,
+                                    bf16 *__restrict__ out) {
+  int rh = blockIdx.x, d = threadIdx.x;
+  const float sc = rsqrtf((float)HD) * 1.4426950408889634f;
+  float M = -INFINITY;
+  for (int s = 0; s < nsplit; s++) M = fmaxf(M, part_ml[((size_t)s * nrh + rh) * 2]);
+  float acc = 0.0f, l = 0.0f;
+  for (int s = 0; s < nsplit; s++) {
+    float m = part_ml[((size_t)s * nrh + rh) * 2], ls = part_ml[((size_t)s * nrh + rh) * 2 + 1];
+    if (m == -INFINITY) continue;
+    float w = exp2f((m - M) * sc);
+    acc += w * part_o[((size_t)s * nrh + rh) * HD + d];
+    l += w * ls;
+  }
+  out[(size_t)rh * HD + d] = __float2bfloat16_rn(l > 0.0f ? acc / l : 0.0f);
+}
+
+int pick_splits(int seqs, int G, int mtiles, int max_ctx_tiles) {
+  int base = seqs * G * mtiles;
+  int want = (2 * 148 + base - 1) / base;
+  int s = want < max_ctx_tiles ? want : max_ctx_tiles;
+  if (s > MAX_SPLITS) s = MAX_SPLITS;
+  return s < 1 ? 1 : s;
+}
+
+}  // namespace
+
+bool attn_fast_supported(int head_dim, int group) { return (head_dim == 64 || head_dim == 128) && group >= 1; }
+
+size_t attn_fast_scratch_bytes(int rows, int n_heads, int head_dim, int max_ctx) {
+  (void)max_ctx;
+  return (size_t)MAX_SPLITS * rows * n_heads * (head_dim + 2) * sizeof(float) + 256;
+}
+
 int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail_len, bf16 *out, int rows, int H, int G,
-                     int hd, int max_ctx, void *scratch, cudaStream_t s) {
-  return 0;
+                     int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s) {
+  if (rps < 1 || rows % rps) rps = 1;
+  int seqs = rows / rps, grp = H / G;
+  int mtiles = (rps * grp + MT - 1) / MT;
+  int ntiles_hint = (ctx_hint + tail_len + KT - 1) / KT;
+  int nsplit = scratch ? pick_splits(seqs, G, mtiles, ntiles_hint < 1 ? 1 : ntiles_hint) : 1;
+  AttnParams p;
+  p.q = q; p.kpool = (const bf16 *)pool.k; p.vpool = (const bf16 *)pool.v; p.pm = pm; p.m = m; p.tail_len = tail_len;
+  p.rows = rows; p.H = H; p.G = G; p.rps = rps; p.nsplit = nsplit; p.out = out;
+  p.part_o = (float *)scratch;
+  p.part_ml = p.part_o ? p.part_o + (size_t)MAX_SPLITS * rows * H * hd : nullptr;
+  dim3 grid(mtiles, nsplit, seqs * G);
+  size_t smem = (size_t)4 * KT * hd * 2;
+  if (smem < (size_t)MT * hd * 2) smem = (size_t)MT * hd * 2;
+  static bool attr[2] = {false, false};
+  if (hd == 128) {
+    if (!attr[1]) { cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[1] = true; }
+    attn_mma_kernel<128><<<grid, 256, smem, s>>>(p);
+    if (nsplit > 1) attn_combine_kernel<128><<<rows * H, 128, 0, s>>>(p.part_o, p.part_ml, nsplit, rows * H, out);
+  } else {
+    if (!attr[0]) { cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[0] = true; }
+    attn_mma_kernel<64><<<grid, 256, smem, s>>>(p);
+    if (nsplit > 1) attn_combine_kernel<64><<<rows * H, 64, 0, s>>>(p.part_o, p.part_ml, nsplit, rows * H, out);
+  }
+  return nsplit > 1 ? 2 : 1;
 }
 
 }  // namespace spec

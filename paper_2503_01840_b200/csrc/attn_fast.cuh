@@ -6,8 +6,10 @@ namespace spec {
 
 bool attn_fast_supported(int head_dim, int group);
 size_t attn_fast_scratch_bytes(int rows, int n_heads, int head_dim, int max_ctx);
-// returns the number of kernels launched
+// rows are grouped as rows/rps consecutive blocks of rps rows that belong to one sequence (rps = 1 when
+// nothing is known); ctx_hint sizes the key split (any value is correct); scratch may be NULL (one
+// split).  Returns the number of kernels launched.
 int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail_len, bf16 *out, int rows, int H, int G,
-                     int hd, int max_ctx, void *scratch, cudaStream_t s);
+                     int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s);
 
 }  // namespace spec
