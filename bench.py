@@ -240,6 +240,7 @@ def main():
     t0 = time.time()
     dec.prefill(prompts, reserve)
     t_prefill = time.time() - t0
+    prefill_launches = dec.launches_per_step()
 
     counts = torch.zeros(max(args.steps, args.warmup), B, dtype=torch.int32, device=dev)
     timed_steps(dec, args.warmup, counts)
@@ -309,7 +310,8 @@ def main():
             "clocks": clocks, "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": d2h,
                                       "note": "spec_step with host outputs, synchronised every step; a step has no host input"},
             "gpu_launches": launches * args.steps, "roofline": roofline,
-            "setup_s": {"weights": round(t_gen, 2), "prefill": round(t_prefill, 2)}}
+            "setup_s": {"weights": round(t_gen, 2), "prefill": round(t_prefill, 2)},
+            "launches": {"per_step": launches, "prefill": prefill_launches}}
 
     if rank == 0 and world == 1 and not args.no_extras:
         extras = {}
