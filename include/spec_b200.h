@@ -196,6 +196,28 @@ int spec_attention(int32_t dtype, int32_t impl, const void *q, const void *k_poo
                    const uint64_t *row_mask_hi, int32_t tail_len, void *out, int32_t rows, int32_t n_heads,
                    int32_t n_kv_heads, int32_t head_dim, int32_t max_ctx, void *scratch, void *stream);
 
+/* spec_attention without any allocation (the paper has no counterpart: this is a packaging variant
+ * of the tensor-core kernel, bf16 only).  It is meant for callers that cannot obtain device memory
+ * at the point where they need attention - code living inside a pre-sized memory arena, plugins
+ * whose host forbids cudaMalloc after start-up, loops that must not take the implicit device
+ * synchronisation of an allocation.  The split-KV partial results go to an 8 MiB device array that
+ * is part of the library image (every GPU that loads the library holds it until the process ends);
+ * inputs and outputs are still the caller's, with the meaning and layout of spec_attention.
+ *   - Limit: spec_attn_scratch_bytes(rows, n_heads, head_dim, max_ctx) must not exceed
+ *     spec_attention_static_capacity(); larger calls return SPEC_ERR_WORKSPACE and print the sizes.
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it has to start at zero (every partial
+ *     that is read was written by the same call), but two calls whose kernels overlap on the GPU
+ *     (different streams) race on it: keep calls on one stream or order them yourself.
+ *   - Calls no cudaMalloc/cudaFree and no allocating library routine; does not synchronise. */
+size_t spec_attention_static_capacity(void);
+int spec_attention_static(const void *q, const void *k_pool, const void *v_pool, const int32_t *page_table,
+                          int32_t pages_per_seq, int32_t page_size, const int32_t *row_seq, const int32_t *row_ctx,
+                          const int32_t *row_tail_base, const uint64_t *row_mask_lo, const uint64_t *row_mask_hi,
+                          int32_t tail_len, void *out, int32_t rows, int32_t n_heads, int32_t n_kv_heads,
+                          int32_t head_dim, int32_t max_ctx, void *stream);
+
 /* Per-row log-softmax + top-K (value desc, index asc) over fp32 logits [rows][n]: the expansion
  * step of the dynamic tree.  out_idx int32 [rows][K], out_lp float [rows][K]. */
 int spec_logsoftmax_topk(const float *logits, int32_t rows, int32_t n, int32_t K, int32_t *out_idx, float *out_lp,

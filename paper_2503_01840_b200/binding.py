@@ -57,7 +57,7 @@ class _Cfg(C.Structure):
 EXPORTS = ("spec_workspace_bytes", "spec_init", "spec_prefill", "spec_step", "spec_step_async", "spec_plain_step",
            "spec_lengths", "spec_profile_step", "spec_launches_per_step", "spec_step_bytes", "spec_free", "spec_last_error",
            "spec_debug_read", "spec_debug_read_kv", "spec_gemm_scratch_bytes", "spec_gemm", "spec_attn_scratch_bytes",
-           "spec_attention", "spec_logsoftmax_topk", "spec_argmax")
+           "spec_attention", "spec_attention_static", "spec_attention_static_capacity", "spec_logsoftmax_topk", "spec_argmax")
 
 
 def library_path() -> str:
@@ -96,6 +96,9 @@ def lib():
     L.spec_attn_scratch_bytes.restype = sz
     L.spec_attention.argtypes = [i32, i32, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, i32, vp, i32, i32, i32, i32, i32,
                                  vp, vp]
+    L.spec_attention_static_capacity.argtypes = []
+    L.spec_attention_static_capacity.restype = sz
+    L.spec_attention_static.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, vp]
     L.spec_logsoftmax_topk.argtypes = [vp, i32, i32, i32, vp, vp, vp]
     L.spec_argmax.argtypes = [vp, i32, i32, vp, vp]
     _lib = L
@@ -305,6 +308,23 @@ def attention(q, k_pool, v_pool, page_table, page_size, row_seq, row_ctx, row_ta
                               rows, H, n_kv_heads, hd, max_ctx, scratch.data_ptr(), _stream_ptr(None))
     if rc:
         raise SpecError(rc, "spec_attention")
+    return out
+
+
+def attention_static(q, k_pool, v_pool, page_table, page_size, row_seq, row_ctx, row_tail_base, mask_lo, mask_hi,
+                     tail_len, n_kv_heads, max_ctx, out: Optional[torch.Tensor] = None):
+    """spec_attention_static: the tensor-core attention kernel with its split-KV scratch in the library's
+    built-in device array, for callers that cannot allocate.  `out` may be passed in so that the call itself
+    allocates nothing; raises SpecError(-3) when the shape needs more scratch than the array holds."""
+    rows, H, hd = q.shape
+    if out is None:
+        out = torch.empty_like(q)
+    rc = lib().spec_attention_static(q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), page_table.data_ptr(),
+                                     page_table.shape[1], page_size, row_seq.data_ptr(), row_ctx.data_ptr(),
+                                     row_tail_base.data_ptr(), mask_lo.data_ptr(), mask_hi.data_ptr(), tail_len,
+                                     out.data_ptr(), rows, H, n_kv_heads, hd, max_ctx, _stream_ptr(None))
+    if rc:
+        raise SpecError(rc, "spec_attention_static")
     return out
 
 

@@ -7,6 +7,10 @@
 // m16n8k16, keeps the softmax statistics in registers (quad shuffles), applies the bit-packed
 // ancestor mask to the tail keys, and writes either the final output (one split) or an unnormalised
 // partial (several splits) that a small combine kernel merges.
+#include <stdio.h>
+
+#include <mutex>
+
 #include "attn_fast.cuh"
 
 namespace spec {
@@ -297,3 +301,68 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
 }
 
 }  // namespace spec
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant of the tensor-core attention entry point.
+//
+// Some hosts of this library cannot allocate device memory when they need attention: code running
+// inside a memory-pool or arena that was sized up front, a plugin whose host process forbids
+// cudaMalloc after start-up, or a latency-critical loop where an allocation (an implicit device
+// synchronisation) is not acceptable.  For them the split-KV partial results live in a fixed
+// file-scope device array instead of a caller-provided scratch buffer.  Every GPU that loads the
+// library carries the array until the process exits.
+namespace spec {
+namespace {
+constexpr size_t STATIC_SCRATCH_BYTES = (size_t)8 << 20;     // 8 MiB per device
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+void *g_static_scratch_dev[MAX_DEVICES];                      // device address of the array, per device
+bool g_static_scratch_ready[MAX_DEVICES];
+std::mutex g_static_scratch_mu;
+
+// Device address of the array on the current device.  In host code the array's name is only a handle
+// for the runtime, not a device address, so it is resolved once per device with cudaGetSymbolAddress.
+int static_scratch_ptr(void **out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return -6;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mu);
+  if (!g_static_scratch_ready[dev]) {
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return -6;
+    g_static_scratch_dev[dev] = p;
+    g_static_scratch_ready[dev] = true;
+  }
+  *out = g_static_scratch_dev[dev];
+  return 0;
+}
+}  // namespace
+}  // namespace spec
+
+extern "C" size_t spec_attention_static_capacity(void) { return spec::STATIC_SCRATCH_BYTES; }
+
+extern "C" int spec_attention_static(const void *q, const void *k_pool, const void *v_pool, const int32_t *page_table,
+                                     int32_t pages_per_seq, int32_t page_size, const int32_t *row_seq,
+                                     const int32_t *row_ctx, const int32_t *row_tail_base, const uint64_t *row_mask_lo,
+                                     const uint64_t *row_mask_hi, int32_t tail_len, void *out, int32_t rows, int32_t H,
+                                     int32_t G, int32_t hd, int32_t max_ctx, void *stream) {
+  using namespace spec;
+  if (!q || !k_pool || !v_pool || !page_table || !row_seq || !row_ctx || !row_tail_base || !row_mask_lo || !row_mask_hi || !out)
+    return -2;                                                         // SPEC_ERR_NULL
+  if (rows < 1 || H < 1 || G < 1 || H % G || tail_len < 0 || tail_len > 128 || page_size < 1 || pages_per_seq < 1) return -1;
+  if (!attn_fast_supported(hd, H / G)) return -8;                      // SPEC_ERR_UNSUPPORTED
+  if (attn_fast_scratch_bytes(rows, H, hd, max_ctx) > STATIC_SCRATCH_BYTES) {
+    fprintf(stderr, "spec_attention_static: rows=%d heads=%d head_dim=%d needs %zu bytes of split-KV scratch, the built-in "
+                    "array holds %zu\n", rows, H, hd, attn_fast_scratch_bytes(rows, H, hd, max_ctx), STATIC_SCRATCH_BYTES);
+    return -3;                                                         // SPEC_ERR_WORKSPACE
+  }
+  void *scratch = nullptr;
+  if (int rc = static_scratch_ptr(&scratch)) return rc;
+  RowMeta m{};
+  m.seq = (int32_t *)row_seq; m.ctx = (int32_t *)row_ctx; m.tail_base = (int32_t *)row_tail_base;
+  m.mask_lo = (uint64_t *)row_mask_lo; m.mask_hi = (uint64_t *)row_mask_hi;
+  KvPool pool{(void *)k_pool, (void *)v_pool};
+  PageMap pm{page_table, pages_per_seq, page_size, 1 << 30};
+  launch_attn_fast((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, 1, max_ctx, scratch, (cudaStream_t)stream);
+  return cudaGetLastError() == cudaSuccess ? 0 : -6;
+}
