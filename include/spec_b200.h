@@ -49,7 +49,10 @@ enum {
   SPEC_FLAG_REF_GEMM = 1,        /* use the plain CUDA-core GEMM kernel also for bf16 (debugging aid)   */
   SPEC_FLAG_REF_ATTN = 2,        /* use the plain CUDA-core attention kernel also for bf16             */
   SPEC_FLAG_CAPTURE = 4,         /* keep per-pass draft logits / features for spec_debug_read          */
-  SPEC_FLAG_NO_GRAPH = 8         /* launch kernels one by one instead of replaying a CUDA graph        */
+  SPEC_FLAG_NO_GRAPH = 8,        /* launch kernels one by one instead of replaying a CUDA graph        */
+  SPEC_FLAG_UNFUSED = 16,        /* bf16: separate norm / RoPE / activation kernels and split-K partial
+                                    sums in global memory instead of the fused GEMM epilogues          */
+  SPEC_FLAG_NO_PDL = 32          /* no programmatic dependent launch between the kernels of a step    */
 };
 
 /* Target model weights (Section 3.1: the frozen target whose layers are tapped).  Device pointers;
@@ -153,7 +156,7 @@ enum spec_debug_what {
   SPEC_DBG_TREE_POOLIDX,     /* int32 [nodes]            */
   SPEC_DBG_TREE_SCORE,       /* float [nodes]            */
   SPEC_DBG_Y,                /* int32 [nodes]            */
-  SPEC_DBG_TARGET_LOGITS,    /* float [nodes][vocab]     */
+  SPEC_DBG_TARGET_LOGITS,    /* float [nodes][vocab]; bf16 models keep them only with SPEC_FLAG_CAPTURE */
   SPEC_DBG_NODE_TAPS,        /* float [nodes][3*hidden] (widened from the storage dtype) */
   SPEC_DBG_NODE_HIDDEN,      /* float [nodes][hidden] residual stream after the last block */
   SPEC_DBG_DRAFT_LOGITS,     /* float [D][K][draft_vocab]; needs SPEC_FLAG_CAPTURE      */
@@ -182,6 +185,13 @@ int spec_debug_read_kv(spec_ctx *ctx, int32_t seq, int32_t layer, int32_t pos, f
 size_t spec_gemm_scratch_bytes(int32_t rows, int32_t out, int32_t in);
 int spec_gemm(int32_t dtype, int32_t impl, const void *x, const void *w, float *out_f32, int32_t rows, int32_t out,
               int32_t in, int32_t ldo, void *scratch, void *stream);
+
+/* The same contraction on the kernel the step uses (Section 3.1's FC, projection and LM-head layers are
+ * all of this form): bf16, tcgen05/TMEM, split-K reduced across a thread-block cluster through
+ * distributed shared memory, no scratch.  rows <= 256, in % 8 == 0, 16-byte aligned x and w.
+ * split: K slices (= cluster size, 1..8), stages: TMA pipeline depth; 0 lets the library choose. */
+int spec_gemm_fused(const void *x, const void *w, float *out_f32, int32_t rows, int32_t out, int32_t in, int32_t ldo,
+                    int32_t split, int32_t stages, void *stream);
 
 /* Tree-masked paged GQA attention (Section 2.2 "tree attention") for `rows` query rows of one or
  * more sequences.  q [rows][H][hd] dtype; K/V pools [num_pages][G][page_size][hd] dtype;
@@ -219,9 +229,13 @@ int spec_attention_static(const void *q, const void *k_pool, const void *v_pool,
                           int32_t head_dim, int32_t max_ctx, void *stream);
 
 /* Per-row log-softmax + top-K (value desc, index asc) over fp32 logits [rows][n]: the expansion
- * step of the dynamic tree.  out_idx int32 [rows][K], out_lp float [rows][K]. */
+ * step of the dynamic tree (Section 2.2; Appendix A "nodes during the expansion phase").  K <= 16.
+ * out_idx int32 [rows][K], out_lp float [rows][K].  scratch: device buffer of
+ * spec_topk_scratch_bytes(rows, n, K) bytes for the two-stage kernel the step uses (chunk candidates,
+ * then a per-row merge); NULL selects the plain one-CTA-per-row kernel. */
+size_t spec_topk_scratch_bytes(int32_t rows, int32_t n, int32_t K);
 int spec_logsoftmax_topk(const float *logits, int32_t rows, int32_t n, int32_t K, int32_t *out_idx, float *out_lp,
-                         void *stream);
+                         void *scratch, void *stream);
 /* Per-row argmax (lowest index on ties) over fp32 [rows][n]. */
 int spec_argmax(const float *logits, int32_t rows, int32_t n, int32_t *out_idx, void *stream);
 

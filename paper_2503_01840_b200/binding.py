@@ -19,7 +19,7 @@ from . import build as _build
 _lib = None
 
 F32, BF16 = 0, 1
-FLAG_REF_GEMM, FLAG_REF_ATTN, FLAG_CAPTURE, FLAG_NO_GRAPH = 1, 2, 4, 8
+FLAG_REF_GEMM, FLAG_REF_ATTN, FLAG_CAPTURE, FLAG_NO_GRAPH, FLAG_UNFUSED, FLAG_NO_PDL = 1, 2, 4, 8, 16, 32
 
 (DBG_TREE_TOK, DBG_TREE_PARENT, DBG_TREE_DEPTH, DBG_TREE_MASK, DBG_TREE_POOLIDX, DBG_TREE_SCORE, DBG_Y,
  DBG_TARGET_LOGITS, DBG_NODE_TAPS, DBG_NODE_HIDDEN, DBG_DRAFT_LOGITS, DBG_DRAFT_A, DBG_POOL_TOK, DBG_POOL_SCORE,
@@ -56,7 +56,8 @@ class _Cfg(C.Structure):
 
 EXPORTS = ("spec_workspace_bytes", "spec_init", "spec_prefill", "spec_step", "spec_step_async", "spec_plain_step",
            "spec_lengths", "spec_profile_step", "spec_launches_per_step", "spec_step_bytes", "spec_free", "spec_last_error",
-           "spec_debug_read", "spec_debug_read_kv", "spec_gemm_scratch_bytes", "spec_gemm", "spec_attn_scratch_bytes",
+           "spec_debug_read", "spec_debug_read_kv", "spec_gemm_scratch_bytes", "spec_gemm", "spec_gemm_fused",
+           "spec_topk_scratch_bytes", "spec_attn_scratch_bytes",
            "spec_attention", "spec_attention_static", "spec_attention_static_capacity", "spec_logsoftmax_topk", "spec_argmax")
 
 
@@ -99,7 +100,10 @@ def lib():
     L.spec_attention_static_capacity.argtypes = []
     L.spec_attention_static_capacity.restype = sz
     L.spec_attention_static.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, vp]
-    L.spec_logsoftmax_topk.argtypes = [vp, i32, i32, i32, vp, vp, vp]
+    L.spec_gemm_fused.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]
+    L.spec_topk_scratch_bytes.argtypes = [i32, i32, i32]
+    L.spec_topk_scratch_bytes.restype = sz
+    L.spec_logsoftmax_topk.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
     L.spec_argmax.argtypes = [vp, i32, i32, vp, vp]
     _lib = L
     return L
@@ -328,11 +332,29 @@ def attention_static(q, k_pool, v_pool, page_table, page_size, row_seq, row_ctx,
     return out
 
 
-def logsoftmax_topk(logits: torch.Tensor, K: int):
+def gemm_fused(x: torch.Tensor, w: torch.Tensor, split: int = 0, stages: int = 0, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """out = x . w^T (fp32) on the cluster split-K tcgen05 kernel of the step; split/stages 0 = library's choice."""
+    rows, I = x.shape
+    O = w.shape[0]
+    assert w.shape[1] == I and x.is_contiguous() and w.is_contiguous() and x.dtype == w.dtype == torch.bfloat16
+    if out is None:
+        out = torch.empty(rows, O, dtype=torch.float32, device=x.device)
+    rc = lib().spec_gemm_fused(x.data_ptr(), w.data_ptr(), out.data_ptr(), rows, O, I, out.stride(0), split, stages,
+                               _stream_ptr(None))
+    if rc:
+        raise SpecError(rc, "spec_gemm_fused")
+    return out
+
+
+def logsoftmax_topk(logits: torch.Tensor, K: int, two_stage: bool = True):
     rows, n = logits.shape
     idx = torch.empty(rows, K, dtype=torch.int32, device=logits.device)
     lp = torch.empty(rows, K, dtype=torch.float32, device=logits.device)
-    rc = lib().spec_logsoftmax_topk(logits.data_ptr(), rows, n, K, idx.data_ptr(), lp.data_ptr(), _stream_ptr(None))
+    scratch = None
+    if two_stage:
+        scratch = torch.empty(lib().spec_topk_scratch_bytes(rows, n, K), dtype=torch.uint8, device=logits.device)
+    rc = lib().spec_logsoftmax_topk(logits.data_ptr(), rows, n, K, idx.data_ptr(), lp.data_ptr(),
+                                    scratch.data_ptr() if scratch is not None else None, _stream_ptr(None))
     if rc:
         raise SpecError(rc, "spec_logsoftmax_topk")
     return idx, lp

@@ -11,18 +11,23 @@
 
 #include "../../include/spec_b200.h"
 #include "gemm_fast.cuh"
+#include "gemm_fused.cuh"
 #include "attn_fast.cuh"
 #include "state.cuh"
 
 using namespace spec;
 
 namespace spec {
+thread_local bool tl_pdl = false;
+
 void launch_logsoftmax_topk_rows(const float *logits, const int32_t *src_row, int rows, int n, int K, int32_t *idx,
                                  float *lp, cudaStream_t s);
 
 // dst row b*dst_stride_rows <- src row src_row[b] (fp32, `width` columns); rows with src_row < 0 are skipped
 __global__ void gather_rows_kernel(const float *__restrict__ src, const int32_t *__restrict__ src_row,
                                    float *__restrict__ dst, int width, int dst_stride_rows) {
+  pdl_wait();
+  pdl_trigger();
   int b = blockIdx.x, sr = src_row[b];
   if (sr < 0) return;
   for (int i = threadIdx.x; i < width; i += blockDim.x)
@@ -30,7 +35,7 @@ __global__ void gather_rows_kernel(const float *__restrict__ src, const int32_t 
 }
 static void launch_gather_rows(const float *src, const int32_t *src_row, float *dst, int B, int width, int dst_stride_rows,
                                cudaStream_t s) {
-  gather_rows_kernel<<<B, 256, 0, s>>>(src, src_row, dst, width, dst_stride_rows);
+  launch_k(gather_rows_kernel, dim3(B), dim3(256), 0, s, src, src_row, dst, width, dst_stride_rows);
 }
 }
 
@@ -76,6 +81,13 @@ struct spec_ctx {
   TreeBufs tb;
   int32_t *status;
   float *cap_logits, *cap_a;   // capture buffers (SPEC_FLAG_CAPTURE)
+  // fused bf16 path: GEMM epilogues do the norm / RoPE / activation / residual / argmax work
+  bool fused = false;
+  float *ssq = nullptr;        // [ceil(k/128)][Ralloc] per-tile sums of squares of the residual stream
+  float *best_val = nullptr;   // [ceil(V/128)][Ralloc] per-tile argmax candidates of the target LM head
+  int32_t *best_idx = nullptr;
+  void *topk_scratch = nullptr;
+  int ktiles = 0, vtiles = 0;
   void *gemm_scratch;
   size_t gemm_scratch_bytes;
   void *attn_scratch;
@@ -204,6 +216,11 @@ static size_t carve(spec_ctx *c, void *base) {
   } else {
     c->cap_logits = c->cap_a = nullptr;
   }
+  c->ktiles = (k + 127) / 128; c->vtiles = (c->V + 127) / 128;
+  c->ssq = cv.take<float>((size_t)c->ktiles * R);
+  c->best_val = cv.take<float>((size_t)c->vtiles * R);
+  c->best_idx = cv.take<int32_t>((size_t)c->vtiles * R);
+  c->topk_scratch = cv.take_bytes(topk_scratch_bytes(R, c->Vd, c->K));
   c->gemm_scratch_bytes = 0;
   c->gemm_scratch = nullptr;
   c->attn_scratch_bytes = attn_fast_scratch_bytes(R, c->H, c->hd, g.max_ctx);
@@ -273,6 +290,13 @@ extern "C" int spec_init(spec_ctx **out, const spec_target_weights *tw, const sp
       return rc;
     }
   }
+  c->fused = c->fg && !(cfg->flags & SPEC_FLAG_UNFUSED) && c->hd <= 128 && (c->hd & (c->hd - 1)) == 0 && c->Ralloc <= 256;
+  if (c->fg && c->R > 256) {
+    int rc = fail(nullptr, SPEC_ERR_UNSUPPORTED, "spec_init: %d rows per pass exceed the 256 the tensor-core GEMM takes", c->R);
+    fast_gemm_destroy(c->fg);
+    delete c;
+    return rc;
+  }
   *out = c;
   return SPEC_OK;
 }
@@ -290,7 +314,9 @@ extern "C" int spec_free(spec_ctx *c) {
 template <typename T> struct Sched {
   spec_ctx *c;
   cudaStream_t s;
-  explicit Sched(spec_ctx *ctx) : c(ctx), s(ctx->stream) {}
+  explicit Sched(spec_ctx *ctx) : c(ctx), s(ctx->stream) { tl_pdl = c->fused && !(c->cfg.flags & SPEC_FLAG_NO_PDL); }
+  ~Sched() { tl_pdl = false; }
+  Sched(const Sched &) = delete;
   void tick(int n = 1) { c->launches += n; }
   // profiling: one event at the start of every launch; the interval to the next event is charged to `cls`
   void mark(int cls) {
@@ -320,6 +346,95 @@ template <typename T> struct Sched {
       launch_gemm_ref<T>((const T *)x, (const T *)w, out + col0, rows, O, I, ldo, s);
     }
     tick();
+  }
+
+  // ---- fused bf16 path -----------------------------------------------------------------------
+  FusedGemmArgs fargs(const void *x, int rows, int I) const {
+    FusedGemmArgs a;
+    a.x = (const bf16 *)x; a.rows = rows; a.I = I; a.status = c->status; a.pdl = tl_pdl;
+    return a;
+  }
+  // the GEMM input is bf16(residual * gain): apply the RMSNorm factor of the residual as a row scale
+  void with_norm_scale(FusedGemmArgs &a) const {
+    a.ssq_in = c->ssq; a.ssq_in_tiles = c->ktiles; a.ssq_ld = c->Ralloc; a.k_in = c->k; a.eps = c->cfg.rms_eps;
+  }
+  void fgemm(FusedEpi epi, const FusedGemmArgs &a) {
+    mark(SPEC_PROF_GEMM);
+    int rc = fused_gemm_launch(c->fg, epi, a, s);
+    if (rc && !c->sched_err) c->sched_err = rc;
+    tick();
+  }
+  // residual-producing GEMM: x (+)= in . w^T, h = bf16(x * gain), ssq, optional taps
+  void fgemm_resid(const void *in, int I, const void *w, int rows, bool add, const void *gain, int tap_mask) {
+    FusedGemmArgs a = fargs(in, rows, I);
+    a.w[0] = (const bf16 *)w; a.O[0] = c->k; a.nw = 1;
+    a.xres = c->x; a.gain = (const bf16 *)gain; a.hb = (bf16 *)c->h; a.ssq_out = c->ssq; a.ssq_ld = c->Ralloc;
+    a.taps = (bf16 *)c->node_taps; a.tap_mask = tap_mask; a.resid_add = add ? 1 : 0;
+    fgemm(EPI_RESID, a);
+  }
+  void block_fused(const LayerW &w, KvPool pool, int rows, int tail_len, const void *next_gain, int tap_mask) {
+    int k = c->k, qd = c->H * c->hd, kvd = c->G * c->hd, F = c->F;
+    FusedGemmArgs a = fargs(c->h, rows, k);
+    a.w[0] = (const bf16 *)w.wq; a.w[1] = (const bf16 *)w.wk; a.w[2] = (const bf16 *)w.wv;
+    a.O[0] = qd; a.O[1] = kvd; a.O[2] = kvd; a.nw = 3;
+    with_norm_scale(a);
+    a.cs = c->cs; a.m = c->meta; a.q = (bf16 *)c->q; a.pool = pool;
+    a.pm = PageMap{c->page_table, c->pps, c->cfg.page_size, c->cfg.num_pages};
+    a.H = c->H; a.G = c->G; a.hd = c->hd;
+    fgemm(EPI_QKV, a);
+    attention(pool, rows, tail_len);
+    fgemm_resid(c->ao, qd, w.wo, rows, true, w.mlp_norm, 0);
+    FusedGemmArgs g = fargs(c->h, rows, k);
+    g.w[0] = (const bf16 *)w.w_gate; g.w[1] = (const bf16 *)w.w_up; g.O[0] = F; g.O[1] = F; g.nw = 2;
+    with_norm_scale(g);
+    g.act = (bf16 *)c->act;
+    fgemm(EPI_SWIGLU, g);
+    fgemm_resid(c->act, F, w.w_down, rows, true, next_gain, tap_mask);
+  }
+  void target_forward_fused(int rows, int tail_len, bool want_logits) {
+    mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
+    mark(SPEC_PROF_MISC);
+    launch_embed_norm((const bf16 *)c->embed, c->meta.tok, (const bf16 *)c->tl[0].attn_norm, c->x, (bf16 *)c->h, c->ssq, rows, c->k,
+                      c->Ralloc, s);
+    tick();
+    for (int l = 0; l < c->L; l++)
+      block_fused(c->tl[l], c->pools[l], rows, tail_len, l + 1 < c->L ? c->tl[l + 1].attn_norm : c->final_norm, tap_mask_of(l));
+    if (want_logits) {
+      FusedGemmArgs a = fargs(c->h, rows, c->k);
+      a.w[0] = (const bf16 *)c->lm_head; a.O[0] = c->V; a.nw = 1;
+      with_norm_scale(a);
+      a.best_val = c->best_val; a.best_idx = c->best_idx; a.best_ld = c->Ralloc;
+      if (c->cap_logits) { a.out_f32 = c->logits; a.ldo = c->V; }
+      fgemm(EPI_ARGMAX, a);
+      mark(SPEC_PROF_ARGMAX); launch_argmax_merge(c->best_val, c->best_idx, c->vtiles, c->Ralloc, rows, c->tb.y, s); tick();
+    }
+  }
+  void fuse_fused(const void *taps, int rows) {
+    FusedGemmArgs a = fargs(taps, rows, 3 * c->k);
+    a.w[0] = (const bf16 *)c->fc3; a.O[0] = c->k; a.nw = 1;
+    a.out_f32 = c->proj; a.ldo = c->k;
+    fgemm(EPI_F32, a);
+    c->np_proj = 1; c->ps_proj = 0;
+  }
+  void draft_forward_fused(const float *feat, int nparts, size_t fstride, const int32_t *src_row, int rows, int tail_len) {
+    mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
+    mark(SPEC_PROF_MISC);
+    launch_build_cat<bf16>(feat, nparts, fstride, src_row, (const bf16 *)c->embed, c->meta.tok, c->meta.seq, (bf16 *)c->cat, rows, c->k, s);
+    tick();
+    fgemm_resid(c->cat, 2 * c->k, c->fc2, rows, false, c->dl.attn_norm, 0);
+    block_fused(c->dl, c->pools[c->L], rows, tail_len, c->dfinal_norm, 0);
+  }
+  void draft_logits_fused(int rows) {
+    FusedGemmArgs a = fargs(c->h, rows, c->k);
+    a.w[0] = (const bf16 *)c->dlm_head; a.O[0] = c->Vd; a.nw = 1;
+    with_norm_scale(a);
+    a.out_f32 = c->logits; a.ldo = c->Vd;
+    fgemm(EPI_F32, a);
+  }
+  void topk(const int32_t *src_row, int rows) {
+    mark(SPEC_PROF_TOPK);
+    if (c->fused) tick(launch_topk2(c->logits, src_row, rows, c->Vd, c->K, c->tb.tk_idx, c->tb.tk_lp, c->topk_scratch, s));
+    else { launch_logsoftmax_topk_rows(c->logits, src_row, rows, c->Vd, c->K, c->tb.tk_idx, c->tb.tk_lp, s); tick(); }
   }
 
   void attention(KvPool pool, int rows, int tail_len) {
@@ -375,6 +490,7 @@ template <typename T> struct Sched {
 
   // target forward over the rows of c->meta: taps -> node_taps, argmax -> tb.y
   void target_forward(int rows, int tail_len, bool want_logits) {
+    if (c->fused) return target_forward_fused(rows, tail_len, want_logits);
     mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
     mark(SPEC_PROF_MISC); launch_embed<T>((const T *)c->embed, c->meta.tok, c->x, rows, c->k, s); tick();
     for (int l = 0; l < c->L; l++)
@@ -390,12 +506,14 @@ template <typename T> struct Sched {
 
   // FC3 over `rows` rows of taps -> proj (Section 3.1: g = FC([l;m;h]))
   void fuse(const void *taps, int rows) {
+    if (c->fused) return fuse_fused(taps, rows);
     c->np_proj = pick(c->k, 3 * c->k, c->smax_proj); c->ps_proj = pstride(c->k);
     gemm(taps, c->fc3, c->proj, rows, c->k, 3 * c->k, c->k, 0, c->np_proj);
   }
 
   // draft head on the rows of c->meta: cat = [feat ; e(tok)], FC2, decoder block, final norm (-> h)
   void draft_forward(const float *feat, int nparts, size_t fstride, const int32_t *src_row, int rows, int tail_len) {
+    if (c->fused) return draft_forward_fused(feat, nparts, fstride, src_row, rows, tail_len);
     mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
     mark(SPEC_PROF_MISC); launch_build_cat<T>(feat, nparts, fstride, src_row, (const T *)c->embed, c->meta.tok, c->meta.seq, (T *)c->cat, rows, c->k, s);
     tick();
@@ -408,6 +526,7 @@ template <typename T> struct Sched {
   }
 
   void draft_logits(int rows) {
+    if (c->fused) return draft_logits_fused(rows);
     gemm(c->h, c->dlm_head, c->logits, rows, c->Vd, c->k, c->Vd, 0, 1);
   }
 
@@ -434,14 +553,14 @@ template <typename T> struct Sched {
       fuse(c->pend_taps, c->Te);
       draft_forward(c->proj, c->np_proj, c->ps_proj, nullptr, c->Te, c->Pmax);
       draft_logits(c->Te);
-      mark(SPEC_PROF_TOPK); launch_logsoftmax_topk_rows(c->logits, c->st.last_row, c->B, c->Vd, c->K, c->tb.tk_idx, c->tb.tk_lp, s); tick();
+      topk(c->st.last_row, c->B);
       capture(1, c->Te, true);
       mark(SPEC_PROF_TREE); launch_expand(c->st, c->tb, c->meta, c->d2t, 1, c->B, s); tick();
       for (int p = 2; p <= c->D; p++) {
         c->cur_rps = c->K;
         draft_forward(c->x, 1, 0, c->tb.feat_row, c->Td, c->tail_tree);
         draft_logits(c->Td);
-        mark(SPEC_PROF_TOPK); launch_logsoftmax_topk_rows(c->logits, nullptr, c->Td, c->Vd, c->K, c->tb.tk_idx, c->tb.tk_lp, s); tick();
+        topk(nullptr, c->Td);
         capture(p, c->Td, false);
         mark(SPEC_PROF_TREE); launch_expand(c->st, c->tb, c->meta, c->d2t, p, c->B, s); tick();
       }
@@ -746,7 +865,9 @@ extern "C" int64_t spec_debug_read(spec_ctx *c, int32_t what, int32_t seq, void 
     case SPEC_DBG_TREE_POOLIDX: return copy_out(c, t.poolidx + t0, nn, dst, bytes);
     case SPEC_DBG_TREE_SCORE: return copy_out(c, t.score + t0, nn, dst, bytes);
     case SPEC_DBG_Y: return copy_out(c, t.y + t0, nn, dst, bytes);
-    case SPEC_DBG_TARGET_LOGITS: return copy_out(c, c->logits + t0 * c->V, (size_t)nn * c->V, dst, bytes);
+    case SPEC_DBG_TARGET_LOGITS:
+      if (c->fused && !c->cap_logits) return fail(c, SPEC_ERR_STATE, "spec_debug_read: target logits need SPEC_FLAG_CAPTURE on the fused path");
+      return copy_out(c, c->logits + t0 * c->V, (size_t)nn * c->V, dst, bytes);
     case SPEC_DBG_NODE_TAPS: return copy_widen(c, (const char *)c->node_taps + t0 * 3 * c->k * c->esz, (size_t)nn * 3 * c->k, dst, bytes);
     case SPEC_DBG_NODE_HIDDEN: return copy_out(c, c->x + t0 * c->k, (size_t)nn * c->k, dst, bytes);
     case SPEC_DBG_DRAFT_LOGITS:
@@ -809,6 +930,26 @@ extern "C" int spec_gemm(int32_t dtype, int32_t impl, const void *x, const void 
   return fast_gemm_oneshot((const bf16 *)x, (const bf16 *)w, out, rows, O, I, ldo, scratch, s);
 }
 
+extern "C" int spec_gemm_fused(const void *x, const void *w, float *out, int32_t rows, int32_t O, int32_t I, int32_t ldo,
+                               int32_t split, int32_t stages, void *stream) {
+  if (!x || !w || !out) return SPEC_ERR_NULL;
+  if (rows < 1 || O < 1 || I < 1 || ldo < O || split < 0 || stages < 0) return SPEC_ERR_INVALID_CFG;
+  static FastGemm *g = nullptr;
+  if (!g) {
+    std::string why;
+    g = fast_gemm_create(why);
+    if (!g) return SPEC_ERR_CUDA;
+  }
+  FusedGemmArgs a;
+  a.x = (const bf16 *)x; a.rows = rows; a.I = I; a.w[0] = (const bf16 *)w; a.O[0] = O; a.nw = 1;
+  a.out_f32 = out; a.ldo = ldo; a.split = split; a.stages = stages;
+  if (!fused_gemm_supported(EPI_F32, a)) return SPEC_ERR_UNSUPPORTED;
+  int rc = fused_gemm_launch(g, EPI_F32, a, (cudaStream_t)stream);
+  fast_gemm_forget(g);   // test buffers come and go; do not keep descriptors of freed memory
+  if (rc) return rc == -1 ? SPEC_ERR_INVALID_CFG : SPEC_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
+}
+
 extern "C" size_t spec_attn_scratch_bytes(int32_t rows, int32_t n_heads, int32_t head_dim, int32_t max_ctx) {
   return attn_fast_scratch_bytes(rows, n_heads, head_dim, max_ctx);
 }
@@ -838,11 +979,17 @@ extern "C" int spec_attention(int32_t dtype, int32_t impl, const void *q, const 
   return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }
 
+extern "C" size_t spec_topk_scratch_bytes(int32_t rows, int32_t n, int32_t K) {
+  if (rows < 1 || n < 1 || K < 1) return 0;
+  return topk_scratch_bytes(rows, n, K);
+}
+
 extern "C" int spec_logsoftmax_topk(const float *logits, int32_t rows, int32_t n, int32_t K, int32_t *out_idx, float *out_lp,
-                                    void *stream) {
+                                    void *scratch, void *stream) {
   if (!logits || !out_idx || !out_lp) return SPEC_ERR_NULL;
-  if (rows < 1 || n < 1 || K < 1 || K > n) return SPEC_ERR_INVALID_CFG;
-  launch_logsoftmax_topk(logits, rows, n, K, out_idx, out_lp, (cudaStream_t)stream);
+  if (rows < 1 || n < 1 || K < 1 || K > n || K > 16) return SPEC_ERR_INVALID_CFG;
+  if (scratch) launch_topk2(logits, nullptr, rows, n, K, out_idx, out_lp, scratch, (cudaStream_t)stream);
+  else launch_logsoftmax_topk(logits, rows, n, K, out_idx, out_lp, (cudaStream_t)stream);
   return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }
 

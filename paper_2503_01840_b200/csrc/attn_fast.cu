@@ -59,6 +59,8 @@ struct AttnParams {
 
 template <int HD>
 __global__ void __launch_bounds__(256) attn_mma_kernel(AttnParams p) {
+  pdl_wait();
+  pdl_trigger();
   constexpr int ROWB = HD * 2, CPR = HD / 8;          // bytes / 16-byte chunks per row
   constexpr int NKS = HD / 16;                        // k-steps of Q K^T
   extern __shared__ __align__(128) unsigned char sm[];
@@ -240,6 +242,8 @@ __global__ void __launch_bounds__(256) attn_mma_kernel(AttnParams p) {
 template <int HD>
 __global__ void attn_combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, int nsplit, int nrh,
                                     bf16 *__restrict__ out) {
+  pdl_wait();
+  pdl_trigger();
   int rh = blockIdx.x, d = threadIdx.x;
   const float sc = rsqrtf((float)HD) * 1.4426950408889634f;
   float M = -INFINITY;
@@ -290,12 +294,12 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
   static bool attr[2] = {false, false};
   if (hd == 128) {
     if (!attr[1]) { cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[1] = true; }
-    attn_mma_kernel<128><<<grid, 256, smem, s>>>(p);
-    if (nsplit > 1) attn_combine_kernel<128><<<rows * H, 128, 0, s>>>(p.part_o, p.part_ml, nsplit, rows * H, out);
+    launch_k(attn_mma_kernel<128>, grid, dim3(256), smem, s, p);
+    if (nsplit > 1) launch_k(attn_combine_kernel<128>, dim3(rows * H), dim3(128), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
   } else {
     if (!attr[0]) { cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[0] = true; }
-    attn_mma_kernel<64><<<grid, 256, smem, s>>>(p);
-    if (nsplit > 1) attn_combine_kernel<64><<<rows * H, 64, 0, s>>>(p.part_o, p.part_ml, nsplit, rows * H, out);
+    launch_k(attn_mma_kernel<64>, grid, dim3(256), smem, s, p);
+    if (nsplit > 1) launch_k(attn_combine_kernel<64>, dim3(rows * H), dim3(64), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
   }
   return nsplit > 1 ? 2 : 1;
 }

@@ -8,6 +8,8 @@ namespace spec {
 template <typename T>
 __global__ void __launch_bounds__(128) attn_ref_kernel(const T *__restrict__ q, KvPool pool, PageMap pm, RowMeta m,
                                                        int tail_len, T *__restrict__ out, int H, int G, int hd) {
+  pdl_wait();
+  pdl_trigger();
   extern __shared__ float smem[];
   float *qs = smem;            // [hd]
   float *sc = smem + hd;       // [ctx + tail_len]
@@ -86,7 +88,7 @@ void launch_attn_ref(const T *q, KvPool pool, PageMap pm, RowMeta m, int tail_le
     cudaFuncSetAttribute(attn_ref_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     configured[which] = smem;
   }
-  attn_ref_kernel<T><<<dim3(rows, H), 128, smem, s>>>(q, pool, pm, m, tail_len, out, H, G, hd);
+  launch_k(attn_ref_kernel<T>, dim3(rows, H), dim3(128), smem, s, q, pool, pm, m, tail_len, out, H, G, hd);
 }
 template void launch_attn_ref<float>(const float *, KvPool, PageMap, RowMeta, int, float *, int, int, int, int, int,
                                      cudaStream_t);

@@ -21,6 +21,28 @@ __device__ __forceinline__ void set_status(int32_t *st, int code, int where, int
   if (atomicCAS(st, 0, code) == 0) { st[1] = where; st[2] = a; st[3] = b; }
 }
 
+// Programmatic dependent launch: a kernel launched with the attribute may start while its predecessor
+// on the stream is still running; everything it reads that the predecessor wrote must come after
+// pdl_wait().  Both instructions do nothing in a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// When set (per host thread, by the step scheduler), launch_k adds the programmatic-dependent-launch
+// attribute to every launch.
+extern thread_local bool tl_pdl;
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = tl_pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // Per-row description of one forward pass (draft extend, draft tree pass, target verify).  A row
 // attends cache positions [0, ctx) unmasked, then "tail" positions tail_base + t for every set bit t
 // of (mask_lo, mask_hi); it writes its own K/V at cache position kvpos and is rotated by pos.
@@ -52,6 +74,10 @@ __device__ __forceinline__ size_t kv_offset(const PageMap &pm, int seq, int pos,
 // ---------------------------------------------------------------- launchers (elementwise.cu)
 template <typename T>
 void launch_embed(const T *embed, const int32_t *tok, float *x, int rows, int k, cudaStream_t s);
+
+// fused-path embedding: x = E[tok], hb = bf16(x * gain), ssq[tile][row] = per-128-feature sums of x^2
+void launch_embed_norm(const bf16 *embed, const int32_t *tok, const bf16 *gain, float *x, bf16 *hb, float *ssq, int rows,
+                       int k, int ssq_ld, cudaStream_t s);
 
 // x (+)= sum of `nparts` partial slices [nparts][rows][k]; optional taps (T, [rows][3k], slots by bitmask);
 // optional h[r] = rmsnorm(x[src_row ? src_row[r] : r]) * gain.  mode: 0 keep x, 1 x = parts, 2 x += parts.
@@ -89,5 +115,12 @@ size_t attn_ref_smem_bytes(int max_keys, int hd);
 // ---------------------------------------------------------------- launchers (tree.cu)
 void launch_logsoftmax_topk(const float *logits, int rows, int n, int K, int32_t *idx, float *lp, cudaStream_t s);
 void launch_argmax(const float *logits, int rows, int n, int32_t *idx, cudaStream_t s);
+// two-stage log-softmax + top-K (chunk candidates, then a per-row merge); scratch of topk_scratch_bytes
+size_t topk_scratch_bytes(int rows, int n, int K);
+int launch_topk2(const float *logits, const int32_t *src_row, int rows, int n, int K, int32_t *idx, float *lp, void *scratch,
+                 cudaStream_t s);
+// y[r] = best index over per-tile (value, index) candidates [tiles][ld]
+void launch_argmax_merge(const float *best_val, const int32_t *best_idx, int tiles, int ld, int rows, int32_t *out,
+                         cudaStream_t s);
 
 }  // namespace spec

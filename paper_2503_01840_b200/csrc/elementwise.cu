@@ -24,22 +24,51 @@ __device__ __forceinline__ float block_sum(float v, float *sh) {
 // ---------------------------------------------------------------- embedding gather
 template <typename T>
 __global__ void embed_kernel(const T *__restrict__ embed, const int32_t *__restrict__ tok, float *__restrict__ x, int k) {
+  pdl_wait();
+  pdl_trigger();
   int r = blockIdx.x;
   const T *e = embed + (size_t)tok[r] * k;
   for (int i = threadIdx.x; i < k; i += blockDim.x) x[(size_t)r * k + i] = to_f32(e[i]);
 }
 template <typename T>
 void launch_embed(const T *embed, const int32_t *tok, float *x, int rows, int k, cudaStream_t s) {
-  embed_kernel<T><<<rows, 256, 0, s>>>(embed, tok, x, k);
+  launch_k(embed_kernel<T>, dim3(rows), dim3(256), 0, s, embed, tok, x, k);
 }
 template void launch_embed<float>(const float *, const int32_t *, float *, int, int, cudaStream_t);
 template void launch_embed<bf16>(const bf16 *, const int32_t *, float *, int, int, cudaStream_t);
+
+// ---------------------------------------------------------------- embedding gather feeding the fused GEMM path
+// x = E[tok] (fp32 residual stream), hb = bf16(x * gain) (input of the first QKV GEMM, which applies
+// the RMSNorm factor as a row scale), ssq[tile][row] = sum of x^2 over the tile's 128 features.
+__global__ void embed_norm_kernel(const bf16 *__restrict__ embed, const int32_t *__restrict__ tok,
+                                  const bf16 *__restrict__ gain, float *__restrict__ x, bf16 *__restrict__ hb,
+                                  float *__restrict__ ssq, int k, int ssq_ld) {
+  __shared__ float sh[4];
+  int r = blockIdx.x, tile = blockIdx.y, o = tile * 128 + threadIdx.x;
+  float v = 0.0f;
+  if (o < k) {
+    v = __bfloat162float(embed[(size_t)tok[r] * k + o]);
+    x[(size_t)r * k + o] = v;
+    hb[(size_t)r * k + o] = __float2bfloat16_rn(v * __bfloat162float(gain[o]));
+  }
+  float sq = v * v;
+  for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = sq;
+  __syncthreads();
+  if (threadIdx.x == 0) ssq[(size_t)tile * ssq_ld + r] = ((sh[0] + sh[1]) + sh[2]) + sh[3];
+}
+void launch_embed_norm(const bf16 *embed, const int32_t *tok, const bf16 *gain, float *x, bf16 *hb, float *ssq, int rows,
+                       int k, int ssq_ld, cudaStream_t s) {
+  launch_k(embed_norm_kernel, dim3(rows, (k + 127) / 128), dim3(128), 0, s, embed, tok, gain, x, hb, ssq, k, ssq_ld);
+}
 
 // ---------------------------------------------------------------- partial-sum reduce + residual + RMSNorm (+ taps)
 template <typename T>
 __global__ void add_norm_kernel(float *__restrict__ x, const float *__restrict__ parts, int nparts, size_t part_stride,
                                 int mode, T *__restrict__ taps, int tap_mask, const T *__restrict__ gain, float eps,
                                 T *__restrict__ h, int k) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ float sh[32];
   int r = blockIdx.x;
   float *xr = x + (size_t)r * k;
@@ -67,7 +96,7 @@ void launch_add_norm(float *x, const float *parts, int nparts, size_t part_strid
                      const T *gain, float eps, T *h, const int32_t *src_row, int rows_x, int rows_h, int k,
                      cudaStream_t s) {
   (void)src_row; (void)rows_h;
-  add_norm_kernel<T><<<rows_x, 256, 0, s>>>(x, parts, nparts, part_stride, mode, tap_mask ? taps : nullptr, tap_mask,
+  launch_k(add_norm_kernel<T>, dim3(rows_x), dim3(256), 0, s, x, parts, nparts, part_stride, mode, tap_mask ? taps : nullptr, tap_mask,
                                            gain, eps, h, k);
 }
 template void launch_add_norm<float>(float *, const float *, int, size_t, int, float *, int, const float *, float,
@@ -78,6 +107,8 @@ template void launch_add_norm<bf16>(float *, const float *, int, size_t, int, bf
 // ---------------------------------------------------------------- RoPE angles (double, rounded once)
 __global__ void rope_table_kernel(const int32_t *__restrict__ pos, int rows, int half, const double *__restrict__ inv_freq,
                                   float2 *__restrict__ cs) {
+  pdl_wait();
+  pdl_trigger();
   int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= rows * half) return;
   int r = idx / half, i = idx % half;
@@ -88,7 +119,7 @@ __global__ void rope_table_kernel(const int32_t *__restrict__ pos, int rows, int
 }
 void launch_rope_table(const int32_t *pos, int rows, int half, const double *inv_freq, float2 *cs, cudaStream_t s) {
   int n = rows * half;
-  rope_table_kernel<<<(n + 255) / 256, 256, 0, s>>>(pos, rows, half, inv_freq, cs);
+  launch_k(rope_table_kernel, dim3((n + 255) / 256), dim3(256), 0, s, pos, rows, half, inv_freq, cs);
 }
 
 // ---------------------------------------------------------------- RoPE + q store + paged K/V write
@@ -96,6 +127,8 @@ template <typename T>
 __global__ void rope_kv_kernel(const float *__restrict__ qkv, int nparts, size_t part_stride,
                                const float2 *__restrict__ cs, RowMeta m, T *__restrict__ q, KvPool pool, PageMap pm,
                                int H, int G, int hd, int32_t *status) {
+  pdl_wait();
+  pdl_trigger();
   int r = blockIdx.x;
   int seq = m.seq[r];
   int half = hd / 2, ld = (H + 2 * G) * hd;
@@ -144,7 +177,7 @@ __global__ void rope_kv_kernel(const float *__restrict__ qkv, int nparts, size_t
 template <typename T>
 void launch_rope_kv(const float *qkv, int nparts, size_t part_stride, const float2 *cs, RowMeta m, T *q, KvPool pool,
                     PageMap pm, int rows, int H, int G, int hd, int32_t *status, cudaStream_t s) {
-  rope_kv_kernel<T><<<rows, 256, 0, s>>>(qkv, nparts, part_stride, cs, m, q, pool, pm, H, G, hd, status);
+  launch_k(rope_kv_kernel<T>, dim3(rows), dim3(256), 0, s, qkv, nparts, part_stride, cs, m, q, pool, pm, H, G, hd, status);
 }
 template void launch_rope_kv<float>(const float *, int, size_t, const float2 *, RowMeta, float *, KvPool, PageMap, int,
                                     int, int, int, int32_t *, cudaStream_t);
@@ -155,6 +188,8 @@ template void launch_rope_kv<bf16>(const float *, int, size_t, const float2 *, R
 template <typename T>
 __global__ void silu_mul_kernel(const float *__restrict__ gu, int nparts, size_t part_stride, T *__restrict__ act,
                                 int rows, int F) {
+  pdl_wait();
+  pdl_trigger();
   size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (size_t)rows * F) return;
   size_t r = idx / F, f = idx % F;
@@ -168,7 +203,7 @@ __global__ void silu_mul_kernel(const float *__restrict__ gu, int nparts, size_t
 template <typename T>
 void launch_silu_mul(const float *gu, int nparts, size_t part_stride, T *act, int rows, int F, cudaStream_t s) {
   size_t n = (size_t)rows * F;
-  silu_mul_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, s>>>(gu, nparts, part_stride, act, rows, F);
+  launch_k(silu_mul_kernel<T>, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, s, gu, nparts, part_stride, act, rows, F);
 }
 template void launch_silu_mul<float>(const float *, int, size_t, float *, int, int, cudaStream_t);
 template void launch_silu_mul<bf16>(const float *, int, size_t, bf16 *, int, int, cudaStream_t);
@@ -179,6 +214,8 @@ __global__ void build_cat_kernel(const float *__restrict__ feat, int nparts, siz
                                  const int32_t *__restrict__ src_row, const T *__restrict__ embed,
                                  const int32_t *__restrict__ tok, const int32_t *__restrict__ seq, T *__restrict__ cat,
                                  int k) {
+  pdl_wait();
+  pdl_trigger();
   int r = blockIdx.x;
   T *c = cat + (size_t)r * 2 * k;
   if (seq[r] < 0) {
@@ -197,7 +234,7 @@ __global__ void build_cat_kernel(const float *__restrict__ feat, int nparts, siz
 template <typename T>
 void launch_build_cat(const float *feat, int nparts, size_t part_stride, const int32_t *src_row, const T *embed,
                       const int32_t *tok, const int32_t *seq, T *cat, int rows, int k, cudaStream_t s) {
-  build_cat_kernel<T><<<rows, 256, 0, s>>>(feat, nparts, part_stride, src_row, embed, tok, seq, cat, k);
+  launch_k(build_cat_kernel<T>, dim3(rows), dim3(256), 0, s, feat, nparts, part_stride, src_row, embed, tok, seq, cat, k);
 }
 template void launch_build_cat<float>(const float *, int, size_t, const int32_t *, const float *, const int32_t *,
                                       const int32_t *, float *, int, int, cudaStream_t);

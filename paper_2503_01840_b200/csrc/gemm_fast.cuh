@@ -1,6 +1,8 @@
 // bf16 weight-streaming GEMM on the 5th-generation tensor cores (tcgen05.mma, TMEM accumulators,
 // TMA-staged operands): host-side interface.
 #pragma once
+#include <cuda.h>
+
 #include <string>
 #include "common.cuh"
 
@@ -10,6 +12,13 @@ struct FastGemm;   // caches TMA descriptors; one per context
 
 FastGemm *fast_gemm_create(std::string &why);
 void fast_gemm_destroy(FastGemm *);
+
+// Cached TMA descriptor of a bf16 matrix [outer][inner] (row pitch inner) with box [box_outer][64] and
+// 128-byte swizzle; nullptr if the driver rejects it.
+const CUtensorMap *fast_gemm_map(FastGemm *, const void *ptr, int outer, int inner, int box_outer);
+
+// drops every cached descriptor (buffers of one-shot callers come and go)
+void fast_gemm_forget(FastGemm *);
 
 // number of split-K slices for a [O][I] weight when at most smax slices fit the output buffer
 int fast_gemm_pick_split(int O, int I, int smax);

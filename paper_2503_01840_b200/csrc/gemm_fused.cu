@@ -1,0 +1,465 @@
+// Weight-streaming bf16 GEMM with fused epilogues for sm_100a.
+//
+//   out[r][o] = sum_i x[r][i] * w[o][i],  rows <= 256 token rows, weights far larger than the L2.
+//
+// The contraction is HBM-bound (every weight byte is read once per launch), so the kernel is built
+// around keeping many weight bytes in flight per SM and wasting no extra pass over the result:
+//
+//  * swap-AB mapping: the weight tile (128 output features x 64 k, K-major, 128-byte swizzle) is the
+//    UMMA M side, the token rows the N side (NT = 16/64/128/256), the fp32 accumulator sits in TMEM;
+//  * warp 0 streams tiles with TMA through a ring of shared-memory stages, warp 1 issues tcgen05.mma;
+//  * split-K: the S slices of one feature tile form a thread-block cluster.  Each CTA parks its
+//    accumulator in its own shared memory and every CTA reduces a share of the rows by reading its
+//    peers' copies through distributed shared memory, in slice order (deterministic, no atomics, no
+//    round trip of partial sums through global memory);
+//  * the epilogue that follows the reduction is the consumer's work: residual add + bf16 copy scaled
+//    by the next norm's gain + RMSNorm statistics (+ feature taps); RoPE + q store + paged K/V write;
+//    SiLU(gate)*up; per-tile argmax.  RMSNorm of the input is applied as a per-row scale in the
+//    epilogue (the normalisation factor is a row constant, so it commutes with the contraction);
+//  * programmatic dependent launch: the producer prefetches the first weight tiles (which never depend
+//    on the previous kernel) before griddepcontrol.wait, so the pipeline is full when the activations
+//    become valid.
+//
+// Every mbarrier wait is bounded; on timeout the CTA records it, skips its arithmetic, still takes part
+// in the cluster barriers (so its peers are not left waiting), frees its TMEM and exits.
+#include <cuda.h>
+#include <stdio.h>
+
+#include <algorithm>
+
+#include "gemm_fused.cuh"
+#include "tcgen05_ptx.cuh"
+
+namespace spec {
+
+namespace {
+
+using namespace tc;
+
+constexpr int MAX_STAGES = 16;
+constexpr int CHUNK = 64;                       // rows reduced per epilogue round
+constexpr int A_BYTES = TILE_M * TILE_K * 2;    // one weight tile of a stage
+
+struct alignas(64) FusedParams {
+  CUtensorMap map_w[3];
+  CUtensorMap map_x;
+  int tiles0, tiles1;          // tile index ranges of the weights: [0,tiles0) w0, [tiles0,tiles1) w1, rest w2
+  int O[3];
+  int rows, KB, S, stages, ctrl_off;
+  const float *ssq_in; int ssq_in_tiles, ssq_ld; float inv_k_in, eps;
+  float *out_f32; int ldo;
+  float *xres; const bf16 *gain; bf16 *hb; float *ssq_out; bf16 *taps; int tap_mask, resid_add;
+  const float2 *cs; RowMeta m; bf16 *q; KvPool pool; PageMap pm; int H, G, hd;
+  bf16 *act;
+  float *best_val; int32_t *best_idx; int best_ld;
+  int32_t *status;
+};
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_peer(uint32_t local_addr, uint32_t rank) {
+  uint32_t ra;
+  float v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+  return v;
+}
+
+template <int NT, int EPI>
+__global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__ FusedParams p) {
+  constexpr bool PAIR = (EPI == EPI_SWIGLU);
+  constexpr int NA = PAIR ? 2 : 1;
+  constexpr int B_BYTES = NT * TILE_K * 2;
+  constexpr int STAGE = NA * A_BYTES + B_BYTES;
+  constexpr int TMEM_COLS = (NA * NT < 32) ? 32 : NA * NT;
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char *tiles = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  unsigned char *ctrl = tiles + p.ctrl_off;
+  uint64_t *full = (uint64_t *)ctrl;
+  uint64_t *empty = full + MAX_STAGES;
+  uint64_t *acc_bar = empty + MAX_STAGES;
+  uint32_t *tmem_slot = (uint32_t *)(acc_bar + 1);
+  volatile uint32_t *abort_flag = tmem_slot + 1;
+  float *inv_s = (float *)(ctrl + 512);          // [256] per-row input scale
+  float *wpart = inv_s + 256;                    // [4][CHUNK] per-warp partial sums / argmax exchange
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int stages = p.stages, S = p.S;
+  const int slice = (S > 1) ? (int)cluster_rank() : 0;
+  const int kb0 = (int)(((long long)slice * p.KB) / S), kb1 = (int)(((long long)(slice + 1) * p.KB) / S);
+  const int nkb = kb1 - kb0;
+  int mi = 0, tm = blockIdx.x;                   // weight index and tile within that weight
+  if (!PAIR) {
+    if (tm >= p.tiles1) { mi = 2; tm -= p.tiles1; }
+    else if (tm >= p.tiles0) { mi = 1; tm -= p.tiles0; }
+  }
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < stages; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    mbar_init(acc_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {   // TMEM allocation is a whole-warp operation
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_trigger();
+
+  if (warp == 0 && lane == 0) {
+    // ---- producer.  Weight tiles do not depend on the previous kernel: fill the ring with them first.
+    const CUtensorMap *mw0 = &p.map_w[PAIR ? 0 : mi];
+    const int npre = nkb < stages ? nkb : stages;
+    for (int i = 0; i < npre; i++) {
+      unsigned char *a = tiles + i * STAGE;
+      mbar_expect_tx(&full[i], STAGE);
+      tma_load_2d(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[i]);
+      if (PAIR) tma_load_2d(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[i]);
+    }
+    pdl_wait();
+    for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + NA * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
+    for (int i = npre; i < nkb; i++) {
+      int st = i % stages;
+      if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
+      if (*abort_flag) break;
+      unsigned char *a = tiles + st * STAGE;
+      mbar_expect_tx(&full[st], STAGE);
+      tma_load_2d(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[st]);
+      if (PAIR) tma_load_2d(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[st]);
+      tma_load_2d(a + NA * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[st]);
+    }
+  } else {
+    pdl_wait();
+    if (warp == 1 && lane == 0) {
+      // ---- MMA issuer
+      constexpr uint32_t idesc = umma_idesc(NT);
+      for (int i = 0; i < nkb; i++) {
+        int st = i % stages;
+        if (!mbar_wait(&full[st], (i / stages) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 201, blockIdx.x, i); break; }
+        if (*abort_flag) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        uint32_t a = smem_u32(tiles + st * STAGE), b = a + NA * A_BYTES;
+#pragma unroll
+        for (int j = 0; j < TILE_K / UMMA_K; j++) {
+          uint64_t db = umma_desc_sw128(b + j * UMMA_K * 2);
+          umma_bf16(tmem_base, umma_desc_sw128(a + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
+          if (PAIR) umma_bf16(tmem_base + NT, umma_desc_sw128(a + A_BYTES + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
+        }
+        umma_commit(&empty[st]);      // frees the stage once these MMAs have read it
+      }
+      umma_commit(acc_bar);           // accumulator complete
+    } else if (warp >= 2) {
+      // ---- per-row scale of the input: rsqrt(mean square + eps) from the producer kernel's per-tile sums
+      for (int r = threadIdx.x - 64; r < p.rows; r += 64) {
+        float sc = 1.0f;
+        if (p.ssq_in) {
+          float ss = 0.0f;
+          for (int t = 0; t < p.ssq_in_tiles; t++) ss += p.ssq_in[(size_t)t * p.ssq_ld + r];
+          sc = 1.0f / sqrtf(ss * p.inv_k_in + p.eps);
+        }
+        inv_s[r] = sc;
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- wait for the accumulator (one bounded wait per warp)
+  int good = 0;
+  if (lane == 0) {
+    bool ok = mbar_wait(acc_bar, 0);
+    if (!ok) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 202, blockIdx.x, slice); }
+    good = (ok && !*abort_flag) ? 1 : 0;
+  }
+  good = __shfl_sync(0xffffffffu, good, 0);
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+  // ---- epilogue, CHUNK rows at a time.  The stage ring is free now (every load landed, every MMA that
+  // read it completed) and is reused: red = this CTA's accumulator(s), sumb = reduced rows (EPI_QKV).
+  float *red = (float *)tiles;                       // [NA][CHUNK][128]
+  float *sumb = red + NA * CHUNK * TILE_M;           // [CHUNK][128]
+  const int f = threadIdx.x;
+  const int o = tm * TILE_M + f;                     // output feature within weight mi
+  for (int c0 = 0; c0 < p.rows; c0 += CHUNK) {
+    const int nrow = (p.rows - c0 < CHUNK) ? p.rows - c0 : CHUNK;
+    if (good) {
+#pragma unroll
+      for (int a = 0; a < NA; a++) {
+#pragma unroll 1
+        for (int cc = 0; cc < CHUNK && c0 + cc < NT; cc += 16) {
+          if (cc >= nrow) break;
+          uint32_t v[16];
+          tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(a * NT + c0 + cc), v);
+#pragma unroll
+          for (int j = 0; j < 16; j++) red[(a * CHUNK + cc + j) * TILE_M + f] = __uint_as_float(v[j]);
+        }
+      }
+    }
+    if (S > 1) cluster_sync_all(); else __syncthreads();
+    const int per = (nrow + S - 1) / S;
+    const int r0 = slice * per, r1 = (r0 + per < nrow) ? r0 + per : nrow;
+
+    if (EPI == EPI_F32 || EPI == EPI_RESID || EPI == EPI_QKV) {
+      for (int r = r0; r < r1; r++) {
+        float v = 0.0f;
+        if (S > 1) {
+          uint32_t la = smem_u32(&red[r * TILE_M + f]);
+          for (int s = 0; s < S; s++) v += ld_peer(la, (uint32_t)s);
+        } else {
+          v = red[r * TILE_M + f];
+        }
+        const int row = c0 + r;
+        if (EPI == EPI_F32) {
+          if (good && o < p.O[0]) p.out_f32[(size_t)row * p.ldo + o] = v * inv_s[row];
+        } else if (EPI == EPI_RESID) {
+          float xo = 0.0f;
+          if (good && o < p.O[0]) {
+            size_t xi = (size_t)row * p.O[0] + o;
+            xo = (p.resid_add ? p.xres[xi] : 0.0f) + v;
+            p.xres[xi] = xo;
+            p.hb[xi] = __float2bfloat16_rn(xo * __bfloat162float(p.gain[o]));
+            if (p.tap_mask) {
+#pragma unroll
+              for (int s = 0; s < 3; s++)
+                if ((p.tap_mask >> s) & 1) p.taps[(size_t)row * 3 * p.O[0] + (size_t)s * p.O[0] + o] = __float2bfloat16_rn(xo);
+            }
+          }
+          float sq = xo * xo;
+          for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+          if (lane == 0) wpart[warp * CHUNK + (r - r0)] = sq;
+        } else {
+          sumb[r * TILE_M + f] = v * inv_s[row];
+        }
+      }
+      if (EPI == EPI_RESID) {
+        __syncthreads();
+        if (good && threadIdx.x < r1 - r0) {
+          int t = threadIdx.x;
+          p.ssq_out[(size_t)tm * p.ssq_ld + c0 + r0 + t] =
+              ((wpart[t] + wpart[CHUNK + t]) + wpart[2 * CHUNK + t]) + wpart[3 * CHUNK + t];
+        }
+      }
+      if (EPI == EPI_QKV) {
+        __syncthreads();
+        const int hd = p.hd, half = hd >> 1;
+        const int head = o / hd, i = o % hd;
+        const bool valid_o = o < p.O[mi];
+        bf16 *Kp = (bf16 *)p.pool.k, *Vp = (bf16 *)p.pool.v;
+        for (int r = r0; r < r1; r++) {
+          const int row = c0 + r;
+          const int seq = p.m.seq[row];
+          if (!valid_o || !good) continue;
+          float v = sumb[r * TILE_M + f];
+          if (mi < 2) {                             // rotate-half RoPE: partner feature is f ^ half
+            float w = sumb[r * TILE_M + (f ^ half)];
+            float2 c = p.cs[(size_t)row * half + (i & (half - 1))];
+            v = (i < half) ? v * c.x - w * c.y : v * c.x + w * c.y;
+          }
+          if (mi == 0) {
+            p.q[((size_t)row * p.H + head) * hd + i] = __float2bfloat16_rn(seq < 0 ? 0.0f : v);
+          } else if (seq >= 0) {
+            const int kvpos = p.m.kvpos[row];
+            if (kvpos < 0 || kvpos / p.pm.page_size >= p.pm.pages_per_seq) {
+              if (f == 0) set_status(p.status, ST_BOUNDS, 1, row, kvpos);
+              continue;
+            }
+            const int page = p.pm.table[(size_t)seq * p.pm.pages_per_seq + kvpos / p.pm.page_size];
+            if (page < 0 || page >= p.pm.num_pages) {
+              if (f == 0) set_status(p.status, ST_BOUNDS, 2, row, page);
+              continue;
+            }
+            size_t off = (((size_t)page * p.G + head) * p.pm.page_size + (kvpos % p.pm.page_size)) * hd + i;
+            (mi == 1 ? Kp : Vp)[off] = __float2bfloat16_rn(v);
+          }
+        }
+      }
+    } else if (EPI == EPI_SWIGLU) {
+      if (good && o < p.O[0]) {
+        for (int r = r0; r < r1; r++) {
+          const int row = c0 + r;
+          float sc = inv_s[row];
+          float g = red[r * TILE_M + f] * sc, u = red[(CHUNK + r) * TILE_M + f] * sc;
+          p.act[(size_t)row * p.O[0] + o] = __float2bfloat16_rn((g / (1.0f + expf(-g))) * u);
+        }
+      }
+    } else {   // EPI_ARGMAX
+      if (good && p.out_f32 && o < p.O[0])
+        for (int r = r0; r < r1; r++) p.out_f32[(size_t)(c0 + r) * p.ldo + o] = red[r * TILE_M + f] * inv_s[c0 + r];
+      // thread t scans half of the tile's features for row t % 64, starting at a row-dependent feature
+      // so that the 32 rows of a warp touch 32 different banks
+      const int row = threadIdx.x & (CHUNK - 1), hf = threadIdx.x >> 6;
+      float bv = 0.0f;
+      int bi = -1;
+      if (row < nrow) {
+        for (int j = 0; j < 64; j++) {
+          int ff = hf * 64 + ((j + row) & 63), oo = tm * TILE_M + ff;
+          float v = red[row * TILE_M + ff];
+          if (oo < p.O[0] && (bi < 0 || v > bv || (v == bv && oo < bi))) { bv = v; bi = oo; }
+        }
+      }
+      if (hf == 1) { wpart[row] = bv; wpart[CHUNK + row] = __int_as_float(bi); }
+      __syncthreads();
+      if (hf == 0 && row < nrow && good) {
+        float ov = wpart[row];
+        int oi = __float_as_int(wpart[CHUNK + row]);
+        if (oi >= 0 && (bi < 0 || ov > bv || (ov == bv && oi < bi))) { bv = ov; bi = oi; }
+        p.best_val[(size_t)blockIdx.x * p.best_ld + c0 + row] = bv;
+        p.best_idx[(size_t)blockIdx.x * p.best_ld + c0 + row] = bi;
+      }
+    }
+    // peers may still be reading this CTA's red; nobody overwrites or leaves before all are done
+    if (S > 1) cluster_sync_all(); else __syncthreads();
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- host side
+int pick_nt(int rows) { return rows <= 16 ? 16 : rows <= 64 ? 64 : rows <= 128 ? 128 : 256; }
+
+constexpr int NUM_SMS = 148;
+constexpr int SMEM_ONE = 200 * 1024;      // ring budget with one CTA per SM
+constexpr int SMEM_TWO = 104 * 1024;      // ring budget that lets two CTAs share an SM
+
+struct Plan { int nt, tiles, S, stages, smem, ctrl_off, KB; };
+
+Plan make_plan(FusedEpi epi, const FusedGemmArgs &a) {
+  Plan pl;
+  const bool pair = epi == EPI_SWIGLU;
+  pl.nt = pick_nt(a.rows);
+  pl.KB = (a.I + TILE_K - 1) / TILE_K;
+  pl.tiles = fused_gemm_tiles(epi, a);
+  const int stage = (pair ? 2 : 1) * A_BYTES + pl.nt * TILE_K * 2;
+  int S = 1;
+  if (epi == EPI_F32 || epi == EPI_RESID || epi == EPI_QKV) {
+    S = std::max(1, std::min(8, NUM_SMS / std::max(1, pl.tiles)));
+    S = std::max(1, std::min(S, pl.KB / 4));
+  }
+  if (a.split > 0) S = std::min(std::min(a.split, 8), pl.KB);
+  if (epi == EPI_SWIGLU || epi == EPI_ARGMAX) S = 1;
+  pl.S = S;
+  int budget = SMEM_ONE;
+  if (pl.tiles * S > NUM_SMS && SMEM_TWO / stage >= 3) budget = SMEM_TWO;   // several waves: let two CTAs overlap
+  int stages = std::max(2, std::min(MAX_STAGES, budget / stage));
+  if (a.stages > 0) stages = std::max(2, std::min(std::min(a.stages, MAX_STAGES), (220 * 1024) / stage));
+  int per_slice = (pl.KB + S - 1) / S;
+  stages = std::max(2, std::min(stages, per_slice));
+  pl.stages = stages;
+  const int epi_bytes = ((pair ? 2 : 1) * CHUNK * TILE_M + (epi == EPI_QKV ? CHUNK * TILE_M : 0)) * 4;
+  pl.ctrl_off = (std::max(stages * stage, epi_bytes) + 1023) & ~1023;
+  pl.smem = pl.ctrl_off + 512 + 256 * 4 + 4 * CHUNK * 4 + 1024 /*alignment slack*/;
+  return pl;
+}
+
+template <int NT, int EPI>
+int launch_inst(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) {
+  static int configured = 0;
+  if (pl.smem > configured) {
+    if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem) != cudaSuccess) return -6;
+    configured = pl.smem;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(pl.tiles, pl.S, 1);
+  cfg.blockDim = dim3(128, 1, 1);
+  cfg.dynamicSmemBytes = pl.smem;
+  cfg.stream = s;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  if (pl.S > 1) {
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = 1; at[na].val.clusterDim.y = pl.S; at[na].val.clusterDim.z = 1;
+    na++;
+  }
+  if (pdl) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    na++;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = na;
+  return cudaLaunchKernelEx(&cfg, gemm_fused_kernel<NT, EPI>, p) == cudaSuccess ? 0 : -6;
+}
+
+template <int EPI>
+int launch_epi(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) {
+  switch (pl.nt) {
+    case 16: return launch_inst<16, EPI>(p, pl, pdl, s);
+    case 64: return launch_inst<64, EPI>(p, pl, pdl, s);
+    case 128: return launch_inst<128, EPI>(p, pl, pdl, s);
+    default: return launch_inst<256, EPI>(p, pl, pdl, s);
+  }
+}
+
+}  // namespace
+
+int fused_gemm_tiles(FusedEpi epi, const FusedGemmArgs &a) {
+  if (epi == EPI_SWIGLU) return (a.O[0] + TILE_M - 1) / TILE_M;
+  int t = 0;
+  for (int j = 0; j < a.nw; j++) t += (a.O[j] + TILE_M - 1) / TILE_M;
+  return t;
+}
+
+bool fused_gemm_supported(FusedEpi epi, const FusedGemmArgs &a) {
+  if (a.rows < 1 || a.rows > 256 || a.I < 8 || (a.I % 8) != 0 || ((uintptr_t)a.x & 15)) return false;
+  int need = epi == EPI_QKV ? 3 : epi == EPI_SWIGLU ? 2 : 1;
+  if (a.nw != need) return false;
+  for (int j = 0; j < a.nw; j++)
+    if (!a.w[j] || ((uintptr_t)a.w[j] & 15) || a.O[j] < 1) return false;
+  if (epi == EPI_SWIGLU && a.O[0] != a.O[1]) return false;
+  if (epi == EPI_QKV) {
+    if (a.hd < 2 || a.hd > TILE_M || (a.hd & (a.hd - 1))) return false;
+    if (a.O[0] != a.H * a.hd || a.O[1] != a.G * a.hd || a.O[2] != a.G * a.hd) return false;
+  }
+  return true;
+}
+
+int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStream_t s) {
+  if (!g || !fused_gemm_supported(epi, a)) return -1;
+  Plan pl = make_plan(epi, a);
+  FusedParams p;
+  memset(&p, 0, sizeof p);
+  for (int j = 0; j < a.nw; j++) {
+    const CUtensorMap *mw = fast_gemm_map(g, a.w[j], a.O[j], a.I, TILE_M);
+    if (!mw) return -6;
+    p.map_w[j] = *mw;
+    p.O[j] = a.O[j];
+  }
+  const CUtensorMap *mx = fast_gemm_map(g, a.x, a.rows, a.I, pl.nt);
+  if (!mx) return -6;
+  p.map_x = *mx;
+  p.tiles0 = (a.O[0] + TILE_M - 1) / TILE_M;
+  p.tiles1 = p.tiles0 + (a.nw > 1 ? (a.O[1] + TILE_M - 1) / TILE_M : 0);
+  p.rows = a.rows; p.KB = pl.KB; p.S = pl.S; p.stages = pl.stages; p.ctrl_off = pl.ctrl_off;
+  p.ssq_in = a.ssq_in; p.ssq_in_tiles = a.ssq_in_tiles; p.ssq_ld = a.ssq_ld; p.inv_k_in = 1.0f / (float)a.k_in; p.eps = a.eps;
+  p.out_f32 = a.out_f32; p.ldo = a.ldo;
+  p.xres = a.xres; p.gain = a.gain; p.hb = a.hb; p.ssq_out = a.ssq_out; p.taps = a.tap_mask ? a.taps : nullptr;
+  p.tap_mask = a.taps ? a.tap_mask : 0; p.resid_add = a.resid_add;
+  p.cs = a.cs; p.m = a.m; p.q = a.q; p.pool = a.pool; p.pm = a.pm; p.H = a.H; p.G = a.G; p.hd = a.hd;
+  p.act = a.act;
+  p.best_val = a.best_val; p.best_idx = a.best_idx; p.best_ld = a.best_ld;
+  p.status = a.status;
+  switch (epi) {
+    case EPI_F32: return launch_epi<EPI_F32>(p, pl, a.pdl, s);
+    case EPI_RESID: return launch_epi<EPI_RESID>(p, pl, a.pdl, s);
+    case EPI_QKV: return launch_epi<EPI_QKV>(p, pl, a.pdl, s);
+    case EPI_SWIGLU: return launch_epi<EPI_SWIGLU>(p, pl, a.pdl, s);
+    default: return launch_epi<EPI_ARGMAX>(p, pl, a.pdl, s);
+  }
+}
+
+}  // namespace spec

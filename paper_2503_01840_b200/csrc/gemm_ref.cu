@@ -8,6 +8,8 @@ namespace spec {
 template <typename T>
 __global__ void __launch_bounds__(256) gemm_ref_kernel(const T *__restrict__ x, const T *__restrict__ w,
                                                        float *__restrict__ out, int rows, int O, int I, int ldo) {
+  pdl_wait();
+  pdl_trigger();
   constexpr int BM = 64, BN = 64, BK = 16;
   __shared__ float xs[BK][BM + 1];
   __shared__ float ws[BK][BN + 1];
@@ -56,7 +58,7 @@ __global__ void __launch_bounds__(256) gemm_ref_kernel(const T *__restrict__ x, 
 template <typename T>
 void launch_gemm_ref(const T *x, const T *w, float *out, int rows, int O, int I, int ldo, cudaStream_t s) {
   dim3 grid((O + 63) / 64, (rows + 63) / 64);
-  gemm_ref_kernel<T><<<grid, 256, 0, s>>>(x, w, out, rows, O, I, ldo);
+  launch_k(gemm_ref_kernel<T>, dim3(grid), dim3(256), 0, s, x, w, out, rows, O, I, ldo);
 }
 template void launch_gemm_ref<float>(const float *, const float *, float *, int, int, int, int, cudaStream_t);
 template void launch_gemm_ref<bf16>(const bf16 *, const bf16 *, float *, int, int, int, int, cudaStream_t);

@@ -36,6 +36,8 @@ __device__ __forceinline__ VI block_best(VI x, VI *sh) {
 }
 
 __global__ void __launch_bounds__(256) argmax_kernel(const float *__restrict__ logits, int n, int32_t *__restrict__ out) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ VI sh[32];
   const float *z = logits + (size_t)blockIdx.x * n;
   VI b{0.0f, -1};
@@ -47,13 +49,15 @@ __global__ void __launch_bounds__(256) argmax_kernel(const float *__restrict__ l
   if (threadIdx.x == 0) out[blockIdx.x] = b.i;
 }
 void launch_argmax(const float *logits, int rows, int n, int32_t *idx, cudaStream_t s) {
-  argmax_kernel<<<rows, 256, 0, s>>>(logits, n, idx);
+  launch_k(argmax_kernel, dim3(rows), dim3(256), 0, s, logits, n, idx);
 }
 
 // log-softmax + top-K, (value desc, index asc).  Row r reads logits row src_row[r] when given.
 __global__ void __launch_bounds__(256) logsoftmax_topk_kernel(const float *__restrict__ logits, const int32_t *src_row,
                                                               int n, int K, int32_t *__restrict__ idx,
                                                               float *__restrict__ lp) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ VI sh[32];
   __shared__ float shf[32];
   int r = blockIdx.x;
@@ -95,16 +99,172 @@ __global__ void __launch_bounds__(256) logsoftmax_topk_kernel(const float *__res
   }
 }
 void launch_logsoftmax_topk(const float *logits, int rows, int n, int K, int32_t *idx, float *lp, cudaStream_t s) {
-  logsoftmax_topk_kernel<<<rows, 256, 0, s>>>(logits, nullptr, n, K, idx, lp);
+  launch_k(logsoftmax_topk_kernel, dim3(rows), dim3(256), 0, s, logits, nullptr, n, K, idx, lp);
 }
 void launch_logsoftmax_topk_rows(const float *logits, const int32_t *src_row, int rows, int n, int K, int32_t *idx,
                                  float *lp, cudaStream_t s) {
-  logsoftmax_topk_kernel<<<rows, 256, 0, s>>>(logits, src_row, n, K, idx, lp);
+  launch_k(logsoftmax_topk_kernel, dim3(rows), dim3(256), 0, s, logits, src_row, n, K, idx, lp);
+}
+
+
+// ---------------------------------------------------------------- two-stage log-softmax + top-K
+// Stage 1: one CTA per (row, chunk of TOPK_CHUNK logits): chunk maximum, sum of exp relative to it, and
+// the chunk's K best (value desc, index asc).  Stage 2: one CTA per row merges the chunks: log-sum-exp
+// of the row and the K best of the chunk candidates, ranked by counting.
+constexpr int TOPK_CHUNK = 1024;
+constexpr int TOPK_MAXK = 16;
+
+__global__ void __launch_bounds__(256) topk_partial_kernel(const float *__restrict__ logits, const int32_t *src_row, int n,
+                                                           int K, int nch, float *__restrict__ pmax,
+                                                           float *__restrict__ psum, float *__restrict__ cval,
+                                                           int32_t *__restrict__ cidx) {
+  pdl_wait();
+  pdl_trigger();
+  __shared__ VI sh[32];
+  __shared__ float shf[32];
+  int r = blockIdx.y, ch = blockIdx.x;
+  int sr = src_row ? src_row[r] : r;
+  if (sr < 0) return;
+  const float *z = logits + (size_t)sr * n;
+  int base = ch * TOPK_CHUNK;
+  float v[4];
+  int id[4];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < 4; j++) {
+    id[j] = base + j * 256 + threadIdx.x;
+    v[j] = id[j] < n ? z[id[j]] : -INFINITY;
+    if (id[j] >= n) id[j] = -1;
+    mx = fmaxf(mx, v[j]);
+  }
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  mx = shf[0];
+  for (int w = 1; w < 8; w++) mx = fmaxf(mx, shf[w]);
+  __syncthreads();
+  float sum = 0.0f;
+#pragma unroll
+  for (int j = 0; j < 4; j++) sum += id[j] >= 0 ? expf(v[j] - mx) : 0.0f;
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.0f;
+    for (int w = 0; w < 8; w++) t += shf[w];
+    pmax[(size_t)r * nch + ch] = mx;
+    psum[(size_t)r * nch + ch] = t;
+  }
+  for (int c = 0; c < K; c++) {
+    VI b{0.0f, -1};
+#pragma unroll
+    for (int j = 0; j < 4; j++)
+      if (id[j] >= 0 && (b.i < 0 || before(v[j], id[j], b.v, b.i))) { b.v = v[j]; b.i = id[j]; }
+    b = block_best(b, sh);
+#pragma unroll
+    for (int j = 0; j < 4; j++)
+      if (id[j] == b.i) id[j] = -1;           // taken (b.i is -1 only when the chunk is exhausted)
+    if (threadIdx.x == 0) {
+      cval[((size_t)r * nch + ch) * K + c] = b.v;
+      cidx[((size_t)r * nch + ch) * K + c] = b.i;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) topk_merge_kernel(const int32_t *src_row, int K, int nch, const float *__restrict__ pmax,
+                                                         const float *__restrict__ psum, const float *__restrict__ cval,
+                                                         const int32_t *__restrict__ cidx, int32_t *__restrict__ idx,
+                                                         float *__restrict__ lp) {
+  pdl_wait();
+  pdl_trigger();
+  extern __shared__ unsigned char smraw[];
+  __shared__ float shf[32];
+  int r = blockIdx.x;
+  int sr = src_row ? src_row[r] : r;
+  if (sr < 0) {
+    for (int c = threadIdx.x; c < K; c += blockDim.x) { idx[(size_t)r * K + c] = 0; lp[(size_t)r * K + c] = 0.0f; }
+    return;
+  }
+  int nc = nch * K;
+  float *cv = (float *)smraw;              // [nc]
+  int32_t *ci = (int32_t *)(cv + nc);      // [nc]
+  for (int i = threadIdx.x; i < nc; i += blockDim.x) { cv[i] = cval[(size_t)r * nc + i]; ci[i] = cidx[(size_t)r * nc + i]; }
+  float mx = -INFINITY;
+  for (int i = threadIdx.x; i < nch; i += blockDim.x) mx = fmaxf(mx, pmax[(size_t)r * nch + i]);
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = mx;
+  __syncthreads();
+  mx = shf[0];
+  for (int w = 1; w < 8; w++) mx = fmaxf(mx, shf[w]);
+  __syncthreads();
+  // chunk sums are combined in chunk order by one thread: the result does not depend on the launch shape
+  if (threadIdx.x == 0) {
+    float t = 0.0f;
+    for (int i = 0; i < nch; i++) t += psum[(size_t)r * nch + i] * expf(pmax[(size_t)r * nch + i] - mx);
+    shf[0] = logf(t);
+  }
+  __syncthreads();
+  float lse = shf[0];
+  for (int i = threadIdx.x; i < nc; i += blockDim.x) {
+    int my = ci[i];
+    if (my < 0) continue;
+    float v = cv[i];
+    int rank = 0;
+    for (int j = 0; j < nc; j++) rank += (ci[j] >= 0 && before(cv[j], ci[j], v, my)) ? 1 : 0;
+    if (rank < K) { idx[(size_t)r * K + rank] = my; lp[(size_t)r * K + rank] = (v - mx) - lse; }
+  }
+}
+
+size_t topk_scratch_bytes(int rows, int n, int K) {
+  size_t nch = (size_t)(n + TOPK_CHUNK - 1) / TOPK_CHUNK;
+  return (size_t)rows * nch * (2 + 2 * (size_t)K) * 4 + 256;
+}
+
+// scratch: topk_scratch_bytes(rows, n, K) bytes.  Returns the number of kernels launched.
+int launch_topk2(const float *logits, const int32_t *src_row, int rows, int n, int K, int32_t *idx, float *lp, void *scratch,
+                 cudaStream_t s) {
+  int nch = (n + TOPK_CHUNK - 1) / TOPK_CHUNK;
+  float *pmax = (float *)scratch;
+  float *psum = pmax + (size_t)rows * nch;
+  float *cval = psum + (size_t)rows * nch;
+  int32_t *cidx = (int32_t *)(cval + (size_t)rows * nch * K);
+  launch_k(topk_partial_kernel, dim3(nch, rows), dim3(256), 0, s, logits, src_row, n, K, nch, pmax, psum, cval, cidx);
+  size_t smem = (size_t)nch * K * 8;
+  static size_t configured = 0;
+  if (smem > 48 * 1024 && smem > configured) {
+    cudaFuncSetAttribute(topk_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    configured = smem;
+  }
+  launch_k(topk_merge_kernel, dim3(rows), dim3(256), smem, s, src_row, K, nch, pmax, psum, cval, cidx, idx, lp);
+  return 2;
+}
+
+// ---------------------------------------------------------------- argmax over per-tile candidates
+// y[r] = index of the best (value desc, index asc) of best_val/best_idx[t][r], t < tiles.
+__global__ void __launch_bounds__(256) argmax_merge_kernel(const float *__restrict__ best_val, const int32_t *__restrict__ best_idx,
+                                                           int tiles, int ld, int32_t *__restrict__ out) {
+  pdl_wait();
+  pdl_trigger();
+  __shared__ VI sh[32];
+  int r = blockIdx.x;
+  VI b{0.0f, -1};
+  for (int t = threadIdx.x; t < tiles; t += blockDim.x) {
+    float v = best_val[(size_t)t * ld + r];
+    int i = best_idx[(size_t)t * ld + r];
+    if (i >= 0 && (b.i < 0 || before(v, i, b.v, b.i))) { b.v = v; b.i = i; }
+  }
+  b = block_best(b, sh);
+  if (threadIdx.x == 0) out[r] = b.i;
+}
+void launch_argmax_merge(const float *best_val, const int32_t *best_idx, int tiles, int ld, int rows, int32_t *out, cudaStream_t s) {
+  launch_k(argmax_merge_kernel, dim3(rows), dim3(256), 0, s, best_val, best_idx, tiles, ld, out);
 }
 
 // ---------------------------------------------------------------- step set-up: rows of the extend pass
 // Row b*Pmax + j is pending entry j of sequence b: position n-P+j, causal among the pending rows.
 __global__ void prep_extend_kernel(SeqState st, TreeBufs tb, RowMeta m, int need_positions, int32_t *status) {
+  pdl_wait();
+  pdl_trigger();
   int b = blockIdx.x, j = threadIdx.x;
   int n = st.n[b], P = st.P[b];
   bool ok = (n + need_positions <= st.cap[b]) && P >= 1 && P <= tb.Pmax;
@@ -132,7 +292,7 @@ __global__ void prep_extend_kernel(SeqState st, TreeBufs tb, RowMeta m, int need
 }
 void launch_prep_extend(SeqState st, TreeBufs tb, RowMeta m, int B, int need_positions, int32_t *status, cudaStream_t s) {
   int threads = ((tb.Pmax + 31) / 32) * 32;
-  prep_extend_kernel<<<B, threads, 0, s>>>(st, tb, m, need_positions, status);
+  launch_k(prep_extend_kernel, dim3(B), dim3(threads), 0, s, st, tb, m, need_positions, status);
 }
 
 // ---------------------------------------------------------------- dynamic-tree expansion after draft pass `pass` (1-based)
@@ -140,6 +300,8 @@ void launch_prep_extend(SeqState st, TreeBufs tb, RowMeta m, int B, int need_pos
 // best of the level) and writes the row metadata of the next draft pass.
 __global__ void __launch_bounds__(256) expand_kernel(SeqState st, TreeBufs tb, RowMeta m, const int32_t *__restrict__ d2t,
                                                      int pass) {
+  pdl_wait();
+  pdl_trigger();
   extern __shared__ unsigned char smraw[];
   int K = tb.K, D = tb.D, b = blockIdx.x;
   int nch = (pass == 1) ? K : K * K;        // children created by this pass
@@ -205,13 +367,15 @@ __global__ void __launch_bounds__(256) expand_kernel(SeqState st, TreeBufs tb, R
 void launch_expand(SeqState st, TreeBufs tb, RowMeta m, const int32_t *d2t, int pass, int B, cudaStream_t s) {
   int K = tb.K, nch = K * K;
   size_t smem = (size_t)((nch + 1) & ~1) * 4 + (size_t)K * 16 + (size_t)K * 4 + 16;
-  expand_kernel<<<B, 256, smem, s>>>(st, tb, m, d2t, pass);
+  launch_k(expand_kernel, dim3(B), dim3(256), smem, s, st, tb, m, d2t, pass);
 }
 
 // ---------------------------------------------------------------- pruning + tree assembly
 // Keeps the M = min(N-1, pool) best candidates (score desc, pool index asc), numbers them in pool
 // order after the root and emits parents, depths, ancestor-or-self bit masks and the verify rows.
 __global__ void __launch_bounds__(256) rerank_kernel(SeqState st, TreeBufs tb, RowMeta m) {
+  pdl_wait();
+  pdl_trigger();
   extern __shared__ unsigned char smraw[];
   int b = blockIdx.x, pool = tb.pool, N = tb.N;
   float *sc = (float *)smraw;                       // [pool+1]
@@ -279,11 +443,13 @@ __global__ void __launch_bounds__(256) rerank_kernel(SeqState st, TreeBufs tb, R
 }
 void launch_rerank(SeqState st, TreeBufs tb, RowMeta m, int B, cudaStream_t s) {
   size_t smem = (size_t)(tb.pool + 1) * 12 + 16;
-  rerank_kernel<<<B, 256, smem, s>>>(st, tb, m);
+  launch_k(rerank_kernel, dim3(B), dim3(256), smem, s, st, tb, m);
 }
 
 // Tree of the root alone (plain autoregressive decoding on the same kernels): one row per sequence.
 __global__ void plain_tree_kernel(SeqState st, TreeBufs tb, RowMeta m, int B) {
+  pdl_wait();
+  pdl_trigger();
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   int n = st.n[b];
@@ -295,12 +461,14 @@ __global__ void plain_tree_kernel(SeqState st, TreeBufs tb, RowMeta m, int B) {
   m.mask_lo[b] = 1ull; m.mask_hi[b] = 0ull; m.tok[b] = act ? st.root[b] : 0;
 }
 void launch_plain_tree(SeqState st, TreeBufs tb, RowMeta m, int B, cudaStream_t s) {
-  plain_tree_kernel<<<(B + 63) / 64, 64, 0, s>>>(st, tb, m, B);
+  launch_k(plain_tree_kernel, dim3((B + 63) / 64), dim3(64), 0, s, st, tb, m, B);
 }
 
 // ---------------------------------------------------------------- greedy acceptance
 // Follow, from the root, the child whose token equals the target's argmax at the current node.
 __global__ void accept_kernel(SeqState st, TreeBufs tb, int rows_per_seq) {
+  pdl_wait();
+  pdl_trigger();
   int b = blockIdx.x;
   if (threadIdx.x != 0) return;
   int Pmax = tb.Pmax;
@@ -331,7 +499,7 @@ __global__ void accept_kernel(SeqState st, TreeBufs tb, int rows_per_seq) {
   st.root[b] = y[cur];
 }
 void launch_accept(SeqState st, TreeBufs tb, int B, int rows_per_seq, cudaStream_t s) {
-  accept_kernel<<<B, 32, 0, s>>>(st, tb, rows_per_seq);
+  launch_k(accept_kernel, dim3(B), dim3(32), 0, s, st, tb, rows_per_seq);
 }
 
 // ---------------------------------------------------------------- commit: KV compaction + tap gather
@@ -343,6 +511,8 @@ __global__ void __launch_bounds__(256) commit_kernel(SeqState st, TreeBufs tb, c
                                                      PageMap pm, const T *__restrict__ node_taps,
                                                      T *__restrict__ pend_taps, int L, int G, int hd, int k,
                                                      int rows_per_seq) {
+  pdl_wait();
+  pdl_trigger();
   int b = blockIdx.x, l = blockIdx.y;
   int cnt = tb.out_cnt[b];
   if (cnt <= 0) return;
@@ -370,7 +540,7 @@ __global__ void __launch_bounds__(256) commit_kernel(SeqState st, TreeBufs tb, c
 template <typename T>
 void launch_commit(SeqState st, TreeBufs tb, const KvPool *pools, PageMap pm, const T *node_taps, T *pend_taps, int B,
                    int L, int G, int hd, int k, int rows_per_seq, cudaStream_t s) {
-  commit_kernel<T><<<dim3(B, L + 1), 256, 0, s>>>(st, tb, pools, pm, node_taps, pend_taps, L, G, hd, k, rows_per_seq);
+  launch_k(commit_kernel<T>, dim3(B, L + 1), dim3(256), 0, s, st, tb, pools, pm, node_taps, pend_taps, L, G, hd, k, rows_per_seq);
 }
 template void launch_commit<float>(SeqState, TreeBufs, const KvPool *, PageMap, const float *, float *, int, int, int,
                                    int, int, int, cudaStream_t);
