@@ -137,6 +137,14 @@ enum spec_prof_class {
 };
 int spec_profile_step(spec_ctx *ctx, float *class_ms, int32_t *class_launches);
 
+/* Performance knobs (the defaults are tuned for B200; results never depend on them).
+ *   SPEC_TUNE_L2_LEAD_MB  how many MB of the weights that follow in a step's read order each GEMM launch
+ *                         keeps prefetched in L2 (0 = no prefetch)
+ *   SPEC_TUNE_GEMM_CTAS   CTAs a weight-streaming GEMM launch aims at (process-wide) */
+enum spec_tune_knob { SPEC_TUNE_L2_LEAD_MB = 1, SPEC_TUNE_GEMM_CTAS = 2,
+                      SPEC_TUNE_DEBUG_LAUNCH_BUDGET = 3 /* debugging: run only the first n kernels of each step (-1: all) */ };
+int spec_tune(spec_ctx *ctx, int32_t what, int32_t value);
+
 /* Number of kernels one spec_step launches (for launch accounting). */
 int spec_launches_per_step(const spec_ctx *ctx);
 
@@ -167,7 +175,10 @@ enum spec_debug_what {
   SPEC_DBG_FRONTIER,         /* int32 [D][K]             */
   SPEC_DBG_PATH,             /* int32 [count]            */
   SPEC_DBG_STATUS,           /* int32 [4] device status words */
-  SPEC_DBG_PAGE_TABLE        /* int32 [pages of seq]     */
+  SPEC_DBG_PAGE_TABLE,       /* int32 [pages of seq]     */
+  /* raw activation buffers of the last pass as floats, all allocated rows (debugging) */
+  SPEC_DBG_RAW_X = 100, SPEC_DBG_RAW_H, SPEC_DBG_RAW_Q, SPEC_DBG_RAW_AO, SPEC_DBG_RAW_ACT, SPEC_DBG_RAW_CAT,
+  SPEC_DBG_RAW_SSQ, SPEC_DBG_RAW_LOGITS
 };
 /* Copies up to `bytes` of item `what` of sequence `seq` (last step) to host_dst; returns bytes
  * available (>= 0) or a negative status. */

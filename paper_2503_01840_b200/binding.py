@@ -24,7 +24,8 @@ FLAG_REF_GEMM, FLAG_REF_ATTN, FLAG_CAPTURE, FLAG_NO_GRAPH, FLAG_UNFUSED, FLAG_NO
 (DBG_TREE_TOK, DBG_TREE_PARENT, DBG_TREE_DEPTH, DBG_TREE_MASK, DBG_TREE_POOLIDX, DBG_TREE_SCORE, DBG_Y,
  DBG_TARGET_LOGITS, DBG_NODE_TAPS, DBG_NODE_HIDDEN, DBG_DRAFT_LOGITS, DBG_DRAFT_A, DBG_POOL_TOK, DBG_POOL_SCORE,
  DBG_POOL_PARENT, DBG_FRONTIER, DBG_PATH, DBG_STATUS, DBG_PAGE_TABLE) = range(1, 20)
-_DBG_DTYPE = {DBG_TREE_TOK: np.int32, DBG_TREE_PARENT: np.int32, DBG_TREE_DEPTH: np.int32, DBG_TREE_MASK: np.uint64,
+DBG_RAW_X, DBG_RAW_H, DBG_RAW_Q, DBG_RAW_AO, DBG_RAW_ACT, DBG_RAW_CAT, DBG_RAW_SSQ, DBG_RAW_LOGITS = range(100, 108)
+_DBG_DTYPE = {**{i: np.float32 for i in range(100, 108)}, DBG_TREE_TOK: np.int32, DBG_TREE_PARENT: np.int32, DBG_TREE_DEPTH: np.int32, DBG_TREE_MASK: np.uint64,
               DBG_TREE_POOLIDX: np.int32, DBG_TREE_SCORE: np.float32, DBG_Y: np.int32, DBG_TARGET_LOGITS: np.float32,
               DBG_NODE_TAPS: np.float32, DBG_NODE_HIDDEN: np.float32, DBG_DRAFT_LOGITS: np.float32,
               DBG_DRAFT_A: np.float32, DBG_POOL_TOK: np.int32, DBG_POOL_SCORE: np.float32, DBG_POOL_PARENT: np.int32,
@@ -55,7 +56,7 @@ class _Cfg(C.Structure):
 
 
 EXPORTS = ("spec_workspace_bytes", "spec_init", "spec_prefill", "spec_step", "spec_step_async", "spec_plain_step",
-           "spec_lengths", "spec_profile_step", "spec_launches_per_step", "spec_step_bytes", "spec_free", "spec_last_error",
+           "spec_lengths", "spec_profile_step", "spec_tune", "spec_launches_per_step", "spec_step_bytes", "spec_free", "spec_last_error",
            "spec_debug_read", "spec_debug_read_kv", "spec_gemm_scratch_bytes", "spec_gemm", "spec_gemm_fused",
            "spec_topk_scratch_bytes", "spec_attn_scratch_bytes",
            "spec_attention", "spec_attention_static", "spec_attention_static_capacity", "spec_logsoftmax_topk", "spec_argmax")
@@ -82,6 +83,7 @@ def lib():
     L.spec_plain_step.argtypes = [vp, vp]
     L.spec_lengths.argtypes = [vp, vp]
     L.spec_launches_per_step.argtypes = [vp]
+    L.spec_tune.argtypes = [vp, i32, i32]
     L.spec_profile_step.argtypes = [vp, vp, vp]
     L.spec_step_bytes.argtypes = [vp, C.POINTER(C.c_double)]
     L.spec_free.argtypes = [vp]
@@ -251,6 +253,11 @@ class SpecDecoder:
         n = np.zeros(len(self.PROF_CLASSES), np.int32)
         self._check(lib().spec_profile_step(self.h, ms.ctypes.data, n.ctypes.data))
         return {c: (float(ms[i]), int(n[i])) for i, c in enumerate(self.PROF_CLASSES)}
+
+    TUNE_L2_LEAD_MB, TUNE_GEMM_CTAS, TUNE_DEBUG_LAUNCH_BUDGET = 1, 2, 3
+
+    def tune(self, what: int, value: int):
+        self._check(lib().spec_tune(self.h, what, value))
 
     def launches_per_step(self) -> int:
         return lib().spec_launches_per_step(self.h)

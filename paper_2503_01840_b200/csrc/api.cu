@@ -19,6 +19,7 @@ using namespace spec;
 
 namespace spec {
 thread_local bool tl_pdl = false;
+thread_local int tl_launch_budget = -1;
 
 void launch_logsoftmax_topk_rows(const float *logits, const int32_t *src_row, int rows, int n, int K, int32_t *idx,
                                  float *lp, cudaStream_t s);
@@ -88,6 +89,15 @@ struct spec_ctx {
   int32_t *best_idx = nullptr;
   void *topk_scratch = nullptr;
   int ktiles = 0, vtiles = 0;
+  // weights in the order one speculative step reads them (cyclic: the stream of the next step follows);
+  // every GEMM launch prefetches its share of the window [own end, own end + lead) into L2
+  struct WSeg { const void *ptr; size_t bytes; };
+  std::vector<WSeg> wstream;
+  std::vector<size_t> wcum;      // wcum[i] = bytes before entry i; wcum.back() = total
+  int wcur = -1;                 // stream entry of the next GEMM launch (-1: no prefetching)
+  size_t pf_front = 0;           // stream position up to which earlier launches of this step prefetched
+  size_t pf_lead = 0;             // bytes each launch keeps prefetched ahead (off by default: measured slower on B200)
+  int dbg_launch_budget = -1;   // debugging aid: kernels of the next step to run (-1: all)
   void *gemm_scratch;
   size_t gemm_scratch_bytes;
   void *attn_scratch;
@@ -291,6 +301,20 @@ extern "C" int spec_init(spec_ctx **out, const spec_target_weights *tw, const sp
     }
   }
   c->fused = c->fg && !(cfg->flags & SPEC_FLAG_UNFUSED) && c->hd <= 128 && (c->hd & (c->hd - 1)) == 0 && c->Ralloc <= 256;
+  if (c->fused) {
+    size_t e = 2, k = c->k, qd = (size_t)c->H * c->hd, kvd = (size_t)c->G * c->hd, F = c->F;
+    auto push = [&](const void *p, size_t elems) { c->wstream.push_back({p, elems * e}); };
+    auto layer = [&](const LayerW &w) {
+      push(w.wq, qd * k); push(w.wk, kvd * k); push(w.wv, kvd * k); push(w.wo, k * qd);
+      push(w.w_gate, F * k); push(w.w_up, F * k); push(w.w_down, k * F);
+    };
+    push(c->fc3, k * 3 * k);
+    for (int d = 0; d < c->D; d++) { push(c->fc2, k * 2 * k); layer(c->dl); push(c->dlm_head, (size_t)c->Vd * k); }
+    for (int l = 0; l < c->L; l++) layer(c->tl[l]);
+    push(c->lm_head, (size_t)c->V * k);
+    c->wcum.assign(c->wstream.size() + 1, 0);
+    for (size_t i = 0; i < c->wstream.size(); i++) c->wcum[i + 1] = c->wcum[i] + c->wstream[i].bytes;
+  }
   if (c->fg && c->R > 256) {
     int rc = fail(nullptr, SPEC_ERR_UNSUPPORTED, "spec_init: %d rows per pass exceed the 256 the tensor-core GEMM takes", c->R);
     fast_gemm_destroy(c->fg);
@@ -358,8 +382,34 @@ template <typename T> struct Sched {
   void with_norm_scale(FusedGemmArgs &a) const {
     a.ssq_in = c->ssq; a.ssq_in_tiles = c->ktiles; a.ssq_ld = c->Ralloc; a.k_in = c->k; a.eps = c->cfg.rms_eps;
   }
-  void fgemm(FusedEpi epi, const FusedGemmArgs &a) {
+  // Assigns this launch its share of the L2 prefetch window and advances the stream cursor.
+  void assign_prefetch(FusedGemmArgs &a) {
+    if (c->wcur < 0 || c->pf_lead == 0) return;
+    const int n = (int)c->wstream.size();
+    if (c->wcur + a.nw > n || c->wstream[c->wcur].ptr != (const void *)a.w[0]) { c->wcur = -1; return; }   // not the step's order
+    const size_t total = c->wcum[n];
+    const size_t own_end = c->wcum[c->wcur + a.nw];
+    size_t lo = std::max(own_end, c->pf_front), hi = own_end + c->pf_lead;
+    c->wcur += a.nw;
+    if (hi <= lo) return;
+    // entries overlapping [lo, hi) in the cyclic stream
+    size_t pos = lo;
+    int idx = (int)(std::upper_bound(c->wcum.begin(), c->wcum.end(), pos % total) - c->wcum.begin()) - 1;
+    while (pos < hi && a.npf < FusedGemmArgs::MAX_PREFETCH) {
+      idx %= n;
+      size_t seg_lo = pos % total - c->wcum[idx];
+      size_t take = std::min(c->wstream[idx].bytes - seg_lo, hi - pos);
+      a.pf_ptr[a.npf] = (const char *)c->wstream[idx].ptr + seg_lo;
+      a.pf_bytes[a.npf] = take;
+      a.npf++;
+      pos += take;
+      idx++;
+    }
+    c->pf_front = pos;
+  }
+  void fgemm(FusedEpi epi, FusedGemmArgs a) {
     mark(SPEC_PROF_GEMM);
+    assign_prefetch(a);
     int rc = fused_gemm_launch(c->fg, epi, a, s);
     if (rc && !c->sched_err) c->sched_err = rc;
     tick();
@@ -538,7 +588,7 @@ template <typename T> struct Sched {
     if (first) {
       launch_gather_rows(c->logits, c->st.last_row, c->cap_logits + lo * c->Vd, c->B, c->Vd, c->K, s);
       launch_gather_rows(c->x, c->st.last_row, c->cap_a + lo * c->k, c->B, c->k, c->K, s);
-    } else {
+    } else if (tl_launch_budget != 0) {
       cudaMemcpyAsync(c->cap_logits + lo * c->Vd, c->logits, (size_t)rows * c->Vd * 4, cudaMemcpyDeviceToDevice, s);
       cudaMemcpyAsync(c->cap_a + lo * c->k, c->x, (size_t)rows * c->k * 4, cudaMemcpyDeviceToDevice, s);
     }
@@ -547,6 +597,10 @@ template <typename T> struct Sched {
 
   void step(bool plain) {
     int rows = plain ? c->B : c->Tv, rps = plain ? 1 : c->N;
+    // the previous step's last launches already covered the first `lead` bytes of this step's stream
+    c->wcur = (!plain && c->fused) ? 0 : -1;
+    c->pf_front = c->pf_lead;
+    tl_launch_budget = c->dbg_launch_budget;
     if (!plain) {
       mark(SPEC_PROF_TREE); launch_prep_extend(c->st, c->tb, c->meta, c->B, c->need_pos, c->status, s); tick();
       c->cur_rps = c->Pmax;
@@ -576,6 +630,8 @@ template <typename T> struct Sched {
                      c->k, rps, s);
     tick();
     mark(-1);
+    c->wcur = -1;
+    tl_launch_budget = -1;
   }
 };
 
@@ -808,6 +864,23 @@ extern "C" int spec_profile_step(spec_ctx *c, float *class_ms, int32_t *class_la
   return sync_lengths(c);
 }
 
+extern "C" int spec_tune(spec_ctx *c, int32_t what, int32_t value) {
+  if (!c) return SPEC_ERR_NULL;
+  if (what == SPEC_TUNE_L2_LEAD_MB) {
+    if (value < 0 || value > 120) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the L2 prefetch distance must be 0..120 MB");
+    c->pf_lead = (size_t)value << 20;
+  } else if (what == SPEC_TUNE_DEBUG_LAUNCH_BUDGET) {
+    c->dbg_launch_budget = value;
+  } else if (what == SPEC_TUNE_GEMM_CTAS) {
+    if (value < 32 || value > 2048) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the GEMM CTA target must be 32..2048");
+    fused_gemm_set_target_ctas(value);
+  } else {
+    return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: unknown knob %d", what);
+  }
+  if (c->graph) { cudaStreamSynchronize(c->stream); cudaGraphExecDestroy(c->graph); c->graph = nullptr; }   // re-capture with the new plan
+  return SPEC_OK;
+}
+
 extern "C" int spec_launches_per_step(const spec_ctx *c) { return c ? c->launches : 0; }
 
 extern "C" int spec_step_bytes(spec_ctx *c, double *bytes) {
@@ -890,6 +963,14 @@ extern "C" int64_t spec_debug_read(spec_ctx *c, int32_t what, int32_t seq, void 
     case SPEC_DBG_PATH: return copy_out(c, t.path + (size_t)seq * c->Pmax, cnt, dst, bytes);
     case SPEC_DBG_STATUS: return copy_out(c, c->status, 4, dst, bytes);
     case SPEC_DBG_PAGE_TABLE: return copy_out(c, c->page_table + (size_t)seq * c->pps, c->n_pages_host[seq], dst, bytes);
+    case SPEC_DBG_RAW_X: return copy_out(c, c->x, (size_t)c->Ralloc * c->k, dst, bytes);
+    case SPEC_DBG_RAW_H: return copy_widen(c, c->h, (size_t)c->Ralloc * c->k, dst, bytes);
+    case SPEC_DBG_RAW_Q: return copy_widen(c, c->q, (size_t)c->Ralloc * c->H * c->hd, dst, bytes);
+    case SPEC_DBG_RAW_AO: return copy_widen(c, c->ao, (size_t)c->Ralloc * c->H * c->hd, dst, bytes);
+    case SPEC_DBG_RAW_ACT: return copy_widen(c, c->act, (size_t)c->Ralloc * c->F, dst, bytes);
+    case SPEC_DBG_RAW_CAT: return copy_widen(c, c->cat, (size_t)c->Ralloc * 2 * c->k, dst, bytes);
+    case SPEC_DBG_RAW_SSQ: return copy_out(c, c->ssq, (size_t)c->ktiles * c->Ralloc, dst, bytes);
+    case SPEC_DBG_RAW_LOGITS: return copy_out(c, c->logits, (size_t)c->Ralloc * c->Vd, dst, bytes);
     default: return fail(c, SPEC_ERR_INVALID_CFG, "spec_debug_read: unknown item %d", what);
   }
 }

@@ -30,9 +30,19 @@ __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.lau
 // When set (per host thread, by the step scheduler), launch_k adds the programmatic-dependent-launch
 // attribute to every launch.
 extern thread_local bool tl_pdl;
+// Debugging aid: when >= 0, the number of kernel launches still allowed on this host thread; further
+// launches are dropped (lets a test look at intermediate buffers after the n-th kernel of a step).
+extern thread_local int tl_launch_budget;
+inline bool launch_allowed() {
+  if (tl_launch_budget < 0) return true;
+  if (tl_launch_budget == 0) return false;
+  tl_launch_budget--;
+  return true;
+}
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  if (!launch_allowed()) return cudaSuccess;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
   cudaLaunchAttribute at[1];

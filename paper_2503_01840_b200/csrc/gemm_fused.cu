@@ -14,7 +14,8 @@
 //    round trip of partial sums through global memory);
 //  * the epilogue that follows the reduction is the consumer's work: residual add + bf16 copy scaled
 //    by the next norm's gain + RMSNorm statistics (+ feature taps); RoPE + q store + paged K/V write;
-//    SiLU(gate)*up; per-tile argmax.  RMSNorm of the input is applied as a per-row scale in the
+//    SiLU(gate)*up (the gate and up tiles of a feature range are two members of the same cluster);
+//    per-tile argmax.  RMSNorm of the input is applied as a per-row scale in the
 //    epilogue (the normalisation factor is a row constant, so it commutes with the contraction);
 //  * programmatic dependent launch: the producer prefetches the first weight tiles (which never depend
 //    on the previous kernel) before griddepcontrol.wait, so the pipeline is full when the activations
@@ -45,15 +46,20 @@ struct alignas(64) FusedParams {
   CUtensorMap map_x;
   int tiles0, tiles1;          // tile index ranges of the weights: [0,tiles0) w0, [tiles0,tiles1) w1, rest w2
   int O[3];
-  int rows, KB, S, stages, ctrl_off;
+  int rows, KB, S, Sk, stages, ctrl_off;   // S = cluster size, Sk = K slices (S = 2 Sk for EPI_SWIGLU)
   const float *ssq_in; int ssq_in_tiles, ssq_ld; float inv_k_in, eps;
   float *out_f32; int ldo;
   float *xres; const bf16 *gain; bf16 *hb; float *ssq_out; bf16 *taps; int tap_mask, resid_add;
   const float2 *cs; RowMeta m; bf16 *q; KvPool pool; PageMap pm; int H, G, hd;
   bf16 *act;
   float *best_val; int32_t *best_idx; int best_ld;
+  const unsigned char *pf_ptr[FusedGemmArgs::MAX_PREFETCH];
+  unsigned long long pf_bytes[FusedGemmArgs::MAX_PREFETCH];
+  int npf;
   int32_t *status;
 };
+
+constexpr unsigned PF_CHUNK = 32768;   // bytes per L2 prefetch instruction
 
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
@@ -73,11 +79,9 @@ __device__ __forceinline__ float ld_peer(uint32_t local_addr, uint32_t rank) {
 
 template <int NT, int EPI>
 __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__ FusedParams p) {
-  constexpr bool PAIR = (EPI == EPI_SWIGLU);
-  constexpr int NA = PAIR ? 2 : 1;
   constexpr int B_BYTES = NT * TILE_K * 2;
-  constexpr int STAGE = NA * A_BYTES + B_BYTES;
-  constexpr int TMEM_COLS = (NA * NT < 32) ? 32 : NA * NT;
+  constexpr int STAGE = A_BYTES + B_BYTES;
+  constexpr int TMEM_COLS = (NT < 32) ? 32 : NT;
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char *tiles = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -91,12 +95,15 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
   float *wpart = inv_s + 256;                    // [4][CHUNK] per-warp partial sums / argmax exchange
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int stages = p.stages, S = p.S;
-  const int slice = (S > 1) ? (int)cluster_rank() : 0;
-  const int kb0 = (int)(((long long)slice * p.KB) / S), kb1 = (int)(((long long)(slice + 1) * p.KB) / S);
+  const int stages = p.stages, S = p.S, Sk = p.Sk;
+  const int slice = (S > 1) ? (int)cluster_rank() : 0;        // rank in the cluster
+  const int ksl = (EPI == EPI_SWIGLU) ? slice % Sk : slice;   // K slice
+  const int kb0 = (int)(((long long)ksl * p.KB) / Sk), kb1 = (int)(((long long)(ksl + 1) * p.KB) / Sk);
   const int nkb = kb1 - kb0;
   int mi = 0, tm = blockIdx.x;                   // weight index and tile within that weight
-  if (!PAIR) {
+  if (EPI == EPI_SWIGLU) {
+    mi = slice / Sk;                             // ranks [0,Sk) stream the gate tile, [Sk,2Sk) the up tile
+  } else {
     if (tm >= p.tiles1) { mi = 2; tm -= p.tiles1; }
     else if (tm >= p.tiles0) { mi = 1; tm -= p.tiles0; }
   }
@@ -120,25 +127,38 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
 
   if (warp == 0 && lane == 0) {
     // ---- producer.  Weight tiles do not depend on the previous kernel: fill the ring with them first.
-    const CUtensorMap *mw0 = &p.map_w[PAIR ? 0 : mi];
+    const CUtensorMap *mw0 = &p.map_w[mi];
+    const uint64_t pol = l2_policy_evict_first();
     const int npre = nkb < stages ? nkb : stages;
     for (int i = 0; i < npre; i++) {
       unsigned char *a = tiles + i * STAGE;
       mbar_expect_tx(&full[i], STAGE);
-      tma_load_2d(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[i]);
-      if (PAIR) tma_load_2d(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[i]);
+      tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[i], pol);
+    }
+    // pull the weights of the launches that follow into L2: the memory system stays busy across this
+    // kernel's epilogue and the next kernel's start-up, and those kernels then stream from L2
+    if (p.npf > 0) {
+      const unsigned ncta = gridDim.x * gridDim.y, me = blockIdx.y * gridDim.x + blockIdx.x;
+      for (int sgm = 0; sgm < p.npf; sgm++) {
+        const unsigned long long nb = p.pf_bytes[sgm];
+        const unsigned long long nch = (nb + PF_CHUNK - 1) / PF_CHUNK;
+        for (unsigned long long ch = me; ch < nch; ch += ncta) {
+          unsigned long long off = ch * PF_CHUNK;
+          unsigned len = (unsigned)((nb - off < PF_CHUNK) ? nb - off : PF_CHUNK);
+          l2_prefetch_bulk(p.pf_ptr[sgm] + off, len);
+        }
+      }
     }
     pdl_wait();
-    for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + NA * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
+    for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
     for (int i = npre; i < nkb; i++) {
       int st = i % stages;
       if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
       if (*abort_flag) break;
       unsigned char *a = tiles + st * STAGE;
       mbar_expect_tx(&full[st], STAGE);
-      tma_load_2d(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[st]);
-      if (PAIR) tma_load_2d(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[st]);
-      tma_load_2d(a + NA * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[st]);
+      tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
+      tma_load_2d(a + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[st]);
     }
   } else {
     pdl_wait();
@@ -150,12 +170,11 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
         if (!mbar_wait(&full[st], (i / stages) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 201, blockIdx.x, i); break; }
         if (*abort_flag) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        uint32_t a = smem_u32(tiles + st * STAGE), b = a + NA * A_BYTES;
+        uint32_t a = smem_u32(tiles + st * STAGE), b = a + A_BYTES;
 #pragma unroll
         for (int j = 0; j < TILE_K / UMMA_K; j++) {
           uint64_t db = umma_desc_sw128(b + j * UMMA_K * 2);
           umma_bf16(tmem_base, umma_desc_sw128(a + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
-          if (PAIR) umma_bf16(tmem_base + NT, umma_desc_sw128(a + A_BYTES + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
         }
         umma_commit(&empty[st]);      // frees the stage once these MMAs have read it
       }
@@ -187,28 +206,25 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
 
   // ---- epilogue, CHUNK rows at a time.  The stage ring is free now (every load landed, every MMA that
   // read it completed) and is reused: red = this CTA's accumulator(s), sumb = reduced rows (EPI_QKV).
-  float *red = (float *)tiles;                       // [NA][CHUNK][128]
-  float *sumb = red + NA * CHUNK * TILE_M;           // [CHUNK][128]
+  float *red = (float *)tiles;                       // [CHUNK][128]
+  float *sumb = red + CHUNK * TILE_M;                // [CHUNK][128]
   const int f = threadIdx.x;
   const int o = tm * TILE_M + f;                     // output feature within weight mi
   for (int c0 = 0; c0 < p.rows; c0 += CHUNK) {
     const int nrow = (p.rows - c0 < CHUNK) ? p.rows - c0 : CHUNK;
     if (good) {
-#pragma unroll
-      for (int a = 0; a < NA; a++) {
 #pragma unroll 1
-        for (int cc = 0; cc < CHUNK && c0 + cc < NT; cc += 16) {
-          if (cc >= nrow) break;
-          uint32_t v[16];
-          tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(a * NT + c0 + cc), v);
+      for (int cc = 0; cc < CHUNK && c0 + cc < NT; cc += 16) {
+        if (cc >= nrow) break;
+        uint32_t v[16];
+        tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + cc), v);
 #pragma unroll
-          for (int j = 0; j < 16; j++) red[(a * CHUNK + cc + j) * TILE_M + f] = __uint_as_float(v[j]);
-        }
+        for (int j = 0; j < 16; j++) red[(cc + j) * TILE_M + f] = __uint_as_float(v[j]);
       }
     }
     if (S > 1) cluster_sync_all(); else __syncthreads();
     const int per = (nrow + S - 1) / S;
-    const int r0 = slice * per, r1 = (r0 + per < nrow) ? r0 + per : nrow;
+    const int r0 = (slice * per < nrow) ? slice * per : nrow, r1 = (r0 + per < nrow) ? r0 + per : nrow;   // r0 <= r1
 
     if (EPI == EPI_F32 || EPI == EPI_RESID || EPI == EPI_QKV) {
       for (int r = r0; r < r1; r++) {
@@ -244,7 +260,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       }
       if (EPI == EPI_RESID) {
         __syncthreads();
-        if (good && threadIdx.x < r1 - r0) {
+        if (good && (int)threadIdx.x < r1 - r0) {
           int t = threadIdx.x;
           p.ssq_out[(size_t)tm * p.ssq_ld + c0 + r0 + t] =
               ((wpart[t] + wpart[CHUNK + t]) + wpart[2 * CHUNK + t]) + wpart[3 * CHUNK + t];
@@ -285,13 +301,15 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
         }
       }
     } else if (EPI == EPI_SWIGLU) {
-      if (good && o < p.O[0]) {
-        for (int r = r0; r < r1; r++) {
-          const int row = c0 + r;
-          float sc = inv_s[row];
-          float g = red[r * TILE_M + f] * sc, u = red[(CHUNK + r) * TILE_M + f] * sc;
-          p.act[(size_t)row * p.O[0] + o] = __float2bfloat16_rn((g / (1.0f + expf(-g))) * u);
-        }
+      for (int r = r0; r < r1; r++) {
+        const int row = c0 + r;
+        uint32_t la = smem_u32(&red[r * TILE_M + f]);
+        float g = 0.0f, u = 0.0f;
+        for (int s = 0; s < Sk; s++) g += ld_peer(la, (uint32_t)s);
+        for (int s = 0; s < Sk; s++) u += ld_peer(la, (uint32_t)(Sk + s));
+        float sc = inv_s[row];
+        g *= sc; u *= sc;
+        if (good && o < p.O[0]) p.act[(size_t)row * p.O[0] + o] = __float2bfloat16_rn((g / (1.0f + expf(-g))) * u);
       }
     } else {   // EPI_ARGMAX
       if (good && p.out_f32 && o < p.O[0])
@@ -336,31 +354,37 @@ constexpr int NUM_SMS = 148;
 constexpr int SMEM_ONE = 200 * 1024;      // ring budget with one CTA per SM
 constexpr int SMEM_TWO = 104 * 1024;      // ring budget that lets two CTAs share an SM
 
-struct Plan { int nt, tiles, S, stages, smem, ctrl_off, KB; };
+struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB; };
+
+// CTAs are sized so that two of them share an SM (one CTA alone cannot hide its MMA and epilogue time
+// behind its own loads) and the grid covers all SMs about twice: S K-slices per feature tile.
+int g_target_ctas = 2 * NUM_SMS;
 
 Plan make_plan(FusedEpi epi, const FusedGemmArgs &a) {
   Plan pl;
-  const bool pair = epi == EPI_SWIGLU;
   pl.nt = pick_nt(a.rows);
   pl.KB = (a.I + TILE_K - 1) / TILE_K;
   pl.tiles = fused_gemm_tiles(epi, a);
-  const int stage = (pair ? 2 : 1) * A_BYTES + pl.nt * TILE_K * 2;
-  int S = 1;
-  if (epi == EPI_F32 || epi == EPI_RESID || epi == EPI_QKV) {
-    S = std::max(1, std::min(8, NUM_SMS / std::max(1, pl.tiles)));
-    S = std::max(1, std::min(S, pl.KB / 4));
+  const int stage = A_BYTES + pl.nt * TILE_K * 2;
+  const int wmul = epi == EPI_SWIGLU ? 2 : 1;          // cluster members per K slice
+  const int smax = 8 / wmul;
+  int Sk = 1;
+  if (epi != EPI_ARGMAX) {
+    Sk = (g_target_ctas + pl.tiles * wmul / 2) / std::max(1, pl.tiles * wmul);   // nearest
+    Sk = std::max(1, std::min(Sk, smax));
+    Sk = std::max(1, std::min(Sk, pl.KB / 4));
   }
-  if (a.split > 0) S = std::min(std::min(a.split, 8), pl.KB);
-  if (epi == EPI_SWIGLU || epi == EPI_ARGMAX) S = 1;
-  pl.S = S;
-  int budget = SMEM_ONE;
-  if (pl.tiles * S > NUM_SMS && SMEM_TWO / stage >= 3) budget = SMEM_TWO;   // several waves: let two CTAs overlap
+  if (a.split > 0) Sk = std::max(1, std::min(std::min(a.split, smax), pl.KB));
+  pl.Sk = Sk;
+  pl.S = Sk * wmul;
+  int budget = SMEM_TWO;
+  if (SMEM_TWO / stage < 3) budget = SMEM_ONE;         // 256-row tiles: one CTA per SM
   int stages = std::max(2, std::min(MAX_STAGES, budget / stage));
   if (a.stages > 0) stages = std::max(2, std::min(std::min(a.stages, MAX_STAGES), (220 * 1024) / stage));
-  int per_slice = (pl.KB + S - 1) / S;
+  int per_slice = (pl.KB + Sk - 1) / Sk;
   stages = std::max(2, std::min(stages, per_slice));
   pl.stages = stages;
-  const int epi_bytes = ((pair ? 2 : 1) * CHUNK * TILE_M + (epi == EPI_QKV ? CHUNK * TILE_M : 0)) * 4;
+  const int epi_bytes = (CHUNK * TILE_M + (epi == EPI_QKV ? CHUNK * TILE_M : 0)) * 4;
   pl.ctrl_off = (std::max(stages * stage, epi_bytes) + 1023) & ~1023;
   pl.smem = pl.ctrl_off + 512 + 256 * 4 + 4 * CHUNK * 4 + 1024 /*alignment slack*/;
   return pl;
@@ -373,6 +397,7 @@ int launch_inst(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) 
     if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem) != cudaSuccess) return -6;
     configured = pl.smem;
   }
+  if (!launch_allowed()) return 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(pl.tiles, pl.S, 1);
   cfg.blockDim = dim3(128, 1, 1);
@@ -406,6 +431,8 @@ int launch_epi(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) {
 }
 
 }  // namespace
+
+void fused_gemm_set_target_ctas(int n) { g_target_ctas = n; }
 
 int fused_gemm_tiles(FusedEpi epi, const FusedGemmArgs &a) {
   if (epi == EPI_SWIGLU) return (a.O[0] + TILE_M - 1) / TILE_M;
@@ -444,7 +471,7 @@ int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStr
   p.map_x = *mx;
   p.tiles0 = (a.O[0] + TILE_M - 1) / TILE_M;
   p.tiles1 = p.tiles0 + (a.nw > 1 ? (a.O[1] + TILE_M - 1) / TILE_M : 0);
-  p.rows = a.rows; p.KB = pl.KB; p.S = pl.S; p.stages = pl.stages; p.ctrl_off = pl.ctrl_off;
+  p.rows = a.rows; p.KB = pl.KB; p.S = pl.S; p.Sk = pl.Sk; p.stages = pl.stages; p.ctrl_off = pl.ctrl_off;
   p.ssq_in = a.ssq_in; p.ssq_in_tiles = a.ssq_in_tiles; p.ssq_ld = a.ssq_ld; p.inv_k_in = 1.0f / (float)a.k_in; p.eps = a.eps;
   p.out_f32 = a.out_f32; p.ldo = a.ldo;
   p.xres = a.xres; p.gain = a.gain; p.hb = a.hb; p.ssq_out = a.ssq_out; p.taps = a.tap_mask ? a.taps : nullptr;
@@ -453,6 +480,13 @@ int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStr
   p.act = a.act;
   p.best_val = a.best_val; p.best_idx = a.best_idx; p.best_ld = a.best_ld;
   p.status = a.status;
+  p.npf = 0;
+  for (int j = 0; j < a.npf && j < FusedGemmArgs::MAX_PREFETCH; j++) {
+    if (!a.pf_ptr[j] || ((uintptr_t)a.pf_ptr[j] & 15) || a.pf_bytes[j] < 16) continue;
+    p.pf_ptr[p.npf] = (const unsigned char *)a.pf_ptr[j];
+    p.pf_bytes[p.npf] = a.pf_bytes[j] & ~(size_t)15;
+    p.npf++;
+  }
   switch (epi) {
     case EPI_F32: return launch_epi<EPI_F32>(p, pl, a.pdl, s);
     case EPI_RESID: return launch_epi<EPI_RESID>(p, pl, a.pdl, s);

@@ -50,6 +50,11 @@ struct FusedGemmArgs {
   float *best_val = nullptr;    // [tiles][best_ld]
   int32_t *best_idx = nullptr;
   int best_ld = 0;
+  // ---- weights of later launches to pull into L2 while this one runs (addresses and sizes multiples of 16)
+  static constexpr int MAX_PREFETCH = 6;
+  const void *pf_ptr[MAX_PREFETCH] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  size_t pf_bytes[MAX_PREFETCH] = {0, 0, 0, 0, 0, 0};
+  int npf = 0;
   // ---- launch
   int32_t *status = nullptr;    // device status words
   int split = 0, stages = 0;    // 0 = chosen by the library
@@ -61,6 +66,8 @@ struct FusedGemmArgs {
 bool fused_gemm_supported(FusedEpi epi, const FusedGemmArgs &a);
 // number of 128-feature tiles of the launch (EPI_ARGMAX: rows of best_val / best_idx needed)
 int fused_gemm_tiles(FusedEpi epi, const FusedGemmArgs &a);
+// CTAs a launch aims at (K slices are chosen to come close to it); process-wide.
+void fused_gemm_set_target_ctas(int n);
 // Returns 0 or a negative code.
 int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStream_t s);
 
