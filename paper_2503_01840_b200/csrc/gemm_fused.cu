@@ -77,6 +77,33 @@ __device__ __forceinline__ float ld_peer(uint32_t local_addr, uint32_t rank) {
   return v;
 }
 
+// 16-byte load from the same shared-memory offset in cluster member `rank`.  Deliberately without a
+// "memory" clobber: consecutive loads stay in program order (volatile) but do not wait for one another,
+// so a thread keeps several remote requests in flight.
+__device__ __forceinline__ float4 ld_peer4(uint32_t local_addr, uint32_t rank) {
+  uint32_t ra;
+  float4 v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(ra));
+  return v;
+}
+// sum over cluster members [s0, s0+n) (n <= 16) of the float4 at local_addr, added in member order
+__device__ __forceinline__ float4 sum_peers4(uint32_t local_addr, int s0, int n) {
+  float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll
+  for (int b = 0; b < 16; b += 8) {
+    if (b >= n) break;
+    float4 v[8];
+#pragma unroll
+    for (int s = 0; s < 8; s++)
+      if (b + s < n) v[s] = ld_peer4(local_addr, (uint32_t)(s0 + b + s));
+#pragma unroll
+    for (int s = 0; s < 8; s++)
+      if (b + s < n) { acc.x += v[s].x; acc.y += v[s].y; acc.z += v[s].z; acc.w += v[s].w; }
+  }
+  return acc;
+}
+
 template <int NT, int EPI>
 __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__ FusedParams p) {
   constexpr int B_BYTES = NT * TILE_K * 2;
@@ -135,8 +162,19 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       mbar_expect_tx(&full[i], STAGE);
       tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[i], pol);
     }
-    // pull the weights of the launches that follow into L2: the memory system stays busy across this
-    // kernel's epilogue and the next kernel's start-up, and those kernels then stream from L2
+    pdl_wait();
+    for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
+    for (int i = npre; i < nkb; i++) {
+      int st = i % stages;
+      if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
+      if (*abort_flag) break;
+      unsigned char *a = tiles + st * STAGE;
+      mbar_expect_tx(&full[st], STAGE);
+      tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
+      tma_load_2d(a + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[st]);
+    }
+    // all of this CTA's loads are issued: pull the first weights of the launches that follow into L2, so that
+    // the memory system stays busy across this kernel's epilogue and the next kernel's start-up
     if (p.npf > 0) {
       const unsigned ncta = gridDim.x * gridDim.y, me = blockIdx.y * gridDim.x + blockIdx.x;
       for (int sgm = 0; sgm < p.npf; sgm++) {
@@ -148,17 +186,6 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
           l2_prefetch_bulk(p.pf_ptr[sgm] + off, len);
         }
       }
-    }
-    pdl_wait();
-    for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
-    for (int i = npre; i < nkb; i++) {
-      int st = i % stages;
-      if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
-      if (*abort_flag) break;
-      unsigned char *a = tiles + st * STAGE;
-      mbar_expect_tx(&full[st], STAGE);
-      tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
-      tma_load_2d(a + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[st]);
     }
   } else {
     pdl_wait();
@@ -205,9 +232,9 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
   // ---- epilogue, CHUNK rows at a time.  The stage ring is free now (every load landed, every MMA that
-  // read it completed) and is reused: red = this CTA's accumulator(s), sumb = reduced rows (EPI_QKV).
+  // read it completed) and is reused: red = this CTA's accumulator, sumb = this CTA's rows after the cluster sum.
   float *red = (float *)tiles;                       // [CHUNK][128]
-  float *sumb = red + CHUNK * TILE_M;                // [CHUNK][128]
+  float *sumb = red + CHUNK * TILE_M;                // [CHUNK][128] (EPI_SWIGLU: gate rows, then up rows at CHUNK/2)
   const int f = threadIdx.x;
   const int o = tm * TILE_M + f;                     // output feature within weight mi
   for (int c0 = 0; c0 < p.rows; c0 += CHUNK) {
@@ -226,76 +253,110 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
     const int per = (nrow + S - 1) / S;
     const int r0 = (slice * per < nrow) ? slice * per : nrow, r1 = (r0 + per < nrow) ? r0 + per : nrow;   // r0 <= r1
 
-    if (EPI == EPI_F32 || EPI == EPI_RESID || EPI == EPI_QKV) {
-      for (int r = r0; r < r1; r++) {
-        float v = 0.0f;
-        if (S > 1) {
-          uint32_t la = smem_u32(&red[r * TILE_M + f]);
-          for (int s = 0; s < S; s++) v += ld_peer(la, (uint32_t)s);
-        } else {
-          v = red[r * TILE_M + f];
-        }
-        const int row = c0 + r;
-        if (EPI == EPI_F32) {
-          if (good && o < p.O[0]) p.out_f32[(size_t)row * p.ldo + o] = v * inv_s[row];
-        } else if (EPI == EPI_RESID) {
-          float xo = 0.0f;
-          if (good && o < p.O[0]) {
-            size_t xi = (size_t)row * p.O[0] + o;
-            xo = (p.resid_add ? p.xres[xi] : 0.0f) + v;
-            p.xres[xi] = xo;
-            p.hb[xi] = __float2bfloat16_rn(xo * __bfloat162float(p.gain[o]));
-            if (p.tap_mask) {
+    // ---- phase A (clusters): this CTA's rows, summed over the K slices, land in its own sumb.  Each thread
+    // takes (row, 4 features) items and keeps all its remote loads in flight before adding them up.
+    const float *src = red + r0 * TILE_M;              // S == 1: the accumulator dump is the sum
+    if (S > 1) {
+      const int nitems = (r1 - r0) * 32;
+      for (int item = threadIdx.x; item < nitems; item += 128) {
+        const int i = item >> 5, qd = item & 31;
+        const uint32_t la = smem_u32(&red[(r0 + i) * TILE_M + qd * 4]);
+        *(float4 *)&sumb[i * TILE_M + qd * 4] = sum_peers4(la, 0, Sk);
+        if (EPI == EPI_SWIGLU) *(float4 *)&sumb[(CHUNK / 2 + i) * TILE_M + qd * 4] = sum_peers4(la, Sk, Sk);
+      }
+      __syncthreads();
+      src = sumb;
+    }
+    // ---- phase B: per-feature epilogue from local shared memory (thread = feature f of the tile).  Rows go
+    // in batches of RB: all global loads of a batch are issued before its first store, so the loop is not
+    // a chain of dependent L2 round trips.
+    constexpr int RB = 8;
+    if (EPI == EPI_F32) {
+      for (int r = r0; r < r1; r++)
+        if (good && o < p.O[0]) p.out_f32[(size_t)(c0 + r) * p.ldo + o] = src[(r - r0) * TILE_M + f] * inv_s[c0 + r];
+    } else if (EPI == EPI_RESID) {
+      const bool act_o = good && o < p.O[0];
+      const float gn = act_o ? __bfloat162float(p.gain[o]) : 0.0f;
+      for (int rb = r0; rb < r1; rb += RB) {
+        float xin[RB];
 #pragma unroll
-              for (int s = 0; s < 3; s++)
-                if ((p.tap_mask >> s) & 1) p.taps[(size_t)row * 3 * p.O[0] + (size_t)s * p.O[0] + o] = __float2bfloat16_rn(xo);
+        for (int j = 0; j < RB; j++)
+          xin[j] = (act_o && p.resid_add && rb + j < r1) ? p.xres[(size_t)(c0 + rb + j) * p.O[0] + o] : 0.0f;
+#pragma unroll
+        for (int j = 0; j < RB; j++) {
+          const int r = rb + j;
+          if (r < r1) {              // uniform over the CTA
+            const int row = c0 + r;
+            float xo = 0.0f;
+            if (act_o) {
+              size_t xi = (size_t)row * p.O[0] + o;
+              xo = xin[j] + src[(r - r0) * TILE_M + f];
+              p.xres[xi] = xo;
+              p.hb[xi] = __float2bfloat16_rn(xo * gn);
+              if (p.tap_mask) {
+#pragma unroll
+                for (int s = 0; s < 3; s++)
+                  if ((p.tap_mask >> s) & 1) p.taps[(size_t)row * 3 * p.O[0] + (size_t)s * p.O[0] + o] = __float2bfloat16_rn(xo);
+              }
             }
+            float sq = xo * xo;
+            for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+            if (lane == 0) wpart[warp * CHUNK + (r - r0)] = sq;
           }
-          float sq = xo * xo;
-          for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
-          if (lane == 0) wpart[warp * CHUNK + (r - r0)] = sq;
-        } else {
-          sumb[r * TILE_M + f] = v * inv_s[row];
         }
       }
-      if (EPI == EPI_RESID) {
-        __syncthreads();
-        if (good && (int)threadIdx.x < r1 - r0) {
-          int t = threadIdx.x;
-          p.ssq_out[(size_t)tm * p.ssq_ld + c0 + r0 + t] =
-              ((wpart[t] + wpart[CHUNK + t]) + wpart[2 * CHUNK + t]) + wpart[3 * CHUNK + t];
-        }
+      __syncthreads();
+      if (good && (int)threadIdx.x < r1 - r0) {
+        int t = threadIdx.x;
+        p.ssq_out[(size_t)tm * p.ssq_ld + c0 + r0 + t] =
+            ((wpart[t] + wpart[CHUNK + t]) + wpart[2 * CHUNK + t]) + wpart[3 * CHUNK + t];
       }
-      if (EPI == EPI_QKV) {
-        __syncthreads();
-        const int hd = p.hd, half = hd >> 1;
-        const int head = o / hd, i = o % hd;
-        const bool valid_o = o < p.O[mi];
-        bf16 *Kp = (bf16 *)p.pool.k, *Vp = (bf16 *)p.pool.v;
-        for (int r = r0; r < r1; r++) {
+    } else if (EPI == EPI_QKV) {
+      const int hd = p.hd, half = hd >> 1;
+      const int head = o / hd, i = o % hd;
+      const bool valid_o = (o < p.O[mi]) && good;
+      bf16 *Kp = (bf16 *)p.pool.k, *Vp = (bf16 *)p.pool.v;
+      // per-row cache slot of this CTA's rows: one thread per row resolves sequence -> position -> page
+      int32_t *slot_s = (int32_t *)wpart;              // [CHUNK] element offset / hd of the row's K/V slot, -1: none
+      int32_t *seq_s = slot_s + CHUNK;                 // [CHUNK]
+      if ((int)threadIdx.x < r1 - r0) {
+        const int row = c0 + r0 + threadIdx.x;
+        const int seq = p.m.seq[row];
+        int slot = -1;
+        if (seq >= 0 && mi > 0) {
+          const int kvpos = p.m.kvpos[row];
+          if (kvpos < 0 || kvpos / p.pm.page_size >= p.pm.pages_per_seq) {
+            set_status(p.status, ST_BOUNDS, 1, row, kvpos);
+          } else {
+            const int page = p.pm.table[(size_t)seq * p.pm.pages_per_seq + kvpos / p.pm.page_size];
+            if (page < 0 || page >= p.pm.num_pages) set_status(p.status, ST_BOUNDS, 2, row, page);
+            else slot = (page * p.G) * p.pm.page_size + (kvpos % p.pm.page_size);   // + head * page_size below
+          }
+        }
+        slot_s[threadIdx.x] = slot;
+        seq_s[threadIdx.x] = seq;
+      }
+      __syncthreads();
+      for (int rb = r0; rb < r1; rb += RB) {
+        float2 cs[RB];
+#pragma unroll
+        for (int j = 0; j < RB; j++)
+          cs[j] = (valid_o && mi < 2 && rb + j < r1) ? p.cs[(size_t)(c0 + rb + j) * half + (i & (half - 1))] : make_float2(1.0f, 0.0f);
+#pragma unroll
+        for (int j = 0; j < RB; j++) {
+          const int r = rb + j;
+          if (r >= r1 || !valid_o) continue;
           const int row = c0 + r;
-          const int seq = p.m.seq[row];
-          if (!valid_o || !good) continue;
-          float v = sumb[r * TILE_M + f];
+          const float sc = inv_s[row];
+          float v = src[(r - r0) * TILE_M + f] * sc;
           if (mi < 2) {                             // rotate-half RoPE: partner feature is f ^ half
-            float w = sumb[r * TILE_M + (f ^ half)];
-            float2 c = p.cs[(size_t)row * half + (i & (half - 1))];
-            v = (i < half) ? v * c.x - w * c.y : v * c.x + w * c.y;
+            float w = src[(r - r0) * TILE_M + (f ^ half)] * sc;
+            v = (i < half) ? v * cs[j].x - w * cs[j].y : v * cs[j].x + w * cs[j].y;
           }
           if (mi == 0) {
-            p.q[((size_t)row * p.H + head) * hd + i] = __float2bfloat16_rn(seq < 0 ? 0.0f : v);
-          } else if (seq >= 0) {
-            const int kvpos = p.m.kvpos[row];
-            if (kvpos < 0 || kvpos / p.pm.page_size >= p.pm.pages_per_seq) {
-              if (f == 0) set_status(p.status, ST_BOUNDS, 1, row, kvpos);
-              continue;
-            }
-            const int page = p.pm.table[(size_t)seq * p.pm.pages_per_seq + kvpos / p.pm.page_size];
-            if (page < 0 || page >= p.pm.num_pages) {
-              if (f == 0) set_status(p.status, ST_BOUNDS, 2, row, page);
-              continue;
-            }
-            size_t off = (((size_t)page * p.G + head) * p.pm.page_size + (kvpos % p.pm.page_size)) * hd + i;
+            p.q[((size_t)row * p.H + head) * hd + i] = __float2bfloat16_rn(seq_s[r - r0] < 0 ? 0.0f : v);
+          } else if (slot_s[r - r0] >= 0) {
+            size_t off = ((size_t)slot_s[r - r0] + (size_t)head * p.pm.page_size) * hd + i;
             (mi == 1 ? Kp : Vp)[off] = __float2bfloat16_rn(v);
           }
         }
@@ -303,12 +364,8 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
     } else if (EPI == EPI_SWIGLU) {
       for (int r = r0; r < r1; r++) {
         const int row = c0 + r;
-        uint32_t la = smem_u32(&red[r * TILE_M + f]);
-        float g = 0.0f, u = 0.0f;
-        for (int s = 0; s < Sk; s++) g += ld_peer(la, (uint32_t)s);
-        for (int s = 0; s < Sk; s++) u += ld_peer(la, (uint32_t)(Sk + s));
-        float sc = inv_s[row];
-        g *= sc; u *= sc;
+        const float sc = inv_s[row];
+        const float g = src[(r - r0) * TILE_M + f] * sc, u = src[(CHUNK / 2 + r - r0) * TILE_M + f] * sc;
         if (good && o < p.O[0]) p.act[(size_t)row * p.O[0] + o] = __float2bfloat16_rn((g / (1.0f + expf(-g))) * u);
       }
     } else {   // EPI_ARGMAX
@@ -356,9 +413,11 @@ constexpr int SMEM_TWO = 104 * 1024;      // ring budget that lets two CTAs shar
 
 struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB; };
 
-// CTAs are sized so that two of them share an SM (one CTA alone cannot hide its MMA and epilogue time
-// behind its own loads) and the grid covers all SMs about twice: S K-slices per feature tile.
-int g_target_ctas = 2 * NUM_SMS;
+// K slices per feature tile.  An SM streams at a capped rate whether one or two CTAs feed it, so the time
+// of a launch goes with (CTAs on the busiest SM) x (k-blocks per CTA + a fixed cost per CTA); two CTAs per SM
+// are needed to hide one CTA's MMA and epilogue time behind the other's loads.
+int g_target_ctas = 222;   // measured best on the 8B shapes (1.5 CTAs per SM)
+constexpr int MAX_CLUSTER = 8;
 
 Plan make_plan(FusedEpi epi, const FusedGemmArgs &a) {
   Plan pl;
@@ -367,10 +426,10 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a) {
   pl.tiles = fused_gemm_tiles(epi, a);
   const int stage = A_BYTES + pl.nt * TILE_K * 2;
   const int wmul = epi == EPI_SWIGLU ? 2 : 1;          // cluster members per K slice
-  const int smax = 8 / wmul;
+  const int smax = MAX_CLUSTER / wmul;
   int Sk = 1;
   if (epi != EPI_ARGMAX) {
-    Sk = (g_target_ctas + pl.tiles * wmul / 2) / std::max(1, pl.tiles * wmul);   // nearest
+    Sk = (g_target_ctas + pl.tiles * wmul / 2) / std::max(1, pl.tiles * wmul);   // nearest to the target CTA count
     Sk = std::max(1, std::min(Sk, smax));
     Sk = std::max(1, std::min(Sk, pl.KB / 4));
   }
@@ -384,7 +443,7 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a) {
   int per_slice = (pl.KB + Sk - 1) / Sk;
   stages = std::max(2, std::min(stages, per_slice));
   pl.stages = stages;
-  const int epi_bytes = (CHUNK * TILE_M + (epi == EPI_QKV ? CHUNK * TILE_M : 0)) * 4;
+  const int epi_bytes = 2 * CHUNK * TILE_M * 4;   // accumulator dump + reduced rows
   pl.ctrl_off = (std::max(stages * stage, epi_bytes) + 1023) & ~1023;
   pl.smem = pl.ctrl_off + 512 + 256 * 4 + 4 * CHUNK * 4 + 1024 /*alignment slack*/;
   return pl;
@@ -396,6 +455,11 @@ int launch_inst(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) 
   if (pl.smem > configured) {
     if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem) != cudaSuccess) return -6;
     configured = pl.smem;
+  }
+  static bool nonportable = false;
+  if (pl.S > 8 && !nonportable) {
+    if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return -6;
+    nonportable = true;
   }
   if (!launch_allowed()) return 0;
   cudaLaunchConfig_t cfg = {};
