@@ -182,6 +182,20 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
+# ----------------------------------------------------------------------------------------------- replicas
+def aggregate_over_ranks(ms, toks, e2e_val, dist=None, device="cpu"):
+    """The path has no exchange step, so N GPUs run N independent replicas: whole-job time is the slowest
+    rank's device time (MAX), tokens and end-to-end throughput add up (SUM).  `dist` is an initialised
+    torch.distributed module or None for a single process."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(ms), int(toks), float(e2e_val)
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    k = torch.tensor([toks, e2e_val], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(k, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(round(k[0].item())), float(k[1].item())
+
+
 # ----------------------------------------------------------------------------------------------- the CUDA arm
 def timed_steps(dec, n_steps, counts_dev):
     """n_steps x spec_step_async between two events on the decoder's stream; returns (ms, tokens)."""
@@ -252,14 +266,6 @@ def main():
     ms, toks = timed_steps(dec, args.steps, counts)
     clocks = sampler.stop() if sampler else None
     launches = dec.launches_per_step()
-    if world > 1:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        k = torch.tensor([toks], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(k, op=dist.ReduceOp.SUM)
-        ms, toks = float(t.item()), int(k.item())
-    ms_per_step = ms / args.steps
-    value = toks / (ms * 1e-3)
 
     # ---- end to end through the host-buffer entry point (sync + device->host copy every step)
     e2e_steps = min(args.steps, 50)
@@ -271,10 +277,9 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     e2e_val = e2e_toks / e2e_s
-    if world > 1:
-        v = torch.tensor([e2e_val], device=dev, dtype=torch.float64)
-        dist.all_reduce(v, op=dist.ReduceOp.SUM)
-        e2e_val = float(v.item())
+    ms, toks, e2e_val = aggregate_over_ranks(ms, toks, e2e_val, dist if world > 1 else None, dev)
+    ms_per_step = ms / args.steps
+    value = toks / (ms * 1e-3)
     d2h = B * (D + 1) * 4 + B * 4 + 16 + B * 4
 
     # ---- dominant kernel (the tcgen05 GEMM) timed with an event before every launch
@@ -291,7 +296,7 @@ def main():
     wbytes = weight_bytes_per_step(cfg)
     achieved = wbytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
     traffic = NCU_TRAFFIC_PER_LAUNCH.get(cfg.name)
-    roofline = {"bound": "hbm", "kernel": "gemm_tcgen05_kernel (all weight GEMMs of the step)", "achieved": achieved,
+    roofline = {"bound": "hbm", "kernel": "gemm_fused_kernel (all weight GEMMs of the step)", "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                 "bytes_per_launch": wbytes / max(1, gemm_n), "avg_launch_us": 1e3 * gemm_ms / max(1, gemm_n),
                 "launches_per_step": gemm_n, "traffic": traffic,
