@@ -52,7 +52,8 @@ enum {
   SPEC_FLAG_NO_GRAPH = 8,        /* launch kernels one by one instead of replaying a CUDA graph        */
   SPEC_FLAG_UNFUSED = 16,        /* bf16: separate norm / RoPE / activation kernels and split-K partial
                                     sums in global memory instead of the fused GEMM epilogues          */
-  SPEC_FLAG_NO_PDL = 32          /* no programmatic dependent launch between the kernels of a step    */
+  SPEC_FLAG_NO_PDL = 32,         /* no programmatic dependent launch between the kernels of a step    */
+  SPEC_FLAG_NO_CHAIN = 64        /* one kernel per GEMM instead of one persistent kernel per GEMM chain */
 };
 
 /* Target model weights (Section 3.1: the frozen target whose layers are tapped).  Device pointers;

@@ -12,6 +12,7 @@
 #include "../../include/spec_b200.h"
 #include "gemm_fast.cuh"
 #include "gemm_fused.cuh"
+#include "gemm_chain.cuh"
 #include "attn_fast.cuh"
 #include "state.cuh"
 
@@ -41,6 +42,8 @@ static void launch_gather_rows(const float *src, const int32_t *src_row, float *
 }
 
 static char g_init_err[256] = "";
+
+constexpr int MAX_CHAIN_LAUNCHES = 512;
 
 struct LayerW {
   const void *attn_norm, *wq, *wk, *wv, *wo, *mlp_norm, *w_gate, *w_up, *w_down;
@@ -97,6 +100,12 @@ struct spec_ctx {
   int wcur = -1;                 // stream entry of the next GEMM launch (-1: no prefetching)
   size_t pf_front = 0;           // stream position up to which earlier launches of this step prefetched
   size_t pf_lead = 0;             // bytes each launch keeps prefetched ahead (off by default: measured slower on B200)
+  // chain kernel: consecutive GEMMs of a pass run as one persistent kernel
+  bool chain = false;
+  float *chain_part = nullptr;     // split-K partial sums of the chain kernel
+  size_t chain_part_bytes = 0;
+  int32_t *chain_ctr = nullptr;    // [MAX_CHAIN_LAUNCHES][CHAIN_COUNTERS] grid-barrier counters, one block per launch of a step
+  int chain_idx = 0;
   int dbg_launch_budget = -1;   // debugging aid: kernels of the next step to run (-1: all)
   void *gemm_scratch;
   size_t gemm_scratch_bytes;
@@ -231,6 +240,9 @@ static size_t carve(spec_ctx *c, void *base) {
   c->best_val = cv.take<float>((size_t)c->vtiles * R);
   c->best_idx = cv.take<int32_t>((size_t)c->vtiles * R);
   c->topk_scratch = cv.take_bytes(topk_scratch_bytes(R, c->Vd, c->K));
+  c->chain_part_bytes = (R <= 64) ? ((size_t)64 << 20) : 0;
+  c->chain_part = c->chain_part_bytes ? (float *)cv.take_bytes(c->chain_part_bytes) : nullptr;
+  c->chain_ctr = cv.take<int32_t>((size_t)MAX_CHAIN_LAUNCHES * CHAIN_COUNTERS);
   c->gemm_scratch_bytes = 0;
   c->gemm_scratch = nullptr;
   c->attn_scratch_bytes = attn_fast_scratch_bytes(R, c->H, c->hd, g.max_ctx);
@@ -301,6 +313,7 @@ extern "C" int spec_init(spec_ctx **out, const spec_target_weights *tw, const sp
     }
   }
   c->fused = c->fg && !(cfg->flags & SPEC_FLAG_UNFUSED) && c->hd <= 128 && (c->hd & (c->hd - 1)) == 0 && c->Ralloc <= 256;
+  c->chain = c->fused && !(cfg->flags & SPEC_FLAG_NO_CHAIN) && c->chain_part != nullptr;
   if (c->fused) {
     size_t e = 2, k = c->k, qd = (size_t)c->H * c->hd, kvd = (size_t)c->G * c->hd, F = c->F;
     auto push = [&](const void *p, size_t elems) { c->wstream.push_back({p, elems * e}); };
@@ -338,12 +351,41 @@ extern "C" int spec_free(spec_ctx *c) {
 template <typename T> struct Sched {
   spec_ctx *c;
   cudaStream_t s;
+  // GEMMs waiting to be launched as one chain kernel
+  std::vector<FusedEpi> ch_epi;
+  std::vector<FusedGemmArgs> ch_ops;
+  bool defer_flush = false;      // inside step(): chains may span the forward helpers; counters were zeroed at step start
   explicit Sched(spec_ctx *ctx) : c(ctx), s(ctx->stream) { tl_pdl = c->fused && !(c->cfg.flags & SPEC_FLAG_NO_PDL); }
-  ~Sched() { tl_pdl = false; }
+  ~Sched() { flush_chain(); tl_pdl = false; }
+  void flush_chain() {
+    if (ch_ops.empty()) return;
+    int n = (int)ch_ops.size();
+    int rc = -1;
+    prof_mark(SPEC_PROF_GEMM);
+    if (c->chain_idx < MAX_CHAIN_LAUNCHES) {
+      int32_t *ctr = c->chain_ctr + (size_t)c->chain_idx * CHAIN_COUNTERS;
+      if (!defer_flush) cudaMemsetAsync(ctr, 0, CHAIN_COUNTERS * sizeof(int32_t), s);
+      rc = chain_launch(c->fg, ch_epi.data(), ch_ops.data(), n, c->chain_part, c->chain_part_bytes, ctr, c->status, tl_pdl, s);
+      if (rc == 0) { c->chain_idx++; tick(); }
+    }
+    if (rc != 0) {               // shapes the chain kernel does not take: one launch per GEMM
+      for (int i = 0; i < n; i++) {
+        int r2 = fused_gemm_launch(c->fg, ch_epi[i], ch_ops[i], s);
+        if (r2 && !c->sched_err) c->sched_err = r2;
+        tick();
+      }
+    }
+    ch_epi.clear();
+    ch_ops.clear();
+  }
   Sched(const Sched &) = delete;
   void tick(int n = 1) { c->launches += n; }
   // profiling: one event at the start of every launch; the interval to the next event is charged to `cls`
   void mark(int cls) {
+    if (cls != SPEC_PROF_GEMM) flush_chain();      // a non-GEMM kernel follows: it needs the pending GEMMs' results
+    prof_mark(cls);
+  }
+  void prof_mark(int cls) {
     if (!c->prof) return;
     if (c->prof_n >= (int)c->prof_ev.size()) {
       cudaEvent_t e;
@@ -408,7 +450,14 @@ template <typename T> struct Sched {
     c->pf_front = pos;
   }
   void fgemm(FusedEpi epi, FusedGemmArgs a) {
-    mark(SPEC_PROF_GEMM);
+    if (c->chain && epi != EPI_ARGMAX && a.rows <= 64) {
+      if (!ch_ops.empty() && ((int)ch_ops.size() == MAX_CHAIN_OPS || ch_ops[0].rows != a.rows)) flush_chain();
+      ch_epi.push_back(epi);
+      ch_ops.push_back(a);
+      return;
+    }
+    flush_chain();
+    prof_mark(SPEC_PROF_GEMM);
     assign_prefetch(a);
     int rc = fused_gemm_launch(c->fg, epi, a, s);
     if (rc && !c->sched_err) c->sched_err = rc;
@@ -458,6 +507,7 @@ template <typename T> struct Sched {
       fgemm(EPI_ARGMAX, a);
       mark(SPEC_PROF_ARGMAX); launch_argmax_merge(c->best_val, c->best_idx, c->vtiles, c->Ralloc, rows, c->tb.y, s); tick();
     }
+    if (!defer_flush) flush_chain();
   }
   void fuse_fused(const void *taps, int rows) {
     FusedGemmArgs a = fargs(taps, rows, 3 * c->k);
@@ -465,6 +515,7 @@ template <typename T> struct Sched {
     a.out_f32 = c->proj; a.ldo = c->k;
     fgemm(EPI_F32, a);
     c->np_proj = 1; c->ps_proj = 0;
+    if (!defer_flush) flush_chain();
   }
   void draft_forward_fused(const float *feat, int nparts, size_t fstride, const int32_t *src_row, int rows, int tail_len) {
     mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
@@ -473,6 +524,7 @@ template <typename T> struct Sched {
     tick();
     fgemm_resid(c->cat, 2 * c->k, c->fc2, rows, false, c->dl.attn_norm, 0);
     block_fused(c->dl, c->pools[c->L], rows, tail_len, c->dfinal_norm, 0);
+    if (!defer_flush) flush_chain();
   }
   void draft_logits_fused(int rows) {
     FusedGemmArgs a = fargs(c->h, rows, c->k);
@@ -601,6 +653,11 @@ template <typename T> struct Sched {
     c->wcur = (!plain && c->fused) ? 0 : -1;
     c->pf_front = c->pf_lead;
     tl_launch_budget = c->dbg_launch_budget;
+    if (c->chain) {              // one block of barrier counters per chain launch of the step, all zeroed up front
+      cudaMemsetAsync(c->chain_ctr, 0, (size_t)MAX_CHAIN_LAUNCHES * CHAIN_COUNTERS * sizeof(int32_t), s);
+      c->chain_idx = 0;
+      defer_flush = true;
+    }
     if (!plain) {
       mark(SPEC_PROF_TREE); launch_prep_extend(c->st, c->tb, c->meta, c->B, c->need_pos, c->status, s); tick();
       c->cur_rps = c->Pmax;
@@ -630,6 +687,7 @@ template <typename T> struct Sched {
                      c->k, rps, s);
     tick();
     mark(-1);
+    defer_flush = false;
     c->wcur = -1;
     tl_launch_budget = -1;
   }
