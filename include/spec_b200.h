@@ -53,7 +53,9 @@ enum {
   SPEC_FLAG_UNFUSED = 16,        /* bf16: separate norm / RoPE / activation kernels and split-K partial
                                     sums in global memory instead of the fused GEMM epilogues          */
   SPEC_FLAG_NO_PDL = 32,         /* no programmatic dependent launch between the kernels of a step    */
-  SPEC_FLAG_NO_CHAIN = 64        /* one kernel per GEMM instead of one persistent kernel per GEMM chain */
+  SPEC_FLAG_CHAIN = 64           /* run the GEMMs between two attention calls as ONE persistent kernel (balanced
+                                    unit ranges, partial sums through L2, grid counters) instead of one
+                                    cluster split-K kernel per GEMM; measured slower on B200, kept as an option */
 };
 
 /* Target model weights (Section 3.1: the frozen target whose layers are tapped).  Device pointers;
@@ -143,7 +145,8 @@ int spec_profile_step(spec_ctx *ctx, float *class_ms, int32_t *class_launches);
  *                         keeps prefetched in L2 (0 = no prefetch)
  *   SPEC_TUNE_GEMM_CTAS   CTAs a weight-streaming GEMM launch aims at (process-wide) */
 enum spec_tune_knob { SPEC_TUNE_L2_LEAD_MB = 1, SPEC_TUNE_GEMM_CTAS = 2,
-                      SPEC_TUNE_DEBUG_LAUNCH_BUDGET = 3 /* debugging: run only the first n kernels of each step (-1: all) */ };
+                      SPEC_TUNE_DEBUG_LAUNCH_BUDGET = 3 /* debugging: run only the first n kernels of each step (-1: all) */,
+                      SPEC_TUNE_CHAIN_TIMING = 5 /* profiling: record phase time stamps of the n-th chain launch of a step (-1: none) */ };
 int spec_tune(spec_ctx *ctx, int32_t what, int32_t value);
 
 /* Number of kernels one spec_step launches (for launch accounting). */
@@ -179,7 +182,8 @@ enum spec_debug_what {
   SPEC_DBG_PAGE_TABLE,       /* int32 [pages of seq]     */
   /* raw activation buffers of the last pass as floats, all allocated rows (debugging) */
   SPEC_DBG_RAW_X = 100, SPEC_DBG_RAW_H, SPEC_DBG_RAW_Q, SPEC_DBG_RAW_AO, SPEC_DBG_RAW_ACT, SPEC_DBG_RAW_CAT,
-  SPEC_DBG_RAW_SSQ, SPEC_DBG_RAW_LOGITS
+  SPEC_DBG_RAW_SSQ, SPEC_DBG_RAW_LOGITS,
+  SPEC_DBG_CHAIN_TIMING      /* int64 [chain CTAs][4 ops][8] globaltimer stamps (ns), see SPEC_TUNE_CHAIN_TIMING */
 };
 /* Copies up to `bytes` of item `what` of sequence `seq` (last step) to host_dst; returns bytes
  * available (>= 0) or a negative status. */

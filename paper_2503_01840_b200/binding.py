@@ -19,13 +19,13 @@ from . import build as _build
 _lib = None
 
 F32, BF16 = 0, 1
-FLAG_REF_GEMM, FLAG_REF_ATTN, FLAG_CAPTURE, FLAG_NO_GRAPH, FLAG_UNFUSED, FLAG_NO_PDL, FLAG_NO_CHAIN = 1, 2, 4, 8, 16, 32, 64
+FLAG_REF_GEMM, FLAG_REF_ATTN, FLAG_CAPTURE, FLAG_NO_GRAPH, FLAG_UNFUSED, FLAG_NO_PDL, FLAG_CHAIN = 1, 2, 4, 8, 16, 32, 64
 
 (DBG_TREE_TOK, DBG_TREE_PARENT, DBG_TREE_DEPTH, DBG_TREE_MASK, DBG_TREE_POOLIDX, DBG_TREE_SCORE, DBG_Y,
  DBG_TARGET_LOGITS, DBG_NODE_TAPS, DBG_NODE_HIDDEN, DBG_DRAFT_LOGITS, DBG_DRAFT_A, DBG_POOL_TOK, DBG_POOL_SCORE,
  DBG_POOL_PARENT, DBG_FRONTIER, DBG_PATH, DBG_STATUS, DBG_PAGE_TABLE) = range(1, 20)
-DBG_RAW_X, DBG_RAW_H, DBG_RAW_Q, DBG_RAW_AO, DBG_RAW_ACT, DBG_RAW_CAT, DBG_RAW_SSQ, DBG_RAW_LOGITS = range(100, 108)
-_DBG_DTYPE = {**{i: np.float32 for i in range(100, 108)}, DBG_TREE_TOK: np.int32, DBG_TREE_PARENT: np.int32, DBG_TREE_DEPTH: np.int32, DBG_TREE_MASK: np.uint64,
+DBG_RAW_X, DBG_RAW_H, DBG_RAW_Q, DBG_RAW_AO, DBG_RAW_ACT, DBG_RAW_CAT, DBG_RAW_SSQ, DBG_RAW_LOGITS, DBG_CHAIN_TIMING = range(100, 109)
+_DBG_DTYPE = {**{i: np.float32 for i in range(100, 108)}, DBG_CHAIN_TIMING: np.int64, DBG_TREE_TOK: np.int32, DBG_TREE_PARENT: np.int32, DBG_TREE_DEPTH: np.int32, DBG_TREE_MASK: np.uint64,
               DBG_TREE_POOLIDX: np.int32, DBG_TREE_SCORE: np.float32, DBG_Y: np.int32, DBG_TARGET_LOGITS: np.float32,
               DBG_NODE_TAPS: np.float32, DBG_NODE_HIDDEN: np.float32, DBG_DRAFT_LOGITS: np.float32,
               DBG_DRAFT_A: np.float32, DBG_POOL_TOK: np.int32, DBG_POOL_SCORE: np.float32, DBG_POOL_PARENT: np.int32,
@@ -254,7 +254,7 @@ class SpecDecoder:
         self._check(lib().spec_profile_step(self.h, ms.ctypes.data, n.ctypes.data))
         return {c: (float(ms[i]), int(n[i])) for i, c in enumerate(self.PROF_CLASSES)}
 
-    TUNE_L2_LEAD_MB, TUNE_GEMM_CTAS, TUNE_DEBUG_LAUNCH_BUDGET = 1, 2, 3
+    TUNE_L2_LEAD_MB, TUNE_GEMM_CTAS, TUNE_DEBUG_LAUNCH_BUDGET, TUNE_CHAIN_TIMING = 1, 2, 3, 5
 
     def tune(self, what: int, value: int):
         self._check(lib().spec_tune(self.h, what, value))

@@ -106,6 +106,8 @@ struct spec_ctx {
   size_t chain_part_bytes = 0;
   int32_t *chain_ctr = nullptr;    // [MAX_CHAIN_LAUNCHES][CHAIN_COUNTERS] grid-barrier counters, one block per launch of a step
   int chain_idx = 0;
+  long long *chain_timing = nullptr;   // [CTAs][MAX_CHAIN_OPS][8] phase stamps of one chain launch (profiling aid)
+  int chain_timing_launch = -1;        // index of the chain launch of a step to record (-1: none)
   int dbg_launch_budget = -1;   // debugging aid: kernels of the next step to run (-1: all)
   void *gemm_scratch;
   size_t gemm_scratch_bytes;
@@ -243,6 +245,7 @@ static size_t carve(spec_ctx *c, void *base) {
   c->chain_part_bytes = (R <= 64) ? ((size_t)64 << 20) : 0;
   c->chain_part = c->chain_part_bytes ? (float *)cv.take_bytes(c->chain_part_bytes) : nullptr;
   c->chain_ctr = cv.take<int32_t>((size_t)MAX_CHAIN_LAUNCHES * CHAIN_COUNTERS);
+  c->chain_timing = cv.take<long long>((size_t)1024 * MAX_CHAIN_OPS * 16);
   c->gemm_scratch_bytes = 0;
   c->gemm_scratch = nullptr;
   c->attn_scratch_bytes = attn_fast_scratch_bytes(R, c->H, c->hd, g.max_ctx);
@@ -313,7 +316,7 @@ extern "C" int spec_init(spec_ctx **out, const spec_target_weights *tw, const sp
     }
   }
   c->fused = c->fg && !(cfg->flags & SPEC_FLAG_UNFUSED) && c->hd <= 128 && (c->hd & (c->hd - 1)) == 0 && c->Ralloc <= 256;
-  c->chain = c->fused && !(cfg->flags & SPEC_FLAG_NO_CHAIN) && c->chain_part != nullptr;
+  c->chain = c->fused && (cfg->flags & SPEC_FLAG_CHAIN) && c->chain_part != nullptr;
   if (c->fused) {
     size_t e = 2, k = c->k, qd = (size_t)c->H * c->hd, kvd = (size_t)c->G * c->hd, F = c->F;
     auto push = [&](const void *p, size_t elems) { c->wstream.push_back({p, elems * e}); };
@@ -365,7 +368,8 @@ template <typename T> struct Sched {
     if (c->chain_idx < MAX_CHAIN_LAUNCHES) {
       int32_t *ctr = c->chain_ctr + (size_t)c->chain_idx * CHAIN_COUNTERS;
       if (!defer_flush) cudaMemsetAsync(ctr, 0, CHAIN_COUNTERS * sizeof(int32_t), s);
-      rc = chain_launch(c->fg, ch_epi.data(), ch_ops.data(), n, c->chain_part, c->chain_part_bytes, ctr, c->status, tl_pdl, s);
+      rc = chain_launch(c->fg, ch_epi.data(), ch_ops.data(), n, c->chain_part, c->chain_part_bytes, ctr, c->status, tl_pdl, s,
+                        (defer_flush && c->chain_idx == c->chain_timing_launch) ? c->chain_timing : nullptr);
       if (rc == 0) { c->chain_idx++; tick(); }
     }
     if (rc != 0) {               // shapes the chain kernel does not take: one launch per GEMM
@@ -927,6 +931,8 @@ extern "C" int spec_tune(spec_ctx *c, int32_t what, int32_t value) {
   if (what == SPEC_TUNE_L2_LEAD_MB) {
     if (value < 0 || value > 120) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the L2 prefetch distance must be 0..120 MB");
     c->pf_lead = (size_t)value << 20;
+  } else if (what == SPEC_TUNE_CHAIN_TIMING) {
+    c->chain_timing_launch = value;
   } else if (what == SPEC_TUNE_DEBUG_LAUNCH_BUDGET) {
     c->dbg_launch_budget = value;
   } else if (what == SPEC_TUNE_GEMM_CTAS) {
@@ -1028,6 +1034,7 @@ extern "C" int64_t spec_debug_read(spec_ctx *c, int32_t what, int32_t seq, void 
     case SPEC_DBG_RAW_ACT: return copy_widen(c, c->act, (size_t)c->Ralloc * c->F, dst, bytes);
     case SPEC_DBG_RAW_CAT: return copy_widen(c, c->cat, (size_t)c->Ralloc * 2 * c->k, dst, bytes);
     case SPEC_DBG_RAW_SSQ: return copy_out(c, c->ssq, (size_t)c->ktiles * c->Ralloc, dst, bytes);
+    case SPEC_DBG_CHAIN_TIMING: return copy_out(c, c->chain_timing, (size_t)chain_ctas() * MAX_CHAIN_OPS * 16, dst, bytes);
     case SPEC_DBG_RAW_LOGITS: return copy_out(c, c->logits, (size_t)c->Ralloc * c->Vd, dst, bytes);
     default: return fail(c, SPEC_ERR_INVALID_CFG, "spec_debug_read: unknown item %d", what);
   }

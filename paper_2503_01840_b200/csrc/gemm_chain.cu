@@ -47,7 +47,7 @@ struct ChainOp {
   CUtensorMap map_x;
   int epi, tiles0, tiles1, ntiles, etiles, KB, maxslots;
   int O[3];
-  long long U;                 // ntiles * KB
+  unsigned U;                  // ntiles * KB (U * P < 2^31, checked on the host, so all unit arithmetic is 32-bit)
   int Pj;                      // CTAs that take units of this op: min(P, U), so that every one of them has work
   const float *ssq_in; int ssq_in_tiles; float inv_k_in, eps;
   float *out_f32; int ldo;
@@ -64,7 +64,18 @@ struct alignas(64) ChainParams {
   float *part;
   int32_t *ctr;
   int32_t *status;
+  long long *timing;           // optional [P][MAX_CHAIN_OPS][8] globaltimer stamps (profiling aid)
 };
+
+__device__ __forceinline__ long long global_ns() {
+  long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// stamps per (CTA, op): 0 producer: activations of the op available, 1 producer: last load of the op issued,
+// 2 MMA: last MMA of the op issued, 3 drain: first accumulator ready, 4 drain: partials written,
+// 5 drain: all partials of the grid present, 6 drain: epilogue share done, 7 kernel entry
+#define CSTAMP(j, i) do { if (p.timing) p.timing[((size_t)blockIdx.x * MAX_CHAIN_OPS + (j)) * 16 + (i)] = global_ns(); } while (0)
 
 __device__ __forceinline__ int ld_acquire(const int32_t *p) {
   int v;
@@ -75,7 +86,7 @@ __device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(smem_u32(bar)), "r"(parity)
@@ -87,8 +98,18 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
 }
 __device__ __forceinline__ void bar_epi() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 // CTA that owns unit u when U units are split over P CTAs as [c U / P, (c + 1) U / P)
-__device__ __forceinline__ int owner_of(long long u, long long U, int P) { return (int)(((u + 1) * P - 1) / U); }
+__device__ __forceinline__ int owner_of(unsigned u, unsigned U, int P) { return (int)(((u + 1u) * (unsigned)P - 1u) / U); }
 
+constexpr int FLAG_BASE = 2 * MAX_CHAIN_OPS;   // ctr[FLAG_BASE + b] != 0: all CTAs arrived at barrier b
+// counts this CTA in at barrier b; the last CTA to arrive publishes the barrier's flag, which is what waiters poll
+// (a word nobody does atomics on)
+__device__ __forceinline__ void arrive_and_publish(int32_t *ctr, int b, int P) {
+  __threadfence();
+  if (atomicAdd(ctr + b, 1) == P - 1) {
+    __threadfence();
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ctr + FLAG_BASE + b), "r"(1) : "memory");
+  }
+}
 // waits until counter >= target; false on timeout or abort
 __device__ __forceinline__ bool wait_counter(const int32_t *ctr, int target, const int32_t *abort_word) {
   for (uint32_t it = 0; it < GRID_SPIN_LIMIT; it++) {
@@ -97,6 +118,172 @@ __device__ __forceinline__ bool wait_counter(const int32_t *ctr, int target, con
     __nanosleep(20);
   }
   return false;
+}
+
+
+__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c2, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c2, d);
+  return make_uint2(*(uint32_t *)&lo, *(uint32_t *)&hi);
+}
+
+// One warp's share of an op's (tile, row) items.  RB items are handled together and every global load of the
+// group (slice partial sums, norm statistics, residual, gain, RoPE angles) is issued before the first use, so a
+// group costs about one L2 round trip.  CAP = slices of one tile loaded per round.  Lane l owns features 4l..4l+3.
+template <int RB, int CAP, int NTI>
+__device__ __forceinline__ void epilogue_items(const ChainParams &p, const ChainOp &op, int P, int c, int warp, int lane,
+                                               const int32_t *slot_s, const int32_t *seq_s, long long *tm_out) {
+  const int rows = p.rows;
+  long long t_idx = 0, t_wait = 0, t_rest = 0, n_groups = 0;
+  const unsigned N = (unsigned)op.etiles * (unsigned)rows;
+  const unsigned i0 = (unsigned)c * N / (unsigned)P, i1 = (unsigned)(c + 1) * N / (unsigned)P;
+  const size_t sstride = (size_t)rows * TILE_M;              // floats between two slices of a tile
+  for (unsigned it0 = i0 + warp; it0 < i1; it0 += 4 * RB) {
+    int et[RB], row[RB], ns[RB][NTI];
+    const float *base[RB][NTI];
+    bool valid[RB];
+    float4 acc[RB][NTI];
+    float ss[RB];
+    float4 xin[RB];
+    uint2 gn[RB];
+    float4 csv[RB][2];
+    long long ta = global_ns();
+    // ---- loads
+#pragma unroll
+    for (int b = 0; b < RB; b++) {
+      const unsigned it = it0 + 4 * b;
+      valid[b] = it < i1;
+      et[b] = valid[b] ? (int)(it / (unsigned)rows) : 0;
+      row[b] = valid[b] ? (int)(it - (unsigned)et[b] * (unsigned)rows) : 0;
+      ss[b] = 0.0f;
+      xin[b] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+      gn[b] = make_uint2(0u, 0u);
+      csv[b][0] = csv[b][1] = make_float4(1.0f, 0.0f, 1.0f, 0.0f);
+#pragma unroll
+      for (int w2 = 0; w2 < NTI; w2++) {
+        acc[b][w2] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        ns[b][w2] = 0;
+        base[b][w2] = p.part;
+        if (!valid[b]) continue;
+        const int T = et[b] + w2 * op.etiles;
+        const int cf = owner_of((unsigned)T * (unsigned)op.KB, op.U, op.Pj), cl = owner_of((unsigned)(T + 1) * (unsigned)op.KB - 1u, op.U, op.Pj);
+        ns[b][w2] = cl - cf + 1;
+        base[b][w2] = p.part + (((size_t)T * op.maxslots) * rows + row[b]) * TILE_M + lane * 4;
+      }
+    }
+    long long tb = global_ns();
+    float4 v[RB][NTI][CAP];
+#pragma unroll
+    for (int b = 0; b < RB; b++)
+#pragma unroll
+      for (int w2 = 0; w2 < NTI; w2++)
+#pragma unroll
+        for (int s2 = 0; s2 < CAP; s2++)
+          if (s2 < ns[b][w2]) v[b][w2][s2] = __ldcg((const float4 *)(base[b][w2] + (size_t)s2 * sstride));
+#pragma unroll
+    for (int b = 0; b < RB; b++) {
+      if (!valid[b]) continue;
+      if (op.ssq_in)
+        for (int tt = lane; tt < op.ssq_in_tiles; tt += 32) ss[b] += __ldcg(op.ssq_in + (size_t)tt * p.ssq_ld + row[b]);
+      const int o = (op.epi == EPI_QKV ? 0 : et[b] * TILE_M) + lane * 4;
+      if (op.epi == EPI_RESID && o < op.O[0]) {
+        if (op.resid_add) xin[b] = __ldcg((const float4 *)(op.xres + (size_t)row[b] * op.O[0] + o));
+        gn[b] = *(const uint2 *)(op.gain + o);
+      } else if (op.epi == EPI_QKV && et[b] < op.tiles1) {          // q and k tiles are rotated
+        int tm = et[b] >= op.tiles0 ? et[b] - op.tiles0 : et[b];
+        const int half = op.hd >> 1, i = (tm * TILE_M + lane * 4) % op.hd;
+        const float4 *cp = (const float4 *)(op.cs + (size_t)row[b] * half + (i & (half - 1)));
+        csv[b][0] = cp[0];
+        csv[b][1] = cp[1];
+      }
+    }
+    // ---- slice sums in slice order (further rounds only for tiles cut into more than CAP slices)
+#pragma unroll
+    for (int b = 0; b < RB; b++)
+#pragma unroll
+      for (int w2 = 0; w2 < NTI; w2++) {
+#pragma unroll
+        for (int s2 = 0; s2 < CAP; s2++)
+          if (s2 < ns[b][w2]) { acc[b][w2].x += v[b][w2][s2].x; acc[b][w2].y += v[b][w2][s2].y; acc[b][w2].z += v[b][w2][s2].z; acc[b][w2].w += v[b][w2][s2].w; }
+        for (int s2 = CAP; s2 < ns[b][w2]; s2++) {
+          float4 t4 = __ldcg((const float4 *)(base[b][w2] + (size_t)s2 * sstride));
+          acc[b][w2].x += t4.x; acc[b][w2].y += t4.y; acc[b][w2].z += t4.z; acc[b][w2].w += t4.w;
+        }
+      }
+    long long tc = global_ns();
+    // ---- epilogue
+#pragma unroll
+    for (int b = 0; b < RB; b++) {
+      float sc = 1.0f;
+      if (op.ssq_in) {                                            // all lanes take part in the shuffles
+        float t = ss[b];
+        for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+        sc = 1.0f / sqrtf(t * op.inv_k_in + op.eps);
+      }
+      float v4[4] = {acc[b][0].x * sc, acc[b][0].y * sc, acc[b][0].z * sc, acc[b][0].w * sc};
+      const int r = row[b];
+      if (NTI == 1 && op.epi == EPI_F32) {
+        const int o = et[b] * TILE_M + lane * 4;
+        if (valid[b] && o < op.O[0]) *(float4 *)(op.out_f32 + (size_t)r * op.ldo + o) = make_float4(v4[0], v4[1], v4[2], v4[3]);
+      } else if (NTI == 1 && op.epi == EPI_RESID) {
+        const int o = et[b] * TILE_M + lane * 4;
+        float sq = 0.0f;
+        if (valid[b] && o < op.O[0]) {
+          const size_t xi = (size_t)r * op.O[0] + o;
+          const float x0 = xin[b].x + v4[0], x1 = xin[b].y + v4[1], x2 = xin[b].z + v4[2], x3 = xin[b].w + v4[3];
+          *(float4 *)(op.xres + xi) = make_float4(x0, x1, x2, x3);
+          const __nv_bfloat162 g01 = *(const __nv_bfloat162 *)&gn[b].x, g23 = *(const __nv_bfloat162 *)&gn[b].y;
+          *(uint2 *)(op.hb + xi) = pack4_bf16(x0 * __low2float(g01), x1 * __high2float(g01), x2 * __low2float(g23), x3 * __high2float(g23));
+          if (op.tap_mask) {
+            const uint2 tp = pack4_bf16(x0, x1, x2, x3);
+#pragma unroll
+            for (int s2 = 0; s2 < 3; s2++)
+              if ((op.tap_mask >> s2) & 1) *(uint2 *)(op.taps + (size_t)r * 3 * op.O[0] + (size_t)s2 * op.O[0] + o) = tp;
+          }
+          sq = x0 * x0 + x1 * x1 + x2 * x2 + x3 * x3;
+        }
+        for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+        if (valid[b] && lane == 0) op.ssq_out[(size_t)et[b] * p.ssq_ld + r] = sq;
+      } else if (NTI == 2) {
+        const int o = et[b] * TILE_M + lane * 4;
+        const float u4[4] = {acc[b][NTI - 1].x * sc, acc[b][NTI - 1].y * sc, acc[b][NTI - 1].z * sc, acc[b][NTI - 1].w * sc};
+        if (valid[b] && o < op.O[0]) {
+          float a4[4];
+#pragma unroll
+          for (int e = 0; e < 4; e++) a4[e] = (v4[e] / (1.0f + expf(-v4[e]))) * u4[e];
+          *(uint2 *)(op.act + (size_t)r * op.O[0] + o) = pack4_bf16(a4[0], a4[1], a4[2], a4[3]);
+        }
+      } else if (NTI == 1 && op.epi == EPI_QKV) {
+        int mi = 0, tm = et[b];
+        if (tm >= op.tiles1) { mi = 2; tm -= op.tiles1; }
+        else if (tm >= op.tiles0) { mi = 1; tm -= op.tiles0; }
+        const int hd = op.hd, half = hd >> 1;
+        const int o = tm * TILE_M + lane * 4;                  // feature within weight mi; 4 features stay in one half
+        const int head = o / hd, i = o % hd;
+        float w4[4];
+#pragma unroll
+        for (int e = 0; e < 4; e++) w4[e] = __shfl_xor_sync(0xffffffffu, v4[e], half >> 2);   // rotate-half partner
+        if (valid[b] && o < op.O[mi]) {
+          if (mi < 2) {
+            const float cc[4] = {csv[b][0].x, csv[b][0].z, csv[b][1].x, csv[b][1].z}, sn[4] = {csv[b][0].y, csv[b][0].w, csv[b][1].y, csv[b][1].w};
+#pragma unroll
+            for (int e = 0; e < 4; e++) v4[e] = (i < half) ? v4[e] * cc[e] - w4[e] * sn[e] : v4[e] * cc[e] + w4[e] * sn[e];
+          }
+          const int seq = seq_s[r];
+          if (mi == 0) {
+            const bool z = seq < 0;
+            *(uint2 *)(op.q + ((size_t)r * op.H + head) * hd + i) = pack4_bf16(z ? 0.0f : v4[0], z ? 0.0f : v4[1], z ? 0.0f : v4[2], z ? 0.0f : v4[3]);
+          } else if (slot_s[r] >= 0) {
+            const int kvpos = p.m.kvpos[r];
+            const size_t off = (((size_t)slot_s[r] * op.G + head) * p.pm.page_size + (kvpos % p.pm.page_size)) * hd + i;
+            *(uint2 *)((bf16 *)(mi == 1 ? op.pool.k : op.pool.v) + off) = pack4_bf16(v4[0], v4[1], v4[2], v4[3]);
+          }
+        }
+      }
+    }
+    long long td = global_ns();
+    t_idx += tb - ta; t_wait += tc - tb; t_rest += td - tc; n_groups++;
+  }
+  if (tm_out && warp == 0 && lane == 0) { tm_out[8] = t_idx; tm_out[9] = t_wait; tm_out[10] = t_rest; tm_out[11] = n_groups; }
 }
 
 template <int NT>
@@ -137,6 +324,7 @@ __global__ void __launch_bounds__(192, 2) chain_kernel(const __grid_constant__ C
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) CSTAMP(0, 7);
 
   if (warp == 4) {
     // ================================================================== producer
@@ -144,32 +332,33 @@ __global__ void __launch_bounds__(192, 2) chain_kernel(const __grid_constant__ C
       const uint64_t pol = l2_policy_evict_first();
       int kbs[MAX_STAGES];                       // k-block held by each stage (for deferred activation loads)
       const CUtensorMap *xmap[MAX_STAGES];
-      long long g = 0;                           // stage items issued so far (all ops)
+      unsigned g = 0;                            // stage items issued so far (all ops)
       bool dead = false;
       for (int j = 0; j < p.nops && !dead; j++) {
         const ChainOp &op = p.op[j];
-        const long long u0 = c < op.Pj ? (long long)c * op.U / op.Pj : op.U, u1 = c < op.Pj ? (long long)(c + 1) * op.U / op.Pj : op.U;
+        const unsigned u0 = c < op.Pj ? (unsigned)c * op.U / (unsigned)op.Pj : op.U, u1 = c < op.Pj ? (unsigned)(c + 1) * op.U / (unsigned)op.Pj : op.U;
         bool dep_ok = false;
-        long long pend_lo = g;                   // first item of this op whose activation tile is not issued yet
-        auto dep_ready = [&]() -> bool { return j > 0 && ld_acquire(p.ctr + 2 * (j - 1) + 1) >= P; };
+        unsigned pend_lo = g;                    // first item of this op whose activation tile is not issued yet
+        auto dep_ready = [&]() -> bool { return j > 0 && ld_acquire(p.ctr + FLAG_BASE + 2 * (j - 1) + 1) != 0; };
         auto dep_wait = [&]() -> bool {
           if (j == 0) { pdl_wait(); return true; }
-          return wait_counter(p.ctr + 2 * (j - 1) + 1, P, abort_word);
+          return wait_counter(p.ctr + FLAG_BASE + 2 * (j - 1) + 1, 1, abort_word);
         };
         auto flush_b = [&]() {
           asm volatile("fence.proxy.async;" ::: "memory");   // other CTAs' generic-proxy stores -> this CTA's TMA reads
-          for (long long gi = pend_lo; gi < g; gi++) {
-            int st = (int)(gi % stages);
+          for (unsigned gi = pend_lo; gi < g; gi++) {
+            int st = (int)(gi % (unsigned)stages);
             tma_load_2d(tiles + st * STAGE + A_BYTES, xmap[st], kbs[st] * TILE_K, 0, &full[st]);
           }
           pend_lo = g;
+          CSTAMP(j, 0);
         };
-        int t = (int)(u0 / op.KB), kb = (int)(u0 - (long long)t * op.KB);
-        for (long long u = u0; u < u1 && !dead; u++) {
-          const int st = (int)(g % stages);
-          if (g >= stages) {
-            const uint32_t par = (uint32_t)(((g / stages) - 1) & 1);
-            if (!dep_ok && g - stages >= pend_lo) {
+        int t = (int)(u0 / (unsigned)op.KB), kb = (int)(u0 - (unsigned)t * (unsigned)op.KB);
+        for (unsigned u = u0; u < u1 && !dead; u++) {
+          const int st = (int)(g % (unsigned)stages);
+          if (g >= (unsigned)stages) {
+            const uint32_t par = ((g / (unsigned)stages) - 1u) & 1u;
+            if (!dep_ok && g - (unsigned)stages >= pend_lo) {
               // the stage still holds an item of this op that waits for its activations: resolve the dependency first
               if (!dep_wait()) { dead = true; break; }
               dep_ok = true;
@@ -194,6 +383,7 @@ __global__ void __launch_bounds__(192, 2) chain_kernel(const __grid_constant__ C
           else if (dep_ok) { tma_load_2d(tiles + st * STAGE + A_BYTES, &op.map_x, kb * TILE_K, 0, &full[st]); pend_lo = g; }
           if (++kb == op.KB) { kb = 0; t++; }
         }
+        CSTAMP(j, 1);
         if (!dead && !dep_ok) {
           if (!dep_wait()) { dead = true; set_status(p.status, ST_TIMEOUT, 301, c, j); }
           else { dep_ok = true; flush_b(); }
@@ -205,22 +395,22 @@ __global__ void __launch_bounds__(192, 2) chain_kernel(const __grid_constant__ C
     // ================================================================== MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc(NT);
-      long long g = 0;
+      unsigned g = 0;
       int pc = 0;                                // tile fragments processed so far
       bool dead = false;
       for (int j = 0; j < p.nops && !dead; j++) {
         const ChainOp &op = p.op[j];
-        const long long u0 = c < op.Pj ? (long long)c * op.U / op.Pj : op.U, u1 = c < op.Pj ? (long long)(c + 1) * op.U / op.Pj : op.U;
-        long long u = u0;
-        int kb_lo = (int)(u0 % op.KB);
+        const unsigned u0 = c < op.Pj ? (unsigned)c * op.U / (unsigned)op.Pj : op.U, u1 = c < op.Pj ? (unsigned)(c + 1) * op.U / (unsigned)op.Pj : op.U;
+        unsigned u = u0;
+        int kb_lo = (int)(u0 % (unsigned)op.KB);
         while (u < u1 && !dead) {
-          const int kb_hi = (int)std::min<long long>(op.KB, kb_lo + (u1 - u));
+          const int kb_hi = (int)min((unsigned)op.KB, (unsigned)kb_lo + (u1 - u));
           const int buf = pc & 1;
           if (pc >= 2 && !mbar_wait(&acc_empty[buf], (uint32_t)(((pc >> 1) - 1) & 1))) { dead = true; set_status(p.status, ST_TIMEOUT, 310, c, j); break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           for (int kb = kb_lo; kb < kb_hi; kb++) {
-            const int st = (int)(g % stages);
-            if (!mbar_wait(&full[st], (uint32_t)((g / stages) & 1)) || *abort_flag) { dead = true; set_status(p.status, ST_TIMEOUT, 311, c, j); break; }
+            const int st = (int)(g % (unsigned)stages);
+            if (!mbar_wait(&full[st], ((g / (unsigned)stages) & 1u)) || *abort_flag) { dead = true; set_status(p.status, ST_TIMEOUT, 311, c, j); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t a = smem_u32(tiles + st * STAGE), b = a + A_BYTES;
 #pragma unroll
@@ -236,6 +426,7 @@ __global__ void __launch_bounds__(192, 2) chain_kernel(const __grid_constant__ C
           u += kb_hi - kb_lo;
           kb_lo = 0;
         }
+        CSTAMP(j, 2);
       }
       if (dead) { *abort_flag = 1; atomicExch(p.ctr + ABORT_WORD, 1); }
     }
@@ -265,17 +456,18 @@ __global__ void __launch_bounds__(192, 2) chain_kernel(const __grid_constant__ C
     bool dead = false;
     for (int j = 0; j < p.nops; j++) {
       const ChainOp &op = p.op[j];
-      const long long u0 = c < op.Pj ? (long long)c * op.U / op.Pj : op.U, u1 = c < op.Pj ? (long long)(c + 1) * op.U / op.Pj : op.U;
+      const unsigned u0 = c < op.Pj ? (unsigned)c * op.U / (unsigned)op.Pj : op.U, u1 = c < op.Pj ? (unsigned)(c + 1) * op.U / (unsigned)op.Pj : op.U;
       // ---- 1. fragment partial sums -> scratch
       {
-        long long u = u0;
-        int t = (int)(u0 / op.KB), kb_lo = (int)(u0 - (long long)t * op.KB);
+        unsigned u = u0;
+        int t = (int)(u0 / (unsigned)op.KB), kb_lo = (int)(u0 - (unsigned)t * (unsigned)op.KB);
         while (u < u1 && !dead) {
-          const int kb_hi = (int)std::min<long long>(op.KB, kb_lo + (u1 - u));
+          const int kb_hi = (int)min((unsigned)op.KB, (unsigned)kb_lo + (u1 - u));
           const int buf = pc & 1;
           if (!mbar_wait(&acc_full[buf], (uint32_t)((pc >> 1) & 1)) || *abort_flag) { dead = true; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const int slot = c - owner_of((long long)t * op.KB, op.U, op.Pj);
+          if (threadIdx.x == 0 && u == u0) CSTAMP(j, 3);
+          const int slot = c - owner_of((unsigned)t * (unsigned)op.KB, op.U, op.Pj);
           float *dst = p.part + (((size_t)t * op.maxslots + slot) * rows) * TILE_M + threadIdx.x;
 #pragma unroll 1
           for (int cc = 0; cc < rows; cc += 16) {
@@ -297,117 +489,29 @@ __global__ void __launch_bounds__(192, 2) chain_kernel(const __grid_constant__ C
       // ---- 2. all partial sums of the op are in memory (grid-wide)
       __threadfence();
       bar_epi();
-      if (threadIdx.x == 0) atomicAdd(p.ctr + 2 * j, 1);
-      if (!dead && lane == 0) dead = !wait_counter(p.ctr + 2 * j, P, abort_word);
-      dead = __shfl_sync(0xffffffffu, dead ? 1 : 0, 0) != 0;
+      if (threadIdx.x == 0) {
+        arrive_and_publish(p.ctr, 2 * j, P);
+        CSTAMP(j, 4);
+        if (!wait_counter(p.ctr + FLAG_BASE + 2 * j, 1, abort_word)) *abort_flag = 1;
+      }
+      bar_epi();
+      dead = dead || *abort_flag != 0;
+      if (threadIdx.x == 0) CSTAMP(j, 5);
       // ---- 3. this warp's share of the (tile, row) items: reduce in slice order + epilogue
       if (!dead) {
-        const long long N = (long long)op.etiles * rows;
-        const long long i0 = (long long)c * N / P, i1 = (long long)(c + 1) * N / P;
-        const size_t sstride = (size_t)rows * TILE_M;              // floats between two slices of a tile
-        for (long long it = i0 + warp; it < i1; it += 4) {
-          const int et = (int)(it / rows), row = (int)(it - (long long)et * rows);
-          // slices of the tile(s) of this item
-          float4 acc[2];
-          const int nt_item = op.epi == EPI_SWIGLU ? 2 : 1;
-#pragma unroll
-          for (int w2 = 0; w2 < 2; w2++) {
-            acc[w2] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            if (w2 >= nt_item) continue;
-            const int T = et + w2 * op.etiles;
-            const int cf = owner_of((long long)T * op.KB, op.U, op.Pj), cl = owner_of((long long)(T + 1) * op.KB - 1, op.U, op.Pj);
-            const int ns = cl - cf + 1;
-            const float *base = p.part + (((size_t)T * op.maxslots) * rows + row) * TILE_M + lane * 4;
-            for (int s0 = 0; s0 < ns; s0 += 8) {
-              float4 v[8];
-#pragma unroll
-              for (int s = 0; s < 8; s++)
-                if (s0 + s < ns) v[s] = __ldcg((const float4 *)(base + (size_t)(s0 + s) * sstride));
-#pragma unroll
-              for (int s = 0; s < 8; s++)
-                if (s0 + s < ns) { acc[w2].x += v[s].x; acc[w2].y += v[s].y; acc[w2].z += v[s].z; acc[w2].w += v[s].w; }
-            }
-          }
-          // per-row scale of the input (RMSNorm factor), every lane gets the total
-          float sc = 1.0f;
-          if (op.ssq_in) {
-            float ss = 0.0f;
-            for (int tt = lane; tt < op.ssq_in_tiles; tt += 32) ss += __ldcg(op.ssq_in + (size_t)tt * p.ssq_ld + row);
-            for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
-            sc = 1.0f / sqrtf(ss * op.inv_k_in + op.eps);
-          }
-          float v4[4] = {acc[0].x * sc, acc[0].y * sc, acc[0].z * sc, acc[0].w * sc};
-          if (op.epi == EPI_F32) {
-            const int o = et * TILE_M + lane * 4;
-#pragma unroll
-            for (int e = 0; e < 4; e++)
-              if (o + e < op.O[0]) op.out_f32[(size_t)row * op.ldo + o + e] = v4[e];
-          } else if (op.epi == EPI_RESID) {
-            const int o = et * TILE_M + lane * 4;
-            float sq = 0.0f;
-#pragma unroll
-            for (int e = 0; e < 4; e++) {
-              if (o + e < op.O[0]) {
-                const size_t xi = (size_t)row * op.O[0] + o + e;
-                const float xo = (op.resid_add ? __ldcg(op.xres + xi) : 0.0f) + v4[e];
-                op.xres[xi] = xo;
-                op.hb[xi] = __float2bfloat16_rn(xo * __bfloat162float(op.gain[o + e]));
-                if (op.tap_mask) {
-#pragma unroll
-                  for (int s = 0; s < 3; s++)
-                    if ((op.tap_mask >> s) & 1) op.taps[(size_t)row * 3 * op.O[0] + (size_t)s * op.O[0] + o + e] = __float2bfloat16_rn(xo);
-                }
-                sq += xo * xo;
-              }
-            }
-            for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
-            if (lane == 0) op.ssq_out[(size_t)et * p.ssq_ld + row] = sq;
-          } else if (op.epi == EPI_SWIGLU) {
-            const int o = et * TILE_M + lane * 4;
-            const float u4[4] = {acc[1].x * sc, acc[1].y * sc, acc[1].z * sc, acc[1].w * sc};
-#pragma unroll
-            for (int e = 0; e < 4; e++)
-              if (o + e < op.O[0]) op.act[(size_t)row * op.O[0] + o + e] = __float2bfloat16_rn((v4[e] / (1.0f + expf(-v4[e]))) * u4[e]);
-          } else if (op.epi == EPI_QKV) {
-            int mi = 0, tm = et;
-            if (tm >= op.tiles1) { mi = 2; tm -= op.tiles1; }
-            else if (tm >= op.tiles0) { mi = 1; tm -= op.tiles0; }
-            const int hd = op.hd, half = hd >> 1;
-            const int o = tm * TILE_M + lane * 4;                  // feature within weight mi; 4 features stay in one half
-            const int head = o / hd, i = o % hd;
-            if (mi < 2) {                                          // rotate-half RoPE: partner features sit half/4 lanes away
-              float w4[4];
-#pragma unroll
-              for (int e = 0; e < 4; e++) w4[e] = __shfl_xor_sync(0xffffffffu, v4[e], half >> 2);
-              if (o < op.O[mi]) {
-#pragma unroll
-                for (int e = 0; e < 4; e++) {
-                  const float2 cs = op.cs[(size_t)row * half + ((i + e) & (half - 1))];
-                  v4[e] = (i < half) ? v4[e] * cs.x - w4[e] * cs.y : v4[e] * cs.x + w4[e] * cs.y;
-                }
-              }
-            }
-            if (o < op.O[mi]) {
-              const int seq = seq_s[row];
-              if (mi == 0) {
-#pragma unroll
-                for (int e = 0; e < 4; e++) op.q[((size_t)row * op.H + head) * hd + i + e] = __float2bfloat16_rn(seq < 0 ? 0.0f : v4[e]);
-              } else if (slot_s[row] >= 0) {
-                const int kvpos = p.m.kvpos[row];
-                const size_t off = (((size_t)slot_s[row] * op.G + head) * p.pm.page_size + (kvpos % p.pm.page_size)) * hd + i;
-                bf16 *dst = (bf16 *)(mi == 1 ? op.pool.k : op.pool.v) + off;
-#pragma unroll
-                for (int e = 0; e < 4; e++) dst[e] = __float2bfloat16_rn(v4[e]);
-              }
-            }
-          }
+        if (op.epi == EPI_SWIGLU) {
+          if (op.maxslots <= 3) epilogue_items<2, 3, 2>(p, op, P, c, warp, lane, slot_s, seq_s, p.timing ? p.timing + ((size_t)blockIdx.x * MAX_CHAIN_OPS + j) * 16 : nullptr);
+          else epilogue_items<1, 6, 2>(p, op, P, c, warp, lane, slot_s, seq_s, p.timing ? p.timing + ((size_t)blockIdx.x * MAX_CHAIN_OPS + j) * 16 : nullptr);
+        } else {
+          if (op.maxslots <= 6) epilogue_items<2, 6, 1>(p, op, P, c, warp, lane, slot_s, seq_s, p.timing ? p.timing + ((size_t)blockIdx.x * MAX_CHAIN_OPS + j) * 16 : nullptr);
+          else epilogue_items<1, 12, 1>(p, op, P, c, warp, lane, slot_s, seq_s, p.timing ? p.timing + ((size_t)blockIdx.x * MAX_CHAIN_OPS + j) * 16 : nullptr);
         }
       }
       // ---- 4. outputs of the op are complete (grid-wide): the producers may load the next op's activations
       asm volatile("fence.proxy.async;" ::: "memory");
       __threadfence();
       bar_epi();
-      if (threadIdx.x == 0) atomicAdd(p.ctr + 2 * j + 1, 1);
+      if (threadIdx.x == 0) { arrive_and_publish(p.ctr, 2 * j + 1, P); CSTAMP(j, 6); }
     }
     if (dead && lane == 0) { *abort_flag = 1; atomicExch(p.ctr + ABORT_WORD, 1); set_status(p.status, ST_TIMEOUT, 320, c, 0); }
   }
@@ -441,6 +545,8 @@ int max_slots(int ntiles, int KB, int P) {
 
 }  // namespace
 
+int chain_ctas() { return pick_P(); }
+
 bool chain_supported(const FusedEpi *epi, const FusedGemmArgs *ops, int nops) {
   if (nops < 1 || nops > MAX_CHAIN_OPS) return false;
   for (int j = 0; j < nops; j++) {
@@ -448,6 +554,10 @@ bool chain_supported(const FusedEpi *epi, const FusedGemmArgs *ops, int nops) {
     if (ops[j].rows != ops[0].rows || ops[j].rows > 64) return false;
     if (epi[j] == EPI_QKV && (ops[j].hd < 16)) return false;
     if (epi[j] == EPI_F32 && (ops[j].ldo % 4)) return false;
+    for (int w = 0; w < ops[j].nw; w++)
+      if (ops[j].O[w] % 4) return false;                       // a lane's four features are stored as one vector
+    long long U = (long long)ntiles_of(epi[j], ops[j]) * ((ops[j].I + TILE_K - 1) / TILE_K);
+    if ((U + 1) * pick_P() >= (1ll << 31) || (long long)ntiles_of(epi[j], ops[j]) * 64 * pick_P() >= (1ll << 31)) return false;
   }
   return true;
 }
@@ -464,7 +574,7 @@ size_t chain_scratch_bytes(const FusedEpi *epi, const FusedGemmArgs *ops, int no
 }
 
 int chain_launch(FastGemm *g, const FusedEpi *epi, const FusedGemmArgs *ops, int nops, float *scratch, size_t scratch_bytes,
-                 int32_t *counters, int32_t *status, bool pdl, cudaStream_t s) {
+                 int32_t *counters, int32_t *status, bool pdl, cudaStream_t s, long long *timing) {
   if (!g || !chain_supported(epi, ops, nops) || !scratch || !counters) return -1;
   if (chain_scratch_bytes(epi, ops, nops) > scratch_bytes) return -3;
   static ChainParams p;                          // ~5 KB: kept off the stack; launches are issued by one host thread at a time
@@ -489,8 +599,8 @@ int chain_launch(FastGemm *g, const FusedEpi *epi, const FusedGemmArgs *ops, int
     o.ntiles = ntiles_of(epi[j], a);
     o.etiles = epi[j] == EPI_SWIGLU ? o.tiles0 : o.ntiles;
     o.KB = (a.I + TILE_K - 1) / TILE_K;
-    o.U = (long long)o.ntiles * o.KB;
-    o.Pj = (int)std::min<long long>(P, o.U);
+    o.U = (unsigned)o.ntiles * (unsigned)o.KB;
+    o.Pj = (int)std::min<long long>(P, (long long)o.U);
     o.maxslots = max_slots(o.ntiles, o.KB, o.Pj);
     o.ssq_in = a.ssq_in; o.ssq_in_tiles = a.ssq_in_tiles; o.inv_k_in = 1.0f / (float)a.k_in; o.eps = a.eps;
     o.out_f32 = a.out_f32; o.ldo = a.ldo;
@@ -505,7 +615,7 @@ int chain_launch(FastGemm *g, const FusedEpi *epi, const FusedGemmArgs *ops, int
   p.stages = std::max(2, std::min(MAX_STAGES, (100 * 1024) / stage));
   p.ctrl_off = (p.stages * stage + 1023) & ~1023;
   const int smem = p.ctrl_off + 512 + 2 * 64 * 4 + 1024;
-  p.nops = nops; p.rows = rows; p.part = scratch; p.ctr = counters; p.status = status;
+  p.nops = nops; p.rows = rows; p.part = scratch; p.ctr = counters; p.status = status; p.timing = timing;
   static int configured_nt[2] = {0, 0};          // the two instantiations have the same function type: one slot each
   auto launch = [&](auto kern) -> int {
     int &configured = configured_nt[nt == 16 ? 0 : 1];

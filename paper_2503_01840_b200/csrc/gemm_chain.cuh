@@ -16,6 +16,8 @@ size_t chain_scratch_bytes(const FusedEpi *epi, const FusedGemmArgs *ops, int no
 // counters: CHAIN_COUNTERS zeroed int32 words owned by this launch (zeroed by the caller before the launch runs).
 // meta / pm: row metadata and page map shared by the ops with an EPI_QKV epilogue.  Returns 0 or a negative code.
 int chain_launch(FastGemm *g, const FusedEpi *epi, const FusedGemmArgs *ops, int nops, float *scratch, size_t scratch_bytes,
-                 int32_t *counters, int32_t *status, bool pdl, cudaStream_t s);
+                 int32_t *counters, int32_t *status, bool pdl, cudaStream_t s, long long *timing = nullptr);
+// CTAs of a chain launch
+int chain_ctas();
 
 }  // namespace spec

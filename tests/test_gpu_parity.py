@@ -146,7 +146,8 @@ def test_c1_full_trajectory_fp32(flags):
     assert st.tokens >= 32 and st.exact_tree >= 1 and st.same_tree >= 24 and st.exact_out >= 24
 
 
-@pytest.mark.parametrize("flags", [0, sb.FLAG_NO_PDL | sb.FLAG_NO_GRAPH, sb.FLAG_UNFUSED, sb.FLAG_REF_GEMM | sb.FLAG_REF_ATTN])
+@pytest.mark.parametrize("flags", [0, sb.FLAG_NO_PDL | sb.FLAG_NO_GRAPH, sb.FLAG_CHAIN, sb.FLAG_CHAIN | sb.FLAG_NO_GRAPH, sb.FLAG_UNFUSED,
+                                   sb.FLAG_REF_GEMM | sb.FLAG_REF_ATTN])
 def test_tiny_bf16_trajectory(flags):
     tw, dw = _weights(T1)
     prompts = [p.numpy() for p in synth.make_prompts(T1)]
@@ -155,10 +156,11 @@ def test_tiny_bf16_trajectory(flags):
     assert st.same_tree >= 4
 
 
-def test_small_bf16_hd128_trajectory():
+@pytest.mark.parametrize("flags", [0, sb.FLAG_CHAIN])
+def test_small_bf16_hd128_trajectory(flags):
     tw, dw = _weights(T2)
     prompts = [p.numpy() for p in synth.make_prompts(T2)]
-    st, _ = parity.run_trajectory(T2, tw, dw, prompts, n_steps=10, tol=2e-2, tap_tol=3e-2)
+    st, _ = parity.run_trajectory(T2, tw, dw, prompts, n_steps=10, tol=2e-2, tap_tol=3e-2, flags=flags)
     print("T2", st)
 
 
@@ -266,12 +268,13 @@ def test_plain_decode_matches_oracle_greedy():
     dec.close()
 
 
-def test_c2_two_layer_truncation_first_steps():
+@pytest.mark.parametrize("flags", [0, sb.FLAG_CHAIN])
+def test_c2_two_layer_truncation_first_steps(flags):
     """8B-shaped widths (hidden 4096, 32/8 heads of 128, FFN 14336, vocab 128256 / 32000, depth 6, top-k 10,
     60 nodes) on a 2-layer truncation, first steps, bf16."""
     cfg = synth.C2.truncated(2, prompt_len=48)
     tw = synth.make_target_weights(cfg, device="cuda")
     dw = synth.make_draft_weights(cfg, device="cuda")
     prompts = [p.numpy() for p in synth.make_prompts(cfg)]
-    st, _ = parity.run_trajectory(cfg, parity.to_cpu(tw), parity.to_cpu(dw), prompts, n_steps=2, tol=2e-2, tap_tol=3e-2)
+    st, _ = parity.run_trajectory(cfg, parity.to_cpu(tw), parity.to_cpu(dw), prompts, n_steps=2, tol=2e-2, tap_tol=3e-2, flags=flags)
     print("C2-L2", st)
