@@ -53,6 +53,7 @@ enum {
   SPEC_FLAG_UNFUSED = 16,        /* bf16: separate norm / RoPE / activation kernels and split-K partial
                                     sums in global memory instead of the fused GEMM epilogues          */
   SPEC_FLAG_NO_PDL = 32,         /* no programmatic dependent launch between the kernels of a step    */
+  SPEC_FLAG_NO_TMA_ATTN = 128,   /* attention K/V tiles through cp.async instead of TMA page copies             */
   SPEC_FLAG_CHAIN = 64           /* run the GEMMs between two attention calls as ONE persistent kernel (balanced
                                     unit ranges, partial sums through L2, grid counters) instead of one
                                     cluster split-K kernel per GEMM; measured slower on B200, kept as an option */
@@ -213,7 +214,9 @@ int spec_gemm_fused(const void *x, const void *w, float *out_f32, int32_t rows, 
  * more sequences.  q [rows][H][hd] dtype; K/V pools [num_pages][G][page_size][hd] dtype;
  * page_table int32 [n_seq][pages_per_seq]; per row: seq, ctx_len (positions 0..ctx_len-1 all visible),
  * tail_base (first tail position), mask lo/hi (bit t: tail position tail_base+t visible);
- * out [rows][H][hd] dtype.  impl 0: tensor-core kernel (bf16), 1: plain kernel.
+ * out [rows][H][hd] dtype.  impl 0: tensor-core kernel (bf16), 1: plain kernel, 2: tensor-core kernel with
+ * TMA-staged K/V pages (bf16; needs row_tail_base[r] == row_ctx[r] for every row and page_size 16, 32 or 64;
+ * other shapes fall back to impl 0).
  * scratch: spec_attn_scratch_bytes(...) bytes of device memory for split-KV partial results. */
 size_t spec_attn_scratch_bytes(int32_t rows, int32_t n_heads, int32_t head_dim, int32_t max_ctx);
 int spec_attention(int32_t dtype, int32_t impl, const void *q, const void *k_pool, const void *v_pool,

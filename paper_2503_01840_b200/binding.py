@@ -19,7 +19,7 @@ from . import build as _build
 _lib = None
 
 F32, BF16 = 0, 1
-FLAG_REF_GEMM, FLAG_REF_ATTN, FLAG_CAPTURE, FLAG_NO_GRAPH, FLAG_UNFUSED, FLAG_NO_PDL, FLAG_CHAIN = 1, 2, 4, 8, 16, 32, 64
+FLAG_REF_GEMM, FLAG_REF_ATTN, FLAG_CAPTURE, FLAG_NO_GRAPH, FLAG_UNFUSED, FLAG_NO_PDL, FLAG_CHAIN, FLAG_NO_TMA_ATTN = 1, 2, 4, 8, 16, 32, 64, 128
 
 (DBG_TREE_TOK, DBG_TREE_PARENT, DBG_TREE_DEPTH, DBG_TREE_MASK, DBG_TREE_POOLIDX, DBG_TREE_SCORE, DBG_Y,
  DBG_TARGET_LOGITS, DBG_NODE_TAPS, DBG_NODE_HIDDEN, DBG_DRAFT_LOGITS, DBG_DRAFT_A, DBG_POOL_TOK, DBG_POOL_SCORE,

@@ -551,7 +551,7 @@ template <typename T> struct Sched {
       int hint = 0;
       for (int b = 0; b < c->B; b++) hint = std::max(hint, c->n_upper[b]);
       tick(launch_attn_fast((const bf16 *)c->q, pool, pm, c->meta, tail_len, (bf16 *)c->ao, rows, c->H, c->G, c->hd,
-                            c->cur_rps, hint, c->attn_scratch, s));
+                            c->cur_rps, hint, c->attn_scratch, s, !(c->cfg.flags & SPEC_FLAG_NO_TMA_ATTN), c->status));
     } else {
       launch_attn_ref<T>((const T *)c->q, pool, pm, c->meta, tail_len, (T *)c->ao, rows, c->H, c->G, c->hd,
                          c->cfg.max_ctx + tail_len, s);
@@ -1114,6 +1114,7 @@ extern "C" int spec_attention(int32_t dtype, int32_t impl, const void *q, const 
   m.mask_lo = (uint64_t *)row_mask_lo; m.mask_hi = (uint64_t *)row_mask_hi;
   KvPool pool{(void *)k_pool, (void *)v_pool};
   PageMap pm{page_table, pages_per_seq, page_size, 1 << 30};
+  if (impl < 0 || impl > 2) return SPEC_ERR_INVALID_CFG;
   if (impl == 1) {
     if (dtype == SPEC_F32) launch_attn_ref<float>((const float *)q, pool, pm, m, tail_len, (float *)out, rows, H, G, hd, max_ctx + tail_len, s);
     else if (dtype == SPEC_BF16) launch_attn_ref<bf16>((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, max_ctx + tail_len, s);
@@ -1121,7 +1122,8 @@ extern "C" int spec_attention(int32_t dtype, int32_t impl, const void *q, const 
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
   }
   if (dtype != SPEC_BF16 || !attn_fast_supported(hd, H / G)) return SPEC_ERR_UNSUPPORTED;
-  launch_attn_fast((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, 1, max_ctx, scratch, s);
+  launch_attn_fast((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, 1, max_ctx, scratch, s, impl == 2, nullptr);
+  attn_fast_forget_maps();
   return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }
 

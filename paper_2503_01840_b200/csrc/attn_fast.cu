@@ -11,6 +11,11 @@
 
 #include <mutex>
 
+#include <cuda.h>
+
+#include <map>
+#include <tuple>
+
 #include "attn_fast.cuh"
 
 namespace spec {
@@ -238,6 +243,249 @@ __global__ void __launch_bounds__(256) attn_mma_kernel(AttnParams p) {
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// TMA-staged variant.  One page of one KV head ([page_size][hd], contiguous) is fetched by ONE tensor copy
+// (cp.async.bulk.tensor, 128-byte swizzle) per K and per V; a producer warp keeps STAGES 64-key tiles in flight
+// through full/empty mbarriers, eight consumer warps run the tensor-core math of the kernel above.  Needs the
+// tail keys to follow the context directly (tail_base == ctx, true for every pass of a speculative step) and a
+// page size of 16, 32 or 64 keys.  Waits are bounded; a timeout is recorded in the status words.
+constexpr uint32_t ATT_SPIN_LIMIT = 1u << 20;
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t addr = smem_u32(bar);
+  for (uint32_t it = 0; it < ATT_SPIN_LIMIT; it++) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_3d(void *smem_dst, const CUtensorMap *map, int c0, int c1, int c2, uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+template <int HD, int STAGES>
+__global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ CUtensorMap map_k,
+                                                       const __grid_constant__ CUtensorMap map_v, AttnParams p, int32_t *status) {
+  pdl_wait();
+  pdl_trigger();
+  constexpr int ROWB = HD * 2, CPR = HD / 8;
+  constexpr int NKS = HD / 16;
+  constexpr int TILEB = KT * ROWB;                     // bytes of one K (or V) tile
+  extern __shared__ __align__(1024) unsigned char sm[];
+  unsigned char *sQ = sm + (STAGES - 1) * 2 * TILEB;   // the Q tile borrows the last stage until its fragments are in registers
+  uint64_t *full = (uint64_t *)(sm + STAGES * 2 * TILEB);
+  uint64_t *empty = full + STAGES;
+  uint64_t *q_bar = empty + STAGES;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int grp = p.H / p.G;
+  const int b = blockIdx.z / p.G, g = blockIdx.z % p.G;
+  const int M = p.rps * grp;
+  const int m0 = blockIdx.x * MT;
+  const int row0 = b * p.rps;
+  const int ps = p.pm.page_size;                       // keys per page = rows per tensor copy
+  int seq = -1, ctx = 0;
+  for (int i = 0; i < p.rps; i++) {
+    int s = p.m.seq[row0 + i];
+    if (s >= 0) { seq = s; ctx = p.m.ctx[row0 + i]; break; }
+  }
+  const int nkeys = (seq >= 0) ? ctx + p.tail_len : 0;
+  const int ntiles = (nkeys + KT - 1) / KT;
+  const int t_begin = (int)(((long long)blockIdx.y * ntiles) / p.nsplit);
+  const int t_end = (int)(((long long)(blockIdx.y + 1) * ntiles) / p.nsplit);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 8); }
+    mbar_init(q_bar, 8);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // ---- Q tile -> shared (swizzled) -> A fragments (consumer warps)
+  if (warp < 8) {
+    for (int id = threadIdx.x; id < MT * CPR; id += 256) {
+      int lr = id / CPR, c = id % CPR, mrow = m0 + lr;
+      bool v = mrow < M;
+      int i = v ? mrow / grp : 0, hq = v ? mrow % grp : 0;
+      v = v && p.m.seq[row0 + i] >= 0;
+      const bf16 *src = p.q + ((size_t)(row0 + i) * p.H + g * grp + hq) * HD + c * 8;
+      cp_async16(smem_u32(sQ + swz<ROWB>(lr, c)), src, v);
+    }
+    cp_async_commit();
+    cp_async_wait<0>();
+  }
+  __syncthreads();
+
+  if (warp == 8) {
+    // ================================================================ producer
+    if (lane == 0 && seq >= 0) {
+      const int32_t *tbl = p.pm.table + (size_t)seq * p.pm.pages_per_seq;
+      const int fallback = tbl[0];                     // keys past the last page are masked; they still need a valid source
+      const int ppt = KT / ps;                         // pages per tile
+      for (int t = t_begin; t < t_end; t++) {
+        const int i = t - t_begin, st = i % STAGES;
+        if (i == STAGES - 1 && !mbar_wait(q_bar, 0)) { if (status) set_status(status, ST_TIMEOUT, 400, blockIdx.z, t); break; }
+        if (i >= STAGES && !mbar_wait(&empty[st], (uint32_t)(((i / STAGES) - 1) & 1))) { if (status) set_status(status, ST_TIMEOUT, 401, blockIdx.z, t); break; }
+        unsigned char *kb = sm + st * 2 * TILEB, *vb = kb + TILEB;
+        mbar_expect_tx(&full[st], 2 * TILEB);
+        for (int pg = 0; pg < ppt; pg++) {
+          const int pidx = (t * KT) / ps + pg;
+          int page = pidx < p.pm.pages_per_seq ? tbl[pidx] : -1;
+          if (page < 0 || page >= p.pm.num_pages) page = fallback;
+          const int row = (page * p.G + g) * ps;
+          tma_load_3d(kb + pg * ps * ROWB, &map_k, 0, row, 0, &full[st]);
+          tma_load_3d(vb + pg * ps * ROWB, &map_v, 0, row, 0, &full[st]);
+        }
+      }
+    }
+    return;
+  }
+
+  // ================================================================== consumers (8 warps x 16 query rows)
+  uint32_t qf[NKS][4];
+#pragma unroll
+  for (int ks = 0; ks < NKS; ks++) {
+    int r = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = ks * 2 + (lane >> 4);
+    ldsm_x4(smem_u32(sQ + swz<ROWB>(r, c)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+  }
+  __syncwarp();
+  if (lane == 0) mbar_arrive(q_bar);
+  // byte offset of 16-byte chunk c of key kr inside a tile: [page][half of hd][key in page][128 B], chunks XOR-swizzled
+  const int psb = ps * ROWB;
+  auto koff = [&](int kr, int c) -> uint32_t {
+    return (uint32_t)((kr / ps) * psb + (c >> 3) * (ps * 128) + (kr % ps) * 128 + (((c & 7) ^ (kr & 7)) << 4));
+  };
+  const int tb = ctx;                                   // tail keys follow the context
+  (void)tb;
+  // rows owned by this thread: rA = quad row, rB = rA + 8 (within the warp's 16 rows)
+  const int mA = m0 + warp * 16 + (lane >> 2), mB = mA + 8;
+  uint64_t loA = 0, hiA = 0, loB = 0, hiB = 0;
+  bool vA = false, vB = false;
+  if (mA < M) { int r = row0 + mA / grp; vA = p.m.seq[r] >= 0; if (vA) { loA = p.m.mask_lo[r]; hiA = p.m.mask_hi[r]; } }
+  if (mB < M) { int r = row0 + mB / grp; vB = p.m.seq[r] >= 0; if (vB) { loB = p.m.mask_lo[r]; hiB = p.m.mask_hi[r]; } }
+
+  float o[HD / 8][4];
+#pragma unroll
+  for (int n = 0; n < HD / 8; n++) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.0f; }
+  float mxA = -INFINITY, mxB = -INFINITY, lA = 0.0f, lB = 0.0f;
+  const float sc = rsqrtf((float)HD) * 1.4426950408889634f;    // softmax scale folded into exp2
+
+
+  bool alive = true;
+  for (int t = t_begin; t < t_end && alive; t++) {
+    const int i = t - t_begin, st = i % STAGES;
+    if (!mbar_wait(&full[st], (uint32_t)((i / STAGES) & 1))) { if (lane == 0) if (status) set_status(status, ST_TIMEOUT, 402, blockIdx.z, t); alive = false; break; }
+    const unsigned char *kbase = sm + st * 2 * TILEB, *vbase = kbase + TILEB;
+    // ---- S = Q K^T for 64 keys: 8 n-tiles of 8 keys
+    float s[KT / 8][4];
+#pragma unroll
+    for (int n = 0; n < KT / 8; n++) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.0f; }
+#pragma unroll
+    for (int ks = 0; ks < NKS; ks++) {
+#pragma unroll
+      for (int n2 = 0; n2 < KT / 16; n2++) {
+        uint32_t b0, b1, b2, b3;
+        int kr = n2 * 16 + (lane & 7) + (lane >> 4) * 8, c = ks * 2 + ((lane >> 3) & 1);
+        ldsm_x4(smem_u32(kbase + koff(kr, c)), b0, b1, b2, b3);
+        mma_bf16(s[2 * n2], qf[ks], b0, b1);
+        mma_bf16(s[2 * n2 + 1], qf[ks], b2, b3);
+      }
+    }
+    // ---- mask + online softmax (two rows per thread, reductions across the quad)
+    float tmA = -INFINITY, tmB = -INFINITY;
+#pragma unroll
+    for (int n = 0; n < KT / 8; n++) {
+#pragma unroll
+      for (int e = 0; e < 2; e++) {
+        int key = t * KT + n * 8 + (lane & 3) * 2 + e;
+        bool in_ctx = key < ctx;
+        int tt = key - ctx;
+        bool in_tail = !in_ctx && tt < p.tail_len;
+        bool okA = vA && (in_ctx || (in_tail && ((tt < 64 ? (loA >> tt) : (hiA >> (tt - 64))) & 1ull)));
+        bool okB = vB && (in_ctx || (in_tail && ((tt < 64 ? (loB >> tt) : (hiB >> (tt - 64))) & 1ull)));
+        s[n][e] = okA ? s[n][e] : -INFINITY;
+        s[n][2 + e] = okB ? s[n][2 + e] : -INFINITY;
+        tmA = fmaxf(tmA, s[n][e]);
+        tmB = fmaxf(tmB, s[n][2 + e]);
+      }
+    }
+    tmA = fmaxf(tmA, __shfl_xor_sync(0xffffffffu, tmA, 1)); tmA = fmaxf(tmA, __shfl_xor_sync(0xffffffffu, tmA, 2));
+    tmB = fmaxf(tmB, __shfl_xor_sync(0xffffffffu, tmB, 1)); tmB = fmaxf(tmB, __shfl_xor_sync(0xffffffffu, tmB, 2));
+    float nmA = fmaxf(mxA, tmA), nmB = fmaxf(mxB, tmB);
+    float fA = (nmA == -INFINITY) ? 1.0f : exp2f((mxA - nmA) * sc), fB = (nmB == -INFINITY) ? 1.0f : exp2f((mxB - nmB) * sc);
+    float baseA = (nmA == -INFINITY) ? 0.0f : nmA, baseB = (nmB == -INFINITY) ? 0.0f : nmB;
+    float rsA = 0.0f, rsB = 0.0f;
+    uint32_t pf[KT / 16][4];
+#pragma unroll
+    for (int n = 0; n < KT / 8; n++) {
+      float p0 = exp2f((s[n][0] - baseA) * sc), p1 = exp2f((s[n][1] - baseA) * sc);
+      float p2 = exp2f((s[n][2] - baseB) * sc), p3 = exp2f((s[n][3] - baseB) * sc);
+      rsA += p0 + p1; rsB += p2 + p3;
+      pf[n >> 1][(n & 1) * 2] = pack_bf16(p0, p1);
+      pf[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
+    }
+    rsA += __shfl_xor_sync(0xffffffffu, rsA, 1); rsA += __shfl_xor_sync(0xffffffffu, rsA, 2);
+    rsB += __shfl_xor_sync(0xffffffffu, rsB, 1); rsB += __shfl_xor_sync(0xffffffffu, rsB, 2);
+    lA = lA * fA + rsA; lB = lB * fB + rsB;
+    mxA = nmA; mxB = nmB;
+#pragma unroll
+    for (int n = 0; n < HD / 8; n++) { o[n][0] *= fA; o[n][1] *= fA; o[n][2] *= fB; o[n][3] *= fB; }
+    // ---- O += P V
+#pragma unroll
+    for (int kk = 0; kk < KT / 16; kk++) {
+#pragma unroll
+      for (int d2 = 0; d2 < HD / 16; d2++) {
+        uint32_t b0, b1, b2, b3;
+        int kr = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, c = d2 * 2 + (lane >> 4);
+        ldsm_x4_t(smem_u32(vbase + koff(kr, c)), b0, b1, b2, b3);
+        mma_bf16(o[2 * d2], pf[kk], b0, b1);
+        mma_bf16(o[2 * d2 + 1], pf[kk], b2, b3);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&empty[st]);              // this warp is done with the stage
+  }
+
+  // ---- write: final (one split) or partial
+  const int qcol = (lane & 3) * 2;
+#pragma unroll
+  for (int half = 0; half < 2; half++) {
+    int mrow = half ? mB : mA;
+    if (mrow >= M) continue;
+    int r = row0 + mrow / grp, h = g * grp + mrow % grp;
+    float l = half ? lB : lA, mx = half ? mxB : mxA;
+    if (p.nsplit == 1) {
+      float inv = l > 0.0f ? 1.0f / l : 0.0f;
+      bf16 *dst = p.out + ((size_t)r * p.H + h) * HD;
+#pragma unroll
+      for (int n = 0; n < HD / 8; n++)
+        *(uint32_t *)(dst + n * 8 + qcol) = pack_bf16(o[n][half * 2] * inv, o[n][half * 2 + 1] * inv);
+    } else {
+      size_t idx = (size_t)blockIdx.y * p.rows * p.H + (size_t)r * p.H + h;
+      float *dst = p.part_o + idx * HD;
+#pragma unroll
+      for (int n = 0; n < HD / 8; n++) *(float2 *)(dst + n * 8 + qcol) = make_float2(o[n][half * 2], o[n][half * 2 + 1]);
+      if ((lane & 3) == 0) { p.part_ml[idx * 2] = mx; p.part_ml[idx * 2 + 1] = l; }
+    }
+  }
+}
+
 // merge the splits: out = sum_s 2^((m_s - M) c) O_s / sum_s 2^((m_s - M) c) l_s
 template <int HD>
 __global__ void attn_combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, int nsplit, int nrh,
@@ -276,8 +524,60 @@ size_t attn_fast_scratch_bytes(int rows, int n_heads, int head_dim, int max_ctx)
   return (size_t)MAX_SPLITS * rows * n_heads * (head_dim + 2) * sizeof(float) + 256;
 }
 
+namespace {
+typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                             const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn g_encode = nullptr;
+bool g_encode_tried = false;
+std::map<std::tuple<const void *, int, int, int, int>, CUtensorMap> g_kv_maps;   // (pool, pages, G, page size, hd)
+
+// 3-D view of a K or V pool [num_pages][G][page_size][hd]: dim0 = 64 elements (128 bytes), dim1 = every key row of
+// the pool (pitch hd * 2 bytes), dim2 = the hd / 64 column halves (128 bytes apart).  One box = one page of one head.
+const CUtensorMap *kv_map(const void *pool, int num_pages, int G, int ps, int hd) {
+  if (!g_encode_tried) {
+    g_encode_tried = true;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      g_encode = (EncodeFn)fn;
+  }
+  if (!g_encode) return nullptr;
+  if (num_pages > (1 << 20)) num_pages = 1 << 20;      // callers without a pool size: the page table is trusted
+  auto key = std::make_tuple(pool, num_pages, G, ps, hd);
+  auto it = g_kv_maps.find(key);
+  if (it != g_kv_maps.end()) return &it->second;
+  CUtensorMap m;
+  cuuint64_t dims[3] = {64, (cuuint64_t)num_pages * G * ps, (cuuint64_t)(hd / 64)};
+  cuuint64_t strides[2] = {(cuuint64_t)hd * 2, 128};
+  cuuint32_t box[3] = {64, (cuuint32_t)ps, (cuuint32_t)(hd / 64)};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void *)pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return nullptr;
+  if (g_kv_maps.size() > 4096) g_kv_maps.clear();
+  return &(g_kv_maps[key] = m);
+}
+
+template <int HD>
+int launch_tma(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorMap *mv, int32_t *status, cudaStream_t s) {
+  constexpr int STAGES = HD == 128 ? 3 : 4;
+  const int smem = STAGES * 2 * KT * HD * 2 + 256;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(attn_tma_kernel<HD, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -1;
+    configured = true;
+  }
+  launch_k(attn_tma_kernel<HD, STAGES>, grid, dim3(288), (size_t)smem, s, *mk, *mv, p, status);
+  return 0;
+}
+}  // namespace
+
+void attn_fast_forget_maps() { g_kv_maps.clear(); }
+
 int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail_len, bf16 *out, int rows, int H, int G,
-                     int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s) {
+                     int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s, bool contiguous_tail, int32_t *status) {
   if (rps < 1 || rows % rps) rps = 1;
   int seqs = rows / rps, grp = H / G;
   int mtiles = (rps * grp + MT - 1) / MT;
@@ -289,6 +589,21 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
   p.part_o = (float *)scratch;
   p.part_ml = p.part_o ? p.part_o + (size_t)MAX_SPLITS * rows * H * hd : nullptr;
   dim3 grid(mtiles, nsplit, seqs * G);
+  // TMA-staged kernel when the tail follows the context and a page is a whole number of 128-byte-swizzle boxes
+  const int ps = pm.page_size;
+  if (contiguous_tail && (ps == 16 || ps == 32 || ps == 64) && (hd == 64 || hd == 128)) {
+    const CUtensorMap *mk = kv_map(pool.k, pm.num_pages, G, ps, hd), *mv = kv_map(pool.v, pm.num_pages, G, ps, hd);
+    if (mk && mv) {
+      int rc = hd == 128 ? launch_tma<128>(p, grid, mk, mv, status, s) : launch_tma<64>(p, grid, mk, mv, status, s);
+      if (rc == 0) {
+        if (nsplit > 1) {
+          if (hd == 128) launch_k(attn_combine_kernel<128>, dim3(rows * H), dim3(128), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
+          else launch_k(attn_combine_kernel<64>, dim3(rows * H), dim3(64), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
+        }
+        return nsplit > 1 ? 2 : 1;
+      }
+    }
+  }
   size_t smem = (size_t)4 * KT * hd * 2;
   if (smem < (size_t)MT * hd * 2) smem = (size_t)MT * hd * 2;
   static bool attr[2] = {false, false};
@@ -367,6 +682,6 @@ extern "C" int spec_attention_static(const void *q, const void *k_pool, const vo
   m.mask_lo = (uint64_t *)row_mask_lo; m.mask_hi = (uint64_t *)row_mask_hi;
   KvPool pool{(void *)k_pool, (void *)v_pool};
   PageMap pm{page_table, pages_per_seq, page_size, 1 << 30};
-  launch_attn_fast((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, 1, max_ctx, scratch, (cudaStream_t)stream);
+  launch_attn_fast((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, 1, max_ctx, scratch, (cudaStream_t)stream, false, nullptr);
   return cudaGetLastError() == cudaSuccess ? 0 : -6;
 }

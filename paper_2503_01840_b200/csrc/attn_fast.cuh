@@ -10,6 +10,11 @@ size_t attn_fast_scratch_bytes(int rows, int n_heads, int head_dim, int max_ctx)
 // nothing is known); ctx_hint sizes the key split (any value is correct); scratch may be NULL (one
 // split).  Returns the number of kernels launched.
 int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail_len, bf16 *out, int rows, int H, int G,
-                     int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s);
+                     int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s, bool contiguous_tail = false,
+                     int32_t *status = nullptr);
+// contiguous_tail: every row's tail_base equals its ctx (the tail keys follow the context in the cache), which lets the
+// TMA-staged kernel fetch whole pages; status: device status words for its bounded waits (may be NULL).
+// Drops the cached K/V tensor maps (pools of one-shot callers come and go).
+void attn_fast_forget_maps();
 
 }  // namespace spec

@@ -127,7 +127,8 @@ def test_c3_shape_two_layers_batch64_losslessness():
     assert mismatches <= 16, mismatches
 
 
-def test_c4_long_context_attention_sampled_vs_oracle():
+@pytest.mark.parametrize("impl", [0, 2], ids=["cp_async", "tma"])
+def test_c4_long_context_attention_sampled_vs_oracle(impl):
     """Tree-masked attention over a 16384-token paged context (many key splits + combine), 60 nodes x 32 heads;
     sampled (node, head) pairs against the oracle's per-head routine."""
     H, G, hd, ps, ctx, tail = 32, 8, 128, 16, 16384, 60
@@ -143,7 +144,7 @@ def test_c4_long_context_attention_sampled_vs_oracle():
     lo = torch.randint(0, 2 ** 59, (rows,), generator=g, dtype=torch.int64) | 1
     hi = torch.zeros(rows, dtype=torch.int64)
     out = sb.attention(q.cuda(), kp.cuda(), vp.cuda(), perm.cuda(), ps, seq.cuda(), rctx.cuda(), rctx.cuda(), lo.cuda(),
-                       hi.cuda(), tail, G, ctx + 64, impl=0).float().cpu().numpy()
+                       hi.cuda(), tail, G, ctx + 64, impl=impl).float().cpu().numpy()
     pos_ctx = np.arange(ctx)
     page_of = perm[0].numpy()
     for r, h in [(0, 0), (7, 5), (31, 17), (59, 31), (44, 12)]:
