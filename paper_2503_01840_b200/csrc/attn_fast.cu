@@ -312,9 +312,11 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
   const int t_begin = (int)(((long long)blockIdx.y * ntiles) / p.nsplit);
   const int t_end = (int)(((long long)(blockIdx.y + 1) * ntiles) / p.nsplit);
 
+  // consumer warps that own at least one query row; the others leave after the Q phase
+  const int nactive = (M - m0 >= MT) ? 8 : (M - m0 + 15) / 16;
   if (threadIdx.x == 0) {
-    for (int i = 0; i < STAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 8); }
-    mbar_init(q_bar, 8);
+    for (int i = 0; i < STAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], nactive); }
+    mbar_init(q_bar, nactive);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // ---- Q tile -> shared (swizzled) -> A fragments (consumer warps)
@@ -358,6 +360,7 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
   }
 
   // ================================================================== consumers (8 warps x 16 query rows)
+  if (warp >= nactive) return;
   uint32_t qf[NKS][4];
 #pragma unroll
   for (int ks = 0; ks < NKS; ks++) {
@@ -409,20 +412,29 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
     }
     // ---- mask + online softmax (two rows per thread, reductions across the quad)
     float tmA = -INFINITY, tmB = -INFINITY;
+    if (t * KT + KT <= ctx && vA && vB) {
+      // every key of the tile is context and both rows are real: nothing to mask
 #pragma unroll
-    for (int n = 0; n < KT / 8; n++) {
+      for (int n = 0; n < KT / 8; n++) {
+        tmA = fmaxf(tmA, fmaxf(s[n][0], s[n][1]));
+        tmB = fmaxf(tmB, fmaxf(s[n][2], s[n][3]));
+      }
+    } else {
 #pragma unroll
-      for (int e = 0; e < 2; e++) {
-        int key = t * KT + n * 8 + (lane & 3) * 2 + e;
-        bool in_ctx = key < ctx;
-        int tt = key - ctx;
-        bool in_tail = !in_ctx && tt < p.tail_len;
-        bool okA = vA && (in_ctx || (in_tail && ((tt < 64 ? (loA >> tt) : (hiA >> (tt - 64))) & 1ull)));
-        bool okB = vB && (in_ctx || (in_tail && ((tt < 64 ? (loB >> tt) : (hiB >> (tt - 64))) & 1ull)));
-        s[n][e] = okA ? s[n][e] : -INFINITY;
-        s[n][2 + e] = okB ? s[n][2 + e] : -INFINITY;
-        tmA = fmaxf(tmA, s[n][e]);
-        tmB = fmaxf(tmB, s[n][2 + e]);
+      for (int n = 0; n < KT / 8; n++) {
+  #pragma unroll
+        for (int e = 0; e < 2; e++) {
+          int key = t * KT + n * 8 + (lane & 3) * 2 + e;
+          bool in_ctx = key < ctx;
+          int tt = key - ctx;
+          bool in_tail = !in_ctx && tt < p.tail_len;
+          bool okA = vA && (in_ctx || (in_tail && ((tt < 64 ? (loA >> tt) : (hiA >> (tt - 64))) & 1ull)));
+          bool okB = vB && (in_ctx || (in_tail && ((tt < 64 ? (loB >> tt) : (hiB >> (tt - 64))) & 1ull)));
+          s[n][e] = okA ? s[n][e] : -INFINITY;
+          s[n][2 + e] = okB ? s[n][2 + e] : -INFINITY;
+          tmA = fmaxf(tmA, s[n][e]);
+          tmB = fmaxf(tmB, s[n][2 + e]);
+        }
       }
     }
     tmA = fmaxf(tmA, __shfl_xor_sync(0xffffffffu, tmA, 1)); tmA = fmaxf(tmA, __shfl_xor_sync(0xffffffffu, tmA, 2));
@@ -509,7 +521,8 @@ __global__ void attn_combine_kernel(const float *__restrict__ part_o, const floa
 
 int pick_splits(int seqs, int G, int mtiles, int max_ctx_tiles) {
   int base = seqs * G * mtiles;
-  int want = (2 * 148 + base - 1) / base;
+  int want = (148 + base / 2) / base;                // the kernels run one CTA per SM (register-bound): aim at one wave
+  if (want < 1) want = 1;
   int s = want < max_ctx_tiles ? want : max_ctx_tiles;
   if (s > MAX_SPLITS) s = MAX_SPLITS;
   return s < 1 ? 1 : s;
