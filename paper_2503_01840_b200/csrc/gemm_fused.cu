@@ -417,7 +417,7 @@ struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB; };
 // of a launch goes with (CTAs on the busiest SM) x (k-blocks per CTA + a fixed cost per CTA); two CTAs per SM
 // are needed to hide one CTA's MMA and epilogue time behind the other's loads.
 int g_target_ctas = 222;   // measured best on the 8B shapes (1.5 CTAs per SM)
-constexpr int MAX_CLUSTER = 8;
+constexpr int MAX_CLUSTER = 8;    // portable cluster sizes only: size 9 (non-portable) measured 20 % slower per step
 
 Plan make_plan(FusedEpi epi, const FusedGemmArgs &a) {
   Plan pl;
