@@ -33,9 +33,12 @@ from paper_2503_01840_b200 import synth  # noqa: E402
 METRIC = "spec_step accepted tok/s"
 UNIT = "tok/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMM kernel from the ncu capture
-# summarised in profiles/ (None until a capture exists for that workload)
-NCU_TRAFFIC_PER_LAUNCH = {}
+# DRAM traffic of the GEMM kernel relative to its weight bytes, from the ncu capture summarised in
+# profiles/gemm_fused_kernel_C2_shapes_ncu_full.md: (dram__bytes_read.sum + dram__bytes_write.sum) of the four GEMMs
+# of an 8B-shaped layer = 448.5 MB for 436.2 MB of weights.  The capture ran on the 2-layer truncation (same kernels,
+# same shapes); a full step's traffic is that ratio times its weight bytes (traffic grows with the weight bytes).
+# Valid for the 8B shapes at 60 rows only; None elsewhere.
+NCU_TRAFFIC_RATIO = {"C2-8B-b1": 448.5 / 436.2}
 
 
 def peaks():
@@ -295,7 +298,8 @@ def main():
     gemm_ms, gemm_n = breakdown["gemm"]
     wbytes = weight_bytes_per_step(cfg)
     achieved = wbytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
-    traffic = NCU_TRAFFIC_PER_LAUNCH.get(cfg.name)
+    ratio = NCU_TRAFFIC_RATIO.get(cfg.name)
+    traffic = ratio * wbytes / max(1, gemm_n) if ratio else None
     roofline = {"bound": "hbm", "kernel": "gemm_fused_kernel (all weight GEMMs of the step)", "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                 "bytes_per_launch": wbytes / max(1, gemm_n), "avg_launch_us": 1e3 * gemm_ms / max(1, gemm_n),

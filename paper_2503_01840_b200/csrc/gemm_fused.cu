@@ -427,17 +427,20 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a) {
   const int stage = A_BYTES + pl.nt * TILE_K * 2;
   const int wmul = epi == EPI_SWIGLU ? 2 : 1;          // cluster members per K slice
   const int smax = MAX_CLUSTER / wmul;
+  const bool one_per_sm = SMEM_TWO / stage < 3;        // 256-row tiles: the ring of one CTA takes the SM
+  const int target = one_per_sm ? NUM_SMS : g_target_ctas;   // one wave
   int Sk = 1;
   if (epi != EPI_ARGMAX) {
-    Sk = (g_target_ctas + pl.tiles * wmul / 2) / std::max(1, pl.tiles * wmul);   // nearest to the target CTA count
+    Sk = one_per_sm ? target / std::max(1, pl.tiles * wmul)  // never more CTAs than SMs
+                    : (target + pl.tiles * wmul / 2) / std::max(1, pl.tiles * wmul);   // nearest to the target CTA count
     Sk = std::max(1, std::min(Sk, smax));
     Sk = std::max(1, std::min(Sk, pl.KB / 4));
   }
   if (a.split > 0) Sk = std::max(1, std::min(std::min(a.split, smax), pl.KB));
   pl.Sk = Sk;
   pl.S = Sk * wmul;
-  int budget = SMEM_TWO;
-  if (SMEM_TWO / stage < 3) budget = SMEM_ONE;         // 256-row tiles: one CTA per SM
+  // more tiles than SMs and a ring that fills the SM: two CTAs with two stages each beat two waves of one
+  const int budget = !one_per_sm ? SMEM_TWO : (pl.tiles * wmul * Sk > NUM_SMS ? 2 * stage : SMEM_ONE);
   int stages = std::max(2, std::min(MAX_STAGES, budget / stage));
   if (a.stages > 0) stages = std::max(2, std::min(std::min(a.stages, MAX_STAGES), (220 * 1024) / stage));
   int per_slice = (pl.KB + Sk - 1) / Sk;
