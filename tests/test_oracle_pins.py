@@ -425,3 +425,17 @@ def test_rerank_unit_ties_and_closure():
     assert r["cut_margin"] == 0.0
     r = po.rerank(score, parent, tok, depth, 64, 100)
     assert r["n"] == 7 and math.isinf(r["cut_margin"])
+
+
+def test_golden_c1_trajectory_is_reproduced_and_lossless():
+    """tests/golden/c1_oracle_trajectory.json (written by tests/golden/make_golden.py from the oracle alone)."""
+    import json
+    import os
+    import sys
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    sys.path.insert(0, here)
+    import make_golden
+    stored = json.load(open(os.path.join(here, "c1_oracle_trajectory.json")))
+    assert stored["tokens"] == stored["greedy"][: len(stored["tokens"])]          # Section 2.1: lossless at temperature 0
+    assert all(1 <= c <= C1.tree_depth + 1 for c in stored["counts"]) and sum(stored["counts"]) == len(stored["tokens"]) - 1
+    assert make_golden.trajectory() == stored
