@@ -498,6 +498,204 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// TMA-staged variant for at most 16 query rows per (sequence, KV head): chain drafts at batch (one node x the GQA
+// group) and single-token decoding.  One 16-row tile would leave seven of eight row-parallel warps idle, so here
+// the four consumer warps share the rows and split the KEYS of every 64-key tile (16 keys each); each keeps its own
+// online-softmax state and the four states are merged through shared memory at the end.
+template <int HD, int STAGES>
+__global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_constant__ CUtensorMap map_k,
+                                                             const __grid_constant__ CUtensorMap map_v, AttnParams p, int32_t *status) {
+  pdl_wait();
+  pdl_trigger();
+  constexpr int ROWB = HD * 2, CPR = HD / 8;
+  constexpr int NKS = HD / 16;
+  constexpr int TILEB = KT * ROWB;
+  constexpr int NW = 4;                                // consumer warps
+  extern __shared__ __align__(1024) unsigned char sm[];
+  uint64_t *full = (uint64_t *)(sm + STAGES * 2 * TILEB);
+  uint64_t *empty = full + STAGES;
+  unsigned char *sQ = sm + STAGES * 2 * TILEB + 256;   // [16][HD] bf16, swizzled
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int grp = p.H / p.G;
+  const int b = blockIdx.z / p.G, g = blockIdx.z % p.G;
+  const int M = p.rps * grp;                           // <= 16
+  const int row0 = b * p.rps;
+  const int ps = p.pm.page_size;
+  int seq = -1, ctx = 0;
+  for (int i = 0; i < p.rps; i++) {
+    int s = p.m.seq[row0 + i];
+    if (s >= 0) { seq = s; ctx = p.m.ctx[row0 + i]; break; }
+  }
+  const int nkeys = (seq >= 0) ? ctx + p.tail_len : 0;
+  const int ntiles = (nkeys + KT - 1) / KT;
+  const int t_begin = (int)(((long long)blockIdx.y * ntiles) / p.nsplit);
+  const int t_end = (int)(((long long)(blockIdx.y + 1) * ntiles) / p.nsplit);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], NW); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int id = threadIdx.x; id < 16 * CPR; id += 160) {
+    int lr = id / CPR, c = id % CPR;
+    bool v = lr < M;
+    int i = v ? lr / grp : 0, hq = v ? lr % grp : 0;
+    v = v && p.m.seq[row0 + i] >= 0;
+    const bf16 *src = p.q + ((size_t)(row0 + i) * p.H + g * grp + hq) * HD + c * 8;
+    cp_async16(smem_u32(sQ + swz<ROWB>(lr, c)), src, v);
+  }
+  cp_async_commit();
+  cp_async_wait<0>();
+  __syncthreads();
+
+  if (warp == NW) {
+    if (lane == 0 && seq >= 0) {
+      const int32_t *tbl = p.pm.table + (size_t)seq * p.pm.pages_per_seq;
+      const int fallback = tbl[0];
+      const int ppt = KT / ps;
+      for (int t = t_begin; t < t_end; t++) {
+        const int i = t - t_begin, st = i % STAGES;
+        if (i >= STAGES && !mbar_wait(&empty[st], (uint32_t)(((i / STAGES) - 1) & 1))) { if (status) set_status(status, ST_TIMEOUT, 411, blockIdx.z, t); break; }
+        unsigned char *kb = sm + st * 2 * TILEB, *vb = kb + TILEB;
+        mbar_expect_tx(&full[st], 2 * TILEB);
+        for (int pg = 0; pg < ppt; pg++) {
+          const int pidx = (t * KT) / ps + pg;
+          int page = pidx < p.pm.pages_per_seq ? tbl[pidx] : -1;
+          if (page < 0 || page >= p.pm.num_pages) page = fallback;
+          const int row = (page * p.G + g) * ps;
+          tma_load_3d(kb + pg * ps * ROWB, &map_k, 0, row, 0, &full[st]);
+          tma_load_3d(vb + pg * ps * ROWB, &map_v, 0, row, 0, &full[st]);
+        }
+      }
+    }
+  } else {
+    // ---- consumers: all four warps hold the same 16-row Q tile
+    uint32_t qf[NKS][4];
+#pragma unroll
+    for (int ks = 0; ks < NKS; ks++) {
+      int r = (lane & 7) + ((lane >> 3) & 1) * 8, c = ks * 2 + (lane >> 4);
+      ldsm_x4(smem_u32(sQ + swz<ROWB>(r, c)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+    }
+    const int psb = ps * ROWB;
+    auto koff = [&](int kr, int c) -> uint32_t {
+      return (uint32_t)((kr / ps) * psb + (c >> 3) * (ps * 128) + (kr % ps) * 128 + (((c & 7) ^ (kr & 7)) << 4));
+    };
+    const int mA = lane >> 2, mB = mA + 8;
+    uint64_t loA = 0, hiA = 0, loB = 0, hiB = 0;
+    bool vA = false, vB = false;
+    if (mA < M) { int r = row0 + mA / grp; vA = p.m.seq[r] >= 0; if (vA) { loA = p.m.mask_lo[r]; hiA = p.m.mask_hi[r]; } }
+    if (mB < M) { int r = row0 + mB / grp; vB = p.m.seq[r] >= 0; if (vB) { loB = p.m.mask_lo[r]; hiB = p.m.mask_hi[r]; } }
+    float o[HD / 8][4];
+#pragma unroll
+    for (int n = 0; n < HD / 8; n++) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.0f; }
+    float mxA = -INFINITY, mxB = -INFINITY, lA = 0.0f, lB = 0.0f;
+    const float sc = rsqrtf((float)HD) * 1.4426950408889634f;
+    const int k0w = warp * 16;                          // this warp's keys inside a tile
+    for (int t = t_begin; t < t_end; t++) {
+      const int i = t - t_begin, st = i % STAGES;
+      if (!mbar_wait(&full[st], (uint32_t)((i / STAGES) & 1))) { if (lane == 0 && status) set_status(status, ST_TIMEOUT, 412, blockIdx.z, t); break; }
+      const unsigned char *kbase = sm + st * 2 * TILEB, *vbase = kbase + TILEB;
+      float s[2][4];
+#pragma unroll
+      for (int n = 0; n < 2; n++) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.0f; }
+#pragma unroll
+      for (int ks = 0; ks < NKS; ks++) {
+        uint32_t b0, b1, b2, b3;
+        int kr = k0w + (lane & 7) + (lane >> 4) * 8, c = ks * 2 + ((lane >> 3) & 1);
+        ldsm_x4(smem_u32(kbase + koff(kr, c)), b0, b1, b2, b3);
+        mma_bf16(s[0], qf[ks], b0, b1);
+        mma_bf16(s[1], qf[ks], b2, b3);
+      }
+      float tmA = -INFINITY, tmB = -INFINITY;
+#pragma unroll
+      for (int n = 0; n < 2; n++) {
+#pragma unroll
+        for (int e = 0; e < 2; e++) {
+          int key = t * KT + k0w + n * 8 + (lane & 3) * 2 + e;
+          bool in_ctx = key < ctx;
+          int tt = key - ctx;
+          bool in_tail = !in_ctx && tt < p.tail_len;
+          bool okA = vA && (in_ctx || (in_tail && ((tt < 64 ? (loA >> tt) : (hiA >> (tt - 64))) & 1ull)));
+          bool okB = vB && (in_ctx || (in_tail && ((tt < 64 ? (loB >> tt) : (hiB >> (tt - 64))) & 1ull)));
+          s[n][e] = okA ? s[n][e] : -INFINITY;
+          s[n][2 + e] = okB ? s[n][2 + e] : -INFINITY;
+          tmA = fmaxf(tmA, s[n][e]);
+          tmB = fmaxf(tmB, s[n][2 + e]);
+        }
+      }
+      tmA = fmaxf(tmA, __shfl_xor_sync(0xffffffffu, tmA, 1)); tmA = fmaxf(tmA, __shfl_xor_sync(0xffffffffu, tmA, 2));
+      tmB = fmaxf(tmB, __shfl_xor_sync(0xffffffffu, tmB, 1)); tmB = fmaxf(tmB, __shfl_xor_sync(0xffffffffu, tmB, 2));
+      float nmA = fmaxf(mxA, tmA), nmB = fmaxf(mxB, tmB);
+      float fA = (nmA == -INFINITY) ? 1.0f : exp2f((mxA - nmA) * sc), fB = (nmB == -INFINITY) ? 1.0f : exp2f((mxB - nmB) * sc);
+      float baseA = (nmA == -INFINITY) ? 0.0f : nmA, baseB = (nmB == -INFINITY) ? 0.0f : nmB;
+      float rsA = 0.0f, rsB = 0.0f;
+      uint32_t pf[4];
+#pragma unroll
+      for (int n = 0; n < 2; n++) {
+        float p0 = exp2f((s[n][0] - baseA) * sc), p1 = exp2f((s[n][1] - baseA) * sc);
+        float p2 = exp2f((s[n][2] - baseB) * sc), p3 = exp2f((s[n][3] - baseB) * sc);
+        rsA += p0 + p1; rsB += p2 + p3;
+        pf[n * 2] = pack_bf16(p0, p1);
+        pf[n * 2 + 1] = pack_bf16(p2, p3);
+      }
+      rsA += __shfl_xor_sync(0xffffffffu, rsA, 1); rsA += __shfl_xor_sync(0xffffffffu, rsA, 2);
+      rsB += __shfl_xor_sync(0xffffffffu, rsB, 1); rsB += __shfl_xor_sync(0xffffffffu, rsB, 2);
+      lA = lA * fA + rsA; lB = lB * fB + rsB;
+      mxA = nmA; mxB = nmB;
+#pragma unroll
+      for (int n = 0; n < HD / 8; n++) { o[n][0] *= fA; o[n][1] *= fA; o[n][2] *= fB; o[n][3] *= fB; }
+#pragma unroll
+      for (int d2 = 0; d2 < HD / 16; d2++) {
+        uint32_t b0, b1, b2, b3;
+        int kr = k0w + (lane & 7) + ((lane >> 3) & 1) * 8, c = d2 * 2 + (lane >> 4);
+        ldsm_x4_t(smem_u32(vbase + koff(kr, c)), b0, b1, b2, b3);
+        mma_bf16(o[2 * d2], pf, b0, b1);
+        mma_bf16(o[2 * d2 + 1], pf, b2, b3);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[st]);
+    }
+    // ---- merge the four key subsets: every warp parks (o, max, sum) in shared memory
+    float *so = (float *)sm;                            // [NW][16][HD]: the ring is free once every warp has left the loop
+    float *sml = so + NW * 16 * HD;                     // [NW][16][2]
+    asm volatile("bar.sync 1, 128;" ::: "memory");      // all warps are done with the last stage
+    const int qcol = (lane & 3) * 2;
+#pragma unroll
+    for (int half = 0; half < 2; half++) {
+      const int lr = (lane >> 2) + half * 8;
+#pragma unroll
+      for (int n = 0; n < HD / 8; n++) *(float2 *)(so + (warp * 16 + lr) * HD + n * 8 + qcol) = make_float2(o[n][half * 2], o[n][half * 2 + 1]);
+      if ((lane & 3) == 0) { sml[(warp * 16 + lr) * 2] = half ? mxB : mxA; sml[(warp * 16 + lr) * 2 + 1] = half ? lB : lA; }
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    const int tid = threadIdx.x;                        // 0..127
+    for (int e = tid; e < 16 * HD; e += 128) {
+      const int lr = e / HD, d = e % HD;
+      if (lr >= M) continue;
+      float Mx = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < NW; w++) Mx = fmaxf(Mx, sml[(w * 16 + lr) * 2]);
+      float acc = 0.0f, l = 0.0f;
+#pragma unroll
+      for (int w = 0; w < NW; w++) {
+        const float m = sml[(w * 16 + lr) * 2];
+        if (m == -INFINITY) continue;
+        const float wt = exp2f((m - Mx) * sc);
+        acc += wt * so[(w * 16 + lr) * HD + d];
+        l += wt * sml[(w * 16 + lr) * 2 + 1];
+      }
+      const int r = row0 + lr / grp, h = g * grp + lr % grp;
+      if (p.nsplit == 1) {
+        p.out[((size_t)r * p.H + h) * HD + d] = __float2bfloat16_rn(l > 0.0f ? acc / l : 0.0f);
+      } else {
+        const size_t idx = (size_t)blockIdx.y * p.rows * p.H + (size_t)r * p.H + h;
+        p.part_o[idx * HD + d] = acc;
+        if (d == 0) { p.part_ml[idx * 2] = Mx; p.part_ml[idx * 2 + 1] = l; }
+      }
+    }
+  }
+}
+
 // merge the splits: out = sum_s 2^((m_s - M) c) O_s / sum_s 2^((m_s - M) c) l_s
 template <int HD>
 __global__ void attn_combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, int nsplit, int nrh,
@@ -574,7 +772,21 @@ const CUtensorMap *kv_map(const void *pool, int num_pages, int G, int ps, int hd
 }
 
 template <int HD>
+int launch_tma_small(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorMap *mv, int32_t *status, cudaStream_t s) {
+  constexpr int STAGES = HD == 128 ? 3 : 4;
+  const int smem = STAGES * 2 * KT * HD * 2 + 256 + 16 * HD * 2;   // ring (reused by the final merge) + barriers + Q tile
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(attn_tma_small_kernel<HD, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -1;
+    configured = true;
+  }
+  launch_k(attn_tma_small_kernel<HD, STAGES>, grid, dim3(160), (size_t)smem, s, *mk, *mv, p, status);
+  return 0;
+}
+
+template <int HD>
 int launch_tma(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorMap *mv, int32_t *status, cudaStream_t s) {
+  if (p.rps * (p.H / p.G) <= 16) return launch_tma_small<HD>(p, grid, mk, mv, status, s);
   constexpr int STAGES = HD == 128 ? 3 : 4;
   const int smem = STAGES * 2 * KT * HD * 2 + 256;
   static bool configured = false;

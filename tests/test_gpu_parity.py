@@ -278,3 +278,33 @@ def test_c2_two_layer_truncation_first_steps(flags):
     prompts = [p.numpy() for p in synth.make_prompts(cfg)]
     st, _ = parity.run_trajectory(cfg, parity.to_cpu(tw), parity.to_cpu(dw), prompts, n_steps=2, tol=2e-2, tap_tol=3e-2, flags=flags)
     print("C2-L2", st)
+
+
+@pytest.mark.parametrize("H,G,hd,rps", [(32, 8, 128, 4), (8, 2, 128, 1), (4, 2, 64, 3)])
+def test_attention_few_query_rows_key_parallel_kernel(H, G, hd, rps):
+    """At most 16 query rows per (sequence, KV head) (chain drafts at batch, single-token decoding): the key-parallel
+    TMA kernel, several sequences of different lengths, against the oracle's per-head routine."""
+    ps, n_seq, tail = 16, 5, rps
+    g = torch.Generator().manual_seed(70 + H + rps)
+    ctxs = [37, 250, 64, 1, 513]
+    pps = (max(ctxs) + tail + ps - 1) // ps + 1
+    perm = torch.randperm(n_seq * pps, generator=g).to(torch.int32).reshape(n_seq, pps)
+    kp = torch.randn(n_seq * pps, G, ps, hd, generator=g).to(torch.bfloat16)
+    vp = torch.randn(n_seq * pps, G, ps, hd, generator=g).to(torch.bfloat16)
+    rows = n_seq * rps
+    q = torch.randn(rows, H, hd, generator=g).to(torch.bfloat16)
+    seq = torch.tensor([r // rps for r in range(rows)], dtype=torch.int32)
+    rctx = torch.tensor([ctxs[r // rps] for r in range(rows)], dtype=torch.int32)
+    lo = torch.tensor([(1 << ((r % rps) + 1)) - 1 for r in range(rows)], dtype=torch.int64)      # causal chain
+    hi = torch.zeros(rows, dtype=torch.int64)
+    out = sb.attention(q.cuda(), kp.cuda(), vp.cuda(), perm.cuda(), ps, seq.cuda(), rctx.cuda(), rctx.cuda(), lo.cuda(), hi.cuda(),
+                       tail, G, 1024, impl=2).float().cpu().numpy()
+    for r in range(rows):
+        s = int(seq[r])
+        pos = list(range(ctxs[s])) + [ctxs[s] + t for t in range(tail) if (int(lo[r]) >> t) & 1]
+        for h in range(0, H, max(1, H // 4)):
+            gk = h // (H // G)
+            K = np.stack([kp[perm[s, p // ps], gk, p % ps].float().numpy() for p in pos])
+            V = np.stack([vp[perm[s, p // ps], gk, p % ps].float().numpy() for p in pos])
+            ref = po.attend(q[r, h].float().numpy(), K, V)
+            assert np.abs(out[r, h] - ref).max() < 2e-2, (r, h)
