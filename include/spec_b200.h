@@ -147,6 +147,7 @@ int spec_profile_step(spec_ctx *ctx, float *class_ms, int32_t *class_launches);
  *   SPEC_TUNE_GEMM_CTAS   CTAs a weight-streaming GEMM launch aims at (process-wide) */
 enum spec_tune_knob { SPEC_TUNE_L2_LEAD_MB = 1, SPEC_TUNE_GEMM_CTAS = 2,
                       SPEC_TUNE_DEBUG_LAUNCH_BUDGET = 3 /* debugging: run only the first n kernels of each step (-1: all) */,
+                      SPEC_TUNE_ATTN_CTAS = 4 /* CTAs an attention launch aims at when splitting keys (process-wide) */,
                       SPEC_TUNE_CHAIN_TIMING = 5 /* profiling: record phase time stamps of the n-th chain launch of a step (-1: none) */ };
 int spec_tune(spec_ctx *ctx, int32_t what, int32_t value);
 
@@ -209,6 +210,14 @@ int spec_gemm(int32_t dtype, int32_t impl, const void *x, const void *w, float *
  * split: K slices (= cluster size, 1..8), stages: TMA pipeline depth; 0 lets the library choose. */
 int spec_gemm_fused(const void *x, const void *w, float *out_f32, int32_t rows, int32_t out, int32_t in, int32_t ldo,
                     int32_t split, int32_t stages, void *stream);
+
+/* Gate/up half of the decoder layer's MLP (the draft layer and every target layer are LLaMA-style decoder layers,
+ * Section 3.1), on the kernel the step uses: act[r][f] = bf16(silu(g) * u), g = sum_i x[r][i] * w_gate[f][i], u likewise
+ * with w_up, both accumulated in fp32 (a cluster holds the gate and the up tile of the same 128 features and their K
+ * slices).  x [rows][in] bf16, w_gate / w_up [F][in] bf16, act [rows][F] bf16, all device pointers, 16-byte aligned;
+ * rows <= 256, in % 8 == 0.  Returns SPEC_OK or a negative code; nothing is allocated. */
+int spec_gemm_swiglu(const void *x, const void *w_gate, const void *w_up, void *act, int32_t rows, int32_t F, int32_t in,
+                     void *stream);
 
 /* Tree-masked paged GQA attention (Section 2.2 "tree attention") for `rows` query rows of one or
  * more sequences.  q [rows][H][hd] dtype; K/V pools [num_pages][G][page_size][hd] dtype;

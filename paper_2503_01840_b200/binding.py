@@ -57,7 +57,7 @@ class _Cfg(C.Structure):
 
 EXPORTS = ("spec_workspace_bytes", "spec_init", "spec_prefill", "spec_step", "spec_step_async", "spec_plain_step",
            "spec_lengths", "spec_profile_step", "spec_tune", "spec_launches_per_step", "spec_step_bytes", "spec_free", "spec_last_error",
-           "spec_debug_read", "spec_debug_read_kv", "spec_gemm_scratch_bytes", "spec_gemm", "spec_gemm_fused",
+           "spec_debug_read", "spec_debug_read_kv", "spec_gemm_scratch_bytes", "spec_gemm", "spec_gemm_fused", "spec_gemm_swiglu",
            "spec_topk_scratch_bytes", "spec_attn_scratch_bytes",
            "spec_attention", "spec_attention_static", "spec_attention_static_capacity", "spec_logsoftmax_topk", "spec_argmax")
 
@@ -103,6 +103,7 @@ def lib():
     L.spec_attention_static_capacity.restype = sz
     L.spec_attention_static.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, vp]
     L.spec_gemm_fused.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]
+    L.spec_gemm_swiglu.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
     L.spec_topk_scratch_bytes.argtypes = [i32, i32, i32]
     L.spec_topk_scratch_bytes.restype = sz
     L.spec_logsoftmax_topk.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
@@ -254,7 +255,7 @@ class SpecDecoder:
         self._check(lib().spec_profile_step(self.h, ms.ctypes.data, n.ctypes.data))
         return {c: (float(ms[i]), int(n[i])) for i, c in enumerate(self.PROF_CLASSES)}
 
-    TUNE_L2_LEAD_MB, TUNE_GEMM_CTAS, TUNE_DEBUG_LAUNCH_BUDGET, TUNE_CHAIN_TIMING = 1, 2, 3, 5
+    TUNE_L2_LEAD_MB, TUNE_GEMM_CTAS, TUNE_DEBUG_LAUNCH_BUDGET, TUNE_ATTN_CTAS, TUNE_CHAIN_TIMING = 1, 2, 3, 4, 5
 
     def tune(self, what: int, value: int):
         self._check(lib().spec_tune(self.h, what, value))
@@ -351,6 +352,20 @@ def gemm_fused(x: torch.Tensor, w: torch.Tensor, split: int = 0, stages: int = 0
     if rc:
         raise SpecError(rc, "spec_gemm_fused")
     return out
+
+
+def gemm_swiglu(x: torch.Tensor, w_gate: torch.Tensor, w_up: torch.Tensor) -> torch.Tensor:
+    """act = bf16(silu(x . w_gate^T) * (x . w_up^T)) on the step's gate/up kernel."""
+    rows, I = x.shape
+    F = w_gate.shape[0]
+    assert w_gate.shape == w_up.shape == (F, I) and x.dtype == w_gate.dtype == w_up.dtype == torch.bfloat16
+    assert x.is_contiguous() and w_gate.is_contiguous() and w_up.is_contiguous()
+    act = torch.empty(rows, F, dtype=torch.bfloat16, device=x.device)
+    rc = lib().spec_gemm_swiglu(x.data_ptr(), w_gate.data_ptr(), w_up.data_ptr(), act.data_ptr(), rows, F, I,
+                                _stream_ptr(None))
+    if rc:
+        raise SpecError(rc, "spec_gemm_swiglu")
+    return act
 
 
 def logsoftmax_topk(logits: torch.Tensor, K: int, two_stage: bool = True):

@@ -931,6 +931,9 @@ extern "C" int spec_tune(spec_ctx *c, int32_t what, int32_t value) {
   if (what == SPEC_TUNE_L2_LEAD_MB) {
     if (value < 0 || value > 120) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the L2 prefetch distance must be 0..120 MB");
     c->pf_lead = (size_t)value << 20;
+  } else if (what == SPEC_TUNE_ATTN_CTAS) {
+    if (value < 1 || value > 4096) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the attention CTA target must be 1..4096");
+    attn_fast_set_target_ctas(value);
   } else if (what == SPEC_TUNE_CHAIN_TIMING) {
     c->chain_timing_launch = value;
   } else if (what == SPEC_TUNE_DEBUG_LAUNCH_BUDGET) {
@@ -1092,6 +1095,27 @@ extern "C" int spec_gemm_fused(const void *x, const void *w, float *out, int32_t
   if (!fused_gemm_supported(EPI_F32, a)) return SPEC_ERR_UNSUPPORTED;
   int rc = fused_gemm_launch(g, EPI_F32, a, (cudaStream_t)stream);
   fast_gemm_forget(g);   // test buffers come and go; do not keep descriptors of freed memory
+  if (rc) return rc == -1 ? SPEC_ERR_INVALID_CFG : SPEC_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
+}
+
+extern "C" int spec_gemm_swiglu(const void *x, const void *w_gate, const void *w_up, void *act, int32_t rows, int32_t F, int32_t I,
+                                void *stream) {
+  if (!x || !w_gate || !w_up || !act) return SPEC_ERR_NULL;
+  if (rows < 1 || F < 1 || I < 1) return SPEC_ERR_INVALID_CFG;
+  static FastGemm *g = nullptr;
+  if (!g) {
+    std::string why;
+    g = fast_gemm_create(why);
+    if (!g) return SPEC_ERR_CUDA;
+  }
+  FusedGemmArgs a;
+  a.x = (const bf16 *)x; a.rows = rows; a.I = I; a.nw = 2;
+  a.w[0] = (const bf16 *)w_gate; a.w[1] = (const bf16 *)w_up; a.O[0] = a.O[1] = F;
+  a.act = (bf16 *)act;
+  if (!fused_gemm_supported(EPI_SWIGLU, a)) return SPEC_ERR_UNSUPPORTED;
+  int rc = fused_gemm_launch(g, EPI_SWIGLU, a, (cudaStream_t)stream);
+  fast_gemm_forget(g);
   if (rc) return rc == -1 ? SPEC_ERR_INVALID_CFG : SPEC_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }

@@ -696,30 +696,60 @@ __global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_consta
   }
 }
 
-// merge the splits: out = sum_s 2^((m_s - M) c) O_s / sum_s 2^((m_s - M) c) l_s
+// merge the splits: out = sum_s 2^((m_s - M) c) O_s / sum_s 2^((m_s - M) c) l_s.  One warp per (row, head): lanes first
+// fetch the (max, sum) pairs of all splits at once, then every lane adds up its HD/32 output dimensions with the
+// loads of eight splits in flight.
 template <int HD>
-__global__ void attn_combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, int nsplit, int nrh,
-                                    bf16 *__restrict__ out) {
+__global__ void __launch_bounds__(256) attn_combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, int nsplit,
+                                                           int nrh, bf16 *__restrict__ out) {
   pdl_wait();
   pdl_trigger();
-  int rh = blockIdx.x, d = threadIdx.x;
+  constexpr int DPL = HD / 32;                              // dimensions per lane
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rh = blockIdx.x * 8 + warp;
+  if (rh >= nrh) return;
   const float sc = rsqrtf((float)HD) * 1.4426950408889634f;
-  float M = -INFINITY;
-  for (int s = 0; s < nsplit; s++) M = fmaxf(M, part_ml[((size_t)s * nrh + rh) * 2]);
-  float acc = 0.0f, l = 0.0f;
-  for (int s = 0; s < nsplit; s++) {
-    float m = part_ml[((size_t)s * nrh + rh) * 2], ls = part_ml[((size_t)s * nrh + rh) * 2 + 1];
-    if (m == -INFINITY) continue;
-    float w = exp2f((m - M) * sc);
-    acc += w * part_o[((size_t)s * nrh + rh) * HD + d];
-    l += w * ls;
+  float m = -INFINITY, ls = 0.0f;                           // lane s holds split s (nsplit <= 32)
+  if (lane < nsplit) {
+    float2 ml = *(const float2 *)(part_ml + ((size_t)lane * nrh + rh) * 2);
+    m = ml.x; ls = ml.y;
   }
-  out[(size_t)rh * HD + d] = __float2bfloat16_rn(l > 0.0f ? acc / l : 0.0f);
+  float M = m;
+  for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+  const float w = (m == -INFINITY) ? 0.0f : exp2f((m - M) * sc);
+  float l = w * ls;
+  for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+  float acc[DPL];
+#pragma unroll
+  for (int e = 0; e < DPL; e++) acc[e] = 0.0f;
+  for (int s0 = 0; s0 < nsplit; s0 += 8) {
+    float v[8][DPL];
+#pragma unroll
+    for (int s = 0; s < 8; s++)
+      if (s0 + s < nsplit) {
+        const float *src = part_o + ((size_t)(s0 + s) * nrh + rh) * HD + lane * DPL;
+#pragma unroll
+        for (int e = 0; e < DPL; e++) v[s][e] = src[e];
+      }
+#pragma unroll
+    for (int s = 0; s < 8; s++) {
+      const float ws = __shfl_sync(0xffffffffu, w, (s0 + s) & 31);
+      if (s0 + s < nsplit) {
+#pragma unroll
+        for (int e = 0; e < DPL; e++) acc[e] += ws * v[s][e];
+      }
+    }
+  }
+  const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+#pragma unroll
+  for (int e = 0; e < DPL; e++) out[(size_t)rh * HD + lane * DPL + e] = __float2bfloat16_rn(acc[e] * inv);
 }
+
+int g_attn_target_ctas = 148;
 
 int pick_splits(int seqs, int G, int mtiles, int max_ctx_tiles) {
   int base = seqs * G * mtiles;
-  int want = (148 + base / 2) / base;                // the kernels run one CTA per SM (register-bound): aim at one wave
+  int want = (g_attn_target_ctas + base / 2) / base;                // the kernels run one CTA per SM (register-bound): aim at one wave
   if (want < 1) want = 1;
   int s = want < max_ctx_tiles ? want : max_ctx_tiles;
   if (s > MAX_SPLITS) s = MAX_SPLITS;
@@ -800,6 +830,7 @@ int launch_tma(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorMa
 }  // namespace
 
 void attn_fast_forget_maps() { g_kv_maps.clear(); }
+void attn_fast_set_target_ctas(int n) { g_attn_target_ctas = n; }
 
 int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail_len, bf16 *out, int rows, int H, int G,
                      int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s, bool contiguous_tail, int32_t *status) {
@@ -822,8 +853,8 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
       int rc = hd == 128 ? launch_tma<128>(p, grid, mk, mv, status, s) : launch_tma<64>(p, grid, mk, mv, status, s);
       if (rc == 0) {
         if (nsplit > 1) {
-          if (hd == 128) launch_k(attn_combine_kernel<128>, dim3(rows * H), dim3(128), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
-          else launch_k(attn_combine_kernel<64>, dim3(rows * H), dim3(64), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
+          if (hd == 128) launch_k(attn_combine_kernel<128>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
+          else launch_k(attn_combine_kernel<64>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
         }
         return nsplit > 1 ? 2 : 1;
       }
@@ -835,11 +866,11 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
   if (hd == 128) {
     if (!attr[1]) { cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[1] = true; }
     launch_k(attn_mma_kernel<128>, grid, dim3(256), smem, s, p);
-    if (nsplit > 1) launch_k(attn_combine_kernel<128>, dim3(rows * H), dim3(128), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
+    if (nsplit > 1) launch_k(attn_combine_kernel<128>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
   } else {
     if (!attr[0]) { cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[0] = true; }
     launch_k(attn_mma_kernel<64>, grid, dim3(256), smem, s, p);
-    if (nsplit > 1) launch_k(attn_combine_kernel<64>, dim3(rows * H), dim3(64), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
+    if (nsplit > 1) launch_k(attn_combine_kernel<64>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
   }
   return nsplit > 1 ? 2 : 1;
 }

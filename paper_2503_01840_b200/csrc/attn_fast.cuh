@@ -16,5 +16,7 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
 // TMA-staged kernel fetch whole pages; status: device status words for its bounded waits (may be NULL).
 // Drops the cached K/V tensor maps (pools of one-shot callers come and go).
 void attn_fast_forget_maps();
+// CTAs an attention launch aims at when it splits the keys (process-wide; default 148 = one wave)
+void attn_fast_set_target_ctas(int n);
 
 }  // namespace spec

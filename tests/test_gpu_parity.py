@@ -55,6 +55,25 @@ def test_gemm_cluster_split_k_vs_oracle(rows, O, I, split, stages):
     assert np.array_equal(out, again), "the cluster reduction must be deterministic"
 
 
+@pytest.mark.parametrize("rows,F,I", [(1, 768, 512), (7, 896, 704), (10, 1000, 1024), (16, 1024, 520), (33, 2048, 4096),
+                                      (60, 14336, 4096), (64, 1408, 576), (5, 256, 4096), (100, 1024, 512)])
+def test_gemm_swiglu_vs_oracle(rows, F, I):
+    """Gate/up projection with SiLU(gate) * up (one cluster per (gate, up) tile pair and its K slices): an odd number
+    of k-blocks, a ragged last k-block, F not a multiple of 128, every row-tile width."""
+    g = torch.Generator().manual_seed(rows * 1000 + F + I)
+    x = (torch.randn(rows, I, generator=g)).to(torch.bfloat16)
+    wg = (torch.randn(F, I, generator=g) / I ** 0.5).to(torch.bfloat16)
+    wu = (torch.randn(F, I, generator=g) / I ** 0.5).to(torch.bfloat16)
+    xf = x.float().numpy()
+    ref = po.swiglu(po.linear(wg, xf), po.linear(wu, xf))
+    out = sb.gemm_swiglu(x.cuda(), wg.cuda(), wu.cuda()).float().cpu().numpy()
+    assert np.isfinite(out).all()
+    err = np.abs(out - ref) - 2.0 ** -8 * np.abs(ref)          # one bf16 rounding of the result
+    assert err.max() < 2e-3, err.max()
+    again = sb.gemm_swiglu(x.cuda(), wg.cuda(), wu.cuda()).float().cpu().numpy()
+    assert np.array_equal(out, again), "the cluster reduction must be deterministic"
+
+
 def test_gemm_plain_fp32_vs_oracle():
     g = torch.Generator().manual_seed(5)
     x, w = torch.randn(33, 300, generator=g), torch.randn(77, 300, generator=g) / 17
