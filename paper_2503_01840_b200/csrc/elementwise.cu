@@ -216,25 +216,27 @@ __global__ void build_cat_kernel(const float *__restrict__ feat, int nparts, siz
                                  int k) {
   pdl_wait();
   pdl_trigger();
+  // one element per thread (grid.y slices of the row): every load of the launch is in flight at once
   int r = blockIdx.x;
+  int i = blockIdx.y * blockDim.x + threadIdx.x;
+  if (i >= k) return;
   T *c = cat + (size_t)r * 2 * k;
   if (seq[r] < 0) {
-    for (int i = threadIdx.x; i < 2 * k; i += blockDim.x) c[i] = from_f32<T>(0.0f);
+    c[i] = from_f32<T>(0.0f);
+    c[k + i] = from_f32<T>(0.0f);
     return;
   }
   int sr = src_row ? src_row[r] : r;
-  const T *e = embed + (size_t)tok[r] * k;
-  for (int i = threadIdx.x; i < k; i += blockDim.x) {
-    float v = 0.0f;
-    for (int p = 0; p < nparts; p++) v += feat[(size_t)p * part_stride + (size_t)sr * k + i];
-    c[i] = from_f32<T>(v);
-    c[k + i] = e[i];
-  }
+  T e = embed[(size_t)tok[r] * k + i];
+  float v = 0.0f;
+  for (int p = 0; p < nparts; p++) v += feat[(size_t)p * part_stride + (size_t)sr * k + i];
+  c[i] = from_f32<T>(v);
+  c[k + i] = e;
 }
 template <typename T>
 void launch_build_cat(const float *feat, int nparts, size_t part_stride, const int32_t *src_row, const T *embed,
                       const int32_t *tok, const int32_t *seq, T *cat, int rows, int k, cudaStream_t s) {
-  launch_k(build_cat_kernel<T>, dim3(rows), dim3(256), 0, s, feat, nparts, part_stride, src_row, embed, tok, seq, cat, k);
+  launch_k(build_cat_kernel<T>, dim3(rows, (k + 255) / 256), dim3(256), 0, s, feat, nparts, part_stride, src_row, embed, tok, seq, cat, k);
 }
 template void launch_build_cat<float>(const float *, int, size_t, const int32_t *, const float *, const int32_t *,
                                       const int32_t *, float *, int, int, cudaStream_t);

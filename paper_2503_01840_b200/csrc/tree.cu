@@ -188,11 +188,22 @@ __global__ void __launch_bounds__(256) topk_merge_kernel(const int32_t *src_row,
   int nc = nch * K;
   float *cv = (float *)smraw;              // [nc]
   int32_t *ci = (int32_t *)(cv + nc);      // [nc]
+  float *pm = (float *)(ci + nc);          // [nch]
+  float *ps = pm + nch;                    // [nch]
+  __shared__ float sv[TOPK_MAXK * TOPK_MAXK];      // candidates that can still be among the K best
+  __shared__ int32_t si[TOPK_MAXK * TOPK_MAXK];
+  __shared__ int nsurv, thr_i;
+  __shared__ float thr_v;
   for (int i = threadIdx.x; i < nc; i += blockDim.x) { cv[i] = cval[(size_t)r * nc + i]; ci[i] = cidx[(size_t)r * nc + i]; }
   float mx = -INFINITY;
-  for (int i = threadIdx.x; i < nch; i += blockDim.x) mx = fmaxf(mx, pmax[(size_t)r * nch + i]);
+  for (int i = threadIdx.x; i < nch; i += blockDim.x) {
+    float m = pmax[(size_t)r * nch + i];
+    pm[i] = m; ps[i] = psum[(size_t)r * nch + i];
+    mx = fmaxf(mx, m);
+  }
   for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
   if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = mx;
+  if (threadIdx.x == 0) { nsurv = 0; thr_i = -1; thr_v = 0.0f; }
   __syncthreads();
   mx = shf[0];
   for (int w = 1; w < 8; w++) mx = fmaxf(mx, shf[w]);
@@ -200,17 +211,37 @@ __global__ void __launch_bounds__(256) topk_merge_kernel(const int32_t *src_row,
   // chunk sums are combined in chunk order by one thread: the result does not depend on the launch shape
   if (threadIdx.x == 0) {
     float t = 0.0f;
-    for (int i = 0; i < nch; i++) t += psum[(size_t)r * nch + i] * expf(pmax[(size_t)r * nch + i] - mx);
+    for (int i = 0; i < nch; i++) t += ps[i] * expf(pm[i] - mx);
     shf[0] = logf(t);
+  }
+  // A chunk's candidates are stored best first.  With t = the K-th best of the chunks' best candidates, K
+  // candidates are at least as good as t, so a candidate after t cannot be among the K best of the row.
+  for (int ch = (int)threadIdx.x - 32; ch < nch; ch += (int)blockDim.x - 32) {       // warp 0 is busy with the sum
+    if (ch < 0) break;
+    int c0 = ch * K, my = ci[c0];
+    if (my < 0) continue;
+    float v = cv[c0];
+    int rank = 0;
+    for (int j = 0; j < nch; j++) rank += (ci[j * K] >= 0 && before(cv[j * K], ci[j * K], v, my)) ? 1 : 0;
+    if (rank == K - 1) { thr_v = v; thr_i = my; }
   }
   __syncthreads();
   float lse = shf[0];
+  const float tv = thr_v;
+  const int ti = thr_i;
   for (int i = threadIdx.x; i < nc; i += blockDim.x) {
     int my = ci[i];
-    if (my < 0) continue;
-    float v = cv[i];
+    if (my < 0 || (ti >= 0 && before(tv, ti, cv[i], my))) continue;
+    int pos = atomicAdd(&nsurv, 1);        // at most K chunks x K candidates survive; their order does not matter
+    if (pos < TOPK_MAXK * TOPK_MAXK) { sv[pos] = cv[i]; si[pos] = my; }
+  }
+  __syncthreads();
+  int ns = nsurv < TOPK_MAXK * TOPK_MAXK ? nsurv : TOPK_MAXK * TOPK_MAXK;
+  for (int i = threadIdx.x; i < ns; i += blockDim.x) {
+    int my = si[i];
+    float v = sv[i];
     int rank = 0;
-    for (int j = 0; j < nc; j++) rank += (ci[j] >= 0 && before(cv[j], ci[j], v, my)) ? 1 : 0;
+    for (int j = 0; j < ns; j++) rank += before(sv[j], si[j], v, my) ? 1 : 0;
     if (rank < K) { idx[(size_t)r * K + rank] = my; lp[(size_t)r * K + rank] = (v - mx) - lse; }
   }
 }
@@ -229,7 +260,7 @@ int launch_topk2(const float *logits, const int32_t *src_row, int rows, int n, i
   float *cval = psum + (size_t)rows * nch;
   int32_t *cidx = (int32_t *)(cval + (size_t)rows * nch * K);
   launch_k(topk_partial_kernel, dim3(nch, rows), dim3(256), 0, s, logits, src_row, n, K, nch, pmax, psum, cval, cidx);
-  size_t smem = (size_t)nch * K * 8;
+  size_t smem = (size_t)nch * K * 8 + (size_t)nch * 8;
   static size_t configured = 0;
   if (smem > 48 * 1024 && smem > configured) {
     cudaFuncSetAttribute(topk_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
