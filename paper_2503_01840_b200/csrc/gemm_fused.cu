@@ -38,7 +38,8 @@ namespace {
 using namespace tc;
 
 constexpr int MAX_STAGES = 16;
-constexpr int CHUNK = 64;                       // rows reduced per epilogue round
+constexpr int CHUNK = 64;                       // rows reduced per epilogue round (tiles of up to 64 rows)
+constexpr int MAX_CHUNK = 256;                  // wider tiles take as many rows per round as the free ring holds
 constexpr int A_BYTES = TILE_M * TILE_K * 2;    // one weight tile of a stage
 
 struct alignas(64) FusedParams {
@@ -47,6 +48,7 @@ struct alignas(64) FusedParams {
   int tiles0, tiles1;          // tile index ranges of the weights: [0,tiles0) w0, [tiles0,tiles1) w1, rest w2
   int O[3];
   int rows, KB, S, Sk, stages, ctrl_off;   // S = cluster size, Sk = K slices (S = 2 Sk for EPI_SWIGLU)
+  int chunk;                               // rows per epilogue round
   const float *ssq_in; int ssq_in_tiles, ssq_ld; float inv_k_in, eps;
   float *out_f32; int ldo;
   float *xres; const bf16 *gain; bf16 *hb; float *ssq_out; bf16 *taps; int tap_mask, resid_add;
@@ -119,7 +121,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
   uint32_t *tmem_slot = (uint32_t *)(acc_bar + 1);
   volatile uint32_t *abort_flag = tmem_slot + 1;
   float *inv_s = (float *)(ctrl + 512);          // [256] per-row input scale
-  float *wpart = inv_s + 256;                    // [4][CHUNK] per-warp partial sums / argmax exchange
+  float *wpart = inv_s + 256;                    // [4][MAX_CHUNK] per-warp partial sums / argmax exchange
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int stages = p.stages, S = p.S, Sk = p.Sk;
@@ -231,17 +233,18 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
   good = __shfl_sync(0xffffffffu, good, 0);
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
-  // ---- epilogue, CHUNK rows at a time.  The stage ring is free now (every load landed, every MMA that
+  // ---- epilogue, CH rows at a time.  The stage ring is free now (every load landed, every MMA that
   // read it completed) and is reused: red = this CTA's accumulator, sumb = this CTA's rows after the cluster sum.
-  float *red = (float *)tiles;                       // [CHUNK][128]
-  float *sumb = red + CHUNK * TILE_M;                // [CHUNK][128] (EPI_SWIGLU: gate rows, then up rows at CHUNK/2)
+  const int CH = (NT <= CHUNK || EPI == EPI_ARGMAX) ? CHUNK : p.chunk;   // a constant for the narrow tiles
+  float *red = (float *)tiles;                       // [CH][128]
+  float *sumb = red + CH * TILE_M;                   // [rows of this CTA][128] (EPI_SWIGLU: gate rows, then up rows at CH/2)
   const int f = threadIdx.x;
   const int o = tm * TILE_M + f;                     // output feature within weight mi
-  for (int c0 = 0; c0 < p.rows; c0 += CHUNK) {
-    const int nrow = (p.rows - c0 < CHUNK) ? p.rows - c0 : CHUNK;
+  for (int c0 = 0; c0 < p.rows; c0 += CH) {
+    const int nrow = (p.rows - c0 < CH) ? p.rows - c0 : CH;
     if (good) {
 #pragma unroll 1
-      for (int cc = 0; cc < CHUNK && c0 + cc < NT; cc += 16) {
+      for (int cc = 0; cc < CH && c0 + cc < NT; cc += 16) {
         if (cc >= nrow) break;
         uint32_t v[16];
         tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + cc), v);
@@ -262,10 +265,13 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
         const int i = item >> 5, qd = item & 31;
         const uint32_t la = smem_u32(&red[(r0 + i) * TILE_M + qd * 4]);
         *(float4 *)&sumb[i * TILE_M + qd * 4] = sum_peers4(la, 0, Sk);
-        if (EPI == EPI_SWIGLU) *(float4 *)&sumb[(CHUNK / 2 + i) * TILE_M + qd * 4] = sum_peers4(la, Sk, Sk);
+        if (EPI == EPI_SWIGLU) *(float4 *)&sumb[(CH / 2 + i) * TILE_M + qd * 4] = sum_peers4(la, Sk, Sk);
       }
       __syncthreads();
       src = sumb;
+      // this CTA has everything it needs from its peers: announce it now and wait only at the end of the round, so
+      // that the per-feature epilogue below runs while the slower members are still summing
+      asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     }
     // ---- phase B: per-feature epilogue from local shared memory (thread = feature f of the tile).  Rows go
     // in batches of RB: all global loads of a batch are issued before its first store, so the loop is not
@@ -301,26 +307,24 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
             }
             float sq = xo * xo;
             for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
-            if (lane == 0) wpart[warp * CHUNK + (r - r0)] = sq;
+            if (lane == 0) wpart[warp * CH + (r - r0)] = sq;
           }
         }
       }
       __syncthreads();
-      if (good && (int)threadIdx.x < r1 - r0) {
-        int t = threadIdx.x;
-        p.ssq_out[(size_t)tm * p.ssq_ld + c0 + r0 + t] =
-            ((wpart[t] + wpart[CHUNK + t]) + wpart[2 * CHUNK + t]) + wpart[3 * CHUNK + t];
-      }
+      if (good)
+        for (int t = threadIdx.x; t < r1 - r0; t += 128)
+          p.ssq_out[(size_t)tm * p.ssq_ld + c0 + r0 + t] = ((wpart[t] + wpart[CH + t]) + wpart[2 * CH + t]) + wpart[3 * CH + t];
     } else if (EPI == EPI_QKV) {
       const int hd = p.hd, half = hd >> 1;
       const int head = o / hd, i = o % hd;
       const bool valid_o = (o < p.O[mi]) && good;
       bf16 *Kp = (bf16 *)p.pool.k, *Vp = (bf16 *)p.pool.v;
       // per-row cache slot of this CTA's rows: one thread per row resolves sequence -> position -> page
-      int32_t *slot_s = (int32_t *)wpart;              // [CHUNK] element offset / hd of the row's K/V slot, -1: none
-      int32_t *seq_s = slot_s + CHUNK;                 // [CHUNK]
-      if ((int)threadIdx.x < r1 - r0) {
-        const int row = c0 + r0 + threadIdx.x;
+      int32_t *slot_s = (int32_t *)wpart;              // [CH] element offset / hd of the row's K/V slot, -1: none
+      int32_t *seq_s = slot_s + CH;                    // [CH]
+      for (int t = threadIdx.x; t < r1 - r0; t += 128) {
+        const int row = c0 + r0 + t;
         const int seq = p.m.seq[row];
         int slot = -1;
         if (seq >= 0 && mi > 0) {
@@ -333,8 +337,8 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
             else slot = (page * p.G) * p.pm.page_size + (kvpos % p.pm.page_size);   // + head * page_size below
           }
         }
-        slot_s[threadIdx.x] = slot;
-        seq_s[threadIdx.x] = seq;
+        slot_s[t] = slot;
+        seq_s[t] = seq;
       }
       __syncthreads();
       for (int rb = r0; rb < r1; rb += RB) {
@@ -365,7 +369,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       for (int r = r0; r < r1; r++) {
         const int row = c0 + r;
         const float sc = inv_s[row];
-        const float g = src[(r - r0) * TILE_M + f] * sc, u = src[(CHUNK / 2 + r - r0) * TILE_M + f] * sc;
+        const float g = src[(r - r0) * TILE_M + f] * sc, u = src[(CH / 2 + r - r0) * TILE_M + f] * sc;
         if (good && o < p.O[0]) p.act[(size_t)row * p.O[0] + o] = __float2bfloat16_rn((g / (1.0f + expf(-g))) * u);
       }
     } else {   // EPI_ARGMAX
@@ -394,9 +398,8 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       }
     }
     // peers may still be reading this CTA's red; nobody overwrites or leaves before all are done
-    if (S > 1) cluster_sync_all(); else __syncthreads();
+    if (S > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); else __syncthreads();
   }
-
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
@@ -411,7 +414,7 @@ constexpr int NUM_SMS = 148;
 constexpr int SMEM_ONE = 200 * 1024;      // ring budget with one CTA per SM
 constexpr int SMEM_TWO = 104 * 1024;      // ring budget that lets two CTAs share an SM
 
-struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB; };
+struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB, chunk; };
 
 // K slices per feature tile.  An SM streams at a capped rate whether one or two CTAs feed it, so the time
 // of a launch goes with (CTAs on the busiest SM) x (k-blocks per CTA + a fixed cost per CTA); two CTAs per SM
@@ -446,9 +449,19 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a) {
   int per_slice = (pl.KB + Sk - 1) / Sk;
   stages = std::max(2, std::min(stages, per_slice));
   pl.stages = stages;
-  const int epi_bytes = 2 * CHUNK * TILE_M * 4;   // accumulator dump + reduced rows
-  pl.ctrl_off = (std::max(stages * stage, epi_bytes) + 1023) & ~1023;
-  pl.smem = pl.ctrl_off + 512 + 256 * 4 + 4 * CHUNK * 4 + 1024 /*alignment slack*/;
+  // rows per epilogue round: accumulator dump [chunk][128] + this CTA's reduced rows; wide tiles take the most rows
+  // the stage ring (free by then) holds, which saves cluster barriers
+  auto epi_bytes = [&](int ch) {
+    const int mine = pl.S > 1 ? (ch + pl.S - 1) / pl.S : 0;
+    const int sum_rows = pl.S > 1 ? (epi == EPI_SWIGLU ? ch / 2 + mine : mine) : 0;
+    return (ch + sum_rows) * TILE_M * 4;
+  };
+  pl.chunk = CHUNK;
+  if (epi != EPI_ARGMAX)
+    for (int ch = MAX_CHUNK; ch > CHUNK; ch >>= 1)
+      if (ch <= pl.nt && epi_bytes(ch) <= std::max(stages * stage, 2 * CHUNK * TILE_M * 4)) { pl.chunk = ch; break; }
+  pl.ctrl_off = (std::max(stages * stage, std::max(epi_bytes(pl.chunk), 2 * CHUNK * TILE_M * 4)) + 1023) & ~1023;
+  pl.smem = pl.ctrl_off + 512 + 256 * 4 + 4 * MAX_CHUNK * 4 + 1024 /*alignment slack*/;
   return pl;
 }
 
@@ -538,7 +551,7 @@ int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStr
   p.map_x = *mx;
   p.tiles0 = (a.O[0] + TILE_M - 1) / TILE_M;
   p.tiles1 = p.tiles0 + (a.nw > 1 ? (a.O[1] + TILE_M - 1) / TILE_M : 0);
-  p.rows = a.rows; p.KB = pl.KB; p.S = pl.S; p.Sk = pl.Sk; p.stages = pl.stages; p.ctrl_off = pl.ctrl_off;
+  p.rows = a.rows; p.KB = pl.KB; p.S = pl.S; p.Sk = pl.Sk; p.stages = pl.stages; p.ctrl_off = pl.ctrl_off; p.chunk = pl.chunk;
   p.ssq_in = a.ssq_in; p.ssq_in_tiles = a.ssq_in_tiles; p.ssq_ld = a.ssq_ld; p.inv_k_in = 1.0f / (float)a.k_in; p.eps = a.eps;
   p.out_f32 = a.out_f32; p.ldo = a.ldo;
   p.xres = a.xres; p.gain = a.gain; p.hb = a.hb; p.ssq_out = a.ssq_out; p.taps = a.tap_mask ? a.taps : nullptr;
