@@ -407,6 +407,144 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
   }
 }
 
+// ----------------------------------------------------------------------------------------------
+// Gate/up GEMM with SiLU(gate) * up for wide row tiles (129..256 token rows).  At this width the k-block of activations
+// (32 KB) is twice a weight tile, and re-reading it from L2 for every weight tile is what bounds the loop.  Here ONE CTA
+// owns the gate tile AND the up tile of the same 128 features: both MMAs of a k-block share one activation tile
+// (64 KB per stage instead of 96), the two accumulators fill the tensor memory (2 x 256 columns), and since a thread
+// then holds gate and up of its feature for every row the activation is applied straight from the accumulators:
+// no cluster, no shared-memory round trip.
+template <int NT>
+__global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_constant__ FusedParams p) {
+  constexpr int B_BYTES = NT * TILE_K * 2;
+  constexpr int STAGE = 2 * A_BYTES + B_BYTES;
+  constexpr int TMEM_COLS = 2 * NT;
+  static_assert(TMEM_COLS <= 512, "two accumulators must fit the tensor memory");
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char *tiles = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  unsigned char *ctrl = tiles + p.ctrl_off;
+  uint64_t *full = (uint64_t *)ctrl;
+  uint64_t *empty = full + MAX_STAGES;
+  uint64_t *acc_bar = empty + MAX_STAGES;
+  uint32_t *tmem_slot = (uint32_t *)(acc_bar + 1);
+  volatile uint32_t *abort_flag = tmem_slot + 1;
+  float *inv_s = (float *)(ctrl + 512);          // [256] per-row input scale
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int stages = p.stages, KB = p.KB;
+  const int tm = blockIdx.x;                     // feature tile (of gate and of up)
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < stages; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    mbar_init(acc_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_trigger();
+
+  if (warp == 0 && lane == 0) {
+    // ---- producer: the weight tiles do not depend on the previous kernel
+    const uint64_t pol = l2_policy_evict_first();
+    const int npre = KB < stages ? KB : stages;
+    for (int i = 0; i < npre; i++) {
+      unsigned char *a = tiles + i * STAGE;
+      mbar_expect_tx(&full[i], STAGE);
+      tma_load_2d_hint(a, &p.map_w[0], i * TILE_K, tm * TILE_M, &full[i], pol);
+      tma_load_2d_hint(a + A_BYTES, &p.map_w[1], i * TILE_K, tm * TILE_M, &full[i], pol);
+    }
+    pdl_wait();
+    for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + 2 * A_BYTES, &p.map_x, i * TILE_K, 0, &full[i]);
+    for (int i = npre; i < KB; i++) {
+      const int st = i % stages;
+      if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 220, blockIdx.x, i); break; }
+      if (*abort_flag) break;
+      unsigned char *a = tiles + st * STAGE;
+      mbar_expect_tx(&full[st], STAGE);
+      tma_load_2d_hint(a, &p.map_w[0], i * TILE_K, tm * TILE_M, &full[st], pol);
+      tma_load_2d_hint(a + A_BYTES, &p.map_w[1], i * TILE_K, tm * TILE_M, &full[st], pol);
+      tma_load_2d(a + 2 * A_BYTES, &p.map_x, i * TILE_K, 0, &full[st]);
+    }
+  } else {
+    pdl_wait();
+    if (warp == 1 && lane == 0) {
+      // ---- MMA issuer: gate accumulator at column 0, up accumulator at column NT
+      constexpr uint32_t idesc = umma_idesc(NT);
+      for (int i = 0; i < KB; i++) {
+        const int st = i % stages;
+        if (!mbar_wait(&full[st], (i / stages) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 221, blockIdx.x, i); break; }
+        if (*abort_flag) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t ag = smem_u32(tiles + st * STAGE), au = ag + A_BYTES, b = ag + 2 * A_BYTES;
+#pragma unroll
+        for (int j = 0; j < TILE_K / UMMA_K; j++) {
+          const uint64_t db = umma_desc_sw128(b + j * UMMA_K * 2);
+          umma_bf16(tmem_base, umma_desc_sw128(ag + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
+          umma_bf16(tmem_base + NT, umma_desc_sw128(au + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
+        }
+        umma_commit(&empty[st]);
+      }
+      umma_commit(acc_bar);
+    } else if (warp >= 2) {
+      for (int r = threadIdx.x - 64; r < p.rows; r += 64) {
+        float sc = 1.0f;
+        if (p.ssq_in) {
+          float ss = 0.0f;
+          for (int t = 0; t < p.ssq_in_tiles; t++) ss += p.ssq_in[(size_t)t * p.ssq_ld + r];
+          sc = 1.0f / sqrtf(ss * p.inv_k_in + p.eps);
+        }
+        inv_s[r] = sc;
+      }
+    }
+  }
+  __syncthreads();
+
+  int good = 0;
+  if (lane == 0) {
+    bool ok = mbar_wait(acc_bar, 0);
+    if (!ok) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 222, blockIdx.x, 0); }
+    good = (ok && !*abort_flag) ? 1 : 0;
+  }
+  good = __shfl_sync(0xffffffffu, good, 0);
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+  // ---- epilogue: thread = feature f (tensor-memory lane), 16 rows (columns) of both accumulators at a time
+  const int o = tm * TILE_M + threadIdx.x;
+  if (good) {
+#pragma unroll 1
+    for (int cc = 0; cc < p.rows; cc += 16) {
+      uint32_t g[16], u[16];
+      tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)cc, g);
+      tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(NT + cc), u);
+      if (o < p.O[0]) {
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+          const int row = cc + j;
+          if (row < p.rows) {
+            const float sc = inv_s[row];
+            const float gv = __uint_as_float(g[j]) * sc, uv = __uint_as_float(u[j]) * sc;
+            p.act[(size_t)row * p.O[0] + o] = __float2bfloat16_rn((gv / (1.0f + expf(-gv))) * uv);
+          }
+        }
+      }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
 // ---------------------------------------------------------------------------------------------- host side
 int pick_nt(int rows) { return rows <= 16 ? 16 : rows <= 64 ? 64 : rows <= 128 ? 128 : 256; }
 
@@ -422,7 +560,8 @@ struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB, chunk; };
 int g_target_ctas = 222;   // measured best on the 8B shapes (1.5 CTAs per SM)
 constexpr int MAX_CLUSTER = 8;    // portable cluster sizes only: size 9 (non-portable) measured 20 % slower per step
 
-Plan make_plan(FusedEpi epi, const FusedGemmArgs &a) {
+// force_two: plan a wide tile (whose full ring takes the SM) as two CTAs per SM with two-stage rings
+Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false) {
   Plan pl;
   pl.nt = pick_nt(a.rows);
   pl.KB = (a.I + TILE_K - 1) / TILE_K;
@@ -430,7 +569,8 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a) {
   const int stage = A_BYTES + pl.nt * TILE_K * 2;
   const int wmul = epi == EPI_SWIGLU ? 2 : 1;          // cluster members per K slice
   const int smax = MAX_CLUSTER / wmul;
-  const bool one_per_sm = SMEM_TWO / stage < 3;        // 256-row tiles: the ring of one CTA takes the SM
+  const bool wide = SMEM_TWO / stage < 3;              // 256-row tiles: the ring of one CTA takes the SM
+  const bool one_per_sm = wide && !force_two;
   const int target = one_per_sm ? NUM_SMS : g_target_ctas;   // one wave
   int Sk = 1;
   if (epi != EPI_ARGMAX) {
@@ -443,7 +583,7 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a) {
   pl.Sk = Sk;
   pl.S = Sk * wmul;
   // more tiles than SMs and a ring that fills the SM: two CTAs with two stages each beat two waves of one
-  const int budget = !one_per_sm ? SMEM_TWO : (pl.tiles * wmul * Sk > NUM_SMS ? 2 * stage : SMEM_ONE);
+  const int budget = !wide ? SMEM_TWO : ((force_two || pl.tiles * wmul * Sk > NUM_SMS) ? 2 * stage : SMEM_ONE);
   int stages = std::max(2, std::min(MAX_STAGES, budget / stage));
   if (a.stages > 0) stages = std::max(2, std::min(std::min(a.stages, MAX_STAGES), (220 * 1024) / stage));
   int per_slice = (pl.KB + Sk - 1) / Sk;
@@ -500,6 +640,37 @@ int launch_inst(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) 
   return cudaLaunchKernelEx(&cfg, gemm_fused_kernel<NT, EPI>, p) == cudaSuccess ? 0 : -6;
 }
 
+// clusters of the plan's shape that can be resident at once (0: unknown)
+template <int NT, int EPI>
+int resident_clusters_inst(const Plan &pl) {
+  static int cached_smem = -1, cached_S = -1, cached_n = 0;
+  if (cached_smem == pl.smem && cached_S == pl.S) return cached_n;
+  if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem) != cudaSuccess) return 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(pl.tiles, pl.S, 1);
+  cfg.blockDim = dim3(128, 1, 1);
+  cfg.dynamicSmemBytes = pl.smem;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = pl.S; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, gemm_fused_kernel<NT, EPI>, &cfg) != cudaSuccess) { cudaGetLastError(); n = 0; }
+  cached_smem = pl.smem; cached_S = pl.S; cached_n = n;
+  return n;
+}
+int resident_clusters_wide(FusedEpi epi, const Plan &pl) {
+  if (pl.nt != 256) return 0;
+  switch (epi) {
+    case EPI_F32: return resident_clusters_inst<256, EPI_F32>(pl);
+    case EPI_RESID: return resident_clusters_inst<256, EPI_RESID>(pl);
+    case EPI_QKV: return resident_clusters_inst<256, EPI_QKV>(pl);
+    case EPI_SWIGLU: return resident_clusters_inst<256, EPI_SWIGLU>(pl);
+    default: return 0;
+  }
+}
+
 template <int EPI>
 int launch_epi(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) {
   switch (pl.nt) {
@@ -538,6 +709,11 @@ bool fused_gemm_supported(FusedEpi epi, const FusedGemmArgs &a) {
 int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStream_t s) {
   if (!g || !fused_gemm_supported(epi, a)) return -1;
   Plan pl = make_plan(epi, a);
+  if (pl.nt == 256 && pl.S > 1 && a.split == 0 && a.stages == 0 && pl.tiles * pl.S <= NUM_SMS) {
+    // clusters are placed inside one GPC: a grid that counts fewer CTAs than SMs can still need a second wave
+    const int fit = resident_clusters_wide(epi, pl);
+    if (fit > 0 && pl.tiles > fit) pl = make_plan(epi, a, true);
+  }
   FusedParams p;
   memset(&p, 0, sizeof p);
   for (int j = 0; j < a.nw; j++) {
@@ -566,6 +742,31 @@ int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStr
     p.pf_ptr[p.npf] = (const unsigned char *)a.pf_ptr[j];
     p.pf_bytes[p.npf] = a.pf_bytes[j] & ~(size_t)15;
     p.npf++;
+  }
+  if (epi == EPI_SWIGLU && pl.nt == 256 && a.split == 0 && a.stages == 0) {
+    // wide rows: one CTA per (gate tile, up tile) pair sharing the activation tiles
+    constexpr int STAGE2 = 2 * A_BYTES + 256 * TILE_K * 2;
+    p.stages = std::max(2, std::min(SMEM_ONE / STAGE2, pl.KB));
+    p.S = 1; p.Sk = 1;
+    p.ctrl_off = (p.stages * STAGE2 + 1023) & ~1023;
+    const int smem = p.ctrl_off + 512 + 256 * 4 + 1024;
+    static int configured = 0;
+    if (smem > configured) {
+      if (cudaFuncSetAttribute(gemm_swiglu_pair_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -6;
+      configured = smem;
+    }
+    if (!launch_allowed()) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.tiles0, 1, 1);
+    cfg.blockDim = dim3(128, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = a.pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, gemm_swiglu_pair_kernel<256>, p) == cudaSuccess ? 0 : -6;
   }
   switch (epi) {
     case EPI_F32: return launch_epi<EPI_F32>(p, pl, a.pdl, s);
