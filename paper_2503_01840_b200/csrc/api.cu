@@ -215,6 +215,7 @@ static size_t carve(spec_ctx *c, void *base) {
   c->st.n = cv.take<int32_t>(B); c->st.n_prev = cv.take<int32_t>(B); c->st.P = cv.take<int32_t>(B);
   c->st.root = cv.take<int32_t>(B); c->st.cap = cv.take<int32_t>(B); c->st.last_row = cv.take<int32_t>(B);
   c->st.active = cv.take<int32_t>(B);
+  c->st.order = cv.take<int32_t>(B);
   TreeBufs &t = c->tb;
   t.pool = c->pool; t.K = c->K; t.D = c->D; t.N = c->N; t.Pmax = c->Pmax;
   size_t pe = (size_t)B * (c->pool + 1);
@@ -298,6 +299,9 @@ extern "C" int spec_init(spec_ctx **out, const spec_target_weights *tw, const sp
   for (int i = 0; i < c->hd / 2; i++) inv[i] = pow((double)cfg->rope_theta, -2.0 * (double)i / (double)c->hd);
   if (e == cudaSuccess) e = cudaMemcpyAsync(c->inv_freq, inv.data(), inv.size() * 8, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(c->pools_dev, c->pools.data(), sizeof(KvPool) * (c->L + 1), cudaMemcpyHostToDevice, s);
+  std::vector<int32_t> ident(c->B);
+  for (int b = 0; b < c->B; b++) ident[b] = b;
+  if (e == cudaSuccess) e = cudaMemcpyAsync(c->st.order, ident.data(), sizeof(int32_t) * c->B, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) {
     int rc = fail(nullptr, SPEC_ERR_CUDA, "spec_init: %s", cudaGetErrorString(e));
@@ -551,7 +555,8 @@ template <typename T> struct Sched {
       int hint = 0;
       for (int b = 0; b < c->B; b++) hint = std::max(hint, c->n_upper[b]);
       tick(launch_attn_fast((const bf16 *)c->q, pool, pm, c->meta, tail_len, (bf16 *)c->ao, rows, c->H, c->G, c->hd,
-                            c->cur_rps, hint, c->attn_scratch, s, !(c->cfg.flags & SPEC_FLAG_NO_TMA_ATTN), c->status));
+                            c->cur_rps, hint, c->attn_scratch, s, !(c->cfg.flags & SPEC_FLAG_NO_TMA_ATTN), c->status,
+                            c->st.order, c->B));
     } else {
       launch_attn_ref<T>((const T *)c->q, pool, pm, c->meta, tail_len, (T *)c->ao, rows, c->H, c->G, c->hd,
                          c->cfg.max_ctx + tail_len, s);

@@ -60,6 +60,7 @@ struct AttnParams {
   bf16 *out;
   float *part_o;    // [nsplit][rows*H][hd]
   float *part_ml;   // [nsplit][rows*H][2]
+  const int32_t *order;   // row block handled by the i-th CTA group (nullptr: i)
 };
 
 template <int HD>
@@ -297,7 +298,9 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
   uint64_t *q_bar = empty + STAGES;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int grp = p.H / p.G;
-  const int b = blockIdx.z / p.G, g = blockIdx.z % p.G;
+  const int zb = blockIdx.z / p.G, g = blockIdx.z % p.G;
+  int b = p.order ? p.order[zb] : zb;            // row block (sequence) of this CTA
+  if ((unsigned)b >= gridDim.z / (unsigned)p.G) b = zb;
   const int M = p.rps * grp;
   const int m0 = blockIdx.x * MT;
   const int row0 = b * p.rps;
@@ -518,7 +521,9 @@ __global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_consta
   unsigned char *sQ = sm + STAGES * 2 * TILEB + 256;   // [16][HD] bf16, swizzled
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int grp = p.H / p.G;
-  const int b = blockIdx.z / p.G, g = blockIdx.z % p.G;
+  const int zb = blockIdx.z / p.G, g = blockIdx.z % p.G;
+  int b = p.order ? p.order[zb] : zb;            // row block (sequence) of this CTA
+  if ((unsigned)b >= gridDim.z / (unsigned)p.G) b = zb;
   const int M = p.rps * grp;                           // <= 16
   const int row0 = b * p.rps;
   const int ps = p.pm.page_size;
@@ -833,7 +838,8 @@ void attn_fast_forget_maps() { g_kv_maps.clear(); }
 void attn_fast_set_target_ctas(int n) { g_attn_target_ctas = n; }
 
 int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail_len, bf16 *out, int rows, int H, int G,
-                     int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s, bool contiguous_tail, int32_t *status) {
+                     int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s, bool contiguous_tail, int32_t *status,
+                     const int32_t *order, int order_len) {
   if (rps < 1 || rows % rps) rps = 1;
   int seqs = rows / rps, grp = H / G;
   int mtiles = (rps * grp + MT - 1) / MT;
@@ -843,6 +849,7 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
   p.q = q; p.kpool = (const bf16 *)pool.k; p.vpool = (const bf16 *)pool.v; p.pm = pm; p.m = m; p.tail_len = tail_len;
   p.rows = rows; p.H = H; p.G = G; p.rps = rps; p.nsplit = nsplit; p.out = out;
   p.part_o = (float *)scratch;
+  p.order = (order && order_len == seqs) ? order : nullptr;
   p.part_ml = p.part_o ? p.part_o + (size_t)MAX_SPLITS * rows * H * hd : nullptr;
   dim3 grid(mtiles, nsplit, seqs * G);
   // TMA-staged kernel when the tail follows the context and a page is a whole number of 128-byte-swizzle boxes

@@ -12,6 +12,7 @@ struct SeqState {        // arrays of [batch]
   int32_t *cap;          // positions this sequence has pages for
   int32_t *last_row;     // row of the last pending entry in the extend pass
   int32_t *active;       // 0: sequence skipped this step (capacity)
+  int32_t *order;        // sequence indices by decreasing committed length: the order attention CTAs are issued in
 };
 
 struct TreeBufs {

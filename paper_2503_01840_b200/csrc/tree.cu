@@ -291,6 +291,15 @@ void launch_argmax_merge(const float *best_val, const int32_t *best_idx, int til
   launch_k(argmax_merge_kernel, dim3(rows), dim3(256), 0, s, best_val, best_idx, tiles, ld, out);
 }
 
+__device__ __forceinline__ int block_sum_int(int v) {
+  __shared__ int acc;
+  if (threadIdx.x == 0) acc = 0;
+  __syncthreads();
+  if (v) atomicAdd(&acc, v);
+  __syncthreads();
+  return acc;
+}
+
 // ---------------------------------------------------------------- step set-up: rows of the extend pass
 // Row b*Pmax + j is pending entry j of sequence b: position n-P+j, causal among the pending rows.
 __global__ void prep_extend_kernel(SeqState st, TreeBufs tb, RowMeta m, int need_positions, int32_t *status) {
@@ -299,7 +308,16 @@ __global__ void prep_extend_kernel(SeqState st, TreeBufs tb, RowMeta m, int need
   int b = blockIdx.x, j = threadIdx.x;
   int n = st.n[b], P = st.P[b];
   bool ok = (n + need_positions <= st.cap[b]) && P >= 1 && P <= tb.Pmax;
+  // rank of this sequence by (length desc, index asc): longest sequences get their attention CTAs first, which
+  // packs CTAs of unequal length into fewer waves
+  int longer = 0;
+  for (int o = j; o < (int)gridDim.x; o += blockDim.x) {
+    int no = st.n[o];
+    longer += (no > n || (no == n && o < b)) ? 1 : 0;
+  }
+  longer = block_sum_int(longer);
   if (j == 0) {
+    st.order[longer] = b;
     st.active[b] = ok ? 1 : 0;
     st.last_row[b] = ok ? b * tb.Pmax + P - 1 : -1;
     if (!ok) set_status(status, ST_CAPACITY, 10, b, n);
