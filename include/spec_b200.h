@@ -148,7 +148,9 @@ int spec_profile_step(spec_ctx *ctx, float *class_ms, int32_t *class_launches);
 enum spec_tune_knob { SPEC_TUNE_L2_LEAD_MB = 1, SPEC_TUNE_GEMM_CTAS = 2,
                       SPEC_TUNE_DEBUG_LAUNCH_BUDGET = 3 /* debugging: run only the first n kernels of each step (-1: all) */,
                       SPEC_TUNE_ATTN_CTAS = 4 /* CTAs an attention launch aims at when splitting keys (process-wide) */,
-                      SPEC_TUNE_CHAIN_TIMING = 5 /* profiling: record phase time stamps of the n-th chain launch of a step (-1: none) */ };
+                      SPEC_TUNE_CHAIN_TIMING = 5 /* profiling: record phase time stamps of the n-th chain launch of a step (-1: none) */,
+                      SPEC_TUNE_ATTN_UMMA = 6 /* tree passes (head_dim 128): 1 = tcgen05 attention kernel, 0 = mma.sync kernel, 2 (default) = tcgen05
+                                                  when every CTA gets several key tiles, i.e. long contexts (process-wide) */ };
 int spec_tune(spec_ctx *ctx, int32_t what, int32_t value);
 
 /* Number of kernels one spec_step launches (for launch accounting). */
@@ -225,7 +227,9 @@ int spec_gemm_swiglu(const void *x, const void *w_gate, const void *w_up, void *
  * tail_base (first tail position), mask lo/hi (bit t: tail position tail_base+t visible);
  * out [rows][H][hd] dtype.  impl 0: tensor-core kernel (bf16), 1: plain kernel, 2: tensor-core kernel with
  * TMA-staged K/V pages (bf16; needs row_tail_base[r] == row_ctx[r] for every row and page_size 16, 32 or 64;
- * other shapes fall back to impl 0).
+ * other shapes fall back to impl 0), 3: tcgen05 kernel (bf16, head_dim 128, the conditions of impl 2, and ALL rows
+ * belong to one sequence: equal row_seq and row_ctx; S = Q K^T and O += P V on tcgen05.mma with TMEM accumulators;
+ * other shapes fall back to impl 2).
  * scratch: spec_attn_scratch_bytes(...) bytes of device memory for split-KV partial results. */
 size_t spec_attn_scratch_bytes(int32_t rows, int32_t n_heads, int32_t head_dim, int32_t max_ctx);
 int spec_attention(int32_t dtype, int32_t impl, const void *q, const void *k_pool, const void *v_pool,

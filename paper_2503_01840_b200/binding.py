@@ -255,7 +255,7 @@ class SpecDecoder:
         self._check(lib().spec_profile_step(self.h, ms.ctypes.data, n.ctypes.data))
         return {c: (float(ms[i]), int(n[i])) for i, c in enumerate(self.PROF_CLASSES)}
 
-    TUNE_L2_LEAD_MB, TUNE_GEMM_CTAS, TUNE_DEBUG_LAUNCH_BUDGET, TUNE_ATTN_CTAS, TUNE_CHAIN_TIMING = 1, 2, 3, 4, 5
+    TUNE_L2_LEAD_MB, TUNE_GEMM_CTAS, TUNE_DEBUG_LAUNCH_BUDGET, TUNE_ATTN_CTAS, TUNE_CHAIN_TIMING, TUNE_ATTN_UMMA = 1, 2, 3, 4, 5, 6
 
     def tune(self, what: int, value: int):
         self._check(lib().spec_tune(self.h, what, value))

@@ -939,6 +939,9 @@ extern "C" int spec_tune(spec_ctx *c, int32_t what, int32_t value) {
   } else if (what == SPEC_TUNE_ATTN_CTAS) {
     if (value < 1 || value > 4096) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the attention CTA target must be 1..4096");
     attn_fast_set_target_ctas(value);
+  } else if (what == SPEC_TUNE_ATTN_UMMA) {
+    if (value < 0 || value > 2) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the tcgen05 attention mode must be 0, 1 or 2");
+    attn_fast_set_umma(value);
   } else if (what == SPEC_TUNE_CHAIN_TIMING) {
     c->chain_timing_launch = value;
   } else if (what == SPEC_TUNE_DEBUG_LAUNCH_BUDGET) {
@@ -1143,7 +1146,7 @@ extern "C" int spec_attention(int32_t dtype, int32_t impl, const void *q, const 
   m.mask_lo = (uint64_t *)row_mask_lo; m.mask_hi = (uint64_t *)row_mask_hi;
   KvPool pool{(void *)k_pool, (void *)v_pool};
   PageMap pm{page_table, pages_per_seq, page_size, 1 << 30};
-  if (impl < 0 || impl > 2) return SPEC_ERR_INVALID_CFG;
+  if (impl < 0 || impl > 3) return SPEC_ERR_INVALID_CFG;
   if (impl == 1) {
     if (dtype == SPEC_F32) launch_attn_ref<float>((const float *)q, pool, pm, m, tail_len, (float *)out, rows, H, G, hd, max_ctx + tail_len, s);
     else if (dtype == SPEC_BF16) launch_attn_ref<bf16>((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, max_ctx + tail_len, s);
@@ -1151,7 +1154,10 @@ extern "C" int spec_attention(int32_t dtype, int32_t impl, const void *q, const 
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
   }
   if (dtype != SPEC_BF16 || !attn_fast_supported(hd, H / G)) return SPEC_ERR_UNSUPPORTED;
-  launch_attn_fast((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, 1, max_ctx, scratch, s, impl == 2, nullptr);
+  // impl 3: the rows are one block of one sequence, which is what the tcgen05 kernel tiles over
+  attn_fast_override_umma(impl == 3 ? 1 : 0);
+  launch_attn_fast((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, impl == 3 ? rows : 1, max_ctx, scratch, s, impl >= 2, nullptr);
+  attn_fast_override_umma(-1);
   attn_fast_forget_maps();
   return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }

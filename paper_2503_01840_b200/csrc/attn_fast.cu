@@ -17,6 +17,7 @@
 #include <tuple>
 
 #include "attn_fast.cuh"
+#include "tcgen05_ptx.cuh"
 
 namespace spec {
 
@@ -502,6 +503,339 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
 }
 
 // ------------------------------------------------------------------------------------------------
+// tcgen05 variant for head_dim 128 and more than 16 query rows per (sequence, KV head): the tree passes (verify,
+// wide draft levels).  With a long context this pass is bound by the two contractions, not by the cache reads, so
+// they run on the fifth-generation tensor cores:
+//   S = Q K^T : A = the CTA's 128 query rows (K-major, 128-byte swizzle, written once), B = a 64-key K tile as it lands
+//               from TMA ([hd half][key][128 B]), accumulator = 64 columns of tensor memory;
+//   O += P V  : A = P (bf16, written to shared memory by the softmax threads), B = the V tile read MN-major (the keys
+//               are the contraction dimension and the slow axis of the tile), accumulator = 128 columns that stay in
+//               tensor memory for the whole key range.
+// Thread r of the four softmax warps owns query row r = tensor-memory lane r: its row maximum and row sum need no
+// shuffles.  When a row maximum grows, the warp rescales its 32 rows of O in tensor memory (rare once the maximum has
+// settled).  Warp 4 is the TMA producer, warp 5 issues the MMAs.  Same masks, statistics and partial-result format as
+// the kernels above.  Every wait is bounded; a timeout is recorded in the status words and the CTA winds down.
+constexpr int UM_STAGES = 4;
+constexpr int UM_HD = 128;
+constexpr int UM_TILE = KT * UM_HD * 2;            // 16 KB: the K (or the V) tile of 64 keys
+constexpr int UM_HALF = KT * 128;                  // 8 KB: one 64-element half of head_dim for 64 keys
+constexpr int UM_Q_BYTES = MT * UM_HD * 2;         // 32 KB
+constexpr int UM_P_BYTES = MT * KT * 2;            // 16 KB
+constexpr int UM_SMEM = UM_Q_BYTES + UM_P_BYTES + UM_STAGES * 2 * UM_TILE + 128;
+constexpr uint32_t UM_TMEM_COLS = 256;             // S (two buffers): columns 0..127, O: columns 128..255
+
+// MN-major operand tile with 128-byte swizzle: rows (contraction index) of 128 bytes = 64 elements of the MN
+// dimension, 8-row groups 1024 bytes apart, the next 64 MN elements lbo bytes further on.
+__device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t saddr, uint32_t lbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
+  d |= (uint64_t)(lbo >> 4) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// 64 consecutive columns of this thread's tensor-memory lane in one instruction
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&v)[64]) {
+  uint32_t *u = (uint32_t *)v;
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+      "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]), "=r"(u[9]), "=r"(u[10]),
+        "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]),
+        "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]),
+        "=r"(u[31]), "=r"(u[32]), "=r"(u[33]), "=r"(u[34]), "=r"(u[35]), "=r"(u[36]), "=r"(u[37]), "=r"(u[38]), "=r"(u[39]), "=r"(u[40]),
+        "=r"(u[41]), "=r"(u[42]), "=r"(u[43]), "=r"(u[44]), "=r"(u[45]), "=r"(u[46]), "=r"(u[47]), "=r"(u[48]), "=r"(u[49]), "=r"(u[50]),
+        "=r"(u[51]), "=r"(u[52]), "=r"(u[53]), "=r"(u[54]), "=r"(u[55]), "=r"(u[56]), "=r"(u[57]), "=r"(u[58]), "=r"(u[59]), "=r"(u[60]),
+        "=r"(u[61]), "=r"(u[62]), "=r"(u[63])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// 2^x on the special-function unit (x = -inf gives 0)
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
+      "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
+
+__global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant__ CUtensorMap map_k,
+                                                        const __grid_constant__ CUtensorMap map_v, AttnParams p, int32_t *status) {
+  pdl_wait();
+  pdl_trigger();
+  constexpr int HD = UM_HD;
+  extern __shared__ __align__(1024) unsigned char sm[];
+  unsigned char *sQ = sm;                                   // [2 halves][128 rows][128 B]
+  unsigned char *sP = sm + UM_Q_BYTES;                      // [128 rows][128 B]: 64 keys
+  unsigned char *ring = sP + UM_P_BYTES;                    // stage: K [2 halves][64 keys][128 B], then V likewise
+  uint64_t *full = (uint64_t *)(ring + UM_STAGES * 2 * UM_TILE);
+  uint64_t *empty = full + UM_STAGES;
+  uint64_t *s_bar = empty + UM_STAGES, *p_bar = s_bar + 2, *o_bar = p_bar + 1;       // s_bar[2]: one per S buffer
+  uint32_t *tmem_slot = (uint32_t *)(o_bar + 1);
+  volatile uint32_t *abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int grp = p.H / p.G;
+  const int zb = blockIdx.z / p.G, g = blockIdx.z % p.G;
+  int b = p.order ? p.order[zb] : zb;                       // row block (sequence) of this CTA
+  if ((unsigned)b >= gridDim.z / (unsigned)p.G) b = zb;
+  const int M = p.rps * grp;
+  const int m0 = blockIdx.x * MT;
+  const int row0 = b * p.rps;
+  const int ps = p.pm.page_size;
+  int seq = -1, ctx = 0;
+  for (int i = 0; i < p.rps; i++) {
+    int s = p.m.seq[row0 + i];
+    if (s >= 0) { seq = s; ctx = p.m.ctx[row0 + i]; break; }
+  }
+  const int nkeys = (seq >= 0) ? ctx + p.tail_len : 0;
+  const int ntiles = (nkeys + KT - 1) / KT;
+  const int t_begin = (int)(((long long)blockIdx.y * ntiles) / p.nsplit);
+  const int t_end = (int)(((long long)(blockIdx.y + 1) * ntiles) / p.nsplit);
+  const int ntl = t_end - t_begin;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < UM_STAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    mbar_init(&s_bar[0], 1);
+    mbar_init(&s_bar[1], 1);
+    mbar_init(p_bar, 128);
+    mbar_init(o_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(UM_TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // ---- Q tile -> shared in the operand layout: row lr, 16-byte chunk c -> half c / 8, chunk (c % 8) ^ (lr % 8)
+  const int lr = threadIdx.x;                               // softmax threads: query row within the tile
+  const int mrow = m0 + lr;
+  bool rvalid = false;
+  uint64_t mlo = 0, mhi = 0;
+  int qi = 0, qh = 0;
+  if (warp < 4) {
+    if (mrow < M) { qi = mrow / grp; qh = mrow % grp; rvalid = p.m.seq[row0 + qi] >= 0; }
+    if (rvalid) { mlo = p.m.mask_lo[row0 + qi]; mhi = p.m.mask_hi[row0 + qi]; }
+    const uint4 *src = (const uint4 *)(p.q + ((size_t)(row0 + qi) * p.H + g * grp + qh) * HD);
+#pragma unroll
+    for (int c = 0; c < HD / 8; c++) {
+      uint4 v = rvalid ? src[c] : make_uint4(0u, 0u, 0u, 0u);
+      *(uint4 *)(sQ + (c >> 3) * (MT * 128) + lr * 128 + (((c & 7) ^ (lr & 7)) << 4)) = v;
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * KT;
+
+  if (warp == 4) {
+    // ================================================================ producer
+    if (lane == 0 && seq >= 0) {
+      const int32_t *tbl = p.pm.table + (size_t)seq * p.pm.pages_per_seq;
+      const int fallback = tbl[0];                     // keys past the last page are masked; they still need a valid source
+      const int ppt = KT / ps;                         // pages per tile
+      for (int i = 0; i < ntl; i++) {
+        const int t = t_begin + i, st = i % UM_STAGES;
+        if (i >= UM_STAGES && !mbar_wait(&empty[st], (uint32_t)(((i / UM_STAGES) - 1) & 1))) {
+          *abort_flag = 1;
+          if (status) set_status(status, ST_TIMEOUT, 420, blockIdx.z, t);
+          break;
+        }
+        if (*abort_flag) break;
+        unsigned char *kb = ring + st * 2 * UM_TILE, *vb = kb + UM_TILE;
+        mbar_expect_tx(&full[st], 2 * UM_TILE);
+        for (int pg = 0; pg < ppt; pg++) {
+          const int pidx = (t * KT) / ps + pg;
+          int page = pidx < p.pm.pages_per_seq ? tbl[pidx] : -1;
+          if (page < 0 || page >= p.pm.num_pages) page = fallback;
+          const int row = (page * p.G + g) * ps;
+#pragma unroll
+          for (int h = 0; h < 2; h++) {
+            tma_load_3d(kb + h * UM_HALF + pg * ps * 128, &map_k, 0, row, h, &full[st]);
+            tma_load_3d(vb + h * UM_HALF + pg * ps * 128, &map_v, 0, row, h, &full[st]);
+          }
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ================================================================ MMA issuer
+    if (lane == 0 && ntl > 0) {
+      constexpr uint32_t idesc_s = tc::umma_idesc(KT);                       // N = 64 keys, both operands K-major
+      constexpr uint32_t idesc_o = tc::umma_idesc(HD) | (1u << 16);          // N = 128, B (the V tile) MN-major
+      const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP);
+      // S of tile i goes to S buffer i % 2: the scores of tile i + 1 are computed while the softmax threads work on tile i
+      auto issue_s = [&](int i) {
+        const int st = i % UM_STAGES;
+        const uint32_t k_addr = smem_u32(ring + st * 2 * UM_TILE);
+        const uint32_t d = tmem_s + (uint32_t)((i & 1) * KT);
+#pragma unroll
+        for (int h = 0; h < 2; h++)
+#pragma unroll
+          for (int j = 0; j < 64 / tc::UMMA_K; j++)
+            tc::umma_bf16(d, tc::umma_desc_sw128(q_addr + h * (MT * 128) + j * 32), tc::umma_desc_sw128(k_addr + h * UM_HALF + j * 32),
+                          idesc_s, (h | j) ? 1u : 0u);
+        tc::umma_commit(&s_bar[i & 1]);
+      };
+      bool ok = true;
+      for (int i = 0; i < 2 && i < ntl && ok; i++) {
+        ok = mbar_wait(&full[i % UM_STAGES], 0);
+        if (!ok) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 421, blockIdx.z, t_begin + i); break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        issue_s(i);
+      }
+      if (ok) {
+        for (int i = 0; i < ntl; i++) {
+          const int st = i % UM_STAGES;
+          if (!mbar_wait(p_bar, (uint32_t)(i & 1))) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 422, blockIdx.z, t_begin + i); break; }
+          if (*abort_flag) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t v_addr = smem_u32(ring + st * 2 * UM_TILE + UM_TILE);
+#pragma unroll
+          for (int kk = 0; kk < KT / tc::UMMA_K; kk++)
+            tc::umma_bf16(tmem_o, tc::umma_desc_sw128(p_addr + kk * 32), umma_desc_sw128_mn(v_addr + kk * (tc::UMMA_K * 128), UM_HALF), idesc_o,
+                          (i | kk) ? 1u : 0u);
+          tc::umma_commit(o_bar);
+          tc::umma_commit(&empty[st]);
+          if (i + 2 < ntl) {          // S buffer i % 2 is free: the softmax threads read it before they arrived on p_bar
+            const int st2 = (i + 2) % UM_STAGES;
+            if (!mbar_wait(&full[st2], (uint32_t)(((i + 2) / UM_STAGES) & 1))) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 423, blockIdx.z, t_begin + i + 2); break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            issue_s(i + 2);
+          }
+        }
+      }
+    }
+  } else {
+    // ================================================================ softmax: thread = query row = tensor-memory lane
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    float mx = -INFINITY, l = 0.0f;
+    const float sc = rsqrtf((float)HD) * 1.4426950408889634f;    // softmax scale folded into exp2
+    bool alive = true;
+    for (int i = 0; i < ntl; i++) {
+      const int t = t_begin + i;
+      bool ok = mbar_wait(&s_bar[i & 1], (uint32_t)((i >> 1) & 1));
+      ok = __all_sync(0xffffffffu, ok && !*abort_flag);
+      if (!ok) { if (lane == 0) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 424, blockIdx.z, t); } alive = false; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      float s[KT];
+      tmem_ld64(tmem_s + lane_base + (uint32_t)((i & 1) * KT), s);
+      // Padding rows (beyond the tile's last row, or of a skipped sequence) run the loop like real rows and are
+      // zeroed at the end: their Q is zero, and a row that always took the masked path would slow its whole warp.
+      float tm = -INFINITY;
+      if (t * KT + KT <= ctx) {
+#pragma unroll
+        for (int j = 0; j < KT; j++) tm = fmaxf(tm, s[j]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < KT; j++) {
+          const int key = t * KT + j, tt = key - ctx;
+          const bool in_ctx = key < ctx;
+          const bool in_tail = !in_ctx && tt < p.tail_len;
+          const bool okk = in_ctx || (in_tail && (!rvalid || ((tt < 64 ? (mlo >> tt) : (mhi >> (tt - 64))) & 1ull)));
+          s[j] = okk ? s[j] : -INFINITY;
+          tm = fmaxf(tm, s[j]);
+        }
+      }
+      // The reference maximum of a row moves only when the tile maximum exceeds it by more than 2^8 in the exponent:
+      // the probabilities stay below 256 (exact in the fp32 sums, 8 mantissa bits in P as always) and O is rescaled
+      // rarely; the (reference, sum, O) triple stays consistent, which is all the final division or the merge needs.
+      float nm = mx, f = 1.0f;
+      if (tm > mx && (mx == -INFINITY || (tm - mx) * sc > 8.0f)) {
+        nm = tm;
+        f = (mx == -INFINITY) ? 1.0f : ex2_approx((mx - nm) * sc);      // nothing accumulated yet: nothing to rescale
+      }
+      const float nb = (nm == -INFINITY) ? 0.0f : nm * sc;
+      float rs = 0.0f;
+      uint32_t pk[KT / 2];
+#pragma unroll
+      for (int j = 0; j < KT; j += 2) {
+        const float p0 = ex2_approx(fmaf(s[j], sc, -nb)), p1 = ex2_approx(fmaf(s[j + 1], sc, -nb));
+        rs += p0 + p1;
+        pk[j >> 1] = pack_bf16(p0, p1);
+      }
+      l = l * f + rs;
+      mx = nm;
+      // the previous tile's P V must be complete before O is rescaled and before P is overwritten
+      if (i > 0) {
+        bool ok2 = mbar_wait(o_bar, (uint32_t)((i - 1) & 1));
+        ok2 = __all_sync(0xffffffffu, ok2 && !*abort_flag);
+        if (!ok2) { if (lane == 0) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 425, blockIdx.z, t); } alive = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (__any_sync(0xffffffffu, f != 1.0f)) {
+#pragma unroll 1
+          for (int c = 0; c < HD / 16; c++) {
+            uint32_t v[16];
+            tc::tmem_ld16(tmem_o + lane_base + c * 16, v);
+#pragma unroll
+            for (int j = 0; j < 16; j++) v[j] = __float_as_uint(__uint_as_float(v[j]) * f);
+            tmem_st16(tmem_o + lane_base + c * 16, v);
+          }
+          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < KT / 8; c++)
+        *(uint4 *)(sP + lr * 128 + ((c ^ (lr & 7)) << 4)) = make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      mbar_arrive(p_bar);
+    }
+    if (alive && ntl > 0) {
+      bool ok = mbar_wait(o_bar, (uint32_t)((ntl - 1) & 1));
+      ok = __all_sync(0xffffffffu, ok && !*abort_flag);
+      if (!ok) { if (lane == 0) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 426, blockIdx.z, t_end); } alive = false; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    }
+    // ---- write: final (one split) or partial
+    if (alive) {
+      const int r = row0 + qi, h = g * grp + qh;
+      if (!rvalid) { l = 0.0f; mx = -INFINITY; }              // padding row: an empty partial, a zero output
+      const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+      const size_t idx = (size_t)blockIdx.y * p.rows * p.H + (size_t)r * p.H + h;
+#pragma unroll 1
+      for (int c = 0; c < HD / 16; c++) {
+        uint32_t v[16];
+        if (ntl > 0) tc::tmem_ld16(tmem_o + lane_base + c * 16, v);      // the whole warp takes part
+        if (ntl <= 0 || !rvalid) {
+#pragma unroll
+          for (int j = 0; j < 16; j++) v[j] = 0u;
+        }
+        if (mrow < M) {
+          if (p.nsplit == 1) {
+            uint32_t w[8];
+#pragma unroll
+            for (int j = 0; j < 8; j++) w[j] = pack_bf16(__uint_as_float(v[2 * j]) * inv, __uint_as_float(v[2 * j + 1]) * inv);
+            uint4 *dst = (uint4 *)(p.out + ((size_t)r * p.H + h) * HD + c * 16);
+            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+          } else {
+            uint4 *dst = (uint4 *)(p.part_o + idx * HD + c * 16);
+#pragma unroll
+            for (int j = 0; j < 4; j++) dst[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          }
+        }
+      }
+      if (mrow < M && p.nsplit > 1) { p.part_ml[idx * 2] = mx; p.part_ml[idx * 2 + 1] = l; }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(UM_TMEM_COLS) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // TMA-staged variant for at most 16 query rows per (sequence, KV head): chain drafts at batch (one node x the GQA
 // group) and single-token decoding.  One 16-row tile would leave seven of eight row-parallel warps idle, so here
 // the four consumer warps share the rows and split the KEYS of every 64-key tile (16 keys each); each keeps its own
@@ -776,11 +1110,13 @@ typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, voi
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeFn g_encode = nullptr;
 bool g_encode_tried = false;
-std::map<std::tuple<const void *, int, int, int, int>, CUtensorMap> g_kv_maps;   // (pool, pages, G, page size, hd)
+std::map<std::tuple<const void *, int, int, int, int, int>, CUtensorMap> g_kv_maps;   // (pool, pages, G, page size, hd, box depth)
 
 // 3-D view of a K or V pool [num_pages][G][page_size][hd]: dim0 = 64 elements (128 bytes), dim1 = every key row of
 // the pool (pitch hd * 2 bytes), dim2 = the hd / 64 column halves (128 bytes apart).  One box = one page of one head.
-const CUtensorMap *kv_map(const void *pool, int num_pages, int G, int ps, int hd) {
+// depth: 64-column halves per box (hd / 64: one box = one page of one head; 1: one half of it).
+const CUtensorMap *kv_map(const void *pool, int num_pages, int G, int ps, int hd, int depth = 0) {
+  if (depth <= 0) depth = hd / 64;
   if (!g_encode_tried) {
     g_encode_tried = true;
     void *fn = nullptr;
@@ -791,13 +1127,13 @@ const CUtensorMap *kv_map(const void *pool, int num_pages, int G, int ps, int hd
   }
   if (!g_encode) return nullptr;
   if (num_pages > (1 << 20)) num_pages = 1 << 20;      // callers without a pool size: the page table is trusted
-  auto key = std::make_tuple(pool, num_pages, G, ps, hd);
+  auto key = std::make_tuple(pool, num_pages, G, ps, hd, depth);
   auto it = g_kv_maps.find(key);
   if (it != g_kv_maps.end()) return &it->second;
   CUtensorMap m;
   cuuint64_t dims[3] = {64, (cuuint64_t)num_pages * G * ps, (cuuint64_t)(hd / 64)};
   cuuint64_t strides[2] = {(cuuint64_t)hd * 2, 128};
-  cuuint32_t box[3] = {64, (cuuint32_t)ps, (cuuint32_t)(hd / 64)};
+  cuuint32_t box[3] = {64, (cuuint32_t)ps, (cuuint32_t)depth};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void *)pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -819,6 +1155,20 @@ int launch_tma_small(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUte
   return 0;
 }
 
+int g_attn_umma = 2;            // tcgen05 kernel for the tree passes: 0 off, 1 on, 2 on when a CTA gets at least UM_MIN_TILES key tiles
+constexpr int UM_MIN_TILES = 4; // below that the pass is launch- and latency-bound and the mma.sync kernel's shorter prologue wins
+thread_local int tl_attn_umma = -1;   // per-call override (-1: none)
+
+int launch_umma(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorMap *mv, int32_t *status, cudaStream_t s) {
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, UM_SMEM) != cudaSuccess) return -1;
+    configured = true;
+  }
+  launch_k(attn_umma_kernel, grid, dim3(192), (size_t)UM_SMEM, s, *mk, *mv, p, status);
+  return 0;
+}
+
 template <int HD>
 int launch_tma(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorMap *mv, int32_t *status, cudaStream_t s) {
   if (p.rps * (p.H / p.G) <= 16) return launch_tma_small<HD>(p, grid, mk, mv, status, s);
@@ -836,6 +1186,8 @@ int launch_tma(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorMa
 
 void attn_fast_forget_maps() { g_kv_maps.clear(); }
 void attn_fast_set_target_ctas(int n) { g_attn_target_ctas = n; }
+void attn_fast_set_umma(int mode) { g_attn_umma = mode; }
+void attn_fast_override_umma(int v) { tl_attn_umma = v; }
 
 int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail_len, bf16 *out, int rows, int H, int G,
                      int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s, bool contiguous_tail, int32_t *status,
@@ -855,9 +1207,11 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
   // TMA-staged kernel when the tail follows the context and a page is a whole number of 128-byte-swizzle boxes
   const int ps = pm.page_size;
   if (contiguous_tail && (ps == 16 || ps == 32 || ps == 64) && (hd == 64 || hd == 128)) {
-    const CUtensorMap *mk = kv_map(pool.k, pm.num_pages, G, ps, hd), *mv = kv_map(pool.v, pm.num_pages, G, ps, hd);
+    const int um_mode = tl_attn_umma >= 0 ? tl_attn_umma : g_attn_umma;
+    const bool umma = hd == 128 && rps * grp > 16 && (um_mode == 1 || (um_mode == 2 && ntiles_hint >= UM_MIN_TILES * nsplit));
+    const CUtensorMap *mk = kv_map(pool.k, pm.num_pages, G, ps, hd, umma ? 1 : 0), *mv = kv_map(pool.v, pm.num_pages, G, ps, hd, umma ? 1 : 0);
     if (mk && mv) {
-      int rc = hd == 128 ? launch_tma<128>(p, grid, mk, mv, status, s) : launch_tma<64>(p, grid, mk, mv, status, s);
+      int rc = umma ? launch_umma(p, grid, mk, mv, status, s) : hd == 128 ? launch_tma<128>(p, grid, mk, mv, status, s) : launch_tma<64>(p, grid, mk, mv, status, s);
       if (rc == 0) {
         if (nsplit > 1) {
           if (hd == 128) launch_k(attn_combine_kernel<128>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);

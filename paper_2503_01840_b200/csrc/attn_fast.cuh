@@ -20,5 +20,9 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
 void attn_fast_forget_maps();
 // CTAs an attention launch aims at when it splits the keys (process-wide; default 148 = one wave)
 void attn_fast_set_target_ctas(int n);
+// tcgen05 kernel for passes with more than 16 query rows per (sequence, KV head) and head_dim 128 (process-wide):
+// 0 never, 1 always, 2 (default) when every CTA gets several key tiles; and a per-thread override for single calls (-1: none)
+void attn_fast_set_umma(int mode);
+void attn_fast_override_umma(int v);
 
 }  // namespace spec

@@ -125,8 +125,9 @@ def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_to
 
 
 def run_trajectory(cfg, tw, dw, prompts, n_steps, tol, flags=0, max_ctx=None, check_floats=True, tap_tol=None,
-                   page_shuffle_seed=0, num_pages=None):
-    """tw/dw: CPU weight dicts.  Returns Stats; raises AssertionError on a parity violation."""
+                   page_shuffle_seed=0, num_pages=None, tune=()):
+    """tw/dw: CPU weight dicts; tune: (knob, value, value to restore) triples applied to the decoder (process-wide knobs).
+    Returns Stats; raises AssertionError on a parity violation."""
     B = len(prompts)
     reserve = n_steps * (cfg.tree_depth + 1) + 8
     if max_ctx is None:
@@ -135,6 +136,18 @@ def run_trajectory(cfg, tw, dw, prompts, n_steps, tol, flags=0, max_ctx=None, ch
         flags |= sb.FLAG_CAPTURE
     dec = sb.SpecDecoder(cfg, to_dev(tw), to_dev(dw), batch=B, max_ctx=max_ctx, flags=flags,
                          page_shuffle_seed=page_shuffle_seed, num_pages=num_pages)
+    for knob, value, _ in tune:
+        dec.tune(knob, value)
+    try:
+        return _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, check_floats, tap_tol)
+    finally:
+        for knob, _, restore in tune:
+            dec.tune(knob, restore)
+        dec.close()
+
+
+def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, check_floats, tap_tol):
+    B = len(prompts)
     st = Stats()
     first = dec.prefill([np.asarray(p) for p in prompts], reserve)
     orcs = []
@@ -173,5 +186,4 @@ def run_trajectory(cfg, tw, dw, prompts, n_steps, tol, flags=0, max_ctx=None, ch
             if a != r:
                 assert mg[i] <= decision_margin(tol), f"sequence {b}: token {i} differs from greedy decoding with margin {mg[i]}"
                 break
-    dec.close()
     return st, emitted

@@ -127,7 +127,7 @@ def test_c3_shape_two_layers_batch64_losslessness():
     assert mismatches <= 16, mismatches
 
 
-@pytest.mark.parametrize("impl", [0, 2], ids=["cp_async", "tma"])
+@pytest.mark.parametrize("impl", [0, 2, 3], ids=["cp_async", "tma", "tcgen05"])
 def test_c4_long_context_attention_sampled_vs_oracle(impl):
     """Tree-masked attention over a 16384-token paged context (many key splits + combine), 60 nodes x 32 heads;
     sampled (node, head) pairs against the oracle's per-head routine."""

@@ -152,6 +152,41 @@ def test_attention_kernel_vs_oracle(dtype, impl):
             assert np.abs(out[r, h] - ref).max() < tol, (r, h)
 
 
+@pytest.mark.parametrize("rows,H,G,ctx,tail_len", [(60, 32, 8, 517, 60), (5, 8, 2, 64, 5), (24, 8, 2, 1000, 24), (33, 16, 2, 130, 33),
+                                                   (10, 32, 8, 0, 10), (60, 32, 8, 4033, 60)])
+def test_attention_tcgen05_kernel_vs_oracle(rows, H, G, ctx, tail_len):
+    """tcgen05 tree attention (S = Q K^T and O += P V on tcgen05.mma, head_dim 128): one sequence, 128-row tiles that are
+    full, partly filled and spread over two CTAs, contexts that end inside a key tile, an empty context, key splits."""
+    hd, ps = 128, 16
+    g = torch.Generator().manual_seed(rows * 31 + ctx)
+    pps = (ctx + tail_len) // ps + 2
+    perm = torch.randperm(pps, generator=g).to(torch.int32).reshape(1, pps)
+    kp = torch.randn(pps, G, ps, hd, generator=g).to(torch.bfloat16)
+    vp = torch.randn(pps, G, ps, hd, generator=g).to(torch.bfloat16)
+    q = torch.randn(rows, H, hd, generator=g).to(torch.bfloat16)
+    seq = torch.zeros(rows, dtype=torch.int32)
+    seq[rows // 2] = -1                                       # a padding row
+    rctx = torch.full((rows,), ctx, dtype=torch.int32)
+    lo = torch.randint(0, 2 ** min(tail_len, 62), (rows,), generator=g, dtype=torch.int64) | 1
+    hi = torch.zeros(rows, dtype=torch.int64)
+    out = sb.attention(q.cuda(), kp.cuda(), vp.cuda(), perm.cuda(), ps, seq.cuda(), rctx.cuda(), rctx.cuda(), lo.cuda(),
+                       hi.cuda(), tail_len, G, ctx + 64, impl=3).float().cpu().numpy()
+    assert np.isfinite(out).all()
+    page_of = perm[0].numpy()
+    heads = sorted(set([0, H - 1, H // 2, 1]))
+    for r in range(rows):
+        if seq[r] < 0:
+            assert (out[r] == 0).all()
+            continue
+        pos = np.array(list(range(ctx)) + [ctx + t for t in range(tail_len) if (int(lo[r]) >> t) & 1], dtype=np.int64)
+        for h in heads:
+            gk = h // (H // G)
+            K = kp[torch.from_numpy(page_of[pos // ps]).long(), gk, torch.from_numpy(pos % ps)].float().numpy()
+            V = vp[torch.from_numpy(page_of[pos // ps]).long(), gk, torch.from_numpy(pos % ps)].float().numpy()
+            ref = po.attend(q[r, h].float().numpy(), K, V)
+            assert np.abs(out[r, h] - ref).max() < 2e-2, (r, h, np.abs(out[r, h] - ref).max())
+
+
 def _fast_attn_available(hd, group):
     return sb.lib().spec_attn_scratch_bytes(64, 8, hd, 1024) > 0
 
@@ -183,6 +218,18 @@ def test_small_bf16_hd128_trajectory(flags):
     prompts = [p.numpy() for p in synth.make_prompts(T2)]
     st, _ = parity.run_trajectory(T2, tw, dw, prompts, n_steps=10, tol=2e-2, tap_tol=3e-2, flags=flags)
     print("T2", st)
+
+
+@pytest.mark.parametrize("batch", [1, 3])
+def test_small_bf16_hd128_trajectory_tcgen05_attention(batch):
+    """The same model with the tree passes' attention on the tcgen05 kernel (draft levels of 5 nodes x 4 heads, verify
+    passes of 24 x 4 query rows per KV head), one sequence and a batch of three with different lengths."""
+    cfg = T2.replace(name="T2-b%d" % batch, batch=batch, prompt_lo=90, prompt_hi=170) if batch > 1 else T2
+    tw, dw = _weights(cfg)
+    prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+    st, _ = parity.run_trajectory(cfg, tw, dw, prompts, n_steps=6, tol=2e-2, tap_tol=3e-2,
+                                  tune=[(sb.SpecDecoder.TUNE_ATTN_UMMA, 1, 2)])
+    print("T2 tcgen05 attention", st)
 
 
 @pytest.mark.parametrize("cfg", [C1, T1], ids=["fp32", "bf16"])
