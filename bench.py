@@ -35,10 +35,10 @@ UNIT = "tok/s"
 
 # DRAM traffic of the GEMM kernel relative to its weight bytes, from the ncu capture summarised in
 # profiles/gemm_fused_kernel_C2_shapes_ncu_full.md: (dram__bytes_read.sum + dram__bytes_write.sum) of the four GEMMs
-# of an 8B-shaped layer = 448.5 MB for 436.2 MB of weights.  The capture ran on the 2-layer truncation (same kernels,
+# of an 8B-shaped layer = 448.4 MB for 436.2 MB of weights.  The capture ran on the 2-layer truncation (same kernels,
 # same shapes); a full step's traffic is that ratio times its weight bytes (traffic grows with the weight bytes).
 # Valid for the 8B shapes at 60 rows only; None elsewhere.
-NCU_TRAFFIC_RATIO = {"C2-8B-b1": 448.5 / 436.2}
+NCU_TRAFFIC_RATIO = {"C2-8B-b1": 448.4 / 436.2}
 
 
 def peaks():
@@ -332,7 +332,8 @@ def main():
         torch.cuda.synchronize()
         extras["plain_decode_tok_s"] = 20 * B / (time.perf_counter() - t0)
         dec.close()
-        del dec
+        del dec, tw, dw                      # the 70B-shaped weights leave no room for a second model beside them
+        torch.cuda.empty_cache()
         if cfg.batch == 1 and cfg.tree_depth >= 2:
             # designed draft/target agreement: same shapes and bytes, acceptance length near the paper's
             tw2, dw2, _, _ = synth.make_structured(cfg, 0.96, device=dev)
@@ -349,7 +350,6 @@ def main():
         extras["projection_at_paper_tau"] = {"tau": 6.23, "tok_s": 6.23 * B / (ms_per_step * 1e-3),
                                             "note": "paper's mean acceptance length for the 8B target (Table 1) / measured step time"}
         line["extras"] = extras
-        del tw, dw
         torch.cuda.empty_cache()
         line["cpu_baseline"] = cpu_baseline(cfg)
     if rank == 0:
