@@ -284,6 +284,15 @@ __device__ __forceinline__ void tma_load_3d(void *smem_dst, const CUtensorMap *m
       : "memory");
 }
 
+// Page ids of the (at most four) pages of key tile t, as the producer thread needs them: every load is issued
+// before any is used, and the caller asks for tile t + 1 before it starts on tile t, so the table look-ups
+// (dependent global loads) are never on the producer's critical path.
+__device__ __forceinline__ void tile_pages(int (&pg)[4], const int32_t *tbl, int pages_per_seq, int t, int ps) {
+  const int ppt = KT / ps, first = (t * KT) / ps;
+#pragma unroll
+  for (int j = 0; j < 4; j++) pg[j] = (j < ppt && first + j < pages_per_seq) ? tbl[first + j] : -1;
+}
+
 template <int HD, int STAGES>
 __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ CUtensorMap map_k,
                                                        const __grid_constant__ CUtensorMap map_v, AttnParams p, int32_t *status) {
@@ -344,20 +353,26 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
       const int32_t *tbl = p.pm.table + (size_t)seq * p.pm.pages_per_seq;
       const int fallback = tbl[0];                     // keys past the last page are masked; they still need a valid source
       const int ppt = KT / ps;                         // pages per tile
+      int cur[4], nxt[4] = {-1, -1, -1, -1};
+      if (t_begin < t_end) tile_pages(cur, tbl, p.pm.pages_per_seq, t_begin, ps);
       for (int t = t_begin; t < t_end; t++) {
         const int i = t - t_begin, st = i % STAGES;
+        if (t + 1 < t_end) tile_pages(nxt, tbl, p.pm.pages_per_seq, t + 1, ps);
         if (i == STAGES - 1 && !mbar_wait(q_bar, 0)) { if (status) set_status(status, ST_TIMEOUT, 400, blockIdx.z, t); break; }
         if (i >= STAGES && !mbar_wait(&empty[st], (uint32_t)(((i / STAGES) - 1) & 1))) { if (status) set_status(status, ST_TIMEOUT, 401, blockIdx.z, t); break; }
         unsigned char *kb = sm + st * 2 * TILEB, *vb = kb + TILEB;
         mbar_expect_tx(&full[st], 2 * TILEB);
-        for (int pg = 0; pg < ppt; pg++) {
-          const int pidx = (t * KT) / ps + pg;
-          int page = pidx < p.pm.pages_per_seq ? tbl[pidx] : -1;
+#pragma unroll
+        for (int pg = 0; pg < 4; pg++) {
+          if (pg >= ppt) break;
+          int page = cur[pg];
           if (page < 0 || page >= p.pm.num_pages) page = fallback;
           const int row = (page * p.G + g) * ps;
           tma_load_3d(kb + pg * ps * ROWB, &map_k, 0, row, 0, &full[st]);
           tma_load_3d(vb + pg * ps * ROWB, &map_v, 0, row, 0, &full[st]);
         }
+#pragma unroll
+        for (int pg = 0; pg < 4; pg++) cur[pg] = nxt[pg];
       }
     }
     return;
@@ -643,8 +658,11 @@ __global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant
       const int32_t *tbl = p.pm.table + (size_t)seq * p.pm.pages_per_seq;
       const int fallback = tbl[0];                     // keys past the last page are masked; they still need a valid source
       const int ppt = KT / ps;                         // pages per tile
+      int cur[4], nxt[4] = {-1, -1, -1, -1};
+      if (ntl > 0) tile_pages(cur, tbl, p.pm.pages_per_seq, t_begin, ps);
       for (int i = 0; i < ntl; i++) {
         const int t = t_begin + i, st = i % UM_STAGES;
+        if (i + 1 < ntl) tile_pages(nxt, tbl, p.pm.pages_per_seq, t + 1, ps);
         if (i >= UM_STAGES && !mbar_wait(&empty[st], (uint32_t)(((i / UM_STAGES) - 1) & 1))) {
           *abort_flag = 1;
           if (status) set_status(status, ST_TIMEOUT, 420, blockIdx.z, t);
@@ -653,9 +671,10 @@ __global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant
         if (*abort_flag) break;
         unsigned char *kb = ring + st * 2 * UM_TILE, *vb = kb + UM_TILE;
         mbar_expect_tx(&full[st], 2 * UM_TILE);
-        for (int pg = 0; pg < ppt; pg++) {
-          const int pidx = (t * KT) / ps + pg;
-          int page = pidx < p.pm.pages_per_seq ? tbl[pidx] : -1;
+#pragma unroll
+        for (int pg = 0; pg < 4; pg++) {
+          if (pg >= ppt) break;
+          int page = cur[pg];
           if (page < 0 || page >= p.pm.num_pages) page = fallback;
           const int row = (page * p.G + g) * ps;
 #pragma unroll
@@ -664,6 +683,8 @@ __global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant
             tma_load_3d(vb + h * UM_HALF + pg * ps * 128, &map_v, 0, row, h, &full[st]);
           }
         }
+#pragma unroll
+        for (int pg = 0; pg < 4; pg++) cur[pg] = nxt[pg];
       }
     }
   } else if (warp == 5) {
@@ -892,19 +913,25 @@ __global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_consta
       const int32_t *tbl = p.pm.table + (size_t)seq * p.pm.pages_per_seq;
       const int fallback = tbl[0];
       const int ppt = KT / ps;
+      int cur[4], nxt[4] = {-1, -1, -1, -1};
+      if (t_begin < t_end) tile_pages(cur, tbl, p.pm.pages_per_seq, t_begin, ps);
       for (int t = t_begin; t < t_end; t++) {
         const int i = t - t_begin, st = i % STAGES;
+        if (t + 1 < t_end) tile_pages(nxt, tbl, p.pm.pages_per_seq, t + 1, ps);
         if (i >= STAGES && !mbar_wait(&empty[st], (uint32_t)(((i / STAGES) - 1) & 1))) { if (status) set_status(status, ST_TIMEOUT, 411, blockIdx.z, t); break; }
         unsigned char *kb = sm + st * 2 * TILEB, *vb = kb + TILEB;
         mbar_expect_tx(&full[st], 2 * TILEB);
-        for (int pg = 0; pg < ppt; pg++) {
-          const int pidx = (t * KT) / ps + pg;
-          int page = pidx < p.pm.pages_per_seq ? tbl[pidx] : -1;
+#pragma unroll
+        for (int pg = 0; pg < 4; pg++) {
+          if (pg >= ppt) break;
+          int page = cur[pg];
           if (page < 0 || page >= p.pm.num_pages) page = fallback;
           const int row = (page * p.G + g) * ps;
           tma_load_3d(kb + pg * ps * ROWB, &map_k, 0, row, 0, &full[st]);
           tma_load_3d(vb + pg * ps * ROWB, &map_v, 0, row, 0, &full[st]);
         }
+#pragma unroll
+        for (int pg = 0; pg < 4; pg++) cur[pg] = nxt[pg];
       }
     }
   } else {
