@@ -536,8 +536,10 @@ constexpr int UM_TILE = KT * UM_HD * 2;            // 16 KB: the K (or the V) ti
 constexpr int UM_HALF = KT * 128;                  // 8 KB: one 64-element half of head_dim for 64 keys
 constexpr int UM_Q_BYTES = MT * UM_HD * 2;         // 32 KB
 constexpr int UM_P_BYTES = MT * KT * 2;            // 16 KB
-constexpr int UM_SMEM = UM_Q_BYTES + UM_P_BYTES + UM_STAGES * 2 * UM_TILE + 128;
-constexpr uint32_t UM_TMEM_COLS = 256;             // S (two buffers): columns 0..127, O: columns 128..255
+constexpr int UM_XCHG_BYTES = 2 * MT * 4;          // row statistics handed from softmax warpgroup 1 to warpgroup 0
+constexpr int UM_SMEM = UM_Q_BYTES + 2 * UM_P_BYTES + UM_STAGES * 2 * UM_TILE + 128 + UM_XCHG_BYTES;
+constexpr int UM_THREADS = 320;                    // two softmax warpgroups, the TMA producer warp, the MMA warp
+constexpr uint32_t UM_TMEM_COLS = 512;             // S of the two warpgroups: columns 0..127, their O: columns 128..383
 
 // MN-major operand tile with 128-byte swizzle: rows (contraction index) of 128 bytes = 64 elements of the MN
 // dimension, 8-row groups 1024 bytes apart, the next 64 MN elements lbo bytes further on.
@@ -581,20 +583,21 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
       : "memory");
 }
 
-__global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant__ CUtensorMap map_k,
+__global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_constant__ CUtensorMap map_k,
                                                         const __grid_constant__ CUtensorMap map_v, AttnParams p, int32_t *status) {
   pdl_wait();
   pdl_trigger();
   constexpr int HD = UM_HD;
   extern __shared__ __align__(1024) unsigned char sm[];
   unsigned char *sQ = sm;                                   // [2 halves][128 rows][128 B]
-  unsigned char *sP = sm + UM_Q_BYTES;                      // [128 rows][128 B]: 64 keys
-  unsigned char *ring = sP + UM_P_BYTES;                    // stage: K [2 halves][64 keys][128 B], then V likewise
+  unsigned char *sP = sm + UM_Q_BYTES;                      // one [128 rows][128 B] tile (64 keys) per softmax warpgroup
+  unsigned char *ring = sP + 2 * UM_P_BYTES;                    // stage: K [2 halves][64 keys][128 B], then V likewise
   uint64_t *full = (uint64_t *)(ring + UM_STAGES * 2 * UM_TILE);
   uint64_t *empty = full + UM_STAGES;
-  uint64_t *s_bar = empty + UM_STAGES, *p_bar = s_bar + 2, *o_bar = p_bar + 1;       // s_bar[2]: one per S buffer
-  uint32_t *tmem_slot = (uint32_t *)(o_bar + 1);
+  uint64_t *s_bar = empty + UM_STAGES, *p_bar = s_bar + 2, *o_bar = p_bar + 2;       // [2] each: one per warpgroup
+  uint32_t *tmem_slot = (uint32_t *)(o_bar + 2);
   volatile uint32_t *abort_flag = tmem_slot + 1;
+  float *xchg = (float *)(sm + UM_SMEM - UM_XCHG_BYTES);    // [2][128]: reference maximum and sum of warpgroup 1's rows
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int grp = p.H / p.G;
@@ -620,8 +623,7 @@ __global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant
     for (int i = 0; i < UM_STAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     mbar_init(&s_bar[0], 1);
     mbar_init(&s_bar[1], 1);
-    mbar_init(p_bar, 128);
-    mbar_init(o_bar, 1);
+    for (int i = 0; i < 2; i++) { mbar_init(&p_bar[i], 128); mbar_init(&o_bar[i], 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -630,17 +632,22 @@ __global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // ---- Q tile -> shared in the operand layout: row lr, 16-byte chunk c -> half c / 8, chunk (c % 8) ^ (lr % 8)
-  const int lr = threadIdx.x;                               // softmax threads: query row within the tile
+  // Two softmax warpgroups (warps 0..3 and 4..7).  Warpgroup w takes the key tiles i with i % 2 == w as an independent
+  // online-softmax stream with its own score buffer, P tile and O accumulator; thread t of either group owns query row
+  // t % 128 = tensor-memory lane t % 128.  The two streams are merged at the end like two key splits.
+  const int wg = (warp >> 2) & 1;
+  const int lr = threadIdx.x & 127;
   const int mrow = m0 + lr;
   bool rvalid = false;
   uint64_t mlo = 0, mhi = 0;
   int qi = 0, qh = 0;
-  if (warp < 4) {
+  if (warp < 8) {
     if (mrow < M) { qi = mrow / grp; qh = mrow % grp; rvalid = p.m.seq[row0 + qi] >= 0; }
     if (rvalid) { mlo = p.m.mask_lo[row0 + qi]; mhi = p.m.mask_hi[row0 + qi]; }
     const uint4 *src = (const uint4 *)(p.q + ((size_t)(row0 + qi) * p.H + g * grp + qh) * HD);
 #pragma unroll
-    for (int c = 0; c < HD / 8; c++) {
+    for (int cc = 0; cc < 8; cc++) {                        // each of the row's two threads copies one half of it
+      const int c = wg * 8 + cc;
       uint4 v = rvalid ? src[c] : make_uint4(0u, 0u, 0u, 0u);
       *(uint4 *)(sQ + (c >> 3) * (MT * 128) + lr * 128 + (((c & 7) ^ (lr & 7)) << 4)) = v;
     }
@@ -650,9 +657,9 @@ __global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * KT;
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * KT;     // S[w] at column 64 w, O[w] at column 128 + 128 w
 
-  if (warp == 4) {
+  if (warp == 8) {
     // ================================================================ producer
     if (lane == 0 && seq >= 0) {
       const int32_t *tbl = p.pm.table + (size_t)seq * p.pm.pages_per_seq;
@@ -687,13 +694,14 @@ __global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant
         for (int pg = 0; pg < 4; pg++) cur[pg] = nxt[pg];
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     // ================================================================ MMA issuer
     if (lane == 0 && ntl > 0) {
       constexpr uint32_t idesc_s = tc::umma_idesc(KT);                       // N = 64 keys, both operands K-major
       constexpr uint32_t idesc_o = tc::umma_idesc(HD) | (1u << 16);          // N = 128, B (the V tile) MN-major
       const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP);
-      // S of tile i goes to S buffer i % 2: the scores of tile i + 1 are computed while the softmax threads work on tile i
+      // S of tile i goes to the score buffer of warpgroup i % 2: while one group is in its softmax the tensor pipe
+      // works for the other
       auto issue_s = [&](int i) {
         const int st = i % UM_STAGES;
         const uint32_t k_addr = smem_u32(ring + st * 2 * UM_TILE);
@@ -716,17 +724,17 @@ __global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant
       if (ok) {
         for (int i = 0; i < ntl; i++) {
           const int st = i % UM_STAGES;
-          if (!mbar_wait(p_bar, (uint32_t)(i & 1))) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 422, blockIdx.z, t_begin + i); break; }
+          if (!mbar_wait(&p_bar[i & 1], (uint32_t)((i >> 1) & 1))) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 422, blockIdx.z, t_begin + i); break; }
           if (*abort_flag) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t v_addr = smem_u32(ring + st * 2 * UM_TILE + UM_TILE);
 #pragma unroll
           for (int kk = 0; kk < KT / tc::UMMA_K; kk++)
-            tc::umma_bf16(tmem_o, tc::umma_desc_sw128(p_addr + kk * 32), umma_desc_sw128_mn(v_addr + kk * (tc::UMMA_K * 128), UM_HALF), idesc_o,
-                          (i | kk) ? 1u : 0u);
-          tc::umma_commit(o_bar);
+            tc::umma_bf16(tmem_o + (uint32_t)((i & 1) * HD), tc::umma_desc_sw128(p_addr + (i & 1) * UM_P_BYTES + kk * 32),
+                          umma_desc_sw128_mn(v_addr + kk * (tc::UMMA_K * 128), UM_HALF), idesc_o, ((i >> 1) | kk) ? 1u : 0u);
+          tc::umma_commit(&o_bar[i & 1]);
           tc::umma_commit(&empty[st]);
-          if (i + 2 < ntl) {          // S buffer i % 2 is free: the softmax threads read it before they arrived on p_bar
+          if (i + 2 < ntl) {          // this group's score buffer is free: its threads read it before they arrived on p_bar
             const int st2 = (i + 2) % UM_STAGES;
             if (!mbar_wait(&full[st2], (uint32_t)(((i + 2) / UM_STAGES) & 1))) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 423, blockIdx.z, t_begin + i + 2); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -737,33 +745,36 @@ __global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant
     }
   } else {
     // ================================================================ softmax: thread = query row = tensor-memory lane
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t my_s = tmem_s + lane_base + (uint32_t)(wg * KT), my_o = tmem_o + lane_base + (uint32_t)(wg * HD);
+    unsigned char *my_p = sP + wg * UM_P_BYTES;
     float mx = -INFINITY, l = 0.0f;
     const float sc = rsqrtf((float)HD) * 1.4426950408889634f;    // softmax scale folded into exp2
     bool alive = true;
-    for (int i = 0; i < ntl; i++) {
-      const int t = t_begin + i;
-      bool ok = mbar_wait(&s_bar[i & 1], (uint32_t)((i >> 1) & 1));
+    int nmine = 0;                                               // tiles this warpgroup has finished
+    for (int i = wg; i < ntl; i += 2) {
+      const int t = t_begin + i, j = i >> 1;                     // j: index within this group's stream
+      bool ok = mbar_wait(&s_bar[wg], (uint32_t)(j & 1));
       ok = __all_sync(0xffffffffu, ok && !*abort_flag);
       if (!ok) { if (lane == 0) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 424, blockIdx.z, t); } alive = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       float s[KT];
-      tmem_ld64(tmem_s + lane_base + (uint32_t)((i & 1) * KT), s);
+      tmem_ld64(my_s, s);
       // Padding rows (beyond the tile's last row, or of a skipped sequence) run the loop like real rows and are
       // zeroed at the end: their Q is zero, and a row that always took the masked path would slow its whole warp.
       float tm = -INFINITY;
       if (t * KT + KT <= ctx) {
 #pragma unroll
-        for (int j = 0; j < KT; j++) tm = fmaxf(tm, s[j]);
+        for (int e = 0; e < KT; e++) tm = fmaxf(tm, s[e]);
       } else {
 #pragma unroll
-        for (int j = 0; j < KT; j++) {
-          const int key = t * KT + j, tt = key - ctx;
+        for (int e = 0; e < KT; e++) {
+          const int key = t * KT + e, tt = key - ctx;
           const bool in_ctx = key < ctx;
           const bool in_tail = !in_ctx && tt < p.tail_len;
           const bool okk = in_ctx || (in_tail && (!rvalid || ((tt < 64 ? (mlo >> tt) : (mhi >> (tt - 64))) & 1ull)));
-          s[j] = okk ? s[j] : -INFINITY;
-          tm = fmaxf(tm, s[j]);
+          s[e] = okk ? s[e] : -INFINITY;
+          tm = fmaxf(tm, s[e]);
         }
       }
       // The reference maximum of a row moves only when the tile maximum exceeds it by more than 2^8 in the exponent:
@@ -778,16 +789,16 @@ __global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant
       float rs = 0.0f;
       uint32_t pk[KT / 2];
 #pragma unroll
-      for (int j = 0; j < KT; j += 2) {
-        const float p0 = ex2_approx(fmaf(s[j], sc, -nb)), p1 = ex2_approx(fmaf(s[j + 1], sc, -nb));
+      for (int e = 0; e < KT; e += 2) {
+        const float p0 = ex2_approx(fmaf(s[e], sc, -nb)), p1 = ex2_approx(fmaf(s[e + 1], sc, -nb));
         rs += p0 + p1;
-        pk[j >> 1] = pack_bf16(p0, p1);
+        pk[e >> 1] = pack_bf16(p0, p1);
       }
       l = l * f + rs;
       mx = nm;
-      // the previous tile's P V must be complete before O is rescaled and before P is overwritten
-      if (i > 0) {
-        bool ok2 = mbar_wait(o_bar, (uint32_t)((i - 1) & 1));
+      // this group's previous P V must be complete before its O is rescaled and before its P tile is overwritten
+      if (j > 0) {
+        bool ok2 = mbar_wait(&o_bar[wg], (uint32_t)((j - 1) & 1));
         ok2 = __all_sync(0xffffffffu, ok2 && !*abort_flag);
         if (!ok2) { if (lane == 0) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 425, blockIdx.z, t); } alive = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -795,53 +806,69 @@ __global__ void __launch_bounds__(192, 1) attn_umma_kernel(const __grid_constant
 #pragma unroll 1
           for (int c = 0; c < HD / 16; c++) {
             uint32_t v[16];
-            tc::tmem_ld16(tmem_o + lane_base + c * 16, v);
+            tc::tmem_ld16(my_o + c * 16, v);
 #pragma unroll
-            for (int j = 0; j < 16; j++) v[j] = __float_as_uint(__uint_as_float(v[j]) * f);
-            tmem_st16(tmem_o + lane_base + c * 16, v);
+            for (int e = 0; e < 16; e++) v[e] = __float_as_uint(__uint_as_float(v[e]) * f);
+            tmem_st16(my_o + c * 16, v);
           }
           asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         }
       }
 #pragma unroll
       for (int c = 0; c < KT / 8; c++)
-        *(uint4 *)(sP + lr * 128 + ((c ^ (lr & 7)) << 4)) = make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
+        *(uint4 *)(my_p + lr * 128 + ((c ^ (lr & 7)) << 4)) = make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(p_bar);
+      mbar_arrive(&p_bar[wg]);
+      nmine++;
     }
-    if (alive && ntl > 0) {
-      bool ok = mbar_wait(o_bar, (uint32_t)((ntl - 1) & 1));
+    if (alive && nmine > 0) {
+      bool ok = mbar_wait(&o_bar[wg], (uint32_t)((nmine - 1) & 1));
       ok = __all_sync(0xffffffffu, ok && !*abort_flag);
       if (!ok) { if (lane == 0) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 426, blockIdx.z, t_end); } alive = false; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     }
+    // ---- merge of the two streams: group 1 hands over its rows' statistics, group 0 reads both O accumulators.
+    // Every softmax thread reaches this barrier exactly once, whether or not its group gave up.
+    if (wg == 1) { xchg[lr] = mx; xchg[128 + lr] = l; }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const bool has1 = ntl > 1;                                   // group 1 accumulated something
     // ---- write: final (one split) or partial
-    if (alive) {
+    if (wg == 0 && alive) {
+      const float m1 = has1 ? xchg[lr] : -INFINITY, l1 = has1 ? xchg[128 + lr] : 0.0f;
+      const float mm = fmaxf(mx, m1);
+      const float f0 = (mx == -INFINITY) ? 0.0f : ex2_approx((mx - mm) * sc), f1 = (m1 == -INFINITY) ? 0.0f : ex2_approx((m1 - mm) * sc);
+      l = l * f0 + l1 * f1;
+      mx = mm;
       const int r = row0 + qi, h = g * grp + qh;
       if (!rvalid) { l = 0.0f; mx = -INFINITY; }              // padding row: an empty partial, a zero output
       const float inv = l > 0.0f ? 1.0f / l : 0.0f;
       const size_t idx = (size_t)blockIdx.y * p.rows * p.H + (size_t)r * p.H + h;
 #pragma unroll 1
       for (int c = 0; c < HD / 16; c++) {
-        uint32_t v[16];
-        if (ntl > 0) tc::tmem_ld16(tmem_o + lane_base + c * 16, v);      // the whole warp takes part
-        if (ntl <= 0 || !rvalid) {
+        uint32_t v[16], w1[16];
+        if (ntl > 0) tc::tmem_ld16(tmem_o + lane_base + c * 16, v);              // the whole warp takes part
+        if (has1) tc::tmem_ld16(tmem_o + lane_base + HD + c * 16, w1);
 #pragma unroll
-          for (int j = 0; j < 16; j++) v[j] = 0u;
+        for (int e = 0; e < 16; e++) {
+          float o0 = (ntl > 0 && rvalid && f0 != 0.0f) ? __uint_as_float(v[e]) * f0 : 0.0f;
+          float o1 = (has1 && rvalid && f1 != 0.0f) ? __uint_as_float(w1[e]) * f1 : 0.0f;
+          v[e] = __float_as_uint(o0 + o1);
         }
         if (mrow < M) {
           if (p.nsplit == 1) {
             uint32_t w[8];
 #pragma unroll
-            for (int j = 0; j < 8; j++) w[j] = pack_bf16(__uint_as_float(v[2 * j]) * inv, __uint_as_float(v[2 * j + 1]) * inv);
+            for (int e = 0; e < 8; e++) w[e] = pack_bf16(__uint_as_float(v[2 * e]) * inv, __uint_as_float(v[2 * e + 1]) * inv);
             uint4 *dst = (uint4 *)(p.out + ((size_t)r * p.H + h) * HD + c * 16);
             dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
             dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
           } else {
             uint4 *dst = (uint4 *)(p.part_o + idx * HD + c * 16);
 #pragma unroll
-            for (int j = 0; j < 4; j++) dst[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            for (int e = 0; e < 4; e++) dst[e] = make_uint4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
           }
         }
       }
@@ -1192,7 +1219,7 @@ int launch_umma(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorM
     if (cudaFuncSetAttribute(attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, UM_SMEM) != cudaSuccess) return -1;
     configured = true;
   }
-  launch_k(attn_umma_kernel, grid, dim3(192), (size_t)UM_SMEM, s, *mk, *mv, p, status);
+  launch_k(attn_umma_kernel, grid, dim3(UM_THREADS), (size_t)UM_SMEM, s, *mk, *mv, p, status);
   return 0;
 }
 
