@@ -232,6 +232,30 @@ def test_small_bf16_hd128_trajectory_tcgen05_attention(batch):
     print("T2 tcgen05 attention", st)
 
 
+DEGENERATE = {
+    "depth1": dict(tree_depth=1, tree_topk=4, tree_nodes=5),                 # one draft pass, the tree is a star
+    "chain_b1": dict(tree_depth=3, tree_topk=1, tree_nodes=4),               # top-1 chain at batch 1
+    "pool_smaller_than_tree": dict(tree_depth=2, tree_topk=3, tree_nodes=40),  # N - 1 > K + (D-1) K^2: every candidate kept, padding rows
+    "two_word_masks": dict(tree_depth=8, tree_topk=10, tree_nodes=60),       # (D-1) K = 70 draft tail keys: bits beyond 64
+    "two_nodes": dict(tree_depth=2, tree_topk=2, tree_nodes=2),              # the root and one candidate
+    "short_prompt": dict(tree_depth=3, tree_topk=4, tree_nodes=16, prompt_len=2),
+}
+
+
+@pytest.mark.parametrize("base", [C1, T1], ids=["fp32", "bf16"])
+@pytest.mark.parametrize("case", sorted(DEGENERATE))
+def test_degenerate_tree_shapes_trajectory(base, case):
+    """Edge shapes of the draft tree against the oracle: depth 1, a chain, a pool smaller than the node budget, more than
+    64 tail keys (two-word ancestor masks), a two-node tree, a two-token prompt."""
+    cfg = base.replace(name=base.name + "-" + case, **DEGENERATE[case])
+    tw, dw = _weights(cfg)
+    prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+    tol = 1e-4 if cfg.dtype == "fp32" else 2e-2
+    st, _ = parity.run_trajectory(cfg, tw, dw, prompts, n_steps=5, tol=tol, tap_tol=None if cfg.dtype == "fp32" else 3e-2)
+    print(case, st)
+    assert st.steps == 5
+
+
 @pytest.mark.parametrize("cfg", [C1, T1], ids=["fp32", "bf16"])
 def test_structured_weights_accept_more_than_one(cfg):
     """Designed agreement between draft and target: counts > 1, KV compaction and multi-entry extend."""
