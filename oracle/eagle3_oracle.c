@@ -223,6 +223,67 @@ int32_t orc_accept(const int32_t *tok, const int32_t *parent, const int32_t *y, 
   return a + 1;
 }
 
+/* Stochastic acceptance at temperature T > 0 on the draft tree.  Section 2.1 gives the rule for a chain whose
+ * tokens were sampled from the draft distribution p^: accept with probability min(1, p / p^), else resample from
+ * norm(max(0, p - p^)).  The tree of Section 2.2 is not sampled: the children of a node are the draft's top-K, a
+ * deterministic set, so the proposal that puts child c forward is the point mass on tok[c] (p^ = 1 there, 0
+ * elsewhere).  The rule then reads: accept c with probability p(tok[c]); on rejection the residual
+ * norm(max(0, p - p^)) is p with tok[c] removed and renormalised, and the next child is tried against it.  When no
+ * child is left the token is drawn from the residual.  By sequential conditioning the emitted token has exactly
+ * distribution p = softmax(z / T), whatever the tree.
+ *
+ * logits [nn][V]; u [2 * n_max]: u[c] decides node c (1 <= c < nn), u[n_max + cur] draws the final token at node
+ * cur by inverse CDF over the ids in increasing order.  acc_p[c] = the probability c was tried against (-1: not
+ * tried); *bonus_lo / *bonus_hi = the CDF interval of the drawn token as fractions of the residual mass. */
+int32_t orc_accept_sampled(const int32_t *tok, const int32_t *parent, const float *logits, int32_t V, int32_t nn,
+                           int32_t n_max, float temperature, const float *u, int32_t *path, int32_t *out_ids,
+                           float *acc_p, double *bonus_lo, double *bonus_hi) {
+  double *e = (double *)xcalloc((size_t)V, sizeof(double));
+  int cur = 0, a = 0;
+  path[0] = 0;
+  for (int i = 0; i < nn; i++) acc_p[i] = -1.0f;
+  for (;;) {
+    const float *z = logits + (size_t)cur * V;
+    float zmax = z[0];
+    for (int v = 1; v < V; v++) if (z[v] > zmax) zmax = z[v];
+    double mass = 0.0;
+    for (int v = 0; v < V; v++) { e[v] = exp(((double)z[v] - (double)zmax) / (double)temperature); mass += e[v]; }
+    int nxt = -1;
+    for (int c = cur + 1; c < nn && nxt < 0; c++) {
+      if (parent[c] != cur) continue;
+      double pc = mass > 0.0 ? e[tok[c]] / mass : 0.0;
+      acc_p[c] = (float)pc;
+      if ((double)u[c] < pc) nxt = c;
+      else { mass -= e[tok[c]]; e[tok[c]] = 0.0; }
+    }
+    if (nxt >= 0) {
+      out_ids[a] = tok[nxt];
+      cur = nxt;
+      path[++a] = cur;
+      continue;
+    }
+    /* inverse CDF over the residual, ids in increasing order */
+    double total = 0.0;
+    for (int v = 0; v < V; v++) total += e[v];
+    double target = (double)u[n_max + cur] * total, cum = 0.0;
+    int pick = -1, last = 0;
+    double lo = 0.0;
+    for (int v = 0; v < V; v++) {
+      if (e[v] <= 0.0) continue;
+      last = v;
+      if (cum + e[v] > target) { pick = v; lo = cum; break; }
+      cum += e[v];
+    }
+    if (pick < 0) { pick = last; lo = total - e[last]; }
+    out_ids[a] = pick;
+    if (bonus_lo) *bonus_lo = total > 0.0 ? lo / total : 0.0;
+    if (bonus_hi) *bonus_hi = total > 0.0 ? (lo + e[pick]) / total : 1.0;
+    break;
+  }
+  free(e);
+  return a + 1;
+}
+
 /* ------------------------------------------------------------------ context */
 typedef struct {
   const void *attn_norm, *wq, *wk, *wv, *wo, *mlp_norm, *w_gate, *w_up, *w_down;
@@ -246,6 +307,8 @@ struct orc_ctx {
   int32_t y[ORC_MAX_NODES], path[ORC_MAX_NODES];
   uint64_t mask[ORC_MAX_NODES];
   float score[ORC_MAX_NODES], y_margin[ORC_MAX_NODES];
+  float acc_p[ORC_MAX_NODES];   /* sampled acceptance: probability each tried node was tested against */
+  double bonus_iv[2];           /* CDF interval of the drawn token */
   float *target_logits, *node_taps, *node_hidden;       /* [N][V], [N][3k], [N][k] */
   float *draft_logits, *draft_a;                        /* [D][K][Vd], [D][K][k] */
   int32_t *pool_tok, *pool_parent, *pool_depth;         /* [pool+1] */
@@ -528,7 +591,7 @@ int orc_force_state(orc_ctx *c, const int32_t *ids, int32_t n, int32_t P) {
 }
 
 /* ------------------------------------------------------------------ the speculative step */
-int orc_step(orc_ctx *c, int32_t *out_ids, int32_t *count) {
+static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float temperature, const float *u) {
   const orc_cfg *g = &c->cfg;
   int n = c->n, P = c->n - c->dn, K = g->tree_topk, D = g->tree_depth, N = g->tree_nodes;
   int k = g->hidden, Vd = g->draft_vocab, V = g->vocab, L = g->n_layers, kvd = g->n_kv_heads * g->head_dim;
@@ -636,8 +699,11 @@ int orc_step(orc_ctx *c, int32_t *out_ids, int32_t *count) {
     free(pos); free(nc); free(ts); free(ne); free(ex);
   }
 
-  /* 6. greedy acceptance */
-  int cnt = orc_accept(c->tok, c->parent, c->y, nn, c->path, out_ids);
+  /* 6. acceptance: greedy, or the stochastic rule when a temperature and uniforms are given */
+  int cnt = (temperature > 0.0f && u)
+                ? orc_accept_sampled(c->tok, c->parent, c->target_logits, V, nn, N, temperature, u, c->path, out_ids, c->acc_p,
+                                     &c->bonus_iv[0], &c->bonus_iv[1])
+                : orc_accept(c->tok, c->parent, c->y, nn, c->path, out_ids);
   c->count = cnt;
   if (count) *count = cnt;
 
@@ -656,6 +722,13 @@ int orc_step(orc_ctx *c, int32_t *out_ids, int32_t *count) {
   c->dn = n;
   free(lp); free(tid); free(tval); free(front);
   return 0;
+}
+
+int orc_step(orc_ctx *c, int32_t *out_ids, int32_t *count) { return step_impl(c, out_ids, count, 0.0f, NULL); }
+
+int orc_step_sampled(orc_ctx *c, float temperature, const float *u, int32_t *out_ids, int32_t *count) {
+  if (!(temperature > 0.0f) || !u) return -1;
+  return step_impl(c, out_ids, count, temperature, u);
 }
 
 const void *orc_get(const orc_ctx *c, int32_t what, int64_t *count) {
@@ -685,6 +758,8 @@ const void *orc_get(const orc_ctx *c, int32_t what, int64_t *count) {
     case ORC_RERANK_MARGIN: p = &c->rerank_margin; cn = 1; break;
     case ORC_PATH: p = c->path; cn = c->count; break;
     case ORC_G_PENDING: p = c->g_pending; cn = (int64_t)c->P_in * g->hidden; break;
+    case ORC_ACC_P: p = c->acc_p; cn = c->nn; break;
+    case ORC_BONUS_INTERVAL: p = c->bonus_iv; cn = 2; break;
     default: break;
   }
   if (count) *count = cn;

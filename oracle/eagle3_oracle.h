@@ -62,6 +62,13 @@ int orc_prefill(orc_ctx *, const int32_t *ids, int32_t n, int32_t *first_id);
  * token), 1 <= count <= D+1. */
 int orc_step(orc_ctx *, int32_t *out_ids, int32_t *count);
 
+/* The same cycle at temperature T > 0 (Section 2.1's acceptance rule on the deterministic top-K tree of Section 2.2:
+ * child c of the current node is accepted with probability p(tok[c]) under the residual of softmax(z / T), a rejected
+ * token is removed from the residual, and when no child is left the token is drawn from the residual).  The random
+ * numbers are inputs: u [2 * tree_nodes] in [0, 1); u[c] decides node c, u[tree_nodes + cur] draws the final token at
+ * node cur (inverse CDF over increasing ids).  The emitted tokens are distributed exactly as plain sampling. */
+int orc_step_sampled(orc_ctx *, float temperature, const float *u, int32_t *out_ids, int32_t *count);
+
 /* Plain greedy autoregressive decoding of the target (the paper's "vanilla" baseline): continue the
  * current state by `gen` tokens, one target forward per token.  Needs a prefilled ctx. */
 int orc_greedy(orc_ctx *, int32_t gen, int32_t *out_ids);
@@ -99,7 +106,9 @@ enum {
   ORC_FRONTIER_MARGIN,   /* float [D] score gap at the frontier cut (inf if no cut) */
   ORC_RERANK_MARGIN,     /* float [1] score gap at the rerank cut (inf if no cut)   */
   ORC_PATH,              /* int32 [count] accepted node indices, root first */
-  ORC_G_PENDING          /* float [P_in][k] fused features of the step's pending entries */
+  ORC_G_PENDING,         /* float [P_in][k] fused features of the step's pending entries */
+  ORC_ACC_P,             /* float [nodes] sampled step: probability the node was tested against, -1 if not tried */
+  ORC_BONUS_INTERVAL     /* double [2] sampled step: CDF interval (fractions of the residual mass) of the drawn token */
 };
 const void *orc_get(const orc_ctx *, int32_t what, int64_t *count);
 
@@ -128,6 +137,9 @@ int32_t orc_rerank(const float *pool_score, const int32_t *pool_parent, const in
                    int32_t root_tok, int32_t *tok, int32_t *parent, int32_t *depth, uint64_t *mask,
                    int32_t *poolidx, float *score, float *cut_margin);
 /* greedy acceptance walk; returns count, writes path (node indices, root first) and ids */
+int32_t orc_accept_sampled(const int32_t *tok, const int32_t *parent, const float *logits, int32_t V, int32_t n_nodes,
+                           int32_t n_max, float temperature, const float *u, int32_t *path, int32_t *out_ids,
+                           float *acc_p, double *bonus_lo, double *bonus_hi);
 int32_t orc_accept(const int32_t *tok, const int32_t *parent, const int32_t *y, int32_t n_nodes,
                    int32_t *path, int32_t *out_ids);
 

@@ -20,13 +20,14 @@ _lib = None
 
 (TREE_TOK, TREE_PARENT, TREE_DEPTH, TREE_MASK, TREE_POOLIDX, TREE_SCORE, Y, Y_MARGIN, TARGET_LOGITS,
  NODE_TAPS, NODE_HIDDEN, DRAFT_LOGITS, DRAFT_A, POOL_TOK, POOL_SCORE, POOL_PARENT, FRONTIER,
- TOPK_MARGIN, FRONTIER_MARGIN, RERANK_MARGIN, PATH, G_PENDING) = range(1, 23)
+ TOPK_MARGIN, FRONTIER_MARGIN, RERANK_MARGIN, PATH, G_PENDING, ACC_P, BONUS_INTERVAL) = range(1, 25)
 _DTYPES = {TREE_TOK: np.int32, TREE_PARENT: np.int32, TREE_DEPTH: np.int32, TREE_MASK: np.uint64,
            TREE_POOLIDX: np.int32, TREE_SCORE: np.float32, Y: np.int32, Y_MARGIN: np.float32,
            TARGET_LOGITS: np.float32, NODE_TAPS: np.float32, NODE_HIDDEN: np.float32,
            DRAFT_LOGITS: np.float32, DRAFT_A: np.float32, POOL_TOK: np.int32, POOL_SCORE: np.float32,
            POOL_PARENT: np.int32, FRONTIER: np.int32, TOPK_MARGIN: np.float32,
-           FRONTIER_MARGIN: np.float32, RERANK_MARGIN: np.float32, PATH: np.int32, G_PENDING: np.float32}
+           FRONTIER_MARGIN: np.float32, RERANK_MARGIN: np.float32, PATH: np.int32, G_PENDING: np.float32,
+           ACC_P: np.float32, BONUS_INTERVAL: np.float64}
 
 
 class _Cfg(C.Structure):
@@ -59,6 +60,7 @@ def lib():
         L.orc_destroy.argtypes = [C.c_void_p]
         L.orc_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
         L.orc_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.orc_step_sampled.argtypes = [C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_greedy.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
         L.orc_greedy_margins.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.orc_force_state.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32]
@@ -192,6 +194,26 @@ def accept(tok, parent, y):
     return cnt, path[:cnt].copy(), out[:cnt].copy()
 
 
+def accept_sampled(tok, parent, logits, temperature, u, n_max=None):
+    """The stochastic acceptance rule on a given tree: logits [nodes][V], u [2 * n_max].  Returns
+    (count, path, out_ids, acc_p, (bonus_lo, bonus_hi))."""
+    tok = _np(tok, np.int32); parent = _np(parent, np.int32)
+    logits = _np(logits, np.float32)
+    nn, V = logits.shape
+    n_max = nn if n_max is None else n_max
+    u = _np(u, np.float32)
+    assert u.size == 2 * n_max and tok.size == nn
+    path = np.zeros(64, np.int32); out = np.zeros(64, np.int32)
+    acc_p = np.zeros(nn, np.float32)
+    lo = C.c_double(0.0); hi = C.c_double(0.0)
+    f = lib().orc_accept_sampled
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_void_p, C.c_void_p,
+                  C.c_void_p, C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    cnt = f(_p(tok), _p(parent), _p(logits), V, nn, n_max, float(temperature), _p(u), _p(path), _p(out), _p(acc_p),
+            C.byref(lo), C.byref(hi))
+    return cnt, path[:cnt].copy(), out[:cnt].copy(), acc_p, (lo.value, hi.value)
+
+
 # ------------------------------------------------------------------ the model
 class Oracle:
     """One sequence.  `cfg` is a synth.ModelCfg-like object; weights are the synth dicts."""
@@ -263,6 +285,17 @@ class Oracle:
         rc = lib().orc_step(self.h, _p(out), _p(cnt))
         if rc:
             raise RuntimeError("orc_step failed (capacity?)")
+        return out[: int(cnt[0])].copy()
+
+    def step_sampled(self, temperature: float, u) -> np.ndarray:
+        """One step with the stochastic acceptance rule; u: 2 * tree_nodes uniforms in [0, 1) (see the header)."""
+        u = _np(u, np.float32)
+        assert u.size == 2 * self.cfg.tree_nodes
+        out = np.zeros(self.cfg.tree_depth + 1, np.int32)
+        cnt = np.zeros(1, np.int32)
+        rc = lib().orc_step_sampled(self.h, float(temperature), _p(u), _p(out), _p(cnt))
+        if rc:
+            raise RuntimeError("orc_step_sampled failed (capacity, temperature?)")
         return out[: int(cnt[0])].copy()
 
     def greedy(self, gen: int) -> np.ndarray:

@@ -412,6 +412,123 @@ def test_accept_walk_unit():
     assert (cnt, path.tolist(), out.tolist()) == (3, [0, 2, 5], [11, 30, 5])
 
 
+# ----------------------------------------------------------------------------- stochastic acceptance (T > 0)
+_ST_TOK = [7, 1, 2, 5, 3, 4, 0]
+_ST_PAR = [-1, 0, 0, 0, 1, 1, 2]     # root -> {1, 2, 3}; node 1 -> {4, 5}; node 2 -> {6}
+
+
+def _st_logits(V=8, seed=0):
+    return np.random.default_rng(seed).normal(0.0, 1.5, size=(len(_ST_TOK), V)).astype(np.float32)
+
+
+def test_sampled_acceptance_is_lossless_on_a_small_tree():
+    """Section 2.1: speculative sampling leaves the output distribution unchanged.  Over many draws of the uniforms, the
+    first emitted token is distributed as softmax(z_root / T), and, given that the first token was accepted child c, the
+    second as softmax(z_c / T), whatever the tree offers (chi-square against the exact probabilities)."""
+    V, T, n_draws = 8, 0.8, 60000
+    z = _st_logits(V)
+    p = lambda row: np.exp((row - row.max()) / T) / np.exp((row - row.max()) / T).sum()
+    rng = np.random.default_rng(1)
+    first = np.zeros(V)
+    second = {1: np.zeros(V), 2: np.zeros(V), 3: np.zeros(V)}
+    counts = np.zeros(4, int)
+    for _ in range(n_draws):
+        u = rng.random(2 * len(_ST_TOK), dtype=np.float32)
+        cnt, path, out, _, _ = po.accept_sampled(_ST_TOK, _ST_PAR, z, T, u)
+        assert 1 <= cnt <= 3 and path[0] == 0
+        counts[cnt] += 1
+        first[out[0]] += 1
+        if cnt >= 2:
+            second[int(path[1])][out[1]] += 1
+
+    def chi2_ok(obs, prob):
+        n = obs.sum()
+        exp_ = n * prob
+        stat = ((obs - exp_) ** 2 / exp_).sum()
+        return stat < 30.0          # 7 degrees of freedom: P(chi2 > 30) ~ 1e-4
+
+    assert chi2_ok(first, p(z[0].astype(np.float64)))
+    for c in (1, 2, 3):
+        assert second[c].sum() > 500
+        assert chi2_ok(second[c], p(z[c].astype(np.float64)))
+    assert counts[2] > 0 and counts[3] > 0
+
+
+def test_sampled_acceptance_probabilities_and_edges():
+    """The probability child c is tested against is p(tok c) under the residual left by its rejected elder siblings;
+    u = 0 accepts every first child, u -> 1 rejects all and draws the last id with mass left; T -> 0 is the greedy rule."""
+    V, T = 8, 1.0
+    z = _st_logits(V, seed=3)
+    pr = np.exp(z[0].astype(np.float64) - z[0].max()); pr /= pr.sum()
+    u = np.full(2 * len(_ST_TOK), 0.999999, np.float32)
+    cnt, path, out, acc_p, (lo, hi) = po.accept_sampled(_ST_TOK, _ST_PAR, z, T, u)
+    assert cnt == 1 and path.tolist() == [0]
+    # children 1, 2, 3 carry tokens 1, 2, 5: each tested against the mass its elder siblings left
+    assert abs(acc_p[1] - pr[1]) < 1e-6
+    assert abs(acc_p[2] - pr[2] / (1 - pr[1])) < 1e-6
+    assert abs(acc_p[3] - pr[5] / (1 - pr[1] - pr[2])) < 1e-6
+    assert acc_p[4] == -1 and acc_p[6] == -1
+    assert out[0] == 7 and hi == pytest.approx(1.0)            # ids 1, 2, 5 are gone; 7 is the last id with mass
+    rest = pr.copy(); rest[[1, 2, 5]] = 0
+    assert lo == pytest.approx(1 - rest[7] / rest.sum(), abs=1e-9)
+    u0 = np.zeros(2 * len(_ST_TOK), np.float32)
+    cnt, path, out, _, _ = po.accept_sampled(_ST_TOK, _ST_PAR, z, T, u0)
+    assert path.tolist() == [0, 1, 4] and out.tolist()[:2] == [1, 3] and cnt == 3
+    # inverse CDF: u picks the id whose interval contains it
+    cdf = np.cumsum(pr)
+    for ub in (0.0, 0.3, 0.77, 0.9999):
+        u = np.full(2 * len(_ST_TOK), 0.999999, np.float32)
+        one = np.array([7], np.int32)                                  # a tree of the root alone
+        u1 = np.array([0.5, ub], np.float32)
+        cnt, _, out, _, (lo, hi) = po.accept_sampled(one, [-1], z[:1], T, u1)
+        assert cnt == 1 and out[0] == int(np.searchsorted(cdf, ub * cdf[-1], side="right"))
+        assert lo <= ub < hi + 1e-12
+    # T -> 0: equals the greedy walk for any uniforms that are not exactly 0
+    for seed in range(5):
+        zz = _st_logits(V, seed=10 + seed)
+        y = zz.argmax(axis=1).astype(np.int32)
+        cg, pg, og = po.accept(_ST_TOK, _ST_PAR, y)
+        u = np.random.default_rng(seed).uniform(0.01, 0.99, 2 * len(_ST_TOK)).astype(np.float32)
+        top2 = np.sort(zz, axis=1)[:, -2:]
+        assert (top2[:, 1] - top2[:, 0]).min() > 5e-4          # far above the temperature: no near ties
+        cs, ps, os_, _, _ = po.accept_sampled(_ST_TOK, _ST_PAR, zz, 1e-5, u)
+        assert (cs, ps.tolist(), os_.tolist()) == (cg, pg.tolist(), og.tolist())
+
+
+def test_sampled_step_wiring_and_greedy_limit(c1):
+    """The sampled step applies the rule to the step's own tree and target logits, commits like the greedy step (cache ==
+    fresh prefill of the committed tokens), and at T -> 0 emits the greedy tokens."""
+    tw, dw, ids = c1
+    N = C1.tree_nodes
+    o = _mk(C1, tw, dw)
+    g = _mk(C1, tw, dw)
+    assert o.prefill(ids) == g.prefill(ids)
+    rng = np.random.default_rng(5)
+    for _ in range(4):
+        u = rng.uniform(0.01, 0.99, 2 * N).astype(np.float32)
+        assert o.step_sampled(1e-5, u).tolist() == g.step().tolist()
+    o = _mk(C1, tw, dw)
+    o.prefill(ids)
+    emitted = []
+    for _ in range(6):
+        u = rng.random(2 * N, dtype=np.float32)
+        n0 = o.n
+        out = o.step_sampled(1.0, u)
+        nn = o.get(po.TREE_TOK).size
+        logits = o.get(po.TARGET_LOGITS).reshape(nn, C1.vocab)
+        cnt, path, ref, acc_p, iv = po.accept_sampled(o.get(po.TREE_TOK), o.get(po.TREE_PARENT), logits, 1.0, u, n_max=N)
+        assert out.tolist() == ref.tolist() and o.get(po.PATH).tolist() == path.tolist()
+        assert np.array_equal(o.get(po.ACC_P), acc_p) and o.get(po.BONUS_INTERVAL).tolist() == list(iv)
+        assert o.n == n0 + len(out) and o.pending == len(out)
+        emitted += out.tolist()
+    fresh = _mk(C1, tw, dw)
+    fresh.prefill(o.ids[: o.n])
+    for pos in (0, o.n // 2, o.n - 1):
+        for layer in range(C1.n_layers):
+            k1, v1 = o.target_kv(layer, pos); k2, v2 = fresh.target_kv(layer, pos)
+            assert np.abs(k1 - k2).max() < TOL and np.abs(v1 - v2).max() < TOL
+
+
 def test_rerank_unit_ties_and_closure():
     # pool: 1,2 children of root; 3,4 children of 1; 5,6 children of 2; log-prob 0 children tie with parents
     score = np.array([0, -0.5, -1.0, -0.5, -2.0, -1.0, -1.0], np.float32)
