@@ -331,6 +331,24 @@ def main():
             dec.plain_step()
         torch.cuda.synchronize()
         extras["plain_decode_tok_s"] = 20 * B / (time.perf_counter() - t0)
+        # temperature 1: the same step ending in the stochastic acceptance kernel (host API, synchronised per step, uniforms
+        # drawn on the host); after the plain tokens the draft cache is stale, so this leg runs on a fresh prefill
+        dec.close()
+        dec = sb.SpecDecoder(cfg, tw, dw, batch=B, max_ctx=max(len(p) for p in prompts) + 40 * (D + 1) + 256,
+                             page_shuffle_seed=cfg.seed)
+        dec.prefill(prompts, 40 * (D + 1))
+        rng = np.random.default_rng(0)
+        us = rng.random((25, B, 2 * cfg.tree_nodes), dtype=np.float32)
+        for i in range(5):
+            dec.step_sampled(1.0, us[i])
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        toks_s = 0
+        for i in range(5, 25):
+            toks_s += sum(len(o) for o in dec.step_sampled(1.0, us[i]))
+        dt = time.perf_counter() - t0
+        extras["sampled_T1"] = {"ms_per_step": 1e3 * dt / 20, "accepted_tok_s": toks_s / dt,
+                                "note": "spec_step_sampled, wall clock with host synchronisation every step"}
         dec.close()
         del dec, tw, dw                      # the 70B-shaped weights leave no room for a second model beside them
         torch.cuda.empty_cache()

@@ -125,6 +125,17 @@ int spec_step(spec_ctx *ctx, int32_t *out_ids, int32_t *out_counts);
  * committed lengths (each async step may add tree_depth+1). */
 int spec_step_async(spec_ctx *ctx, int32_t *dev_ids, int32_t *dev_counts);
 
+/* One speculative step at temperature T > 0 (the non-greedy setting of Section 2.1 / Table 1): drafting and the
+ * tree-masked target forward are those of spec_step; acceptance is stochastic.  Section 2.1 states the rule for a chain
+ * whose tokens were sampled from the draft distribution; the tree of Section 2.2 is the draft's deterministic top-K, so a
+ * tried child is a point-mass proposal: child c of the current node is accepted with probability p(tok[c]) under what
+ * is left of softmax(logits / T) after its rejected elder siblings were removed, and when no child is left the token is
+ * drawn from that residual (inverse CDF over increasing ids).  The emitted tokens are distributed as plain sampling
+ * from the target.  The random numbers are inputs: u host float [batch][2 * tree_nodes] in [0, 1); u[b][c] decides
+ * node c of sequence b, u[b][tree_nodes + cur] draws the final token at node cur.  out_ids / out_counts as spec_step.
+ * 0 < temperature <= 1e4.  Synchronises. */
+int spec_step_sampled(spec_ctx *ctx, float temperature, const float *u, int32_t *out_ids, int32_t *out_counts);
+
 /* Plain greedy decoding of the target on the same kernels (the paper's "vanilla" baseline): one target
  * forward per token for every sequence, draft untouched.  out_ids host [batch]. Synchronises. */
 int spec_plain_step(spec_ctx *ctx, int32_t *out_ids);

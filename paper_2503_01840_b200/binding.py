@@ -55,7 +55,7 @@ class _Cfg(C.Structure):
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p)]
 
 
-EXPORTS = ("spec_workspace_bytes", "spec_init", "spec_prefill", "spec_step", "spec_step_async", "spec_plain_step",
+EXPORTS = ("spec_workspace_bytes", "spec_init", "spec_prefill", "spec_step", "spec_step_async", "spec_step_sampled", "spec_plain_step",
            "spec_lengths", "spec_profile_step", "spec_tune", "spec_launches_per_step", "spec_step_bytes", "spec_free", "spec_last_error",
            "spec_debug_read", "spec_debug_read_kv", "spec_gemm_scratch_bytes", "spec_gemm", "spec_gemm_fused", "spec_gemm_swiglu",
            "spec_topk_scratch_bytes", "spec_attn_scratch_bytes",
@@ -81,6 +81,7 @@ def lib():
     L.spec_step.argtypes = [vp, vp, vp]
     L.spec_step_async.argtypes = [vp, vp, vp]
     L.spec_plain_step.argtypes = [vp, vp]
+    L.spec_step_sampled.argtypes = [vp, C.c_float, vp, vp, vp]
     L.spec_lengths.argtypes = [vp, vp]
     L.spec_launches_per_step.argtypes = [vp]
     L.spec_tune.argtypes = [vp, i32, i32]
@@ -154,6 +155,7 @@ class SpecDecoder:
         self.m = model_cfg
         self.batch = batch
         self.Pmax = model_cfg.tree_depth + 1
+        self.tree_nodes = model_cfg.tree_nodes
         if num_pages is None:
             num_pages = batch * ((max_ctx + model_cfg.page_size - 1) // model_cfg.page_size)
         self._keep = [target_w, draft_w]
@@ -235,6 +237,14 @@ class SpecDecoder:
     def step_async(self, dev_ids: Optional[torch.Tensor] = None, dev_counts: Optional[torch.Tensor] = None):
         self._check(lib().spec_step_async(self.h, dev_ids.data_ptr() if dev_ids is not None else None,
                                           dev_counts.data_ptr() if dev_counts is not None else None))
+
+    def step_sampled(self, temperature: float, u) -> List[np.ndarray]:
+        """One step with the stochastic acceptance rule; u: float32 [batch][2 * tree_nodes] uniforms in [0, 1)."""
+        u = np.ascontiguousarray(u, dtype=np.float32).reshape(self.batch, 2 * self.tree_nodes)
+        ids = np.zeros((self.batch, self.Pmax), np.int32)
+        cnt = np.zeros(self.batch, np.int32)
+        self._check(lib().spec_step_sampled(self.h, float(temperature), u.ctypes.data, ids.ctypes.data, cnt.ctypes.data))
+        return [ids[b, : cnt[b]].copy() for b in range(self.batch)]
 
     def plain_step(self) -> np.ndarray:
         out = np.zeros(self.batch, np.int32)

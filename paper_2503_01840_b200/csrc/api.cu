@@ -122,7 +122,10 @@ struct spec_ctx {
   std::vector<int32_t> page_table_host;
   bool prefilled = false, draft_stale = false;
   cudaGraphExec_t graph = nullptr;
-  int launches = 0, launches_graph = 0;
+  cudaGraphExec_t graph_sampled = nullptr;   // the same step with the stochastic acceptance kernel
+  int launches = 0, launches_graph = 0, launches_graph_sampled = 0;
+  bool sampled = false;        // the step being scheduled ends with the stochastic acceptance
+  float *u_dev = nullptr;      // [B][2N] uniforms of the sampled step, then 1 / temperature
   int sched_err = 0;
   int cur_rps = 1;             // rows per sequence of the pass being scheduled
   bool prof = false;
@@ -231,6 +234,7 @@ static size_t carve(spec_ctx *c, void *base) {
   t.nn = cv.take<int32_t>(B); t.y = cv.take<int32_t>(ne);
   t.path = cv.take<int32_t>((size_t)B * c->Pmax); t.out_ids = cv.take<int32_t>((size_t)B * c->Pmax);
   t.out_cnt = cv.take<int32_t>(B); t.pend_tok = cv.take<int32_t>((size_t)B * c->Pmax);
+  c->u_dev = cv.take<float>((size_t)B * 2 * c->N + 1);
   c->status = cv.take<int32_t>(8);
   if (g.flags & SPEC_FLAG_CAPTURE) {
     c->cap_logits = cv.take<float>((size_t)c->D * c->Td * c->Vd);
@@ -348,6 +352,7 @@ extern "C" int spec_init(spec_ctx **out, const spec_target_weights *tw, const sp
 extern "C" int spec_free(spec_ctx *c) {
   if (!c) return SPEC_OK;
   if (c->graph) cudaGraphExecDestroy(c->graph);
+  if (c->graph_sampled) cudaGraphExecDestroy(c->graph_sampled);
   if (c->fg) fast_gemm_destroy(c->fg);
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   delete c;
@@ -511,7 +516,7 @@ template <typename T> struct Sched {
       a.w[0] = (const bf16 *)c->lm_head; a.O[0] = c->V; a.nw = 1;
       with_norm_scale(a);
       a.best_val = c->best_val; a.best_idx = c->best_idx; a.best_ld = c->Ralloc;
-      if (c->cap_logits) { a.out_f32 = c->logits; a.ldo = c->V; }
+      if (c->cap_logits || c->sampled) { a.out_f32 = c->logits; a.ldo = c->V; }
       fgemm(EPI_ARGMAX, a);
       mark(SPEC_PROF_ARGMAX); launch_argmax_merge(c->best_val, c->best_idx, c->vtiles, c->Ralloc, rows, c->tb.y, s); tick();
     }
@@ -690,7 +695,10 @@ template <typename T> struct Sched {
     }
     c->cur_rps = rps;
     target_forward(rows, rps, true);
-    mark(SPEC_PROF_TREE); launch_accept(c->st, c->tb, c->B, rps, s); tick();
+    mark(SPEC_PROF_TREE);
+    if (c->sampled && !plain) launch_accept_sampled(c->st, c->tb, c->logits, c->V, c->u_dev, c->B, rps, s);
+    else launch_accept(c->st, c->tb, c->B, rps, s);
+    tick();
     PageMap pm{c->page_table, c->pps, c->cfg.page_size, c->cfg.num_pages};
     mark(SPEC_PROF_COMMIT); launch_commit<T>(c->st, c->tb, c->pools_dev, pm, (const T *)c->node_taps, (T *)c->pend_taps, c->B, c->L, c->G, c->hd,
                      c->k, rps, s);
@@ -814,6 +822,7 @@ template <typename T> static int do_prefill(spec_ctx *c, const int32_t *ids, con
   c->prefilled = true;
   c->draft_stale = false;
   if (c->graph) { cudaGraphExecDestroy(c->graph); c->graph = nullptr; }
+  if (c->graph_sampled) { cudaGraphExecDestroy(c->graph_sampled); c->graph_sampled = nullptr; }
   return read_status(c);
 }
 
@@ -833,20 +842,22 @@ static int launch_step(spec_ctx *c, bool plain) {
     if (c->sched_err) return fail(c, SPEC_ERR_CUDA, "a GEMM launch was rejected (code %d)", c->sched_err);
     return SPEC_OK;
   }
-  if (!c->graph) {
+  cudaGraphExec_t &graph = c->sampled ? c->graph_sampled : c->graph;
+  int &launches_graph = c->sampled ? c->launches_graph_sampled : c->launches_graph;
+  if (!graph) {
     cudaGraph_t gr;
     CUDA_TRY(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
     if (c->cfg.dtype == SPEC_F32) Sched<float>(c).step(false); else Sched<bf16>(c).step(false);
     cudaError_t e = cudaStreamEndCapture(c->stream, &gr);
     if (e != cudaSuccess) return fail(c, SPEC_ERR_CUDA, "graph capture: %s", cudaGetErrorString(e));
     if (c->sched_err) { cudaGraphDestroy(gr); return fail(c, SPEC_ERR_CUDA, "a GEMM launch was rejected (code %d)", c->sched_err); }
-    e = cudaGraphInstantiate(&c->graph, gr, 0);
+    e = cudaGraphInstantiate(&graph, gr, 0);
     cudaGraphDestroy(gr);
-    if (e != cudaSuccess) { c->graph = nullptr; return fail(c, SPEC_ERR_CUDA, "graph instantiate: %s", cudaGetErrorString(e)); }
-    c->launches_graph = c->launches;
+    if (e != cudaSuccess) { graph = nullptr; return fail(c, SPEC_ERR_CUDA, "graph instantiate: %s", cudaGetErrorString(e)); }
+    launches_graph = c->launches;
   }
-  c->launches = c->launches_graph;
-  CUDA_TRY(c, cudaGraphLaunch(c->graph, c->stream));
+  c->launches = launches_graph;
+  CUDA_TRY(c, cudaGraphLaunch(graph, c->stream));
   return SPEC_OK;
 }
 
@@ -886,6 +897,28 @@ extern "C" int spec_step(spec_ctx *c, int32_t *out_ids, int32_t *out_counts) {
   CUDA_TRY(c, cudaMemcpyAsync(out_ids, c->tb.out_ids, (size_t)c->B * c->Pmax * 4, cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaMemcpyAsync(out_counts, c->tb.out_cnt, (size_t)c->B * 4, cudaMemcpyDeviceToHost, c->stream));
   if (int rc = read_status(c)) return rc;
+  return sync_lengths(c);
+}
+
+extern "C" int spec_step_sampled(spec_ctx *c, float temperature, const float *u, int32_t *out_ids, int32_t *out_counts) {
+  if (!c) return SPEC_ERR_NULL;
+  if (!u || !out_ids || !out_counts) return fail(c, SPEC_ERR_NULL, "spec_step_sampled: NULL argument");
+  if (!(temperature > 0.0f) || !(temperature <= 1e4f)) return fail(c, SPEC_ERR_INVALID_CFG, "spec_step_sampled: the temperature must be in (0, 1e4]");
+  if (c->draft_stale) return fail(c, SPEC_ERR_STATE, "spec_step_sampled after spec_plain_step: the draft cache is stale, prefill again");
+  if (int rc = check_capacity(c, c->Pmax, "spec_step_sampled")) return rc;
+  const size_t nu = (size_t)c->B * 2 * c->N;
+  const float inv_t = 1.0f / temperature;
+  CUDA_TRY(c, cudaMemcpyAsync(c->u_dev, u, nu * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(c->u_dev + nu, &inv_t, sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));           // inv_t lives on this stack frame
+  c->sampled = true;
+  int rc = launch_step(c, false);
+  c->sampled = false;
+  if (rc) return rc;
+  for (int b = 0; b < c->B; b++) c->n_upper[b] += c->Pmax;
+  CUDA_TRY(c, cudaMemcpyAsync(out_ids, c->tb.out_ids, (size_t)c->B * c->Pmax * 4, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaMemcpyAsync(out_counts, c->tb.out_cnt, (size_t)c->B * 4, cudaMemcpyDeviceToHost, c->stream));
+  if (int rc2 = read_status(c)) return rc2;
   return sync_lengths(c);
 }
 
@@ -953,6 +986,7 @@ extern "C" int spec_tune(spec_ctx *c, int32_t what, int32_t value) {
     return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: unknown knob %d", what);
   }
   if (c->graph) { cudaStreamSynchronize(c->stream); cudaGraphExecDestroy(c->graph); c->graph = nullptr; }   // re-capture with the new plan
+  if (c->graph_sampled) { cudaStreamSynchronize(c->stream); cudaGraphExecDestroy(c->graph_sampled); c->graph_sampled = nullptr; }
   return SPEC_OK;
 }
 

@@ -40,6 +40,10 @@ void launch_expand(SeqState st, TreeBufs tb, RowMeta m, const int32_t *d2t, int 
 void launch_rerank(SeqState st, TreeBufs tb, RowMeta m, int B, cudaStream_t s);
 void launch_plain_tree(SeqState st, TreeBufs tb, RowMeta m, int B, cudaStream_t s);
 void launch_accept(SeqState st, TreeBufs tb, int B, int rows_per_seq, cudaStream_t s);
+// Stochastic acceptance: logits fp32 [B * rows_per_seq][V] of the verify pass; u = B x 2N uniforms followed by one float,
+// 1 / temperature (all device memory).
+void launch_accept_sampled(SeqState st, TreeBufs tb, const float *logits, int V, const float *u, int B, int rows_per_seq,
+                           cudaStream_t s);
 template <typename T>
 void launch_commit(SeqState st, TreeBufs tb, const KvPool *pools /*device array [L]*/, PageMap pm, const T *node_taps,
                    T *pend_taps, int B, int L, int G, int hd, int k, int rows_per_seq, cudaStream_t s);

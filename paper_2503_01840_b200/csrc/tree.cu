@@ -551,6 +551,155 @@ void launch_accept(SeqState st, TreeBufs tb, int B, int rows_per_seq, cudaStream
   launch_k(accept_kernel, dim3(B), dim3(32), 0, s, st, tb, rows_per_seq);
 }
 
+// ---------------------------------------------------------------- stochastic acceptance (temperature > 0)
+// Section 2.1's rule on the deterministic top-K tree: child c of the current node is accepted with probability
+// p(tok[c]) under what is left of softmax(z / T) after its rejected elder siblings were removed; when no child is
+// left the token is drawn from the residual by inverse CDF over increasing ids.  The uniforms are inputs:
+// u[b][c] decides node c, u[b][N + cur] draws the final token at node cur.  One CTA per sequence; every reduction
+// has a fixed order, so a step is reproducible on this kernel.
+constexpr int ACC_THREADS = 1024;
+constexpr int ACC_MAX_REJ = 64;
+
+__device__ __forceinline__ float block_reduce_max(float v, float *sh) {
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = sh[0];
+  for (int w = 1; w < ACC_THREADS / 32; w++) r = fmaxf(r, sh[w]);
+  __syncthreads();
+  return r;
+}
+__device__ __forceinline__ float block_reduce_sum(float v, float *sh) {
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = 0.0f;
+  for (int w = 0; w < ACC_THREADS / 32; w++) r += sh[w];      // every thread adds the 32 warp sums in the same order
+  __syncthreads();
+  return r;
+}
+
+__global__ void __launch_bounds__(ACC_THREADS) accept_sampled_kernel(SeqState st, TreeBufs tb, const float *__restrict__ logits,
+                                                                     int V, const float *__restrict__ u, int rows_per_seq) {
+  pdl_wait();
+  pdl_trigger();
+  __shared__ float red[ACC_THREADS / 32];
+  __shared__ float part[ACC_THREADS];
+  __shared__ int32_t rej[ACC_MAX_REJ];
+  __shared__ int s_next, s_nrej, s_pick, s_owner;
+  __shared__ float s_target;
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int Pmax = tb.Pmax, N = tb.N;
+  const int nn = tb.nn[b];
+  if (!st.active[b] || nn < 1) {
+    if (tid == 0) tb.out_cnt[b] = 0;
+    return;
+  }
+  const int32_t *tok = tb.tok + (size_t)b * rows_per_seq, *par = tb.parent + (size_t)b * rows_per_seq;
+  const float *ub = u + (size_t)b * 2 * N;
+  const float inv_T = u[(size_t)gridDim.x * 2 * N];          // 1 / temperature follows the uniforms
+  int cur = 0, a = 0;
+  if (tid == 0) tb.path[b * Pmax] = 0;
+  for (;;) {
+    const float *z = logits + ((size_t)b * rows_per_seq + cur) * V;
+    float m = -INFINITY;
+    for (int v = tid; v < V; v += ACC_THREADS) m = fmaxf(m, z[v]);
+    const float zmax = block_reduce_max(m, red);
+    float sum = 0.0f;
+    for (int v = tid; v < V; v += ACC_THREADS) sum += expf((z[v] - zmax) * inv_T);
+    float mass = block_reduce_sum(sum, red);
+    // ---- the children of cur in node order, tried by one thread
+    if (tid == 0) {
+      int nxt = -1, nrej = 0;
+      if (a + 1 < Pmax) {
+        for (int c = cur + 1; c < nn && nxt < 0; c++) {
+          if (par[c] != cur) continue;
+          const float e = expf((z[tok[c]] - zmax) * inv_T);
+          const float pc = mass > 0.0f ? e / mass : 0.0f;
+          if (ub[c] < pc) nxt = c;
+          else { mass -= e; if (nrej < ACC_MAX_REJ) rej[nrej++] = tok[c]; }
+        }
+      }
+      s_next = nxt; s_nrej = nrej;
+    }
+    __syncthreads();
+    const int nxt = s_next, nrej = s_nrej;
+    if (nxt >= 0) {
+      if (tid == 0) {
+        tb.out_ids[b * Pmax + a] = tok[nxt];
+        tb.pend_tok[b * Pmax + a] = tok[nxt];
+        tb.path[b * Pmax + a + 1] = nxt;
+      }
+      cur = nxt;
+      a++;
+      __syncthreads();
+      continue;
+    }
+    // ---- the final token: inverse CDF over the residual.  Thread t owns the ids [t * C, (t + 1) * C).
+    const int C = (V + ACC_THREADS - 1) / ACC_THREADS;
+    const int v0 = tid * C, v1 = (v0 + C < V) ? v0 + C : V;
+    float loc = 0.0f;
+    for (int v = v0; v < v1; v++) {
+      bool gone = false;
+      for (int r = 0; r < nrej; r++) gone |= (rej[r] == v);
+      if (!gone) loc += expf((z[v] - zmax) * inv_T);
+    }
+    part[tid] = loc;
+    __syncthreads();
+    if (tid == 0) {
+      float total = 0.0f;
+      for (int t = 0; t < ACC_THREADS; t++) total += part[t];
+      const float target = ub[N + cur] * total;
+      float cum = 0.0f;
+      int owner = -1;
+      for (int t = 0; t < ACC_THREADS; t++) {
+        if (part[t] > 0.0f && cum + part[t] > target) { owner = t; break; }
+        cum += part[t];
+      }
+      if (owner < 0) {                                   // rounding at the upper end: the last thread with mass
+        cum = total;
+        for (int t = ACC_THREADS - 1; t >= 0; t--)
+          if (part[t] > 0.0f) { owner = t; cum = total - part[t]; break; }
+      }
+      s_owner = owner; s_target = target - cum; s_pick = 0;
+    }
+    __syncthreads();
+    if (tid == s_owner) {
+      const float target = s_target;
+      float cum = 0.0f;
+      int pick = -1, last = v0;
+      for (int v = v0; v < v1; v++) {
+        bool gone = false;
+        for (int r = 0; r < nrej; r++) gone |= (rej[r] == v);
+        if (gone) continue;
+        const float e = expf((z[v] - zmax) * inv_T);
+        if (e <= 0.0f) continue;
+        last = v;
+        if (cum + e > target) { pick = v; break; }
+        cum += e;
+      }
+      s_pick = pick >= 0 ? pick : last;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      const int bonus = s_pick;
+      tb.out_ids[b * Pmax + a] = bonus;
+      tb.pend_tok[b * Pmax + a] = bonus;
+      for (int j = a + 1; j < Pmax; j++) tb.out_ids[b * Pmax + j] = -1;
+      tb.out_cnt[b] = a + 1;
+      const int n = st.n[b];
+      st.n_prev[b] = n;
+      st.n[b] = n + a + 1;
+      st.P[b] = a + 1;
+      st.root[b] = bonus;
+    }
+    break;
+  }
+}
+void launch_accept_sampled(SeqState st, TreeBufs tb, const float *logits, int V, const float *u, int B, int rows_per_seq, cudaStream_t s) {
+  launch_k(accept_sampled_kernel, dim3(B), dim3(ACC_THREADS), 0, s, st, tb, logits, V, u, rows_per_seq);
+}
+
 // ---------------------------------------------------------------- commit: KV compaction + tap gather
 // Accepted node path[j] (K/V at cache position n+path[j]) moves to position n+j in every layer; its
 // taps become pending entry j.  path[j] >= j and is increasing, and a thread copies the same element

@@ -49,9 +49,9 @@ class Stats:
                 f"tokens={self.tokens} | {errs}")
 
 
-def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_tol=None):
+def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_tol=None, sampled=None):
     """`orc` has just executed the same step from the same state.  Returns True if outputs were
-    required to be (and were) identical."""
+    required to be (and were) identical.  sampled = (temperature, u) for a step with stochastic acceptance."""
     K, D, N, Vd, k, V = cfg.tree_topk, cfg.tree_depth, cfg.tree_nodes, cfg.draft_vocab, cfg.hidden, cfg.vocab
     tap_tol = tol if tap_tol is None else tap_tol
     MARGIN = decision_margin(tol)
@@ -116,6 +116,8 @@ def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_to
         gy, oy, ym = dec.debug(sb.DBG_Y, seq), orc.get(po.Y), orc.get(po.Y_MARGIN)
         big = ym > MARGIN
         assert np.array_equal(gy[big], oy[big]), "argmax differs at a node with margin"
+        if sampled is not None:
+            return check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, *sampled)
         o_path = orc.get(po.PATH)
         if big[o_path].all():
             g_path = dec.debug(sb.DBG_PATH, seq)
@@ -124,9 +126,61 @@ def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_to
     return exact_out
 
 
+def check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, temperature, u):
+    """Stochastic acceptance on the same tree: every decision of the CUDA path (accept / reject of each tried child, the
+    drawn token) must be one the oracle's probabilities allow within the slack that the logit tolerance implies (a logit
+    error of tol moves a probability ratio by exp(2 tol / T) - 1), and equal to the oracle's decision wherever the
+    oracle's own margin exceeds that slack.  Returns True when the outputs had to be (and were) identical."""
+    V, N = cfg.vocab, cfg.tree_nodes
+    tok, par = orc.get(po.TREE_TOK), orc.get(po.TREE_PARENT)
+    nn = tok.size
+    z = orc.get(po.TARGET_LOGITS).reshape(nn, V).astype(np.float64)
+    g_path = dec.debug(sb.DBG_PATH, seq)
+    assert len(gpu_out) == len(g_path) and g_path[0] == 0
+    delta = float(np.expm1(2.0 * tol / temperature)) + 1e-5
+    cur, forced = 0, True
+    for j in range(len(g_path)):
+        e = np.exp((z[cur] - z[cur].max()) / temperature)
+        mass = e.sum()
+        nxt = int(g_path[j + 1]) if j + 1 < len(g_path) else -1
+        accepted = False
+        for c in range(cur + 1, nn):
+            if par[c] != cur:
+                continue
+            pc = e[tok[c]] / mass
+            uc = float(u[c])
+            if abs(uc - pc) <= delta * pc + 1e-7:
+                forced = False
+            if c == nxt:
+                assert uc < pc * (1 + delta) + 1e-7, f"node {c} accepted with u={uc} against p={pc}"
+                assert gpu_out[j] == tok[c]
+                accepted = True
+                break
+            assert uc >= pc * (1 - delta) - 1e-7, f"node {c} rejected with u={uc} against p={pc}"
+            mass -= e[tok[c]]
+            e[tok[c]] = 0.0
+        if accepted:
+            cur = nxt
+            continue
+        assert nxt == -1, "the path continues through a node that is not a child of the current one"
+        bonus = int(gpu_out[j])
+        assert 0 <= bonus < V and e[bonus] > 0.0, "the drawn token has no mass in the residual"
+        cdf = np.cumsum(e) / e.sum()
+        lo, hi = (cdf[bonus - 1] if bonus else 0.0), cdf[bonus]
+        ub = float(u[N + cur])
+        assert lo - delta - 1e-6 <= ub <= hi + delta + 1e-6, f"token {bonus} drawn with u={ub} outside [{lo}, {hi})"
+        if min(ub - lo, hi - ub) <= delta + 1e-6:
+            forced = False
+    if forced:
+        o_path = orc.get(po.PATH)
+        assert np.array_equal(g_path, o_path), (g_path, o_path)
+    return forced
+
+
 def run_trajectory(cfg, tw, dw, prompts, n_steps, tol, flags=0, max_ctx=None, check_floats=True, tap_tol=None,
-                   page_shuffle_seed=0, num_pages=None, tune=()):
+                   page_shuffle_seed=0, num_pages=None, tune=(), sampling=None):
     """tw/dw: CPU weight dicts; tune: (knob, value, value to restore) triples applied to the decoder (process-wide knobs).
+    sampling = (temperature, seed): every step uses the stochastic acceptance rule with uniforms drawn from that seed.
     Returns Stats; raises AssertionError on a parity violation."""
     B = len(prompts)
     reserve = n_steps * (cfg.tree_depth + 1) + 8
@@ -139,15 +193,16 @@ def run_trajectory(cfg, tw, dw, prompts, n_steps, tol, flags=0, max_ctx=None, ch
     for knob, value, _ in tune:
         dec.tune(knob, value)
     try:
-        return _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, check_floats, tap_tol)
+        return _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, check_floats, tap_tol, sampling)
     finally:
         for knob, _, restore in tune:
             dec.tune(knob, restore)
         dec.close()
 
 
-def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, check_floats, tap_tol):
+def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, check_floats, tap_tol, sampling=None):
     B = len(prompts)
+    rng = np.random.default_rng(sampling[1]) if sampling else None
     st = Stats()
     first = dec.prefill([np.asarray(p) for p in prompts], reserve)
     orcs = []
@@ -158,14 +213,16 @@ def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, c
         orcs.append(o)
     emitted = [[] for _ in range(B)]
     for step in range(n_steps):
-        outs = dec.step()
+        u = rng.random((B, 2 * cfg.tree_nodes), dtype=np.float32) if sampling else None
+        outs = dec.step_sampled(sampling[0], u) if sampling else dec.step()
         for b in range(B):
             o = orcs[b]
             ids_before, n_before = o.ids, o.n
-            o_out = o.step()
+            o_out = o.step_sampled(sampling[0], u[b]) if sampling else o.step()
             g_out = outs[b]
             assert 1 <= len(g_out) <= cfg.tree_depth + 1
-            exact = compare_step(dec, o, b, cfg, tol, st, g_out, check_floats, tap_tol)
+            exact = compare_step(dec, o, b, cfg, tol, st, g_out, check_floats, tap_tol,
+                                 sampled=(sampling[0], u[b]) if sampling else None)
             if exact:
                 assert np.array_equal(g_out, o_out), (g_out, o_out)
                 st.exact_out += 1
@@ -178,7 +235,7 @@ def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, c
         st.steps += 1
         assert np.array_equal(dec.lengths(), [o.n for o in orcs])
     # losslessness against plain greedy decoding of the oracle, up to the first low-margin token
-    for b in range(B):
+    for b in range(B if not sampling else 0):
         g = po.Oracle(cfg, tw, dw, max_ctx)
         g.prefill(np.asarray(prompts[b]))
         ref, mg = g.greedy_margins(len(emitted[b]))

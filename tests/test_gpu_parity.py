@@ -256,6 +256,55 @@ def test_degenerate_tree_shapes_trajectory(base, case):
     assert st.steps == 5
 
 
+@pytest.mark.parametrize("temperature", [1.0, 0.3])
+@pytest.mark.parametrize("base", [C1, T1, T2], ids=["fp32", "bf16", "bf16_hd128"])
+def test_sampled_acceptance_trajectory(base, temperature):
+    """Temperature > 0: the stochastic acceptance kernel against the oracle's rule with the same uniforms, step by step
+    (every accept / reject and the drawn token allowed by the oracle's probabilities within the logit tolerance, identical
+    where the oracle's margin exceeds it), on the fp32 model, the tiny bf16 model and a batch of the head_dim-128 model."""
+    cfg = base if base is not T2 else T2.replace(name="T2-b2-sampled", batch=2, prompt_lo=60, prompt_hi=120)
+    tw, dw = _weights(cfg)
+    prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+    tol = 1e-4 if cfg.dtype == "fp32" else 2e-2
+    st, emitted = parity.run_trajectory(cfg, tw, dw, prompts, n_steps=10, tol=tol, tap_tol=None if cfg.dtype == "fp32" else 3e-2,
+                                        sampling=(temperature, 17))
+    print("sampled", cfg.name, temperature, st)
+    assert st.steps == 10 and st.same_tree >= 3
+    if cfg.dtype == "fp32":
+        assert st.resyncs <= 1          # float errors of ~4e-6: the outputs coincide with the oracle's
+
+
+@pytest.mark.parametrize("cfg", [C1, T1], ids=["fp32", "bf16"])
+def test_sampled_acceptance_with_structured_weights_accepts_drafts(cfg):
+    """Designed draft/target agreement at temperature 1: accepted paths longer than one node, multi-entry commit and
+    extend under the stochastic rule."""
+    tw, dw, pi, pi2 = synth.make_structured(cfg, 0.85, residual_scale=0.05)
+    prompt = synth.structured_prompt(cfg, dw["d2t"], 48).numpy()
+    tol = 1e-4 if cfg.dtype == "fp32" else 2e-2
+    st, emitted = parity.run_trajectory(cfg, tw, dw, [prompt], n_steps=12, tol=tol, tap_tol=tol * 1.5, sampling=(1.0, 5))
+    print("structured sampled", cfg.name, st)
+    assert st.tokens > 12 + 6, "the structured workload must accept draft tokens"
+
+
+def test_sampled_step_low_temperature_is_greedy():
+    """T -> 0: the sampled step emits what the greedy step emits (same kernels, same state)."""
+    tw, dw = _weights(T1)
+    prompts = [p.numpy() for p in synth.make_prompts(T1)]
+    outs = []
+    for sampled in (False, True):
+        dec = sb.SpecDecoder(T1, parity.to_dev(tw), parity.to_dev(dw), batch=1, max_ctx=len(prompts[0]) + 200)
+        dec.prefill(prompts, 100)
+        rng = np.random.default_rng(3)
+        acc = []
+        for _ in range(8):
+            u = rng.uniform(0.01, 0.99, (1, 2 * T1.tree_nodes)).astype(np.float32)
+            acc += (dec.step_sampled(1e-4, u) if sampled else dec.step())[0].tolist()
+        outs.append(acc)
+        dec.close()
+    n = min(len(outs[0]), len(outs[1]))
+    assert outs[0][:n] == outs[1][:n]
+
+
 @pytest.mark.parametrize("cfg", [C1, T1], ids=["fp32", "bf16"])
 def test_structured_weights_accept_more_than_one(cfg):
     """Designed agreement between draft and target: counts > 1, KV compaction and multi-entry extend."""

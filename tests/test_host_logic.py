@@ -76,4 +76,5 @@ def test_single_kernel_entry_points_reject_null():
     assert L.spec_logsoftmax_topk(None, 1, 1, 1, None, None, None, None) == -2
     assert L.spec_gemm_fused(None, None, None, 1, 1, 8, 1, 0, 0, None) == -2
     assert L.spec_gemm_swiglu(None, None, None, None, 1, 128, 8, None) == -2
+    assert L.spec_step_sampled(None, 1.0, None, None, None) == -2
     assert L.spec_topk_scratch_bytes(10, 32000, 10) > 0
