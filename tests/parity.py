@@ -106,6 +106,9 @@ def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_to
             p = int(g_par[i])
             assert 0 <= p < i and g_dep[i] == g_dep[p] + 1 and int(g_mask[i]) == (int(g_mask[p]) | (1 << i))
     exact_out = False
+    if sampled is not None and not same_tree and check_floats:
+        check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, *sampled, own_inputs=True)
+        st.max_err["sampled_own_inputs_checks"] = st.max_err.get("sampled_own_inputs_checks", 0.0) + 1
     if same_tree:
         nn = ints["tok"][0].size
         assert st.err("tree_score", dec.debug(sb.DBG_TREE_SCORE, seq), orc.get(po.TREE_SCORE)) <= tol
@@ -126,15 +129,23 @@ def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_to
     return exact_out
 
 
-def check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, temperature, u):
+def check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, temperature, u, own_inputs=False):
     """Stochastic acceptance on the same tree: every decision of the CUDA path (accept / reject of each tried child, the
     drawn token) must be one the oracle's probabilities allow within the slack that the logit tolerance implies (a logit
     error of tol moves a probability ratio by exp(2 tol / T) - 1), and equal to the oracle's decision wherever the
     oracle's own margin exceeds that slack.  Returns True when the outputs had to be (and were) identical."""
     V, N = cfg.vocab, cfg.tree_nodes
-    tok, par = orc.get(po.TREE_TOK), orc.get(po.TREE_PARENT)
-    nn = tok.size
-    z = orc.get(po.TARGET_LOGITS).reshape(nn, V).astype(np.float64)
+    if own_inputs:
+        # the trees differ (a low-margin draft decision): the acceptance kernel is still checked, as a function of its
+        # own inputs (the CUDA path's tree and verify logits), with the slack of the summation order only
+        tok, par = dec.debug(sb.DBG_TREE_TOK, seq), dec.debug(sb.DBG_TREE_PARENT, seq)
+        nn = tok.size
+        z = dec.debug(sb.DBG_TARGET_LOGITS, seq).reshape(nn, V).astype(np.float64)
+        tol = 1e-5
+    else:
+        tok, par = orc.get(po.TREE_TOK), orc.get(po.TREE_PARENT)
+        nn = tok.size
+        z = orc.get(po.TARGET_LOGITS).reshape(nn, V).astype(np.float64)
     g_path = dec.debug(sb.DBG_PATH, seq)
     assert len(gpu_out) == len(g_path) and g_path[0] == 0
     delta = float(np.expm1(2.0 * tol / temperature)) + 1e-5
@@ -171,6 +182,11 @@ def check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, temperature, u):
         assert lo - delta - 1e-6 <= ub <= hi + delta + 1e-6, f"token {bonus} drawn with u={ub} outside [{lo}, {hi})"
         if min(ub - lo, hi - ub) <= delta + 1e-6:
             forced = False
+    if own_inputs:
+        if forced:      # the oracle's rule on the same inputs must give the same walk and token
+            cnt, o_path, o_out, _, _ = po.accept_sampled(tok, par, z.astype(np.float32), temperature, u, n_max=N)
+            assert np.array_equal(g_path, o_path) and np.array_equal(np.asarray(gpu_out), o_out), (g_path, o_path, gpu_out, o_out)
+        return False
     if forced:
         o_path = orc.get(po.PATH)
         assert np.array_equal(g_path, o_path), (g_path, o_path)

@@ -421,6 +421,18 @@ def test_c2_two_layer_truncation_first_steps(flags):
     print("C2-L2", st)
 
 
+def test_c2_two_layer_truncation_sampled_steps():
+    """The same 8B-shaped truncation at temperature 0.7: softmax, residual and inverse CDF over the 128256-entry
+    vocabulary of 60 verify nodes against the oracle's rule."""
+    cfg = synth.C2.truncated(2, prompt_len=48)
+    tw = synth.make_target_weights(cfg, device="cuda")
+    dw = synth.make_draft_weights(cfg, device="cuda")
+    prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+    st, _ = parity.run_trajectory(cfg, parity.to_cpu(tw), parity.to_cpu(dw), prompts, n_steps=2, tol=2e-2, tap_tol=3e-2,
+                                  sampling=(0.7, 23))
+    print("C2-L2 sampled", st)
+
+
 @pytest.mark.parametrize("H,G,hd,rps", [(32, 8, 128, 4), (8, 2, 128, 1), (4, 2, 64, 3)])
 def test_attention_few_query_rows_key_parallel_kernel(H, G, hd, rps):
     """At most 16 query rows per (sequence, KV head) (chain drafts at batch, single-token decoding): the key-parallel
