@@ -172,6 +172,9 @@ static const char *check_cfg(const spec_cfg *c) {
   return nullptr;
 }
 
+// Prompt positions per prefill pass: the chunk's rows are each other's tail keys, causal through the two-word masks.
+constexpr int PREFILL_CHUNK = 128;
+
 // Derives sizes and carves every buffer; with c->cfg.workspace == nullptr (measure mode) only sizes.
 static size_t carve(spec_ctx *c, void *base) {
   const spec_cfg &g = c->cfg;
@@ -181,7 +184,7 @@ static size_t carve(spec_ctx *c, void *base) {
   c->pool = c->K + (c->D - 1) * c->K * c->K;
   c->esz = g.dtype == SPEC_F32 ? 4 : 2;
   c->Te = c->B * c->Pmax; c->Td = c->B * c->K; c->Tv = c->B * c->N;
-  c->R = std::max(std::max(c->Te, c->Td), std::max(c->Tv, 64));
+  c->R = std::max(std::max(c->Te, c->Td), std::max(c->Tv, PREFILL_CHUNK));
   c->Ralloc = (c->R + 63) / 64 * 64;
   c->pps = (g.max_ctx + g.page_size - 1) / g.page_size;
   c->tail_tree = std::max(1, (c->D - 1) * c->K);
@@ -759,7 +762,7 @@ template <typename T> static int do_prefill(spec_ctx *c, const int32_t *ids, con
   CUDA_TRY(c, cudaStreamSynchronize(s));
 
   Sched<T> sc(c);
-  const int CH = 64;
+  const int CH = PREFILL_CHUNK;
   std::vector<int32_t> mseq(CH), mpos(CH), mctx(CH), mtok(CH), mzero(CH, 0);
   std::vector<uint64_t> mlo(CH), mhi(CH, 0);
   auto upload_meta = [&](int nvalid, int b, int start, const int32_t *toks) -> cudaError_t {
@@ -767,6 +770,7 @@ template <typename T> static int do_prefill(spec_ctx *c, const int32_t *ids, con
       bool v = r < nvalid;
       mseq[r] = v ? b : -1; mpos[r] = v ? start + r : 0; mctx[r] = v ? start : 0; mtok[r] = v ? toks[r] : 0;
       mlo[r] = v ? (r >= 63 ? ~0ull : ((1ull << (r + 1)) - 1ull)) : 0ull;
+      mhi[r] = (v && r >= 64) ? (r >= 127 ? ~0ull : ((1ull << (r - 63)) - 1ull)) : 0ull;
     }
     cudaError_t e = cudaMemcpyAsync(c->meta.seq, mseq.data(), CH * 4, cudaMemcpyHostToDevice, s);
     if (!e) e = cudaMemcpyAsync(c->meta.pos, mpos.data(), CH * 4, cudaMemcpyHostToDevice, s);
