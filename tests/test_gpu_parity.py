@@ -232,6 +232,22 @@ def test_small_bf16_hd128_trajectory_tcgen05_attention(batch):
     print("T2 tcgen05 attention", st)
 
 
+# multi-head attention (one KV head per query head), as in the Vicuna-13B-shaped targets of the paper's Table 1
+T3_MHA = synth.ModelCfg("T3-small-bf16-mha", "bf16", 2, 512, 4, 4, 128, 1024, 4096, 1024, (0, 1, 1), 1e4,
+                        prompt_len=90, tree_depth=5, tree_topk=8, tree_nodes=50, seed=21)
+
+
+@pytest.mark.parametrize("batch", [1, 2])
+def test_mha_model_trajectory(batch):
+    """G = H (no grouping): 50-node trees, 8 x 4 = 32 draft rows per pass, also at batch 2 (trees at batch)."""
+    cfg = T3_MHA if batch == 1 else T3_MHA.replace(name="T3-b2", batch=2, prompt_lo=40, prompt_hi=100)
+    tw, dw = _weights(cfg)
+    prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+    st, _ = parity.run_trajectory(cfg, tw, dw, prompts, n_steps=6, tol=2e-2, tap_tol=3e-2)
+    print("T3 MHA", batch, st)
+    assert st.steps == 6
+
+
 DEGENERATE = {
     "depth1": dict(tree_depth=1, tree_topk=4, tree_nodes=5),                 # one draft pass, the tree is a star
     "chain_b1": dict(tree_depth=3, tree_topk=1, tree_nodes=4),               # top-1 chain at batch 1
