@@ -579,12 +579,17 @@ __device__ __forceinline__ float block_reduce_sum(float v, float *sh) {
   return r;
 }
 
+// exp on the special-function unit (ex2.approx): every term of a row goes through the same routine, so the
+// probabilities stay consistent; its relative error (~1e-6 near the maximum) is far inside the parity slack
+__device__ __forceinline__ float acc_exp(float x) { return __expf(x); }
+
 __global__ void __launch_bounds__(ACC_THREADS) accept_sampled_kernel(SeqState st, TreeBufs tb, const float *__restrict__ logits,
                                                                      int V, const float *__restrict__ u, int rows_per_seq) {
   pdl_wait();
   pdl_trigger();
   __shared__ float red[ACC_THREADS / 32];
-  __shared__ float part[ACC_THREADS];
+  __shared__ float part[ACC_THREADS / 32];
+  extern __shared__ float seg[];                           // [ceil(V / 32)] residual terms of the range that holds the drawn token
   __shared__ int32_t rej[ACC_MAX_REJ];
   __shared__ int s_next, s_nrej, s_pick, s_owner;
   __shared__ float s_target;
@@ -595,18 +600,44 @@ __global__ void __launch_bounds__(ACC_THREADS) accept_sampled_kernel(SeqState st
     if (tid == 0) tb.out_cnt[b] = 0;
     return;
   }
-  const int32_t *tok = tb.tok + (size_t)b * rows_per_seq, *par = tb.parent + (size_t)b * rows_per_seq;
-  const float *ub = u + (size_t)b * 2 * N;
+  // the tree and the uniforms go to shared memory once: the walk below is serial, and a global load per node would
+  // put an L2 round trip into every iteration
+  __shared__ int32_t tok[64], par[64];
+  __shared__ float ub[128];
+  if (tid < nn && tid < 64) { tok[tid] = tb.tok[(size_t)b * rows_per_seq + tid]; par[tid] = tb.parent[(size_t)b * rows_per_seq + tid]; }
+  if (tid < 2 * N && tid < 128) ub[tid] = u[(size_t)b * 2 * N + tid];
   const float inv_T = u[(size_t)gridDim.x * 2 * N];          // 1 / temperature follows the uniforms
+  __syncthreads();
   int cur = 0, a = 0;
   if (tid == 0) tb.path[b * Pmax] = 0;
   for (;;) {
     const float *z = logits + ((size_t)b * rows_per_seq + cur) * V;
+    // one SM reads the row from L2: wide, unrolled loads keep enough requests in flight
+    const bool vec = (V & 3) == 0;                       // rows are then 16-byte aligned
+    const float4 *z4 = (const float4 *)z;
     float m = -INFINITY;
-    for (int v = tid; v < V; v += ACC_THREADS) m = fmaxf(m, z[v]);
+    if (vec) {
+#pragma unroll 4
+      for (int i = tid; i < V / 4; i += ACC_THREADS) {
+        const float4 q = z4[i];
+        m = fmaxf(m, fmaxf(fmaxf(q.x, q.y), fmaxf(q.z, q.w)));
+      }
+    } else {
+#pragma unroll 8
+      for (int v = tid; v < V; v += ACC_THREADS) m = fmaxf(m, z[v]);
+    }
     const float zmax = block_reduce_max(m, red);
     float sum = 0.0f;
-    for (int v = tid; v < V; v += ACC_THREADS) sum += expf((z[v] - zmax) * inv_T);
+    if (vec) {
+#pragma unroll 4
+      for (int i = tid; i < V / 4; i += ACC_THREADS) {
+        const float4 q = z4[i];
+        sum += (acc_exp((q.x - zmax) * inv_T) + acc_exp((q.y - zmax) * inv_T)) + (acc_exp((q.z - zmax) * inv_T) + acc_exp((q.w - zmax) * inv_T));
+      }
+    } else {
+#pragma unroll 8
+      for (int v = tid; v < V; v += ACC_THREADS) sum += acc_exp((z[v] - zmax) * inv_T);
+    }
     float mass = block_reduce_sum(sum, red);
     // ---- the children of cur in node order, tried by one thread
     if (tid == 0) {
@@ -614,7 +645,7 @@ __global__ void __launch_bounds__(ACC_THREADS) accept_sampled_kernel(SeqState st
       if (a + 1 < Pmax) {
         for (int c = cur + 1; c < nn && nxt < 0; c++) {
           if (par[c] != cur) continue;
-          const float e = expf((z[tok[c]] - zmax) * inv_T);
+          const float e = acc_exp((z[tok[c]] - zmax) * inv_T);
           const float pc = mass > 0.0f ? e / mass : 0.0f;
           if (ub[c] < pc) nxt = c;
           else { mass -= e; if (nrej < ACC_MAX_REJ) rej[nrej++] = tok[c]; }
@@ -635,50 +666,71 @@ __global__ void __launch_bounds__(ACC_THREADS) accept_sampled_kernel(SeqState st
       __syncthreads();
       continue;
     }
-    // ---- the final token: inverse CDF over the residual.  Thread t owns the ids [t * C, (t + 1) * C).
-    const int C = (V + ACC_THREADS - 1) / ACC_THREADS;
-    const int v0 = tid * C, v1 = (v0 + C < V) ? v0 + C : V;
+    // ---- the final token: inverse CDF over the residual, in two levels.  Warp w owns the ids [w * CW, (w + 1) * CW):
+    // its lanes read them coalesced and the warp sum goes to part[w]; one thread finds the warp whose range holds the
+    // target; that warp then walks its range 32 ids at a time with a warp prefix sum.
+    const int NWARP = ACC_THREADS / 32, wid = tid >> 5, ln = tid & 31;
+    const int CW = (V + NWARP - 1) / NWARP;
+    const int w0 = wid * CW, w1 = (w0 + CW < V) ? w0 + CW : V;
     float loc = 0.0f;
-    for (int v = v0; v < v1; v++) {
-      bool gone = false;
-      for (int r = 0; r < nrej; r++) gone |= (rej[r] == v);
-      if (!gone) loc += expf((z[v] - zmax) * inv_T);
-    }
-    part[tid] = loc;
+#pragma unroll 8
+    for (int v = w0 + ln; v < w1; v += 32) loc += acc_exp((z[v] - zmax) * inv_T);
+    for (int o = 16; o > 0; o >>= 1) loc += __shfl_xor_sync(0xffffffffu, loc, o);
+    if (ln == 0) part[wid] = loc;
     __syncthreads();
     if (tid == 0) {
+      for (int r = 0; r < nrej; r++) {                   // the rejected tokens leave the residual
+        const float e = acc_exp((z[rej[r]] - zmax) * inv_T);
+        const int w = rej[r] / CW;
+        part[w] = fmaxf(part[w] - e, 0.0f);
+      }
       float total = 0.0f;
-      for (int t = 0; t < ACC_THREADS; t++) total += part[t];
+      for (int w = 0; w < NWARP; w++) total += part[w];
       const float target = ub[N + cur] * total;
       float cum = 0.0f;
       int owner = -1;
-      for (int t = 0; t < ACC_THREADS; t++) {
-        if (part[t] > 0.0f && cum + part[t] > target) { owner = t; break; }
-        cum += part[t];
+      for (int w = 0; w < NWARP; w++) {
+        if (part[w] > 0.0f && cum + part[w] > target) { owner = w; break; }
+        cum += part[w];
       }
-      if (owner < 0) {                                   // rounding at the upper end: the last thread with mass
+      if (owner < 0) {                                   // rounding at the upper end: the last warp with mass
         cum = total;
-        for (int t = ACC_THREADS - 1; t >= 0; t--)
-          if (part[t] > 0.0f) { owner = t; cum = total - part[t]; break; }
+        for (int w = NWARP - 1; w >= 0; w--)
+          if (part[w] > 0.0f) { owner = w; cum = total - part[w]; break; }
       }
       s_owner = owner; s_target = target - cum; s_pick = 0;
     }
     __syncthreads();
-    if (tid == s_owner) {
+    // the owning warp's range goes to shared memory with every thread's help (one parallel, coalesced pass), so the
+    // ordered walk below reads no global memory
+    {
+      const int o0 = s_owner * CW, o1 = (o0 + CW < V) ? o0 + CW : V;
+      for (int v = o0 + tid; v < o1; v += ACC_THREADS) {
+        float e = acc_exp((z[v] - zmax) * inv_T);
+        for (int r = 0; r < nrej; r++) if (rej[r] == v) e = 0.0f;
+        seg[v - o0] = e;
+      }
+    }
+    __syncthreads();
+    if (wid == s_owner) {
       const float target = s_target;
       float cum = 0.0f;
-      int pick = -1, last = v0;
-      for (int v = v0; v < v1; v++) {
-        bool gone = false;
-        for (int r = 0; r < nrej; r++) gone |= (rej[r] == v);
-        if (gone) continue;
-        const float e = expf((z[v] - zmax) * inv_T);
-        if (e <= 0.0f) continue;
-        last = v;
-        if (cum + e > target) { pick = v; break; }
-        cum += e;
+      int pick = -1, last = -1;
+      for (int base = w0; base < w1 && pick < 0; base += 32) {
+        const int v = base + ln;
+        const float e = v < w1 ? seg[v - w0] : 0.0f;
+        float inc = e;                                   // inclusive prefix sum over the 32 lanes
+        for (int o = 1; o < 32; o <<= 1) {
+          const float t = __shfl_up_sync(0xffffffffu, inc, o);
+          if (ln >= o) inc += t;
+        }
+        const bool hit = e > 0.0f && cum + inc > target;
+        const unsigned hits = __ballot_sync(0xffffffffu, hit), alive = __ballot_sync(0xffffffffu, e > 0.0f);
+        if (alive) last = base + 31 - __clz(alive);
+        if (hits) pick = base + __ffs(hits) - 1;
+        cum += __shfl_sync(0xffffffffu, inc, 31);
       }
-      s_pick = pick >= 0 ? pick : last;
+      if (ln == 0) s_pick = pick >= 0 ? pick : (last >= 0 ? last : w0);
     }
     __syncthreads();
     if (tid == 0) {
@@ -697,7 +749,13 @@ __global__ void __launch_bounds__(ACC_THREADS) accept_sampled_kernel(SeqState st
   }
 }
 void launch_accept_sampled(SeqState st, TreeBufs tb, const float *logits, int V, const float *u, int B, int rows_per_seq, cudaStream_t s) {
-  launch_k(accept_sampled_kernel, dim3(B), dim3(ACC_THREADS), 0, s, st, tb, logits, V, u, rows_per_seq);
+  const size_t smem = (size_t)((V + ACC_THREADS / 32 - 1) / (ACC_THREADS / 32)) * sizeof(float);
+  static size_t configured = 0;
+  if (smem > 40 * 1024 && smem > configured) {
+    cudaFuncSetAttribute(accept_sampled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    configured = smem;
+  }
+  launch_k(accept_sampled_kernel, dim3(B), dim3(ACC_THREADS), smem, s, st, tb, logits, V, u, rows_per_seq);
 }
 
 // ---------------------------------------------------------------- commit: KV compaction + tap gather
