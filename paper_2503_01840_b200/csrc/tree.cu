@@ -519,12 +519,18 @@ __global__ void accept_kernel(SeqState st, TreeBufs tb, int rows_per_seq) {
   pdl_wait();
   pdl_trigger();
   int b = blockIdx.x;
-  if (threadIdx.x != 0) return;
   int Pmax = tb.Pmax;
   int nn = tb.nn[b];
+  // the walk is serial: the tree goes to shared memory first, so that no iteration waits for a global load
+  __shared__ int32_t tok[64], par[64], y[64];
+  for (int i = threadIdx.x; i < nn && i < 64; i += blockDim.x) {
+    tok[i] = tb.tok[(size_t)b * rows_per_seq + i];
+    par[i] = tb.parent[(size_t)b * rows_per_seq + i];
+    y[i] = tb.y[(size_t)b * rows_per_seq + i];
+  }
+  __syncthreads();
+  if (threadIdx.x != 0) return;
   if (!st.active[b] || nn < 1) { tb.out_cnt[b] = 0; return; }
-  const int32_t *tok = tb.tok + (size_t)b * rows_per_seq, *par = tb.parent + (size_t)b * rows_per_seq;
-  const int32_t *y = tb.y + (size_t)b * rows_per_seq;
   int cur = 0, a = 0;
   tb.path[b * Pmax] = 0;
   while (a + 1 < Pmax) {
@@ -773,23 +779,50 @@ __global__ void __launch_bounds__(256) commit_kernel(SeqState st, TreeBufs tb, c
   int cnt = tb.out_cnt[b];
   if (cnt <= 0) return;
   int n0 = st.n_prev[b], Pmax = tb.Pmax;
+  constexpr int VEC = 16 / (int)sizeof(T);           // elements per 16-byte vector (head_dim is a multiple of 16)
+  constexpr int JB = 8;                              // accepted nodes moved per batch
+  __shared__ int32_t path_s[64];
+  for (int j = threadIdx.x; j < cnt && j < 64; j += blockDim.x) path_s[j] = tb.path[b * Pmax + j];
+  __syncthreads();
   if (l < L) {
+    // A thread owns the same 16-byte vectors of every position.  Per batch of JB accepted nodes it issues all its loads
+    // before its first store: a destination slot j can only be the source of an earlier node (path[j'] >= j'), never
+    // of a later batch, and within a batch every load has been issued before any store.
     T *Kp = (T *)pools[l].k, *Vp = (T *)pools[l].v;
-    for (int j = 0; j < cnt; j++) {
-      int src = n0 + tb.path[b * Pmax + j], dst = n0 + j;
-      if (src == dst) continue;
-      for (int e = threadIdx.x; e < G * hd; e += blockDim.x) {
-        int g = e / hd, i = e % hd;
-        size_t so = kv_offset(pm, b, src, g, G, hd) + i, dof = kv_offset(pm, b, dst, g, G, hd) + i;
-        Kp[dof] = Kp[so];
-        Vp[dof] = Vp[so];
+    const int nvec = G * hd / VEC;
+    for (int t = threadIdx.x; t < nvec; t += blockDim.x) {
+      const int g = (t * VEC) / hd, i = (t * VEC) % hd;
+      for (int j0 = 0; j0 < cnt; j0 += JB) {
+        uint4 kv[JB], vv[JB];
+        size_t dof[JB];
+        bool mv[JB];
+#pragma unroll
+        for (int jj = 0; jj < JB; jj++) {
+          const int j = j0 + jj;
+          mv[jj] = false;
+          if (j < cnt) {
+            const int src = n0 + path_s[j], dst = n0 + j;
+            mv[jj] = src != dst;
+            if (mv[jj]) {
+              const size_t so = kv_offset(pm, b, src, g, G, hd) + i;
+              dof[jj] = kv_offset(pm, b, dst, g, G, hd) + i;
+              kv[jj] = *(const uint4 *)(Kp + so);
+              vv[jj] = *(const uint4 *)(Vp + so);
+            }
+          }
+        }
+#pragma unroll
+        for (int jj = 0; jj < JB; jj++)
+          if (mv[jj]) { *(uint4 *)(Kp + dof[jj]) = kv[jj]; *(uint4 *)(Vp + dof[jj]) = vv[jj]; }
       }
     }
   } else {
+    // taps of the accepted nodes -> pending entries (different buffers: no ordering needed)
+    const int nvec = 3 * k / VEC;
     for (int j = 0; j < cnt; j++) {
-      const T *src = node_taps + ((size_t)b * rows_per_seq + tb.path[b * Pmax + j]) * 3 * k;
-      T *dst = pend_taps + ((size_t)b * Pmax + j) * 3 * k;
-      for (int e = threadIdx.x; e < 3 * k; e += blockDim.x) dst[e] = src[e];
+      const uint4 *src = (const uint4 *)(node_taps + ((size_t)b * rows_per_seq + path_s[j]) * 3 * k);
+      uint4 *dst = (uint4 *)(pend_taps + ((size_t)b * Pmax + j) * 3 * k);
+      for (int e = threadIdx.x; e < nvec; e += blockDim.x) dst[e] = src[e];
     }
   }
 }
