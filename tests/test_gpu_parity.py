@@ -248,6 +248,28 @@ def test_mha_model_trajectory(batch):
     assert st.steps == 6
 
 
+@pytest.mark.parametrize("base", [C1, T1], ids=["fp32", "bf16"])
+def test_prefill_chunk_boundaries(base):
+    """Prompts of 127, 128, 129 and 257 tokens: the prefill runs 128-position chunks whose rows see each other through
+    the two-word causal masks; the first token, the first steps and the committed K/V must match the oracle."""
+    for n in (127, 128, 129, 257):
+        cfg = base.replace(name=f"{base.name}-p{n}", prompt_len=n)
+        tw, dw = _weights(cfg)
+        prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+        assert len(prompts[0]) == n
+        tol = 1e-4 if cfg.dtype == "fp32" else 2e-2
+        st, _ = parity.run_trajectory(cfg, tw, dw, prompts, n_steps=2, tol=tol, tap_tol=None if cfg.dtype == "fp32" else 3e-2)
+        dec = sb.SpecDecoder(cfg, parity.to_dev(tw), parity.to_dev(dw), batch=1, max_ctx=n + 64)
+        orc = po.Oracle(cfg, tw, dw, n + 64)
+        assert dec.prefill(prompts, 8)[0] == orc.prefill(prompts[0])
+        for pos in (0, 63, 64, 126, n - 2, n - 1):
+            for layer in range(cfg.n_layers):
+                gk, gv = dec.read_kv(0, layer, pos)
+                ok, ov = orc.target_kv(layer, pos)
+                assert np.abs(gk - ok).max() < 4 * tol and np.abs(gv - ov).max() < 4 * tol, (n, pos, layer)
+        dec.close()
+
+
 DEGENERATE = {
     "depth1": dict(tree_depth=1, tree_topk=4, tree_nodes=5),                 # one draft pass, the tree is a star
     "chain_b1": dict(tree_depth=3, tree_topk=1, tree_nodes=4),               # top-1 chain at batch 1
