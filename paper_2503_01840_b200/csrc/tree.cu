@@ -120,25 +120,29 @@ __global__ void __launch_bounds__(256) topk_partial_kernel(const float *__restri
                                                            int32_t *__restrict__ cidx) {
   pdl_wait();
   pdl_trigger();
-  __shared__ VI sh[32];
-  __shared__ float shf[32];
-  int r = blockIdx.y, ch = blockIdx.x;
-  int sr = src_row ? src_row[r] : r;
+  // Warp w owns the 128 consecutive logits base + 128 w ...: it finds its own K best with shuffles only (no block
+  // barrier per round); the 8 x K warp candidates are then ranked against each other by counting.
+  __shared__ float shf[8];
+  __shared__ float wv[8 * TOPK_MAXK];
+  __shared__ int32_t wi[8 * TOPK_MAXK];
+  const int r = blockIdx.y, ch = blockIdx.x;
+  const int sr = src_row ? src_row[r] : r;
   if (sr < 0) return;
   const float *z = logits + (size_t)sr * n;
-  int base = ch * TOPK_CHUNK;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int base = ch * TOPK_CHUNK + warp * 128;
   float v[4];
   int id[4];
   float mx = -INFINITY;
 #pragma unroll
   for (int j = 0; j < 4; j++) {
-    id[j] = base + j * 256 + threadIdx.x;
+    id[j] = base + j * 32 + lane;
     v[j] = id[j] < n ? z[id[j]] : -INFINITY;
     if (id[j] >= n) id[j] = -1;
     mx = fmaxf(mx, v[j]);
   }
   for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-  if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = mx;
+  if (lane == 0) shf[warp] = mx;
   __syncthreads();
   mx = shf[0];
   for (int w = 1; w < 8; w++) mx = fmaxf(mx, shf[w]);
@@ -147,7 +151,24 @@ __global__ void __launch_bounds__(256) topk_partial_kernel(const float *__restri
 #pragma unroll
   for (int j = 0; j < 4; j++) sum += id[j] >= 0 ? expf(v[j] - mx) : 0.0f;
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-  if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = sum;
+  if (lane == 0) shf[warp] = sum;
+  // ---- this warp's K best, best first
+  for (int c = 0; c < K; c++) {
+    float bv = 0.0f;
+    int bi = -1;
+#pragma unroll
+    for (int j = 0; j < 4; j++)
+      if (id[j] >= 0 && (bi < 0 || before(v[j], id[j], bv, bi))) { bv = v[j]; bi = id[j]; }
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (oi >= 0 && (bi < 0 || before(ov, oi, bv, bi))) { bv = ov; bi = oi; }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; j++)
+      if (id[j] == bi) id[j] = -1;            // taken (bi is -1 only when the warp's range is exhausted)
+    if (lane == 0) { wv[warp * K + c] = bv; wi[warp * K + c] = bi; }
+  }
   __syncthreads();
   if (threadIdx.x == 0) {
     float t = 0.0f;
@@ -155,19 +176,23 @@ __global__ void __launch_bounds__(256) topk_partial_kernel(const float *__restri
     pmax[(size_t)r * nch + ch] = mx;
     psum[(size_t)r * nch + ch] = t;
   }
-  for (int c = 0; c < K; c++) {
-    VI b{0.0f, -1};
-#pragma unroll
-    for (int j = 0; j < 4; j++)
-      if (id[j] >= 0 && (b.i < 0 || before(v[j], id[j], b.v, b.i))) { b.v = v[j]; b.i = id[j]; }
-    b = block_best(b, sh);
-#pragma unroll
-    for (int j = 0; j < 4; j++)
-      if (id[j] == b.i) id[j] = -1;           // taken (b.i is -1 only when the chunk is exhausted)
-    if (threadIdx.x == 0) {
-      cval[((size_t)r * nch + ch) * K + c] = b.v;
-      cidx[((size_t)r * nch + ch) * K + c] = b.i;
+  // ---- the chunk's K best of the 8 K warp candidates, by rank (value desc, index asc)
+  const int nc = 8 * K;
+  int my = -1;
+  float mv = 0.0f;
+  if ((int)threadIdx.x < nc) { my = wi[threadIdx.x]; mv = wv[threadIdx.x]; }
+  const int nvalid = __syncthreads_count(my >= 0);
+  if (my >= 0) {
+    int rank = 0;
+    for (int j = 0; j < nc; j++) rank += (wi[j] >= 0 && before(wv[j], wi[j], mv, my)) ? 1 : 0;
+    if (rank < K) {
+      cval[((size_t)r * nch + ch) * K + rank] = mv;
+      cidx[((size_t)r * nch + ch) * K + rank] = my;
     }
+  }
+  for (int c = nvalid + (int)threadIdx.x; c < K; c += blockDim.x) {      // fewer than K logits in the chunk
+    cval[((size_t)r * nch + ch) * K + c] = 0.0f;
+    cidx[((size_t)r * nch + ch) * K + c] = -1;
   }
 }
 
@@ -358,28 +383,33 @@ __global__ void __launch_bounds__(256) expand_kernel(SeqState st, TreeBufs tb, R
   uint64_t *pm_lo = (uint64_t *)(cs + ((nch + 1) & ~1));   // [K] parent masks
   uint64_t *pm_hi = pm_lo + K;
   int32_t *newf = (int32_t *)(pm_hi + K);   // [K] local child index of the new frontier
-  if (!st.active[b]) {   // skipped sequence: its rows of the next pass are padding
+  int32_t *ctok = newf + K;                 // [nch] child tokens (target ids)
+  // every load that does not depend on another is issued up front: the kernel is a chain of L2 round trips otherwise
+  const int active = st.active[b], n = st.n[b], last_row = st.last_row[b];
+  if (!active) {   // skipped sequence: its rows of the next pass are padding
     for (int rr = threadIdx.x; rr < K; rr += blockDim.x) { m.seq[b * K + rr] = -1; m.tok[b * K + rr] = 0; m.pos[b * K + rr] = 0; }
     return;
   }
   size_t pb = (size_t)b * (tb.pool + 1);
   int base = (pass == 1) ? 0 : K + (pass - 2) * K * K;     // pool index of child 0 is base + 1
-  int n = st.n[b];
+  for (int r = threadIdx.x; r < K; r += blockDim.x) {
+    pm_lo[r] = (pass == 1) ? 0ull : m.mask_lo[b * K + r];
+    pm_hi[r] = (pass == 1) ? 0ull : m.mask_hi[b * K + r];
+  }
   for (int c = threadIdx.x; c < nch; c += blockDim.x) {
     int r = (pass == 1) ? 0 : c / K, cc = (pass == 1) ? c : c % K;
     int row = (pass == 1) ? b : b * K + r;                  // row of the top-k output
     int u = (pass == 1) ? 0 : tb.front_cur[b * K + r];
-    float sc = tb.pool_score[pb + u] + tb.tk_lp[(size_t)row * K + cc];
+    const float lp = tb.tk_lp[(size_t)row * K + cc];
+    const int tokid = d2t[tb.tk_idx[(size_t)row * K + cc]];
+    float sc = tb.pool_score[pb + u] + lp;
     int ci = base + c + 1;
-    tb.pool_tok[pb + ci] = d2t[tb.tk_idx[(size_t)row * K + cc]];
+    tb.pool_tok[pb + ci] = tokid;
+    ctok[c] = tokid;
     tb.pool_parent[pb + ci] = u;
     tb.pool_depth[pb + ci] = pass;
     tb.pool_score[pb + ci] = sc;
     cs[c] = sc;
-  }
-  for (int r = threadIdx.x; r < K; r += blockDim.x) {
-    pm_lo[r] = (pass == 1) ? 0ull : m.mask_lo[b * K + r];
-    pm_hi[r] = (pass == 1) ? 0ull : m.mask_hi[b * K + r];
   }
   __syncthreads();
   if (pass >= D) return;
@@ -391,7 +421,6 @@ __global__ void __launch_bounds__(256) expand_kernel(SeqState st, TreeBufs tb, R
     if (rank < K) newf[rank] = c;
   }
   __syncthreads();
-  int last_row = st.last_row[b];
   for (int rr = threadIdx.x; rr < K; rr += blockDim.x) {
     int c = newf[rr];
     int ci = base + c + 1;
@@ -410,12 +439,12 @@ __global__ void __launch_bounds__(256) expand_kernel(SeqState st, TreeBufs tb, R
     m.tail_base[row] = n;
     m.mask_lo[row] = lo;
     m.mask_hi[row] = hi;
-    m.tok[row] = tb.pool_tok[pb + ci];
+    m.tok[row] = ctok[c];
   }
 }
 void launch_expand(SeqState st, TreeBufs tb, RowMeta m, const int32_t *d2t, int pass, int B, cudaStream_t s) {
   int K = tb.K, nch = K * K;
-  size_t smem = (size_t)((nch + 1) & ~1) * 4 + (size_t)K * 16 + (size_t)K * 4 + 16;
+  size_t smem = (size_t)((nch + 1) & ~1) * 4 + (size_t)K * 16 + (size_t)K * 4 + (size_t)nch * 4 + 16;
   launch_k(expand_kernel, dim3(B), dim3(256), smem, s, st, tb, m, d2t, pass);
 }
 
