@@ -33,8 +33,22 @@ def trajectory():
     g = po.Oracle(cfg, tw, dw, 256)
     g.prefill(prompt)
     greedy = [first] + [int(t) for t in g.greedy(len(tokens) - 1)]
+    # the same start at temperature 1 with stored uniforms (multiples of 2^-16, so the file holds them exactly): the
+    # stochastic acceptance rule's own trajectory
+    import numpy as np
+    rng = np.random.default_rng(2503)
+    s = po.Oracle(cfg, tw, dw, 256)
+    s.prefill(prompt)
+    sampled_u, sampled_tokens, sampled_counts = [], [first], []
+    for _ in range(8):
+        u = (rng.integers(0, 1 << 16, 2 * cfg.tree_nodes) / float(1 << 16)).astype(np.float32)
+        out = s.step_sampled(1.0, u)
+        sampled_u.append([float(x) for x in u])
+        sampled_counts.append(len(out))
+        sampled_tokens += [int(t) for t in out]
     return {"config": cfg.name, "prompt_head": [int(t) for t in prompt[:8]], "first_token": first, "tokens": tokens,
-            "counts": counts, "greedy": greedy}
+            "counts": counts, "greedy": greedy,
+            "sampled_T1": {"uniforms": sampled_u, "tokens": sampled_tokens, "counts": sampled_counts}}
 
 
 if __name__ == "__main__":

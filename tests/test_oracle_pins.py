@@ -555,4 +555,5 @@ def test_golden_c1_trajectory_is_reproduced_and_lossless():
     stored = json.load(open(os.path.join(here, "c1_oracle_trajectory.json")))
     assert stored["tokens"] == stored["greedy"][: len(stored["tokens"])]          # Section 2.1: lossless at temperature 0
     assert all(1 <= c <= C1.tree_depth + 1 for c in stored["counts"]) and sum(stored["counts"]) == len(stored["tokens"]) - 1
+    assert sum(stored["sampled_T1"]["counts"]) == len(stored["sampled_T1"]["tokens"]) - 1
     assert make_golden.trajectory() == stored
