@@ -1210,7 +1210,7 @@ int launch_tma_small(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUte
 }
 
 int g_attn_umma = 2;            // tcgen05 kernel for the tree passes: 0 off, 1 on, 2 on when a CTA gets at least UM_MIN_TILES key tiles
-constexpr int UM_MIN_TILES = 4; // below that the pass is launch- and latency-bound and the mma.sync kernel's shorter prologue wins
+constexpr int UM_MIN_TILES = 3; // below that the pass is launch- and latency-bound and the mma.sync kernel's shorter prologue wins
 thread_local int tl_attn_umma = -1;   // per-call override (-1: none)
 
 int launch_umma(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorMap *mv, int32_t *status, cudaStream_t s) {
