@@ -220,7 +220,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="C2", help="C1..C5, optionally ':L=<layers>' for a truncation")
+    ap.add_argument("--workload", default="C2", help="C1..C8, optionally ':L=<layers>' for a truncation")
     ap.add_argument("--no-extras", action="store_true", help="skip plain-decode / structured-acceptance / CPU legs")
     ap.add_argument("--flags", type=int, default=0)
     args = ap.parse_args()

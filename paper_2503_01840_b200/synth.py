@@ -86,7 +86,14 @@ C3 = C2.replace(name="C3-8B-b64-chain", batch=64, prompt_lo=256, prompt_hi=2048,
 C4 = C2.replace(name="C4-8B-16k", prompt_len=16384, gen_tokens=1024, tree_depth=8, seed=4)
 C5 = ModelCfg("C5-70B-b1", "bf16", 80, 8192, 64, 8, 128, 28672, 128256, 32000, (2, 40, 77), 5e5,
               batch=1, prompt_len=4096, gen_tokens=128, tree_depth=6, tree_topk=10, tree_nodes=60, seed=5)
-CONFIGS = {"C1": C1, "C2": C2, "C3": C3, "C4": C4, "C5": C5}
+# Further workloads of the paper's evaluation (Section 4, Appendix A): full trees at a small batch, a 13B-shaped
+# multi-head-attention target (vocabulary 32000, 50 tree nodes, depth 8) and the serving study's chain of 2.
+C6 = C2.replace(name="C6-8B-b4-tree", batch=4, prompt_lo=256, prompt_hi=2048, gen_tokens=128, seed=6)
+C7 = ModelCfg("C7-13B-mha-b1", "bf16", 40, 5120, 40, 40, 128, 13824, 32000, 32000, (2, 20, 37), 1e4,
+              batch=1, prompt_len=512, gen_tokens=256, tree_depth=8, tree_topk=10, tree_nodes=50, seed=7)
+C8 = C2.replace(name="C8-8B-b56-chain2", batch=56, prompt_lo=256, prompt_hi=2048, gen_tokens=128,
+                tree_depth=2, tree_topk=1, tree_nodes=3, seed=8)
+CONFIGS = {"C1": C1, "C2": C2, "C3": C3, "C4": C4, "C5": C5, "C6": C6, "C7": C7, "C8": C8}
 
 
 # ----------------------------------------------------------------------------- hash

@@ -127,6 +127,54 @@ def test_c3_shape_two_layers_batch64_losslessness():
     assert mismatches <= 16, mismatches
 
 
+def test_c6_shape_two_layers_batch4_full_trees_losslessness():
+    """8B widths, batch 4, full trees (depth 6, top-k 10, 60 nodes: 240 rows per verify pass), 2-layer truncation:
+    every sequence's tree is a valid tree and the speculative output equals plain greedy decoding on the same kernels
+    (a low-margin token may differ)."""
+    cfg = synth.C6.truncated(2)
+    tw = synth.make_target_weights(cfg, device="cuda")
+    dw = synth.make_draft_weights(cfg, device="cuda")
+    prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+    assert len(prompts) == 4
+    for seq in (0, 3):
+        dec, out, mismatches = _spec_vs_plain(cfg, tw, dw, prompts, n_steps=4, capture_seq=seq)
+        dec.close()
+        assert mismatches <= 1, mismatches
+
+
+def test_c8_shape_two_layers_batch56_chain2_losslessness():
+    """The serving study's setting (Section 4.3: no tree, chains of at most 2 draft tokens), batch 56, 8B widths,
+    2-layer truncation."""
+    cfg = synth.C8.truncated(2)
+    tw = synth.make_target_weights(cfg, device="cuda")
+    dw = synth.make_draft_weights(cfg, device="cuda")
+    prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+    dec, out, mismatches = _spec_vs_plain(cfg, tw, dw, prompts, n_steps=4, capture_seq=55)
+    dec.close()
+    assert mismatches <= 14, mismatches
+
+
+def test_c7_full_size_mha_losslessness_and_sampled_lm_head():
+    """13B-shaped multi-head-attention target (40 layers, 40 heads = 40 KV heads, vocabulary 32000 = draft vocabulary)
+    with the paper's tree for that size (Appendix A: 50 nodes, depth 8, top-k 10) at full depth."""
+    cfg = synth.C7
+    tw = synth.make_target_weights(cfg, device="cuda")
+    dw = synth.make_draft_weights(cfg, device="cuda")
+    prompts = [p.numpy() for p in synth.make_prompts(cfg)]
+    dec, out, _ = _spec_vs_plain(cfg, tw, dw, prompts, n_steps=4)
+    nn = dec.debug(sb.DBG_TREE_TOK, 0).size
+    hidden = dec.debug(sb.DBG_NODE_HIDDEN, 0).reshape(nn, cfg.hidden)
+    logits = dec.debug(sb.DBG_TARGET_LOGITS, 0).reshape(nn, cfg.vocab)
+    rows = np.random.default_rng(0).choice(cfg.vocab, 96, replace=False)
+    rows[:2] = [0, cfg.vocab - 1]
+    w_rows = tw["lm_head"][torch.from_numpy(rows).cuda()].cpu()
+    for node in (0, nn // 2, nn - 1):
+        h = po.rmsnorm(tw["final_norm"].cpu(), hidden[node:node + 1], cfg.rms_eps)
+        ref = po.linear(w_rows, h)[0]
+        assert np.abs(ref - logits[node, rows]).max() < 2e-2
+    dec.close()
+
+
 @pytest.mark.parametrize("impl", [0, 2, 3], ids=["cp_async", "tma", "tcgen05"])
 def test_c4_long_context_attention_sampled_vs_oracle(impl):
     """Tree-masked attention over a 16384-token paged context (many key splits + combine), 60 nodes x 32 heads;
