@@ -49,6 +49,24 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *(uint32_t *)&v;
 }
+
+// Tail masks as one word per 64-key tile.  clip_tail drops mask bits at and past tail_len; tile_allow returns the word
+// whose bit j says whether key k0 + j may be attended: every context key (k0 + j < ctx), and tail key
+// tt = k0 + j - ctx by bit tt of the row's two-word mask.
+__device__ __forceinline__ void clip_tail(uint64_t &lo, uint64_t &hi, int tail_len) {
+  if (tail_len < 64) { lo &= (tail_len <= 0) ? 0ull : (~0ull >> (64 - tail_len)); hi = 0ull; }
+  else if (tail_len < 128) hi &= (tail_len == 64) ? 0ull : (~0ull >> (128 - tail_len));
+}
+__device__ __forceinline__ uint64_t tile_allow(uint64_t lo, uint64_t hi, int ctx, int k0) {
+  const int sft = k0 - ctx;                     // tail index of the tile's first key (negative: context keys first)
+  if (sft <= -64) return ~0ull;
+  if (sft < 0) return (~0ull >> (64 + sft)) | (lo << (-sft));
+  if (sft == 0) return lo;
+  if (sft < 64) return (lo >> sft) | (hi << (64 - sft));
+  if (sft == 64) return hi;
+  if (sft < 128) return hi >> (sft - 64);
+  return 0ull;
+}
 // byte offset of 16-byte chunk `c` of row `row` in a tile with ROWB bytes per row, XOR-swizzled
 template <int ROWB> __device__ __forceinline__ uint32_t swz(int row, int c) { return (uint32_t)(row * ROWB + ((c ^ (row & 7)) << 4)); }
 
@@ -401,6 +419,8 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
   bool vA = false, vB = false;
   if (mA < M) { int r = row0 + mA / grp; vA = p.m.seq[r] >= 0; if (vA) { loA = p.m.mask_lo[r]; hiA = p.m.mask_hi[r]; } }
   if (mB < M) { int r = row0 + mB / grp; vB = p.m.seq[r] >= 0; if (vB) { loB = p.m.mask_lo[r]; hiB = p.m.mask_hi[r]; } }
+  clip_tail(loA, hiA, p.tail_len);
+  clip_tail(loB, hiB, p.tail_len);
 
   float o[HD / 8][4];
 #pragma unroll
@@ -439,16 +459,16 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
         tmB = fmaxf(tmB, fmaxf(s[n][2], s[n][3]));
       }
     } else {
+      // one allow word per row for the tile, shifted so that this lane's keys sit at bits 8 n + e
+      const uint64_t wA = (vA ? tile_allow(loA, hiA, ctx, t * KT) : 0ull) >> ((lane & 3) * 2);
+      const uint64_t wB = (vB ? tile_allow(loB, hiB, ctx, t * KT) : 0ull) >> ((lane & 3) * 2);
+      const uint32_t wA0 = (uint32_t)wA, wA1 = (uint32_t)(wA >> 32), wB0 = (uint32_t)wB, wB1 = (uint32_t)(wB >> 32);
 #pragma unroll
       for (int n = 0; n < KT / 8; n++) {
-  #pragma unroll
+#pragma unroll
         for (int e = 0; e < 2; e++) {
-          int key = t * KT + n * 8 + (lane & 3) * 2 + e;
-          bool in_ctx = key < ctx;
-          int tt = key - ctx;
-          bool in_tail = !in_ctx && tt < p.tail_len;
-          bool okA = vA && (in_ctx || (in_tail && ((tt < 64 ? (loA >> tt) : (hiA >> (tt - 64))) & 1ull)));
-          bool okB = vB && (in_ctx || (in_tail && ((tt < 64 ? (loB >> tt) : (hiB >> (tt - 64))) & 1ull)));
+          const uint32_t bit = 1u << ((n & 3) * 8 + e);
+          const bool okA = ((n < 4 ? wA0 : wA1) & bit) != 0u, okB = ((n < 4 ? wB0 : wB1) & bit) != 0u;
           s[n][e] = okA ? s[n][e] : -INFINITY;
           s[n][2 + e] = okB ? s[n][2 + e] : -INFINITY;
           tmA = fmaxf(tmA, s[n][e]);
@@ -644,6 +664,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
   if (warp < 8) {
     if (mrow < M) { qi = mrow / grp; qh = mrow % grp; rvalid = p.m.seq[row0 + qi] >= 0; }
     if (rvalid) { mlo = p.m.mask_lo[row0 + qi]; mhi = p.m.mask_hi[row0 + qi]; }
+    else { mlo = ~0ull; mhi = ~0ull; }                         // a padding row attends every tail key (zeroed at the end)
+    clip_tail(mlo, mhi, p.tail_len);
     const uint4 *src = (const uint4 *)(p.q + ((size_t)(row0 + qi) * p.H + g * grp + qh) * HD);
 #pragma unroll
     for (int cc = 0; cc < 8; cc++) {                        // each of the row's two threads copies one half of it
@@ -767,12 +789,11 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
 #pragma unroll
         for (int e = 0; e < KT; e++) tm = fmaxf(tm, s[e]);
       } else {
+        const uint64_t w = tile_allow(mlo, mhi, ctx, t * KT);
+        const uint32_t w0 = (uint32_t)w, w1 = (uint32_t)(w >> 32);
 #pragma unroll
         for (int e = 0; e < KT; e++) {
-          const int key = t * KT + e, tt = key - ctx;
-          const bool in_ctx = key < ctx;
-          const bool in_tail = !in_ctx && tt < p.tail_len;
-          const bool okk = in_ctx || (in_tail && (!rvalid || ((tt < 64 ? (mlo >> tt) : (mhi >> (tt - 64))) & 1ull)));
+          const bool okk = ((e < 32 ? w0 : w1) & (1u << (e & 31))) != 0u;
           s[e] = okk ? s[e] : -INFINITY;
           tm = fmaxf(tm, s[e]);
         }
