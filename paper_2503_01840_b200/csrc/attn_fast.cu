@@ -327,16 +327,17 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int grp = p.H / p.G;
   const int zb = blockIdx.z / p.G, g = blockIdx.z % p.G;
-  int b = p.order ? p.order[zb] : zb;            // row block (sequence) of this CTA
-  if ((unsigned)b >= gridDim.z / (unsigned)p.G) b = zb;
+  const unsigned nblk = gridDim.z / (unsigned)p.G;
+  int b = (p.order && nblk > 1) ? p.order[zb] : zb;    // row block (sequence) of this CTA
+  if ((unsigned)b >= nblk) b = zb;
   const int M = p.rps * grp;
   const int m0 = blockIdx.x * MT;
   const int row0 = b * p.rps;
   const int ps = p.pm.page_size;                       // keys per page = rows per tensor copy
   int seq = -1, ctx = 0;
   for (int i = 0; i < p.rps; i++) {
-    int s = p.m.seq[row0 + i];
-    if (s >= 0) { seq = s; ctx = p.m.ctx[row0 + i]; break; }
+    const int s = p.m.seq[row0 + i], cx = p.m.ctx[row0 + i];   // both loads in flight together
+    if (s >= 0) { seq = s; ctx = cx; break; }
   }
   const int nkeys = (seq >= 0) ? ctx + p.tail_len : 0;
   const int ntiles = (nkeys + KT - 1) / KT;
@@ -345,12 +346,9 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
 
   // consumer warps that own at least one query row; the others leave after the Q phase
   const int nactive = (M - m0 >= MT) ? 8 : (M - m0 + 15) / 16;
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < STAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], nactive); }
-    mbar_init(q_bar, nactive);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  // ---- Q tile -> shared (swizzled) -> A fragments (consumer warps)
+  // The producer warp sets up the barriers and starts the first K/V copies while the consumer warps fetch Q: the
+  // page-table look-up and the copies overlap the Q round trip.  Named barrier 1 (288 threads): the producer only
+  // arrives, the consumers wait there for the barrier set-up and for each other's part of the Q tile.
   if (warp < 8) {
     for (int id = threadIdx.x; id < MT * CPR; id += 256) {
       int lr = id / CPR, c = id % CPR, mrow = m0 + lr;
@@ -362,11 +360,17 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
     }
     cp_async_commit();
     cp_async_wait<0>();
-  }
-  __syncthreads();
-
-  if (warp == 8) {
+    asm volatile("bar.sync 1, 288;" ::: "memory");
+  } else {
     // ================================================================ producer
+    if (lane == 0) {
+      for (int i = 0; i < STAGES; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], nactive); }
+      mbar_init(q_bar, nactive);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      __threadfence_block();
+    }
+    __syncwarp();
+    asm volatile("bar.arrive 1, 288;" ::: "memory");
     if (lane == 0 && seq >= 0) {
       const int32_t *tbl = p.pm.table + (size_t)seq * p.pm.pages_per_seq;
       const int fallback = tbl[0];                     // keys past the last page are masked; they still need a valid source
@@ -407,9 +411,9 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
   __syncwarp();
   if (lane == 0) mbar_arrive(q_bar);
   // byte offset of 16-byte chunk c of key kr inside a tile: [page][half of hd][key in page][128 B], chunks XOR-swizzled
-  const int psb = ps * ROWB;
+  const int psb = ps * ROWB, psh = __ffs(ps) - 1;      // the page size is a power of two
   auto koff = [&](int kr, int c) -> uint32_t {
-    return (uint32_t)((kr / ps) * psb + (c >> 3) * (ps * 128) + (kr % ps) * 128 + (((c & 7) ^ (kr & 7)) << 4));
+    return (uint32_t)((kr >> psh) * psb + (c >> 3) * (ps * 128) + (kr & (ps - 1)) * 128 + (((c & 7) ^ (kr & 7)) << 4));
   };
   const int tb = ctx;                                   // tail keys follow the context
   (void)tb;
@@ -990,9 +994,9 @@ __global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_consta
       int r = (lane & 7) + ((lane >> 3) & 1) * 8, c = ks * 2 + (lane >> 4);
       ldsm_x4(smem_u32(sQ + swz<ROWB>(r, c)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
     }
-    const int psb = ps * ROWB;
+    const int psb = ps * ROWB, psh = __ffs(ps) - 1;    // the page size is a power of two
     auto koff = [&](int kr, int c) -> uint32_t {
-      return (uint32_t)((kr / ps) * psb + (c >> 3) * (ps * 128) + (kr % ps) * 128 + (((c & 7) ^ (kr & 7)) << 4));
+      return (uint32_t)((kr >> psh) * psb + (c >> 3) * (ps * 128) + (kr & (ps - 1)) * 128 + (((c & 7) ^ (kr & 7)) << 4));
     };
     const int mA = lane >> 2, mB = mA + 8;
     uint64_t loA = 0, hiA = 0, loB = 0, hiB = 0;
@@ -1124,10 +1128,19 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const float *__restri
   if (rh >= nrh) return;
   const float sc = rsqrtf((float)HD) * 1.4426950408889634f;
   float m = -INFINITY, ls = 0.0f;                           // lane s holds split s (nsplit <= 32)
-  if (lane < nsplit) {
-    float2 ml = *(const float2 *)(part_ml + ((size_t)lane * nrh + rh) * 2);
-    m = ml.x; ls = ml.y;
-  }
+  float2 ml = make_float2(-INFINITY, 0.0f);
+  if (lane < nsplit) ml = *(const float2 *)(part_ml + ((size_t)lane * nrh + rh) * 2);
+  constexpr int NB = 12;                                    // partial rows in flight per lane
+  // the first NB partial rows are requested together with the statistics: one round trip instead of two
+  float v[NB][DPL];
+#pragma unroll
+  for (int s = 0; s < NB; s++)
+    if (s < nsplit) {
+      const float *src = part_o + ((size_t)s * nrh + rh) * HD + lane * DPL;
+#pragma unroll
+      for (int e = 0; e < DPL; e++) v[s][e] = src[e];
+    }
+  m = ml.x; ls = ml.y;
   float M = m;
   for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
   const float w = (m == -INFINITY) ? 0.0f : exp2f((m - M) * sc);
@@ -1136,17 +1149,18 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const float *__restri
   float acc[DPL];
 #pragma unroll
   for (int e = 0; e < DPL; e++) acc[e] = 0.0f;
-  for (int s0 = 0; s0 < nsplit; s0 += 8) {
-    float v[8][DPL];
+  for (int s0 = 0; s0 < nsplit; s0 += NB) {
+    if (s0 > 0) {
 #pragma unroll
-    for (int s = 0; s < 8; s++)
-      if (s0 + s < nsplit) {
-        const float *src = part_o + ((size_t)(s0 + s) * nrh + rh) * HD + lane * DPL;
+      for (int s = 0; s < NB; s++)
+        if (s0 + s < nsplit) {
+          const float *src = part_o + ((size_t)(s0 + s) * nrh + rh) * HD + lane * DPL;
 #pragma unroll
-        for (int e = 0; e < DPL; e++) v[s][e] = src[e];
-      }
+          for (int e = 0; e < DPL; e++) v[s][e] = src[e];
+        }
+    }
 #pragma unroll
-    for (int s = 0; s < 8; s++) {
+    for (int s = 0; s < NB; s++) {
       const float ws = __shfl_sync(0xffffffffu, w, (s0 + s) & 31);
       if (s0 + s < nsplit) {
 #pragma unroll
