@@ -284,7 +284,15 @@ int launch_topk2(const float *logits, const int32_t *src_row, int rows, int n, i
   float *psum = pmax + (size_t)rows * nch;
   float *cval = psum + (size_t)rows * nch;
   int32_t *cidx = (int32_t *)(cval + (size_t)rows * nch * K);
-  launch_k(topk_partial_kernel, dim3(nch, rows), dim3(256), 0, s, logits, src_row, n, K, nch, pmax, psum, cval, cidx);
+  {
+    // Launched without the programmatic-dependent-launch attribute: pre-launched under the LM-head GEMM, the
+    // rows x nch small CTAs become resident wherever that kernel leaves room, packed onto a few SMs instead of spread
+    // over all of them, and the pair ran 8 us slower per draft pass (measured on the 8B shapes).
+    const bool pdl = tl_pdl;
+    tl_pdl = false;
+    launch_k(topk_partial_kernel, dim3(nch, rows), dim3(256), 0, s, logits, src_row, n, K, nch, pmax, psum, cval, cidx);
+    tl_pdl = pdl;
+  }
   size_t smem = (size_t)nch * K * 8 + (size_t)nch * 8;
   static size_t configured = 0;
   if (smem > 48 * 1024 && smem > configured) {
