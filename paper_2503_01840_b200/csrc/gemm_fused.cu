@@ -106,11 +106,18 @@ __device__ __forceinline__ float4 sum_peers4(uint32_t local_addr, int s0, int n)
   return acc;
 }
 
-template <int NT, int EPI>
+// PAIR (EPI_SWIGLU only): the CTA streams the gate tile AND the up tile of its 128 features for its K slice, both
+// MMAs of a k-block share one activation tile (half the activation fill traffic of the form in which gate and up are
+// separate cluster members), the two accumulators sit side by side in tensor memory, and the cluster holds only the
+// Sk K slices.
+template <int NT, int EPI, bool PAIR = false>
 __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__ FusedParams p) {
+  static_assert(!PAIR || EPI == EPI_SWIGLU, "two weight tiles per CTA exist for the gate/up epilogue only");
+  constexpr int A_TILES = PAIR ? 2 : 1;
   constexpr int B_BYTES = NT * TILE_K * 2;
-  constexpr int STAGE = A_BYTES + B_BYTES;
-  constexpr int TMEM_COLS = (NT < 32) ? 32 : NT;
+  constexpr int STAGE = A_TILES * A_BYTES + B_BYTES;
+  constexpr int TMEM_COLS = (A_TILES * NT < 32) ? 32 : A_TILES * NT;
+  static_assert(TMEM_COLS <= 512, "accumulators must fit the tensor memory");
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char *tiles = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -126,12 +133,12 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int stages = p.stages, S = p.S, Sk = p.Sk;
   const int slice = (S > 1) ? (int)cluster_rank() : 0;        // rank in the cluster
-  const int ksl = (EPI == EPI_SWIGLU) ? slice % Sk : slice;   // K slice
+  const int ksl = (EPI == EPI_SWIGLU && !PAIR) ? slice % Sk : slice;   // K slice
   const int kb0 = (int)(((long long)ksl * p.KB) / Sk), kb1 = (int)(((long long)(ksl + 1) * p.KB) / Sk);
   const int nkb = kb1 - kb0;
   int mi = 0, tm = blockIdx.x;                   // weight index and tile within that weight
   if (EPI == EPI_SWIGLU) {
-    mi = slice / Sk;                             // ranks [0,Sk) stream the gate tile, [Sk,2Sk) the up tile
+    mi = PAIR ? 0 : slice / Sk;                  // ranks [0,Sk) stream the gate tile, [Sk,2Sk) the up tile
   } else {
     if (tm >= p.tiles1) { mi = 2; tm -= p.tiles1; }
     else if (tm >= p.tiles0) { mi = 1; tm -= p.tiles0; }
@@ -163,9 +170,10 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       unsigned char *a = tiles + i * STAGE;
       mbar_expect_tx(&full[i], STAGE);
       tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[i], pol);
+      if (PAIR) tma_load_2d_hint(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[i], pol);
     }
     pdl_wait();
-    for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
+    for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + A_TILES * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
     for (int i = npre; i < nkb; i++) {
       int st = i % stages;
       if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
@@ -173,7 +181,8 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       unsigned char *a = tiles + st * STAGE;
       mbar_expect_tx(&full[st], STAGE);
       tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
-      tma_load_2d(a + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[st]);
+      if (PAIR) tma_load_2d_hint(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
+      tma_load_2d(a + A_TILES * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[st]);
     }
     // all of this CTA's loads are issued: pull the first weights of the launches that follow into L2, so that
     // the memory system stays busy across this kernel's epilogue and the next kernel's start-up
@@ -199,11 +208,12 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
         if (!mbar_wait(&full[st], (i / stages) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 201, blockIdx.x, i); break; }
         if (*abort_flag) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        uint32_t a = smem_u32(tiles + st * STAGE), b = a + A_BYTES;
+        uint32_t a = smem_u32(tiles + st * STAGE), b = a + A_TILES * A_BYTES;
 #pragma unroll
         for (int j = 0; j < TILE_K / UMMA_K; j++) {
           uint64_t db = umma_desc_sw128(b + j * UMMA_K * 2);
           umma_bf16(tmem_base, umma_desc_sw128(a + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
+          if (PAIR) umma_bf16(tmem_base + NT, umma_desc_sw128(a + A_BYTES + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
         }
         umma_commit(&empty[st]);      // frees the stage once these MMAs have read it
       }
@@ -237,7 +247,8 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
   // read it completed) and is reused: red = this CTA's accumulator, sumb = this CTA's rows after the cluster sum.
   const int CH = (NT <= CHUNK || EPI == EPI_ARGMAX) ? CHUNK : p.chunk;   // a constant for the narrow tiles
   float *red = (float *)tiles;                       // [CH][128]
-  float *sumb = red + CH * TILE_M;                   // [rows of this CTA][128] (EPI_SWIGLU: gate rows, then up rows at CH/2)
+  float *red_u = red + CH * TILE_M;                  // PAIR: the up accumulator, [CH][128]
+  float *sumb = red + A_TILES * CH * TILE_M;         // [rows of this CTA][128] (EPI_SWIGLU: gate rows, then up rows at CH/2)
   const int f = threadIdx.x;
   const int o = tm * TILE_M + f;                     // output feature within weight mi
   for (int c0 = 0; c0 < p.rows; c0 += CH) {
@@ -250,6 +261,11 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
         tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + cc), v);
 #pragma unroll
         for (int j = 0; j < 16; j++) red[(cc + j) * TILE_M + f] = __uint_as_float(v[j]);
+        if (PAIR) {
+          tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(NT + c0 + cc), v);
+#pragma unroll
+          for (int j = 0; j < 16; j++) red_u[(cc + j) * TILE_M + f] = __uint_as_float(v[j]);
+        }
       }
     }
     if (S > 1) cluster_sync_all(); else __syncthreads();
@@ -259,16 +275,21 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
     // ---- phase A (clusters): this CTA's rows, summed over the K slices, land in its own sumb.  Each thread
     // takes (row, 4 features) items and keeps all its remote loads in flight before adding them up.
     const float *src = red + r0 * TILE_M;              // S == 1: the accumulator dump is the sum
+    const float *src_u = red_u + r0 * TILE_M;          // EPI_SWIGLU: the up values of the same rows
     if (S > 1) {
       const int nitems = (r1 - r0) * 32;
       for (int item = threadIdx.x; item < nitems; item += 128) {
         const int i = item >> 5, qd = item & 31;
         const uint32_t la = smem_u32(&red[(r0 + i) * TILE_M + qd * 4]);
         *(float4 *)&sumb[i * TILE_M + qd * 4] = sum_peers4(la, 0, Sk);
-        if (EPI == EPI_SWIGLU) *(float4 *)&sumb[(CH / 2 + i) * TILE_M + qd * 4] = sum_peers4(la, Sk, Sk);
+        if (EPI == EPI_SWIGLU) {
+          if (PAIR) *(float4 *)&sumb[(CH / 2 + i) * TILE_M + qd * 4] = sum_peers4(smem_u32(&red_u[(r0 + i) * TILE_M + qd * 4]), 0, Sk);
+          else *(float4 *)&sumb[(CH / 2 + i) * TILE_M + qd * 4] = sum_peers4(la, Sk, Sk);
+        }
       }
       __syncthreads();
       src = sumb;
+      src_u = sumb + (CH / 2) * TILE_M;
       // this CTA has everything it needs from its peers: announce it now and wait only at the end of the round, so
       // that the per-feature epilogue below runs while the slower members are still summing
       asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -369,7 +390,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       for (int r = r0; r < r1; r++) {
         const int row = c0 + r;
         const float sc = inv_s[row];
-        const float g = src[(r - r0) * TILE_M + f] * sc, u = src[(CH / 2 + r - r0) * TILE_M + f] * sc;
+        const float g = src[(r - r0) * TILE_M + f] * sc, u = src_u[(r - r0) * TILE_M + f] * sc;
         if (good && o < p.O[0]) p.act[(size_t)row * p.O[0] + o] = __float2bfloat16_rn((g / (1.0f + expf(-g))) * u);
       }
     } else {   // EPI_ARGMAX
@@ -552,12 +573,13 @@ constexpr int NUM_SMS = 148;
 constexpr int SMEM_ONE = 200 * 1024;      // ring budget with one CTA per SM
 constexpr int SMEM_TWO = 104 * 1024;      // ring budget that lets two CTAs share an SM
 
-struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB, chunk; };
+struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB, chunk; bool pair; };
 
 // K slices per feature tile.  An SM streams at a capped rate whether one or two CTAs feed it, so the time
 // of a launch goes with (CTAs on the busiest SM) x (k-blocks per CTA + a fixed cost per CTA); two CTAs per SM
 // are needed to hide one CTA's MMA and epilogue time behind the other's loads.
 int g_target_ctas = 222;   // measured best on the 8B shapes (1.5 CTAs per SM)
+bool g_swiglu_pair = true;
 constexpr int MAX_CLUSTER = 8;    // portable cluster sizes only: size 9 (non-portable) measured 20 % slower per step
 
 // force_two: plan a wide tile (whose full ring takes the SM) as two CTAs per SM with two-stage rings
@@ -566,10 +588,12 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false) {
   pl.nt = pick_nt(a.rows);
   pl.KB = (a.I + TILE_K - 1) / TILE_K;
   pl.tiles = fused_gemm_tiles(epi, a);
-  const int stage = A_BYTES + pl.nt * TILE_K * 2;
-  const int wmul = epi == EPI_SWIGLU ? 2 : 1;          // cluster members per K slice
+  // gate/up below 256 rows: gate and up tile in ONE CTA (256 rows: the pair kernel without K split)
+  pl.pair = epi == EPI_SWIGLU && pl.nt <= 128 && g_swiglu_pair;
+  const int stage = (pl.pair ? 2 : 1) * A_BYTES + pl.nt * TILE_K * 2;
+  const int wmul = (epi == EPI_SWIGLU && !pl.pair) ? 2 : 1;   // cluster members per K slice
   const int smax = MAX_CLUSTER / wmul;
-  const bool wide = SMEM_TWO / stage < 3;              // 256-row tiles: the ring of one CTA takes the SM
+  const bool wide = SMEM_TWO / stage < (pl.pair ? 2 : 3);     // 256-row tiles: the ring of one CTA takes the SM
   const bool one_per_sm = wide && !force_two;
   const int target = one_per_sm ? NUM_SMS : g_target_ctas;   // one wave
   int Sk = 1;
@@ -594,7 +618,7 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false) {
   auto epi_bytes = [&](int ch) {
     const int mine = pl.S > 1 ? (ch + pl.S - 1) / pl.S : 0;
     const int sum_rows = pl.S > 1 ? (epi == EPI_SWIGLU ? ch / 2 + mine : mine) : 0;
-    return (ch + sum_rows) * TILE_M * 4;
+    return ((pl.pair ? 2 : 1) * ch + sum_rows) * TILE_M * 4;
   };
   pl.chunk = CHUNK;
   if (epi != EPI_ARGMAX)
@@ -605,16 +629,16 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false) {
   return pl;
 }
 
-template <int NT, int EPI>
+template <int NT, int EPI, bool PAIR = false>
 int launch_inst(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) {
   static int configured = 0;
   if (pl.smem > configured) {
-    if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem) != cudaSuccess) return -6;
+    if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem) != cudaSuccess) return -6;
     configured = pl.smem;
   }
   static bool nonportable = false;
   if (pl.S > 8 && !nonportable) {
-    if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return -6;
+    if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI, PAIR>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return -6;
     nonportable = true;
   }
   if (!launch_allowed()) return 0;
@@ -637,7 +661,7 @@ int launch_inst(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) 
   }
   cfg.attrs = at;
   cfg.numAttrs = na;
-  return cudaLaunchKernelEx(&cfg, gemm_fused_kernel<NT, EPI>, p) == cudaSuccess ? 0 : -6;
+  return cudaLaunchKernelEx(&cfg, gemm_fused_kernel<NT, EPI, PAIR>, p) == cudaSuccess ? 0 : -6;
 }
 
 // clusters of the plan's shape that can be resident at once (0: unknown)
@@ -678,6 +702,13 @@ int launch_epi(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) {
     case 64: return launch_inst<64, EPI>(p, pl, pdl, s);
     case 128: return launch_inst<128, EPI>(p, pl, pdl, s);
     default: return launch_inst<256, EPI>(p, pl, pdl, s);
+  }
+}
+int launch_swiglu_pair(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) {
+  switch (pl.nt) {
+    case 16: return launch_inst<16, EPI_SWIGLU, true>(p, pl, pdl, s);
+    case 64: return launch_inst<64, EPI_SWIGLU, true>(p, pl, pdl, s);
+    default: return launch_inst<128, EPI_SWIGLU, true>(p, pl, pdl, s);
   }
 }
 
@@ -772,7 +803,7 @@ int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStr
     case EPI_F32: return launch_epi<EPI_F32>(p, pl, a.pdl, s);
     case EPI_RESID: return launch_epi<EPI_RESID>(p, pl, a.pdl, s);
     case EPI_QKV: return launch_epi<EPI_QKV>(p, pl, a.pdl, s);
-    case EPI_SWIGLU: return launch_epi<EPI_SWIGLU>(p, pl, a.pdl, s);
+    case EPI_SWIGLU: return pl.pair ? launch_swiglu_pair(p, pl, a.pdl, s) : launch_epi<EPI_SWIGLU>(p, pl, a.pdl, s);
     default: return launch_epi<EPI_ARGMAX>(p, pl, a.pdl, s);
   }
 }
