@@ -57,11 +57,12 @@ def test_gemm_cluster_split_k_vs_oracle(rows, O, I, split, stages):
 
 @pytest.mark.parametrize("rows,F,I", [(1, 768, 512), (7, 896, 704), (10, 1000, 1024), (16, 1024, 520), (33, 2048, 4096),
                                       (60, 14336, 4096), (64, 1408, 576), (5, 256, 4096), (100, 1024, 512), (130, 1000, 520),
-                                      (200, 1408, 576), (256, 2048, 1024)])
+                                      (200, 1408, 576), (256, 2048, 1024), (60, 28672, 512), (12, 20480, 256)])
 def test_gemm_swiglu_vs_oracle(rows, F, I):
-    """Gate/up projection with SiLU(gate) * up (up to 128 rows: one cluster per (gate, up) tile pair and its K slices;
-    wider: one CTA per pair with two accumulators): an odd number of k-blocks, a ragged last k-block, F not a multiple
-    of 128, every row-tile width."""
+    """Gate/up projection with SiLU(gate) * up: one CTA holds the gate and the up tile of its 128 features (two
+    accumulators); up to 128 rows the K slices of a tile pair form a cluster, wider tiles run without K split.  An odd
+    number of k-blocks, a ragged last k-block, F not a multiple of 128, every row-tile width, and feature counts large
+    enough that a tile pair gets a single K slice (no cluster)."""
     g = torch.Generator().manual_seed(rows * 1000 + F + I)
     x = (torch.randn(rows, I, generator=g)).to(torch.bfloat16)
     wg = (torch.randn(F, I, generator=g) / I ** 0.5).to(torch.bfloat16)
