@@ -573,25 +573,24 @@ constexpr int NUM_SMS = 148;
 constexpr int SMEM_ONE = 200 * 1024;      // ring budget with one CTA per SM
 constexpr int SMEM_TWO = 104 * 1024;      // ring budget that lets two CTAs share an SM
 
-struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB, chunk; bool pair, bumped; };
+struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB, chunk; bool pair; };
 
 // K slices per feature tile.  An SM streams at a capped rate whether one or two CTAs feed it, so the time
 // of a launch goes with (CTAs on the busiest SM) x (k-blocks per CTA + a fixed cost per CTA); two CTAs per SM
 // are needed to hide one CTA's MMA and epilogue time behind the other's loads.
 int g_target_ctas = 222;   // measured best on the 8B shapes (1.5 CTAs per SM)
-bool g_swiglu_pair = true;
 constexpr int MAX_CLUSTER = 8;    // portable cluster sizes only: size 9 (non-portable) measured 20 % slower per step
 
 // force_two: plan a wide tile (whose full ring takes the SM) as two CTAs per SM with two-stage rings
 constexpr int NUM_GPCS = 8;
 constexpr int MAX_BUMPED_CTAS = 266;   // 90 % of the 296 CTA slots: fuller grids fail to place all their clusters
-Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false, bool no_bump = false) {
+Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false) {
   Plan pl;
   pl.nt = pick_nt(a.rows);
   pl.KB = (a.I + TILE_K - 1) / TILE_K;
   pl.tiles = fused_gemm_tiles(epi, a);
   // gate/up below 256 rows: gate and up tile in ONE CTA (256 rows: the pair kernel without K split)
-  pl.pair = epi == EPI_SWIGLU && pl.nt <= 128 && g_swiglu_pair;
+  pl.pair = epi == EPI_SWIGLU && pl.nt <= 128;
   const int stage = (pl.pair ? 2 : 1) * A_BYTES + pl.nt * TILE_K * 2;
   const int wmul = (epi == EPI_SWIGLU && !pl.pair) ? 2 : 1;   // cluster members per K slice
   const int smax = MAX_CLUSTER / wmul;
@@ -609,8 +608,7 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false, boo
   // of the 70B shapes, 4 slices make 256 CTAs of 112 k-blocks against 192 of 150) and every cluster can still be
   // placed in the first wave: a cluster lives inside one GPC, and with two CTAs per SM a GPC of at least 16 SMs holds 32 / S clusters of S CTAs.  (The
   // occupancy query counts one CTA per SM for these launches, so the bound is spelled out here.)
-  pl.bumped = false;
-  if (!one_per_sm && epi != EPI_ARGMAX && a.split == 0 && !no_bump) {
+  if (!one_per_sm && epi != EPI_ARGMAX && a.split == 0) {
     auto queue = [&](int sk) { return ((pl.tiles * wmul * sk + NUM_SMS - 1) / NUM_SMS) * ((pl.KB + sk - 1) / sk); };
     const int up = Sk + 1, s_up = up * wmul;
     // only up to clusters of 4: with 7 -> 8 slices on the 8B shapes the longer reduction and the fuller grid (less
@@ -618,7 +616,6 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false, boo
     if (s_up <= 4 && up <= smax && up <= pl.KB / 4 && pl.tiles * s_up <= MAX_BUMPED_CTAS && pl.tiles <= NUM_GPCS * (32 / s_up) &&
         queue(up) < queue(Sk)) {
       Sk = up;
-      pl.bumped = true;
     }
   }
   if (a.split > 0) Sk = std::max(1, std::min(std::min(a.split, smax), pl.KB));
