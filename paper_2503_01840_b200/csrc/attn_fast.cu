@@ -1178,7 +1178,7 @@ int g_attn_target_ctas = 148;
 
 int pick_splits(int seqs, int G, int mtiles, int max_ctx_tiles) {
   int base = seqs * G * mtiles;
-  int want = (g_attn_target_ctas + base / 2) / base;                // the kernels run one CTA per SM (register-bound): aim at one wave
+  int want = g_attn_target_ctas / base;                             // the kernels run one CTA per SM (register-bound): never more CTAs than one wave
   if (want < 1) want = 1;
   int s = want < max_ctx_tiles ? want : max_ctx_tiles;
   if (s > MAX_SPLITS) s = MAX_SPLITS;
