@@ -731,6 +731,35 @@ int orc_step_sampled(orc_ctx *c, float temperature, const float *u, int32_t *out
   return step_impl(c, out_ids, count, temperature, u);
 }
 
+/* Step 5 (Section 2.2, tree attention) on a caller-given tree: node i carries tok[i], sits at RoPE position
+ * n_ctx + depth[i], and attends the committed positions [0, n_ctx) plus the nodes j with bit j of mask[i].  Only the
+ * per-step tail scratch is written, the committed caches are read; n_ctx may be smaller than the committed length
+ * (the state before the last step). */
+int orc_verify_tree(orc_ctx *c, int32_t n_ctx, int32_t nn, const int32_t *tok, const int32_t *depth, const uint64_t *mask,
+                    float *logits, float *hidden, float *taps) {
+  const orc_cfg *g = &c->cfg;
+  int N = g->tree_nodes;
+  if (n_ctx < 0 || n_ctx > c->n || nn < 1 || nn > N || n_ctx + N > g->max_ctx) return -1;
+  for (int i = 0; i < nn; i++)
+    if (tok[i] < 0 || tok[i] >= g->vocab || depth[i] < 0 || !((mask[i] >> i) & 1ull) || (i + 1 < 64 && (mask[i] >> (i + 1)))) return -1;
+  int *pos = (int *)xcalloc((size_t)nn, sizeof(int)), *nc = (int *)xcalloc((size_t)nn, sizeof(int));
+  int *ts = (int *)xcalloc((size_t)nn, sizeof(int)), *ne = (int *)xcalloc((size_t)nn, sizeof(int));
+  int *ex = (int *)xcalloc((size_t)nn * ORC_MAX_NODES, sizeof(int));
+  for (int i = 0; i < nn; i++) {
+    pos[i] = n_ctx + depth[i]; nc[i] = n_ctx; ts[i] = i;
+    int len = 0;
+    for (int j = 0; j <= i; j++) if ((mask[i] >> j) & 1ull) ex[(size_t)i * ORC_MAX_NODES + len++] = j;
+    ne[i] = len;
+  }
+  attn_spec sp; memset(&sp, 0, sizeof sp);
+  sp.tail_slot = ts; sp.n_cache = nc; sp.extra = ex; sp.n_extra = ne; sp.extra_stride = ORC_MAX_NODES;
+  float *tp = taps ? taps : (float *)xcalloc((size_t)nn * 3 * g->hidden, 4);
+  target_forward(c, nn, tok, pos, sp, N, tp, hidden, 0, logits);
+  if (!taps) free(tp);
+  free(pos); free(nc); free(ts); free(ne); free(ex);
+  return 0;
+}
+
 const void *orc_get(const orc_ctx *c, int32_t what, int64_t *count) {
   const orc_cfg *g = &c->cfg;
   int64_t cn = 0; const void *p = NULL;

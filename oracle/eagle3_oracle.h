@@ -75,6 +75,14 @@ int orc_greedy(orc_ctx *, int32_t gen, int32_t *out_ids);
 /* same, also reporting the top1 - top2 logit gap of every emitted token */
 int orc_greedy_margins(orc_ctx *, int32_t gen, int32_t *out_ids, float *margins);
 
+/* Step 5 alone (Section 2.2: one target forward over all tree nodes with tree attention) on a tree the caller
+ * gives: node i holds tok[i] at RoPE position n_ctx + depth[i] and attends the committed positions [0, n_ctx) and
+ * the nodes in mask[i] (ancestor-or-self bits, bit i set, none above i).  n_ctx <= committed length.  Outputs:
+ * logits [nn][vocab], hidden [nn][hidden] (either may be NULL), taps [nn][3*hidden] (may be NULL).  Writes only the
+ * step's tail scratch.  Lets a harness check a verify pass on a tree that differs from the oracle's own. */
+int orc_verify_tree(orc_ctx *, int32_t n_ctx, int32_t nn, const int32_t *tok, const int32_t *depth, const uint64_t *mask,
+                    float *logits, float *hidden, float *taps);
+
 /* Put the ctx into the state "ids[0..n-1] committed, ids[n] is the root, P pending entries",
  * recomputing whatever the current caches do not already hold (common prefix is kept). */
 int orc_force_state(orc_ctx *, const int32_t *ids, int32_t n, int32_t P);

@@ -64,6 +64,8 @@ def lib():
         L.orc_greedy.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
         L.orc_greedy_margins.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.orc_force_state.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32]
+        L.orc_verify_tree.restype = C.c_int
+        L.orc_verify_tree.argtypes = [C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 6
         L.orc_n.argtypes = [C.c_void_p]
         L.orc_pending.argtypes = [C.c_void_p]
         L.orc_ids.argtypes = [C.c_void_p]
@@ -316,6 +318,17 @@ class Oracle:
         assert ids.size >= n + 1
         if lib().orc_force_state(self.h, _p(ids), n, P):
             raise RuntimeError("orc_force_state failed")
+
+    def verify_tree(self, n_ctx: int, tok, depth, mask):
+        """The verify pass (step 5) on a given tree over the committed prefix [0, n_ctx): returns (logits [nn][V],
+        hidden [nn][k], taps [nn][3k])."""
+        tok = _np(tok, np.int32); depth = _np(depth, np.int32); mask = _np(mask, np.uint64)
+        nn, k, V = tok.size, self.cfg.hidden, self.cfg.vocab
+        logits = np.empty((nn, V), np.float32); hidden = np.empty((nn, k), np.float32); taps = np.empty((nn, 3 * k), np.float32)
+        rc = lib().orc_verify_tree(self.h, n_ctx, nn, _p(tok), _p(depth), _p(mask), _p(logits), _p(hidden), _p(taps))
+        if rc:
+            raise RuntimeError("orc_verify_tree rejected the tree")
+        return logits, hidden, taps
 
     @property
     def n(self) -> int:

@@ -1236,11 +1236,8 @@ template <int HD>
 int launch_tma_small(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorMap *mv, int32_t *status, cudaStream_t s) {
   constexpr int STAGES = HD == 128 ? 3 : 4;
   const int smem = STAGES * 2 * KT * HD * 2 + 256 + 16 * HD * 2;   // ring (reused by the final merge) + barriers + Q tile
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(attn_tma_small_kernel<HD, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -1;
-    configured = true;
-  }
+  static SmemLimit limit;
+  if (!limit.ensure(attn_tma_small_kernel<HD, STAGES>, (int)smem)) return -1;
   launch_k(attn_tma_small_kernel<HD, STAGES>, grid, dim3(160), (size_t)smem, s, *mk, *mv, p, status);
   return 0;
 }
@@ -1250,11 +1247,8 @@ constexpr int UM_MIN_TILES = 3; // below that the pass is launch- and latency-bo
 thread_local int tl_attn_umma = -1;   // per-call override (-1: none)
 
 int launch_umma(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorMap *mv, int32_t *status, cudaStream_t s) {
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, UM_SMEM) != cudaSuccess) return -1;
-    configured = true;
-  }
+  static SmemLimit limit;
+  if (!limit.ensure(attn_umma_kernel, (int)UM_SMEM)) return -1;
   launch_k(attn_umma_kernel, grid, dim3(UM_THREADS), (size_t)UM_SMEM, s, *mk, *mv, p, status);
   return 0;
 }
@@ -1264,11 +1258,8 @@ int launch_tma(AttnParams &p, dim3 grid, const CUtensorMap *mk, const CUtensorMa
   if (p.rps * (p.H / p.G) <= 16) return launch_tma_small<HD>(p, grid, mk, mv, status, s);
   constexpr int STAGES = HD == 128 ? 3 : 4;
   const int smem = STAGES * 2 * KT * HD * 2 + 256;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(attn_tma_kernel<HD, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -1;
-    configured = true;
-  }
+  static SmemLimit limit;
+  if (!limit.ensure(attn_tma_kernel<HD, STAGES>, (int)smem)) return -1;
   launch_k(attn_tma_kernel<HD, STAGES>, grid, dim3(288), (size_t)smem, s, *mk, *mv, p, status);
   return 0;
 }
@@ -1313,13 +1304,13 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
   }
   size_t smem = (size_t)4 * KT * hd * 2;
   if (smem < (size_t)MT * hd * 2) smem = (size_t)MT * hd * 2;
-  static bool attr[2] = {false, false};
+  static SmemLimit limit[2];
   if (hd == 128) {
-    if (!attr[1]) { cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[1] = true; }
+    if (!limit[1].ensure(attn_mma_kernel<128>, (int)smem)) return -1;
     launch_k(attn_mma_kernel<128>, grid, dim3(256), smem, s, p);
     if (nsplit > 1) launch_k(attn_combine_kernel<128>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
   } else {
-    if (!attr[0]) { cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr[0] = true; }
+    if (!limit[0].ensure(attn_mma_kernel<64>, (int)smem)) return -1;
     launch_k(attn_mma_kernel<64>, grid, dim3(256), smem, s, p);
     if (nsplit > 1) launch_k(attn_combine_kernel<64>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
   }

@@ -53,6 +53,20 @@ inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
+// Kernel function attributes belong to one device: remembers, per device ordinal, the largest dynamic
+// shared-memory size a kernel has been configured with, and raises the limit on the current device when needed.
+struct SmemLimit {
+  int have[64] = {};
+  template <typename F> bool ensure(F kern, int smem) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (dev >= 0 && dev < 64 && smem <= have[dev]) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+    if (dev >= 0 && dev < 64) have[dev] = smem;
+    return true;
+  }
+};
+
 // Per-row description of one forward pass (draft extend, draft tree pass, target verify).  A row
 // attends cache positions [0, ctx) unmasked, then "tail" positions tail_base + t for every set bit t
 // of (mask_lo, mask_hi); it writes its own K/V at cache position kvpos and is rotated by pos.

@@ -43,6 +43,10 @@ template void launch_embed<bf16>(const bf16 *, const int32_t *, float *, int, in
 __global__ void embed_norm_kernel(const bf16 *__restrict__ embed, const int32_t *__restrict__ tok,
                                   const bf16 *__restrict__ gain, float *__restrict__ x, bf16 *__restrict__ hb,
                                   float *__restrict__ ssq, int k, int ssq_ld) {
+  // The wait also orders this kernel's successors after its predecessor: the first QKV GEMM waits only for this
+  // kernel and reads the RoPE table the kernel before it wrote.
+  pdl_wait();
+  pdl_trigger();
   __shared__ float sh[4];
   int r = blockIdx.x, tile = blockIdx.y, o = tile * 128 + threadIdx.x;
   float v = 0.0f;

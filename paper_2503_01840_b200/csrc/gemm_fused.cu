@@ -646,16 +646,9 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false) {
 
 template <int NT, int EPI, bool PAIR = false>
 int launch_inst(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) {
-  static int configured = 0;
-  if (pl.smem > configured) {
-    if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem) != cudaSuccess) return -6;
-    configured = pl.smem;
-  }
-  static bool nonportable = false;
-  if (pl.S > 8 && !nonportable) {
-    if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI, PAIR>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return -6;
-    nonportable = true;
-  }
+  static SmemLimit limit;
+  if (!limit.ensure(gemm_fused_kernel<NT, EPI, PAIR>, pl.smem)) return -6;
+  if (pl.S > 8) return -1;   // portable cluster sizes only
   if (!launch_allowed()) return 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(pl.tiles, pl.S, 1);
@@ -796,11 +789,8 @@ int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStr
     p.S = 1; p.Sk = 1;
     p.ctrl_off = (p.stages * STAGE2 + 1023) & ~1023;
     const int smem = p.ctrl_off + 512 + 256 * 4 + 1024;
-    static int configured = 0;
-    if (smem > configured) {
-      if (cudaFuncSetAttribute(gemm_swiglu_pair_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -6;
-      configured = smem;
-    }
+    static SmemLimit limit;
+    if (!limit.ensure(gemm_swiglu_pair_kernel<256>, smem)) return -6;
     if (!launch_allowed()) return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.tiles0, 1, 1);

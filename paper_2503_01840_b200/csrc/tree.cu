@@ -294,11 +294,8 @@ int launch_topk2(const float *logits, const int32_t *src_row, int rows, int n, i
     tl_pdl = pdl;
   }
   size_t smem = (size_t)nch * K * 8 + (size_t)nch * 8;
-  static size_t configured = 0;
-  if (smem > 48 * 1024 && smem > configured) {
-    cudaFuncSetAttribute(topk_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    configured = smem;
-  }
+  static SmemLimit limit;
+  if (smem > 48 * 1024) limit.ensure(topk_merge_kernel, (int)smem);
   launch_k(topk_merge_kernel, dim3(rows), dim3(256), smem, s, src_row, K, nch, pmax, psum, cval, cidx, idx, lp);
   return 2;
 }
@@ -793,11 +790,8 @@ __global__ void __launch_bounds__(ACC_THREADS) accept_sampled_kernel(SeqState st
 }
 void launch_accept_sampled(SeqState st, TreeBufs tb, const float *logits, int V, const float *u, int B, int rows_per_seq, cudaStream_t s) {
   const size_t smem = (size_t)((V + ACC_THREADS / 32 - 1) / (ACC_THREADS / 32)) * sizeof(float);
-  static size_t configured = 0;
-  if (smem > 40 * 1024 && smem > configured) {
-    cudaFuncSetAttribute(accept_sampled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    configured = smem;
-  }
+  static SmemLimit limit;
+  if (smem > 40 * 1024) limit.ensure(accept_sampled_kernel, (int)smem);
   launch_k(accept_sampled_kernel, dim3(B), dim3(ACC_THREADS), smem, s, st, tb, logits, V, u, rows_per_seq);
 }
 

@@ -11,13 +11,15 @@ import pyoracle as po
 from paper_2503_01840_b200 import binding as sb
 from paper_2503_01840_b200 import synth
 
-MARGIN = 1e-2
+MARGIN = 1e-2          # the stated rule: an integer decision whose oracle margin exceeds this must be bit-exact
 
 
 def decision_margin(tol):
-    """Oracle margin above which an integer decision of the CUDA path must be bit-exact.  The stated rule is 1e-2; it
-    presumes float errors well below that.  The bf16 bound on logits is 2e-2 per value, and two competing logits can
-    each be off by it, so for bf16 models a decision is only forced when the margin exceeds twice the tolerance."""
+    """Oracle margin above which an integer decision of the CUDA path is REQUIRED to be bit-exact.  The stated rule
+    (1e-2) presumes float errors well below it.  The bf16 bound on a logit is 2e-2, and two competing logits may each be
+    off by it, so for bf16 models the requirement starts at twice the tolerance; decisions whose margin lies in the band
+    (1e-2, 2 tol] are still compared and counted (Stats.band_total / band_diff) so that a run reports how many of them
+    actually differed."""
     return MARGIN if tol < 1e-3 else max(MARGIN, 2.0 * tol)
 
 
@@ -34,8 +36,24 @@ def to_cpu(w):
 
 
 class Stats:
+    """What a trajectory actually compared.  Every test asserts minimums on these, so that a run which diverged early
+    and compared nothing cannot pass."""
+    COUNTERS = ("steps", "tokens", "resyncs",
+                "passes",            # draft passes whose logits and features were compared element by element
+                "topk_forced",       # top-k rows (own margin above the threshold) required to match, order included
+                "topk_set_forced",   # rows whose K-th vs (K+1)-th gap alone is above the threshold: the SET had to match
+                "frontier_forced",   # frontier selections required to match
+                "exact_tree",        # steps whose whole tree (tokens, parents, depths, masks, pool indices) had to match
+                "same_tree",         # steps whose tree did match the oracle's
+                "verify_compared",   # steps whose verify logits / hidden states / taps were compared element by element
+                "accept_checked",    # steps whose accepted path and ids equal the oracle's walk over the same tree and argmax
+                "argmax_forced",     # verify nodes whose argmax had to match
+                "exact_out",         # steps whose accepted path and emitted ids had to match
+                "band_total", "band_diff")   # decisions with oracle margin in (1e-2, threshold]: seen / differed
+
     def __init__(self):
-        self.steps = self.exact_tree = self.same_tree = self.exact_out = self.resyncs = self.tokens = 0
+        for n in self.COUNTERS:
+            setattr(self, n, 0)
         self.max_err = {}
 
     def err(self, name, a, b):
@@ -43,59 +61,97 @@ class Stats:
         self.max_err[name] = max(self.max_err.get(name, 0.0), e)
         return e
 
+    def decide(self, margin, threshold, same, what):
+        """One integer decision with oracle margin `margin`: required to match above `threshold`, counted in the band
+        between the stated 1e-2 and the threshold.  Returns True when it was required."""
+        if margin > threshold:
+            assert same, f"{what} differs although its oracle margin {margin:.4g} exceeds {threshold:.4g}"
+            return True
+        if margin > MARGIN:
+            self.band_total += 1
+            self.band_diff += int(not same)
+        return False
+
     def __repr__(self):
         errs = ", ".join(f"{k}={v:.2e}" for k, v in sorted(self.max_err.items()))
-        return (f"steps={self.steps} exact_tree={self.exact_tree} same_tree={self.same_tree} exact_out={self.exact_out} resyncs={self.resyncs} "
-                f"tokens={self.tokens} | {errs}")
+        return " ".join(f"{n}={getattr(self, n)}" for n in self.COUNTERS) + " | " + errs
 
 
-def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_tol=None, sampled=None):
-    """`orc` has just executed the same step from the same state.  Returns True if outputs were
-    required to be (and were) identical.  sampled = (temperature, u) for a step with stochastic acceptance."""
+def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_tol=None, sampled=None, n_ctx=None):
+    """`orc` has just executed the same step from the same state.  Every integer decision is gated on its OWN oracle
+    margin: a top-k row, a frontier selection, the final cut of the candidate pool, each verify node's argmax and the
+    accepted path.  Returns True if the outputs were required to be (and were) identical.
+    sampled = (temperature, u) for a step with stochastic acceptance.  n_ctx = committed length before the step: when
+    the trees differ (a low-margin draft decision), the oracle runs its verify pass on the CUDA path's tree over that
+    prefix, so that the verify floats, the argmax and the acceptance walk are compared in every step."""
     K, D, N, Vd, k, V = cfg.tree_topk, cfg.tree_depth, cfg.tree_nodes, cfg.draft_vocab, cfg.hidden, cfg.vocab
     tap_tol = tol if tap_tol is None else tap_tol
-    MARGIN = decision_margin(tol)
+    thr = decision_margin(tol)
     o_front = orc.get(po.FRONTIER).reshape(D, K)
     g_front = dec.debug(sb.DBG_FRONTIER, seq).reshape(D, K)
     tk_m = orc.get(po.TOPK_MARGIN).reshape(D, K)
     fr_m = orc.get(po.FRONTIER_MARGIN)
     rr_m = float(orc.get(po.RERANK_MARGIN)[0])
     capture = check_floats
+    o_dl = orc.get(po.DRAFT_LOGITS).reshape(D, K, Vd)
     if capture:
         g_dl = dec.debug(sb.DBG_DRAFT_LOGITS, seq).reshape(D, K, Vd)
         g_da = dec.debug(sb.DBG_DRAFT_A, seq).reshape(D, K, k)
-        o_dl = orc.get(po.DRAFT_LOGITS).reshape(D, K, Vd)
         o_da = orc.get(po.DRAFT_A).reshape(D, K, k)
-    # draft passes: comparable while the frontier (and its order) is the same
-    safe = True                                    # every decision so far had margin
     o_ptok, g_ptok = orc.get(po.POOL_TOK), dec.debug(sb.DBG_POOL_TOK, seq)
+    pool_same = True                 # every candidate drafted so far is the same on both sides
+    front_required = True            # the frontier of the next pass has to match (all decisions behind it were required)
     for d in range(D):
         rows = 1 if d == 0 else K
         # same nodes in the same order, carrying the same tokens (a swapped near-tie inside one top-k
         # row keeps the pool indices but exchanges the tokens)
         same_front = d == 0 or (np.array_equal(o_front[d], g_front[d]) and
                                 np.array_equal(o_ptok[o_front[d]], g_ptok[g_front[d]]))
-        if d > 0 and safe:
-            assert same_front, f"frontier of pass {d} differs although all margins > {MARGIN}: {o_front[d]} vs {g_front[d]}"
+        if d > 0 and front_required:
+            assert same_front, f"frontier of pass {d} differs although every decision behind it had margin > {thr}: {o_front[d]} vs {g_front[d]}"
+            st.frontier_forced += 1
         if not same_front:
-            safe = False
+            pool_same = False
             break
         if capture:
             assert st.err("draft_logits", g_dl[d, :rows], o_dl[d, :rows]) <= tol, (d, st.max_err)
             assert st.err("draft_a", g_da[d, :rows], o_da[d, :rows]) <= tol, (d, st.max_err)
-        if tk_m[d, :rows].min() <= MARGIN or (d + 1 < D and d >= 1 and fr_m[d] <= MARGIN):
-            safe = False
-            # later passes may still coincide; keep comparing floats only if frontiers match
-    safe_tree = bool((tk_m[np.isfinite(tk_m)] > MARGIN).all() and (fr_m[np.isfinite(fr_m)] > MARGIN).all() and rr_m > MARGIN)
+            st.passes += 1
+        # the K children of every row of this pass: pool entries base + r K + 1 .. base + r K + K
+        base = 0 if d == 0 else K + (d - 1) * K * K
+        rows_same = True
+        for r in range(rows):
+            lo = base + r * K + 1
+            o_t, g_t = o_ptok[lo:lo + K], g_ptok[lo:lo + K]
+            same = bool(np.array_equal(o_t, g_t))
+            if st.decide(float(tk_m[d, r]), thr, same, f"top-{K} of pass {d} row {r}"):
+                st.topk_forced += 1
+            else:
+                # membership alone: the K-th against the (K+1)-th log-probability of the oracle's row
+                z = o_dl[d, r].astype(np.float64)
+                top = np.sort(z)[::-1][:K + 1]
+                set_margin = float(top[K - 1] - top[K]) if Vd > K else np.inf
+                same_set = set(o_t.tolist()) == set(g_t.tolist())
+                if st.decide(set_margin, thr, same_set, f"top-{K} set of pass {d} row {r}"):
+                    st.topk_set_forced += 1
+            rows_same = rows_same and same
+        pool_same = pool_same and rows_same
+        # the next frontier: level 1 is taken whole, later levels are the K best children of the level
+        if d + 1 < D:
+            front_required = rows_same and (d == 0 or float(fr_m[d]) > thr)
+            if rows_same and d >= 1 and MARGIN < float(fr_m[d]) <= thr:
+                st.band_total += 1
+                st.band_diff += int(not (np.array_equal(o_front[d + 1], g_front[d + 1])))
     ints = {n: (dec.debug(g, seq), orc.get(o)) for n, g, o in (
         ("tok", sb.DBG_TREE_TOK, po.TREE_TOK), ("parent", sb.DBG_TREE_PARENT, po.TREE_PARENT),
         ("depth", sb.DBG_TREE_DEPTH, po.TREE_DEPTH), ("mask", sb.DBG_TREE_MASK, po.TREE_MASK),
         ("poolidx", sb.DBG_TREE_POOLIDX, po.TREE_POOLIDX))}
     same_tree = all(np.array_equal(a, b) for a, b in ints.values())
     st.same_tree += int(same_tree)
-    if safe_tree:
+    # the cut of the pool: required when both sides ranked the same candidates and the oracle's cut has margin
+    if pool_same and st.decide(rr_m, thr, same_tree, "pruned tree"):
         for n, (a, b) in ints.items():
-            assert np.array_equal(a, b), f"tree {n} differs although all margins > {MARGIN}\n{a}\n{b}"
+            assert np.array_equal(a, b), f"tree {n} differs although the pool matches and the cut margin > {thr}\n{a}\n{b}"
         st.exact_tree += 1
     # GPU tree must be a valid tree whatever the margins
     g_par, g_dep, g_mask = ints["parent"][0], ints["depth"][0], ints["mask"][0]
@@ -109,21 +165,38 @@ def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_to
     if sampled is not None and not same_tree and check_floats:
         check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, *sampled, own_inputs=True)
         st.max_err["sampled_own_inputs_checks"] = st.max_err.get("sampled_own_inputs_checks", 0.0) + 1
+    g_tok, g_par = ints["tok"][0], ints["parent"][0]
+    nn = g_tok.size
+    gy = dec.debug(sb.DBG_Y, seq)
     if same_tree:
-        nn = ints["tok"][0].size
         assert st.err("tree_score", dec.debug(sb.DBG_TREE_SCORE, seq), orc.get(po.TREE_SCORE)) <= tol
-        if check_floats:
-            assert st.err("target_logits", dec.debug(sb.DBG_TARGET_LOGITS, seq), orc.get(po.TARGET_LOGITS)) <= tol, st.max_err
-            assert st.err("node_hidden", dec.debug(sb.DBG_NODE_HIDDEN, seq), orc.get(po.NODE_HIDDEN)) <= tol, st.max_err
-            assert st.err("node_taps", dec.debug(sb.DBG_NODE_TAPS, seq), orc.get(po.NODE_TAPS)) <= tap_tol, st.max_err
-        gy, oy, ym = dec.debug(sb.DBG_Y, seq), orc.get(po.Y), orc.get(po.Y_MARGIN)
-        big = ym > MARGIN
-        assert np.array_equal(gy[big], oy[big]), "argmax differs at a node with margin"
-        if sampled is not None:
-            return check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, *sampled)
+        o_logits, o_hidden, o_taps = orc.get(po.TARGET_LOGITS), orc.get(po.NODE_HIDDEN), orc.get(po.NODE_TAPS)
+        oy, ym = orc.get(po.Y), orc.get(po.Y_MARGIN)
+    elif check_floats and n_ctx is not None:
+        # the oracle's verify pass on the CUDA path's (valid) tree
+        o_logits, o_hidden, o_taps = orc.verify_tree(n_ctx, g_tok, g_dep, g_mask)
+        top2 = np.partition(o_logits, -2, axis=1)[:, -2:]
+        oy, ym = np.argmax(o_logits, axis=1), top2[:, 1] - top2[:, 0]
+    else:
+        return False
+    if check_floats:
+        assert st.err("target_logits", dec.debug(sb.DBG_TARGET_LOGITS, seq), np.ravel(o_logits)) <= tol, st.max_err
+        assert st.err("node_hidden", dec.debug(sb.DBG_NODE_HIDDEN, seq), np.ravel(o_hidden)) <= tol, st.max_err
+        assert st.err("node_taps", dec.debug(sb.DBG_NODE_TAPS, seq), np.ravel(o_taps)) <= tap_tol, st.max_err
+        st.verify_compared += 1
+    for i in range(nn):
+        if st.decide(float(ym[i]), thr, gy[i] == oy[i], f"argmax of verify node {i}"):
+            st.argmax_forced += 1
+    if sampled is not None:
+        return check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, *sampled) if same_tree else False
+    # the acceptance walk is integer work: on the CUDA path's own tree and argmax it must equal the oracle's walk
+    cnt, w_path, w_out = po.accept(g_tok, g_par, gy)
+    g_path = dec.debug(sb.DBG_PATH, seq)
+    assert np.array_equal(g_path, w_path) and np.array_equal(np.asarray(gpu_out), w_out), (g_path, w_path, gpu_out, w_out)
+    st.accept_checked += 1
+    if same_tree:
         o_path = orc.get(po.PATH)
-        if big[o_path].all():
-            g_path = dec.debug(sb.DBG_PATH, seq)
+        if (ym[o_path] > thr).all():
             assert np.array_equal(g_path, o_path), (g_path, o_path)
             exact_out = True
     return exact_out
@@ -238,7 +311,7 @@ def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, c
             g_out = outs[b]
             assert 1 <= len(g_out) <= cfg.tree_depth + 1
             exact = compare_step(dec, o, b, cfg, tol, st, g_out, check_floats, tap_tol,
-                                 sampled=(sampling[0], u[b]) if sampling else None)
+                                 sampled=(sampling[0], u[b]) if sampling else None, n_ctx=n_before)
             if exact:
                 assert np.array_equal(g_out, o_out), (g_out, o_out)
                 st.exact_out += 1
@@ -250,6 +323,20 @@ def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, c
             st.tokens += len(g_out)
         st.steps += 1
         assert np.array_equal(dec.lengths(), [o.n for o in orcs])
+    # committed caches: K/V of sampled positions in the first and last target layer and in the draft layer against the
+    # oracle (which is in the CUDA path's committed state after every step)
+    for b in sorted(set([0, B // 2, B - 1])):
+        o = orcs[b]
+        n = o.n
+        for pos in sorted(set([0, n // 2, n - 2, n - 1])):
+            for layer in sorted(set([0, cfg.n_layers - 1])):
+                gk, gv = dec.read_kv(b, layer, pos)
+                ok, ov = o.target_kv(layer, pos)
+                assert st.err("kv_target", gk, ok) <= 4 * tol and st.err("kv_target", gv, ov) <= 4 * tol, (b, pos, layer)
+            if pos < n - o.pending:
+                gk, gv = dec.read_kv(b, -1, pos)
+                ok, ov = o.draft_kv(pos)
+                assert st.err("kv_draft", gk, ok) <= 4 * tol and st.err("kv_draft", gv, ov) <= 4 * tol, (b, pos)
     # losslessness against plain greedy decoding of the oracle, up to the first low-margin token
     for b in range(B if not sampling else 0):
         g = po.Oracle(cfg, tw, dw, max_ctx)

@@ -78,3 +78,43 @@ def test_single_kernel_entry_points_reject_null():
     assert L.spec_gemm_swiglu(None, None, None, None, 1, 128, 8, None) == -2
     assert L.spec_step_sampled(None, 1.0, None, None, None) == -2
     assert L.spec_topk_scratch_bytes(10, 32000, 10) > 0
+
+
+def _kernel_bodies():
+    """(file, kernel name, body text) of every __global__ function of the CUDA sources."""
+    csrc = os.path.join(ROOT, "paper_2503_01840_b200", "csrc")
+    for fn in sorted(os.listdir(csrc)):
+        if not fn.endswith(".cu"):
+            continue
+        s = open(os.path.join(csrc, fn)).read()
+        for m in re.finditer(r"__global__\s+void\s+(?:__launch_bounds__\([^)]*\)\s*)?(\w+)\s*\(", s):
+            i = s.index("{", m.end())
+            depth, j = 0, i
+            while True:
+                depth += {"{": 1, "}": -1}.get(s[j], 0)
+                if depth == 0:
+                    break
+                j += 1
+            yield fn, m.group(1), s[i:j]
+
+
+def test_every_step_kernel_orders_itself_behind_its_predecessor():
+    """Kernels of a step are launched with programmatic dependent launch: a kernel may start before its predecessor
+    has finished, and its successor waits only for IT.  A kernel without griddepcontrol.wait would let its successor
+    overtake the kernel before it (the first QKV GEMM reading a RoPE table that is still being written), so every
+    kernel the scheduler launches with the attribute must wait, and must do so before it touches global memory."""
+    never_pdl = {"gemm_tcgen05_kernel", "reduce_slices_kernel"}      # launched without the attribute
+    seen = 0
+    for fn, name, body in _kernel_bodies():
+        if name in never_pdl:
+            continue
+        seen += 1
+        assert "pdl_wait()" in body, f"{fn}: {name} never calls pdl_wait()"
+        assert "pdl_trigger()" in body, f"{fn}: {name} never calls pdl_trigger()"
+    assert seen >= 25
+    # the elementwise / tree kernels wait first thing: nothing but declarations may precede the wait
+    for fn, name, body in _kernel_bodies():
+        if fn in ("elementwise.cu", "tree.cu", "gemm_ref.cu", "attn_ref.cu") and name not in never_pdl:
+            head = body[: body.index("pdl_wait()")]
+            head = "\n".join(l for l in head.split("\n") if "__shared__" not in l)
+            assert "[" not in head and "->" not in head, f"{fn}: {name} touches memory before pdl_wait()"

@@ -335,6 +335,49 @@ def test_tree_forward_equals_per_path_sequential_bitwise(c1):
         assert np.array_equal(s.taps(n0 + dep[i]), taps[i])          # bit-identical
 
 
+def test_verify_tree_on_a_given_tree_equals_sequential_decoding(c1):
+    """orc_verify_tree (step 5 on a caller-given tree): a hand-built tree whose branches are arbitrary token runs must
+    give, at every node, the logits, hidden state and taps of an ordinary causal run over prompt + that node's path
+    (a fresh prefill, bit for bit), also when the committed state has already moved past n_ctx."""
+    tw, dw, ids = c1
+    o = _mk(C1, tw, dw)
+    o.prefill(ids)
+    n0 = o.n
+    root = int(o.ids[n0])
+    #       0
+    #     / | \
+    #    1  2  3
+    #    |     |\
+    #    4     5 6
+    #    |
+    #    7
+    tok = np.array([root, 11, 22, 33, 44, 55, 66, 77], np.int32)
+    par = [-1, 0, 0, 0, 1, 3, 3, 4]
+    dep = np.array([0, 1, 1, 1, 2, 2, 2, 3], np.int32)
+    mask = np.zeros(8, np.uint64)
+    for i, p_ in enumerate(par):
+        mask[i] = np.uint64((int(mask[p_]) if p_ >= 0 else 0) | (1 << i))
+    base = o.ids[:n0].copy()
+    for advance in (False, True):
+        if advance:
+            o.step()                                      # commits past n0; the call below still verifies at n0
+        lg, hid, taps = o.verify_tree(n0, tok, dep, mask)
+        for i in range(8):
+            chain, v = [], i
+            while v != -1:
+                chain.append(int(tok[v]))
+                v = par[v]
+            chain.reverse()
+            s = _mk(C1, tw, dw)
+            nxt = s.prefill(np.concatenate([base, np.array(chain, np.int32)]))
+            assert nxt == int(np.argmax(lg[i]))
+            assert np.array_equal(s.taps(n0 + dep[i]), taps[i])
+    # rejects masks that are not ancestor-or-self sets below the node
+    bad = mask.copy(); bad[2] = np.uint64(1 << 5 | 1 << 2)
+    with pytest.raises(RuntimeError):
+        o.verify_tree(n0, tok, dep, bad)
+
+
 def test_commit_equals_fresh_prefill(c1):
     tw, dw, ids = c1
     tws, dws, pi, pi2 = synth.make_structured(C1, 0.8, residual_scale=0.05)

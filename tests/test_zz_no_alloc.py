@@ -5,9 +5,11 @@ pre-sized arena, hosts that forbid cudaMalloc after start-up, loops that must no
 implicit synchronisation).  For them the split-KV scratch lives in a device array built into the library.
 This file is collected last on purpose: if it fails, a run that stops at the first failure has already
 run every other test.  It passes alone in a fresh process and after the other tests."""
+import numpy as np
 import pytest
 import torch
 
+import pyoracle as po
 from paper_2503_01840_b200 import binding as sb
 
 pytestmark = pytest.mark.gpu
@@ -44,6 +46,18 @@ def test_static_scratch_attention_matches_the_allocating_entry_point_twice():
         err = (got - want).abs().max().item()
         assert err <= TOL, err
         assert (got[5] == 0).all()                                 # padding rows stay zero
+        # and against the CPU oracle's per-head attention for a few (row, head) pairs
+        kp, vp, perm = c["k_pool"].cpu(), c["v_pool"].cpu(), c["page_table"].cpu()
+        q, lo, seq, rctx = c["q"].cpu(), c["mask_lo"].cpu(), c["row_seq"].cpu(), c["row_ctx"].cpu()
+        H, G, ps = q.shape[1], c["n_kv_heads"], c["page_size"]
+        for r, h in ((0, 0), (7, 3), (12, 5), (23, 7)):
+            s_, n = int(seq[r]), int(rctx[r])
+            pos = list(range(n)) + [n + t for t in range(c["tail_len"]) if (int(lo[r]) >> t) & 1]
+            gk = h // (H // G)
+            K = np.stack([kp[perm[s_, p // ps], gk, p % ps].float().numpy() for p in pos])
+            V = np.stack([vp[perm[s_, p // ps], gk, p % ps].float().numpy() for p in pos])
+            ref = po.attend(q[r, h].float().numpy(), K, V)
+            assert np.abs(got[r, h].cpu().numpy() - ref).max() <= TOL, (r, h)
 
 
 def test_static_scratch_attention_rejects_shapes_beyond_its_capacity():
