@@ -165,24 +165,10 @@ int32_t orc_argmax(const float *v, int32_t n, float *margin) {
 
 /* Pruning at the end of drafting (Section 2.2): keep the M = min(N-1, pool) best-scored candidates,
  * (score desc, pool index asc); nodes are then numbered in pool-index order after the root. */
-int32_t orc_rerank(const float *pscore, const int32_t *pparent, const int32_t *ptok, const int32_t *pdepth,
-                   int32_t pool, int32_t nmax, int32_t root_tok, int32_t *tok, int32_t *parent,
-                   int32_t *depth, uint64_t *mask, int32_t *poolidx, float *score, float *cut_margin) {
-  int M = nmax - 1 < pool ? nmax - 1 : pool;
-  char *sel = (char *)xcalloc((size_t)pool + 1, 1);
-  float last = INFINITY;
-  for (int r = 0; r < M; r++) {
-    int best = -1;
-    for (int i = 1; i <= pool; i++)
-      if (!sel[i] && (best < 0 || pscore[i] > pscore[best])) best = i;
-    sel[best] = 1;
-    last = pscore[best];
-  }
-  if (cut_margin) {
-    float nxt = -INFINITY;
-    for (int i = 1; i <= pool; i++) if (!sel[i] && pscore[i] > nxt) nxt = pscore[i];
-    *cut_margin = (M < pool && M > 0) ? last - nxt : INFINITY;
-  }
+/* numbers the selected candidates in pool-index order after the root and fills the tree arrays */
+static int32_t tree_from_selection(const char *sel, const float *pscore, const int32_t *pparent, const int32_t *ptok,
+                                   const int32_t *pdepth, int32_t pool, int32_t root_tok, int32_t *tok, int32_t *parent,
+                                   int32_t *depth, uint64_t *mask, int32_t *poolidx, float *score) {
   int32_t *node_of = (int32_t *)xcalloc((size_t)pool + 1, sizeof(int32_t));
   int nn = 1;
   tok[0] = root_tok; parent[0] = -1; depth[0] = 0; mask[0] = 1ull; poolidx[0] = 0; score[0] = 0.0f;
@@ -198,8 +184,35 @@ int32_t orc_rerank(const float *pscore, const int32_t *pparent, const int32_t *p
     score[nn] = pscore[i];
     nn++;
   }
-  free(sel);
   free(node_of);
+  return nn;
+}
+
+/* the M best-scored candidates, (score desc, pool index asc); returns the last selected score and the best unselected */
+static void rerank_select(const float *pscore, int32_t pool, int M, char *sel, float *last_out, float *next_out) {
+  float last = INFINITY;
+  for (int r = 0; r < M; r++) {
+    int best = -1;
+    for (int i = 1; i <= pool; i++)
+      if (!sel[i] && (best < 0 || pscore[i] > pscore[best])) best = i;
+    sel[best] = 1;
+    last = pscore[best];
+  }
+  float nxt = -INFINITY;
+  for (int i = 1; i <= pool; i++) if (!sel[i] && pscore[i] > nxt) nxt = pscore[i];
+  *last_out = last; *next_out = nxt;
+}
+
+int32_t orc_rerank(const float *pscore, const int32_t *pparent, const int32_t *ptok, const int32_t *pdepth,
+                   int32_t pool, int32_t nmax, int32_t root_tok, int32_t *tok, int32_t *parent,
+                   int32_t *depth, uint64_t *mask, int32_t *poolidx, float *score, float *cut_margin) {
+  int M = nmax - 1 < pool ? nmax - 1 : pool;
+  char *sel = (char *)xcalloc((size_t)pool + 1, 1);
+  float last, nxt;
+  rerank_select(pscore, pool, M, sel, &last, &nxt);
+  if (cut_margin) *cut_margin = (M < pool && M > 0) ? last - nxt : INFINITY;
+  int nn = tree_from_selection(sel, pscore, pparent, ptok, pdepth, pool, root_tok, tok, parent, depth, mask, poolidx, score);
+  free(sel);
   return nn;
 }
 
@@ -590,8 +603,64 @@ int orc_force_state(orc_ctx *c, const int32_t *ids, int32_t n, int32_t P) {
   return 0;
 }
 
+/* ------------------------------------------------------------------ following another implementation's decisions
+ * A harness that compares a second implementation with this one loses everything after the first near-tie that the
+ * two resolve differently.  In follow mode the step takes the other side's integer decisions (the K children of every
+ * row, every frontier, the pruned set) wherever they are VALID on this oracle's own values: a followed choice of K
+ * items is valid when its order is non-increasing within eps and no item left out beats the worst chosen one by more
+ * than eps.  All values (log-probabilities, scores) stay the oracle's own.  Each decision is also compared with the
+ * oracle's own choice: above `require` of its own margin a difference is recorded as a violation. */
+static void follow_note(orc_follow *fw, int same, float own_margin, int valid) {
+  fw->checked++;
+  if (!valid) { fw->invalid++; return; }
+  if (!same) fw->differs++;
+  if (own_margin > fw->require) { fw->required++; if (!same) fw->required_differs++; }
+  else if (own_margin > fw->band_lo) { fw->band_total++; if (!same) fw->band_differs++; }
+}
+
+/* v[n]: the oracle's values; own[K]: its own choice; cand[K]: the followed choice (indices into v, -1 = unknown).
+ * Returns 1 and overwrites own/own_val with the followed choice when that is valid. */
+static int follow_choice(orc_follow *fw, const float *v, int n, int K, int32_t *own, float *own_val, const int32_t *cand,
+                         float own_margin) {
+  int valid = 1, same = 1;
+  for (int r = 0; r < K && valid; r++) {
+    if (cand[r] < 0 || cand[r] >= n) valid = 0;
+    for (int q = 0; q < r && valid; q++) if (cand[q] == cand[r]) valid = 0;
+  }
+  float worst = INFINITY;
+  for (int r = 0; r < K && valid; r++) {
+    if (r + 1 < K && v[cand[r]] < v[cand[r + 1]] - fw->eps) valid = 0;
+    if (v[cand[r]] < worst) worst = v[cand[r]];
+    if (cand[r] != own[r]) same = 0;
+  }
+  if (valid) {
+    for (int i = 0; i < n && valid; i++) {
+      if (v[i] <= worst + fw->eps) continue;
+      int chosen = 0;
+      for (int r = 0; r < K; r++) if (cand[r] == i) chosen = 1;
+      if (!chosen) valid = 0;
+    }
+  }
+  follow_note(fw, same, own_margin, valid);
+  if (!valid) return 0;
+  for (int r = 0; r < K; r++) { own[r] = cand[r]; own_val[r] = v[cand[r]]; }
+  return 1;
+}
+
+/* draft id of a target token (d2t is strictly increasing), -1 if the draft cannot emit it */
+static int32_t d2t_inverse(const orc_ctx *c, int32_t target_id) {
+  int lo = 0, hi = c->cfg.draft_vocab - 1;
+  while (lo <= hi) {
+    int mid = (lo + hi) / 2;
+    int32_t t = c->dw.d2t[mid];
+    if (t == target_id) return mid;
+    if (t < target_id) lo = mid + 1; else hi = mid - 1;
+  }
+  return -1;
+}
+
 /* ------------------------------------------------------------------ the speculative step */
-static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float temperature, const float *u) {
+static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float temperature, const float *u, orc_follow *fw) {
   const orc_cfg *g = &c->cfg;
   int n = c->n, P = c->n - c->dn, K = g->tree_topk, D = g->tree_depth, N = g->tree_nodes;
   int k = g->hidden, Vd = g->draft_vocab, V = g->vocab, L = g->n_layers, kvd = g->n_kv_heads * g->head_dim;
@@ -602,6 +671,8 @@ static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float tempera
   float *lp = (float *)xcalloc((size_t)Vd, 4);
   int32_t *tid = (int32_t *)xcalloc((size_t)K, 4);
   float *tval = (float *)xcalloc((size_t)K + 1, 4);
+  int32_t *cand = (int32_t *)xcalloc((size_t)K, 4);
+  if (fw) fw->checked = fw->differs = fw->invalid = fw->required = fw->required_differs = fw->band_total = fw->band_differs = 0;
 
   /* 1+2. fuse the pending taps (FC 3k->k) and run the draft layer over the pending entries */
   draft_extend(c, n - P, n, c->g_pending, c->a_store, c->draft_logits);
@@ -614,6 +685,12 @@ static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float tempera
   for (int r = 0; r < K; r++) {
     float gap = tval[r] - tval[r + 1];
     if (gap < c->topk_margin[0]) c->topk_margin[0] = gap;
+  }
+  if (fw) {
+    for (int r = 0; r < K; r++) cand[r] = d2t_inverse(c, fw->pool_tok[1 + r]);
+    follow_choice(fw, lp, Vd, K, tid, tval, cand, c->topk_margin[0]);
+  }
+  for (int r = 0; r < K; r++) {
     c->pool_tok[1 + r] = c->dw.d2t[tid[r]];
     c->pool_parent[1 + r] = 0; c->pool_depth[1 + r] = 1; c->pool_score[1 + r] = tval[r];
   }
@@ -654,6 +731,12 @@ static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float tempera
       for (int cc = 0; cc < K; cc++) {
         float gap = tval[cc] - tval[cc + 1];
         if (gap < mg) mg = gap;
+      }
+      if (fw) {
+        for (int cc = 0; cc < K; cc++) cand[cc] = d2t_inverse(c, fw->pool_tok[base + r * K + cc + 1]);
+        follow_choice(fw, lp, Vd, K, tid, tval, cand, mg);
+      }
+      for (int cc = 0; cc < K; cc++) {
         int ci = base + r * K + cc + 1;
         c->pool_tok[ci] = c->dw.d2t[tid[cc]];
         c->pool_parent[ci] = u; c->pool_depth[ci] = d;
@@ -666,12 +749,16 @@ static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float tempera
       float *sc = c->pool_score + base + 1;
       float nxt = -INFINITY;
       orc_topk(sc, K * K, K, tid, tval, &nxt);
-      for (int r = 0; r < K; r++) front[r] = base + 1 + tid[r];
       if (K * K > K) {
         float mg = tval[K - 1] - nxt;
         for (int r = 0; r + 1 < K; r++) if (tval[r] - tval[r + 1] < mg) mg = tval[r] - tval[r + 1];
         c->frontier_margin[d - 1] = mg;
       }
+      if (fw) {
+        for (int r = 0; r < K; r++) cand[r] = fw->frontier[(size_t)d * K + r] - (base + 1);
+        follow_choice(fw, sc, K * K, K, tid, tval, cand, c->frontier_margin[d - 1]);
+      }
+      for (int r = 0; r < K; r++) front[r] = base + 1 + tid[r];
     }
     free(f); free(a); free(tk); free(pos); free(nc); free(ts); free(ne); free(ex);
   }
@@ -679,6 +766,29 @@ static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float tempera
   /* 4. prune to the N-1 best candidates and number the nodes */
   int nn = orc_rerank(c->pool_score, c->pool_parent, c->pool_tok, c->pool_depth, c->pool, N, c->ids[n],
                       c->tok, c->parent, c->depth, c->mask, c->poolidx, c->score, &c->rerank_margin);
+  if (fw) {
+    /* the followed pruned set: as many candidates, none left out that beats the worst kept one by more than eps,
+     * every kept candidate's parent kept */
+    int M = N - 1 < c->pool ? N - 1 : c->pool, valid = fw->nsel == M + 1, same = valid && fw->nsel == nn;
+    char *sel = (char *)xcalloc((size_t)c->pool + 1, 1);
+    float worst = INFINITY;
+    for (int i = 1; i < fw->nsel && valid; i++) {
+      int pi = fw->sel_poolidx[i];
+      if (pi < 1 || pi > c->pool || sel[pi] || (i > 1 && pi <= fw->sel_poolidx[i - 1])) { valid = 0; break; }
+      sel[pi] = 1;
+      if (c->pool_score[pi] < worst) worst = c->pool_score[pi];
+      if (same && c->poolidx[i] != pi) same = 0;
+    }
+    for (int i = 1; i <= c->pool && valid; i++) {
+      if (sel[i] && c->pool_parent[i] != 0 && !sel[c->pool_parent[i]]) valid = 0;
+      if (!sel[i] && c->pool_score[i] > worst + fw->eps) valid = 0;
+    }
+    follow_note(fw, same, c->rerank_margin, valid);
+    if (valid)
+      nn = tree_from_selection(sel, c->pool_score, c->pool_parent, c->pool_tok, c->pool_depth, c->pool, c->ids[n],
+                               c->tok, c->parent, c->depth, c->mask, c->poolidx, c->score);
+    free(sel);
+  }
   c->nn = nn;
 
   /* 5. one target forward over all nodes with tree attention */
@@ -720,15 +830,21 @@ static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float tempera
   }
   c->n = n + cnt;
   c->dn = n;
-  free(lp); free(tid); free(tval); free(front);
+  free(lp); free(tid); free(tval); free(front); free(cand);
   return 0;
 }
 
-int orc_step(orc_ctx *c, int32_t *out_ids, int32_t *count) { return step_impl(c, out_ids, count, 0.0f, NULL); }
+int orc_step(orc_ctx *c, int32_t *out_ids, int32_t *count) { return step_impl(c, out_ids, count, 0.0f, NULL, NULL); }
+
+int orc_step_follow(orc_ctx *c, orc_follow *fw, float temperature, const float *u, int32_t *out_ids, int32_t *count) {
+  if (!fw || !fw->pool_tok || !fw->frontier || !fw->sel_poolidx || !(fw->eps >= 0.0f)) return -1;
+  if (temperature > 0.0f && !u) return -1;
+  return step_impl(c, out_ids, count, temperature > 0.0f ? temperature : 0.0f, temperature > 0.0f ? u : NULL, fw);
+}
 
 int orc_step_sampled(orc_ctx *c, float temperature, const float *u, int32_t *out_ids, int32_t *count) {
   if (!(temperature > 0.0f) || !u) return -1;
-  return step_impl(c, out_ids, count, temperature, u);
+  return step_impl(c, out_ids, count, temperature, u, NULL);
 }
 
 /* Step 5 (Section 2.2, tree attention) on a caller-given tree: node i carries tok[i], sits at RoPE position

@@ -69,6 +69,24 @@ int orc_step(orc_ctx *, int32_t *out_ids, int32_t *count);
  * node cur (inverse CDF over increasing ids).  The emitted tokens are distributed exactly as plain sampling. */
 int orc_step_sampled(orc_ctx *, float temperature, const float *u, int32_t *out_ids, int32_t *count);
 
+/* The same cycle (greedy when temperature <= 0, else the stochastic rule with uniforms u) FOLLOWING another
+ * implementation's integer decisions, so that a harness can compare every later stage after a near-tie the two sides
+ * resolved differently.  Inputs: the other side's candidate tokens in pool layout (pool_tok [pool+1], target ids), its
+ * frontier per pass (frontier [D][K], pool indices) and the pool indices of its pruned tree (sel_poolidx [nsel],
+ * ascending, entry 0 = the root).  A followed choice of K items is adopted when it is valid on the oracle's own
+ * values: order non-increasing within eps, nothing left out that beats the worst chosen item by more than eps (for the
+ * pruned set also: parents kept).  An invalid choice is counted and the oracle's own is used.  Values (log-probs,
+ * scores, logits) are always the oracle's own arithmetic.  Outputs: decisions looked at, how many differed from the
+ * oracle's own choice, how many were invalid; of those whose own margin exceeds `require`: how many, and how many
+ * differed (must be 0 for a conforming implementation); the same two counts for margins in (band_lo, require]. */
+typedef struct {
+  const int32_t *pool_tok, *frontier, *sel_poolidx;
+  int32_t nsel;
+  float eps, require, band_lo;
+  int32_t checked, differs, invalid, required, required_differs, band_total, band_differs;
+} orc_follow;
+int orc_step_follow(orc_ctx *, orc_follow *, float temperature, const float *u, int32_t *out_ids, int32_t *count);
+
 /* Plain greedy autoregressive decoding of the target (the paper's "vanilla" baseline): continue the
  * current state by `gen` tokens, one target forward per token.  Needs a prefilled ctx. */
 int orc_greedy(orc_ctx *, int32_t gen, int32_t *out_ids);

@@ -41,6 +41,13 @@ class _Cfg(C.Structure):
 _PP = C.POINTER(C.c_void_p)
 
 
+class _Follow(C.Structure):
+    _fields_ = [("pool_tok", C.c_void_p), ("frontier", C.c_void_p), ("sel_poolidx", C.c_void_p), ("nsel", C.c_int32),
+                ("eps", C.c_float), ("require", C.c_float), ("band_lo", C.c_float)] + \
+               [(n, C.c_int32) for n in ("checked", "differs", "invalid", "required", "required_differs", "band_total",
+                                         "band_differs")]
+
+
 class _TW(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("final_norm", C.c_void_p), ("lm_head", C.c_void_p)] + \
                [(n, _PP) for n in ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up", "w_down")]
@@ -64,6 +71,8 @@ def lib():
         L.orc_greedy.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
         L.orc_greedy_margins.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.orc_force_state.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32]
+        L.orc_step_follow.restype = C.c_int
+        L.orc_step_follow.argtypes = [C.c_void_p, C.POINTER(_Follow), C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_verify_tree.restype = C.c_int
         L.orc_verify_tree.argtypes = [C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 6
         L.orc_n.argtypes = [C.c_void_p]
@@ -299,6 +308,24 @@ class Oracle:
         if rc:
             raise RuntimeError("orc_step_sampled failed (capacity, temperature?)")
         return out[: int(cnt[0])].copy()
+
+    def step_follow(self, pool_tok, frontier, sel_poolidx, eps: float, require: float, band_lo: float,
+                    temperature: float = 0.0, u=None):
+        """One step that adopts another implementation's decisions wherever they are valid within eps on the oracle's own
+        values (see the header).  Returns (out_ids, counters dict)."""
+        pool_tok = _np(pool_tok, np.int32); frontier = _np(frontier, np.int32); sel = _np(sel_poolidx, np.int32)
+        assert pool_tok.size == self.cfg.pool + 1 and frontier.size == self.cfg.tree_depth * self.cfg.tree_topk
+        fw = _Follow()
+        fw.pool_tok, fw.frontier, fw.sel_poolidx, fw.nsel = pool_tok.ctypes.data, frontier.ctypes.data, sel.ctypes.data, sel.size
+        fw.eps, fw.require, fw.band_lo = eps, require, band_lo
+        uu = _np(u, np.float32) if u is not None else None
+        out = np.zeros(self.cfg.tree_depth + 1, np.int32)
+        cnt = np.zeros(1, np.int32)
+        rc = lib().orc_step_follow(self.h, C.byref(fw), float(temperature), _p(uu) if uu is not None else None, _p(out), _p(cnt))
+        if rc:
+            raise RuntimeError("orc_step_follow failed (capacity, arguments?)")
+        names = ("checked", "differs", "invalid", "required", "required_differs", "band_total", "band_differs")
+        return out[: int(cnt[0])].copy(), {n: int(getattr(fw, n)) for n in names}
 
     def greedy(self, gen: int) -> np.ndarray:
         out = np.zeros(gen, np.int32)

@@ -40,15 +40,15 @@ class Stats:
     and compared nothing cannot pass."""
     COUNTERS = ("steps", "tokens", "resyncs",
                 "passes",            # draft passes whose logits and features were compared element by element
-                "topk_forced",       # top-k rows (own margin above the threshold) required to match, order included
-                "topk_set_forced",   # rows whose K-th vs (K+1)-th gap alone is above the threshold: the SET had to match
-                "frontier_forced",   # frontier selections required to match
-                "exact_tree",        # steps whose whole tree (tokens, parents, depths, masks, pool indices) had to match
-                "same_tree",         # steps whose tree did match the oracle's
+                "decisions",         # draft-side integer decisions checked (top-k rows, frontiers, pruned sets): each valid within 2 tol
+                "decisions_forced",  # ... of which the oracle's own margin required bit-equality (and it held)
+                "decisions_differ",  # ... of which the CUDA path resolved a near-tie differently (valid, followed)
+                "exact_tree",        # steps in which every draft decision was required to be bit-exact
+                "same_tree",         # steps whose tree equals the one the oracle builds on its own
                 "verify_compared",   # steps whose verify logits / hidden states / taps were compared element by element
+                "argmax_forced",     # verify nodes (and first tokens) whose argmax had to match
                 "accept_checked",    # steps whose accepted path and ids equal the oracle's walk over the same tree and argmax
-                "argmax_forced",     # verify nodes whose argmax had to match
-                "exact_out",         # steps whose accepted path and emitted ids had to match
+                "exact_out",         # steps whose emitted ids had to equal the oracle's
                 "band_total", "band_diff")   # decisions with oracle margin in (1e-2, threshold]: seen / differed
 
     def __init__(self):
@@ -77,129 +77,84 @@ class Stats:
         return " ".join(f"{n}={getattr(self, n)}" for n in self.COUNTERS) + " | " + errs
 
 
-def compare_step(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_tol=None, sampled=None, n_ctx=None):
-    """`orc` has just executed the same step from the same state.  Every integer decision is gated on its OWN oracle
-    margin: a top-k row, a frontier selection, the final cut of the candidate pool, each verify node's argmax and the
-    accepted path.  Returns True if the outputs were required to be (and were) identical.
-    sampled = (temperature, u) for a step with stochastic acceptance.  n_ctx = committed length before the step: when
-    the trees differ (a low-margin draft decision), the oracle runs its verify pass on the CUDA path's tree over that
-    prefix, so that the verify floats, the argmax and the acceptance walk are compared in every step."""
+def step_and_compare(dec, orc, seq, cfg, tol, st, gpu_out, check_floats=True, tap_tol=None, sampled=None):
+    """The CUDA path has just executed a step; `orc` is in the same state before it.  The oracle now runs the step
+    FOLLOWING the CUDA path's integer decisions (the K children of every draft row, every frontier, the pruned set):
+    each must be valid on the oracle's own values within 2 tol (order non-increasing, nothing better left out), and
+    bit-equal to the oracle's own choice wherever that choice has margin above the threshold.  Both sides then hold
+    the same tree, so every float of the step is compared: draft logits and features of all D passes, tree scores,
+    verify logits, hidden states, taps; each verify argmax is gated on its own margin; the acceptance walk must equal
+    the oracle's walk over the same tree and argmax.  Returns (oracle's emitted ids, True if the emitted ids were
+    required to be identical).  sampled = (temperature, u) for a step with stochastic acceptance."""
     K, D, N, Vd, k, V = cfg.tree_topk, cfg.tree_depth, cfg.tree_nodes, cfg.draft_vocab, cfg.hidden, cfg.vocab
     tap_tol = tol if tap_tol is None else tap_tol
     thr = decision_margin(tol)
-    o_front = orc.get(po.FRONTIER).reshape(D, K)
-    g_front = dec.debug(sb.DBG_FRONTIER, seq).reshape(D, K)
-    tk_m = orc.get(po.TOPK_MARGIN).reshape(D, K)
-    fr_m = orc.get(po.FRONTIER_MARGIN)
-    rr_m = float(orc.get(po.RERANK_MARGIN)[0])
-    capture = check_floats
-    o_dl = orc.get(po.DRAFT_LOGITS).reshape(D, K, Vd)
-    if capture:
+    g_pool = dec.debug(sb.DBG_POOL_TOK, seq)
+    g_front = dec.debug(sb.DBG_FRONTIER, seq)
+    g_sel = dec.debug(sb.DBG_TREE_POOLIDX, seq)
+    o_out, cnt = orc.step_follow(g_pool, g_front, g_sel, eps=2.0 * tol, require=thr, band_lo=MARGIN,
+                                 temperature=sampled[0] if sampled else 0.0, u=sampled[1] if sampled else None)
+    assert cnt["invalid"] == 0, f"{cnt['invalid']} draft decision(s) of the CUDA path are not valid within {2 * tol} on the oracle's values: {cnt}"
+    assert cnt["required_differs"] == 0, f"a draft decision differs although its oracle margin exceeds {thr}: {cnt}"
+    st.decisions += cnt["checked"]
+    st.decisions_forced += cnt["required"]
+    st.decisions_differ += cnt["differs"]
+    st.band_total += cnt["band_total"]
+    st.band_diff += cnt["band_differs"]
+    st.same_tree += int(cnt["differs"] == 0)
+    st.exact_tree += int(cnt["required"] == cnt["checked"])
+    # ---- draft passes: all of them
+    assert np.array_equal(g_pool, orc.get(po.POOL_TOK)), "candidate pools differ after following"
+    if check_floats:
         g_dl = dec.debug(sb.DBG_DRAFT_LOGITS, seq).reshape(D, K, Vd)
         g_da = dec.debug(sb.DBG_DRAFT_A, seq).reshape(D, K, k)
+        o_dl = orc.get(po.DRAFT_LOGITS).reshape(D, K, Vd)
         o_da = orc.get(po.DRAFT_A).reshape(D, K, k)
-    o_ptok, g_ptok = orc.get(po.POOL_TOK), dec.debug(sb.DBG_POOL_TOK, seq)
-    pool_same = True                 # every candidate drafted so far is the same on both sides
-    front_required = True            # the frontier of the next pass has to match (all decisions behind it were required)
-    for d in range(D):
-        rows = 1 if d == 0 else K
-        # same nodes in the same order, carrying the same tokens (a swapped near-tie inside one top-k
-        # row keeps the pool indices but exchanges the tokens)
-        same_front = d == 0 or (np.array_equal(o_front[d], g_front[d]) and
-                                np.array_equal(o_ptok[o_front[d]], g_ptok[g_front[d]]))
-        if d > 0 and front_required:
-            assert same_front, f"frontier of pass {d} differs although every decision behind it had margin > {thr}: {o_front[d]} vs {g_front[d]}"
-            st.frontier_forced += 1
-        if not same_front:
-            pool_same = False
-            break
-        if capture:
+        for d in range(D):
+            rows = 1 if d == 0 else K
             assert st.err("draft_logits", g_dl[d, :rows], o_dl[d, :rows]) <= tol, (d, st.max_err)
             assert st.err("draft_a", g_da[d, :rows], o_da[d, :rows]) <= tol, (d, st.max_err)
             st.passes += 1
-        # the K children of every row of this pass: pool entries base + r K + 1 .. base + r K + K
-        base = 0 if d == 0 else K + (d - 1) * K * K
-        rows_same = True
-        for r in range(rows):
-            lo = base + r * K + 1
-            o_t, g_t = o_ptok[lo:lo + K], g_ptok[lo:lo + K]
-            same = bool(np.array_equal(o_t, g_t))
-            if st.decide(float(tk_m[d, r]), thr, same, f"top-{K} of pass {d} row {r}"):
-                st.topk_forced += 1
-            else:
-                # membership alone: the K-th against the (K+1)-th log-probability of the oracle's row
-                z = o_dl[d, r].astype(np.float64)
-                top = np.sort(z)[::-1][:K + 1]
-                set_margin = float(top[K - 1] - top[K]) if Vd > K else np.inf
-                same_set = set(o_t.tolist()) == set(g_t.tolist())
-                if st.decide(set_margin, thr, same_set, f"top-{K} set of pass {d} row {r}"):
-                    st.topk_set_forced += 1
-            rows_same = rows_same and same
-        pool_same = pool_same and rows_same
-        # the next frontier: level 1 is taken whole, later levels are the K best children of the level
-        if d + 1 < D:
-            front_required = rows_same and (d == 0 or float(fr_m[d]) > thr)
-            if rows_same and d >= 1 and MARGIN < float(fr_m[d]) <= thr:
-                st.band_total += 1
-                st.band_diff += int(not (np.array_equal(o_front[d + 1], g_front[d + 1])))
+    assert st.err("pool_score", dec.debug(sb.DBG_POOL_SCORE, seq)[1:], orc.get(po.POOL_SCORE)[1:]) <= D * tol
+    # ---- the tree: identical integers, valid structure
     ints = {n: (dec.debug(g, seq), orc.get(o)) for n, g, o in (
         ("tok", sb.DBG_TREE_TOK, po.TREE_TOK), ("parent", sb.DBG_TREE_PARENT, po.TREE_PARENT),
         ("depth", sb.DBG_TREE_DEPTH, po.TREE_DEPTH), ("mask", sb.DBG_TREE_MASK, po.TREE_MASK),
         ("poolidx", sb.DBG_TREE_POOLIDX, po.TREE_POOLIDX))}
-    same_tree = all(np.array_equal(a, b) for a, b in ints.values())
-    st.same_tree += int(same_tree)
-    # the cut of the pool: required when both sides ranked the same candidates and the oracle's cut has margin
-    if pool_same and st.decide(rr_m, thr, same_tree, "pruned tree"):
-        for n, (a, b) in ints.items():
-            assert np.array_equal(a, b), f"tree {n} differs although the pool matches and the cut margin > {thr}\n{a}\n{b}"
-        st.exact_tree += 1
-    # GPU tree must be a valid tree whatever the margins
-    g_par, g_dep, g_mask = ints["parent"][0], ints["depth"][0], ints["mask"][0]
-    for i in range(g_par.size):
+    for n, (a, b) in ints.items():
+        assert np.array_equal(a, b), f"tree {n} differs on identical decisions\n{a}\n{b}"
+    g_tok, g_par, g_dep, g_mask = ints["tok"][0], ints["parent"][0], ints["depth"][0], ints["mask"][0]
+    nn = g_tok.size
+    assert 1 <= nn <= N
+    for i in range(nn):
         if i == 0:
             assert g_par[0] == -1 and g_dep[0] == 0 and int(g_mask[0]) == 1
         else:
             p = int(g_par[i])
             assert 0 <= p < i and g_dep[i] == g_dep[p] + 1 and int(g_mask[i]) == (int(g_mask[p]) | (1 << i))
-    exact_out = False
-    if sampled is not None and not same_tree and check_floats:
-        check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, *sampled, own_inputs=True)
-        st.max_err["sampled_own_inputs_checks"] = st.max_err.get("sampled_own_inputs_checks", 0.0) + 1
-    g_tok, g_par = ints["tok"][0], ints["parent"][0]
-    nn = g_tok.size
-    gy = dec.debug(sb.DBG_Y, seq)
-    if same_tree:
-        assert st.err("tree_score", dec.debug(sb.DBG_TREE_SCORE, seq), orc.get(po.TREE_SCORE)) <= tol
-        o_logits, o_hidden, o_taps = orc.get(po.TARGET_LOGITS), orc.get(po.NODE_HIDDEN), orc.get(po.NODE_TAPS)
-        oy, ym = orc.get(po.Y), orc.get(po.Y_MARGIN)
-    elif check_floats and n_ctx is not None:
-        # the oracle's verify pass on the CUDA path's (valid) tree
-        o_logits, o_hidden, o_taps = orc.verify_tree(n_ctx, g_tok, g_dep, g_mask)
-        top2 = np.partition(o_logits, -2, axis=1)[:, -2:]
-        oy, ym = np.argmax(o_logits, axis=1), top2[:, 1] - top2[:, 0]
-    else:
-        return False
+    assert st.err("tree_score", dec.debug(sb.DBG_TREE_SCORE, seq), orc.get(po.TREE_SCORE)) <= D * tol
+    # ---- verify pass
     if check_floats:
-        assert st.err("target_logits", dec.debug(sb.DBG_TARGET_LOGITS, seq), np.ravel(o_logits)) <= tol, st.max_err
-        assert st.err("node_hidden", dec.debug(sb.DBG_NODE_HIDDEN, seq), np.ravel(o_hidden)) <= tol, st.max_err
-        assert st.err("node_taps", dec.debug(sb.DBG_NODE_TAPS, seq), np.ravel(o_taps)) <= tap_tol, st.max_err
+        assert st.err("target_logits", dec.debug(sb.DBG_TARGET_LOGITS, seq), orc.get(po.TARGET_LOGITS)) <= tol, st.max_err
+        assert st.err("node_hidden", dec.debug(sb.DBG_NODE_HIDDEN, seq), orc.get(po.NODE_HIDDEN)) <= tol, st.max_err
+        assert st.err("node_taps", dec.debug(sb.DBG_NODE_TAPS, seq), orc.get(po.NODE_TAPS)) <= tap_tol, st.max_err
         st.verify_compared += 1
+    gy, oy, ym = dec.debug(sb.DBG_Y, seq), orc.get(po.Y), orc.get(po.Y_MARGIN)
     for i in range(nn):
         if st.decide(float(ym[i]), thr, gy[i] == oy[i], f"argmax of verify node {i}"):
             st.argmax_forced += 1
     if sampled is not None:
-        return check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, *sampled) if same_tree else False
-    # the acceptance walk is integer work: on the CUDA path's own tree and argmax it must equal the oracle's walk
-    cnt, w_path, w_out = po.accept(g_tok, g_par, gy)
+        return o_out, check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, *sampled)
+    # the acceptance walk is integer work: on the CUDA path's own argmax it must equal the oracle's walk
+    _, w_path, w_out = po.accept(g_tok, g_par, gy)
     g_path = dec.debug(sb.DBG_PATH, seq)
     assert np.array_equal(g_path, w_path) and np.array_equal(np.asarray(gpu_out), w_out), (g_path, w_path, gpu_out, w_out)
     st.accept_checked += 1
-    if same_tree:
-        o_path = orc.get(po.PATH)
-        if (ym[o_path] > thr).all():
-            assert np.array_equal(g_path, o_path), (g_path, o_path)
-            exact_out = True
-    return exact_out
+    o_path = orc.get(po.PATH)
+    exact_out = bool((ym[o_path] > thr).all())
+    if exact_out:
+        assert np.array_equal(g_path, o_path), (g_path, o_path)
+    return o_out, exact_out
 
 
 def check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, temperature, u, own_inputs=False):
@@ -267,7 +222,7 @@ def check_sampled_decisions(dec, orc, seq, cfg, tol, gpu_out, temperature, u, ow
 
 
 def run_trajectory(cfg, tw, dw, prompts, n_steps, tol, flags=0, max_ctx=None, check_floats=True, tap_tol=None,
-                   page_shuffle_seed=0, num_pages=None, tune=(), sampling=None):
+                   page_shuffle_seed=0, num_pages=None, tune=(), sampling=None, greedy_check=True):
     """tw/dw: CPU weight dicts; tune: (knob, value, value to restore) triples applied to the decoder (process-wide knobs).
     sampling = (temperature, seed): every step uses the stochastic acceptance rule with uniforms drawn from that seed.
     Returns Stats; raises AssertionError on a parity violation."""
@@ -282,14 +237,16 @@ def run_trajectory(cfg, tw, dw, prompts, n_steps, tol, flags=0, max_ctx=None, ch
     for knob, value, _ in tune:
         dec.tune(knob, value)
     try:
-        return _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, check_floats, tap_tol, sampling)
+        return _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, check_floats, tap_tol, sampling,
+                               greedy_check)
     finally:
         for knob, _, restore in tune:
             dec.tune(knob, restore)
         dec.close()
 
 
-def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, check_floats, tap_tol, sampling=None):
+def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, check_floats, tap_tol, sampling=None,
+                    greedy_check=True):
     B = len(prompts)
     rng = np.random.default_rng(sampling[1]) if sampling else None
     st = Stats()
@@ -298,7 +255,16 @@ def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, c
     for b in range(B):
         o = po.Oracle(cfg, tw, dw, max_ctx)
         f = o.prefill(np.asarray(prompts[b]))
-        assert f == first[b], f"first token differs for sequence {b}: {f} vs {first[b]}"
+        # the first token is an argmax like any other: it has to match where the oracle's top-1 margin allows
+        n0 = len(prompts[b])
+        lg, _, _ = o.verify_tree(n0 - 1, prompts[b][-1:], [0], [1])
+        top2 = np.partition(lg[0], -2)[-2:]
+        st.err("prefill_logit_top1", lg[0, f], top2[1])
+        if st.decide(float(top2[1] - top2[0]), decision_margin(tol), f == first[b], f"first token of sequence {b} ({f} vs {first[b]})"):
+            st.argmax_forced += 1
+        if f != first[b]:
+            st.resyncs += 1
+            o.force_state(np.concatenate([prompts[b], [first[b]]]).astype(np.int32), n0, 1)
         orcs.append(o)
     emitted = [[] for _ in range(B)]
     for step in range(n_steps):
@@ -307,11 +273,10 @@ def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, c
         for b in range(B):
             o = orcs[b]
             ids_before, n_before = o.ids, o.n
-            o_out = o.step_sampled(sampling[0], u[b]) if sampling else o.step()
             g_out = outs[b]
             assert 1 <= len(g_out) <= cfg.tree_depth + 1
-            exact = compare_step(dec, o, b, cfg, tol, st, g_out, check_floats, tap_tol,
-                                 sampled=(sampling[0], u[b]) if sampling else None, n_ctx=n_before)
+            o_out, exact = step_and_compare(dec, o, b, cfg, tol, st, g_out, check_floats, tap_tol,
+                                            sampled=(sampling[0], u[b]) if sampling else None)
             if exact:
                 assert np.array_equal(g_out, o_out), (g_out, o_out)
                 st.exact_out += 1
@@ -338,7 +303,7 @@ def _run_trajectory(dec, cfg, tw, dw, prompts, n_steps, tol, max_ctx, reserve, c
                 ok, ov = o.draft_kv(pos)
                 assert st.err("kv_draft", gk, ok) <= 4 * tol and st.err("kv_draft", gv, ov) <= 4 * tol, (b, pos)
     # losslessness against plain greedy decoding of the oracle, up to the first low-margin token
-    for b in range(B if not sampling else 0):
+    for b in range(B if (greedy_check and not sampling) else 0):
         g = po.Oracle(cfg, tw, dw, max_ctx)
         g.prefill(np.asarray(prompts[b]))
         ref, mg = g.greedy_margins(len(emitted[b]))

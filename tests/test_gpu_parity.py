@@ -200,7 +200,8 @@ def test_c1_full_trajectory_fp32(flags):
     prompts = [p.numpy() for p in synth.make_prompts(C1)]
     st, emitted = parity.run_trajectory(C1, tw, dw, prompts, n_steps=32, tol=1e-4, flags=flags)
     print("C1", st)
-    assert st.tokens >= 32 and st.exact_tree >= 1 and st.same_tree >= 24 and st.exact_out >= 24
+    assert st.tokens >= 32 and st.passes == 32 * 3 and st.verify_compared == 32 and st.accept_checked == 32, st
+    assert st.exact_tree >= 20 and st.same_tree >= 30 and st.exact_out >= 24 and st.band_total == 0, st
 
 
 @pytest.mark.parametrize("flags", [0, sb.FLAG_NO_PDL | sb.FLAG_NO_GRAPH, sb.FLAG_CHAIN, sb.FLAG_CHAIN | sb.FLAG_NO_GRAPH, sb.FLAG_UNFUSED,
@@ -210,7 +211,8 @@ def test_tiny_bf16_trajectory(flags):
     prompts = [p.numpy() for p in synth.make_prompts(T1)]
     st, _ = parity.run_trajectory(T1, tw, dw, prompts, n_steps=16, tol=2e-2, flags=flags, tap_tol=3e-2)
     print("T1", flags, st)
-    assert st.same_tree >= 4
+    assert st.passes == 16 * 3 and st.verify_compared == 16 and st.accept_checked == 16, st
+    assert st.decisions_forced >= 40 and st.same_tree >= 4 and st.argmax_forced >= 150, st
 
 
 @pytest.mark.parametrize("flags", [0, sb.FLAG_CHAIN])
@@ -219,6 +221,7 @@ def test_small_bf16_hd128_trajectory(flags):
     prompts = [p.numpy() for p in synth.make_prompts(T2)]
     st, _ = parity.run_trajectory(T2, tw, dw, prompts, n_steps=10, tol=2e-2, tap_tol=3e-2, flags=flags)
     print("T2", st)
+    assert st.passes == 10 * 4 and st.verify_compared == 10 and st.decisions_forced >= 20 and st.argmax_forced >= 150, st
 
 
 @pytest.mark.parametrize("batch", [1, 3])
@@ -231,6 +234,7 @@ def test_small_bf16_hd128_trajectory_tcgen05_attention(batch):
     st, _ = parity.run_trajectory(cfg, tw, dw, prompts, n_steps=6, tol=2e-2, tap_tol=3e-2,
                                   tune=[(sb.SpecDecoder.TUNE_ATTN_UMMA, 1, 2)])
     print("T2 tcgen05 attention", st)
+    assert st.passes == 6 * 4 * batch and st.verify_compared == 6 * batch and st.argmax_forced >= 80 * batch, st
 
 
 # multi-head attention (one KV head per query head), as in the Vicuna-13B-shaped targets of the paper's Table 1
@@ -246,7 +250,7 @@ def test_mha_model_trajectory(batch):
     prompts = [p.numpy() for p in synth.make_prompts(cfg)]
     st, _ = parity.run_trajectory(cfg, tw, dw, prompts, n_steps=6, tol=2e-2, tap_tol=3e-2)
     print("T3 MHA", batch, st)
-    assert st.steps == 6
+    assert st.steps == 6 and st.passes == 6 * 5 * batch and st.verify_compared == 6 * batch and st.decisions_forced >= 10, st
 
 
 @pytest.mark.parametrize("base", [C1, T1], ids=["fp32", "bf16"])
@@ -292,7 +296,7 @@ def test_degenerate_tree_shapes_trajectory(base, case):
     tol = 1e-4 if cfg.dtype == "fp32" else 2e-2
     st, _ = parity.run_trajectory(cfg, tw, dw, prompts, n_steps=5, tol=tol, tap_tol=None if cfg.dtype == "fp32" else 3e-2)
     print(case, st)
-    assert st.steps == 5
+    assert st.steps == 5 and st.passes == 5 * cfg.tree_depth and st.verify_compared == 5 and st.accept_checked == 5, st
 
 
 @pytest.mark.parametrize("temperature", [1.0, 0.3])
@@ -308,7 +312,7 @@ def test_sampled_acceptance_trajectory(base, temperature):
     st, emitted = parity.run_trajectory(cfg, tw, dw, prompts, n_steps=10, tol=tol, tap_tol=None if cfg.dtype == "fp32" else 3e-2,
                                         sampling=(temperature, 17))
     print("sampled", cfg.name, temperature, st)
-    assert st.steps == 10 and st.same_tree >= 3
+    assert st.steps == 10 and st.same_tree >= 3 and st.verify_compared == 10 * cfg.batch and st.passes == 10 * cfg.batch * cfg.tree_depth, st
     if cfg.dtype == "fp32":
         assert st.resyncs <= 1          # float errors of ~4e-6: the outputs coincide with the oracle's
 
@@ -384,6 +388,7 @@ def test_batch_chain_with_shuffled_pages():
     prompts = [p.numpy() for p in synth.make_prompts(cfg)]
     st, _ = parity.run_trajectory(cfg, tw, dw, prompts, n_steps=8, tol=2e-2, tap_tol=3e-2, page_shuffle_seed=77)
     print("chain", st)
+    assert st.passes == 8 * 5 * 3 and st.verify_compared == 40 and st.accept_checked == 40 and st.decisions_forced >= 100, st
 
 
 def test_page_permutation_invariance():
@@ -458,6 +463,7 @@ def test_c2_two_layer_truncation_first_steps(flags):
     prompts = [p.numpy() for p in synth.make_prompts(cfg)]
     st, _ = parity.run_trajectory(cfg, parity.to_cpu(tw), parity.to_cpu(dw), prompts, n_steps=2, tol=2e-2, tap_tol=3e-2, flags=flags)
     print("C2-L2", st)
+    assert st.passes == 12 and st.verify_compared == 2 and st.decisions == 2 * (1 + 50 + 4 + 1) and st.argmax_forced >= 60, st
 
 
 def test_c2_two_layer_truncation_sampled_steps():
@@ -470,6 +476,7 @@ def test_c2_two_layer_truncation_sampled_steps():
     st, _ = parity.run_trajectory(cfg, parity.to_cpu(tw), parity.to_cpu(dw), prompts, n_steps=2, tol=2e-2, tap_tol=3e-2,
                                   sampling=(0.7, 23))
     print("C2-L2 sampled", st)
+    assert st.passes == 12 and st.verify_compared == 2, st
 
 
 @pytest.mark.parametrize("H,G,hd,rps", [(32, 8, 128, 4), (8, 2, 128, 1), (4, 2, 64, 3)])

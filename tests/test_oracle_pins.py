@@ -378,6 +378,58 @@ def test_verify_tree_on_a_given_tree_equals_sequential_decoding(c1):
         o.verify_tree(n0, tok, dep, bad)
 
 
+def _own_decisions(o):
+    return o.get(po.POOL_TOK), o.get(po.FRONTIER), o.get(po.TREE_POOLIDX)
+
+
+def test_follow_mode_reproduces_own_step_and_rejects_invalid_choices(c1):
+    """orc_step_follow: (1) fed the oracle's own decisions it is the ordinary step, bit for bit, with no decision
+    reported as different; (2) a followed top-k row with two children exchanged is adopted when their log-probabilities
+    lie within eps and the later stages then run on the exchanged order; (3) with eps = 0 the same exchange, a child
+    replaced by a token outside the top-k, and a pruned set that drops a better candidate are all refused."""
+    tw, dw, ids = c1
+    a, b = _mk(C1, tw, dw), _mk(C1, tw, dw)
+    a.prefill(ids); b.prefill(ids)
+    out_a = a.step()
+    dec_a = _own_decisions(a)
+    out_b, cnt = b.step_follow(*dec_a, eps=0.0, require=1e-2, band_lo=1e-2)
+    K, D = C1.tree_topk, C1.tree_depth
+    assert cnt["invalid"] == 0 and cnt["differs"] == 0 and cnt["required_differs"] == 0
+    assert cnt["checked"] == 1 + (D - 1) * K + (D - 2) + 1          # top-k rows, frontiers, the pruned set
+    assert np.array_equal(out_a, out_b)
+    for what in (po.TREE_TOK, po.TREE_MASK, po.TARGET_LOGITS, po.DRAFT_LOGITS, po.DRAFT_A, po.NODE_TAPS, po.POOL_SCORE):
+        assert np.array_equal(a.get(what), b.get(what)), what
+    # (2) exchange children 2 and 3 of the root: valid within a generous eps, and the step follows it
+    c = _mk(C1, tw, dw); c.prefill(ids)
+    pool, front, sel = (x.copy() for x in dec_a)
+    pool[[2, 3]] = pool[[3, 2]]
+    out_c, cnt_c = c.step_follow(pool, front, sel, eps=10.0, require=1e9, band_lo=1e9)
+    assert cnt_c["invalid"] == 0 and cnt_c["differs"] >= 1
+    assert np.array_equal(c.get(po.POOL_TOK)[:K + 1], pool[:K + 1])
+    sc_a, sc_c = a.get(po.POOL_SCORE), c.get(po.POOL_SCORE)
+    assert sc_c[2] == sc_a[3] and sc_c[3] == sc_a[2]                  # the oracle's own values, in the followed order
+    # (3) eps = 0: refused, the oracle's own choice is used and the step equals the ordinary one
+    for mutate in ("swap", "outsider", "prune"):
+        d = _mk(C1, tw, dw); d.prefill(ids)
+        pool, front, sel = (x.copy() for x in dec_a)
+        if mutate == "swap":
+            pool[[2, 3]] = pool[[3, 2]]
+        elif mutate == "outsider":
+            inside = set(pool[1:K + 1].tolist())
+            pool[K] = next(int(t) for t in dw["d2t"].tolist() if int(t) not in inside)
+        else:
+            unsel = [i for i in range(1, C1.pool + 1) if i not in set(sel.tolist())]
+            worst_unsel = min(unsel, key=lambda i: sc_a[i])
+            leaf = max(sel.tolist())                                  # the highest pool index kept is a leaf
+            if sc_a[worst_unsel] >= sc_a[leaf]:
+                continue
+            sel = np.sort(np.array([i for i in sel.tolist() if i != leaf] + [worst_unsel], np.int32))
+        out_d, cnt_d = d.step_follow(pool, front, sel, eps=0.0, require=1e-2, band_lo=1e-2)
+        assert cnt_d["invalid"] >= 1, mutate
+        if mutate != "prune":
+            assert np.array_equal(d.get(po.POOL_TOK)[:K + 1], dec_a[0][:K + 1]), mutate
+
+
 def test_commit_equals_fresh_prefill(c1):
     tw, dw, ids = c1
     tws, dws, pi, pi2 = synth.make_structured(C1, 0.8, residual_scale=0.05)
