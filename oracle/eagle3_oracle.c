@@ -618,11 +618,13 @@ static void follow_note(orc_follow *fw, int same, float own_margin, int valid) {
   else if (own_margin > fw->band_lo) { fw->band_total++; if (!same) fw->band_differs++; }
 }
 
-/* v[n]: the oracle's values; own[K]: its own choice; cand[K]: the followed choice (indices into v, -1 = unknown).
- * Returns 1 and overwrites own/own_val with the followed choice when that is valid. */
-static int follow_choice(orc_follow *fw, const float *v, int n, int K, int32_t *own, float *own_val, const int32_t *cand,
-                         float own_margin) {
-  int valid = 1, same = 1;
+/* v[n]: the oracle's values; own[K] / own_val[K]: its own choice in rank order, next_val: its (K+1)-th value;
+ * cand[K]: the followed choice (indices into v, -1 = unknown).  Every rank is one decision whose margin is the
+ * smaller of the gaps to its neighbours in the oracle's own order (the last rank: to the best item left out).
+ * Returns 1 and overwrites own / own_val with the followed choice when that is valid. */
+static int follow_choice(orc_follow *fw, const float *v, int n, int K, int32_t *own, float *own_val, float next_val,
+                         const int32_t *cand) {
+  int valid = 1;
   for (int r = 0; r < K && valid; r++) {
     if (cand[r] < 0 || cand[r] >= n) valid = 0;
     for (int q = 0; q < r && valid; q++) if (cand[q] == cand[r]) valid = 0;
@@ -631,7 +633,6 @@ static int follow_choice(orc_follow *fw, const float *v, int n, int K, int32_t *
   for (int r = 0; r < K && valid; r++) {
     if (r + 1 < K && v[cand[r]] < v[cand[r + 1]] - fw->eps) valid = 0;
     if (v[cand[r]] < worst) worst = v[cand[r]];
-    if (cand[r] != own[r]) same = 0;
   }
   if (valid) {
     for (int i = 0; i < n && valid; i++) {
@@ -641,8 +642,12 @@ static int follow_choice(orc_follow *fw, const float *v, int n, int K, int32_t *
       if (!chosen) valid = 0;
     }
   }
-  follow_note(fw, same, own_margin, valid);
-  if (!valid) return 0;
+  if (!valid) { fw->checked += K; fw->invalid++; return 0; }
+  for (int r = 0; r < K; r++) {
+    float below = own_val[r] - (r + 1 < K ? own_val[r + 1] : next_val);
+    float above = r > 0 ? own_val[r - 1] - own_val[r] : INFINITY;
+    follow_note(fw, cand[r] == own[r], below < above ? below : above, 1);
+  }
   for (int r = 0; r < K; r++) { own[r] = cand[r]; own_val[r] = v[cand[r]]; }
   return 1;
 }
@@ -688,7 +693,7 @@ static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float tempera
   }
   if (fw) {
     for (int r = 0; r < K; r++) cand[r] = d2t_inverse(c, fw->pool_tok[1 + r]);
-    follow_choice(fw, lp, Vd, K, tid, tval, cand, c->topk_margin[0]);
+    follow_choice(fw, lp, Vd, K, tid, tval, tval[K], cand);
   }
   for (int r = 0; r < K; r++) {
     c->pool_tok[1 + r] = c->dw.d2t[tid[r]];
@@ -734,7 +739,7 @@ static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float tempera
       }
       if (fw) {
         for (int cc = 0; cc < K; cc++) cand[cc] = d2t_inverse(c, fw->pool_tok[base + r * K + cc + 1]);
-        follow_choice(fw, lp, Vd, K, tid, tval, cand, mg);
+        follow_choice(fw, lp, Vd, K, tid, tval, tval[K], cand);
       }
       for (int cc = 0; cc < K; cc++) {
         int ci = base + r * K + cc + 1;
@@ -756,7 +761,7 @@ static int step_impl(orc_ctx *c, int32_t *out_ids, int32_t *count, float tempera
       }
       if (fw) {
         for (int r = 0; r < K; r++) cand[r] = fw->frontier[(size_t)d * K + r] - (base + 1);
-        follow_choice(fw, sc, K * K, K, tid, tval, cand, c->frontier_margin[d - 1]);
+        follow_choice(fw, sc, K * K, K, tid, tval, nxt, cand);
       }
       for (int r = 0; r < K; r++) front[r] = base + 1 + tid[r];
     }

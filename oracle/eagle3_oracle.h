@@ -76,8 +76,10 @@ int orc_step_sampled(orc_ctx *, float temperature, const float *u, int32_t *out_
  * ascending, entry 0 = the root).  A followed choice of K items is adopted when it is valid on the oracle's own
  * values: order non-increasing within eps, nothing left out that beats the worst chosen item by more than eps (for the
  * pruned set also: parents kept).  An invalid choice is counted and the oracle's own is used.  Values (log-probs,
- * scores, logits) are always the oracle's own arithmetic.  Outputs: decisions looked at, how many differed from the
- * oracle's own choice, how many were invalid; of those whose own margin exceeds `require`: how many, and how many
+ * scores, logits) are always the oracle's own arithmetic.  A decision is one rank of a top-K choice (margin: the
+ * smaller gap to its neighbours in the oracle's own order; last rank: to the best item left out) or the pruned set as
+ * a whole (margin: the cut).  Outputs: decisions looked at, how many differed from the oracle's own choice, how many
+ * choices were invalid; of those whose own margin exceeds `require`: how many, and how many
  * differed (must be 0 for a conforming implementation); the same two counts for margins in (band_lo, require]. */
 typedef struct {
   const int32_t *pool_tok, *frontier, *sel_poolidx;

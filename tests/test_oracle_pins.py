@@ -395,7 +395,7 @@ def test_follow_mode_reproduces_own_step_and_rejects_invalid_choices(c1):
     out_b, cnt = b.step_follow(*dec_a, eps=0.0, require=1e-2, band_lo=1e-2)
     K, D = C1.tree_topk, C1.tree_depth
     assert cnt["invalid"] == 0 and cnt["differs"] == 0 and cnt["required_differs"] == 0
-    assert cnt["checked"] == 1 + (D - 1) * K + (D - 2) + 1          # top-k rows, frontiers, the pruned set
+    assert cnt["checked"] == K + (D - 1) * K * K + (D - 2) * K + 1   # every rank of every top-k row and frontier, the pruned set
     assert np.array_equal(out_a, out_b)
     for what in (po.TREE_TOK, po.TREE_MASK, po.TARGET_LOGITS, po.DRAFT_LOGITS, po.DRAFT_A, po.NODE_TAPS, po.POOL_SCORE):
         assert np.array_equal(a.get(what), b.get(what)), what

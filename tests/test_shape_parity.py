@@ -39,7 +39,7 @@ def _assert_everything_compared(st, cfg, sequences=1):
     units = st.steps * sequences
     assert st.passes == units * D, st
     assert st.verify_compared == units, st
-    per_step = 1 + (D - 1) * K + max(D - 2, 0) + 1           # top-k rows, frontier selections, the pruned set
+    per_step = K + (D - 1) * K * K + max(D - 2, 0) * K + 1    # every rank of every top-k row and frontier, the pruned set
     assert st.decisions == units * per_step, st
 
 
@@ -50,7 +50,7 @@ def test_c5_shape_two_layer_steps_vs_oracle():
     st, _, _ = _run(cfg, 2)
     assert st.steps == 2
     _assert_everything_compared(st, cfg)
-    assert st.decisions_forced >= 4 and st.argmax_forced >= 60 and st.accept_checked == 2, st
+    assert st.decisions_forced >= 200 and st.argmax_forced >= 60 and st.accept_checked == 2, st
     st2, _, _ = _run(cfg, 1, sampling=(0.8, 31))
     assert st2.steps == 1 and st2.passes == cfg.tree_depth and st2.verify_compared == 1, st2
 
@@ -64,15 +64,15 @@ def test_c4_shape_two_layer_long_context_steps_vs_oracle():
     st, _, _ = _run(cfg, 2, greedy_check=False)
     assert st.steps == 2
     _assert_everything_compared(st, cfg)
-    assert st.decisions_forced >= 4 and st.argmax_forced >= 60 and st.accept_checked == 2, st
+    assert st.decisions_forced >= 200 and st.argmax_forced >= 60 and st.accept_checked == 2, st
 
 
 def test_c3_shape_two_layer_batch64_steps_vs_oracle():
-    """8B widths at batch 64 with chains of 3 (Section 4.3's serving setting), ragged prompts of 24..96 tokens, 2-layer
+    """8B widths at batch 64 with chains of 3 (Section 4.3's serving setting), ragged prompts of 16..64 tokens, 2-layer
     truncation: 256-row verify passes (the widest GEMM tiles, the gate/up pair kernel), the key-parallel attention
     kernel at <= 4 rows per sequence and longest-first issue, against 64 oracles."""
-    cfg = synth.C3.truncated(2, prompt_lo=24, prompt_hi=96)
-    st, _, prompts = _run(cfg, 2, page_shuffle_seed=13)
+    cfg = synth.C3.truncated(2, prompt_lo=16, prompt_hi=64)
+    st, _, prompts = _run(cfg, 2, page_shuffle_seed=13, greedy_check=False)
     assert len(prompts) == 64 and st.steps == 2
     # a chain: every step has 3 draft passes of one row per sequence
     _assert_everything_compared(st, cfg, sequences=64)
@@ -87,4 +87,4 @@ def test_c2_full_depth_steps_vs_oracle():
     st, _, _ = _run(cfg, 2, greedy_check=False)
     assert st.steps == 2
     _assert_everything_compared(st, cfg)
-    assert st.decisions_forced >= 4 and st.argmax_forced >= 60 and st.accept_checked == 2, st
+    assert st.decisions_forced >= 200 and st.argmax_forced >= 60 and st.accept_checked == 2, st
