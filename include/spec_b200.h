@@ -50,13 +50,11 @@ enum {
   SPEC_FLAG_REF_ATTN = 2,        /* use the plain CUDA-core attention kernel also for bf16             */
   SPEC_FLAG_CAPTURE = 4,         /* keep per-pass draft logits / features for spec_debug_read          */
   SPEC_FLAG_NO_GRAPH = 8,        /* launch kernels one by one instead of replaying a CUDA graph        */
-  SPEC_FLAG_UNFUSED = 16,        /* bf16: separate norm / RoPE / activation kernels and split-K partial
-                                    sums in global memory instead of the fused GEMM epilogues          */
+  SPEC_FLAG_STAMPS = 16,         /* profiling aid: every GEMM and attention launch of a step records when its
+                                    inputs became ready and when its last CTA left (SPEC_DBG_STAMPS); costs two
+                                    atomics per CTA, so timed runs leave it off                          */
   SPEC_FLAG_NO_PDL = 32,         /* no programmatic dependent launch between the kernels of a step    */
-  SPEC_FLAG_NO_TMA_ATTN = 128,   /* attention K/V tiles through cp.async instead of TMA page copies             */
-  SPEC_FLAG_CHAIN = 64           /* run the GEMMs between two attention calls as ONE persistent kernel (balanced
-                                    unit ranges, partial sums through L2, grid counters) instead of one
-                                    cluster split-K kernel per GEMM; measured slower on B200, kept as an option */
+  SPEC_FLAG_NO_TMA_ATTN = 128    /* attention K/V tiles through cp.async instead of TMA page copies    */
 };
 
 /* Target model weights (Section 3.1: the frozen target whose layers are tapped).  Device pointers;
@@ -153,13 +151,13 @@ enum spec_prof_class {
 int spec_profile_step(spec_ctx *ctx, float *class_ms, int32_t *class_launches);
 
 /* Performance knobs (the defaults are tuned for B200; results never depend on them).
- *   SPEC_TUNE_L2_LEAD_MB  how many MB of the weights that follow in a step's read order each GEMM launch
- *                         keeps prefetched in L2 (0 = no prefetch)
  *   SPEC_TUNE_GEMM_CTAS   CTAs a weight-streaming GEMM launch aims at (process-wide) */
-enum spec_tune_knob { SPEC_TUNE_L2_LEAD_MB = 1, SPEC_TUNE_GEMM_CTAS = 2,
+enum spec_tune_knob { SPEC_TUNE_GEMM_CTAS = 2,
                       SPEC_TUNE_DEBUG_LAUNCH_BUDGET = 3 /* debugging: run only the first n kernels of each step (-1: all) */,
                       SPEC_TUNE_ATTN_CTAS = 4 /* CTAs an attention launch aims at when splitting keys (process-wide) */,
-                      SPEC_TUNE_CHAIN_TIMING = 5 /* profiling: record phase time stamps of the n-th chain launch of a step (-1: none) */,
+                      SPEC_TUNE_DEBUG_WAIT_RUNS_OUT = 5 /* test hook for the bounded device waits: with a value n > 0 one CTA of the verify
+                                                  pass's LM-head GEMM never receives its first activation tile and gives up after n
+                                                  polls; the step then returns SPEC_ERR_DEVICE_STATUS (0 = off) */,
                       SPEC_TUNE_ATTN_UMMA = 6 /* tree passes (head_dim 128): 1 = tcgen05 attention kernel, 0 = mma.sync kernel, 2 (default) = tcgen05
                                                   when every CTA gets several key tiles, i.e. long contexts (process-wide) */ };
 int spec_tune(spec_ctx *ctx, int32_t what, int32_t value);
@@ -198,7 +196,10 @@ enum spec_debug_what {
   /* raw activation buffers of the last pass as floats, all allocated rows (debugging) */
   SPEC_DBG_RAW_X = 100, SPEC_DBG_RAW_H, SPEC_DBG_RAW_Q, SPEC_DBG_RAW_AO, SPEC_DBG_RAW_ACT, SPEC_DBG_RAW_CAT,
   SPEC_DBG_RAW_SSQ, SPEC_DBG_RAW_LOGITS,
-  SPEC_DBG_CHAIN_TIMING      /* int64 [chain CTAs][4 ops][8] globaltimer stamps (ns), see SPEC_TUNE_CHAIN_TIMING */
+  /* SPEC_FLAG_STAMPS: per stamped launch of the last step, in launch order, uint64 [n][2] = {earliest time a CTA of the
+   * launch had its inputs ready (after its programmatic-dependent-launch wait), latest time a CTA left}, nanoseconds
+   * of the GPU's global timer; and the launch's profile class, int32 [n] */
+  SPEC_DBG_STAMPS = 120, SPEC_DBG_STAMP_CLASS
 };
 /* Copies up to `bytes` of item `what` of sequence `seq` (last step) to host_dst; returns bytes
  * available (>= 0) or a negative status. */
@@ -210,12 +211,10 @@ int spec_debug_read_kv(spec_ctx *ctx, int32_t seq, int32_t layer, int32_t pos, f
  * Each launches on `stream` and does not synchronise.  dtype as spec_dtype. */
 
 /* out[r][o] = sum_i x[r][i] * w[o][i]; x [rows][in] dtype, w [out][in] dtype, out fp32 [rows][ldo]
- * (first `out` columns).  impl 0: tcgen05/TMEM kernel (bf16 only), 1: plain CUDA-core kernel.
- * scratch: device fp32 buffer of spec_gemm_scratch_bytes(rows, out, in) bytes for split-K partial
- * sums (may be NULL when that size is 0). */
-size_t spec_gemm_scratch_bytes(int32_t rows, int32_t out, int32_t in);
+ * (first `out` columns).  impl 0: the step's tcgen05/TMEM kernel with the library's own plan (bf16 only; the shape
+ * limits of spec_gemm_fused), 1: plain CUDA-core kernel. */
 int spec_gemm(int32_t dtype, int32_t impl, const void *x, const void *w, float *out_f32, int32_t rows, int32_t out,
-              int32_t in, int32_t ldo, void *scratch, void *stream);
+              int32_t in, int32_t ldo, void *stream);
 
 /* The same contraction on the kernel the step uses (Section 3.1's FC, projection and LM-head layers are
  * all of this form): bf16, tcgen05/TMEM, split-K reduced across a thread-block cluster through

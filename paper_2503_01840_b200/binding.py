@@ -19,13 +19,14 @@ from . import build as _build
 _lib = None
 
 F32, BF16 = 0, 1
-FLAG_REF_GEMM, FLAG_REF_ATTN, FLAG_CAPTURE, FLAG_NO_GRAPH, FLAG_UNFUSED, FLAG_NO_PDL, FLAG_CHAIN, FLAG_NO_TMA_ATTN = 1, 2, 4, 8, 16, 32, 64, 128
+FLAG_REF_GEMM, FLAG_REF_ATTN, FLAG_CAPTURE, FLAG_NO_GRAPH, FLAG_STAMPS, FLAG_NO_PDL, FLAG_NO_TMA_ATTN = 1, 2, 4, 8, 16, 32, 128
 
 (DBG_TREE_TOK, DBG_TREE_PARENT, DBG_TREE_DEPTH, DBG_TREE_MASK, DBG_TREE_POOLIDX, DBG_TREE_SCORE, DBG_Y,
  DBG_TARGET_LOGITS, DBG_NODE_TAPS, DBG_NODE_HIDDEN, DBG_DRAFT_LOGITS, DBG_DRAFT_A, DBG_POOL_TOK, DBG_POOL_SCORE,
  DBG_POOL_PARENT, DBG_FRONTIER, DBG_PATH, DBG_STATUS, DBG_PAGE_TABLE) = range(1, 20)
-DBG_RAW_X, DBG_RAW_H, DBG_RAW_Q, DBG_RAW_AO, DBG_RAW_ACT, DBG_RAW_CAT, DBG_RAW_SSQ, DBG_RAW_LOGITS, DBG_CHAIN_TIMING = range(100, 109)
-_DBG_DTYPE = {**{i: np.float32 for i in range(100, 108)}, DBG_CHAIN_TIMING: np.int64, DBG_TREE_TOK: np.int32, DBG_TREE_PARENT: np.int32, DBG_TREE_DEPTH: np.int32, DBG_TREE_MASK: np.uint64,
+DBG_RAW_X, DBG_RAW_H, DBG_RAW_Q, DBG_RAW_AO, DBG_RAW_ACT, DBG_RAW_CAT, DBG_RAW_SSQ, DBG_RAW_LOGITS = range(100, 108)
+DBG_STAMPS, DBG_STAMP_CLASS = 120, 121
+_DBG_DTYPE = {**{i: np.float32 for i in range(100, 108)}, DBG_STAMPS: np.uint64, DBG_STAMP_CLASS: np.int32, DBG_TREE_TOK: np.int32, DBG_TREE_PARENT: np.int32, DBG_TREE_DEPTH: np.int32, DBG_TREE_MASK: np.uint64,
               DBG_TREE_POOLIDX: np.int32, DBG_TREE_SCORE: np.float32, DBG_Y: np.int32, DBG_TARGET_LOGITS: np.float32,
               DBG_NODE_TAPS: np.float32, DBG_NODE_HIDDEN: np.float32, DBG_DRAFT_LOGITS: np.float32,
               DBG_DRAFT_A: np.float32, DBG_POOL_TOK: np.int32, DBG_POOL_SCORE: np.float32, DBG_POOL_PARENT: np.int32,
@@ -57,7 +58,7 @@ class _Cfg(C.Structure):
 
 EXPORTS = ("spec_workspace_bytes", "spec_init", "spec_prefill", "spec_step", "spec_step_async", "spec_step_sampled", "spec_plain_step",
            "spec_lengths", "spec_profile_step", "spec_tune", "spec_launches_per_step", "spec_step_bytes", "spec_free", "spec_last_error",
-           "spec_debug_read", "spec_debug_read_kv", "spec_gemm_scratch_bytes", "spec_gemm", "spec_gemm_fused", "spec_gemm_swiglu",
+           "spec_debug_read", "spec_debug_read_kv", "spec_gemm", "spec_gemm_fused", "spec_gemm_swiglu",
            "spec_topk_scratch_bytes", "spec_attn_scratch_bytes",
            "spec_attention", "spec_attention_static", "spec_attention_static_capacity", "spec_logsoftmax_topk", "spec_argmax")
 
@@ -93,9 +94,7 @@ def lib():
     L.spec_debug_read.argtypes = [vp, i32, i32, vp, sz]
     L.spec_debug_read.restype = i64
     L.spec_debug_read_kv.argtypes = [vp, i32, i32, i32, vp, vp]
-    L.spec_gemm_scratch_bytes.argtypes = [i32, i32, i32]
-    L.spec_gemm_scratch_bytes.restype = sz
-    L.spec_gemm.argtypes = [i32, i32, vp, vp, vp, i32, i32, i32, i32, vp, vp]
+    L.spec_gemm.argtypes = [i32, i32, vp, vp, vp, i32, i32, i32, i32, vp]
     L.spec_attn_scratch_bytes.argtypes = [i32, i32, i32, i32]
     L.spec_attn_scratch_bytes.restype = sz
     L.spec_attention.argtypes = [i32, i32, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, i32, vp, i32, i32, i32, i32, i32,
@@ -265,7 +264,14 @@ class SpecDecoder:
         self._check(lib().spec_profile_step(self.h, ms.ctypes.data, n.ctypes.data))
         return {c: (float(ms[i]), int(n[i])) for i, c in enumerate(self.PROF_CLASSES)}
 
-    TUNE_L2_LEAD_MB, TUNE_GEMM_CTAS, TUNE_DEBUG_LAUNCH_BUDGET, TUNE_ATTN_CTAS, TUNE_CHAIN_TIMING, TUNE_ATTN_UMMA = 1, 2, 3, 4, 5, 6
+    def kernel_stamps(self):
+        """FLAG_STAMPS: (uint64 [n][2] {inputs ready, last CTA left} in ns of the GPU timer, class names [n]) of the GEMM
+        and attention launches of the last step, in launch order."""
+        st = self.debug(DBG_STAMPS, 0).reshape(-1, 2)
+        cls = self.debug(DBG_STAMP_CLASS, 0)
+        return st, [self.PROF_CLASSES[c] for c in cls[: len(st)]]
+
+    TUNE_GEMM_CTAS, TUNE_DEBUG_LAUNCH_BUDGET, TUNE_ATTN_CTAS, TUNE_DEBUG_WAIT_RUNS_OUT, TUNE_ATTN_UMMA = 2, 3, 4, 5, 6
 
     def tune(self, what: int, value: int):
         self._check(lib().spec_tune(self.h, what, value))
@@ -301,18 +307,15 @@ class SpecDecoder:
 
 
 # ------------------------------------------------------------------ single kernels (tests, timing)
-def gemm(x: torch.Tensor, w: torch.Tensor, impl: int = 0, out: Optional[torch.Tensor] = None,
-         scratch: Optional[torch.Tensor] = None) -> torch.Tensor:
+def gemm(x: torch.Tensor, w: torch.Tensor, impl: int = 0, out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """out[r][o] = sum_i x[r][i] w[o][i] (fp32 out).  impl 0: tcgen05 kernel (bf16), 1: plain kernel."""
     rows, I = x.shape
     O = w.shape[0]
     assert w.shape[1] == I and x.is_contiguous() and w.is_contiguous() and x.dtype == w.dtype
     if out is None:
         out = torch.empty(rows, O, dtype=torch.float32, device=x.device)
-    if scratch is None:
-        scratch = torch.empty(max(64, lib().spec_gemm_scratch_bytes(rows, O, I)), dtype=torch.uint8, device=x.device)
     rc = lib().spec_gemm(_dt(x.dtype), impl, x.data_ptr(), w.data_ptr(), out.data_ptr(), rows, O, I, out.stride(0),
-                         scratch.data_ptr(), _stream_ptr(None))
+                         _stream_ptr(None))
     if rc:
         raise SpecError(rc, "spec_gemm")
     return out

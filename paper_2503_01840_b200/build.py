@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libspec_b200.so")
-SOURCES = ["api.cu", "elementwise.cu", "gemm_ref.cu", "gemm_fast.cu", "gemm_fused.cu", "gemm_chain.cu", "attn_ref.cu", "attn_fast.cu", "tree.cu"]
+SOURCES = ["api.cu", "elementwise.cu", "gemm_ref.cu", "tma_maps.cu", "gemm_fused.cu", "attn_ref.cu", "attn_fast.cu", "tree.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
          "--expt-relaxed-constexpr"]

@@ -10,9 +10,8 @@
 #include <vector>
 
 #include "../../include/spec_b200.h"
-#include "gemm_fast.cuh"
+#include "tma_maps.cuh"
 #include "gemm_fused.cuh"
-#include "gemm_chain.cuh"
 #include "attn_fast.cuh"
 #include "state.cuh"
 
@@ -43,7 +42,7 @@ static void launch_gather_rows(const float *src, const int32_t *src_row, float *
 
 static char g_init_err[256] = "";
 
-constexpr int MAX_CHAIN_LAUNCHES = 512;
+constexpr int MAX_STAMPS = 1024;   // stamped launches of one step (profiling aid)
 
 struct LayerW {
   const void *attn_norm, *wq, *wk, *wv, *wo, *mlp_norm, *w_gate, *w_up, *w_down;
@@ -92,31 +91,17 @@ struct spec_ctx {
   int32_t *best_idx = nullptr;
   void *topk_scratch = nullptr;
   int ktiles = 0, vtiles = 0;
-  // weights in the order one speculative step reads them (cyclic: the stream of the next step follows);
-  // every GEMM launch prefetches its share of the window [own end, own end + lead) into L2
-  struct WSeg { const void *ptr; size_t bytes; };
-  std::vector<WSeg> wstream;
-  std::vector<size_t> wcum;      // wcum[i] = bytes before entry i; wcum.back() = total
-  int wcur = -1;                 // stream entry of the next GEMM launch (-1: no prefetching)
-  size_t pf_front = 0;           // stream position up to which earlier launches of this step prefetched
-  size_t pf_lead = 0;             // bytes each launch keeps prefetched ahead (off by default: measured slower on B200)
-  // chain kernel: consecutive GEMMs of a pass run as one persistent kernel
-  bool chain = false;
-  float *chain_part = nullptr;     // split-K partial sums of the chain kernel
-  size_t chain_part_bytes = 0;
-  int32_t *chain_ctr = nullptr;    // [MAX_CHAIN_LAUNCHES][CHAIN_COUNTERS] grid-barrier counters, one block per launch of a step
-  int chain_idx = 0;
-  long long *chain_timing = nullptr;   // [CTAs][MAX_CHAIN_OPS][8] phase stamps of one chain launch (profiling aid)
-  int chain_timing_launch = -1;        // index of the chain launch of a step to record (-1: none)
+  // profiling aid (SPEC_FLAG_STAMPS): per stamped launch {earliest "inputs ready" time, latest CTA exit} in globaltimer ns
+  unsigned long long *stamps = nullptr;      // [MAX_STAMPS][2]
+  std::vector<int> stamp_cls;                // class of each stamped launch of the last scheduled step
+  int stamp_n = 0;
   int dbg_launch_budget = -1;   // debugging aid: kernels of the next step to run (-1: all)
-  void *gemm_scratch;
-  size_t gemm_scratch_bytes;
+  int dbg_withhold_spin = 0;    // test hook: > 0 makes one CTA of the verify LM-head GEMM run a bounded wait out after that many polls
   void *attn_scratch;
   size_t attn_scratch_bytes;
-  // split-K bookkeeping of the last GEMM into each buffer
+  // partial-sum bookkeeping of the plain (fp32 / debug) schedule: its GEMMs write one slice
   int np_proj = 1, np_qkv = 1, np_gu = 1;
   size_t ps_proj = 0, ps_qkv = 0, ps_gu = 0;
-  int smax_proj, smax_qkv, smax_gu;
   // host mirrors
   std::vector<int32_t> n_upper, cap_host, n_pages_host;
   std::vector<int32_t> page_table_host;
@@ -132,7 +117,7 @@ struct spec_ctx {
   std::vector<cudaEvent_t> prof_ev;
   std::vector<int> prof_cls;
   int prof_n = 0;
-  FastGemm *fg = nullptr;
+  TmaMaps *fg = nullptr;
   char err[256];
 };
 
@@ -189,14 +174,13 @@ static size_t carve(spec_ctx *c, void *base) {
   c->pps = (g.max_ctx + g.page_size - 1) / g.page_size;
   c->tail_tree = std::max(1, (c->D - 1) * c->K);
   c->need_pos = std::max(c->N, c->tail_tree) + 1;
-  c->smax_proj = 16; c->smax_qkv = 8; c->smax_gu = 4;
   int B = c->B, k = c->k, R = c->Ralloc, qd = c->H * c->hd, qkvd = (c->H + 2 * c->G) * c->hd;
   size_t e = c->esz;
   Carver cv(base);
   c->x = cv.take<float>((size_t)R * k);
-  c->proj = cv.take<float>((size_t)c->smax_proj * R * k);
-  c->qkv = cv.take<float>((size_t)c->smax_qkv * R * qkvd);
-  c->gu = cv.take<float>((size_t)c->smax_gu * R * 2 * c->F);
+  c->proj = cv.take<float>((size_t)R * k);
+  c->qkv = cv.take<float>((size_t)R * qkvd);
+  c->gu = cv.take<float>((size_t)R * 2 * c->F);
   c->logits = cv.take<float>((size_t)R * std::max(c->V, c->Vd));
   c->h = cv.take_bytes((size_t)R * k * e);
   c->q = cv.take_bytes((size_t)R * qd * e);
@@ -250,12 +234,7 @@ static size_t carve(spec_ctx *c, void *base) {
   c->best_val = cv.take<float>((size_t)c->vtiles * R);
   c->best_idx = cv.take<int32_t>((size_t)c->vtiles * R);
   c->topk_scratch = cv.take_bytes(topk_scratch_bytes(R, c->Vd, c->K));
-  c->chain_part_bytes = (R <= 64) ? ((size_t)64 << 20) : 0;
-  c->chain_part = c->chain_part_bytes ? (float *)cv.take_bytes(c->chain_part_bytes) : nullptr;
-  c->chain_ctr = cv.take<int32_t>((size_t)MAX_CHAIN_LAUNCHES * CHAIN_COUNTERS);
-  c->chain_timing = cv.take<long long>((size_t)1024 * MAX_CHAIN_OPS * 16);
-  c->gemm_scratch_bytes = 0;
-  c->gemm_scratch = nullptr;
+  c->stamps = (g.flags & SPEC_FLAG_STAMPS) ? cv.take<unsigned long long>((size_t)MAX_STAMPS * 2) : nullptr;
   c->attn_scratch_bytes = attn_fast_scratch_bytes(R, c->H, c->hd, g.max_ctx);
   c->attn_scratch = cv.take_bytes(c->attn_scratch_bytes);
   return (cv.off + 255) & ~(size_t)255;
@@ -319,32 +298,23 @@ extern "C" int spec_init(spec_ctx **out, const spec_target_weights *tw, const sp
   c->page_table_host.assign((size_t)c->B * c->pps, 0);
   if (cfg->dtype == SPEC_BF16 && !((cfg->flags & SPEC_FLAG_REF_GEMM))) {
     std::string why;
-    c->fg = fast_gemm_create(why);
+    c->fg = tma_maps_create(why);
     if (!c->fg) {
       int rc = fail(nullptr, SPEC_ERR_CUDA, "spec_init: tcgen05 GEMM set-up failed: %s", why.c_str());
       delete c;
       return rc;
     }
   }
-  c->fused = c->fg && !(cfg->flags & SPEC_FLAG_UNFUSED) && c->hd <= 128 && (c->hd & (c->hd - 1)) == 0 && c->Ralloc <= 256;
-  c->chain = c->fused && (cfg->flags & SPEC_FLAG_CHAIN) && c->chain_part != nullptr;
-  if (c->fused) {
-    size_t e = 2, k = c->k, qd = (size_t)c->H * c->hd, kvd = (size_t)c->G * c->hd, F = c->F;
-    auto push = [&](const void *p, size_t elems) { c->wstream.push_back({p, elems * e}); };
-    auto layer = [&](const LayerW &w) {
-      push(w.wq, qd * k); push(w.wk, kvd * k); push(w.wv, kvd * k); push(w.wo, k * qd);
-      push(w.w_gate, F * k); push(w.w_up, F * k); push(w.w_down, k * F);
-    };
-    push(c->fc3, k * 3 * k);
-    for (int d = 0; d < c->D; d++) { push(c->fc2, k * 2 * k); layer(c->dl); push(c->dlm_head, (size_t)c->Vd * k); }
-    for (int l = 0; l < c->L; l++) layer(c->tl[l]);
-    push(c->lm_head, (size_t)c->V * k);
-    c->wcum.assign(c->wstream.size() + 1, 0);
-    for (size_t i = 0; i < c->wstream.size(); i++) c->wcum[i + 1] = c->wcum[i] + c->wstream[i].bytes;
+  c->fused = c->fg != nullptr;
+  if (c->fg && !(c->hd <= 128 && (c->hd & (c->hd - 1)) == 0)) {
+    int rc = fail(nullptr, SPEC_ERR_UNSUPPORTED, "spec_init: the bf16 tensor-core path takes a power-of-two head_dim <= 128 (got %d)", c->hd);
+    tma_maps_destroy(c->fg);
+    delete c;
+    return rc;
   }
   if (c->fg && c->R > 256) {
     int rc = fail(nullptr, SPEC_ERR_UNSUPPORTED, "spec_init: %d rows per pass exceed the 256 the tensor-core GEMM takes", c->R);
-    fast_gemm_destroy(c->fg);
+    tma_maps_destroy(c->fg);
     delete c;
     return rc;
   }
@@ -356,7 +326,7 @@ extern "C" int spec_free(spec_ctx *c) {
   if (!c) return SPEC_OK;
   if (c->graph) cudaGraphExecDestroy(c->graph);
   if (c->graph_sampled) cudaGraphExecDestroy(c->graph_sampled);
-  if (c->fg) fast_gemm_destroy(c->fg);
+  if (c->fg) tma_maps_destroy(c->fg);
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   delete c;
   return SPEC_OK;
@@ -366,40 +336,17 @@ extern "C" int spec_free(spec_ctx *c) {
 template <typename T> struct Sched {
   spec_ctx *c;
   cudaStream_t s;
-  // GEMMs waiting to be launched as one chain kernel
-  std::vector<FusedEpi> ch_epi;
-  std::vector<FusedGemmArgs> ch_ops;
-  bool defer_flush = false;      // inside step(): chains may span the forward helpers; counters were zeroed at step start
   explicit Sched(spec_ctx *ctx) : c(ctx), s(ctx->stream) { tl_pdl = c->fused && !(c->cfg.flags & SPEC_FLAG_NO_PDL); }
-  ~Sched() { flush_chain(); tl_pdl = false; }
-  void flush_chain() {
-    if (ch_ops.empty()) return;
-    int n = (int)ch_ops.size();
-    int rc = -1;
-    prof_mark(SPEC_PROF_GEMM);
-    if (c->chain_idx < MAX_CHAIN_LAUNCHES) {
-      int32_t *ctr = c->chain_ctr + (size_t)c->chain_idx * CHAIN_COUNTERS;
-      if (!defer_flush) cudaMemsetAsync(ctr, 0, CHAIN_COUNTERS * sizeof(int32_t), s);
-      rc = chain_launch(c->fg, ch_epi.data(), ch_ops.data(), n, c->chain_part, c->chain_part_bytes, ctr, c->status, tl_pdl, s,
-                        (defer_flush && c->chain_idx == c->chain_timing_launch) ? c->chain_timing : nullptr);
-      if (rc == 0) { c->chain_idx++; tick(); }
-    }
-    if (rc != 0) {               // shapes the chain kernel does not take: one launch per GEMM
-      for (int i = 0; i < n; i++) {
-        int r2 = fused_gemm_launch(c->fg, ch_epi[i], ch_ops[i], s);
-        if (r2 && !c->sched_err) c->sched_err = r2;
-        tick();
-      }
-    }
-    ch_epi.clear();
-    ch_ops.clear();
-  }
+  ~Sched() { tl_pdl = false; }
   Sched(const Sched &) = delete;
   void tick(int n = 1) { c->launches += n; }
   // profiling: one event at the start of every launch; the interval to the next event is charged to `cls`
-  void mark(int cls) {
-    if (cls != SPEC_PROF_GEMM) flush_chain();      // a non-GEMM kernel follows: it needs the pending GEMMs' results
-    prof_mark(cls);
+  void mark(int cls) { prof_mark(cls); }
+  // profiling aid: the next stamped launch's slot (nullptr when stamps are off or the step has more launches than slots)
+  unsigned long long *next_stamp(int cls) {
+    if (!c->stamps || c->stamp_n >= MAX_STAMPS) return nullptr;
+    c->stamp_cls.push_back(cls);
+    return c->stamps + 2 * (size_t)c->stamp_n++;
   }
   void prof_mark(int cls) {
     if (!c->prof) return;
@@ -415,18 +362,14 @@ template <typename T> struct Sched {
   }
 
   // number of split-K slices for a weight of shape [O][I] whose output buffer holds smax slices
-  int pick(int O, int I, int smax) const { return c->fg ? fast_gemm_pick_split(O, I, smax) : 1; }
+  int pick(int, int, int) const { return 1; }
   size_t pstride(int ldo) const { return (size_t)c->Ralloc * ldo; }
 
   // S fp32 partial slices of x . w^T into columns [col0, col0+O) of `out` (row pitch ldo)
   void gemm(const void *x, const void *w, float *out, int rows, int O, int I, int ldo, int col0, int S) {
     mark(SPEC_PROF_GEMM);
-    if (c->fg) {
-      int rc = fast_gemm_run(c->fg, (const bf16 *)x, (const bf16 *)w, out + col0, rows, O, I, ldo, pstride(ldo), S, c->status, s);
-      if (rc && !c->sched_err) c->sched_err = rc;
-    } else {
-      launch_gemm_ref<T>((const T *)x, (const T *)w, out + col0, rows, O, I, ldo, s);
-    }
+    (void)S;
+    launch_gemm_ref<T>((const T *)x, (const T *)w, out + col0, rows, O, I, ldo, s);
     tick();
   }
 
@@ -440,41 +383,9 @@ template <typename T> struct Sched {
   void with_norm_scale(FusedGemmArgs &a) const {
     a.ssq_in = c->ssq; a.ssq_in_tiles = c->ktiles; a.ssq_ld = c->Ralloc; a.k_in = c->k; a.eps = c->cfg.rms_eps;
   }
-  // Assigns this launch its share of the L2 prefetch window and advances the stream cursor.
-  void assign_prefetch(FusedGemmArgs &a) {
-    if (c->wcur < 0 || c->pf_lead == 0) return;
-    const int n = (int)c->wstream.size();
-    if (c->wcur + a.nw > n || c->wstream[c->wcur].ptr != (const void *)a.w[0]) { c->wcur = -1; return; }   // not the step's order
-    const size_t total = c->wcum[n];
-    const size_t own_end = c->wcum[c->wcur + a.nw];
-    size_t lo = std::max(own_end, c->pf_front), hi = own_end + c->pf_lead;
-    c->wcur += a.nw;
-    if (hi <= lo) return;
-    // entries overlapping [lo, hi) in the cyclic stream
-    size_t pos = lo;
-    int idx = (int)(std::upper_bound(c->wcum.begin(), c->wcum.end(), pos % total) - c->wcum.begin()) - 1;
-    while (pos < hi && a.npf < FusedGemmArgs::MAX_PREFETCH) {
-      idx %= n;
-      size_t seg_lo = pos % total - c->wcum[idx];
-      size_t take = std::min(c->wstream[idx].bytes - seg_lo, hi - pos);
-      a.pf_ptr[a.npf] = (const char *)c->wstream[idx].ptr + seg_lo;
-      a.pf_bytes[a.npf] = take;
-      a.npf++;
-      pos += take;
-      idx++;
-    }
-    c->pf_front = pos;
-  }
   void fgemm(FusedEpi epi, FusedGemmArgs a) {
-    if (c->chain && epi != EPI_ARGMAX && a.rows <= 64) {
-      if (!ch_ops.empty() && ((int)ch_ops.size() == MAX_CHAIN_OPS || ch_ops[0].rows != a.rows)) flush_chain();
-      ch_epi.push_back(epi);
-      ch_ops.push_back(a);
-      return;
-    }
-    flush_chain();
     prof_mark(SPEC_PROF_GEMM);
-    assign_prefetch(a);
+    a.stamp = next_stamp(SPEC_PROF_GEMM);
     int rc = fused_gemm_launch(c->fg, epi, a, s);
     if (rc && !c->sched_err) c->sched_err = rc;
     tick();
@@ -520,10 +431,10 @@ template <typename T> struct Sched {
       with_norm_scale(a);
       a.best_val = c->best_val; a.best_idx = c->best_idx; a.best_ld = c->Ralloc;
       if (c->cap_logits || c->sampled) { a.out_f32 = c->logits; a.ldo = c->V; }
+      if (c->dbg_withhold_spin > 0) { a.withhold = true; a.spin_limit = (unsigned)c->dbg_withhold_spin; }
       fgemm(EPI_ARGMAX, a);
       mark(SPEC_PROF_ARGMAX); launch_argmax_merge(c->best_val, c->best_idx, c->vtiles, c->Ralloc, rows, c->tb.y, s); tick();
     }
-    if (!defer_flush) flush_chain();
   }
   void fuse_fused(const void *taps, int rows) {
     FusedGemmArgs a = fargs(taps, rows, 3 * c->k);
@@ -531,7 +442,6 @@ template <typename T> struct Sched {
     a.out_f32 = c->proj; a.ldo = c->k;
     fgemm(EPI_F32, a);
     c->np_proj = 1; c->ps_proj = 0;
-    if (!defer_flush) flush_chain();
   }
   void draft_forward_fused(const float *feat, int nparts, size_t fstride, const int32_t *src_row, int rows, int tail_len) {
     mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
@@ -540,7 +450,6 @@ template <typename T> struct Sched {
     tick();
     fgemm_resid(c->cat, 2 * c->k, c->fc2, rows, false, c->dl.attn_norm, 0);
     block_fused(c->dl, c->pools[c->L], rows, tail_len, c->dfinal_norm, 0);
-    if (!defer_flush) flush_chain();
   }
   void draft_logits_fused(int rows) {
     FusedGemmArgs a = fargs(c->h, rows, c->k);
@@ -564,7 +473,7 @@ template <typename T> struct Sched {
       for (int b = 0; b < c->B; b++) hint = std::max(hint, c->n_upper[b]);
       tick(launch_attn_fast((const bf16 *)c->q, pool, pm, c->meta, tail_len, (bf16 *)c->ao, rows, c->H, c->G, c->hd,
                             c->cur_rps, hint, c->attn_scratch, s, !(c->cfg.flags & SPEC_FLAG_NO_TMA_ATTN), c->status,
-                            c->st.order, c->B));
+                            c->st.order, c->B, next_stamp(SPEC_PROF_ATTN)));
     } else {
       launch_attn_ref<T>((const T *)c->q, pool, pm, c->meta, tail_len, (T *)c->ao, rows, c->H, c->G, c->hd,
                          c->cfg.max_ctx + tail_len, s);
@@ -580,24 +489,24 @@ template <typename T> struct Sched {
     mark(SPEC_PROF_NORM); launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, first_mode, (T *)c->node_taps, tap_mask, (const T *)w.attn_norm,
                        c->cfg.rms_eps, (T *)c->h, nullptr, rows, rows, k, s);
     tick();
-    c->np_qkv = pick(qd, k, c->smax_qkv); c->ps_qkv = pstride(qkvd);
+    c->np_qkv = pick(qd, k, 1); c->ps_qkv = pstride(qkvd);
     gemm(c->h, w.wq, c->qkv, rows, qd, k, qkvd, 0, c->np_qkv);
     gemm(c->h, w.wk, c->qkv, rows, kvd, k, qkvd, qd, c->np_qkv);
     gemm(c->h, w.wv, c->qkv, rows, kvd, k, qkvd, qd + kvd, c->np_qkv);
     mark(SPEC_PROF_ROPE_KV); launch_rope_kv<T>(c->qkv, c->np_qkv, c->ps_qkv, c->cs, c->meta, (T *)c->q, pool, pm, rows, c->H, c->G, c->hd, c->status, s);
     tick();
     attention(pool, rows, tail_len);
-    c->np_proj = pick(k, qd, c->smax_proj); c->ps_proj = pstride(k);
+    c->np_proj = pick(k, qd, 1); c->ps_proj = pstride(k);
     gemm(c->ao, w.wo, c->proj, rows, k, qd, k, 0, c->np_proj);
     mark(SPEC_PROF_NORM); launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, 2, (T *)nullptr, 0, (const T *)w.mlp_norm, c->cfg.rms_eps,
                        (T *)c->h, nullptr, rows, rows, k, s);
     tick();
-    c->np_gu = pick(F, k, c->smax_gu); c->ps_gu = pstride(2 * F);
+    c->np_gu = pick(F, k, 1); c->ps_gu = pstride(2 * F);
     gemm(c->h, w.w_gate, c->gu, rows, F, k, 2 * F, 0, c->np_gu);
     gemm(c->h, w.w_up, c->gu, rows, F, k, 2 * F, F, c->np_gu);
     mark(SPEC_PROF_ACT); launch_silu_mul<T>(c->gu, c->np_gu, c->ps_gu, (T *)c->act, rows, F, s);
     tick();
-    c->np_proj = pick(k, F, c->smax_proj); c->ps_proj = pstride(k);
+    c->np_proj = pick(k, F, 1); c->ps_proj = pstride(k);
     gemm(c->act, w.w_down, c->proj, rows, k, F, k, 0, c->np_proj);
   }
 
@@ -626,7 +535,7 @@ template <typename T> struct Sched {
   // FC3 over `rows` rows of taps -> proj (Section 3.1: g = FC([l;m;h]))
   void fuse(const void *taps, int rows) {
     if (c->fused) return fuse_fused(taps, rows);
-    c->np_proj = pick(c->k, 3 * c->k, c->smax_proj); c->ps_proj = pstride(c->k);
+    c->np_proj = pick(c->k, 3 * c->k, 1); c->ps_proj = pstride(c->k);
     gemm(taps, c->fc3, c->proj, rows, c->k, 3 * c->k, c->k, 0, c->np_proj);
   }
 
@@ -636,7 +545,7 @@ template <typename T> struct Sched {
     mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
     mark(SPEC_PROF_MISC); launch_build_cat<T>(feat, nparts, fstride, src_row, (const T *)c->embed, c->meta.tok, c->meta.seq, (T *)c->cat, rows, c->k, s);
     tick();
-    c->np_proj = pick(c->k, 2 * c->k, c->smax_proj); c->ps_proj = pstride(c->k);
+    c->np_proj = pick(c->k, 2 * c->k, 1); c->ps_proj = pstride(c->k);
     gemm(c->cat, c->fc2, c->proj, rows, c->k, 2 * c->k, c->k, 0, c->np_proj);
     block(c->dl, c->pools[c->L], rows, tail_len, 1, 0);
     mark(SPEC_PROF_NORM); launch_add_norm<T>(c->x, c->proj, c->np_proj, c->ps_proj, 2, (T *)nullptr, 0, (const T *)c->dfinal_norm, c->cfg.rms_eps,
@@ -666,14 +575,11 @@ template <typename T> struct Sched {
 
   void step(bool plain) {
     int rows = plain ? c->B : c->Tv, rps = plain ? 1 : c->N;
-    // the previous step's last launches already covered the first `lead` bytes of this step's stream
-    c->wcur = (!plain && c->fused) ? 0 : -1;
-    c->pf_front = c->pf_lead;
     tl_launch_budget = c->dbg_launch_budget;
-    if (c->chain) {              // one block of barrier counters per chain launch of the step, all zeroed up front
-      cudaMemsetAsync(c->chain_ctr, 0, (size_t)MAX_CHAIN_LAUNCHES * CHAIN_COUNTERS * sizeof(int32_t), s);
-      c->chain_idx = 0;
-      defer_flush = true;
+    c->stamp_n = 0;
+    c->stamp_cls.clear();
+    if (c->stamps) {             // earliest times start at the largest value, latest at zero
+      cudaMemsetAsync(c->stamps, 0xff, (size_t)MAX_STAMPS * 2 * sizeof(unsigned long long), s);
     }
     if (!plain) {
       mark(SPEC_PROF_TREE); launch_prep_extend(c->st, c->tb, c->meta, c->B, c->need_pos, c->status, s); tick();
@@ -707,8 +613,6 @@ template <typename T> struct Sched {
                      c->k, rps, s);
     tick();
     mark(-1);
-    defer_flush = false;
-    c->wcur = -1;
     tl_launch_budget = -1;
   }
 };
@@ -970,19 +874,17 @@ extern "C" int spec_profile_step(spec_ctx *c, float *class_ms, int32_t *class_la
 
 extern "C" int spec_tune(spec_ctx *c, int32_t what, int32_t value) {
   if (!c) return SPEC_ERR_NULL;
-  if (what == SPEC_TUNE_L2_LEAD_MB) {
-    if (value < 0 || value > 120) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the L2 prefetch distance must be 0..120 MB");
-    c->pf_lead = (size_t)value << 20;
-  } else if (what == SPEC_TUNE_ATTN_CTAS) {
+  if (what == SPEC_TUNE_ATTN_CTAS) {
     if (value < 1 || value > 4096) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the attention CTA target must be 1..4096");
     attn_fast_set_target_ctas(value);
   } else if (what == SPEC_TUNE_ATTN_UMMA) {
     if (value < 0 || value > 2) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the tcgen05 attention mode must be 0, 1 or 2");
     attn_fast_set_umma(value);
-  } else if (what == SPEC_TUNE_CHAIN_TIMING) {
-    c->chain_timing_launch = value;
   } else if (what == SPEC_TUNE_DEBUG_LAUNCH_BUDGET) {
     c->dbg_launch_budget = value;
+  } else if (what == SPEC_TUNE_DEBUG_WAIT_RUNS_OUT) {
+    if (value < 0 || value > (1 << 20)) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the poll count must be 0..2^20");
+    c->dbg_withhold_spin = value;
   } else if (what == SPEC_TUNE_GEMM_CTAS) {
     if (value < 32 || value > 2048) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the GEMM CTA target must be 32..2048");
     fused_gemm_set_target_ctas(value);
@@ -1083,7 +985,14 @@ extern "C" int64_t spec_debug_read(spec_ctx *c, int32_t what, int32_t seq, void 
     case SPEC_DBG_RAW_ACT: return copy_widen(c, c->act, (size_t)c->Ralloc * c->F, dst, bytes);
     case SPEC_DBG_RAW_CAT: return copy_widen(c, c->cat, (size_t)c->Ralloc * 2 * c->k, dst, bytes);
     case SPEC_DBG_RAW_SSQ: return copy_out(c, c->ssq, (size_t)c->ktiles * c->Ralloc, dst, bytes);
-    case SPEC_DBG_CHAIN_TIMING: return copy_out(c, c->chain_timing, (size_t)chain_ctas() * MAX_CHAIN_OPS * 16, dst, bytes);
+    case SPEC_DBG_STAMPS:
+      if (!c->stamps) return fail(c, SPEC_ERR_STATE, "spec_debug_read: kernel stamps need SPEC_FLAG_STAMPS");
+      return copy_out(c, c->stamps, (size_t)c->stamp_n * 2, dst, bytes);
+    case SPEC_DBG_STAMP_CLASS: {
+      size_t avail = c->stamp_cls.size() * sizeof(int32_t);
+      if (dst && bytes) memcpy(dst, c->stamp_cls.data(), std::min(avail, bytes));
+      return (int64_t)avail;
+    }
     case SPEC_DBG_RAW_LOGITS: return copy_out(c, c->logits, (size_t)c->Ralloc * c->Vd, dst, bytes);
     default: return fail(c, SPEC_ERR_INVALID_CFG, "spec_debug_read: unknown item %d", what);
   }
@@ -1106,12 +1015,9 @@ extern "C" int spec_debug_read_kv(spec_ctx *c, int32_t seq, int32_t layer, int32
 }
 
 // ------------------------------------------------------------------------------------------ single kernels
-extern "C" size_t spec_gemm_scratch_bytes(int32_t rows, int32_t out, int32_t in) {
-  return fast_gemm_scratch_bytes(rows, out, in);
-}
 
 extern "C" int spec_gemm(int32_t dtype, int32_t impl, const void *x, const void *w, float *out, int32_t rows, int32_t O,
-                         int32_t I, int32_t ldo, void *scratch, void *stream) {
+                         int32_t I, int32_t ldo, void *stream) {
   if (!x || !w || !out) return SPEC_ERR_NULL;
   if (rows < 1 || O < 1 || I < 1 || ldo < O) return SPEC_ERR_INVALID_CFG;
   cudaStream_t s = (cudaStream_t)stream;
@@ -1122,17 +1028,17 @@ extern "C" int spec_gemm(int32_t dtype, int32_t impl, const void *x, const void 
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
   }
   if (dtype != SPEC_BF16) return SPEC_ERR_UNSUPPORTED;
-  return fast_gemm_oneshot((const bf16 *)x, (const bf16 *)w, out, rows, O, I, ldo, scratch, s);
+  return spec_gemm_fused(x, w, out, rows, O, I, ldo, 0, 0, stream);
 }
 
 extern "C" int spec_gemm_fused(const void *x, const void *w, float *out, int32_t rows, int32_t O, int32_t I, int32_t ldo,
                                int32_t split, int32_t stages, void *stream) {
   if (!x || !w || !out) return SPEC_ERR_NULL;
   if (rows < 1 || O < 1 || I < 1 || ldo < O || split < 0 || stages < 0) return SPEC_ERR_INVALID_CFG;
-  static FastGemm *g = nullptr;
+  static TmaMaps *g = nullptr;
   if (!g) {
     std::string why;
-    g = fast_gemm_create(why);
+    g = tma_maps_create(why);
     if (!g) return SPEC_ERR_CUDA;
   }
   FusedGemmArgs a;
@@ -1140,7 +1046,7 @@ extern "C" int spec_gemm_fused(const void *x, const void *w, float *out, int32_t
   a.out_f32 = out; a.ldo = ldo; a.split = split; a.stages = stages;
   if (!fused_gemm_supported(EPI_F32, a)) return SPEC_ERR_UNSUPPORTED;
   int rc = fused_gemm_launch(g, EPI_F32, a, (cudaStream_t)stream);
-  fast_gemm_forget(g);   // test buffers come and go; do not keep descriptors of freed memory
+  tma_maps_forget(g);   // test buffers come and go; do not keep descriptors of freed memory
   if (rc) return rc == -1 ? SPEC_ERR_INVALID_CFG : SPEC_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }
@@ -1149,10 +1055,10 @@ extern "C" int spec_gemm_swiglu(const void *x, const void *w_gate, const void *w
                                 void *stream) {
   if (!x || !w_gate || !w_up || !act) return SPEC_ERR_NULL;
   if (rows < 1 || F < 1 || I < 1) return SPEC_ERR_INVALID_CFG;
-  static FastGemm *g = nullptr;
+  static TmaMaps *g = nullptr;
   if (!g) {
     std::string why;
-    g = fast_gemm_create(why);
+    g = tma_maps_create(why);
     if (!g) return SPEC_ERR_CUDA;
   }
   FusedGemmArgs a;
@@ -1161,7 +1067,7 @@ extern "C" int spec_gemm_swiglu(const void *x, const void *w_gate, const void *w
   a.act = (bf16 *)act;
   if (!fused_gemm_supported(EPI_SWIGLU, a)) return SPEC_ERR_UNSUPPORTED;
   int rc = fused_gemm_launch(g, EPI_SWIGLU, a, (cudaStream_t)stream);
-  fast_gemm_forget(g);
+  tma_maps_forget(g);
   if (rc) return rc == -1 ? SPEC_ERR_INVALID_CFG : SPEC_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }

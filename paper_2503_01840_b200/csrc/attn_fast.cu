@@ -87,12 +87,14 @@ struct AttnParams {
   float *part_o;    // [nsplit][rows*H][hd]
   float *part_ml;   // [nsplit][rows*H][2]
   const int32_t *order;   // row block handled by the i-th CTA group (nullptr: i)
+  unsigned long long *stamp;   // profiling aid (see KernelStamp), may be null
 };
 
 template <int HD>
 __global__ void __launch_bounds__(256) attn_mma_kernel(AttnParams p) {
   pdl_wait();
   pdl_trigger();
+  KernelStamp stamp_guard(p.stamp);
   constexpr int ROWB = HD * 2, CPR = HD / 8;          // bytes / 16-byte chunks per row
   constexpr int NKS = HD / 16;                        // k-steps of Q K^T
   extern __shared__ __align__(128) unsigned char sm[];
@@ -323,6 +325,7 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
                                                        const __grid_constant__ CUtensorMap map_v, AttnParams p, int32_t *status) {
   pdl_wait();
   pdl_trigger();
+  KernelStamp stamp_guard(p.stamp);
   constexpr int ROWB = HD * 2, CPR = HD / 8;
   constexpr int NKS = HD / 16;
   constexpr int TILEB = KT * ROWB;                     // bytes of one K (or V) tile
@@ -612,6 +615,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
                                                         const __grid_constant__ CUtensorMap map_v, AttnParams p, int32_t *status) {
   pdl_wait();
   pdl_trigger();
+  KernelStamp stamp_guard(p.stamp);
   constexpr int HD = UM_HD;
   extern __shared__ __align__(1024) unsigned char sm[];
   unsigned char *sQ = sm;                                   // [2 halves][128 rows][128 B]
@@ -919,6 +923,7 @@ __global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_consta
                                                              const __grid_constant__ CUtensorMap map_v, AttnParams p, int32_t *status) {
   pdl_wait();
   pdl_trigger();
+  KernelStamp stamp_guard(p.stamp);
   constexpr int ROWB = HD * 2, CPR = HD / 8;
   constexpr int NKS = HD / 16;
   constexpr int TILEB = KT * ROWB;
@@ -1120,9 +1125,10 @@ __global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_consta
 // loads of eight splits in flight.
 template <int HD>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, int nsplit,
-                                                           int nrh, bf16 *__restrict__ out) {
+                                                           int nrh, bf16 *__restrict__ out, unsigned long long *stamp) {
   pdl_wait();
   pdl_trigger();
+  KernelStamp stamp_guard(stamp, false);
   constexpr int DPL = HD / 32;                              // dimensions per lane
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rh = blockIdx.x * 8 + warp;
@@ -1272,7 +1278,7 @@ void attn_fast_override_umma(int v) { tl_attn_umma = v; }
 
 int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail_len, bf16 *out, int rows, int H, int G,
                      int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s, bool contiguous_tail, int32_t *status,
-                     const int32_t *order, int order_len) {
+                     const int32_t *order, int order_len, unsigned long long *stamp) {
   if (rps < 1 || rows % rps) rps = 1;
   int seqs = rows / rps, grp = H / G;
   int mtiles = (rps * grp + MT - 1) / MT;
@@ -1283,6 +1289,7 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
   p.rows = rows; p.H = H; p.G = G; p.rps = rps; p.nsplit = nsplit; p.out = out;
   p.part_o = (float *)scratch;
   p.order = (order && order_len == seqs) ? order : nullptr;
+  p.stamp = stamp;
   p.part_ml = p.part_o ? p.part_o + (size_t)MAX_SPLITS * rows * H * hd : nullptr;
   dim3 grid(mtiles, nsplit, seqs * G);
   // TMA-staged kernel when the tail follows the context and a page is a whole number of 128-byte-swizzle boxes
@@ -1295,8 +1302,8 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
       int rc = umma ? launch_umma(p, grid, mk, mv, status, s) : hd == 128 ? launch_tma<128>(p, grid, mk, mv, status, s) : launch_tma<64>(p, grid, mk, mv, status, s);
       if (rc == 0) {
         if (nsplit > 1) {
-          if (hd == 128) launch_k(attn_combine_kernel<128>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
-          else launch_k(attn_combine_kernel<64>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
+          if (hd == 128) launch_k(attn_combine_kernel<128>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out, p.stamp);
+          else launch_k(attn_combine_kernel<64>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out, p.stamp);
         }
         return nsplit > 1 ? 2 : 1;
       }
@@ -1308,11 +1315,11 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
   if (hd == 128) {
     if (!limit[1].ensure(attn_mma_kernel<128>, (int)smem)) return -1;
     launch_k(attn_mma_kernel<128>, grid, dim3(256), smem, s, p);
-    if (nsplit > 1) launch_k(attn_combine_kernel<128>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
+    if (nsplit > 1) launch_k(attn_combine_kernel<128>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out, p.stamp);
   } else {
     if (!limit[0].ensure(attn_mma_kernel<64>, (int)smem)) return -1;
     launch_k(attn_mma_kernel<64>, grid, dim3(256), smem, s, p);
-    if (nsplit > 1) launch_k(attn_combine_kernel<64>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out);
+    if (nsplit > 1) launch_k(attn_combine_kernel<64>, dim3((rows * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, out, p.stamp);
   }
   return nsplit > 1 ? 2 : 1;
 }

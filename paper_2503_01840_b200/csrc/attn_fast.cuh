@@ -11,11 +11,13 @@ size_t attn_fast_scratch_bytes(int rows, int n_heads, int head_dim, int max_ctx)
 // split).  Returns the number of kernels launched.
 int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail_len, bf16 *out, int rows, int H, int G,
                      int hd, int rps, int ctx_hint, void *scratch, cudaStream_t s, bool contiguous_tail = false,
-                     int32_t *status = nullptr, const int32_t *order = nullptr, int order_len = 0);
+                     int32_t *status = nullptr, const int32_t *order = nullptr, int order_len = 0,
+                     unsigned long long *stamp = nullptr);
 // contiguous_tail: every row's tail_base equals its ctx (the tail keys follow the context in the cache), which lets the
 // TMA-staged kernel fetch whole pages; status: device status words for its bounded waits (may be NULL).
 // order: a permutation of the rows / rps row blocks (device, order_len entries; used when order_len == rows / rps): the
 // TMA-staged kernels give block order[i] to the i-th group of CTAs, e.g. longest sequence first.
+// stamp: profiling aid, see KernelStamp (may be NULL).
 // Drops the cached K/V tensor maps (pools of one-shot callers come and go).
 void attn_fast_forget_maps();
 // CTAs an attention launch aims at when it splits the keys (process-wide; default 148 = one wave)

@@ -27,6 +27,24 @@ __device__ __forceinline__ void set_status(int32_t *st, int code, int where, int
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Profiling aid: the GPU's global nanosecond timer, and a guard that records into stamp[0] the earliest time a CTA
+// of the launch got past its dependency wait and into stamp[1] the latest time a warp of the launch left the kernel
+// (early returns included).  A null pointer switches it off.
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+struct KernelStamp {
+  unsigned long long *p;
+  __device__ __forceinline__ KernelStamp(unsigned long long *stamp, bool start = true) : p(stamp) {
+    if (p && start && threadIdx.x == 0) atomicMin(p, global_ns());
+  }
+  __device__ __forceinline__ ~KernelStamp() {
+    if (p && (threadIdx.x & 31) == 0) atomicMax(p + 1, global_ns());
+  }
+};
+
 // When set (per host thread, by the step scheduler), launch_k adds the programmatic-dependent-launch
 // attribute to every launch.
 extern thread_local bool tl_pdl;

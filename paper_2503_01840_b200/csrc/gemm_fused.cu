@@ -55,13 +55,11 @@ struct alignas(64) FusedParams {
   const float2 *cs; RowMeta m; bf16 *q; KvPool pool; PageMap pm; int H, G, hd;
   bf16 *act;
   float *best_val; int32_t *best_idx; int best_ld;
-  const unsigned char *pf_ptr[FusedGemmArgs::MAX_PREFETCH];
-  unsigned long long pf_bytes[FusedGemmArgs::MAX_PREFETCH];
-  int npf;
   int32_t *status;
+  unsigned long long *stamp;
+  unsigned spin;               // polls before a wait gives up
+  int withhold;                // test hook: CTA 0 leaves out the activation load of its first k-block
 };
-
-constexpr unsigned PF_CHUNK = 32768;   // bytes per L2 prefetch instruction
 
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
@@ -127,6 +125,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
   uint64_t *acc_bar = empty + MAX_STAGES;
   uint32_t *tmem_slot = (uint32_t *)(acc_bar + 1);
   volatile uint32_t *abort_flag = tmem_slot + 1;
+  volatile int *n_issued = (volatile int *)(tmem_slot + 2), *n_consumed = (volatile int *)(tmem_slot + 3);   // stage loads issued / seen complete
   float *inv_s = (float *)(ctrl + 512);          // [256] per-row input scale
   float *wpart = inv_s + 256;                    // [4][MAX_CHUNK] per-warp partial sums / argmax exchange
 
@@ -148,6 +147,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
     for (int i = 0; i < stages; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     mbar_init(acc_bar, 1);
     *abort_flag = 0;
+    *n_issued = 0; *n_consumed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {   // TMEM allocation is a whole-warp operation
@@ -173,30 +173,20 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       if (PAIR) tma_load_2d_hint(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[i], pol);
     }
     pdl_wait();
-    for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + A_TILES * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
+    if (p.stamp) atomicMin(p.stamp, global_ns());
+    const bool hold = p.withhold && blockIdx.x == 0 && blockIdx.y == 0;     // test hook: the first stage never completes
+    for (int i = hold ? 1 : 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + A_TILES * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
+    *n_issued = npre;
     for (int i = npre; i < nkb; i++) {
       int st = i % stages;
-      if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
+      if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
       if (*abort_flag) break;
       unsigned char *a = tiles + st * STAGE;
       mbar_expect_tx(&full[st], STAGE);
       tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
       if (PAIR) tma_load_2d_hint(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
       tma_load_2d(a + A_TILES * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[st]);
-    }
-    // all of this CTA's loads are issued: pull the first weights of the launches that follow into L2, so that
-    // the memory system stays busy across this kernel's epilogue and the next kernel's start-up
-    if (p.npf > 0) {
-      const unsigned ncta = gridDim.x * gridDim.y, me = blockIdx.y * gridDim.x + blockIdx.x;
-      for (int sgm = 0; sgm < p.npf; sgm++) {
-        const unsigned long long nb = p.pf_bytes[sgm];
-        const unsigned long long nch = (nb + PF_CHUNK - 1) / PF_CHUNK;
-        for (unsigned long long ch = me; ch < nch; ch += ncta) {
-          unsigned long long off = ch * PF_CHUNK;
-          unsigned len = (unsigned)((nb - off < PF_CHUNK) ? nb - off : PF_CHUNK);
-          l2_prefetch_bulk(p.pf_ptr[sgm] + off, len);
-        }
-      }
+      *n_issued = i + 1;
     }
   } else {
     pdl_wait();
@@ -205,7 +195,8 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       constexpr uint32_t idesc = umma_idesc(NT);
       for (int i = 0; i < nkb; i++) {
         int st = i % stages;
-        if (!mbar_wait(&full[st], (i / stages) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 201, blockIdx.x, i); break; }
+        if (!mbar_wait(&full[st], (i / stages) & 1, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 201, blockIdx.x, i); break; }
+        *n_consumed = i + 1;
         if (*abort_flag) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         uint32_t a = smem_u32(tiles + st * STAGE), b = a + A_TILES * A_BYTES;
@@ -236,8 +227,8 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
   // ---- wait for the accumulator (one bounded wait per warp)
   int good = 0;
   if (lane == 0) {
-    bool ok = mbar_wait(acc_bar, 0);
-    if (!ok) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 202, blockIdx.x, slice); }
+    bool ok = *abort_flag ? false : mbar_wait(acc_bar, 0, p.spin);    // after an abort the accumulator never completes
+    if (!ok && !*abort_flag) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 202, blockIdx.x, slice); }
     good = (ok && !*abort_flag) ? 1 : 0;
   }
   good = __shfl_sync(0xffffffffu, good, 0);
@@ -421,11 +412,17 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
     // peers may still be reading this CTA's red; nobody overwrites or leaves before all are done
     if (S > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); else __syncthreads();
   }
+  if (*abort_flag && threadIdx.x == 0) {
+    // gave up on a wait: no bulk copy may still be landing in this CTA's shared memory when it exits.  Every stage
+    // load that was issued and not seen complete is waited for (bounded; a load that was never issued runs the wait out).
+    for (int i = *n_consumed; i < *n_issued; i++) mbar_wait(&full[i % stages], (i / stages) & 1, p.spin);
+  }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
+  if (p.stamp && threadIdx.x == 0) atomicMax(p.stamp + 1, global_ns());
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -449,6 +446,7 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
   uint64_t *acc_bar = empty + MAX_STAGES;
   uint32_t *tmem_slot = (uint32_t *)(acc_bar + 1);
   volatile uint32_t *abort_flag = tmem_slot + 1;
+  volatile int *n_issued = (volatile int *)(tmem_slot + 2), *n_consumed = (volatile int *)(tmem_slot + 3);
   float *inv_s = (float *)(ctrl + 512);          // [256] per-row input scale
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -459,6 +457,7 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
     for (int i = 0; i < stages; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     mbar_init(acc_bar, 1);
     *abort_flag = 0;
+    *n_issued = 0; *n_consumed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -483,16 +482,19 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
       tma_load_2d_hint(a + A_BYTES, &p.map_w[1], i * TILE_K, tm * TILE_M, &full[i], pol);
     }
     pdl_wait();
+    if (p.stamp) atomicMin(p.stamp, global_ns());
     for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + 2 * A_BYTES, &p.map_x, i * TILE_K, 0, &full[i]);
+    *n_issued = npre;
     for (int i = npre; i < KB; i++) {
       const int st = i % stages;
-      if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 220, blockIdx.x, i); break; }
+      if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 220, blockIdx.x, i); break; }
       if (*abort_flag) break;
       unsigned char *a = tiles + st * STAGE;
       mbar_expect_tx(&full[st], STAGE);
       tma_load_2d_hint(a, &p.map_w[0], i * TILE_K, tm * TILE_M, &full[st], pol);
       tma_load_2d_hint(a + A_BYTES, &p.map_w[1], i * TILE_K, tm * TILE_M, &full[st], pol);
       tma_load_2d(a + 2 * A_BYTES, &p.map_x, i * TILE_K, 0, &full[st]);
+      *n_issued = i + 1;
     }
   } else {
     pdl_wait();
@@ -501,7 +503,8 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
       constexpr uint32_t idesc = umma_idesc(NT);
       for (int i = 0; i < KB; i++) {
         const int st = i % stages;
-        if (!mbar_wait(&full[st], (i / stages) & 1)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 221, blockIdx.x, i); break; }
+        if (!mbar_wait(&full[st], (i / stages) & 1, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 221, blockIdx.x, i); break; }
+        *n_consumed = i + 1;
         if (*abort_flag) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t ag = smem_u32(tiles + st * STAGE), au = ag + A_BYTES, b = ag + 2 * A_BYTES;
@@ -530,8 +533,8 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
 
   int good = 0;
   if (lane == 0) {
-    bool ok = mbar_wait(acc_bar, 0);
-    if (!ok) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 222, blockIdx.x, 0); }
+    bool ok = *abort_flag ? false : mbar_wait(acc_bar, 0, p.spin);
+    if (!ok && !*abort_flag) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 222, blockIdx.x, 0); }
     good = (ok && !*abort_flag) ? 1 : 0;
   }
   good = __shfl_sync(0xffffffffu, good, 0);
@@ -558,12 +561,16 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
       }
     }
   }
+  if (*abort_flag && threadIdx.x == 0) {      // no bulk copy may still be landing when the CTA exits
+    for (int i = *n_consumed; i < *n_issued; i++) mbar_wait(&full[i % stages], (i / stages) & 1, p.spin);
+  }
 
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
+  if (p.stamp && threadIdx.x == 0) atomicMax(p.stamp + 1, global_ns());
 }
 
 // ---------------------------------------------------------------------------------------------- host side
@@ -745,7 +752,7 @@ bool fused_gemm_supported(FusedEpi epi, const FusedGemmArgs &a) {
   return true;
 }
 
-int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStream_t s) {
+int fused_gemm_launch(TmaMaps *g, FusedEpi epi, const FusedGemmArgs &a, cudaStream_t s) {
   if (!g || !fused_gemm_supported(epi, a)) return -1;
   Plan pl = make_plan(epi, a);
   if (pl.nt == 256 && pl.S > 1 && a.split == 0 && a.stages == 0 && pl.tiles * pl.S <= NUM_SMS) {
@@ -756,12 +763,12 @@ int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStr
   FusedParams p;
   memset(&p, 0, sizeof p);
   for (int j = 0; j < a.nw; j++) {
-    const CUtensorMap *mw = fast_gemm_map(g, a.w[j], a.O[j], a.I, TILE_M);
+    const CUtensorMap *mw = tma_maps_get(g, a.w[j], a.O[j], a.I, TILE_M);
     if (!mw) return -6;
     p.map_w[j] = *mw;
     p.O[j] = a.O[j];
   }
-  const CUtensorMap *mx = fast_gemm_map(g, a.x, a.rows, a.I, pl.nt);
+  const CUtensorMap *mx = tma_maps_get(g, a.x, a.rows, a.I, pl.nt);
   if (!mx) return -6;
   p.map_x = *mx;
   p.tiles0 = (a.O[0] + TILE_M - 1) / TILE_M;
@@ -775,13 +782,9 @@ int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStr
   p.act = a.act;
   p.best_val = a.best_val; p.best_idx = a.best_idx; p.best_ld = a.best_ld;
   p.status = a.status;
-  p.npf = 0;
-  for (int j = 0; j < a.npf && j < FusedGemmArgs::MAX_PREFETCH; j++) {
-    if (!a.pf_ptr[j] || ((uintptr_t)a.pf_ptr[j] & 15) || a.pf_bytes[j] < 16) continue;
-    p.pf_ptr[p.npf] = (const unsigned char *)a.pf_ptr[j];
-    p.pf_bytes[p.npf] = a.pf_bytes[j] & ~(size_t)15;
-    p.npf++;
-  }
+  p.stamp = a.stamp;
+  p.spin = a.spin_limit ? a.spin_limit : SPIN_LIMIT;
+  p.withhold = a.withhold ? 1 : 0;
   if (epi == EPI_SWIGLU && pl.nt == 256 && a.split == 0 && a.stages == 0) {
     // wide rows: one CTA per (gate tile, up tile) pair sharing the activation tiles
     constexpr int STAGE2 = 2 * A_BYTES + 256 * TILE_K * 2;

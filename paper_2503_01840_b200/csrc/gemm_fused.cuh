@@ -2,7 +2,7 @@
 // operands, split-K reduced across a thread-block cluster through distributed shared memory):
 // host-side interface.
 #pragma once
-#include "gemm_fast.cuh"
+#include "tma_maps.cuh"
 
 namespace spec {
 
@@ -50,15 +50,18 @@ struct FusedGemmArgs {
   float *best_val = nullptr;    // [tiles][best_ld]
   int32_t *best_idx = nullptr;
   int best_ld = 0;
-  // ---- weights of later launches to pull into L2 while this one runs (addresses and sizes multiples of 16)
-  static constexpr int MAX_PREFETCH = 6;
-  const void *pf_ptr[MAX_PREFETCH] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
-  size_t pf_bytes[MAX_PREFETCH] = {0, 0, 0, 0, 0, 0};
-  int npf = 0;
   // ---- launch
   int32_t *status = nullptr;    // device status words
   int split = 0, stages = 0;    // 0 = chosen by the library
   bool pdl = false;             // programmatic dependent launch (weights are prefetched before the wait)
+  // ---- test hook for the bounded waits: polls before a wait gives up (0 = the library's limit), and, when `withhold`
+  // is set, CTA 0 leaves out the activation load of its first k-block, so that its first wait runs out: the CTA records
+  // ST_TIMEOUT in the status words, skips its arithmetic, keeps its cluster barriers, waits for its loads in flight,
+  // frees its tensor memory and exits
+  unsigned spin_limit = 0;
+  bool withhold = false;
+  // ---- profiling aid: stamp[0] = earliest time (globaltimer ns) a CTA saw its inputs ready, stamp[1] = latest CTA exit
+  unsigned long long *stamp = nullptr;
 };
 
 // true when the shapes fit the fused kernels (rows <= 256, I % 8 == 0, 16-byte aligned pointers, and for
@@ -69,6 +72,6 @@ int fused_gemm_tiles(FusedEpi epi, const FusedGemmArgs &a);
 // CTAs a launch aims at (K slices are chosen to come close to it); process-wide.
 void fused_gemm_set_target_ctas(int n);
 // Returns 0 or a negative code.
-int fused_gemm_launch(FastGemm *g, FusedEpi epi, const FusedGemmArgs &a, cudaStream_t s);
+int fused_gemm_launch(TmaMaps *g, FusedEpi epi, const FusedGemmArgs &a, cudaStream_t s);
 
 }  // namespace spec

@@ -204,8 +204,7 @@ def test_c1_full_trajectory_fp32(flags):
     assert st.decisions_forced >= 800 and st.same_tree >= 30 and st.exact_out >= 24 and st.band_total == 0, st
 
 
-@pytest.mark.parametrize("flags", [0, sb.FLAG_NO_PDL | sb.FLAG_NO_GRAPH, sb.FLAG_CHAIN, sb.FLAG_CHAIN | sb.FLAG_NO_GRAPH, sb.FLAG_UNFUSED,
-                                   sb.FLAG_REF_GEMM | sb.FLAG_REF_ATTN])
+@pytest.mark.parametrize("flags", [0, sb.FLAG_NO_PDL | sb.FLAG_NO_GRAPH, sb.FLAG_STAMPS, sb.FLAG_REF_GEMM | sb.FLAG_REF_ATTN])
 def test_tiny_bf16_trajectory(flags):
     tw, dw = _weights(T1)
     prompts = [p.numpy() for p in synth.make_prompts(T1)]
@@ -215,7 +214,7 @@ def test_tiny_bf16_trajectory(flags):
     assert st.decisions_forced >= 40 and st.same_tree >= 4 and st.argmax_forced >= 150, st
 
 
-@pytest.mark.parametrize("flags", [0, sb.FLAG_CHAIN])
+@pytest.mark.parametrize("flags", [0, sb.FLAG_NO_TMA_ATTN])
 def test_small_bf16_hd128_trajectory(flags):
     tw, dw = _weights(T2)
     prompts = [p.numpy() for p in synth.make_prompts(T2)]
@@ -453,7 +452,7 @@ def test_plain_decode_matches_oracle_greedy():
     dec.close()
 
 
-@pytest.mark.parametrize("flags", [0, sb.FLAG_CHAIN])
+@pytest.mark.parametrize("flags", [0])
 def test_c2_two_layer_truncation_first_steps(flags):
     """8B-shaped widths (hidden 4096, 32/8 heads of 128, FFN 14336, vocab 128256 / 32000, depth 6, top-k 10,
     60 nodes) on a 2-layer truncation, first steps, bf16."""
@@ -507,3 +506,28 @@ def test_attention_few_query_rows_key_parallel_kernel(H, G, hd, rps):
             V = np.stack([vp[perm[s, p // ps], gk, p % ps].float().numpy() for p in pos])
             ref = po.attend(q[r, h].float().numpy(), K, V)
             assert np.abs(out[r, h] - ref).max() < 2e-2, (r, h)
+
+
+def test_bounded_device_wait_runs_out_and_is_reported():
+    """Failure detection without a fault: one CTA of the verify pass's LM-head GEMM never receives its first activation
+    tile (test hook), so its bounded wait runs out.  The CTA records the time-out, skips its arithmetic, waits for its
+    loads in flight, frees its tensor memory and leaves; the step returns SPEC_ERR_DEVICE_STATUS with the site of the
+    wait, the context stays usable, and a fresh context matches the oracle afterwards."""
+    tw, dw = _weights(T1)
+    prompts = [p.numpy() for p in synth.make_prompts(T1)]
+    for flags in (0, sb.FLAG_NO_GRAPH):
+        dec = sb.SpecDecoder(T1, parity.to_dev(tw), parity.to_dev(dw), batch=1, max_ctx=len(prompts[0]) + 200, flags=flags)
+        dec.prefill(prompts, 100)
+        dec.step()                                           # a healthy step first
+        dec.tune(sb.SpecDecoder.TUNE_DEBUG_WAIT_RUNS_OUT, 2000)
+        with pytest.raises(sb.SpecError) as e:
+            dec.step()
+        assert e.value.code == -7 and "site 201" in str(e.value), str(e.value)
+        assert (dec.debug(sb.DBG_STATUS, 0) == 0).all()      # the status words were cleared when they were reported
+        dec.tune(sb.SpecDecoder.TUNE_DEBUG_WAIT_RUNS_OUT, 0)
+        n0 = int(dec.lengths()[0])
+        out = dec.step()[0]                                  # the context still runs steps
+        assert 1 <= len(out) <= T1.tree_depth + 1 and int(dec.lengths()[0]) == n0 + len(out)
+        dec.close()
+    st, _ = parity.run_trajectory(T1, tw, dw, prompts, n_steps=4, tol=2e-2, tap_tol=3e-2)
+    assert st.steps == 4 and st.verify_compared == 4
