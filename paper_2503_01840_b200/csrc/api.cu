@@ -578,7 +578,7 @@ template <typename T> struct Sched {
     tl_launch_budget = c->dbg_launch_budget;
     c->stamp_n = 0;
     c->stamp_cls.clear();
-    if (c->stamps) {             // earliest times start at the largest value, latest at zero
+    if (c->stamps) {             // both slots start from all ones (see KernelStamp)
       cudaMemsetAsync(c->stamps, 0xff, (size_t)MAX_STAMPS * 2 * sizeof(unsigned long long), s);
     }
     if (!plain) {
@@ -987,7 +987,16 @@ extern "C" int64_t spec_debug_read(spec_ctx *c, int32_t what, int32_t seq, void 
     case SPEC_DBG_RAW_SSQ: return copy_out(c, c->ssq, (size_t)c->ktiles * c->Ralloc, dst, bytes);
     case SPEC_DBG_STAMPS:
       if (!c->stamps) return fail(c, SPEC_ERR_STATE, "spec_debug_read: kernel stamps need SPEC_FLAG_STAMPS");
-      return copy_out(c, c->stamps, (size_t)c->stamp_n * 2, dst, bytes);
+    {
+      // the device keeps the exit time complemented (both slots are updated with atomicMin from all ones)
+      size_t cnt = (size_t)c->stamp_n * 2, avail = cnt * sizeof(unsigned long long);
+      if (!dst || !bytes) return (int64_t)avail;
+      std::vector<unsigned long long> tmp(cnt);
+      if (copy_out(c, c->stamps, cnt, tmp.data(), avail) < 0) return SPEC_ERR_CUDA;
+      for (size_t i = 1; i < cnt; i += 2) tmp[i] = ~tmp[i];
+      memcpy(dst, tmp.data(), std::min(avail, bytes));
+      return (int64_t)avail;
+    }
     case SPEC_DBG_STAMP_CLASS: {
       size_t avail = c->stamp_cls.size() * sizeof(int32_t);
       if (dst && bytes) memcpy(dst, c->stamp_cls.data(), std::min(avail, bytes));

@@ -28,8 +28,9 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Profiling aid: the GPU's global nanosecond timer, and a guard that records into stamp[0] the earliest time a CTA
-// of the launch got past its dependency wait and into stamp[1] the latest time a warp of the launch left the kernel
-// (early returns included).  A null pointer switches it off.
+// of the launch got past its dependency wait and into stamp[1] the bitwise complement of the latest time a warp of
+// the launch left the kernel (early returns included), so that both slots start from all ones and are updated with
+// atomicMin.  A null pointer switches it off.
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -41,7 +42,7 @@ struct KernelStamp {
     if (p && start && threadIdx.x == 0) atomicMin(p, global_ns());
   }
   __device__ __forceinline__ ~KernelStamp() {
-    if (p && (threadIdx.x & 31) == 0) atomicMax(p + 1, global_ns());
+    if (p && (threadIdx.x & 31) == 0) atomicMin(p + 1, ~global_ns());
   }
 };
 

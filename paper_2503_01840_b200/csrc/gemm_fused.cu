@@ -422,7 +422,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
-  if (p.stamp && threadIdx.x == 0) atomicMax(p.stamp + 1, global_ns());
+  if (p.stamp && threadIdx.x == 0) atomicMin(p.stamp + 1, ~global_ns());
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -570,7 +570,7 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
-  if (p.stamp && threadIdx.x == 0) atomicMax(p.stamp + 1, global_ns());
+  if (p.stamp && threadIdx.x == 0) atomicMin(p.stamp + 1, ~global_ns());
 }
 
 // ---------------------------------------------------------------------------------------------- host side

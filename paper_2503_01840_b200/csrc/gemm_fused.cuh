@@ -60,7 +60,7 @@ struct FusedGemmArgs {
   // frees its tensor memory and exits
   unsigned spin_limit = 0;
   bool withhold = false;
-  // ---- profiling aid: stamp[0] = earliest time (globaltimer ns) a CTA saw its inputs ready, stamp[1] = latest CTA exit
+  // ---- profiling aid: stamp[0] = earliest time (globaltimer ns) a CTA saw its inputs ready, stamp[1] = complement of the latest CTA exit (both start from all ones)
   unsigned long long *stamp = nullptr;
 };
 
