@@ -223,6 +223,17 @@ int spec_gemm(int32_t dtype, int32_t impl, const void *x, const void *w, float *
 int spec_gemm_fused(const void *x, const void *w, float *out_f32, int32_t rows, int32_t out, int32_t in, int32_t ldo,
                     int32_t split, int32_t stages, void *stream);
 
+/* The draft LM head followed by log-softmax and top-K (Section 2.2: the draft tree is expanded by the draft model's
+ * confidence; Appendix A: nodes per expansion), on the kernels the step uses, without ever writing the logits: the
+ * GEMM's epilogue leaves, per 128-logit tile and row, the tile maximum, the sum of exp relative to it and the tile's K
+ * best logits, and a merge kernel turns them into each row's K best ids (value descending, lower id first on ties) and
+ * their log-probabilities.  x [rows][in] bf16, w [out][in] bf16, out_idx int32 [rows][K], out_lp float [rows][K];
+ * scratch: spec_gemm_topk_scratch_bytes(rows, out, K) bytes of device memory.  rows <= 256, in % 8 == 0, K <= 15,
+ * out <= 32768 and out / 128 * K <= 3200 (SPEC_ERR_UNSUPPORTED otherwise). */
+size_t spec_gemm_topk_scratch_bytes(int32_t rows, int32_t out, int32_t K);
+int spec_gemm_topk(const void *x, const void *w, int32_t rows, int32_t out, int32_t in, int32_t K, int32_t *out_idx,
+                   float *out_lp, void *scratch, void *stream);
+
 /* Gate/up half of the decoder layer's MLP (the draft layer and every target layer are LLaMA-style decoder layers,
  * Section 3.1), on the kernel the step uses: act[r][f] = bf16(silu(g) * u), g = sum_i x[r][i] * w_gate[f][i], u likewise
  * with w_up, both accumulated in fp32 (a cluster holds the gate and the up tile of the same 128 features and their K

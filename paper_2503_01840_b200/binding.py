@@ -58,7 +58,7 @@ class _Cfg(C.Structure):
 
 EXPORTS = ("spec_workspace_bytes", "spec_init", "spec_prefill", "spec_step", "spec_step_async", "spec_step_sampled", "spec_plain_step",
            "spec_lengths", "spec_profile_step", "spec_tune", "spec_launches_per_step", "spec_step_bytes", "spec_free", "spec_last_error",
-           "spec_debug_read", "spec_debug_read_kv", "spec_gemm", "spec_gemm_fused", "spec_gemm_swiglu",
+           "spec_debug_read", "spec_debug_read_kv", "spec_gemm", "spec_gemm_fused", "spec_gemm_swiglu", "spec_gemm_topk_scratch_bytes", "spec_gemm_topk",
            "spec_topk_scratch_bytes", "spec_attn_scratch_bytes",
            "spec_attention", "spec_attention_static", "spec_attention_static_capacity", "spec_logsoftmax_topk", "spec_argmax")
 
@@ -104,6 +104,9 @@ def lib():
     L.spec_attention_static.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, i32, vp, i32, i32, i32, i32, i32, vp]
     L.spec_gemm_fused.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]
     L.spec_gemm_swiglu.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp]
+    L.spec_gemm_topk_scratch_bytes.argtypes = [i32, i32, i32]
+    L.spec_gemm_topk_scratch_bytes.restype = sz
+    L.spec_gemm_topk.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
     L.spec_topk_scratch_bytes.argtypes = [i32, i32, i32]
     L.spec_topk_scratch_bytes.restype = sz
     L.spec_logsoftmax_topk.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
@@ -365,6 +368,22 @@ def gemm_fused(x: torch.Tensor, w: torch.Tensor, split: int = 0, stages: int = 0
     if rc:
         raise SpecError(rc, "spec_gemm_fused")
     return out
+
+
+def gemm_topk(x: torch.Tensor, w: torch.Tensor, K: int):
+    """Top-K ids and log-probabilities of softmax(x . w^T) per row without materialising the logits: (int32 [rows][K],
+    float32 [rows][K])."""
+    rows, I = x.shape
+    O = w.shape[0]
+    assert x.is_contiguous() and w.is_contiguous() and x.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
+    idx = torch.empty(rows, K, dtype=torch.int32, device=x.device)
+    lp = torch.empty(rows, K, dtype=torch.float32, device=x.device)
+    scratch = torch.empty(max(64, lib().spec_gemm_topk_scratch_bytes(rows, O, K)), dtype=torch.uint8, device=x.device)
+    rc = lib().spec_gemm_topk(x.data_ptr(), w.data_ptr(), rows, O, I, K, idx.data_ptr(), lp.data_ptr(), scratch.data_ptr(),
+                              _stream_ptr(None))
+    if rc:
+        raise SpecError(rc, "spec_gemm_topk")
+    return idx, lp
 
 
 def gemm_swiglu(x: torch.Tensor, w_gate: torch.Tensor, w_up: torch.Tensor) -> torch.Tensor:

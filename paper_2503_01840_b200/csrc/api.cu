@@ -90,7 +90,11 @@ struct spec_ctx {
   float *best_val = nullptr;   // [ceil(V/128)][Ralloc] per-tile argmax candidates of the target LM head
   int32_t *best_idx = nullptr;
   void *topk_scratch = nullptr;
-  int ktiles = 0, vtiles = 0;
+  int ktiles = 0, vtiles = 0, dtiles = 0;
+  // per-tile candidates of the draft LM head (fused path): [dtiles][Ralloc][K] values / indices, [dtiles][Ralloc] max / sum
+  float *cand_val = nullptr, *cand_max = nullptr, *cand_sum = nullptr;
+  int32_t *cand_idx = nullptr;
+  bool tree_fused = false;     // one launch between two draft passes (merge + expansion + next pass's inputs)
   // profiling aid (SPEC_FLAG_STAMPS): per stamped launch {earliest "inputs ready" time, latest CTA exit} in globaltimer ns
   unsigned long long *stamps = nullptr;      // [MAX_STAMPS][2]
   std::vector<int> stamp_cls;                // class of each stamped launch of the last scheduled step
@@ -234,6 +238,12 @@ static size_t carve(spec_ctx *c, void *base) {
   c->best_val = cv.take<float>((size_t)c->vtiles * R);
   c->best_idx = cv.take<int32_t>((size_t)c->vtiles * R);
   c->topk_scratch = cv.take_bytes(topk_scratch_bytes(R, c->Vd, c->K));
+  c->dtiles = (c->Vd + 127) / 128;
+  const size_t cld = (size_t)draft_tree_cand_ld(c->dtiles);
+  c->cand_val = cv.take<float>(cld * R * c->K);
+  c->cand_idx = cv.take<int32_t>(cld * R * c->K);
+  c->cand_max = cv.take<float>(cld * R);
+  c->cand_sum = cv.take<float>(cld * R);
   c->stamps = (g.flags & SPEC_FLAG_STAMPS) ? cv.take<unsigned long long>((size_t)MAX_STAMPS * 2) : nullptr;
   c->attn_scratch_bytes = attn_fast_scratch_bytes(R, c->H, c->hd, g.max_ctx);
   c->attn_scratch = cv.take_bytes(c->attn_scratch_bytes);
@@ -306,6 +316,7 @@ extern "C" int spec_init(spec_ctx **out, const spec_target_weights *tw, const sp
     }
   }
   c->fused = c->fg != nullptr;
+  c->tree_fused = c->fused && draft_tree_step_smem(c->dtiles, c->K) > 0;
   if (c->fg && !(c->hd <= 128 && (c->hd & (c->hd - 1)) == 0)) {
     int rc = fail(nullptr, SPEC_ERR_UNSUPPORTED, "spec_init: the bf16 tensor-core path takes a power-of-two head_dim <= 128 (got %d)", c->hd);
     tma_maps_destroy(c->fg);
@@ -443,11 +454,15 @@ template <typename T> struct Sched {
     fgemm(EPI_F32, a);
     c->np_proj = 1; c->ps_proj = 0;
   }
-  void draft_forward_fused(const float *feat, int nparts, size_t fstride, const int32_t *src_row, int rows, int tail_len) {
-    mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
-    mark(SPEC_PROF_MISC);
-    launch_build_cat<bf16>(feat, nparts, fstride, src_row, (const bf16 *)c->embed, c->meta.tok, c->meta.seq, (bf16 *)c->cat, rows, c->k, s);
-    tick();
+  // prebuilt: the launch that closed the previous draft pass already wrote this pass's FC2 input and RoPE angles
+  void draft_forward_fused(const float *feat, int nparts, size_t fstride, const int32_t *src_row, int rows, int tail_len,
+                           bool prebuilt = false) {
+    if (!prebuilt) {
+      mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
+      mark(SPEC_PROF_MISC);
+      launch_build_cat<bf16>(feat, nparts, fstride, src_row, (const bf16 *)c->embed, c->meta.tok, c->meta.seq, (bf16 *)c->cat, rows, c->k, s);
+      tick();
+    }
     fgemm_resid(c->cat, 2 * c->k, c->fc2, rows, false, c->dl.attn_norm, 0);
     block_fused(c->dl, c->pools[c->L], rows, tail_len, c->dfinal_norm, 0);
   }
@@ -457,6 +472,24 @@ template <typename T> struct Sched {
     with_norm_scale(a);
     a.out_f32 = c->logits; a.ldo = c->Vd;
     fgemm(EPI_F32, a);
+  }
+  // draft LM head whose epilogue leaves per-tile softmax statistics and top-K candidates (the logits themselves are
+  // written only when they are captured for inspection)
+  void draft_logits_topk(int rows, const int32_t *want_rows, int n_want) {
+    FusedGemmArgs a = fargs(c->h, rows, c->k);
+    a.w[0] = (const bf16 *)c->dlm_head; a.O[0] = c->Vd; a.nw = 1;
+    with_norm_scale(a);
+    if (c->cap_logits) { a.out_f32 = c->logits; a.ldo = c->Vd; }
+    a.topk = c->K; a.cand_val = c->cand_val; a.cand_idx = c->cand_idx; a.cand_max = c->cand_max; a.cand_sum = c->cand_sum;
+    a.cand_ld = draft_tree_cand_ld(c->dtiles); a.want_rows = want_rows; a.n_want = n_want;
+    fgemm(EPI_TOPK, a);
+  }
+  void tree_step(int pass) {
+    mark(SPEC_PROF_TREE);
+    int rc = launch_draft_tree_step(c->st, c->tb, c->meta, c->d2t, pass, c->cand_val, c->cand_idx, c->cand_max, c->cand_sum, c->dtiles,
+                                    draft_tree_cand_ld(c->dtiles), c->x, (const bf16 *)c->embed, (bf16 *)c->cat, c->k, c->inv_freq, c->cs, c->hd / 2, c->B, s);
+    if (rc && !c->sched_err) c->sched_err = rc;
+    tick();
   }
   void topk(const int32_t *src_row, int rows) {
     mark(SPEC_PROF_TOPK);
@@ -540,8 +573,9 @@ template <typename T> struct Sched {
   }
 
   // draft head on the rows of c->meta: cat = [feat ; e(tok)], FC2, decoder block, final norm (-> h)
-  void draft_forward(const float *feat, int nparts, size_t fstride, const int32_t *src_row, int rows, int tail_len) {
-    if (c->fused) return draft_forward_fused(feat, nparts, fstride, src_row, rows, tail_len);
+  void draft_forward(const float *feat, int nparts, size_t fstride, const int32_t *src_row, int rows, int tail_len,
+                     bool prebuilt = false) {
+    if (c->fused) return draft_forward_fused(feat, nparts, fstride, src_row, rows, tail_len, prebuilt);
     mark(SPEC_PROF_MISC); launch_rope_table(c->meta.pos, rows, c->hd / 2, c->inv_freq, c->cs, s); tick();
     mark(SPEC_PROF_MISC); launch_build_cat<T>(feat, nparts, fstride, src_row, (const T *)c->embed, c->meta.tok, c->meta.seq, (T *)c->cat, rows, c->k, s);
     tick();
@@ -586,17 +620,29 @@ template <typename T> struct Sched {
       c->cur_rps = c->Pmax;
       fuse(c->pend_taps, c->Te);
       draft_forward(c->proj, c->np_proj, c->ps_proj, nullptr, c->Te, c->Pmax);
-      draft_logits(c->Te);
-      topk(c->st.last_row, c->B);
-      capture(1, c->Te, true);
-      mark(SPEC_PROF_TREE); launch_expand(c->st, c->tb, c->meta, c->d2t, 1, c->B, s); tick();
+      if (c->tree_fused) {
+        draft_logits_topk(c->Te, c->st.last_row, c->B);
+        capture(1, c->Te, true);
+        tree_step(1);
+      } else {
+        draft_logits(c->Te);
+        topk(c->st.last_row, c->B);
+        capture(1, c->Te, true);
+        mark(SPEC_PROF_TREE); launch_expand(c->st, c->tb, c->meta, c->d2t, 1, c->B, s); tick();
+      }
       for (int p = 2; p <= c->D; p++) {
         c->cur_rps = c->K;
-        draft_forward(c->x, 1, 0, c->tb.feat_row, c->Td, c->tail_tree);
-        draft_logits(c->Td);
-        topk(nullptr, c->Td);
-        capture(p, c->Td, false);
-        mark(SPEC_PROF_TREE); launch_expand(c->st, c->tb, c->meta, c->d2t, p, c->B, s); tick();
+        draft_forward(c->x, 1, 0, c->tb.feat_row, c->Td, c->tail_tree, c->tree_fused);
+        if (c->tree_fused) {
+          draft_logits_topk(c->Td, nullptr, 0);
+          capture(p, c->Td, false);
+          tree_step(p);
+        } else {
+          draft_logits(c->Td);
+          topk(nullptr, c->Td);
+          capture(p, c->Td, false);
+          mark(SPEC_PROF_TREE); launch_expand(c->st, c->tb, c->meta, c->d2t, p, c->B, s); tick();
+        }
       }
       mark(SPEC_PROF_TREE); launch_rerank(c->st, c->tb, c->meta, c->B, s); tick();
     } else {
@@ -1078,6 +1124,42 @@ extern "C" int spec_gemm_swiglu(const void *x, const void *w_gate, const void *w
   int rc = fused_gemm_launch(g, EPI_SWIGLU, a, (cudaStream_t)stream);
   tma_maps_forget(g);
   if (rc) return rc == -1 ? SPEC_ERR_INVALID_CFG : SPEC_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
+}
+
+extern "C" size_t spec_gemm_topk_scratch_bytes(int32_t rows, int32_t out, int32_t K) {
+  if (rows < 1 || out < 1 || K < 1) return 0;
+  const size_t tiles = ((size_t)out + 127) / 128;
+  return (tiles + 3) * rows * ((size_t)K * 8 + 8) + 1024;
+}
+
+extern "C" int spec_gemm_topk(const void *x, const void *w, int32_t rows, int32_t O, int32_t I, int32_t K, int32_t *out_idx,
+                              float *out_lp, void *scratch, void *stream) {
+  if (!x || !w || !out_idx || !out_lp || !scratch) return SPEC_ERR_NULL;
+  if (rows < 1 || O < 1 || I < 1 || K < 1 || K > O) return SPEC_ERR_INVALID_CFG;
+  const int tiles = (O + 127) / 128;
+  if (!draft_tree_step_smem(tiles, K)) return SPEC_ERR_UNSUPPORTED;
+  static TmaMaps *g = nullptr;
+  if (!g) {
+    std::string why;
+    g = tma_maps_create(why);
+    if (!g) return SPEC_ERR_CUDA;
+  }
+  char *base = (char *)(((uintptr_t)scratch + 255) & ~(uintptr_t)255);
+  FusedGemmArgs a;
+  a.x = (const bf16 *)x; a.rows = rows; a.I = I; a.w[0] = (const bf16 *)w; a.O[0] = O; a.nw = 1;
+  const size_t cld = (size_t)draft_tree_cand_ld(tiles);
+  a.topk = K; a.cand_ld = (int)cld;
+  a.cand_val = (float *)base;
+  a.cand_idx = (int32_t *)(a.cand_val + cld * rows * K);
+  a.cand_max = (float *)(a.cand_idx + cld * rows * K);
+  a.cand_sum = a.cand_max + cld * rows;
+  if (!fused_gemm_supported(EPI_TOPK, a)) return SPEC_ERR_UNSUPPORTED;
+  int rc = fused_gemm_launch(g, EPI_TOPK, a, (cudaStream_t)stream);
+  tma_maps_forget(g);
+  if (rc) return rc == -1 ? SPEC_ERR_INVALID_CFG : SPEC_ERR_CUDA;
+  if (launch_merge_candidates(a.cand_val, a.cand_idx, a.cand_max, a.cand_sum, tiles, (int)cld, rows, K, out_idx, out_lp, (cudaStream_t)stream))
+    return SPEC_ERR_UNSUPPORTED;
   return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }
 

@@ -21,6 +21,28 @@ __device__ __forceinline__ void set_status(int32_t *st, int code, int where, int
   if (atomicCAS(st, 0, code) == 0) { st[1] = where; st[2] = a; st[3] = b; }
 }
 
+// "a before b" in (value desc, index asc) order: the tie-break of every argmax / top-k of the step
+__device__ __forceinline__ bool before(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
+
+// Order-preserving map of a float to an unsigned key (larger float = larger key; -0 is folded into +0 first, so equal
+// floats give equal keys) and back: lets a warp pick its best (value desc, index asc) entry with two redux instructions
+// instead of a five-step shuffle tree.
+__device__ __forceinline__ unsigned ordered_key(float v) {
+  const unsigned u = __float_as_uint(v + 0.0f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_value(unsigned k) { return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k); }
+// Best (key desc, index asc) over the warp; idx < 0 marks a lane without an entry.  Returns the winning index (-1: none)
+// and its key through *key.
+__device__ __forceinline__ int warp_best(unsigned key_in, int idx, unsigned *key) {
+  const unsigned k = idx >= 0 ? key_in : 0u;             // real keys are >= 1 (the key of -inf is 0x007fffff)
+  const unsigned m = __reduce_max_sync(0xffffffffu, k);
+  const unsigned cand = (idx >= 0 && k == m) ? (unsigned)idx : 0xffffffffu;
+  const unsigned w = __reduce_min_sync(0xffffffffu, cand);
+  *key = m;
+  return w == 0xffffffffu ? -1 : (int)w;
+}
+
 // Programmatic dependent launch: a kernel launched with the attribute may start while its predecessor
 // on the stream is still running; everything it reads that the predecessor wrote must come after
 // pdl_wait().  Both instructions do nothing in a kernel launched the ordinary way.

@@ -55,6 +55,7 @@ struct alignas(64) FusedParams {
   const float2 *cs; RowMeta m; bf16 *q; KvPool pool; PageMap pm; int H, G, hd;
   bf16 *act;
   float *best_val; int32_t *best_idx; int best_ld;
+  int topk; float *cand_val, *cand_max, *cand_sum; int32_t *cand_idx; int cand_ld; const int32_t *want_rows; int n_want;
   int32_t *status;
   unsigned long long *stamp;
   unsigned spin;               // polls before a wait gives up
@@ -383,6 +384,69 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
         const float sc = inv_s[row];
         const float g = src[(r - r0) * TILE_M + f] * sc, u = src_u[(r - r0) * TILE_M + f] * sc;
         if (good && o < p.O[0]) p.act[(size_t)row * p.O[0] + o] = __float2bfloat16_rn((g / (1.0f + expf(-g))) * u);
+      }
+    } else if (EPI == EPI_TOPK) {
+      // which rows need candidates (a list made by an earlier kernel: read after the dependency wait, i.e. here)
+      unsigned char *want = (unsigned char *)wpart;                // [256]
+      for (int t = threadIdx.x; t < 256; t += 128) want[t] = p.want_rows ? 0 : 1;
+      __syncthreads();
+      if (p.want_rows)
+        for (int t = threadIdx.x; t < p.n_want; t += 128) { const int wr = p.want_rows[t]; if (wr >= 0 && wr < 256) want[wr] = 1; }
+      __syncthreads();
+      if (good && p.out_f32 && o < p.O[0])
+        for (int r = r0; r < r1; r++) p.out_f32[(size_t)(c0 + r) * p.ldo + o] = src[(r - r0) * TILE_M + f] * inv_s[c0 + r];
+      // One warp takes four rows at a time: their selection rounds are four independent dependency chains, written
+      // without branches so that they interleave (a CTA has only four warps, nothing else hides the latencies).
+      // Lane l holds features l, l+32, l+64, l+96 of the tile as order-preserving keys; id < 0 = nothing there.
+      const int K = p.topk;
+      for (int rb = r0 + warp; rb < r1; rb += 16) {
+        unsigned key[4][4];
+        int id[4][4];
+        bool act[4];
+        size_t slot[4];
+#pragma unroll
+        for (int q = 0; q < 4; q++) {
+          const int r = rb + 4 * q, row = c0 + r;
+          const int rs = r < r1 ? r : r0;                                  // a row that exists (results are masked)
+          act[q] = good && r < r1 && want[row < 256 ? row : 255];          // uniform over the warp
+          slot[q] = (size_t)row * p.cand_ld * K + (size_t)blockIdx.x * K;
+          const float sc = inv_s[c0 + rs];
+          float v[4];
+          float mx = -INFINITY;
+#pragma unroll
+          for (int j2 = 0; j2 < 4; j2++) {
+            const int ff = lane + 32 * j2, oo = tm * TILE_M + ff;
+            id[q][j2] = (act[q] && oo < p.O[0]) ? oo : -1;
+            v[j2] = id[q][j2] >= 0 ? src[(rs - r0) * TILE_M + ff] * sc : -INFINITY;
+            key[q][j2] = ordered_key(v[j2]);
+            mx = fmaxf(mx, v[j2]);
+          }
+          for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+          float sum = 0.0f;
+#pragma unroll
+          for (int j2 = 0; j2 < 4; j2++) sum += id[q][j2] >= 0 ? expf(v[j2] - mx) : 0.0f;
+          for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+          // row-major: all candidates / statistics of a row are contiguous, so that the merge fetches a row in one go
+          if (act[q] && lane == 0) { p.cand_max[(size_t)row * p.cand_ld + blockIdx.x] = mx; p.cand_sum[(size_t)row * p.cand_ld + blockIdx.x] = sum; }
+        }
+        for (int c = 0; c < K; c++) {
+#pragma unroll
+          for (int q = 0; q < 4; q++) {
+            unsigned bk = 0u;
+            int bi = -1;
+#pragma unroll
+            for (int j2 = 0; j2 < 4; j2++) {
+              const bool better = id[q][j2] >= 0 && (bi < 0 || key[q][j2] > bk || (key[q][j2] == bk && id[q][j2] < bi));
+              bk = better ? key[q][j2] : bk;
+              bi = better ? id[q][j2] : bi;
+            }
+            unsigned wk;
+            const int wi = warp_best(bk, bi, &wk);
+#pragma unroll
+            for (int j2 = 0; j2 < 4; j2++) id[q][j2] = (id[q][j2] == wi) ? -1 : id[q][j2];   // taken (wi = -1: tile exhausted)
+            if (act[q] && lane == 0) { p.cand_val[slot[q] + c] = wi < 0 ? 0.0f : key_value(wk); p.cand_idx[slot[q] + c] = wi; }
+          }
+        }
       }
     } else {   // EPI_ARGMAX
       if (good && p.out_f32 && o < p.O[0])
@@ -745,6 +809,7 @@ bool fused_gemm_supported(FusedEpi epi, const FusedGemmArgs &a) {
   for (int j = 0; j < a.nw; j++)
     if (!a.w[j] || ((uintptr_t)a.w[j] & 15) || a.O[j] < 1) return false;
   if (epi == EPI_SWIGLU && a.O[0] != a.O[1]) return false;
+  if (epi == EPI_TOPK && (a.topk < 1 || a.topk > 16 || !a.cand_val || !a.cand_idx || !a.cand_max || !a.cand_sum || a.cand_ld < (a.O[0] + TILE_M - 1) / TILE_M)) return false;
   if (epi == EPI_QKV) {
     if (a.hd < 2 || a.hd > TILE_M || (a.hd & (a.hd - 1))) return false;
     if (a.O[0] != a.H * a.hd || a.O[1] != a.G * a.hd || a.O[2] != a.G * a.hd) return false;
@@ -781,6 +846,8 @@ int fused_gemm_launch(TmaMaps *g, FusedEpi epi, const FusedGemmArgs &a, cudaStre
   p.cs = a.cs; p.m = a.m; p.q = a.q; p.pool = a.pool; p.pm = a.pm; p.H = a.H; p.G = a.G; p.hd = a.hd;
   p.act = a.act;
   p.best_val = a.best_val; p.best_idx = a.best_idx; p.best_ld = a.best_ld;
+  p.topk = a.topk; p.cand_val = a.cand_val; p.cand_max = a.cand_max; p.cand_sum = a.cand_sum; p.cand_idx = a.cand_idx;
+  p.cand_ld = a.cand_ld; p.want_rows = a.want_rows; p.n_want = a.n_want;
   p.status = a.status;
   p.stamp = a.stamp;
   p.spin = a.spin_limit ? a.spin_limit : SPIN_LIMIT;
@@ -812,6 +879,7 @@ int fused_gemm_launch(TmaMaps *g, FusedEpi epi, const FusedGemmArgs &a, cudaStre
     case EPI_RESID: return launch_epi<EPI_RESID>(p, pl, a.pdl, s);
     case EPI_QKV: return launch_epi<EPI_QKV>(p, pl, a.pdl, s);
     case EPI_SWIGLU: return pl.pair ? launch_swiglu_pair(p, pl, a.pdl, s) : launch_epi<EPI_SWIGLU>(p, pl, a.pdl, s);
+    case EPI_TOPK: return launch_epi<EPI_TOPK>(p, pl, a.pdl, s);
     default: return launch_epi<EPI_ARGMAX>(p, pl, a.pdl, s);
   }
 }

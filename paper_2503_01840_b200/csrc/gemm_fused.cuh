@@ -11,7 +11,9 @@ enum FusedEpi {
   EPI_RESID = 1,    // x[r][o] (+)= acc; hb = bf16(x * gain[o]); per-tile sum of squares; optional taps
   EPI_QKV = 2,      // scale, rotate q and k by the row's position, store q, write K/V into the paged cache
   EPI_SWIGLU = 3,   // two weights (gate, up): act = bf16(silu(scale*g) * scale*u)
-  EPI_ARGMAX = 4    // per (feature tile, row) best (value, index); optional fp32 logits
+  EPI_ARGMAX = 4,   // per (feature tile, row) best (value, index); optional fp32 logits
+  EPI_TOPK = 5      // per (feature tile, wanted row): tile maximum, sum of exp relative to it, the tile's K best (value,
+                    // index) best first: what a log-softmax + top-K over all features needs; optional fp32 logits
 };
 
 struct FusedGemmArgs {
@@ -50,6 +52,14 @@ struct FusedGemmArgs {
   float *best_val = nullptr;    // [tiles][best_ld]
   int32_t *best_idx = nullptr;
   int best_ld = 0;
+  // ---- EPI_TOPK: candidates [rows][cand_ld][topk], tile statistics [rows][cand_ld]; cand_ld >= tiles (a multiple of 4
+  // keeps every row 16-byte aligned for the merge)
+  int topk = 0;                 // K (1..16)
+  float *cand_val = nullptr, *cand_max = nullptr, *cand_sum = nullptr;
+  int32_t *cand_idx = nullptr;  // -1: the tile has fewer than K features
+  int cand_ld = 0;
+  const int32_t *want_rows = nullptr;   // device list of the rows that need candidates (entries < 0 ignored); nullptr: all rows
+  int n_want = 0;
   // ---- launch
   int32_t *status = nullptr;    // device status words
   int split = 0, stages = 0;    // 0 = chosen by the library

@@ -37,6 +37,16 @@ struct TreeBufs {
 
 void launch_prep_extend(SeqState st, TreeBufs tb, RowMeta m, int B, int need_positions, int32_t *status, cudaStream_t s);
 void launch_expand(SeqState st, TreeBufs tb, RowMeta m, const int32_t *d2t, int pass, int B, cudaStream_t s);
+// One launch between two draft passes (merge of the LM head's per-tile candidates, expansion, the next pass's row
+// metadata, FC2 input and RoPE angles); returns -1 when the shape does not fit (tiles > 256, K > 15 or too many candidates).
+size_t draft_tree_step_smem(int tiles, int K);
+int draft_tree_cand_ld(int tiles);      // row pitch (in tiles) of the candidate arrays: tiles rounded up to a multiple of 4
+int launch_draft_tree_step(SeqState st, TreeBufs tb, RowMeta m, const int32_t *d2t, int pass, const float *cand_val,
+                           const int32_t *cand_idx, const float *cand_max, const float *cand_sum, int tiles, int ld, const float *x,
+                           const bf16 *embed, bf16 *cat, int k, const double *inv_freq, float2 *cs, int half, int B, cudaStream_t s);
+// the merge of per-tile candidates alone: idx / lp [rows][K]; -1 when the shape does not fit
+int launch_merge_candidates(const float *cand_val, const int32_t *cand_idx, const float *cand_max, const float *cand_sum, int tiles,
+                            int ld, int rows, int K, int32_t *idx, float *lp, cudaStream_t s);
 void launch_rerank(SeqState st, TreeBufs tb, RowMeta m, int B, cudaStream_t s);
 void launch_plain_tree(SeqState st, TreeBufs tb, RowMeta m, int B, cudaStream_t s);
 void launch_accept(SeqState st, TreeBufs tb, int B, int rows_per_seq, cudaStream_t s);

@@ -6,10 +6,11 @@
 
 namespace spec {
 
+size_t draft_tree_step_smem(int tiles, int K);
+int draft_tree_cand_ld(int tiles);
+
 // ---------------------------------------------------------------- block argmax helpers
 struct VI { float v; int i; };
-// "a before b" in (value desc, index asc) order
-__device__ __forceinline__ bool before(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
 
 __device__ __forceinline__ VI block_best(VI x, VI *sh) {
   for (int o = 16; o > 0; o >>= 1) {
@@ -451,6 +452,265 @@ void launch_expand(SeqState st, TreeBufs tb, RowMeta m, const int32_t *d2t, int 
   int K = tb.K, nch = K * K;
   size_t smem = (size_t)((nch + 1) & ~1) * 4 + (size_t)K * 16 + (size_t)K * 4 + (size_t)nch * 4 + 16;
   launch_k(expand_kernel, dim3(B), dim3(256), smem, s, st, tb, m, d2t, pass);
+}
+
+// One warp merges the per-tile candidates of one row (the draft LM head's epilogue left, per 128-logit tile, the tile
+// maximum, the sum of exp relative to it and the tile's K best logits, best first): the row's log-sum-exp and its K best
+// (value desc, index asc) as log-probabilities.  Layout: candidates [row][ld][K], statistics [row][ld], ld a multiple of
+// 4 and the arrays 16-byte aligned, so a row is fetched with 16-byte asynchronous copies that are all in flight at once.
+// stage_v / stage_i: ld * K floats / ints of 16-byte aligned scratch owned by the warp; tiles <= 256, K <= 15.
+__device__ __forceinline__ void merge_tile_candidates(const float *__restrict__ cand_val, const int32_t *__restrict__ cand_idx,
+                                                      const float *__restrict__ cand_max, const float *__restrict__ cand_sum,
+                                                      int tiles, int ld, int row, int K, float *stage_v, int32_t *stage_i,
+                                                      int32_t *out_id, float *out_lp) {
+  const int lane = threadIdx.x & 31;
+  const int nvec = ld * K / 4;                           // ld % 4 == 0
+  const float4 *gv = (const float4 *)(cand_val + (size_t)row * ld * K);
+  const int4 *gi = (const int4 *)(cand_idx + (size_t)row * ld * K);
+  for (int e = lane; e < nvec; e += 32) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(stage_v + 4 * e)), "l"(gv + e) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(stage_i + 4 * e)), "l"(gi + e) : "memory");
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  // the tile statistics meanwhile: at most 8 tiles per lane, all loads issued before the first use
+  float pm[8], ps[8];
+#pragma unroll
+  for (int j = 0; j < 8; j++) {
+    const int t = lane + 32 * j;
+    pm[j] = t < tiles ? cand_max[(size_t)row * ld + t] : -INFINITY;
+    ps[j] = t < tiles ? cand_sum[(size_t)row * ld + t] : 0.0f;
+  }
+  float mx = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < 8; j++) mx = fmaxf(mx, pm[j]);
+  for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+  float sum = 0.0f;                                      // lane l adds its tiles in tile order, then a fixed shuffle tree
+#pragma unroll
+  for (int j = 0; j < 8; j++) sum += (lane + 32 * j < tiles) ? ps[j] * expf(pm[j] - mx) : 0.0f;
+  for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+  const float lse = logf(sum);
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncwarp();
+  // a tile's candidates are stored best first: only its current head can be the next winner.  hp = head position of
+  // each of this lane's (at most 8) tiles, four bits each.
+  unsigned hp = 0;
+  for (int c = 0; c < K; c++) {
+    float bv = 0.0f;
+    int bi = -1, bj = 0;
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+      const int t = lane + 32 * j, h = (hp >> (4 * j)) & 15;
+      if (t < tiles && h < K) {
+        const int ci = stage_i[t * K + h];
+        const float cv = stage_v[t * K + h];
+        if (ci >= 0 && (bi < 0 || before(cv, ci, bv, bi))) { bv = cv; bi = ci; bj = j; }
+      }
+    }
+    unsigned wk;
+    const int wi = warp_best(ordered_key(bv), bi, &wk);  // two redux instructions instead of a shuffle tree
+    if (wi >= 0 && wi == bi) hp += 1u << (4 * bj);       // indices are unique: exactly one lane owns the winner
+    if (lane == 0) { out_id[c] = wi < 0 ? 0 : wi; out_lp[c] = wi < 0 ? 0.0f : (key_value(wk) - mx) - lse; }
+  }
+  __syncwarp();
+}
+
+// The merge alone, one warp per row (per-kernel parity tests of the LM-head epilogue + merge).
+__global__ void __launch_bounds__(256) merge_candidates_kernel(const float *cand_val, const int32_t *cand_idx, const float *cand_max,
+                                                               const float *cand_sum, int tiles, int ld, int rows, int K,
+                                                               int32_t *__restrict__ idx, float *__restrict__ lp) {
+  pdl_wait();
+  pdl_trigger();
+  extern __shared__ __align__(16) unsigned char smraw[];
+  const int warp = threadIdx.x >> 5, row = blockIdx.x * 8 + warp;
+  if (row >= rows) return;
+  float *stage_v = (float *)smraw + (size_t)warp * 2 * ld * K;
+  merge_tile_candidates(cand_val, cand_idx, cand_max, cand_sum, tiles, ld, row, K, stage_v, (int32_t *)(stage_v + ld * K),
+                        idx + (size_t)row * K, lp + (size_t)row * K);
+}
+int launch_merge_candidates(const float *cand_val, const int32_t *cand_idx, const float *cand_max, const float *cand_sum, int tiles,
+                            int ld, int rows, int K, int32_t *idx, float *lp, cudaStream_t s) {
+  const size_t smem = draft_tree_step_smem(tiles, K);
+  if (!smem || ld != draft_tree_cand_ld(tiles)) return -1;
+  static SmemLimit limit;
+  if (smem > 48 * 1024 && !limit.ensure(merge_candidates_kernel, (int)smem)) return -6;
+  launch_k(merge_candidates_kernel, dim3((rows + 7) / 8), dim3(256), smem, s, cand_val, cand_idx, cand_max, cand_sum, tiles, ld, rows, K, idx, lp);
+  return 0;
+}
+
+// ---------------------------------------------------------------- one launch between two draft passes
+// After the draft LM head of pass `pass` (whose epilogue left, per 128-logit tile and row, the tile maximum, the sum of
+// exp relative to it and the tile's K best logits): merges the tiles into each row's log-softmax top-K, adds the children
+// to the candidate pool with cumulative log-probability scores, picks the next frontier, writes the next pass's row
+// metadata, and builds that pass's inputs (the FC2 input [feature ; embedding] of every frontier node and its RoPE
+// angles).  Section 2.2 (dynamic draft tree: expansion by the draft's confidence), Section 3.1 (the draft's own output
+// is the feature of the next step), Appendix A (nodes per expansion).
+//
+// grid (B, Z): the Z CTAs of a sequence each redo the small merge + expansion (same inputs, same order of operations,
+// hence identical results) and then take one Z-th of the elements of the next pass's inputs; only CTA z = 0 writes the
+// tree state.  Nothing a CTA reads is written by another CTA of the launch.
+struct TreeStepArgs {
+  SeqState st; TreeBufs tb; RowMeta m;
+  const int32_t *d2t;
+  int pass;                       // 1-based draft pass that just ran
+  const float *cand_val, *cand_max, *cand_sum; const int32_t *cand_idx; int tiles, ld;   // [rows][ld][K], [rows][ld]
+  const float *x; const bf16 *embed; bf16 *cat; int k;                                    // next pass's FC2 input
+  const double *inv_freq; float2 *cs; int half;                                           // next pass's RoPE angles
+};
+
+constexpr int TREE_WARPS = 10;   // one warp per row of a top-10 level
+__global__ void __launch_bounds__(TREE_WARPS * 32) draft_tree_step_kernel(const TreeStepArgs a) {
+  pdl_wait();
+  pdl_trigger();
+  extern __shared__ __align__(16) unsigned char smraw[];
+  const TreeBufs &tb = a.tb;
+  const int K = tb.K, D = tb.D, b = blockIdx.x, pass = a.pass;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nrows = (pass == 1) ? 1 : K;                 // rows of this sequence in the pass that just ran
+  const int nchild = nrows * K;
+  // shared memory: per-warp candidate staging, then the expansion's small arrays
+  const int ncand = a.ld * K;
+  float *stage_v = (float *)smraw + (size_t)warp * 2 * ncand;      // [ld][K] values, then indices
+  int32_t *stage_i = (int32_t *)(stage_v + ncand);
+  unsigned char *tail = smraw + (size_t)TREE_WARPS * 2 * ncand * 4;
+  float *tk_lp = (float *)tail;                          // [nrows][K]
+  int32_t *tk_id = (int32_t *)(tk_lp + K * K);           // [nrows][K] draft ids
+  float *cscore = (float *)(tk_id + K * K);              // [nchild]
+  int32_t *ctok = (int32_t *)(cscore + K * K);           // [nchild] target ids
+  int32_t *newf = ctok + K * K;                          // [K] child index (within the level) of the new frontier
+  int32_t *par_u = newf + K;                             // [K] pool index of the node each row of this pass processed
+  float *par_sc = (float *)(par_u + K);                  // [K] its score
+  const int active = a.st.active[b], n = a.st.n[b], last_row = a.st.last_row[b];
+  const size_t pb = (size_t)b * (tb.pool + 1);
+  const int base = (pass == 1) ? 0 : K + (pass - 2) * K * K;       // pool index of child 0 is base + 1
+  const bool writer = blockIdx.y == 0;
+  if (!active) {   // skipped sequence: its rows of the next pass are padding
+    if (pass < D) {
+      if (writer)
+        for (int rr = threadIdx.x; rr < K; rr += blockDim.x) { a.m.seq[b * K + rr] = -1; a.m.tok[b * K + rr] = 0; a.m.pos[b * K + rr] = 0; }
+      const size_t total = (size_t)K * 2 * a.k;
+      for (size_t e = (size_t)blockIdx.y * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.y * blockDim.x)
+        a.cat[(size_t)b * K * 2 * a.k + e] = __float2bfloat16_rn(0.0f);
+    }
+    return;
+  }
+  // the parents of this pass's rows (two dependent loads) are fetched while the candidates are on their way
+  if ((int)threadIdx.x < nrows) {
+    const int u = (pass == 1) ? 0 : tb.frontier[((size_t)b * D + pass - 1) * K + threadIdx.x];
+    par_u[threadIdx.x] = u;
+    par_sc[threadIdx.x] = tb.pool_score[pb + u];
+  }
+  // ---- 1. per row: log-sum-exp over the tiles and the K best of the tiles' candidates (value desc, index asc)
+  for (int r = warp; r < nrows; r += TREE_WARPS) {
+    const int row = (pass == 1) ? last_row : b * K + r;
+    merge_tile_candidates(a.cand_val, a.cand_idx, a.cand_max, a.cand_sum, a.tiles, a.ld, row, K, stage_v, stage_i, tk_id + r * K,
+                          tk_lp + r * K);
+  }
+  __syncthreads();
+  if (writer) {   // kept for inspection: the top-K of this pass in the layout of the per-row kernels
+    for (int i = threadIdx.x; i < nchild; i += blockDim.x) {
+      const int row = (pass == 1) ? b : b * K + i / K;
+      tb.tk_idx[(size_t)row * K + i % K] = tk_id[i];
+      tb.tk_lp[(size_t)row * K + i % K] = tk_lp[i];
+    }
+  }
+  // ---- 2. children join the pool with cumulative scores
+  for (int c = threadIdx.x; c < nchild; c += blockDim.x) {
+    const int r = c / K;
+    const int u = par_u[r];                                // the node row r processed
+    const float sc = par_sc[r] + tk_lp[c];
+    const int tokid = a.d2t[tk_id[c]];
+    cscore[c] = sc;
+    ctok[c] = tokid;
+    if (writer) {
+      const int ci = base + c + 1;
+      tb.pool_tok[pb + ci] = tokid;
+      tb.pool_parent[pb + ci] = u;
+      tb.pool_depth[pb + ci] = pass;
+      tb.pool_score[pb + ci] = sc;
+    }
+  }
+  __syncthreads();
+  if (pass >= D) return;
+  // ---- 3. next frontier: the K best children of the level, (score desc, pool index asc)
+  for (int c = threadIdx.x; c < nchild; c += blockDim.x) {
+    const float s = cscore[c];
+    int rank = 0;
+    for (int j = 0; j < nchild; j++) rank += (cscore[j] > s || (cscore[j] == s && j < c)) ? 1 : 0;
+    if (rank < K) newf[rank] = c;
+  }
+  __syncthreads();
+  {
+    // the parents' masks are read by every writing thread before any row of the next pass is written
+    const int rr = threadIdx.x;
+    const bool mine = writer && rr < K;
+    const int c = mine ? newf[rr] : 0;
+    const int pr = c / K;                                  // parent's row in the pass that just ran (0 in pass 1)
+    uint64_t lo = 0ull, hi = 0ull;
+    if (mine && pass > 1) { lo = a.m.mask_lo[b * K + pr]; hi = a.m.mask_hi[b * K + pr]; }
+    __syncthreads();
+    if (mine) {
+      const int ci = base + c + 1;
+      const int row = b * K + rr;
+      const int slot = (pass - 1) * K + rr;
+      if (slot < 64) lo |= 1ull << slot; else hi |= 1ull << (slot - 64);
+      tb.front_cur[b * K + rr] = ci;
+      tb.frontier[((size_t)b * D + pass) * K + rr] = ci;
+      tb.feat_row[row] = (pass == 1) ? last_row : b * K + pr;
+      a.m.seq[row] = b;
+      a.m.pos[row] = n + pass - 1;
+      a.m.kvpos[row] = n + slot;
+      a.m.ctx[row] = n;
+      a.m.tail_base[row] = n;
+      a.m.mask_lo[row] = lo;
+      a.m.mask_hi[row] = hi;
+      a.m.tok[row] = ctok[c];
+    }
+  }
+  // ---- 4. inputs of the next pass: FC2 input [bf16(feature of the parent's row) ; embedding of the node's token] and
+  // the RoPE angles of its position (double precision, rounded once), split over the CTAs of the sequence
+  const int k = a.k, vpr = 2 * k / 8;                      // 8-element vectors per row (hidden % 8 == 0)
+  for (int e = blockIdx.y * blockDim.x + threadIdx.x; e < K * vpr; e += gridDim.y * blockDim.x) {
+    const int rr = e / vpr, i = (e % vpr) * 8;
+    const int c = newf[rr];
+    uint4 out;
+    if (i < k) {
+      const int fr = (pass == 1) ? last_row : b * K + c / K;
+      const float4 lo = *(const float4 *)(a.x + (size_t)fr * k + i), hi = *(const float4 *)(a.x + (size_t)fr * k + i + 4);
+      __nv_bfloat162 p0 = __floats2bfloat162_rn(lo.x, lo.y), p1 = __floats2bfloat162_rn(lo.z, lo.w);
+      __nv_bfloat162 p2 = __floats2bfloat162_rn(hi.x, hi.y), p3 = __floats2bfloat162_rn(hi.z, hi.w);
+      out = make_uint4(*(uint32_t *)&p0, *(uint32_t *)&p1, *(uint32_t *)&p2, *(uint32_t *)&p3);
+    } else {
+      out = *(const uint4 *)(a.embed + (size_t)ctok[c] * k + (i - k));
+    }
+    *(uint4 *)(a.cat + ((size_t)(b * K + rr)) * 2 * k + i) = out;
+  }
+  const int nang = K * a.half;
+  for (int e = blockIdx.y * blockDim.x + threadIdx.x; e < nang; e += gridDim.y * blockDim.x) {
+    const int rr = e / a.half, i = e % a.half;
+    double sn, cs_;
+    sincos((double)(n + pass - 1) * a.inv_freq[i], &sn, &cs_);
+    a.cs[(size_t)(b * K + rr) * a.half + i] = make_float2((float)cs_, (float)sn);
+  }
+}
+
+// shared memory the launch needs; 0 when the shape does not fit the kernel (the caller then uses the separate kernels)
+int draft_tree_cand_ld(int tiles) { return (tiles + 3) & ~3; }
+size_t draft_tree_step_smem(int tiles, int K) {
+  if (tiles > 256 || K > 15) return 0;
+  const size_t need = (size_t)TREE_WARPS * 2 * draft_tree_cand_ld(tiles) * K * 4 + (size_t)K * K * 16 + (size_t)K * 12 + 64;
+  return need <= 220 * 1024 ? need : 0;
+}
+int launch_draft_tree_step(SeqState st, TreeBufs tb, RowMeta m, const int32_t *d2t, int pass, const float *cand_val,
+                           const int32_t *cand_idx, const float *cand_max, const float *cand_sum, int tiles, int ld, const float *x,
+                           const bf16 *embed, bf16 *cat, int k, const double *inv_freq, float2 *cs, int half, int B, cudaStream_t s) {
+  const size_t smem = draft_tree_step_smem(tiles, tb.K);
+  if (!smem || ld != draft_tree_cand_ld(tiles) || (k % 8)) return -1;
+  static SmemLimit limit;
+  if (smem > 48 * 1024 && !limit.ensure(draft_tree_step_kernel, (int)smem)) return -6;
+  TreeStepArgs a{st, tb, m, d2t, pass, cand_val, cand_max, cand_sum, cand_idx, tiles, ld, x, embed, cat, k, inv_freq, cs, half};
+  const int Z = B >= 16 ? 1 : 8;        // CTAs per sequence that share the next pass's input assembly
+  launch_k(draft_tree_step_kernel, dim3(B, Z), dim3(TREE_WARPS * 32), smem, s, a);
+  return 0;
 }
 
 // ---------------------------------------------------------------- pruning + tree assembly

@@ -531,3 +531,33 @@ def test_bounded_device_wait_runs_out_and_is_reported():
         dec.close()
     st, _ = parity.run_trajectory(T1, tw, dw, prompts, n_steps=4, tol=2e-2, tap_tol=3e-2)
     assert st.steps == 4 and st.verify_compared == 4
+
+
+@pytest.mark.parametrize("O,K", [(32000, 10), (32768, 9), (1000, 4), (4096, 15), (130, 1)])
+def test_lm_head_topk_epilogue_and_merge_bit_exact(O, K):
+    """The draft LM head whose epilogue leaves per-tile top-K candidates and softmax statistics, followed by the merge
+    (the logits are never written): ids bit-exact against the oracle's log-softmax + top-k, ties included (lower id
+    first), an all-equal row, a vocabulary that is not a multiple of the tile.  The logits are planted exactly through
+    the GEMM: x is an identity, so logits[r][o] = w[o][r]."""
+    rows, I = 12, 16
+    g = torch.Generator().manual_seed(O + K)
+    z = (torch.randn(rows, O, generator=g) * 1.5).to(torch.bfloat16).float()
+    if O > 300:
+        z[3, 100] = z[3, 200] = z[3].max() + 1.0           # a tie at the top: lowest index first
+        z[7, O - 1] = z[7, 0] = z[7].max() + 0.5           # a tie across the first and the last tile
+    z[5, :] = 0.25                                         # all equal: ids 0..K-1
+    x = torch.zeros(rows, I, dtype=torch.bfloat16)
+    x[torch.arange(rows), torch.arange(rows)] = 1.0
+    w = torch.zeros(O, I, dtype=torch.bfloat16)
+    w[:, :rows] = z.t().to(torch.bfloat16)
+    idx, lp = sb.gemm_topk(x.cuda(), w.cuda(), K)
+    idx, lp = idx.cpu().numpy(), lp.cpu().numpy()
+    for r in range(rows):
+        oi, ov, _ = po.topk(po.log_softmax(z[r].numpy()), K)
+        assert idx[r].tolist() == oi.tolist(), (r, idx[r], oi)
+        assert np.abs(lp[r] - ov).max() < 5e-5, r           # fp32 sums of up to 32768 exp terms in two different orders
+    assert idx[5].tolist() == list(range(K))
+    if O > 300:
+        assert idx[3, 0] == 100 and (K < 2 or idx[3, 1] == 200) and idx[7, 0] == 0 and (K < 2 or idx[7, 1] == O - 1)
+    with pytest.raises(sb.SpecError):
+        sb.gemm_topk(x.cuda(), torch.zeros(40000, I, dtype=torch.bfloat16, device="cuda"), K)     # more than 256 tiles
