@@ -117,6 +117,7 @@ struct spec_ctx {
   float *u_dev = nullptr;      // [B][2N] uniforms of the sampled step, then 1 / temperature
   int sched_err = 0;
   int cur_rps = 1;             // rows per sequence of the pass being scheduled
+  int ctx_hint = -1;           // prefill: context length of the pass being scheduled (sizes the key split); -1: from n_upper
   bool prof = false;
   std::vector<cudaEvent_t> prof_ev;
   std::vector<int> prof_cls;
@@ -161,8 +162,12 @@ static const char *check_cfg(const spec_cfg *c) {
   return nullptr;
 }
 
-// Prompt positions per prefill pass: the chunk's rows are each other's tail keys, causal through the two-word masks.
-constexpr int PREFILL_CHUNK = 128;
+// Prompt positions per prefill pass.  A pass holds PREFILL_CHUNK / PREFILL_BLOCK blocks of PREFILL_BLOCK positions: the
+// rows of a block are each other's tail keys (causal through the two-word masks), and the blocks before it, whose K/V
+// the same pass's QKV epilogue has already written, are plain context.  The widest GEMM tile (256 rows) streams every
+// weight once per 256 prompt positions.
+constexpr int PREFILL_CHUNK = 256;
+constexpr int PREFILL_BLOCK = 128;
 
 // Derives sizes and carves every buffer; with c->cfg.workspace == nullptr (measure mode) only sizes.
 static size_t carve(spec_ctx *c, void *base) {
@@ -502,8 +507,9 @@ template <typename T> struct Sched {
     PageMap pm{c->page_table, c->pps, c->cfg.page_size, c->cfg.num_pages};
     bool fast = c->cfg.dtype == SPEC_BF16 && !(c->cfg.flags & SPEC_FLAG_REF_ATTN) && attn_fast_supported(c->hd, c->H / c->G);
     if (fast) {
-      int hint = 0;
-      for (int b = 0; b < c->B; b++) hint = std::max(hint, c->n_upper[b]);
+      int hint = std::max(0, c->ctx_hint);
+      if (c->ctx_hint < 0)
+        for (int b = 0; b < c->B; b++) hint = std::max(hint, c->n_upper[b]);
       tick(launch_attn_fast((const bf16 *)c->q, pool, pm, c->meta, tail_len, (bf16 *)c->ao, rows, c->H, c->G, c->hd,
                             c->cur_rps, hint, c->attn_scratch, s, !(c->cfg.flags & SPEC_FLAG_NO_TMA_ATTN), c->status,
                             c->st.order, c->B, next_stamp(SPEC_PROF_ATTN)));
@@ -718,9 +724,10 @@ template <typename T> static int do_prefill(spec_ctx *c, const int32_t *ids, con
   auto upload_meta = [&](int nvalid, int b, int start, const int32_t *toks) -> cudaError_t {
     for (int r = 0; r < CH; r++) {
       bool v = r < nvalid;
-      mseq[r] = v ? b : -1; mpos[r] = v ? start + r : 0; mctx[r] = v ? start : 0; mtok[r] = v ? toks[r] : 0;
-      mlo[r] = v ? (r >= 63 ? ~0ull : ((1ull << (r + 1)) - 1ull)) : 0ull;
-      mhi[r] = (v && r >= 64) ? (r >= 127 ? ~0ull : ((1ull << (r - 63)) - 1ull)) : 0ull;
+      const int j = r % PREFILL_BLOCK;               // position inside the block
+      mseq[r] = v ? b : -1; mpos[r] = v ? start + r : 0; mctx[r] = v ? start + r - j : 0; mtok[r] = v ? toks[r] : 0;
+      mlo[r] = v ? (j >= 63 ? ~0ull : ((1ull << (j + 1)) - 1ull)) : 0ull;
+      mhi[r] = (v && j >= 64) ? (j >= 127 ? ~0ull : ((1ull << (j - 63)) - 1ull)) : 0ull;
     }
     cudaError_t e = cudaMemcpyAsync(c->meta.seq, mseq.data(), CH * 4, cudaMemcpyHostToDevice, s);
     if (!e) e = cudaMemcpyAsync(c->meta.pos, mpos.data(), CH * 4, cudaMemcpyHostToDevice, s);
@@ -744,8 +751,9 @@ template <typename T> static int do_prefill(spec_ctx *c, const int32_t *ids, con
       int nv = std::min(CH, n - start);
       bool last = start + nv == n;
       CUDA_TRY(c, upload_meta(nv, b, start, p + start));
-      c->cur_rps = CH;
-      sc.target_forward(CH, CH, last);
+      c->cur_rps = PREFILL_BLOCK;
+      c->ctx_hint = start + CH - PREFILL_BLOCK;
+      sc.target_forward(CH, PREFILL_BLOCK, last);
       if (last) {
         // the last position stays pending: its taps become pending entry 0
         CUDA_TRY(c, cudaMemcpyAsync((char *)c->pend_taps + (size_t)b * c->Pmax * 3 * c->k * c->esz,
@@ -757,10 +765,11 @@ template <typename T> static int do_prefill(spec_ctx *c, const int32_t *ids, con
       if (nd > 0) {
         sc.fuse(c->node_taps, CH);
         CUDA_TRY(c, upload_meta(nd, b, start, p + start + 1));
-        sc.draft_forward(c->proj, c->np_proj, c->ps_proj, nullptr, CH, CH);
+        sc.draft_forward(c->proj, c->np_proj, c->ps_proj, nullptr, CH, PREFILL_BLOCK);
       }
     }
     CUDA_TRY(c, cudaStreamSynchronize(s));
+    c->ctx_hint = -1;
     n_host[b] = n;
     off += n;
   }

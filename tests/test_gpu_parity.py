@@ -254,9 +254,10 @@ def test_mha_model_trajectory(batch):
 
 @pytest.mark.parametrize("base", [C1, T1], ids=["fp32", "bf16"])
 def test_prefill_chunk_boundaries(base):
-    """Prompts of 127, 128, 129 and 257 tokens: the prefill runs 128-position chunks whose rows see each other through
-    the two-word causal masks; the first token, the first steps and the committed K/V must match the oracle."""
-    for n in (127, 128, 129, 257):
+    """Prompts of 127, 128, 129, 255, 256, 257 and 513 tokens: the prefill runs 256-position passes made of two
+    128-position blocks (rows of a block see each other through the two-word causal masks, the earlier block of the same
+    pass is context); the first token, the first steps and the committed K/V must match the oracle."""
+    for n in (127, 128, 129, 255, 256, 257, 513):
         cfg = base.replace(name=f"{base.name}-p{n}", prompt_len=n)
         tw, dw = _weights(cfg)
         prompts = [p.numpy() for p in synth.make_prompts(cfg)]
@@ -266,7 +267,7 @@ def test_prefill_chunk_boundaries(base):
         dec = sb.SpecDecoder(cfg, parity.to_dev(tw), parity.to_dev(dw), batch=1, max_ctx=n + 64)
         orc = po.Oracle(cfg, tw, dw, n + 64)
         assert dec.prefill(prompts, 8)[0] == orc.prefill(prompts[0])
-        for pos in (0, 63, 64, 126, n - 2, n - 1):
+        for pos in sorted(set([0, 63, 64, 126, min(128, n - 1), min(200, n - 1), n - 2, n - 1])):
             for layer in range(cfg.n_layers):
                 gk, gv = dec.read_kv(0, layer, pos)
                 ok, ov = orc.target_kv(layer, pos)
