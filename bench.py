@@ -239,6 +239,8 @@ def main():
     ap.add_argument("--workload", default="C2", help="C1..C8, optionally ':L=<layers>' for a truncation")
     ap.add_argument("--no-extras", action="store_true", help="skip plain-decode / structured-acceptance / CPU legs")
     ap.add_argument("--flags", type=int, default=0)
+    ap.add_argument("--dump-stamps", default="", help="write the per-launch in-graph kernel stamps of one step to this text file")
+    ap.add_argument("--nvtx", action="store_true", help="wrap the timed steps in an NVTX range 'timed_steps' (lets a profiler select them)")
     args = ap.parse_args()
     cfg = workload_cfg(args.workload)
     if args.impl == "reference":
@@ -275,14 +277,18 @@ def main():
     t_prefill = time.time() - t0
     prefill_launches = dec.launches_per_step()
 
-    counts = torch.zeros(max(args.steps, args.warmup), B, dtype=torch.int32, device=dev)
+    counts = torch.zeros(max(args.steps, args.warmup + 16, 16), B, dtype=torch.int32, device=dev)
     timed_steps(dec, args.warmup, counts)
     n_mid = dec.lengths().astype(np.float64)
     bytes_step = dec.step_bytes()
     if world > 1:
         dist.barrier()
     sampler = ClockSampler(local) if rank == 0 else None
+    if args.nvtx:
+        torch.cuda.nvtx.range_push("timed_steps")
     ms, toks = timed_steps(dec, args.steps, counts)
+    if args.nvtx:
+        torch.cuda.nvtx.range_pop()
     clocks = sampler.stop() if sampler else None
     launches = dec.launches_per_step()
 
@@ -328,6 +334,15 @@ def main():
         charged[cls] += max(0, end - start) * 1e-6
         prev_end = end if prev_end is None else max(prev_end, end)
     span_ms = float(stamps[:, 1].max() - stamps[:, 0].min()) * 1e-6 if len(stamps) else 0.0
+    if args.dump_stamps and rank == 0 and len(stamps):
+        t0s, prev = int(stamps[:, 0].min()), None
+        with open(args.dump_stamps, "w") as fh:
+            fh.write("# launch class ready_us end_us duration_us charged_us ready_minus_previous_end_us\n")
+            for i, ((ready, end), cls) in enumerate(zip(stamps.astype(np.int64), classes)):
+                start = ready if prev is None else max(ready, prev)
+                gap = 0 if prev is None else ready - prev
+                fh.write(f"{i} {cls} {(ready - t0s) / 1e3:.2f} {(end - t0s) / 1e3:.2f} {(end - ready) / 1e3:.2f} {max(0, end - start) / 1e3:.2f} {gap / 1e3:.2f}\n")
+                prev = end if prev is None else max(prev, end)
     gemm_ms = charged["gemm"]
     wbytes = weight_bytes_per_step(cfg)
     achieved = wbytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
