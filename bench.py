@@ -344,16 +344,20 @@ def main():
                 fh.write(f"{i} {cls} {(ready - t0s) / 1e3:.2f} {(end - t0s) / 1e3:.2f} {(end - ready) / 1e3:.2f} {max(0, end - start) / 1e3:.2f} {gap / 1e3:.2f}\n")
                 prev = end if prev is None else max(prev, end)
     gemm_ms = charged["gemm"]
+    timing = "in-graph kernel stamps (globaltimer) of one replayed step; non-overlapping charged intervals"
+    if gemm_ms <= 0.0:           # the plain fp32 schedule has no stamped kernels: one event per launch instead
+        gemm_ms = breakdown["gemm"][0]
+        timing = "one CUDA event before every launch (no graph): the plain fp32 kernels carry no stamps"
     wbytes = weight_bytes_per_step(cfg)
     achieved = wbytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
     ratio = NCU_TRAFFIC_RATIO.get(cfg.name)
     traffic = ratio * wbytes / max(1, gemm_n) if ratio else None
     ev_gemm_ms = breakdown["gemm"][0]
-    roofline = {"bound": "hbm", "kernel": "gemm_fused_kernel (all weight GEMMs of the step)", "achieved": achieved,
+    roofline = {"bound": "hbm", "kernel": ("gemm_fused_kernel" if cfg.dtype == "bf16" else "gemm_ref_kernel") + " (all weight GEMMs of the step)", "achieved": achieved,
                 "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                 "bytes_per_launch": wbytes / max(1, gemm_n), "avg_launch_us": 1e3 * gemm_ms / max(1, gemm_n),
                 "launches_per_step": gemm_n, "traffic": traffic,
-                "timing": "in-graph kernel stamps (globaltimer) of one replayed step; non-overlapping charged intervals",
+                "timing": timing,
                 "in_graph_ms": {"gemm": round(gemm_ms, 4), "attention": round(charged["attention"], 4),
                                 "first_ready_to_last_exit": round(span_ms, 4), "step_with_stamps": round(st_ms / 10, 4),
                                 "step": round(ms_per_step, 4)},
