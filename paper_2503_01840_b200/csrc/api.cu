@@ -115,6 +115,7 @@ struct spec_ctx {
   int launches = 0, launches_graph = 0, launches_graph_sampled = 0;
   bool sampled = false;        // the step being scheduled ends with the stochastic acceptance
   float *u_dev = nullptr;      // [B][2N] uniforms of the sampled step, then 1 / temperature
+  int32_t *prompt_dev = nullptr;   // [B * max_ctx] the prompts of the prefill being run, concatenated
   int sched_err = 0;
   int cur_rps = 1;             // rows per sequence of the pass being scheduled
   int ctx_hint = -1;           // prefill: context length of the pass being scheduled (sizes the key split); -1: from n_upper
@@ -231,6 +232,7 @@ static size_t carve(spec_ctx *c, void *base) {
   t.path = cv.take<int32_t>((size_t)B * c->Pmax); t.out_ids = cv.take<int32_t>((size_t)B * c->Pmax);
   t.out_cnt = cv.take<int32_t>(B); t.pend_tok = cv.take<int32_t>((size_t)B * c->Pmax);
   c->u_dev = cv.take<float>((size_t)B * 2 * c->N + 1);
+  c->prompt_dev = cv.take<int32_t>((size_t)B * g.max_ctx + 1);
   c->status = cv.take<int32_t>(8);
   if (g.flags & SPEC_FLAG_CAPTURE) {
     c->cap_logits = cv.take<float>((size_t)c->D * c->Td * c->Vd);
@@ -719,26 +721,15 @@ template <typename T> static int do_prefill(spec_ctx *c, const int32_t *ids, con
 
   Sched<T> sc(c);
   const int CH = PREFILL_CHUNK;
-  std::vector<int32_t> mseq(CH), mpos(CH), mctx(CH), mtok(CH), mzero(CH, 0);
-  std::vector<uint64_t> mlo(CH), mhi(CH, 0);
-  auto upload_meta = [&](int nvalid, int b, int start, const int32_t *toks) -> cudaError_t {
-    for (int r = 0; r < CH; r++) {
-      bool v = r < nvalid;
-      const int j = r % PREFILL_BLOCK;               // position inside the block
-      mseq[r] = v ? b : -1; mpos[r] = v ? start + r : 0; mctx[r] = v ? start + r - j : 0; mtok[r] = v ? toks[r] : 0;
-      mlo[r] = v ? (j >= 63 ? ~0ull : ((1ull << (j + 1)) - 1ull)) : 0ull;
-      mhi[r] = (v && j >= 64) ? (j >= 127 ? ~0ull : ((1ull << (j - 63)) - 1ull)) : 0ull;
-    }
-    cudaError_t e = cudaMemcpyAsync(c->meta.seq, mseq.data(), CH * 4, cudaMemcpyHostToDevice, s);
-    if (!e) e = cudaMemcpyAsync(c->meta.pos, mpos.data(), CH * 4, cudaMemcpyHostToDevice, s);
-    if (!e) e = cudaMemcpyAsync(c->meta.kvpos, mpos.data(), CH * 4, cudaMemcpyHostToDevice, s);
-    if (!e) e = cudaMemcpyAsync(c->meta.ctx, mctx.data(), CH * 4, cudaMemcpyHostToDevice, s);
-    if (!e) e = cudaMemcpyAsync(c->meta.tail_base, mctx.data(), CH * 4, cudaMemcpyHostToDevice, s);
-    if (!e) e = cudaMemcpyAsync(c->meta.tok, mtok.data(), CH * 4, cudaMemcpyHostToDevice, s);
-    if (!e) e = cudaMemcpyAsync(c->meta.mask_lo, mlo.data(), CH * 8, cudaMemcpyHostToDevice, s);
-    if (!e) e = cudaMemcpyAsync(c->meta.mask_hi, mhi.data(), CH * 8, cudaMemcpyHostToDevice, s);
-    if (!e) e = cudaStreamSynchronize(s);   // host vectors are reused by the next chunk
-    return e;
+  // the prompts go to the device once; each pass's row metadata is then built by a small kernel, so the host never
+  // waits inside the loop over passes
+  size_t total_ids = 0;
+  for (int b = 0; b < B; b++) total_ids += (size_t)lens[b];
+  CUDA_TRY(c, cudaMemcpyAsync(c->prompt_dev, ids, total_ids * 4, cudaMemcpyHostToDevice, s));
+  auto upload_meta = [&](int nvalid, int b, int start, const int32_t *toks_dev) -> cudaError_t {
+    launch_prefill_meta(c->meta, toks_dev, b, start, nvalid, CH, PREFILL_BLOCK, s);
+    sc.tick();
+    return cudaGetLastError();
   };
   size_t off = 0;
   std::vector<int32_t> n_host(B), P_host(B, 1), root_host(B);
@@ -750,7 +741,7 @@ template <typename T> static int do_prefill(spec_ctx *c, const int32_t *ids, con
     for (int start = 0; start < n; start += CH) {
       int nv = std::min(CH, n - start);
       bool last = start + nv == n;
-      CUDA_TRY(c, upload_meta(nv, b, start, p + start));
+      CUDA_TRY(c, upload_meta(nv, b, start, c->prompt_dev + off + start));
       c->cur_rps = PREFILL_BLOCK;
       c->ctx_hint = start + CH - PREFILL_BLOCK;
       sc.target_forward(CH, PREFILL_BLOCK, last);
@@ -764,7 +755,7 @@ template <typename T> static int do_prefill(spec_ctx *c, const int32_t *ids, con
       int nd = last ? nv - 1 : nv;        // draft entries j use token j+1; the last position waits for the root
       if (nd > 0) {
         sc.fuse(c->node_taps, CH);
-        CUDA_TRY(c, upload_meta(nd, b, start, p + start + 1));
+        CUDA_TRY(c, upload_meta(nd, b, start, c->prompt_dev + off + start + 1));
         sc.draft_forward(c->proj, c->np_proj, c->ps_proj, nullptr, CH, PREFILL_BLOCK);
       }
     }

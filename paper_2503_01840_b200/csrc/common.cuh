@@ -151,6 +151,10 @@ void launch_add_norm(float *x, const float *parts, int nparts, size_t part_strid
                      const T *gain, float eps, T *h, const int32_t *src_row, int rows_x, int rows_h, int k,
                      cudaStream_t s);
 
+// row metadata of one prefill pass of `rows` rows (a multiple of 64): nvalid prompt positions from `start` of sequence b,
+// tokens toks[0..nvalid) (device), causal blocks of `block` positions
+void launch_prefill_meta(RowMeta m, const int32_t *toks, int b, int start, int nvalid, int rows, int block, cudaStream_t s);
+
 void launch_rope_table(const int32_t *pos, int rows, int half, const double *inv_freq, float2 *cs, cudaStream_t s);
 
 // qkv partial sums [nparts][rows][(H+2G)hd] fp32 -> q (T, [rows][H][hd], rotated) and K/V written into the

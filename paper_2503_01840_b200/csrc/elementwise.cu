@@ -126,6 +126,29 @@ void launch_rope_table(const int32_t *pos, int rows, int half, const double *inv
   launch_k(rope_table_kernel, dim3((n + 255) / 256), dim3(256), 0, s, pos, rows, half, inv_freq, cs);
 }
 
+// ---------------------------------------------------------------- row metadata of one prefill pass
+// Row r < nvalid is prompt position start + r of sequence b, fed with toks[r]; a pass is made of blocks of `block`
+// positions: the rows of a block are each other's tail keys (causal through the two-word masks), everything before the
+// block is context.  Rows >= nvalid are padding.
+__global__ void prefill_meta_kernel(RowMeta m, const int32_t *__restrict__ toks, int b, int start, int nvalid, int block) {
+  pdl_wait();
+  pdl_trigger();
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  const bool v = r < nvalid;
+  const int j = r % block;                           // position inside the block
+  m.seq[r] = v ? b : -1;
+  m.pos[r] = v ? start + r : 0;
+  m.kvpos[r] = v ? start + r : 0;
+  m.ctx[r] = v ? start + r - j : 0;
+  m.tail_base[r] = v ? start + r - j : 0;
+  m.tok[r] = v ? toks[r] : 0;
+  m.mask_lo[r] = v ? (j >= 63 ? ~0ull : ((1ull << (j + 1)) - 1ull)) : 0ull;
+  m.mask_hi[r] = (v && j >= 64) ? (j >= 127 ? ~0ull : ((1ull << (j - 63)) - 1ull)) : 0ull;
+}
+void launch_prefill_meta(RowMeta m, const int32_t *toks, int b, int start, int nvalid, int rows, int block, cudaStream_t s) {
+  launch_k(prefill_meta_kernel, dim3(rows / 64), dim3(64), 0, s, m, toks, b, start, nvalid, block);
+}
+
 // ---------------------------------------------------------------- RoPE + q store + paged K/V write
 template <typename T>
 __global__ void rope_kv_kernel(const float *__restrict__ qkv, int nparts, size_t part_stride,
