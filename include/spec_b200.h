@@ -281,11 +281,34 @@ int spec_attention_static(const void *q, const void *k_pool, const void *v_pool,
                           int32_t tail_len, void *out, int32_t rows, int32_t n_heads, int32_t n_kv_heads,
                           int32_t head_dim, int32_t max_ctx, void *stream);
 
+/* Training-time-test attention, forward (Section 3.2 and its figure of the attention masks: while the draft model is
+ * trained its own outputs are fed back for further simulated steps; a query then sees the original sequence through the
+ * ordinary causal mask and, of every earlier simulated step, only the entry at its own position: the mask is lower
+ * triangular over the native keys and diagonal over every simulated step's keys, so the diagonal part needs no matrix
+ * product, only one dot product per step).  One call = the attention of one simulated step for one sequence:
+ *   out[i][h] = softmax over { q[i][h].K0[p][g] : p <= i } U { q[i][h].Kd[s][i][g] : s < n_steps } (scale hd^-1/2) applied
+ *   to the matching rows of V0 / Vd, with g = h / (n_heads / n_kv_heads).
+ * q, out: bf16 [T rounded up to a multiple of 128][n_heads][128] (rows >= T are padding: read, never used; out rows >= T
+ * are not written).  Pool positions T .. (T rounded up to 128) - 1 that fall in a mapped page are read with weight zero
+ * and must hold finite values.  K0 / V0 (the native step's keys and values, RoPE already applied): a paged pool
+ * [num_pages][n_kv_heads][page_size][128] bf16 with page_table int32 [pages_per_seq] (position p lives in page
+ * page_table[p / page_size]); page_size 16, 32 or 64.  k_diag / v_diag: bf16 [n_steps][T][n_kv_heads][128], the keys and
+ * values each simulated step produced at every position (may be NULL when n_steps is 0: plain causal attention);
+ * n_steps <= 8.  lse: optional float [T * n_heads], the natural-log normaliser of every row (what a backward pass needs).
+ * scratch: spec_ttt_attention_scratch_bytes(...) bytes of device memory.  head_dim must be 128 (SPEC_ERR_UNSUPPORTED
+ * otherwise).  The dense causal part runs on the tcgen05 tile kernel of the tree attention; the backward pass is not
+ * part of this library. */
+size_t spec_ttt_attention_scratch_bytes(int32_t T, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim);
+int spec_ttt_attention(const void *q, const void *k_pool, const void *v_pool, const int32_t *page_table, int32_t pages_per_seq,
+                       int32_t page_size, const void *k_diag, const void *v_diag, int32_t n_steps, void *out, float *lse,
+                       int32_t T, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, void *scratch, void *stream);
+
 /* Per-row log-softmax + top-K (value desc, index asc) over fp32 logits [rows][n]: the expansion
  * step of the dynamic tree (Section 2.2; Appendix A "nodes during the expansion phase").  K <= 16.
  * out_idx int32 [rows][K], out_lp float [rows][K].  scratch: device buffer of
- * spec_topk_scratch_bytes(rows, n, K) bytes for the two-stage kernel the step uses (chunk candidates,
- * then a per-row merge); NULL selects the plain one-CTA-per-row kernel. */
+ * spec_topk_scratch_bytes(rows, n, K) bytes for the two-stage kernel (chunk candidates, then a per-row merge; the step
+ * itself takes its candidates from the draft LM head's epilogue, see spec_gemm_topk); NULL selects the plain
+ * one-CTA-per-row kernel. */
 size_t spec_topk_scratch_bytes(int32_t rows, int32_t n, int32_t K);
 int spec_logsoftmax_topk(const float *logits, int32_t rows, int32_t n, int32_t K, int32_t *out_idx, float *out_lp,
                          void *scratch, void *stream);

@@ -225,6 +225,35 @@ def accept_sampled(tok, parent, logits, temperature, u, n_max=None):
     return cnt, path[:cnt].copy(), out[:cnt].copy(), acc_p, (lo.value, hi.value)
 
 
+def ttt_attention_rows(q, k0, v0, kd, vd, rows):
+    """Training-time-test attention of one simulated step for the positions in `rows`, written out from its definition
+    (Section 3.2, the figure of the attention masks during training-time test) in float64: the query at position i sees
+    the native step's keys 0..i and, of every simulated step s, only the entry at position i.  q [T][H][hd]; k0, v0
+    [T][G][hd]; kd, vd [J][T][G][hd] (J may be 0).  Returns (out [len(rows)][H][hd], lse [len(rows)][H]) as float64."""
+    q = np.asarray(q, np.float64); k0 = np.asarray(k0, np.float64); v0 = np.asarray(v0, np.float64)
+    kd = np.asarray(kd, np.float64); vd = np.asarray(vd, np.float64)
+    T, H, hd = q.shape
+    G = k0.shape[1]
+    J = kd.shape[0] if kd.size else 0
+    out = np.zeros((len(rows), H, hd)); lse = np.zeros((len(rows), H))
+    for n, i in enumerate(rows):
+        for h in range(H):
+            g = h // (H // G)
+            keys = np.concatenate([k0[: i + 1, g]] + [kd[s, i, g][None] for s in range(J)], 0)
+            vals = np.concatenate([v0[: i + 1, g]] + [vd[s, i, g][None] for s in range(J)], 0)
+            sc = keys @ q[i, h] / np.sqrt(hd)
+            m = sc.max()
+            e = np.exp(sc - m)
+            out[n, h] = (e[:, None] * vals).sum(0) / e.sum()
+            lse[n, h] = m + np.log(e.sum())
+    return out, lse
+
+
+def ttt_attention(q, k0, v0, kd, vd):
+    """The same for every position."""
+    return ttt_attention_rows(q, k0, v0, kd, vd, list(range(np.asarray(q).shape[0])))
+
+
 # ------------------------------------------------------------------ the model
 class Oracle:
     """One sequence.  `cfg` is a synth.ModelCfg-like object; weights are the synth dicts."""

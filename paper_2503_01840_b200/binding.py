@@ -58,7 +58,7 @@ class _Cfg(C.Structure):
 
 EXPORTS = ("spec_workspace_bytes", "spec_init", "spec_prefill", "spec_step", "spec_step_async", "spec_step_sampled", "spec_plain_step",
            "spec_lengths", "spec_profile_step", "spec_tune", "spec_launches_per_step", "spec_step_bytes", "spec_free", "spec_last_error",
-           "spec_debug_read", "spec_debug_read_kv", "spec_gemm", "spec_gemm_fused", "spec_gemm_swiglu", "spec_gemm_topk_scratch_bytes", "spec_gemm_topk",
+           "spec_debug_read", "spec_debug_read_kv", "spec_gemm", "spec_gemm_fused", "spec_gemm_swiglu", "spec_gemm_topk_scratch_bytes", "spec_gemm_topk", "spec_ttt_attention_scratch_bytes", "spec_ttt_attention",
            "spec_topk_scratch_bytes", "spec_attn_scratch_bytes",
            "spec_attention", "spec_attention_static", "spec_attention_static_capacity", "spec_logsoftmax_topk", "spec_argmax")
 
@@ -107,6 +107,9 @@ def lib():
     L.spec_gemm_topk_scratch_bytes.argtypes = [i32, i32, i32]
     L.spec_gemm_topk_scratch_bytes.restype = sz
     L.spec_gemm_topk.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
+    L.spec_ttt_attention_scratch_bytes.argtypes = [i32, i32, i32, i32]
+    L.spec_ttt_attention_scratch_bytes.restype = sz
+    L.spec_ttt_attention.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, i32, vp, vp, i32, i32, i32, i32, vp, vp]
     L.spec_topk_scratch_bytes.argtypes = [i32, i32, i32]
     L.spec_topk_scratch_bytes.restype = sz
     L.spec_logsoftmax_topk.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
@@ -384,6 +387,28 @@ def gemm_topk(x: torch.Tensor, w: torch.Tensor, K: int):
     if rc:
         raise SpecError(rc, "spec_gemm_topk")
     return idx, lp
+
+
+def ttt_attention(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, page_table: torch.Tensor, k_diag, v_diag,
+                  want_lse: bool = False):
+    """Training-time-test attention of one simulated step.  q bf16 [T][H][128]; k_pool / v_pool the native step's paged
+    keys / values [pages][G][page_size][128]; page_table int32 [pages_per_seq]; k_diag / v_diag bf16 [J][T][G][128] or None.
+    Returns out bf16 [T][H][128] (and the float32 [T][H] log-normaliser when want_lse)."""
+    T, H, hd = q.shape
+    G, ps = k_pool.shape[1], k_pool.shape[2]
+    rows = (T + 127) // 128 * 128
+    qp = torch.zeros(rows, H, hd, dtype=torch.bfloat16, device=q.device)
+    qp[:T] = q
+    out = torch.zeros_like(qp)
+    J = 0 if k_diag is None else k_diag.shape[0]
+    lse = torch.empty(T, H, dtype=torch.float32, device=q.device) if want_lse else None
+    scratch = torch.empty(max(64, lib().spec_ttt_attention_scratch_bytes(T, H, G, hd)), dtype=torch.uint8, device=q.device)
+    rc = lib().spec_ttt_attention(qp.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(), page_table.data_ptr(), page_table.numel(), ps,
+                                  k_diag.data_ptr() if J else None, v_diag.data_ptr() if J else None, J, out.data_ptr(),
+                                  lse.data_ptr() if want_lse else None, T, H, G, hd, scratch.data_ptr(), _stream_ptr(None))
+    if rc:
+        raise SpecError(rc, "spec_ttt_attention")
+    return (out[:T], lse) if want_lse else out[:T]
 
 
 def gemm_swiglu(x: torch.Tensor, w_gate: torch.Tensor, w_up: torch.Tensor) -> torch.Tensor:

@@ -16,6 +16,7 @@
 #include <map>
 #include <tuple>
 
+#include "../../include/spec_b200.h"
 #include "attn_fast.cuh"
 #include "tcgen05_ptx.cuh"
 
@@ -88,6 +89,7 @@ struct AttnParams {
   float *part_ml;   // [nsplit][rows*H][2]
   const int32_t *order;   // row block handled by the i-th CTA group (nullptr: i)
   unsigned long long *stamp;   // profiling aid (see KernelStamp), may be null
+  int keep_partial;            // 1: write unnormalised partial results and statistics even with a single key split
 };
 
 template <int HD>
@@ -535,7 +537,7 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
     if (mrow >= M) continue;
     int r = row0 + mrow / grp, h = g * grp + mrow % grp;
     float l = half ? lB : lA, mx = half ? mxB : mxA;
-    if (p.nsplit == 1) {
+    if (p.nsplit == 1 && !p.keep_partial) {
       float inv = l > 0.0f ? 1.0f / l : 0.0f;
       bf16 *dst = p.out + ((size_t)r * p.H + h) * HD;
 #pragma unroll
@@ -888,7 +890,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
           v[e] = __float_as_uint(o0 + o1);
         }
         if (mrow < M) {
-          if (p.nsplit == 1) {
+          if (p.nsplit == 1 && !p.keep_partial) {
             uint32_t w[8];
 #pragma unroll
             for (int e = 0; e < 8; e++) w[e] = pack_bf16(__uint_as_float(v[2 * e]) * inv, __uint_as_float(v[2 * e + 1]) * inv);
@@ -902,7 +904,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
           }
         }
       }
-      if (mrow < M && p.nsplit > 1) { p.part_ml[idx * 2] = mx; p.part_ml[idx * 2 + 1] = l; }
+      if (mrow < M && (p.nsplit > 1 || p.keep_partial)) { p.part_ml[idx * 2] = mx; p.part_ml[idx * 2 + 1] = l; }
     }
   }
 
@@ -1182,9 +1184,9 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const float *__restri
 
 int g_attn_target_ctas = 148;
 
-int pick_splits(int seqs, int G, int mtiles, int max_ctx_tiles) {
+int pick_splits(int seqs, int G, int mtiles, int max_ctx_tiles, int target = 0) {
   int base = seqs * G * mtiles;
-  int want = g_attn_target_ctas / base;                             // the kernels run one CTA per SM (register-bound): never more CTAs than one wave
+  int want = (target > 0 ? target : g_attn_target_ctas) / base;                             // the kernels run one CTA per SM (register-bound): never more CTAs than one wave
   if (want < 1) want = 1;
   int s = want < max_ctx_tiles ? want : max_ctx_tiles;
   if (s > MAX_SPLITS) s = MAX_SPLITS;
@@ -1290,6 +1292,7 @@ int launch_attn_fast(const bf16 *q, KvPool pool, PageMap pm, RowMeta m, int tail
   p.part_o = (float *)scratch;
   p.order = (order && order_len == seqs) ? order : nullptr;
   p.stamp = stamp;
+  p.keep_partial = 0;
   p.part_ml = p.part_o ? p.part_o + (size_t)MAX_SPLITS * rows * H * hd : nullptr;
   dim3 grid(mtiles, nsplit, seqs * G);
   // TMA-staged kernel when the tail follows the context and a page is a whole number of 128-byte-swizzle boxes
@@ -1389,4 +1392,142 @@ extern "C" int spec_attention_static(const void *q, const void *k_pool, const vo
   PageMap pm{page_table, pages_per_seq, page_size, 1 << 30};
   launch_attn_fast((const bf16 *)q, pool, pm, m, tail_len, (bf16 *)out, rows, H, G, hd, 1, max_ctx, scratch, (cudaStream_t)stream, false, nullptr);
   return cudaGetLastError() == cudaSuccess ? 0 : -6;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Training-time-test attention (Section 3.2, the figure of the attention masks during training-time test).
+//
+// While the draft model is trained, its own outputs are fed back for further simulated steps.  At simulated step j a
+// query at slot i sees the ORIGINAL sequence causally (keys 0..i of the native step: an ordinary lower-triangular mask)
+// and, of every earlier simulated step s = 1..j, only the entry at its own slot i (a diagonal mask).  The dense causal
+// part runs on the tensor-core tile kernels above (128-slot blocks: the block's slots are each other's tail keys, the
+// slots before the block are context), which leave unnormalised partial results; the diagonal part is j dot products
+// per (slot, head), computed as dot products, and folded into the same softmax by the merge kernel below.
+namespace spec {
+namespace {
+
+__global__ void ttt_meta_kernel(RowMeta m, int T, int block) {
+  pdl_wait();
+  pdl_trigger();
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  const bool v = r < T;
+  const int j = r % block;
+  m.seq[r] = v ? 0 : -1;
+  m.ctx[r] = v ? r - j : 0;
+  m.tail_base[r] = v ? r - j : 0;
+  m.mask_lo[r] = v ? (j >= 63 ? ~0ull : ((1ull << (j + 1)) - 1ull)) : 0ull;
+  m.mask_hi[r] = (v && j >= 64) ? (j >= 127 ? ~0ull : ((1ull << (j - 63)) - 1ull)) : 0ull;
+}
+
+constexpr int TTT_MAX_STEPS = 8;
+
+// One warp per (slot, head): merges the key splits of the dense part with the J diagonal entries.
+// part_o [nsplit][nrh][128] / part_ml [nsplit][nrh][2] as the tile kernels write them (raw maximum, sum and output
+// relative to it); q [rows][H][128]; kd / vd [J][T][G][128]; out [rows][H][128]; lse [T*H] natural-log sum (optional).
+__global__ void __launch_bounds__(256) ttt_merge_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, int nsplit,
+                                                        int nrh_alloc, const bf16 *__restrict__ q, const bf16 *__restrict__ kd,
+                                                        const bf16 *__restrict__ vd, int J, int T, int H, int G,
+                                                        bf16 *__restrict__ out, float *__restrict__ lse) {
+  pdl_wait();
+  pdl_trigger();
+  constexpr int HD = 128, DPL = 4;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rh = blockIdx.x * 8 + warp;
+  if (rh >= T * H) return;
+  const int i = rh / H, h = rh % H, g = h / (H / G);
+  const float sc = rsqrtf((float)HD) * 1.4426950408889634f;
+  float2 ml = make_float2(-INFINITY, 0.0f);                 // lane s holds split s (nsplit <= 32)
+  if (lane < nsplit) ml = *(const float2 *)(part_ml + ((size_t)lane * nrh_alloc + rh) * 2);
+  // the diagonal scores: q . k of the slot's own entry of every simulated step
+  const uint2 qraw = *(const uint2 *)(q + (size_t)rh * HD + lane * DPL);
+  const float2 q01 = __bfloat1622float2(*(const __nv_bfloat162 *)&qraw.x), q23 = __bfloat1622float2(*(const __nv_bfloat162 *)&qraw.y);
+  float d[TTT_MAX_STEPS];
+  uint2 vraw[TTT_MAX_STEPS];
+#pragma unroll
+  for (int s = 0; s < TTT_MAX_STEPS; s++) {
+    d[s] = -INFINITY;
+    if (s < J) {
+      const size_t off = (((size_t)s * T + i) * G + g) * HD + lane * DPL;
+      const uint2 kraw = *(const uint2 *)(kd + off);
+      vraw[s] = *(const uint2 *)(vd + off);
+      const float2 k01 = __bfloat1622float2(*(const __nv_bfloat162 *)&kraw.x), k23 = __bfloat1622float2(*(const __nv_bfloat162 *)&kraw.y);
+      float t = q01.x * k01.x + q01.y * k01.y + q23.x * k23.x + q23.y * k23.y;
+      for (int off2 = 16; off2 > 0; off2 >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off2);
+      d[s] = t;
+    }
+  }
+  float M = ml.x;
+  for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+#pragma unroll
+  for (int s = 0; s < TTT_MAX_STEPS; s++) M = fmaxf(M, d[s]);
+  const float w = (ml.x == -INFINITY) ? 0.0f : exp2f((ml.x - M) * sc);
+  float l = w * ml.y;
+  for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+  float acc[DPL] = {0.0f, 0.0f, 0.0f, 0.0f};
+  for (int s = 0; s < nsplit; s++) {
+    const float ws = __shfl_sync(0xffffffffu, w, s);
+    const float4 o = *(const float4 *)(part_o + ((size_t)s * nrh_alloc + rh) * HD + lane * DPL);
+    acc[0] += ws * o.x; acc[1] += ws * o.y; acc[2] += ws * o.z; acc[3] += ws * o.w;
+  }
+#pragma unroll
+  for (int s = 0; s < TTT_MAX_STEPS; s++)
+    if (s < J) {
+      const float ws = exp2f((d[s] - M) * sc);
+      const float2 v01 = __bfloat1622float2(*(const __nv_bfloat162 *)&vraw[s].x), v23 = __bfloat1622float2(*(const __nv_bfloat162 *)&vraw[s].y);
+      l += ws;
+      acc[0] += ws * v01.x; acc[1] += ws * v01.y; acc[2] += ws * v23.x; acc[3] += ws * v23.y;
+    }
+  const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+  __nv_bfloat162 o01 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv), o23 = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);
+  *(uint2 *)(out + (size_t)rh * HD + lane * DPL) = make_uint2(*(uint32_t *)&o01, *(uint32_t *)&o23);
+  if (lse && lane == 0) lse[rh] = logf(l) + M * rsqrtf((float)HD);
+}
+
+constexpr int TTT_BLOCK = 128;
+constexpr int TTT_TARGET_CTAS = 148;   // fixed (not the tuning knob): the scratch size and the launch must agree
+size_t ttt_meta_bytes(int rows_alloc) { return (((size_t)rows_alloc * (3 * 4 + 2 * 8)) + 255) & ~(size_t)255; }
+
+}  // namespace
+}  // namespace spec
+
+extern "C" size_t spec_ttt_attention_scratch_bytes(int32_t T, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim) {
+  using namespace spec;
+  if (T < 1 || n_heads < 1 || n_kv_heads < 1 || n_heads % n_kv_heads || head_dim != 128) return 0;
+  const int rows = (T + TTT_BLOCK - 1) / TTT_BLOCK * TTT_BLOCK, grp = n_heads / n_kv_heads;
+  const int nsplit = pick_splits(rows / TTT_BLOCK, n_kv_heads, (TTT_BLOCK * grp + MT - 1) / MT, (T + KT - 1) / KT, TTT_TARGET_CTAS);
+  return ttt_meta_bytes(rows) + (size_t)nsplit * rows * n_heads * (head_dim + 2) * sizeof(float) + 256;
+}
+
+extern "C" int spec_ttt_attention(const void *q, const void *k_pool, const void *v_pool, const int32_t *page_table,
+                                  int32_t pages_per_seq, int32_t page_size, const void *k_diag, const void *v_diag, int32_t n_steps,
+                                  void *out, float *lse, int32_t T, int32_t H, int32_t G, int32_t hd, void *scratch, void *stream) {
+  using namespace spec;
+  if (!q || !k_pool || !v_pool || !page_table || !out || !scratch || (n_steps > 0 && (!k_diag || !v_diag))) return SPEC_ERR_NULL;
+  if (T < 1 || H < 1 || G < 1 || H % G || n_steps < 0 || n_steps > TTT_MAX_STEPS) return SPEC_ERR_INVALID_CFG;
+  if (hd != 128 || !(page_size == 16 || page_size == 32 || page_size == 64) || (long long)pages_per_seq * page_size < T)
+    return SPEC_ERR_UNSUPPORTED;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int rows = (T + TTT_BLOCK - 1) / TTT_BLOCK * TTT_BLOCK, grp = H / G;
+  const int mtiles = (TTT_BLOCK * grp + MT - 1) / MT, seqs = rows / TTT_BLOCK;
+  const int nsplit = pick_splits(seqs, G, mtiles, (T + KT - 1) / KT, TTT_TARGET_CTAS);
+  char *base = (char *)(((uintptr_t)scratch + 255) & ~(uintptr_t)255);
+  RowMeta m{};
+  m.seq = (int32_t *)base; m.ctx = m.seq + rows; m.tail_base = m.ctx + rows;
+  m.mask_lo = (uint64_t *)(m.tail_base + rows); m.mask_hi = m.mask_lo + rows;
+  launch_k(ttt_meta_kernel, dim3(rows / 128), dim3(128), 0, s, m, (int)T, TTT_BLOCK);
+  AttnParams p;
+  p.q = (const bf16 *)q; p.kpool = (const bf16 *)k_pool; p.vpool = (const bf16 *)v_pool;
+  p.pm = PageMap{page_table, pages_per_seq, page_size, 1 << 20};
+  p.m = m; p.tail_len = TTT_BLOCK; p.rows = rows; p.H = H; p.G = G; p.rps = TTT_BLOCK; p.nsplit = nsplit; p.out = (bf16 *)out;
+  p.part_o = (float *)(base + ttt_meta_bytes(rows));
+  p.part_ml = p.part_o + (size_t)nsplit * rows * H * hd;
+  p.order = nullptr; p.stamp = nullptr; p.keep_partial = 1;
+  const CUtensorMap *mk = kv_map(k_pool, p.pm.num_pages, G, page_size, hd, 1), *mv = kv_map(v_pool, p.pm.num_pages, G, page_size, hd, 1);
+  if (!mk || !mv) return SPEC_ERR_CUDA;
+  dim3 grid(mtiles, nsplit, seqs * G);
+  if (launch_umma(p, grid, mk, mv, nullptr, s)) return SPEC_ERR_CUDA;
+  launch_k(ttt_merge_kernel, dim3((T * H + 7) / 8), dim3(256), 0, s, p.part_o, p.part_ml, nsplit, rows * H, (const bf16 *)q,
+           (const bf16 *)k_diag, (const bf16 *)v_diag, (int)n_steps, (int)T, (int)H, (int)G, (bf16 *)out, lse);
+  attn_fast_forget_maps();
+  return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }

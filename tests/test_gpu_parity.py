@@ -562,3 +562,35 @@ def test_lm_head_topk_epilogue_and_merge_bit_exact(O, K):
         assert idx[3, 0] == 100 and (K < 2 or idx[3, 1] == 200) and idx[7, 0] == 0 and (K < 2 or idx[7, 1] == O - 1)
     with pytest.raises(sb.SpecError):
         sb.gemm_topk(x.cuda(), torch.zeros(40000, I, dtype=torch.bfloat16, device="cuda"), K)     # more than 256 tiles
+
+
+@pytest.mark.parametrize("T,H,G,J", [(300, 8, 2, 3), (128, 4, 4, 0), (517, 32, 8, 1), (70, 8, 2, 8)])
+def test_ttt_attention_vs_oracle(T, H, G, J):
+    """Training-time-test attention (Section 3.2): dense causal part on the tensor-core tile kernel over 128-position
+    blocks (several blocks and a ragged last one), diagonal entries of J simulated steps as dot products, shuffled pages;
+    sampled positions (all block boundaries among them) x every head against the oracle's definition: outputs within the
+    bf16 tolerance 2e-2, log-normalisers within 2e-2."""
+    hd, ps = 128, 16
+    g = torch.Generator().manual_seed(T * 7 + J)
+    q = torch.randn(T, H, hd, generator=g).to(torch.bfloat16)
+    k0 = torch.randn(T, G, hd, generator=g).to(torch.bfloat16)
+    v0 = torch.randn(T, G, hd, generator=g).to(torch.bfloat16)
+    kd = torch.randn(J, T, G, hd, generator=g).to(torch.bfloat16) if J else None
+    vd = torch.randn(J, T, G, hd, generator=g).to(torch.bfloat16) if J else None
+    pps = (T + ps - 1) // ps + 1
+    perm = torch.randperm(pps + 3, generator=g)[:pps].to(torch.int32)
+    kp = torch.zeros(pps + 3, G, ps, hd, dtype=torch.bfloat16)
+    vp = torch.zeros(pps + 3, G, ps, hd, dtype=torch.bfloat16)
+    for p_ in range(T):
+        kp[perm[p_ // ps], :, p_ % ps] = k0[p_]
+        vp[perm[p_ // ps], :, p_ % ps] = v0[p_]
+    out, lse = sb.ttt_attention(q.cuda(), kp.cuda(), vp.cuda(), perm.cuda(), kd.cuda() if J else None,
+                                vd.cuda() if J else None, want_lse=True)
+    out, lse = out.float().cpu().numpy(), lse.cpu().numpy()
+    assert out.shape == (T, H, hd) and lse.shape == (T, H) and np.isfinite(out).all()
+    rows = sorted(set(range(0, T, 5)) | ({0, 1, 63, 64, 127, 128, 129, 255, 256, 257, T - 2, T - 1} & set(range(T))))
+    zero = np.zeros((0, T, G, hd))
+    o_out, o_lse = po.ttt_attention_rows(q.float().numpy(), k0.float().numpy(), v0.float().numpy(),
+                                         kd.float().numpy() if J else zero, vd.float().numpy() if J else zero, rows)
+    assert np.abs(out[rows] - o_out).max() < 2e-2, np.abs(out[rows] - o_out).max()
+    assert np.abs(lse[rows] - o_lse).max() < 2e-2, np.abs(lse[rows] - o_lse).max()

@@ -652,3 +652,50 @@ def test_golden_c1_trajectory_is_reproduced_and_lossless():
     assert all(1 <= c <= C1.tree_depth + 1 for c in stored["counts"]) and sum(stored["counts"]) == len(stored["tokens"]) - 1
     assert sum(stored["sampled_T1"]["counts"]) == len(stored["sampled_T1"]["tokens"]) - 1
     assert make_golden.trajectory() == stored
+
+
+# ----------------------------------------------------------------------------- training-time-test attention
+def _ttt_case(T, H, G, hd, J, seed):
+    g = torch.Generator().manual_seed(seed)
+    q = torch.randn(T, H, hd, generator=g)
+    k0, v0 = torch.randn(T, G, hd, generator=g), torch.randn(T, G, hd, generator=g)
+    kd, vd = torch.randn(J, T, G, hd, generator=g), torch.randn(J, T, G, hd, generator=g)
+    return q, k0, v0, kd, vd
+
+
+def test_ttt_attention_oracle_against_masked_library_attention():
+    """The oracle's training-time-test attention against torch's scaled_dot_product_attention over the concatenated key
+    set [native step ; simulated step 1 ; ... ; simulated step J] with the mask of Section 3.2's figure built by brute
+    force: lower-triangular on the native block, diagonal on every simulated block.  With J = 0 it must be plain causal
+    attention; a dropped diagonal entry, a shifted causal boundary or a wrong KV-head group fails."""
+    for (T, H, G, hd, J) in [(9, 4, 2, 16, 0), (7, 4, 2, 16, 1), (12, 6, 3, 8, 3), (5, 2, 2, 32, 2)]:
+        q, k0, v0, kd, vd = _ttt_case(T, H, G, hd, J, 100 + T + J)
+        out, lse = po.ttt_attention(q.numpy(), k0.numpy(), v0.numpy(), kd.numpy(), vd.numpy())
+        keys = torch.cat([k0] + [kd[s] for s in range(J)], 0)            # [(1+J) T][G][hd]
+        vals = torch.cat([v0] + [vd[s] for s in range(J)], 0)
+        mask = torch.zeros(T, (1 + J) * T, dtype=torch.bool)
+        for i in range(T):
+            mask[i, : i + 1] = True
+            for s in range(J):
+                mask[i, (1 + s) * T + i] = True
+        grp = H // G
+        kk = keys.permute(1, 0, 2).repeat_interleave(grp, 0).double()   # [H][(1+J) T][hd]
+        vv = vals.permute(1, 0, 2).repeat_interleave(grp, 0).double()
+        ref = torch.nn.functional.scaled_dot_product_attention(q.permute(1, 0, 2).double(), kk, vv, attn_mask=mask)
+        assert np.abs(out - ref.permute(1, 0, 2).numpy()).max() < 1e-9, (T, J)
+        if J == 0:
+            causal = torch.nn.functional.scaled_dot_product_attention(q.permute(1, 0, 2).double(), kk, vv, is_causal=True)
+            assert np.abs(out - causal.permute(1, 0, 2).numpy()).max() < 1e-9
+        # the log-normaliser against a direct log-sum-exp of the allowed scores
+        sc = torch.einsum("thd,hkd->thk", q.double(), kk) / hd ** 0.5
+        ref_lse = torch.logsumexp(sc.masked_fill(~mask[:, None, :], float("-inf")), -1)
+        assert np.abs(lse - ref_lse.numpy()).max() < 1e-9
+
+
+def test_ttt_attention_oracle_closed_form_single_position():
+    """T = 1: the softmax runs over the native key and the J diagonal entries only; with equal keys the output is the
+    plain mean of the 1 + J values."""
+    q = np.ones((1, 1, 4)); k0 = np.ones((1, 1, 4)); v0 = np.full((1, 1, 4), 3.0)
+    kd = np.ones((2, 1, 1, 4)); vd = np.stack([np.full((1, 1, 4), 6.0), np.full((1, 1, 4), 0.0)])
+    out, lse = po.ttt_attention(q, k0, v0, kd, vd)
+    assert np.allclose(out, 3.0) and np.allclose(lse, 4 / 2.0 + np.log(3.0))
