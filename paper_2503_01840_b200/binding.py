@@ -278,6 +278,7 @@ class SpecDecoder:
         return st, [self.PROF_CLASSES[c] for c in cls[: len(st)]]
 
     TUNE_GEMM_CTAS, TUNE_DEBUG_LAUNCH_BUDGET, TUNE_ATTN_CTAS, TUNE_DEBUG_WAIT_RUNS_OUT, TUNE_ATTN_UMMA = 2, 3, 4, 5, 6
+    TUNE_GEMM_PAIRS = 7
 
     def tune(self, what: int, value: int):
         self._check(lib().spec_tune(self.h, what, value))

@@ -78,6 +78,13 @@ __device__ __forceinline__ float ld_peer(uint32_t local_addr, uint32_t rank) {
   return v;
 }
 
+__device__ __forceinline__ uint32_t ld_peer_u32(uint32_t local_addr, uint32_t rank) {
+  uint32_t ra, v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+  asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(ra) : "memory");
+  return v;
+}
+
 // 16-byte load from the same shared-memory offset in cluster member `rank`.  Deliberately without a
 // "memory" clobber: consecutive loads stay in program order (volatile) but do not wait for one another,
 // so a thread keeps several remote requests in flight.
@@ -89,7 +96,7 @@ __device__ __forceinline__ float4 ld_peer4(uint32_t local_addr, uint32_t rank) {
   return v;
 }
 // sum over cluster members [s0, s0+n) (n <= 16) of the float4 at local_addr, added in member order
-__device__ __forceinline__ float4 sum_peers4(uint32_t local_addr, int s0, int n) {
+__device__ __forceinline__ float4 sum_peers4(uint32_t local_addr, int s0, int n, int stride = 1) {
   float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
 #pragma unroll
   for (int b = 0; b < 16; b += 8) {
@@ -97,7 +104,7 @@ __device__ __forceinline__ float4 sum_peers4(uint32_t local_addr, int s0, int n)
     float4 v[8];
 #pragma unroll
     for (int s = 0; s < 8; s++)
-      if (b + s < n) v[s] = ld_peer4(local_addr, (uint32_t)(s0 + b + s));
+      if (b + s < n) v[s] = ld_peer4(local_addr, (uint32_t)(s0 + (b + s) * stride));
 #pragma unroll
     for (int s = 0; s < 8; s++)
       if (b + s < n) { acc.x += v[s].x; acc.y += v[s].y; acc.z += v[s].z; acc.w += v[s].w; }
@@ -109,11 +116,19 @@ __device__ __forceinline__ float4 sum_peers4(uint32_t local_addr, int s0, int n)
 // MMAs of a k-block share one activation tile (half the activation fill traffic of the form in which gate and up are
 // separate cluster members), the two accumulators sit side by side in tensor memory, and the cluster holds only the
 // Sk K slices.
-template <int NT, int EPI, bool PAIR = false>
+//
+// DUO (256-row tiles; EPI_F32 / EPI_RESID / EPI_QKV): two neighbouring feature tiles run as a CTA pair (cta_group::2).
+// Each CTA streams its own weight tile but only HALF of the activation k-block (128 of the 256 rows); the even CTA issues
+// one M = 256 MMA per k-step that reads both CTAs' shared memory, and each CTA's tensor memory receives the accumulator
+// of its own tile.  At 256 rows the activation k-block (32 KB) is twice a weight tile, so the shared-memory fill traffic
+// per weight byte drops from 3 x to 2 x, which is what bounds the loop at this width.  The cluster is (2, S): x = the
+// pair, y = the K slices; the reduction runs over the members with the same x.
+template <int NT, int EPI, bool PAIR = false, bool DUO = false>
 __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__ FusedParams p) {
   static_assert(!PAIR || EPI == EPI_SWIGLU, "two weight tiles per CTA exist for the gate/up epilogue only");
+  static_assert(!DUO || (NT == 256 && !PAIR && (EPI == EPI_F32 || EPI == EPI_RESID || EPI == EPI_QKV)), "CTA pairs serve the 256-row tiles");
   constexpr int A_TILES = PAIR ? 2 : 1;
-  constexpr int B_BYTES = NT * TILE_K * 2;
+  constexpr int B_BYTES = (DUO ? NT / 2 : NT) * TILE_K * 2;
   constexpr int STAGE = A_TILES * A_BYTES + B_BYTES;
   constexpr int TMEM_COLS = (A_TILES * NT < 32) ? 32 : A_TILES * NT;
   static_assert(TMEM_COLS <= 512, "accumulators must fit the tensor memory");
@@ -132,7 +147,9 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int stages = p.stages, S = p.S, Sk = p.Sk;
-  const int slice = (S > 1) ? (int)cluster_rank() : 0;        // rank in the cluster
+  const uint32_t crank = (S > 1 || DUO) ? cluster_rank() : 0u;
+  const int xr = DUO ? (int)(crank & 1u) : 0;                 // DUO: position in the CTA pair (0 issues the MMAs)
+  const int slice = DUO ? (int)(crank >> 1) : (int)crank;     // K slice = rank among the CTAs that share this feature tile
   const int ksl = (EPI == EPI_SWIGLU && !PAIR) ? slice % Sk : slice;   // K slice
   const int kb0 = (int)(((long long)ksl * p.KB) / Sk), kb1 = (int)(((long long)(ksl + 1) * p.KB) / Sk);
   const int nkb = kb1 - kb0;
@@ -149,20 +166,61 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
     mbar_init(acc_bar, 1);
     *abort_flag = 0;
     *n_issued = 0; *n_consumed = 0;
+    // pairs rely on cluster ranks running x first (rank = x + 2 y): checked, never assumed
+    if (DUO && ((crank & 1u) != (blockIdx.x & 1u) || (int)(crank >> 1) != (int)(blockIdx.y % (unsigned)S))) {
+      *abort_flag = 1;
+      set_status(p.status, ST_TIMEOUT, 234, blockIdx.x, (int)crank);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {   // TMEM allocation is a whole-warp operation
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (warp == 1) {   // TMEM allocation is a whole-warp operation (pairs: the same warp of both CTAs, same slot offset)
+    if (DUO) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
+  if (DUO) cluster_sync_all(); else __syncthreads();   // pairs: the partner's barriers must exist before anything signals them
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
   pdl_trigger();
 
-  if (warp == 0 && lane == 0) {
+  if (DUO && *abort_flag) {
+    pdl_wait();            // wrong cluster layout: nothing is loaded or issued; the epilogue below writes nothing
+  } else if (DUO && warp == 0 && lane == 0) {
+    // ---- producer of a CTA pair: own weight tile + own half of the activation rows; every byte of both CTAs is counted
+    // on the even CTA's full barrier (it alone announces the byte count: one arrival per phase).
+    const CUtensorMap *mw0 = &p.map_w[mi];
+    const uint64_t pol = l2_policy_evict_first();
+    const uint32_t lead = crank & ~1u;
+    const int npre = nkb < stages ? nkb : stages;
+    for (int i = 0; i < npre; i++) {
+      if (xr == 0) mbar_expect_tx(&full[i], 2 * STAGE);
+      tma_load_2d_pair_hint(tiles + i * STAGE, mw0, (kb0 + i) * TILE_K, tm * TILE_M, mapa_u32(smem_u32(&full[i]), lead), pol);
+    }
+    pdl_wait();
+    if (p.stamp) atomicMin(p.stamp, global_ns());
+    for (int i = 0; i < npre; i++)
+      tma_load_2d_pair(tiles + i * STAGE + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, xr * (NT / 2), mapa_u32(smem_u32(&full[i]), lead));
+    // steady state: stage and phase advance by increments (no divisions), nothing but the wait and the copies per k-block
+    int i = npre, st = 0;
+    uint32_t ph = 0;
+    for (; i < nkb; i++) {
+      if (!mbar_wait(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 230, blockIdx.x, i); break; }
+      unsigned char *a = tiles + st * STAGE;
+      const uint32_t fb = mapa_u32(smem_u32(&full[st]), lead);
+      if (xr == 0) mbar_expect_tx(&full[st], 2 * STAGE);
+      tma_load_2d_pair_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, fb, pol);
+      tma_load_2d_pair(a + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, xr * (NT / 2), fb);
+      if (++st == stages) { st = 0; ph ^= 1u; }
+    }
+    *n_issued = i;
+  } else if (warp == 0 && lane == 0) {
     // ---- producer.  Weight tiles do not depend on the previous kernel: fill the ring with them first.
     const CUtensorMap *mw0 = &p.map_w[mi];
     const uint64_t pol = l2_policy_evict_first();
@@ -177,38 +235,64 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
     if (p.stamp) atomicMin(p.stamp, global_ns());
     const bool hold = p.withhold && blockIdx.x == 0 && blockIdx.y == 0;     // test hook: the first stage never completes
     for (int i = hold ? 1 : 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + A_TILES * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
-    *n_issued = npre;
-    for (int i = npre; i < nkb; i++) {
-      int st = i % stages;
-      if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
-      if (*abort_flag) break;
+    int i = npre, st = 0;             // the loop runs only when the prefill used every stage: it restarts at stage 0
+    uint32_t ph = 0;
+    for (; i < nkb; i++) {
+      if (!mbar_wait(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
       unsigned char *a = tiles + st * STAGE;
       mbar_expect_tx(&full[st], STAGE);
       tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
       if (PAIR) tma_load_2d_hint(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
       tma_load_2d(a + A_TILES * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[st]);
-      *n_issued = i + 1;
+      if (++st == stages) { st = 0; ph ^= 1u; }
     }
+    *n_issued = i;
   } else {
     pdl_wait();
-    if (warp == 1 && lane == 0) {
-      // ---- MMA issuer
-      constexpr uint32_t idesc = umma_idesc(NT);
-      for (int i = 0; i < nkb; i++) {
-        int st = i % stages;
-        if (!mbar_wait(&full[st], (i / stages) & 1, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 201, blockIdx.x, i); break; }
-        *n_consumed = i + 1;
-        if (*abort_flag) break;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        uint32_t a = smem_u32(tiles + st * STAGE), b = a + A_TILES * A_BYTES;
-#pragma unroll
-        for (int j = 0; j < TILE_K / UMMA_K; j++) {
-          uint64_t db = umma_desc_sw128(b + j * UMMA_K * 2);
-          umma_bf16(tmem_base, umma_desc_sw128(a + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
-          if (PAIR) umma_bf16(tmem_base + NT, umma_desc_sw128(a + A_BYTES + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
-        }
-        umma_commit(&empty[st]);      // frees the stage once these MMAs have read it
+    if (DUO && warp == 1 && lane == 0) {
+      // ---- MMA issuer of a CTA pair (even CTA only): M = 256 over both CTAs' weight tiles, N = both activation halves
+      if (xr == 0) {
+        constexpr uint32_t idesc = umma_idesc_m(NT, 2 * TILE_M);
+        const uint16_t pair_mask = (uint16_t)(3u << crank);       // this CTA and its partner
+        const uint32_t partner_base = ld_peer_u32(smem_u32(tmem_slot), crank | 1u);
+        if (partner_base != tmem_base) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 233, blockIdx.x, (int)partner_base); }
+        const uint64_t desc0 = umma_desc_sw128(smem_u32(tiles));
+        int i = 0, st = 0;
+        uint32_t ph = 0, ready = 0;
+        if (!*abort_flag)
+          for (; i < nkb; i++) {
+            if (!ready && !mbar_wait(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 231, blockIdx.x, i); break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t da = desc0 + (uint64_t)((st * STAGE) >> 4);
+            int nst = st + 1;
+            uint32_t nph = ph;
+            if (nst == stages) { nst = 0; nph ^= 1u; }
+            ready = umma_kblock_peek_pair(tmem_base, da, da + (A_BYTES >> 4), idesc, i ? 1u : 0u, &empty[st], pair_mask, smem_u32(&full[nst]), nph);
+            st = nst; ph = nph;
+          }
+        *n_consumed = i;
+        if (!*abort_flag) umma_commit_pair(acc_bar, pair_mask);   // both accumulators complete
       }
+    } else if (warp == 1 && lane == 0) {
+      // ---- MMA issuer
+      // The issuing thread is what limits a CTA's streaming rate, so the loop is kept to the wait (skipped when the
+      // peek of the previous iteration already saw the stage full), one fence and one instruction sequence per k-block.
+      constexpr uint32_t idesc = umma_idesc(NT);
+      const uint64_t desc0 = umma_desc_sw128(smem_u32(tiles));
+      int i = 0, st = 0;
+      uint32_t ph = 0, ready = 0;
+      for (; i < nkb; i++) {
+        if (!ready && !mbar_wait(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 201, blockIdx.x, i); break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint64_t da = desc0 + (uint64_t)((st * STAGE) >> 4), db = da + (uint64_t)((A_TILES * A_BYTES) >> 4);
+        int nst = st + 1;
+        uint32_t nph = ph;
+        if (nst == stages) { nst = 0; nph ^= 1u; }
+        if (PAIR) umma_kblock(tmem_base + NT, da + (A_BYTES >> 4), db, idesc, i ? 1u : 0u);   // the up accumulator
+        ready = umma_kblock_peek(tmem_base, da, db, idesc, i ? 1u : 0u, &empty[st], smem_u32(&full[nst]), nph);   // + commit: frees the stage
+        st = nst; ph = nph;
+      }
+      *n_consumed = i;
       umma_commit(acc_bar);           // accumulator complete
     } else if (warp >= 2) {
       // ---- per-row scale of the input: rsqrt(mean square + eps) from the producer kernel's per-tile sums
@@ -273,7 +357,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       for (int item = threadIdx.x; item < nitems; item += 128) {
         const int i = item >> 5, qd = item & 31;
         const uint32_t la = smem_u32(&red[(r0 + i) * TILE_M + qd * 4]);
-        *(float4 *)&sumb[i * TILE_M + qd * 4] = sum_peers4(la, 0, Sk);
+        *(float4 *)&sumb[i * TILE_M + qd * 4] = DUO ? sum_peers4(la, xr, Sk, 2) : sum_peers4(la, 0, Sk);
         if (EPI == EPI_SWIGLU) {
           if (PAIR) *(float4 *)&sumb[(CH / 2 + i) * TILE_M + qd * 4] = sum_peers4(smem_u32(&red_u[(r0 + i) * TILE_M + qd * 4]), 0, Sk);
           else *(float4 *)&sumb[(CH / 2 + i) * TILE_M + qd * 4] = sum_peers4(la, Sk, Sk);
@@ -476,15 +560,17 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
     // peers may still be reading this CTA's red; nobody overwrites or leaves before all are done
     if (S > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); else __syncthreads();
   }
-  if (*abort_flag && threadIdx.x == 0) {
+  if (*abort_flag && threadIdx.x == 0 && xr == 0) {
     // gave up on a wait: no bulk copy may still be landing in this CTA's shared memory when it exits.  Every stage
     // load that was issued and not seen complete is waited for (bounded; a load that was never issued runs the wait out).
+    // (Pairs: the even CTA's barriers count both CTAs' bytes, and the odd CTA leaves only after the barrier below.)
     for (int i = *n_consumed; i < *n_issued; i++) mbar_wait(&full[i % stages], (i / stages) & 1, p.spin);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
+  if (DUO) cluster_sync_all(); else __syncthreads();   // pairs: neither CTA frees tensor memory the other's MMAs may still use
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if (DUO) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
   if (p.stamp && threadIdx.x == 0) atomicMin(p.stamp + 1, ~global_ns());
 }
@@ -548,38 +634,38 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
     pdl_wait();
     if (p.stamp) atomicMin(p.stamp, global_ns());
     for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + 2 * A_BYTES, &p.map_x, i * TILE_K, 0, &full[i]);
-    *n_issued = npre;
-    for (int i = npre; i < KB; i++) {
-      const int st = i % stages;
-      if (!mbar_wait(&empty[st], ((i / stages) - 1) & 1, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 220, blockIdx.x, i); break; }
-      if (*abort_flag) break;
+    int i = npre, st = 0;
+    uint32_t ph = 0;
+    for (; i < KB; i++) {
+      if (!mbar_wait(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 220, blockIdx.x, i); break; }
       unsigned char *a = tiles + st * STAGE;
       mbar_expect_tx(&full[st], STAGE);
       tma_load_2d_hint(a, &p.map_w[0], i * TILE_K, tm * TILE_M, &full[st], pol);
       tma_load_2d_hint(a + A_BYTES, &p.map_w[1], i * TILE_K, tm * TILE_M, &full[st], pol);
       tma_load_2d(a + 2 * A_BYTES, &p.map_x, i * TILE_K, 0, &full[st]);
-      *n_issued = i + 1;
+      if (++st == stages) { st = 0; ph ^= 1u; }
     }
+    *n_issued = i;
   } else {
     pdl_wait();
     if (warp == 1 && lane == 0) {
       // ---- MMA issuer: gate accumulator at column 0, up accumulator at column NT
       constexpr uint32_t idesc = umma_idesc(NT);
-      for (int i = 0; i < KB; i++) {
-        const int st = i % stages;
-        if (!mbar_wait(&full[st], (i / stages) & 1, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 221, blockIdx.x, i); break; }
-        *n_consumed = i + 1;
-        if (*abort_flag) break;
+      const uint64_t desc0 = umma_desc_sw128(smem_u32(tiles));
+      int i = 0, st = 0;
+      uint32_t ph = 0, ready = 0;
+      for (; i < KB; i++) {
+        if (!ready && !mbar_wait(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 221, blockIdx.x, i); break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t ag = smem_u32(tiles + st * STAGE), au = ag + A_BYTES, b = ag + 2 * A_BYTES;
-#pragma unroll
-        for (int j = 0; j < TILE_K / UMMA_K; j++) {
-          const uint64_t db = umma_desc_sw128(b + j * UMMA_K * 2);
-          umma_bf16(tmem_base, umma_desc_sw128(ag + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
-          umma_bf16(tmem_base + NT, umma_desc_sw128(au + j * UMMA_K * 2), db, idesc, (i | j) ? 1u : 0u);
-        }
-        umma_commit(&empty[st]);
+        const uint64_t dg = desc0 + (uint64_t)((st * STAGE) >> 4), du = dg + (A_BYTES >> 4), db = dg + ((2 * A_BYTES) >> 4);
+        int nst = st + 1;
+        uint32_t nph = ph;
+        if (nst == stages) { nst = 0; nph ^= 1u; }
+        umma_kblock(tmem_base + NT, du, db, idesc, i ? 1u : 0u);
+        ready = umma_kblock_peek(tmem_base, dg, db, idesc, i ? 1u : 0u, &empty[st], smem_u32(&full[nst]), nph);
+        st = nst; ph = nph;
       }
+      *n_consumed = i;
       umma_commit(acc_bar);
     } else if (warp >= 2) {
       for (int r = threadIdx.x - 64; r < p.rows; r += 64) {
@@ -644,7 +730,7 @@ constexpr int NUM_SMS = 148;
 constexpr int SMEM_ONE = 200 * 1024;      // ring budget with one CTA per SM
 constexpr int SMEM_TWO = 104 * 1024;      // ring budget that lets two CTAs share an SM
 
-struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB, chunk; bool pair; };
+struct Plan { int nt, tiles, S, Sk, stages, smem, ctrl_off, KB, chunk; bool pair, duo; };
 
 // K slices per feature tile.  An SM streams at a capped rate whether one or two CTAs feed it, so the time
 // of a launch goes with (CTAs on the busiest SM) x (k-blocks per CTA + a fixed cost per CTA); two CTAs per SM
@@ -655,17 +741,19 @@ constexpr int MAX_CLUSTER = 8;    // portable cluster sizes only: size 9 (non-po
 // force_two: plan a wide tile (whose full ring takes the SM) as two CTAs per SM with two-stage rings
 constexpr int NUM_GPCS = 8;
 constexpr int MAX_BUMPED_CTAS = 266;   // 90 % of the 296 CTA slots: fuller grids fail to place all their clusters
-Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false) {
+// duo: neighbouring feature tiles as CTA pairs (clusters of 2 x Sk members; the stage holds half of the activation rows)
+Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false, bool duo = false) {
   Plan pl;
+  pl.duo = duo;
   pl.nt = pick_nt(a.rows);
   pl.KB = (a.I + TILE_K - 1) / TILE_K;
   pl.tiles = fused_gemm_tiles(epi, a);
   // gate/up below 256 rows: gate and up tile in ONE CTA (256 rows: the pair kernel without K split)
   pl.pair = epi == EPI_SWIGLU && pl.nt <= 128;
-  const int stage = (pl.pair ? 2 : 1) * A_BYTES + pl.nt * TILE_K * 2;
+  const int stage = (pl.pair ? 2 : 1) * A_BYTES + (duo ? pl.nt / 2 : pl.nt) * TILE_K * 2;
   const int wmul = (epi == EPI_SWIGLU && !pl.pair) ? 2 : 1;   // cluster members per K slice
-  const int smax = MAX_CLUSTER / wmul;
-  const bool wide = SMEM_TWO / stage < (pl.pair ? 2 : 3);     // 256-row tiles: the ring of one CTA takes the SM
+  const int smax = MAX_CLUSTER / (duo ? 2 : wmul);
+  const bool wide = duo || SMEM_TWO / stage < (pl.pair ? 2 : 3);     // 256-row tiles: the ring of one CTA takes the SM
   const bool one_per_sm = wide && !force_two;
   const int target = one_per_sm ? NUM_SMS : g_target_ctas;   // one wave
   int Sk = 1;
@@ -715,11 +803,11 @@ Plan make_plan(FusedEpi epi, const FusedGemmArgs &a, bool force_two = false) {
   return pl;
 }
 
-template <int NT, int EPI, bool PAIR = false>
+template <int NT, int EPI, bool PAIR = false, bool DUO = false>
 int launch_inst(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) {
   static SmemLimit limit;
-  if (!limit.ensure(gemm_fused_kernel<NT, EPI, PAIR>, pl.smem)) return -6;
-  if (pl.S > 8) return -1;   // portable cluster sizes only
+  if (!limit.ensure(gemm_fused_kernel<NT, EPI, PAIR, DUO>, pl.smem)) return -6;
+  if (pl.S * (DUO ? 2 : 1) > 8 || (DUO && (pl.tiles & 1))) return -1;   // portable cluster sizes only; pairs need an even tile count
   if (!launch_allowed()) return 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(pl.tiles, pl.S, 1);
@@ -728,9 +816,9 @@ int launch_inst(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) 
   cfg.stream = s;
   cudaLaunchAttribute at[2];
   int na = 0;
-  if (pl.S > 1) {
+  if (pl.S > 1 || DUO) {
     at[na].id = cudaLaunchAttributeClusterDimension;
-    at[na].val.clusterDim.x = 1; at[na].val.clusterDim.y = pl.S; at[na].val.clusterDim.z = 1;
+    at[na].val.clusterDim.x = DUO ? 2 : 1; at[na].val.clusterDim.y = pl.S; at[na].val.clusterDim.z = 1;
     na++;
   }
   if (pdl) {
@@ -740,7 +828,7 @@ int launch_inst(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) 
   }
   cfg.attrs = at;
   cfg.numAttrs = na;
-  return cudaLaunchKernelEx(&cfg, gemm_fused_kernel<NT, EPI, PAIR>, p) == cudaSuccess ? 0 : -6;
+  return cudaLaunchKernelEx(&cfg, gemm_fused_kernel<NT, EPI, PAIR, DUO>, p) == cudaSuccess ? 0 : -6;
 }
 
 // clusters of the plan's shape that can be resident at once (0: unknown)
@@ -794,6 +882,8 @@ int launch_swiglu_pair(const FusedParams &p, const Plan &pl, bool pdl, cudaStrea
 }  // namespace
 
 void fused_gemm_set_target_ctas(int n) { g_target_ctas = n; }
+namespace { int g_pairs = 0; }   // 256-row tiles of neighbouring feature tiles as CTA pairs (measured: no gain, off by default)
+void fused_gemm_set_pairs(int on) { g_pairs = on ? 1 : 0; }
 
 int fused_gemm_tiles(FusedEpi epi, const FusedGemmArgs &a) {
   if (epi == EPI_SWIGLU) return (a.O[0] + TILE_M - 1) / TILE_M;
@@ -820,7 +910,11 @@ bool fused_gemm_supported(FusedEpi epi, const FusedGemmArgs &a) {
 int fused_gemm_launch(TmaMaps *g, FusedEpi epi, const FusedGemmArgs &a, cudaStream_t s) {
   if (!g || !fused_gemm_supported(epi, a)) return -1;
   Plan pl = make_plan(epi, a);
-  if (pl.nt == 256 && pl.S > 1 && a.split == 0 && a.stages == 0 && pl.tiles * pl.S <= NUM_SMS) {
+  // 256 rows: CTA pairs when every weight's tile count is even (pairs never straddle two weights)
+  bool duo = g_pairs && pl.nt == 256 && (epi == EPI_F32 || epi == EPI_RESID || epi == EPI_QKV);
+  for (int j = 0; j < a.nw; j++) duo = duo && (a.O[j] % (2 * TILE_M)) == 0;
+  if (duo) pl = make_plan(epi, a, false, true);
+  if (!duo && pl.nt == 256 && pl.S > 1 && a.split == 0 && a.stages == 0 && pl.tiles * pl.S <= NUM_SMS) {
     // clusters are placed inside one GPC: a grid that counts fewer CTAs than SMs can still need a second wave
     const int fit = resident_clusters_wide(epi, pl);
     if (fit > 0 && pl.tiles > fit) pl = make_plan(epi, a, true);
@@ -833,7 +927,7 @@ int fused_gemm_launch(TmaMaps *g, FusedEpi epi, const FusedGemmArgs &a, cudaStre
     p.map_w[j] = *mw;
     p.O[j] = a.O[j];
   }
-  const CUtensorMap *mx = tma_maps_get(g, a.x, a.rows, a.I, pl.nt);
+  const CUtensorMap *mx = tma_maps_get(g, a.x, a.rows, a.I, duo ? pl.nt / 2 : pl.nt);   // pairs: each CTA loads half of the rows
   if (!mx) return -6;
   p.map_x = *mx;
   p.tiles0 = (a.O[0] + TILE_M - 1) / TILE_M;
@@ -873,6 +967,13 @@ int fused_gemm_launch(TmaMaps *g, FusedEpi epi, const FusedGemmArgs &a, cudaStre
     cfg.attrs = at;
     cfg.numAttrs = a.pdl ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, gemm_swiglu_pair_kernel<256>, p) == cudaSuccess ? 0 : -6;
+  }
+  if (duo) {
+    switch (epi) {
+      case EPI_F32: return launch_inst<256, EPI_F32, false, true>(p, pl, a.pdl, s);
+      case EPI_RESID: return launch_inst<256, EPI_RESID, false, true>(p, pl, a.pdl, s);
+      default: return launch_inst<256, EPI_QKV, false, true>(p, pl, a.pdl, s);
+    }
   }
   switch (epi) {
     case EPI_F32: return launch_epi<EPI_F32>(p, pl, a.pdl, s);

@@ -81,6 +81,7 @@ bool fused_gemm_supported(FusedEpi epi, const FusedGemmArgs &a);
 int fused_gemm_tiles(FusedEpi epi, const FusedGemmArgs &a);
 // CTAs a launch aims at (K slices are chosen to come close to it); process-wide.
 void fused_gemm_set_target_ctas(int n);
+void fused_gemm_set_pairs(int on);   // 256-row tiles as CTA pairs (cta_group::2); process-wide
 // Returns 0 or a negative code.
 int fused_gemm_launch(TmaMaps *g, FusedEpi epi, const FusedGemmArgs &a, cudaStream_t s);
 

@@ -81,6 +81,101 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t
 __device__ __forceinline__ void umma_commit(uint64_t *bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// ---- CTA pairs (cta_group::2): one MMA spans two CTAs of a cluster whose ranks differ in the lowest bit.  Each CTA
+// holds its own 128-row A tile and HALF of the B tile (N/2 rows) at the same shared-memory offsets; the even-ranked
+// CTA issues the MMA (M = 256), each CTA's tensor memory receives the 128 accumulator rows of its own A tile.
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t local_addr, uint32_t rank) {
+  uint32_t ra;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+  return ra;
+}
+// Tile load whose completion bytes are counted on an mbarrier that may live in the pair's other CTA
+// (bar_cluster_addr: a shared::cluster address, e.g. from mapa_u32).
+__device__ __forceinline__ void tma_load_2d_pair(void *smem_dst, const CUtensorMap *map, int c0, int c1, uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(map), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair_hint(void *smem_dst, const CUtensorMap *map, int c0, int c1, uint32_t bar_cluster_addr,
+                                                      uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(map), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "l"(policy)
+      : "memory");
+}
+// kind::f16, bf16 x bf16 -> fp32, M = m (256 for a CTA pair), N = nt
+__host__ __device__ constexpr uint32_t umma_idesc_m(int nt, int m) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(nt >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives (once the pair's MMAs issued so far have completed) on the mbarrier at this offset in every CTA of cta_mask
+__device__ __forceinline__ void umma_commit_pair(uint64_t *bar, uint16_t cta_mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(smem_u32(bar)),
+               "h"(cta_mask)
+               : "memory");
+}
+// ---- One k-block of the main loop in a single instruction sequence: a non-blocking test of the NEXT stage's "full"
+// barrier is issued first, then the four K = 16 MMAs of this stage (descriptors advance by 32 bytes = 2 units), then
+// the commit that frees the stage; the test's result is read last, so that its latency hides behind the MMA issue.
+// Returns 1 when the tested phase is complete (the caller then skips its wait).  The issuing thread is the bottleneck
+// of a weight-streaming CTA: every instruction saved here is bandwidth.
+#define SPEC_KBLOCK_BODY(MMA, COMMIT)                                                                              \
+  "{\n\t.reg .pred p, q, t;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"                                             \
+  "setp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 t, 0, 0;\n\t"                                                                                     \
+  "mbarrier.test_wait.parity.shared::cta.b64 q, [%7], %8;\n\t"                                                    \
+  "add.s64 a1, %2, 2;\n\tadd.s64 a2, %2, 4;\n\tadd.s64 a3, %2, 6;\n\t"                                           \
+  "add.s64 b1, %3, 2;\n\tadd.s64 b2, %3, 4;\n\tadd.s64 b3, %3, 6;\n\t"                                           \
+  MMA " [%1], %2, %3, %4, p;\n\t"                                                                                 \
+  MMA " [%1], a1, b1, %4, t;\n\t"                                                                                 \
+  MMA " [%1], a2, b2, %4, t;\n\t"                                                                                 \
+  MMA " [%1], a3, b3, %4, t;\n\t"                                                                                 \
+  COMMIT "\n\t"                                                                                                   \
+  "selp.u32 %0, 1, 0, q;\n\t}"
+
+__device__ __forceinline__ uint32_t umma_kblock_peek(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate,
+                                                     uint64_t *commit_bar, uint32_t peek_bar_addr, uint32_t peek_parity) {
+  uint32_t ok;
+  asm volatile(SPEC_KBLOCK_BODY("tcgen05.mma.cta_group::1.kind::f16", "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%6];")
+               : "=r"(ok)
+               : "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(smem_u32(commit_bar)), "r"(peek_bar_addr), "r"(peek_parity)
+               : "memory");
+  return ok;
+}
+// the same for a CTA pair (M = 256 across both CTAs; the commit arrives in every CTA of cta_mask)
+__device__ __forceinline__ uint32_t umma_kblock_peek_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate,
+                                                          uint64_t *commit_bar, uint16_t cta_mask, uint32_t peek_bar_addr, uint32_t peek_parity) {
+  uint32_t ok;
+  asm volatile(SPEC_KBLOCK_BODY("tcgen05.mma.cta_group::2.kind::f16",
+                                "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%6], %9;")
+               : "=r"(ok)
+               : "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(smem_u32(commit_bar)), "r"(peek_bar_addr), "r"(peek_parity),
+                 "h"(cta_mask)
+               : "memory");
+  return ok;
+}
+// four MMAs of a k-block without commit or peek (the second accumulator of a gate/up pair)
+__device__ __forceinline__ void umma_kblock(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, t;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 t, 0, 0;\n\t"
+      "add.s64 a1, %1, 2;\n\tadd.s64 a2, %1, 4;\n\tadd.s64 a3, %1, 6;\n\t"
+      "add.s64 b1, %2, 2;\n\tadd.s64 b2, %2, 4;\n\tadd.s64 b3, %2, 6;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %3, t;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a2, b2, %3, t;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a3, b3, %3, t;\n\t}" ::"r"(tmem_d),
+      "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
