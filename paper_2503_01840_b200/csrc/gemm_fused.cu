@@ -192,64 +192,81 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
 
   if (DUO && *abort_flag) {
     pdl_wait();            // wrong cluster layout: nothing is loaded or issued; the epilogue below writes nothing
-  } else if (DUO && warp == 0 && lane == 0) {
+  } else if (DUO && warp == 0) {
     // ---- producer of a CTA pair: own weight tile + own half of the activation rows; every byte of both CTAs is counted
     // on the even CTA's full barrier (it alone announces the byte count: one arrival per phase).
     const CUtensorMap *mw0 = &p.map_w[mi];
     const uint64_t pol = l2_policy_evict_first();
     const uint32_t lead = crank & ~1u;
     const int npre = nkb < stages ? nkb : stages;
-    for (int i = 0; i < npre; i++) {
-      if (xr == 0) mbar_expect_tx(&full[i], 2 * STAGE);
-      tma_load_2d_pair_hint(tiles + i * STAGE, mw0, (kb0 + i) * TILE_K, tm * TILE_M, mapa_u32(smem_u32(&full[i]), lead), pol);
-    }
+    if (elect_one())
+      for (int i = 0; i < npre; i++) {
+        if (xr == 0) mbar_expect_tx(&full[i], 2 * STAGE);
+        tma_load_2d_pair_hint(tiles + i * STAGE, mw0, (kb0 + i) * TILE_K, tm * TILE_M, mapa_u32(smem_u32(&full[i]), lead), pol);
+      }
+    __syncwarp();
     pdl_wait();
-    if (p.stamp) atomicMin(p.stamp, global_ns());
-    for (int i = 0; i < npre; i++)
-      tma_load_2d_pair(tiles + i * STAGE + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, xr * (NT / 2), mapa_u32(smem_u32(&full[i]), lead));
+    if (elect_one()) {
+      if (p.stamp) atomicMin(p.stamp, global_ns());
+      for (int i = 0; i < npre; i++)
+        tma_load_2d_pair(tiles + i * STAGE + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, xr * (NT / 2), mapa_u32(smem_u32(&full[i]), lead));
+    }
+    __syncwarp();
     // steady state: stage and phase advance by increments (no divisions), nothing but the wait and the copies per k-block
     int i = npre, st = 0;
     uint32_t ph = 0;
     for (; i < nkb; i++) {
       if (!mbar_wait(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 230, blockIdx.x, i); break; }
-      unsigned char *a = tiles + st * STAGE;
-      const uint32_t fb = mapa_u32(smem_u32(&full[st]), lead);
-      if (xr == 0) mbar_expect_tx(&full[st], 2 * STAGE);
-      tma_load_2d_pair_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, fb, pol);
-      tma_load_2d_pair(a + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, xr * (NT / 2), fb);
+      if (elect_one()) {
+        unsigned char *a = tiles + st * STAGE;
+        const uint32_t fb = mapa_u32(smem_u32(&full[st]), lead);
+        if (xr == 0) mbar_expect_tx(&full[st], 2 * STAGE);
+        tma_load_2d_pair_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, fb, pol);
+        tma_load_2d_pair(a + A_BYTES, &p.map_x, (kb0 + i) * TILE_K, xr * (NT / 2), fb);
+      }
+      __syncwarp();
       if (++st == stages) { st = 0; ph ^= 1u; }
     }
-    *n_issued = i;
-  } else if (warp == 0 && lane == 0) {
-    // ---- producer.  Weight tiles do not depend on the previous kernel: fill the ring with them first.
+    if (lane == 0) *n_issued = i;
+  } else if (!DUO && warp == 0) {
+    // ---- producer warp (all lanes walk the loop, the elected lane issues).  Weight tiles do not depend on the previous
+    // kernel: fill the ring with them first.
     const CUtensorMap *mw0 = &p.map_w[mi];
     const uint64_t pol = l2_policy_evict_first();
     const int npre = nkb < stages ? nkb : stages;
-    for (int i = 0; i < npre; i++) {
-      unsigned char *a = tiles + i * STAGE;
-      mbar_expect_tx(&full[i], STAGE);
-      tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[i], pol);
-      if (PAIR) tma_load_2d_hint(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[i], pol);
-    }
+    if (elect_one())
+      for (int i = 0; i < npre; i++) {
+        unsigned char *a = tiles + i * STAGE;
+        mbar_expect_tx(&full[i], STAGE);
+        tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[i], pol);
+        if (PAIR) tma_load_2d_hint(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[i], pol);
+      }
+    __syncwarp();
     pdl_wait();
-    if (p.stamp) atomicMin(p.stamp, global_ns());
-    const bool hold = p.withhold && blockIdx.x == 0 && blockIdx.y == 0;     // test hook: the first stage never completes
-    for (int i = hold ? 1 : 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + A_TILES * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
+    if (elect_one()) {
+      if (p.stamp) atomicMin(p.stamp, global_ns());
+      const bool hold = p.withhold && blockIdx.x == 0 && blockIdx.y == 0;     // test hook: the first stage never completes
+      for (int i = hold ? 1 : 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + A_TILES * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[i]);
+    }
+    __syncwarp();
     int i = npre, st = 0;             // the loop runs only when the prefill used every stage: it restarts at stage 0
     uint32_t ph = 0;
     for (; i < nkb; i++) {
       if (!mbar_wait(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
-      unsigned char *a = tiles + st * STAGE;
-      mbar_expect_tx(&full[st], STAGE);
-      tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
-      if (PAIR) tma_load_2d_hint(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
-      tma_load_2d(a + A_TILES * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[st]);
+      if (elect_one()) {
+        unsigned char *a = tiles + st * STAGE;
+        mbar_expect_tx(&full[st], STAGE);
+        tma_load_2d_hint(a, mw0, (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
+        if (PAIR) tma_load_2d_hint(a + A_BYTES, &p.map_w[1], (kb0 + i) * TILE_K, tm * TILE_M, &full[st], pol);
+        tma_load_2d(a + A_TILES * A_BYTES, &p.map_x, (kb0 + i) * TILE_K, 0, &full[st]);
+      }
+      __syncwarp();
       if (++st == stages) { st = 0; ph ^= 1u; }
     }
-    *n_issued = i;
+    if (lane == 0) *n_issued = i;
   } else {
     pdl_wait();
-    if (DUO && warp == 1 && lane == 0) {
+    if (DUO && warp == 1) {
       // ---- MMA issuer of a CTA pair (even CTA only): M = 256 over both CTAs' weight tiles, N = both activation halves
       if (xr == 0) {
         constexpr uint32_t idesc = umma_idesc_m(NT, 2 * TILE_M);
@@ -267,16 +284,23 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
             int nst = st + 1;
             uint32_t nph = ph;
             if (nst == stages) { nst = 0; nph ^= 1u; }
-            ready = umma_kblock_peek_pair(tmem_base, da, da + (A_BYTES >> 4), idesc, i ? 1u : 0u, &empty[st], pair_mask, smem_u32(&full[nst]), nph);
+            if (elect_one()) {
+#pragma unroll
+              for (int j = 0; j < TILE_K / UMMA_K; j++) umma_bf16_pair(tmem_base, da + 2 * j, da + (A_BYTES >> 4) + 2 * j, idesc, (i | j) ? 1u : 0u);
+              umma_commit_pair(&empty[st], pair_mask);      // frees the stage in both CTAs
+            }
+            __syncwarp();
+            ready = mbar_test(&full[nst], nph) ? 1u : 0u;
             st = nst; ph = nph;
           }
-        *n_consumed = i;
-        if (!*abort_flag) umma_commit_pair(acc_bar, pair_mask);   // both accumulators complete
+        if (lane == 0) *n_consumed = i;
+        __syncwarp();
+        if (!*abort_flag && elect_one()) umma_commit_pair(acc_bar, pair_mask);   // both accumulators complete
       }
-    } else if (warp == 1 && lane == 0) {
-      // ---- MMA issuer
-      // The issuing thread is what limits a CTA's streaming rate, so the loop is kept to the wait (skipped when the
-      // peek of the previous iteration already saw the stage full), one fence and one instruction sequence per k-block.
+    } else if (!DUO && warp == 1) {
+      // ---- MMA issuer warp (all lanes walk the loop, the elected lane issues)
+      // The issuing warp is what limits a CTA's streaming rate, so the loop is kept to a non-blocking look at the
+      // barrier (the blocking wait only when the stage is not full yet), one fence, four MMAs and the commit.
       constexpr uint32_t idesc = umma_idesc(NT);
       const uint64_t desc0 = umma_desc_sw128(smem_u32(tiles));
       int i = 0, st = 0;
@@ -288,12 +312,20 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
         int nst = st + 1;
         uint32_t nph = ph;
         if (nst == stages) { nst = 0; nph ^= 1u; }
-        if (PAIR) umma_kblock(tmem_base + NT, da + (A_BYTES >> 4), db, idesc, i ? 1u : 0u);   // the up accumulator
-        ready = umma_kblock_peek(tmem_base, da, db, idesc, i ? 1u : 0u, &empty[st], smem_u32(&full[nst]), nph);   // + commit: frees the stage
+        if (elect_one()) {
+#pragma unroll
+          for (int j = 0; j < TILE_K / UMMA_K; j++) {      // a K = 16 step advances the descriptors by 32 bytes = 2 units
+            umma_bf16(tmem_base, da + 2 * j, db + 2 * j, idesc, (i | j) ? 1u : 0u);
+            if (PAIR) umma_bf16(tmem_base + NT, da + (A_BYTES >> 4) + 2 * j, db + 2 * j, idesc, (i | j) ? 1u : 0u);   // the up accumulator
+          }
+          umma_commit(&empty[st]);      // frees the stage once these MMAs have read it
+        }
+        __syncwarp();
+        ready = mbar_test(&full[nst], nph) ? 1u : 0u;      // a cheap look at the next stage: mostly spares the wait
         st = nst; ph = nph;
       }
-      *n_consumed = i;
-      umma_commit(acc_bar);           // accumulator complete
+      if (lane == 0) *n_consumed = i;
+      if (elect_one()) umma_commit(acc_bar);           // accumulator complete
     } else if (warp >= 2) {
       // ---- per-row scale of the input: rsqrt(mean square + eps) from the producer kernel's per-tile sums
       for (int r = threadIdx.x - 64; r < p.rows; r += 64) {
@@ -621,35 +653,43 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
   const uint32_t tmem_base = *tmem_slot;
   pdl_trigger();
 
-  if (warp == 0 && lane == 0) {
-    // ---- producer: the weight tiles do not depend on the previous kernel
+  if (warp == 0) {
+    // ---- producer warp (the elected lane issues): the weight tiles do not depend on the previous kernel
     const uint64_t pol = l2_policy_evict_first();
     const int npre = KB < stages ? KB : stages;
-    for (int i = 0; i < npre; i++) {
-      unsigned char *a = tiles + i * STAGE;
-      mbar_expect_tx(&full[i], STAGE);
-      tma_load_2d_hint(a, &p.map_w[0], i * TILE_K, tm * TILE_M, &full[i], pol);
-      tma_load_2d_hint(a + A_BYTES, &p.map_w[1], i * TILE_K, tm * TILE_M, &full[i], pol);
-    }
+    if (elect_one())
+      for (int i = 0; i < npre; i++) {
+        unsigned char *a = tiles + i * STAGE;
+        mbar_expect_tx(&full[i], STAGE);
+        tma_load_2d_hint(a, &p.map_w[0], i * TILE_K, tm * TILE_M, &full[i], pol);
+        tma_load_2d_hint(a + A_BYTES, &p.map_w[1], i * TILE_K, tm * TILE_M, &full[i], pol);
+      }
+    __syncwarp();
     pdl_wait();
-    if (p.stamp) atomicMin(p.stamp, global_ns());
-    for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + 2 * A_BYTES, &p.map_x, i * TILE_K, 0, &full[i]);
+    if (elect_one()) {
+      if (p.stamp) atomicMin(p.stamp, global_ns());
+      for (int i = 0; i < npre; i++) tma_load_2d(tiles + i * STAGE + 2 * A_BYTES, &p.map_x, i * TILE_K, 0, &full[i]);
+    }
+    __syncwarp();
     int i = npre, st = 0;
     uint32_t ph = 0;
     for (; i < KB; i++) {
       if (!mbar_wait(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 220, blockIdx.x, i); break; }
-      unsigned char *a = tiles + st * STAGE;
-      mbar_expect_tx(&full[st], STAGE);
-      tma_load_2d_hint(a, &p.map_w[0], i * TILE_K, tm * TILE_M, &full[st], pol);
-      tma_load_2d_hint(a + A_BYTES, &p.map_w[1], i * TILE_K, tm * TILE_M, &full[st], pol);
-      tma_load_2d(a + 2 * A_BYTES, &p.map_x, i * TILE_K, 0, &full[st]);
+      if (elect_one()) {
+        unsigned char *a = tiles + st * STAGE;
+        mbar_expect_tx(&full[st], STAGE);
+        tma_load_2d_hint(a, &p.map_w[0], i * TILE_K, tm * TILE_M, &full[st], pol);
+        tma_load_2d_hint(a + A_BYTES, &p.map_w[1], i * TILE_K, tm * TILE_M, &full[st], pol);
+        tma_load_2d(a + 2 * A_BYTES, &p.map_x, i * TILE_K, 0, &full[st]);
+      }
+      __syncwarp();
       if (++st == stages) { st = 0; ph ^= 1u; }
     }
-    *n_issued = i;
+    if (lane == 0) *n_issued = i;
   } else {
     pdl_wait();
-    if (warp == 1 && lane == 0) {
-      // ---- MMA issuer: gate accumulator at column 0, up accumulator at column NT
+    if (warp == 1) {
+      // ---- MMA issuer warp (the elected lane issues): gate accumulator at column 0, up accumulator at column NT
       constexpr uint32_t idesc = umma_idesc(NT);
       const uint64_t desc0 = umma_desc_sw128(smem_u32(tiles));
       int i = 0, st = 0;
@@ -661,12 +701,21 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
         int nst = st + 1;
         uint32_t nph = ph;
         if (nst == stages) { nst = 0; nph ^= 1u; }
-        umma_kblock(tmem_base + NT, du, db, idesc, i ? 1u : 0u);
-        ready = umma_kblock_peek(tmem_base, dg, db, idesc, i ? 1u : 0u, &empty[st], smem_u32(&full[nst]), nph);
+        if (elect_one()) {
+#pragma unroll
+          for (int j = 0; j < TILE_K / UMMA_K; j++) {
+            umma_bf16(tmem_base, dg + 2 * j, db + 2 * j, idesc, (i | j) ? 1u : 0u);
+            umma_bf16(tmem_base + NT, du + 2 * j, db + 2 * j, idesc, (i | j) ? 1u : 0u);
+          }
+          umma_commit(&empty[st]);
+        }
+        __syncwarp();
+        ready = mbar_test(&full[nst], nph) ? 1u : 0u;
         st = nst; ph = nph;
       }
-      *n_consumed = i;
-      umma_commit(acc_bar);
+      if (lane == 0) *n_consumed = i;
+      __syncwarp();
+      if (elect_one()) umma_commit(acc_bar);
     } else if (warp >= 2) {
       for (int r = threadIdx.x - 64; r < p.rows; r += 64) {
         float sc = 1.0f;

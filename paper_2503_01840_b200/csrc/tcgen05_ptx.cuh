@@ -14,14 +14,35 @@ constexpr uint32_t SPIN_LIMIT = 1u << 20;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// One lane of a fully converged warp (all 32 lanes must execute this).  The producer and the MMA issuer walk their loops
+// as whole warps and let the elected lane issue the copies / MMAs: issued from a branch on the lane id instead, every
+// tcgen05 / bulk-copy / mbarrier instruction costs the thread far more cycles (measured: the same loop ran 2-3 x slower).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred = 0;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\t@p mov.u32 %0, 1;\n\t}" : "+r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+// non-blocking: has the phase with this parity completed?  (13 cycles for a warp, against ~126 for a try_wait that succeeds at once)
+__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // bounded wait; false on timeout
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint32_t limit = SPIN_LIMIT) {
+  if (mbar_test(bar, parity)) return true;
   uint32_t addr = smem_u32(bar);
   for (uint32_t it = 0; it < limit; it++) {
     uint32_t ok;
@@ -122,59 +143,6 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar, uint16_t cta_mas
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(smem_u32(bar)),
                "h"(cta_mask)
                : "memory");
-}
-// ---- One k-block of the main loop in a single instruction sequence: a non-blocking test of the NEXT stage's "full"
-// barrier is issued first, then the four K = 16 MMAs of this stage (descriptors advance by 32 bytes = 2 units), then
-// the commit that frees the stage; the test's result is read last, so that its latency hides behind the MMA issue.
-// Returns 1 when the tested phase is complete (the caller then skips its wait).  The issuing thread is the bottleneck
-// of a weight-streaming CTA: every instruction saved here is bandwidth.
-#define SPEC_KBLOCK_BODY(MMA, COMMIT)                                                                              \
-  "{\n\t.reg .pred p, q, t;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"                                             \
-  "setp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 t, 0, 0;\n\t"                                                                                     \
-  "mbarrier.test_wait.parity.shared::cta.b64 q, [%7], %8;\n\t"                                                    \
-  "add.s64 a1, %2, 2;\n\tadd.s64 a2, %2, 4;\n\tadd.s64 a3, %2, 6;\n\t"                                           \
-  "add.s64 b1, %3, 2;\n\tadd.s64 b2, %3, 4;\n\tadd.s64 b3, %3, 6;\n\t"                                           \
-  MMA " [%1], %2, %3, %4, p;\n\t"                                                                                 \
-  MMA " [%1], a1, b1, %4, t;\n\t"                                                                                 \
-  MMA " [%1], a2, b2, %4, t;\n\t"                                                                                 \
-  MMA " [%1], a3, b3, %4, t;\n\t"                                                                                 \
-  COMMIT "\n\t"                                                                                                   \
-  "selp.u32 %0, 1, 0, q;\n\t}"
-
-__device__ __forceinline__ uint32_t umma_kblock_peek(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate,
-                                                     uint64_t *commit_bar, uint32_t peek_bar_addr, uint32_t peek_parity) {
-  uint32_t ok;
-  asm volatile(SPEC_KBLOCK_BODY("tcgen05.mma.cta_group::1.kind::f16", "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%6];")
-               : "=r"(ok)
-               : "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(smem_u32(commit_bar)), "r"(peek_bar_addr), "r"(peek_parity)
-               : "memory");
-  return ok;
-}
-// the same for a CTA pair (M = 256 across both CTAs; the commit arrives in every CTA of cta_mask)
-__device__ __forceinline__ uint32_t umma_kblock_peek_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate,
-                                                          uint64_t *commit_bar, uint16_t cta_mask, uint32_t peek_bar_addr, uint32_t peek_parity) {
-  uint32_t ok;
-  asm volatile(SPEC_KBLOCK_BODY("tcgen05.mma.cta_group::2.kind::f16",
-                                "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%6], %9;")
-               : "=r"(ok)
-               : "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(smem_u32(commit_bar)), "r"(peek_bar_addr), "r"(peek_parity),
-                 "h"(cta_mask)
-               : "memory");
-  return ok;
-}
-// four MMAs of a k-block without commit or peek (the second accumulator of a gate/up pair)
-__device__ __forceinline__ void umma_kblock(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p, t;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\tsetp.eq.b32 t, 0, 0;\n\t"
-      "add.s64 a1, %1, 2;\n\tadd.s64 a2, %1, 4;\n\tadd.s64 a3, %1, 6;\n\t"
-      "add.s64 b1, %2, 2;\n\tadd.s64 b2, %2, 4;\n\tadd.s64 b3, %2, 6;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %3, t;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], a2, b2, %3, t;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], a3, b3, %3, t;\n\t}" ::"r"(tmem_d),
-      "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
-      : "memory");
 }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
