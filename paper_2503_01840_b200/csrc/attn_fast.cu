@@ -290,8 +290,21 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One lane of a fully converged warp: the producer and issuer warps walk their loops whole and let this lane issue the
+// copies / MMAs (the same instructions issued from a branch on the lane id cost the warp about 1.5 x the cycles).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred = 0;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\t@p mov.u32 %0, 1;\n\t}" : "+r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
   uint32_t addr = smem_u32(bar);
+  {   // non-blocking test first: a phase that is already complete costs a tenth of a try_wait
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+    if (ok) return true;
+  }
   for (uint32_t it = 0; it < ATT_SPIN_LIMIT; it++) {
     uint32_t ok;
     asm volatile(
@@ -383,7 +396,7 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
     }
     __syncwarp();
     asm volatile("bar.arrive 1, 288;" ::: "memory");
-    if (lane == 0 && seq >= 0) {
+    if (seq >= 0) {     // the whole warp walks the loop (same page ids in every lane), the elected lane issues the copies
       const int32_t *tbl = p.pm.table + (size_t)seq * p.pm.pages_per_seq;
       const int fallback = tbl[0];                     // keys past the last page are masked; they still need a valid source
       const int ppt = KT / ps;                         // pages per tile
@@ -394,17 +407,20 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
         if (t + 1 < t_end) tile_pages(nxt, tbl, p.pm.pages_per_seq, t + 1, ps);
         if (i == STAGES - 1 && !mbar_wait(q_bar, 0)) { if (status) set_status(status, ST_TIMEOUT, 400, blockIdx.z, t); break; }
         if (i >= STAGES && !mbar_wait(&empty[st], (uint32_t)(((i / STAGES) - 1) & 1))) { if (status) set_status(status, ST_TIMEOUT, 401, blockIdx.z, t); break; }
-        unsigned char *kb = sm + st * 2 * TILEB, *vb = kb + TILEB;
-        mbar_expect_tx(&full[st], 2 * TILEB);
+        if (elect_one()) {
+          unsigned char *kb = sm + st * 2 * TILEB, *vb = kb + TILEB;
+          mbar_expect_tx(&full[st], 2 * TILEB);
 #pragma unroll
-        for (int pg = 0; pg < 4; pg++) {
-          if (pg >= ppt) break;
-          int page = cur[pg];
-          if (page < 0 || page >= p.pm.num_pages) page = fallback;
-          const int row = (page * p.G + g) * ps;
-          tma_load_3d(kb + pg * ps * ROWB, &map_k, 0, row, 0, &full[st]);
-          tma_load_3d(vb + pg * ps * ROWB, &map_v, 0, row, 0, &full[st]);
+          for (int pg = 0; pg < 4; pg++) {
+            if (pg >= ppt) break;
+            int page = cur[pg];
+            if (page < 0 || page >= p.pm.num_pages) page = fallback;
+            const int row = (page * p.G + g) * ps;
+            tma_load_3d(kb + pg * ps * ROWB, &map_k, 0, row, 0, &full[st]);
+            tma_load_3d(vb + pg * ps * ROWB, &map_v, 0, row, 0, &full[st]);
+          }
         }
+        __syncwarp();
 #pragma unroll
         for (int pg = 0; pg < 4; pg++) cur[pg] = nxt[pg];
       }
@@ -694,7 +710,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
 
   if (warp == 8) {
     // ================================================================ producer
-    if (lane == 0 && seq >= 0) {
+    if (seq >= 0) {     // the whole warp walks the loop, the elected lane issues the copies
       const int32_t *tbl = p.pm.table + (size_t)seq * p.pm.pages_per_seq;
       const int fallback = tbl[0];                     // keys past the last page are masked; they still need a valid source
       const int ppt = KT / ps;                         // pages per tile
@@ -709,27 +725,30 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
           break;
         }
         if (*abort_flag) break;
-        unsigned char *kb = ring + st * 2 * UM_TILE, *vb = kb + UM_TILE;
-        mbar_expect_tx(&full[st], 2 * UM_TILE);
+        if (elect_one()) {
+          unsigned char *kb = ring + st * 2 * UM_TILE, *vb = kb + UM_TILE;
+          mbar_expect_tx(&full[st], 2 * UM_TILE);
 #pragma unroll
-        for (int pg = 0; pg < 4; pg++) {
-          if (pg >= ppt) break;
-          int page = cur[pg];
-          if (page < 0 || page >= p.pm.num_pages) page = fallback;
-          const int row = (page * p.G + g) * ps;
+          for (int pg = 0; pg < 4; pg++) {
+            if (pg >= ppt) break;
+            int page = cur[pg];
+            if (page < 0 || page >= p.pm.num_pages) page = fallback;
+            const int row = (page * p.G + g) * ps;
 #pragma unroll
-          for (int h = 0; h < 2; h++) {
-            tma_load_3d(kb + h * UM_HALF + pg * ps * 128, &map_k, 0, row, h, &full[st]);
-            tma_load_3d(vb + h * UM_HALF + pg * ps * 128, &map_v, 0, row, h, &full[st]);
+            for (int h = 0; h < 2; h++) {
+              tma_load_3d(kb + h * UM_HALF + pg * ps * 128, &map_k, 0, row, h, &full[st]);
+              tma_load_3d(vb + h * UM_HALF + pg * ps * 128, &map_v, 0, row, h, &full[st]);
+            }
           }
         }
+        __syncwarp();
 #pragma unroll
         for (int pg = 0; pg < 4; pg++) cur[pg] = nxt[pg];
       }
     }
   } else if (warp == 9) {
     // ================================================================ MMA issuer
-    if (lane == 0 && ntl > 0) {
+    if (ntl > 0) {      // the whole warp walks the loop, the elected lane issues the MMAs and commits
       constexpr uint32_t idesc_s = tc::umma_idesc(KT);                       // N = 64 keys, both operands K-major
       constexpr uint32_t idesc_o = tc::umma_idesc(HD) | (1u << 16);          // N = 128, B (the V tile) MN-major
       const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP);
@@ -752,7 +771,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
         ok = mbar_wait(&full[i % UM_STAGES], 0);
         if (!ok) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 421, blockIdx.z, t_begin + i); break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        issue_s(i);
+        if (elect_one()) issue_s(i);
+        __syncwarp();
       }
       if (ok) {
         for (int i = 0; i < ntl; i++) {
@@ -761,17 +781,21 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
           if (*abort_flag) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t v_addr = smem_u32(ring + st * 2 * UM_TILE + UM_TILE);
+          if (elect_one()) {
 #pragma unroll
-          for (int kk = 0; kk < KT / tc::UMMA_K; kk++)
-            tc::umma_bf16(tmem_o + (uint32_t)((i & 1) * HD), tc::umma_desc_sw128(p_addr + (i & 1) * UM_P_BYTES + kk * 32),
-                          umma_desc_sw128_mn(v_addr + kk * (tc::UMMA_K * 128), UM_HALF), idesc_o, ((i >> 1) | kk) ? 1u : 0u);
-          tc::umma_commit(&o_bar[i & 1]);
-          tc::umma_commit(&empty[st]);
+            for (int kk = 0; kk < KT / tc::UMMA_K; kk++)
+              tc::umma_bf16(tmem_o + (uint32_t)((i & 1) * HD), tc::umma_desc_sw128(p_addr + (i & 1) * UM_P_BYTES + kk * 32),
+                            umma_desc_sw128_mn(v_addr + kk * (tc::UMMA_K * 128), UM_HALF), idesc_o, ((i >> 1) | kk) ? 1u : 0u);
+            tc::umma_commit(&o_bar[i & 1]);
+            tc::umma_commit(&empty[st]);
+          }
+          __syncwarp();
           if (i + 2 < ntl) {          // this group's score buffer is free: its threads read it before they arrived on p_bar
             const int st2 = (i + 2) % UM_STAGES;
             if (!mbar_wait(&full[st2], (uint32_t)(((i + 2) / UM_STAGES) & 1))) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 423, blockIdx.z, t_begin + i + 2); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            issue_s(i + 2);
+            if (elect_one()) issue_s(i + 2);
+            __syncwarp();
           }
         }
       }
@@ -969,7 +993,7 @@ __global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_consta
   __syncthreads();
 
   if (warp == NW) {
-    if (lane == 0 && seq >= 0) {
+    if (seq >= 0) {     // the whole warp walks the loop, the elected lane issues the copies
       const int32_t *tbl = p.pm.table + (size_t)seq * p.pm.pages_per_seq;
       const int fallback = tbl[0];
       const int ppt = KT / ps;
@@ -979,17 +1003,20 @@ __global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_consta
         const int i = t - t_begin, st = i % STAGES;
         if (t + 1 < t_end) tile_pages(nxt, tbl, p.pm.pages_per_seq, t + 1, ps);
         if (i >= STAGES && !mbar_wait(&empty[st], (uint32_t)(((i / STAGES) - 1) & 1))) { if (status) set_status(status, ST_TIMEOUT, 411, blockIdx.z, t); break; }
-        unsigned char *kb = sm + st * 2 * TILEB, *vb = kb + TILEB;
-        mbar_expect_tx(&full[st], 2 * TILEB);
+        if (elect_one()) {
+          unsigned char *kb = sm + st * 2 * TILEB, *vb = kb + TILEB;
+          mbar_expect_tx(&full[st], 2 * TILEB);
 #pragma unroll
-        for (int pg = 0; pg < 4; pg++) {
-          if (pg >= ppt) break;
-          int page = cur[pg];
-          if (page < 0 || page >= p.pm.num_pages) page = fallback;
-          const int row = (page * p.G + g) * ps;
-          tma_load_3d(kb + pg * ps * ROWB, &map_k, 0, row, 0, &full[st]);
-          tma_load_3d(vb + pg * ps * ROWB, &map_v, 0, row, 0, &full[st]);
+          for (int pg = 0; pg < 4; pg++) {
+            if (pg >= ppt) break;
+            int page = cur[pg];
+            if (page < 0 || page >= p.pm.num_pages) page = fallback;
+            const int row = (page * p.G + g) * ps;
+            tma_load_3d(kb + pg * ps * ROWB, &map_k, 0, row, 0, &full[st]);
+            tma_load_3d(vb + pg * ps * ROWB, &map_v, 0, row, 0, &full[st]);
+          }
         }
+        __syncwarp();
 #pragma unroll
         for (int pg = 0; pg < 4; pg++) cur[pg] = nxt[pg];
       }
