@@ -35,10 +35,10 @@ UNIT = "tok/s"
 
 # DRAM traffic of the GEMM kernel relative to its weight bytes, from the ncu capture summarised in
 # profiles/gemm_fused_kernel_C2_shapes_ncu_full.md: (dram__bytes_read.sum + dram__bytes_write.sum) of the four GEMMs
-# of an 8B-shaped layer = 449.2 MB for 436.2 MB of weights.  The capture ran on the 2-layer truncation (same kernels,
+# of an 8B-shaped layer = 448.6 MB for 436.2 MB of weights.  The capture ran on the 2-layer truncation (same kernels,
 # same shapes); a full step's traffic is that ratio times its weight bytes (traffic grows with the weight bytes).
 # Valid for the 8B shapes at 60 rows only; None elsewhere.
-NCU_TRAFFIC_RATIO = {"C2-8B-b1": 449.2 / 436.2}
+NCU_TRAFFIC_RATIO = {"C2-8B-b1": 448.6 / 436.2}
 
 
 def peaks():

@@ -338,8 +338,8 @@ __device__ __forceinline__ void tile_pages(int (&pg)[4], const int32_t *tbl, int
 template <int HD, int STAGES>
 __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ CUtensorMap map_k,
                                                        const __grid_constant__ CUtensorMap map_v, AttnParams p, int32_t *status) {
+  pdl_trigger();   // the next kernel may start staging its weights; it still waits for this grid to complete
   pdl_wait();
-  pdl_trigger();
   KernelStamp stamp_guard(p.stamp);
   constexpr int ROWB = HD * 2, CPR = HD / 8;
   constexpr int NKS = HD / 16;
@@ -631,8 +631,8 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
 
 __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_constant__ CUtensorMap map_k,
                                                         const __grid_constant__ CUtensorMap map_v, AttnParams p, int32_t *status) {
+  pdl_trigger();   // the next kernel may start staging its weights; it still waits for this grid to complete
   pdl_wait();
-  pdl_trigger();
   KernelStamp stamp_guard(p.stamp);
   constexpr int HD = UM_HD;
   extern __shared__ __align__(1024) unsigned char sm[];
@@ -947,8 +947,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
 template <int HD, int STAGES>
 __global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_constant__ CUtensorMap map_k,
                                                              const __grid_constant__ CUtensorMap map_v, AttnParams p, int32_t *status) {
+  pdl_trigger();   // the next kernel may start staging its weights; it still waits for this grid to complete
   pdl_wait();
-  pdl_trigger();
   KernelStamp stamp_guard(p.stamp);
   constexpr int ROWB = HD * 2, CPR = HD / 8;
   constexpr int NKS = HD / 16;
@@ -1155,8 +1155,8 @@ __global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_consta
 template <int HD>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml, int nsplit,
                                                            int nrh, bf16 *__restrict__ out, unsigned long long *stamp) {
+  pdl_trigger();   // the next kernel may start staging its weights; it still waits for this grid to complete
   pdl_wait();
-  pdl_trigger();
   KernelStamp stamp_guard(stamp, false);
   constexpr int DPL = HD / 32;                              // dimensions per lane
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
