@@ -14,6 +14,7 @@ runs an independent replica (the path has no collective), so the value is the su
 Prints ONE JSON line on rank 0.
 """
 import argparse
+import gc
 import json
 import os
 import statistics
@@ -415,6 +416,7 @@ def main():
         if cfg.n_layers <= CPU_FULL_DEPTH_MAX_LAYERS:
             line["cpu_baseline"] = cpu_baseline(cfg, tw, dw)          # reuses the weights that are already generated
         del dec, tw, dw                      # the 70B-shaped weights leave no room for a second model beside them
+        gc.collect()
         torch.cuda.empty_cache()
         if cfg.batch == 1 and cfg.tree_depth >= 2:
             # designed draft/target agreement: same shapes and bytes, acceptance length near the paper's

@@ -213,6 +213,8 @@ class SpecDecoder:
         if getattr(self, "h", None):
             lib().spec_free(self.h)
             self.h = None
+        self._keep = []          # the weights and the workspace may be freed once the context is gone
+        self.workspace = None
 
     def __del__(self):
         try:
