@@ -158,7 +158,9 @@ enum spec_tune_knob { SPEC_TUNE_GEMM_CTAS = 2,
                       SPEC_TUNE_DEBUG_WAIT_RUNS_OUT = 5 /* test hook for the bounded device waits: with a value n > 0 one CTA of the verify
                                                   pass's LM-head GEMM never receives its first activation tile and gives up after n
                                                   polls; the step then returns SPEC_ERR_DEVICE_STATUS (0 = off) */,
-                      SPEC_TUNE_GEMM_PAIRS = 7 /* 256-row GEMM tiles of neighbouring feature tiles as CTA pairs (1) or single CTAs (0, default: pairs measured no faster); process-wide; the one knob that may be set with a NULL ctx */,
+                      SPEC_TUNE_GEMM_PAIRS = 7 /* 256-row GEMM tiles of neighbouring feature tiles as CTA pairs (tcgen05 cta_group::2): bit 0 = the split-K
+                                                  kernel (default off: measured no faster), bit 1 = the gate/up kernel (default on); process-wide;
+                                                  the one knob that may be set with a NULL ctx */,
                       SPEC_TUNE_ATTN_UMMA = 6 /* tree passes (head_dim 128): 1 = tcgen05 attention kernel, 0 = mma.sync kernel, 2 (default) = tcgen05
                                                   when every CTA gets several key tiles, i.e. long contexts (process-wide) */ };
 int spec_tune(spec_ctx *ctx, int32_t what, int32_t value);

@@ -921,7 +921,7 @@ extern "C" int spec_profile_step(spec_ctx *c, float *class_ms, int32_t *class_la
 extern "C" int spec_tune(spec_ctx *c, int32_t what, int32_t value) {
   if (!c) {   // the per-kernel entry points have no context: the pair switch alone may be set without one
     if (what != SPEC_TUNE_GEMM_PAIRS) return SPEC_ERR_NULL;
-    if (value < 0 || value > 1) return SPEC_ERR_INVALID_CFG;
+    if (value < 0 || value > 3) return SPEC_ERR_INVALID_CFG;
     fused_gemm_set_pairs(value);
     return SPEC_OK;
   }
@@ -937,7 +937,7 @@ extern "C" int spec_tune(spec_ctx *c, int32_t what, int32_t value) {
     if (value < 0 || value > (1 << 20)) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the poll count must be 0..2^20");
     c->dbg_withhold_spin = value;
   } else if (what == SPEC_TUNE_GEMM_PAIRS) {
-    if (value < 0 || value > 1) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the CTA-pair switch must be 0 or 1");
+    if (value < 0 || value > 3) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the CTA-pair switch must be 0..3");
     fused_gemm_set_pairs(value);
   } else if (what == SPEC_TUNE_GEMM_CTAS) {
     if (value < 32 || value > 2048) return fail(c, SPEC_ERR_INVALID_CFG, "spec_tune: the GEMM CTA target must be 32..2048");

@@ -614,9 +614,12 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
 // (64 KB per stage instead of 96), the two accumulators fill the tensor memory (2 x 256 columns), and since a thread
 // then holds gate and up of its feature for every row the activation is applied straight from the accumulators:
 // no cluster, no shared-memory round trip.
-template <int NT>
+// DUO: two neighbouring feature tiles as a CTA pair (cta_group::2, cluster of 2): each CTA streams its own gate and up
+// tile and HALF of the activation rows, the even CTA issues one M = 256 MMA per accumulator and k-step (fill bytes per
+// k-block 48 KB instead of 64 KB per CTA, four stages instead of three).
+template <int NT, bool DUO = false>
 __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_constant__ FusedParams p) {
-  constexpr int B_BYTES = NT * TILE_K * 2;
+  constexpr int B_BYTES = (DUO ? NT / 2 : NT) * TILE_K * 2;
   constexpr int STAGE = 2 * A_BYTES + B_BYTES;
   constexpr int TMEM_COLS = 2 * NT;
   static_assert(TMEM_COLS <= 512, "two accumulators must fit the tensor memory");
@@ -634,26 +637,73 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int stages = p.stages, KB = p.KB;
   const int tm = blockIdx.x;                     // feature tile (of gate and of up)
+  const uint32_t crank = DUO ? cluster_rank() : 0u;
+  const int xr = (int)(crank & 1u);              // DUO: position in the pair (0 issues the MMAs)
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < stages; i++) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     mbar_init(acc_bar, 1);
     *abort_flag = 0;
     *n_issued = 0; *n_consumed = 0;
+    if (DUO && crank != (blockIdx.x & 1u)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 224, blockIdx.x, (int)crank); }   // pairs = (even, odd) tile
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (DUO) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
+  if (DUO) cluster_sync_all(); else __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
   pdl_trigger();
 
-  if (warp == 0) {
+  if (DUO && *abort_flag) {
+    pdl_wait();
+  } else if (DUO && warp == 0) {
+    // ---- producer warp of a CTA pair: every byte of both CTAs is counted on the even CTA's full barrier
+    const uint64_t pol = l2_policy_evict_first();
+    const int npre = KB < stages ? KB : stages;
+    if (elect_one())
+      for (int i = 0; i < npre; i++) {
+        unsigned char *a = tiles + i * STAGE;
+        const uint32_t fb = mapa_u32(smem_u32(&full[i]), 0u);
+        if (xr == 0) mbar_expect_tx(&full[i], 2 * STAGE);
+        tma_load_2d_pair_hint(a, &p.map_w[0], i * TILE_K, tm * TILE_M, fb, pol);
+        tma_load_2d_pair_hint(a + A_BYTES, &p.map_w[1], i * TILE_K, tm * TILE_M, fb, pol);
+      }
+    __syncwarp();
+    pdl_wait();
+    if (elect_one()) {
+      if (p.stamp) atomicMin(p.stamp, global_ns());
+      for (int i = 0; i < npre; i++)
+        tma_load_2d_pair(tiles + i * STAGE + 2 * A_BYTES, &p.map_x, i * TILE_K, xr * (NT / 2), mapa_u32(smem_u32(&full[i]), 0u));
+    }
+    __syncwarp();
+    int i = npre, st = 0;
+    uint32_t ph = 0;
+    for (; i < KB; i++) {
+      if (!mbar_wait(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 225, blockIdx.x, i); break; }
+      if (elect_one()) {
+        unsigned char *a = tiles + st * STAGE;
+        const uint32_t fb = mapa_u32(smem_u32(&full[st]), 0u);
+        if (xr == 0) mbar_expect_tx(&full[st], 2 * STAGE);
+        tma_load_2d_pair_hint(a, &p.map_w[0], i * TILE_K, tm * TILE_M, fb, pol);
+        tma_load_2d_pair_hint(a + A_BYTES, &p.map_w[1], i * TILE_K, tm * TILE_M, fb, pol);
+        tma_load_2d_pair(a + 2 * A_BYTES, &p.map_x, i * TILE_K, xr * (NT / 2), fb);
+      }
+      __syncwarp();
+      if (++st == stages) { st = 0; ph ^= 1u; }
+    }
+    if (lane == 0) *n_issued = i;
+  } else if (!DUO && warp == 0) {
     // ---- producer warp (the elected lane issues): the weight tiles do not depend on the previous kernel
     const uint64_t pol = l2_policy_evict_first();
     const int npre = KB < stages ? KB : stages;
@@ -688,7 +738,40 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
     if (lane == 0) *n_issued = i;
   } else {
     pdl_wait();
-    if (warp == 1) {
+    if (DUO && warp == 1) {
+      // ---- MMA issuer warp of a CTA pair (even CTA only): M = 256 over both CTAs' gate tiles, then both up tiles
+      if (xr == 0) {
+        constexpr uint32_t idesc = umma_idesc_m(NT, 2 * TILE_M);
+        const uint32_t partner_base = ld_peer_u32(smem_u32(tmem_slot), 1u);
+        if (partner_base != tmem_base) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 226, blockIdx.x, (int)partner_base); }
+        const uint64_t desc0 = umma_desc_sw128(smem_u32(tiles));
+        int i = 0, st = 0;
+        uint32_t ph = 0, ready = 0;
+        if (!*abort_flag)
+          for (; i < KB; i++) {
+            if (!ready && !mbar_wait(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 227, blockIdx.x, i); break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t dg = desc0 + (uint64_t)((st * STAGE) >> 4), du = dg + (A_BYTES >> 4), db = dg + ((2 * A_BYTES) >> 4);
+            int nst = st + 1;
+            uint32_t nph = ph;
+            if (nst == stages) { nst = 0; nph ^= 1u; }
+            if (elect_one()) {
+#pragma unroll
+              for (int j = 0; j < TILE_K / UMMA_K; j++) {
+                umma_bf16_pair(tmem_base, dg + 2 * j, db + 2 * j, idesc, (i | j) ? 1u : 0u);
+                umma_bf16_pair(tmem_base + NT, du + 2 * j, db + 2 * j, idesc, (i | j) ? 1u : 0u);
+              }
+              umma_commit_pair(&empty[st], (uint16_t)3);
+            }
+            __syncwarp();
+            ready = mbar_test(&full[nst], nph) ? 1u : 0u;
+            st = nst; ph = nph;
+          }
+        if (lane == 0) *n_consumed = i;
+        __syncwarp();
+        if (!*abort_flag && elect_one()) umma_commit_pair(acc_bar, (uint16_t)3);
+      }
+    } else if (!DUO && warp == 1) {
       // ---- MMA issuer warp (the elected lane issues): gate accumulator at column 0, up accumulator at column NT
       constexpr uint32_t idesc = umma_idesc(NT);
       const uint64_t desc0 = umma_desc_sw128(smem_u32(tiles));
@@ -760,14 +843,15 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
       }
     }
   }
-  if (*abort_flag && threadIdx.x == 0) {      // no bulk copy may still be landing when the CTA exits
+  if (*abort_flag && threadIdx.x == 0 && xr == 0) {      // no bulk copy may still be landing when the CTA exits
     for (int i = *n_consumed; i < *n_issued; i++) mbar_wait(&full[i % stages], (i / stages) & 1, p.spin);
   }
 
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
+  if (DUO) cluster_sync_all(); else __syncthreads();   // pairs: neither CTA frees tensor memory the other's MMAs may still use
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if (DUO) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
   if (p.stamp && threadIdx.x == 0) atomicMin(p.stamp + 1, ~global_ns());
 }
@@ -931,8 +1015,10 @@ int launch_swiglu_pair(const FusedParams &p, const Plan &pl, bool pdl, cudaStrea
 }  // namespace
 
 void fused_gemm_set_target_ctas(int n) { g_target_ctas = n; }
-namespace { int g_pairs = 0; }   // 256-row tiles of neighbouring feature tiles as CTA pairs (measured: no gain, off by default)
-void fused_gemm_set_pairs(int on) { g_pairs = on ? 1 : 0; }
+// 256-row tiles of neighbouring feature tiles as CTA pairs.  Bit 0: the split-K kernel (measured no faster: off); bit 1: the
+// gate/up kernel (gate/up launch -1 %, C3 step -0.6 %: on)
+namespace { int g_pairs = 0, g_pairs_swiglu = 1; }
+void fused_gemm_set_pairs(int on) { g_pairs = on & 1; g_pairs_swiglu = (on >> 1) & 1; }
 
 int fused_gemm_tiles(FusedEpi epi, const FusedGemmArgs &a) {
   if (epi == EPI_SWIGLU) return (a.O[0] + TILE_M - 1) / TILE_M;
@@ -996,25 +1082,42 @@ int fused_gemm_launch(TmaMaps *g, FusedEpi epi, const FusedGemmArgs &a, cudaStre
   p.spin = a.spin_limit ? a.spin_limit : SPIN_LIMIT;
   p.withhold = a.withhold ? 1 : 0;
   if (epi == EPI_SWIGLU && pl.nt == 256 && a.split == 0 && a.stages == 0) {
-    // wide rows: one CTA per (gate tile, up tile) pair sharing the activation tiles
-    constexpr int STAGE2 = 2 * A_BYTES + 256 * TILE_K * 2;
-    p.stages = std::max(2, std::min(SMEM_ONE / STAGE2, pl.KB));
+    // wide rows: one CTA per (gate tile, up tile) pair sharing the activation tiles; optionally two such CTAs as a
+    // CTA pair that also share the activation k-block (each loads half of the rows)
+    const bool duo2 = g_pairs_swiglu && (p.tiles0 % 2) == 0;
+    const int stage2 = 2 * A_BYTES + (duo2 ? 128 : 256) * TILE_K * 2;
+    if (duo2) {
+      const CUtensorMap *mxh = tma_maps_get(g, a.x, a.rows, a.I, 128);
+      if (!mxh) return -6;
+      p.map_x = *mxh;
+    }
+    p.stages = std::max(2, std::min(SMEM_ONE / stage2, pl.KB));
     p.S = 1; p.Sk = 1;
-    p.ctrl_off = (p.stages * STAGE2 + 1023) & ~1023;
+    p.ctrl_off = (p.stages * stage2 + 1023) & ~1023;
     const int smem = p.ctrl_off + 512 + 256 * 4 + 1024;
-    static SmemLimit limit;
-    if (!limit.ensure(gemm_swiglu_pair_kernel<256>, smem)) return -6;
+    static SmemLimit limit, limit_duo;
+    if (!(duo2 ? limit_duo.ensure(gemm_swiglu_pair_kernel<256, true>, smem) : limit.ensure(gemm_swiglu_pair_kernel<256>, smem))) return -6;
     if (!launch_allowed()) return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.tiles0, 1, 1);
     cfg.blockDim = dim3(128, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute at[2];
+    int na = 0;
+    if (duo2) {
+      at[na].id = cudaLaunchAttributeClusterDimension;
+      at[na].val.clusterDim.x = 2; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
+      na++;
+    }
+    if (a.pdl) {
+      at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      at[na].val.programmaticStreamSerializationAllowed = 1;
+      na++;
+    }
     cfg.attrs = at;
-    cfg.numAttrs = a.pdl ? 1 : 0;
+    cfg.numAttrs = na;
+    if (duo2) return cudaLaunchKernelEx(&cfg, gemm_swiglu_pair_kernel<256, true>, p) == cudaSuccess ? 0 : -6;
     return cudaLaunchKernelEx(&cfg, gemm_swiglu_pair_kernel<256>, p) == cudaSuccess ? 0 : -6;
   }
   if (duo) {

@@ -16,7 +16,7 @@ __global__ void __launch_bounds__(128) k(long long *out, int nt) {
   for (int i = threadIdx.x; i < 96 * 1024 / 4; i += 128) ((uint32_t *)tiles)[i] = 0;
   if (threadIdx.x == 0) { for (int i = 0; i < 8; i++) mbar_init(&bars[i], 1); asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(256) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -44,6 +44,9 @@ __global__ void __launch_bounds__(128) k(long long *out, int nt) {
     T0 for (int i = 0; i < IT; i++) { if (elect_one()) { umma_bf16(tm, da, db, idesc, 1u); umma_bf16(tm, da + 2, db + 2, idesc, 1u); umma_bf16(tm, da + 4, db + 4, idesc, 1u); umma_bf16(tm, da + 6, db + 6, idesc, 1u); } } T1   // 7 four MMAs
     T0 for (int i = 0; i < IT; i++) { if (elect_one()) { umma_bf16(tm, da, db, idesc, 1u); umma_bf16(tm, da + 2, db + 2, idesc, 1u); umma_bf16(tm, da + 4, db + 4, idesc, 1u); umma_bf16(tm, da + 6, db + 6, idesc, 1u); umma_commit(&bars[1 + (i & 3)]); } } T1   // 8 four MMAs + commit
     T0 for (int i = 0; i < IT; i++) { if (lane == 0) { umma_bf16(tm, da, db, idesc, 1u); umma_bf16(tm, da + 2, db + 2, idesc, 1u); umma_bf16(tm, da + 4, db + 4, idesc, 1u); umma_bf16(tm, da + 6, db + 6, idesc, 1u); umma_commit(&bars[1 + (i & 3)]); } } T1   // 9 the same from lane 0
+    {   // two accumulators side by side (gate and up of one feature tile), alternating: 8 MMAs + commit per k-block
+      T0 for (int i = 0; i < IT; i++) { if (elect_one()) { for (int j = 0; j < 4; j++) { umma_bf16(tm, da + 2 * j, db + 2 * j, idesc, 1u); umma_bf16(tm + nt, da + 2 * j + 512, db + 2 * j, idesc, 1u); } umma_commit(&bars[1 + (i & 3)]); } } T1
+    }
     T0 for (int i = 0; i < IT; i++) { if (elect_one()) mbar_expect_tx(&bars[5], 0); } T1       // 10 arrive.expect_tx
     // wait until every MMA has completed before freeing tensor memory
     if (elect_one()) umma_commit(&bars[6]);
@@ -53,13 +56,13 @@ __global__ void __launch_bounds__(128) k(long long *out, int nt) {
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(256) : "memory");
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(512) : "memory");
 }
 int main() {
   long long *d, h[16];
   cudaMalloc(&d, sizeof h);
   cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
-  const char *names[] = {"elect", "redux", "tcgen05.fence", "bounded wait(done)", "test_wait(done)", "commit", "1 mma", "4 mma", "4 mma+commit", "same, lane 0 branch", "arrive.expect_tx"};
+  const char *names[] = {"elect", "redux", "tcgen05.fence", "bounded wait(done)", "test_wait(done)", "commit", "1 mma", "4 mma", "4 mma+commit", "same, lane 0 branch", "8 mma, two accumulators + commit", "arrive.expect_tx"};
   for (int nt : {16, 64, 256}) {
     for (int rep = 0; rep < 2; rep++) {
       cudaMemset(d, 0, sizeof h);
@@ -69,7 +72,7 @@ int main() {
     }
     cudaMemcpy(h, d, sizeof h, cudaMemcpyDeviceToHost);
     printf("N=%d:", nt);
-    for (int i = 0; i < 11; i++) printf("  %s %.0f", names[i], (double)h[i] / IT);
+    for (int i = 0; i < 12; i++) printf("  %s %.0f", names[i], (double)h[i] / IT);
     printf("\n");
   }
   return 0;

@@ -608,13 +608,36 @@ def test_gemm_cta_pairs_bit_equal(rows, O, I, split):
     w = (torch.randn(O, I, generator=g) / I ** 0.5).to(torch.bfloat16).cuda()
     L = sb.lib()
     try:
-        assert L.spec_tune(None, sb.SpecDecoder.TUNE_GEMM_PAIRS, 1) == 0
+        assert L.spec_tune(None, sb.SpecDecoder.TUNE_GEMM_PAIRS, 3) == 0
         paired = sb.gemm_fused(x, w, split=split).clone()
-    finally:
         assert L.spec_tune(None, sb.SpecDecoder.TUNE_GEMM_PAIRS, 0) == 0
-    single = sb.gemm_fused(x, w, split=min(split, 4))
+        single = sb.gemm_fused(x, w, split=min(split, 4)).clone()
+    finally:
+        assert L.spec_tune(None, sb.SpecDecoder.TUNE_GEMM_PAIRS, 2) == 0     # the library's default
     if 1 <= split <= 4:                      # the same K split on both sides
         assert torch.equal(paired, single)
     ref = x.double() @ w.double().t()
     assert (paired.double() - ref).abs().max().item() < 1e-4 * I ** 0.5
     assert (single.double() - ref).abs().max().item() < 1e-4 * I ** 0.5
+
+
+@pytest.mark.parametrize("rows,F,I", [(256, 512, 512), (200, 1024, 4096), (129, 1792, 1024), (256, 384, 1024)])
+def test_gate_up_cta_pairs_bit_equal(rows, F, I):
+    """The 256-row gate/up kernel as CTA pairs (the default) against single CTAs: bit-identical activations, and both
+    within bf16 rounding of SiLU(x Wg^T) * (x Wu^T) computed in float64."""
+    g = torch.Generator().manual_seed(rows + F + I)
+    x = torch.randn(rows, I, generator=g).to(torch.bfloat16).cuda()
+    wg = (torch.randn(F, I, generator=g) / I ** 0.5).to(torch.bfloat16).cuda()
+    wu = (torch.randn(F, I, generator=g) / I ** 0.5).to(torch.bfloat16).cuda()
+    L = sb.lib()
+    try:
+        assert L.spec_tune(None, sb.SpecDecoder.TUNE_GEMM_PAIRS, 2) == 0
+        paired = sb.gemm_swiglu(x, wg, wu).clone()
+        assert L.spec_tune(None, sb.SpecDecoder.TUNE_GEMM_PAIRS, 0) == 0
+        single = sb.gemm_swiglu(x, wg, wu).clone()
+    finally:
+        assert L.spec_tune(None, sb.SpecDecoder.TUNE_GEMM_PAIRS, 2) == 0
+    assert torch.equal(paired, single)
+    gd, ud = x.double() @ wg.double().t(), x.double() @ wu.double().t()
+    ref = torch.nn.functional.silu(gd) * ud
+    assert ((paired.double() - ref).abs() <= 2.0 ** -8 * ref.abs() + 1e-3).all()
