@@ -123,8 +123,14 @@ __device__ __forceinline__ float4 sum_peers4(uint32_t local_addr, int s0, int n,
 // of its own tile.  At 256 rows the activation k-block (32 KB) is twice a weight tile, so the shared-memory fill traffic
 // per weight byte drops from 3 x to 2 x, which is what bounds the loop at this width.  The cluster is (2, S): x = the
 // pair, y = the K slices; the reduction runs over the members with the same x.
+// Threads per CTA: 128 (thread = output feature in the epilogue); the 256-row tiles with a row-wise epilogue run 256, so
+// that two threads share a feature and split the tile's columns / rows between them (the epilogue of a 256-row tile is
+// as long as its main loop).
+constexpr int fused_threads(int nt, int epi) { return (nt == 256 && (epi == EPI_F32 || epi == EPI_RESID || epi == EPI_QKV)) ? 256 : 128; }
+
 template <int NT, int EPI, bool PAIR = false, bool DUO = false>
-__global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__ FusedParams p) {
+__global__ void __launch_bounds__(fused_threads(NT, EPI)) gemm_fused_kernel(const __grid_constant__ FusedParams p) {
+  constexpr int THREADS = fused_threads(NT, EPI), NH = THREADS / 128;
   static_assert(!PAIR || EPI == EPI_SWIGLU, "two weight tiles per CTA exist for the gate/up epilogue only");
   static_assert(!DUO || (NT == 256 && !PAIR && (EPI == EPI_F32 || EPI == EPI_RESID || EPI == EPI_QKV)), "CTA pairs serve the 256-row tiles");
   constexpr int A_TILES = PAIR ? 2 : 1;
@@ -328,7 +334,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       if (elect_one()) umma_commit(acc_bar);           // accumulator complete
     } else if (warp >= 2) {
       // ---- per-row scale of the input: rsqrt(mean square + eps) from the producer kernel's per-tile sums
-      for (int r = threadIdx.x - 64; r < p.rows; r += 64) {
+      for (int r = threadIdx.x - 64; r < p.rows; r += THREADS - 64) {
         float sc = 1.0f;
         if (p.ssq_in) {
           float ss = 0.0f;
@@ -357,20 +363,21 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
   float *red = (float *)tiles;                       // [CH][128]
   float *red_u = red + CH * TILE_M;                  // PAIR: the up accumulator, [CH][128]
   float *sumb = red + A_TILES * CH * TILE_M;         // [rows of this CTA][128] (EPI_SWIGLU: gate rows, then up rows at CH/2)
-  const int f = threadIdx.x;
+  const int f = threadIdx.x & (TILE_M - 1);          // feature of the tile = tensor-memory lane (a warp reads lanes 32 (warp % 4) ..)
+  const int hw = threadIdx.x >> 7;                   // 0, or with 256 threads which half of the columns / rows
   const int o = tm * TILE_M + f;                     // output feature within weight mi
   for (int c0 = 0; c0 < p.rows; c0 += CH) {
     const int nrow = (p.rows - c0 < CH) ? p.rows - c0 : CH;
     if (good) {
 #pragma unroll 1
-      for (int cc = 0; cc < CH && c0 + cc < NT; cc += 16) {
+      for (int cc = hw * (CH / NH); cc < (hw + 1) * (CH / NH) && c0 + cc < NT; cc += 16) {
         if (cc >= nrow) break;
         uint32_t v[16];
-        tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c0 + cc), v);
+        tmem_ld16(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(c0 + cc), v);
 #pragma unroll
         for (int j = 0; j < 16; j++) red[(cc + j) * TILE_M + f] = __uint_as_float(v[j]);
         if (PAIR) {
-          tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(NT + c0 + cc), v);
+          tmem_ld16(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(NT + c0 + cc), v);
 #pragma unroll
           for (int j = 0; j < 16; j++) red_u[(cc + j) * TILE_M + f] = __uint_as_float(v[j]);
         }
@@ -386,7 +393,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
     const float *src_u = red_u + r0 * TILE_M;          // EPI_SWIGLU: the up values of the same rows
     if (S > 1) {
       const int nitems = (r1 - r0) * 32;
-      for (int item = threadIdx.x; item < nitems; item += 128) {
+      for (int item = threadIdx.x; item < nitems; item += THREADS) {
         const int i = item >> 5, qd = item & 31;
         const uint32_t la = smem_u32(&red[(r0 + i) * TILE_M + qd * 4]);
         *(float4 *)&sumb[i * TILE_M + qd * 4] = DUO ? sum_peers4(la, xr, Sk, 2) : sum_peers4(la, 0, Sk);
@@ -407,12 +414,12 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
     // a chain of dependent L2 round trips.
     constexpr int RB = 8;
     if (EPI == EPI_F32) {
-      for (int r = r0; r < r1; r++)
+      for (int r = r0 + hw; r < r1; r += NH)
         if (good && o < p.O[0]) p.out_f32[(size_t)(c0 + r) * p.ldo + o] = src[(r - r0) * TILE_M + f] * inv_s[c0 + r];
     } else if (EPI == EPI_RESID) {
       const bool act_o = good && o < p.O[0];
       const float gn = act_o ? __bfloat162float(p.gain[o]) : 0.0f;
-      for (int rb = r0; rb < r1; rb += RB) {
+      for (int rb = r0 + hw * RB; rb < r1; rb += NH * RB) {
         float xin[RB];
 #pragma unroll
         for (int j = 0; j < RB; j++)
@@ -436,13 +443,13 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
             }
             float sq = xo * xo;
             for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
-            if (lane == 0) wpart[warp * CH + (r - r0)] = sq;
+            if (lane == 0) wpart[(warp & 3) * CH + (r - r0)] = sq;
           }
         }
       }
       __syncthreads();
       if (good)
-        for (int t = threadIdx.x; t < r1 - r0; t += 128)
+        for (int t = threadIdx.x; t < r1 - r0; t += THREADS)
           p.ssq_out[(size_t)tm * p.ssq_ld + c0 + r0 + t] = ((wpart[t] + wpart[CH + t]) + wpart[2 * CH + t]) + wpart[3 * CH + t];
     } else if (EPI == EPI_QKV) {
       const int hd = p.hd, half = hd >> 1;
@@ -452,7 +459,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
       // per-row cache slot of this CTA's rows: one thread per row resolves sequence -> position -> page
       int32_t *slot_s = (int32_t *)wpart;              // [CH] element offset / hd of the row's K/V slot, -1: none
       int32_t *seq_s = slot_s + CH;                    // [CH]
-      for (int t = threadIdx.x; t < r1 - r0; t += 128) {
+      for (int t = threadIdx.x; t < r1 - r0; t += THREADS) {
         const int row = c0 + r0 + t;
         const int seq = p.m.seq[row];
         int slot = -1;
@@ -470,7 +477,7 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
         seq_s[t] = seq;
       }
       __syncthreads();
-      for (int rb = r0; rb < r1; rb += RB) {
+      for (int rb = r0 + hw * RB; rb < r1; rb += NH * RB) {
         float2 cs[RB];
 #pragma unroll
         for (int j = 0; j < RB; j++)
@@ -617,8 +624,11 @@ __global__ void __launch_bounds__(128) gemm_fused_kernel(const __grid_constant__
 // DUO: two neighbouring feature tiles as a CTA pair (cta_group::2, cluster of 2): each CTA streams its own gate and up
 // tile and HALF of the activation rows, the even CTA issues one M = 256 MMA per accumulator and k-step (fill bytes per
 // k-block 48 KB instead of 64 KB per CTA, four stages instead of three).
+// PAIR_THREADS threads: several threads share a feature (tensor-memory lane) and split the rows in the epilogue, which
+// converts 2 x 256 accumulator columns per feature (with 128 threads it took a quarter of the launch).
+constexpr int PAIR_THREADS = 512, PAIR_GROUPS = PAIR_THREADS / 128;
 template <int NT, bool DUO = false>
-__global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_constant__ FusedParams p) {
+__global__ void __launch_bounds__(PAIR_THREADS) gemm_swiglu_pair_kernel(const __grid_constant__ FusedParams p) {
   constexpr int B_BYTES = (DUO ? NT / 2 : NT) * TILE_K * 2;
   constexpr int STAGE = 2 * A_BYTES + B_BYTES;
   constexpr int TMEM_COLS = 2 * NT;
@@ -800,7 +810,7 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
       __syncwarp();
       if (elect_one()) umma_commit(acc_bar);
     } else if (warp >= 2) {
-      for (int r = threadIdx.x - 64; r < p.rows; r += 64) {
+      for (int r = threadIdx.x - 64; r < p.rows; r += PAIR_THREADS - 64) {
         float sc = 1.0f;
         if (p.ssq_in) {
           float ss = 0.0f;
@@ -823,13 +833,14 @@ __global__ void __launch_bounds__(128) gemm_swiglu_pair_kernel(const __grid_cons
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
   // ---- epilogue: thread = feature f (tensor-memory lane), 16 rows (columns) of both accumulators at a time
-  const int o = tm * TILE_M + threadIdx.x;
+  const int o = tm * TILE_M + (threadIdx.x & (TILE_M - 1));
+  const int hw = threadIdx.x >> 7;               // which share of the rows (accumulator columns) this thread converts
   if (good) {
 #pragma unroll 1
-    for (int cc = 0; cc < p.rows; cc += 16) {
+    for (int cc = hw * (NT / PAIR_GROUPS); cc < p.rows && cc < (hw + 1) * (NT / PAIR_GROUPS); cc += 16) {
       uint32_t g[16], u[16];
-      tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)cc, g);
-      tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(NT + cc), u);
+      tmem_ld16(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)cc, g);
+      tmem_ld16(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(NT + cc), u);
       if (o < p.O[0]) {
 #pragma unroll
         for (int j = 0; j < 16; j++) {
@@ -944,7 +955,7 @@ int launch_inst(const FusedParams &p, const Plan &pl, bool pdl, cudaStream_t s) 
   if (!launch_allowed()) return 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(pl.tiles, pl.S, 1);
-  cfg.blockDim = dim3(128, 1, 1);
+  cfg.blockDim = dim3(fused_threads(NT, EPI), 1, 1);
   cfg.dynamicSmemBytes = pl.smem;
   cfg.stream = s;
   cudaLaunchAttribute at[2];
@@ -972,7 +983,7 @@ int resident_clusters_inst(const Plan &pl) {
   if (cudaFuncSetAttribute(gemm_fused_kernel<NT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.smem) != cudaSuccess) return 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(pl.tiles, pl.S, 1);
-  cfg.blockDim = dim3(128, 1, 1);
+  cfg.blockDim = dim3(fused_threads(NT, EPI), 1, 1);
   cfg.dynamicSmemBytes = pl.smem;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
@@ -1100,7 +1111,7 @@ int fused_gemm_launch(TmaMaps *g, FusedEpi epi, const FusedGemmArgs &a, cudaStre
     if (!launch_allowed()) return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.tiles0, 1, 1);
-    cfg.blockDim = dim3(128, 1, 1);
+    cfg.blockDim = dim3(PAIR_THREADS, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute at[2];
