@@ -7,7 +7,9 @@
 //
 //  * swap-AB mapping: the weight tile (128 output features x 64 k, K-major, 128-byte swizzle) is the
 //    UMMA M side, the token rows the N side (NT = 16/64/128/256), the fp32 accumulator sits in TMEM;
-//  * warp 0 streams tiles with TMA through a ring of shared-memory stages, warp 1 issues tcgen05.mma;
+//  * warp 0 streams tiles with TMA through a ring of shared-memory stages, warp 1 issues tcgen05.mma; both walk their
+//    loops as converged warps and one lane chosen by elect.sync issues (the issuing warp, not shared memory or HBM,
+//    is what limits a single CTA: see ubench/issue_loop.cu);
 //  * split-K: the S slices of one feature tile form a thread-block cluster.  Each CTA parks its
 //    accumulator in its own shared memory and every CTA reduces a share of the rows by reading its
 //    peers' copies through distributed shared memory, in slice order (deterministic, no atomics, no
