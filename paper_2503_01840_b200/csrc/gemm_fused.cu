@@ -278,7 +278,7 @@ __global__ void __launch_bounds__(fused_threads(NT, EPI)) gemm_fused_kernel(cons
       // ---- MMA issuer of a CTA pair (even CTA only): M = 256 over both CTAs' weight tiles, N = both activation halves
       if (xr == 0) {
         constexpr uint32_t idesc = umma_idesc_m(NT, 2 * TILE_M);
-        const uint16_t pair_mask = (uint16_t)(3u << crank);       // this CTA and its partner
+        const uint32_t pair_lead = crank;                        // this (even) CTA and its partner crank + 1
         const uint32_t partner_base = ld_peer_u32(smem_u32(tmem_slot), crank | 1u);
         if (partner_base != tmem_base) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 233, blockIdx.x, (int)partner_base); }
         const uint64_t desc0 = umma_desc_sw128(smem_u32(tiles));
@@ -295,7 +295,7 @@ __global__ void __launch_bounds__(fused_threads(NT, EPI)) gemm_fused_kernel(cons
             if (elect_one()) {
 #pragma unroll
               for (int j = 0; j < TILE_K / UMMA_K; j++) umma_bf16_pair(tmem_base, da + 2 * j, da + (A_BYTES >> 4) + 2 * j, idesc, (i | j) ? 1u : 0u);
-              umma_commit_pair(&empty[st], pair_mask);      // frees the stage in both CTAs
+              umma_commit_pair(&empty[st], pair_lead);      // frees the stage in both CTAs
             }
             __syncwarp();
             ready = mbar_test(&full[nst], nph) ? 1u : 0u;
@@ -303,7 +303,7 @@ __global__ void __launch_bounds__(fused_threads(NT, EPI)) gemm_fused_kernel(cons
           }
         if (lane == 0) *n_consumed = i;
         __syncwarp();
-        if (!*abort_flag && elect_one()) umma_commit_pair(acc_bar, pair_mask);   // both accumulators complete
+        if (!*abort_flag && elect_one()) umma_commit_pair(acc_bar, pair_lead);   // both accumulators complete
       }
     } else if (!DUO && warp == 1) {
       // ---- MMA issuer warp (all lanes walk the loop, the elected lane issues)
@@ -773,7 +773,7 @@ __global__ void __launch_bounds__(PAIR_THREADS) gemm_swiglu_pair_kernel(const __
                 umma_bf16_pair(tmem_base, dg + 2 * j, db + 2 * j, idesc, (i | j) ? 1u : 0u);
                 umma_bf16_pair(tmem_base + NT, du + 2 * j, db + 2 * j, idesc, (i | j) ? 1u : 0u);
               }
-              umma_commit_pair(&empty[st], (uint16_t)3);
+              umma_commit_pair(&empty[st], 0u);
             }
             __syncwarp();
             ready = mbar_test(&full[nst], nph) ? 1u : 0u;
@@ -781,7 +781,7 @@ __global__ void __launch_bounds__(PAIR_THREADS) gemm_swiglu_pair_kernel(const __
           }
         if (lane == 0) *n_consumed = i;
         __syncwarp();
-        if (!*abort_flag && elect_one()) umma_commit_pair(acc_bar, (uint16_t)3);
+        if (!*abort_flag && elect_one()) umma_commit_pair(acc_bar, 0u);
       }
     } else if (!DUO && warp == 1) {
       // ---- MMA issuer warp (the elected lane issues): gate accumulator at column 0, up accumulator at column NT

@@ -138,11 +138,12 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t da, uin
       "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// arrives (once the pair's MMAs issued so far have completed) on the mbarrier at this offset in every CTA of cta_mask
-__device__ __forceinline__ void umma_commit_pair(uint64_t *bar, uint16_t cta_mask) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(smem_u32(bar)),
-               "h"(cta_mask)
-               : "memory");
+// arrives (once the pair's MMAs issued so far have completed) on the mbarrier at this offset in BOTH CTAs of the pair
+// whose even member has cluster rank `lead`: one commit per CTA, each addressed through the cluster window
+__device__ __forceinline__ void umma_commit_pair(uint64_t *bar, uint32_t lead) {
+  const uint32_t local = smem_u32(bar);
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mapa_u32(local, lead)) : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mapa_u32(local, lead + 1u)) : "memory");
 }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
