@@ -88,3 +88,19 @@ def test_c2_full_depth_steps_vs_oracle():
     assert st.steps == 2
     _assert_everything_compared(st, cfg)
     assert st.decisions_forced >= 200 and st.argmax_forced >= 60 and st.accept_checked == 2, st
+
+
+def test_c3_shape_with_split_k_cta_pairs_vs_oracle():
+    """The same batch-64 steps with the 256-row split-K GEMMs (QKV with RoPE and KV write, O and down with residual and
+    norm statistics) ALSO running as CTA pairs (an optional mode; the gate/up kernel runs as pairs by default): the whole
+    step is compared with the 64 oracles exactly as above."""
+    L = sb.lib()
+    cfg = synth.C3.truncated(2, prompt_lo=16, prompt_hi=64)
+    try:
+        assert L.spec_tune(None, sb.SpecDecoder.TUNE_GEMM_PAIRS, 3) == 0
+        st, _, prompts = _run(cfg, 2, page_shuffle_seed=13, greedy_check=False)
+    finally:
+        assert L.spec_tune(None, sb.SpecDecoder.TUNE_GEMM_PAIRS, 2) == 0      # the library's default
+    assert len(prompts) == 64 and st.steps == 2
+    _assert_everything_compared(st, cfg, sequences=64)
+    assert st.decisions_forced >= 64 * 4 and st.argmax_forced >= 64 * 4 and st.accept_checked == 128, st
