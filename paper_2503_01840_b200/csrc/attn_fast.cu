@@ -318,6 +318,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
   }
   return false;
 }
+// the same for a converged warp (all 32 lanes call it): one lane's sight of the completed phase counts for all, so that
+// no lane leaves its loop alone and strands the warp's next elect.sync
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity) {
+  const bool ok = mbar_wait(bar, parity);
+  const bool any = __any_sync(0xffffffffu, ok);
+  if (any && !ok) mbar_wait(bar, parity);      // completed: returns at its first test, with this lane's own acquire
+  return any;
+}
 __device__ __forceinline__ void tma_load_3d(void *smem_dst, const CUtensorMap *map, int c0, int c1, int c2, uint64_t *bar) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(
@@ -405,8 +413,8 @@ __global__ void __launch_bounds__(288) attn_tma_kernel(const __grid_constant__ C
       for (int t = t_begin; t < t_end; t++) {
         const int i = t - t_begin, st = i % STAGES;
         if (t + 1 < t_end) tile_pages(nxt, tbl, p.pm.pages_per_seq, t + 1, ps);
-        if (i == STAGES - 1 && !mbar_wait(q_bar, 0)) { if (status) set_status(status, ST_TIMEOUT, 400, blockIdx.z, t); break; }
-        if (i >= STAGES && !mbar_wait(&empty[st], (uint32_t)(((i / STAGES) - 1) & 1))) { if (status) set_status(status, ST_TIMEOUT, 401, blockIdx.z, t); break; }
+        if (i == STAGES - 1 && !mbar_wait_warp(q_bar, 0)) { if (status) set_status(status, ST_TIMEOUT, 400, blockIdx.z, t); break; }
+        if (i >= STAGES && !mbar_wait_warp(&empty[st], (uint32_t)(((i / STAGES) - 1) & 1))) { if (status) set_status(status, ST_TIMEOUT, 401, blockIdx.z, t); break; }
         if (elect_one()) {
           unsigned char *kb = sm + st * 2 * TILEB, *vb = kb + TILEB;
           mbar_expect_tx(&full[st], 2 * TILEB);
@@ -719,7 +727,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
       for (int i = 0; i < ntl; i++) {
         const int t = t_begin + i, st = i % UM_STAGES;
         if (i + 1 < ntl) tile_pages(nxt, tbl, p.pm.pages_per_seq, t + 1, ps);
-        if (i >= UM_STAGES && !mbar_wait(&empty[st], (uint32_t)(((i / UM_STAGES) - 1) & 1))) {
+        if (i >= UM_STAGES && !mbar_wait_warp(&empty[st], (uint32_t)(((i / UM_STAGES) - 1) & 1))) {
           *abort_flag = 1;
           if (status) set_status(status, ST_TIMEOUT, 420, blockIdx.z, t);
           break;
@@ -768,7 +776,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
       };
       bool ok = true;
       for (int i = 0; i < 2 && i < ntl && ok; i++) {
-        ok = mbar_wait(&full[i % UM_STAGES], 0);
+        ok = mbar_wait_warp(&full[i % UM_STAGES], 0);
         if (!ok) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 421, blockIdx.z, t_begin + i); break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (elect_one()) issue_s(i);
@@ -777,7 +785,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
       if (ok) {
         for (int i = 0; i < ntl; i++) {
           const int st = i % UM_STAGES;
-          if (!mbar_wait(&p_bar[i & 1], (uint32_t)((i >> 1) & 1))) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 422, blockIdx.z, t_begin + i); break; }
+          if (!mbar_wait_warp(&p_bar[i & 1], (uint32_t)((i >> 1) & 1))) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 422, blockIdx.z, t_begin + i); break; }
           if (*abort_flag) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t v_addr = smem_u32(ring + st * 2 * UM_TILE + UM_TILE);
@@ -792,7 +800,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1) attn_umma_kernel(const __grid_c
           __syncwarp();
           if (i + 2 < ntl) {          // this group's score buffer is free: its threads read it before they arrived on p_bar
             const int st2 = (i + 2) % UM_STAGES;
-            if (!mbar_wait(&full[st2], (uint32_t)(((i + 2) / UM_STAGES) & 1))) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 423, blockIdx.z, t_begin + i + 2); break; }
+            if (!mbar_wait_warp(&full[st2], (uint32_t)(((i + 2) / UM_STAGES) & 1))) { *abort_flag = 1; if (status) set_status(status, ST_TIMEOUT, 423, blockIdx.z, t_begin + i + 2); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (elect_one()) issue_s(i + 2);
             __syncwarp();
@@ -1002,7 +1010,7 @@ __global__ void __launch_bounds__(160) attn_tma_small_kernel(const __grid_consta
       for (int t = t_begin; t < t_end; t++) {
         const int i = t - t_begin, st = i % STAGES;
         if (t + 1 < t_end) tile_pages(nxt, tbl, p.pm.pages_per_seq, t + 1, ps);
-        if (i >= STAGES && !mbar_wait(&empty[st], (uint32_t)(((i / STAGES) - 1) & 1))) { if (status) set_status(status, ST_TIMEOUT, 411, blockIdx.z, t); break; }
+        if (i >= STAGES && !mbar_wait_warp(&empty[st], (uint32_t)(((i / STAGES) - 1) & 1))) { if (status) set_status(status, ST_TIMEOUT, 411, blockIdx.z, t); break; }
         if (elect_one()) {
           unsigned char *kb = sm + st * 2 * TILEB, *vb = kb + TILEB;
           mbar_expect_tx(&full[st], 2 * TILEB);

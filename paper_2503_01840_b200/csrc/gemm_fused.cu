@@ -224,7 +224,7 @@ __global__ void __launch_bounds__(fused_threads(NT, EPI)) gemm_fused_kernel(cons
     int i = npre, st = 0;
     uint32_t ph = 0;
     for (; i < nkb; i++) {
-      if (!mbar_wait(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 230, blockIdx.x, i); break; }
+      if (!mbar_wait_warp(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 230, blockIdx.x, i); break; }
       if (elect_one()) {
         unsigned char *a = tiles + st * STAGE;
         const uint32_t fb = mapa_u32(smem_u32(&full[st]), lead);
@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(fused_threads(NT, EPI)) gemm_fused_kernel(cons
     int i = npre, st = 0;             // the loop runs only when the prefill used every stage: it restarts at stage 0
     uint32_t ph = 0;
     for (; i < nkb; i++) {
-      if (!mbar_wait(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
+      if (!mbar_wait_warp(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 200, blockIdx.x, i); break; }
       if (elect_one()) {
         unsigned char *a = tiles + st * STAGE;
         mbar_expect_tx(&full[st], STAGE);
@@ -286,7 +286,7 @@ __global__ void __launch_bounds__(fused_threads(NT, EPI)) gemm_fused_kernel(cons
         uint32_t ph = 0, ready = 0;
         if (!*abort_flag)
           for (; i < nkb; i++) {
-            if (!ready && !mbar_wait(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 231, blockIdx.x, i); break; }
+            if (!ready && !mbar_wait_warp(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 231, blockIdx.x, i); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t da = desc0 + (uint64_t)((st * STAGE) >> 4);
             int nst = st + 1;
@@ -298,7 +298,7 @@ __global__ void __launch_bounds__(fused_threads(NT, EPI)) gemm_fused_kernel(cons
               umma_commit_pair(&empty[st], pair_lead);      // frees the stage in both CTAs
             }
             __syncwarp();
-            ready = mbar_test(&full[nst], nph) ? 1u : 0u;
+            ready = mbar_test_warp(&full[nst], nph) ? 1u : 0u;
             st = nst; ph = nph;
           }
         if (lane == 0) *n_consumed = i;
@@ -314,7 +314,7 @@ __global__ void __launch_bounds__(fused_threads(NT, EPI)) gemm_fused_kernel(cons
       int i = 0, st = 0;
       uint32_t ph = 0, ready = 0;
       for (; i < nkb; i++) {
-        if (!ready && !mbar_wait(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 201, blockIdx.x, i); break; }
+        if (!ready && !mbar_wait_warp(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 201, blockIdx.x, i); break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint64_t da = desc0 + (uint64_t)((st * STAGE) >> 4), db = da + (uint64_t)((A_TILES * A_BYTES) >> 4);
         int nst = st + 1;
@@ -329,7 +329,7 @@ __global__ void __launch_bounds__(fused_threads(NT, EPI)) gemm_fused_kernel(cons
           umma_commit(&empty[st]);      // frees the stage once these MMAs have read it
         }
         __syncwarp();
-        ready = mbar_test(&full[nst], nph) ? 1u : 0u;      // a cheap look at the next stage: mostly spares the wait
+        ready = mbar_test_warp(&full[nst], nph) ? 1u : 0u;      // a cheap look at the next stage: mostly spares the wait
         st = nst; ph = nph;
       }
       if (lane == 0) *n_consumed = i;
@@ -702,7 +702,7 @@ __global__ void __launch_bounds__(PAIR_THREADS) gemm_swiglu_pair_kernel(const __
     int i = npre, st = 0;
     uint32_t ph = 0;
     for (; i < KB; i++) {
-      if (!mbar_wait(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 225, blockIdx.x, i); break; }
+      if (!mbar_wait_warp(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 225, blockIdx.x, i); break; }
       if (elect_one()) {
         unsigned char *a = tiles + st * STAGE;
         const uint32_t fb = mapa_u32(smem_u32(&full[st]), 0u);
@@ -736,7 +736,7 @@ __global__ void __launch_bounds__(PAIR_THREADS) gemm_swiglu_pair_kernel(const __
     int i = npre, st = 0;
     uint32_t ph = 0;
     for (; i < KB; i++) {
-      if (!mbar_wait(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 220, blockIdx.x, i); break; }
+      if (!mbar_wait_warp(&empty[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 220, blockIdx.x, i); break; }
       if (elect_one()) {
         unsigned char *a = tiles + st * STAGE;
         mbar_expect_tx(&full[st], STAGE);
@@ -761,7 +761,7 @@ __global__ void __launch_bounds__(PAIR_THREADS) gemm_swiglu_pair_kernel(const __
         uint32_t ph = 0, ready = 0;
         if (!*abort_flag)
           for (; i < KB; i++) {
-            if (!ready && !mbar_wait(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 227, blockIdx.x, i); break; }
+            if (!ready && !mbar_wait_warp(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 227, blockIdx.x, i); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t dg = desc0 + (uint64_t)((st * STAGE) >> 4), du = dg + (A_BYTES >> 4), db = dg + ((2 * A_BYTES) >> 4);
             int nst = st + 1;
@@ -776,7 +776,7 @@ __global__ void __launch_bounds__(PAIR_THREADS) gemm_swiglu_pair_kernel(const __
               umma_commit_pair(&empty[st], 0u);
             }
             __syncwarp();
-            ready = mbar_test(&full[nst], nph) ? 1u : 0u;
+            ready = mbar_test_warp(&full[nst], nph) ? 1u : 0u;
             st = nst; ph = nph;
           }
         if (lane == 0) *n_consumed = i;
@@ -790,7 +790,7 @@ __global__ void __launch_bounds__(PAIR_THREADS) gemm_swiglu_pair_kernel(const __
       int i = 0, st = 0;
       uint32_t ph = 0, ready = 0;
       for (; i < KB; i++) {
-        if (!ready && !mbar_wait(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 221, blockIdx.x, i); break; }
+        if (!ready && !mbar_wait_warp(&full[st], ph, p.spin)) { *abort_flag = 1; set_status(p.status, ST_TIMEOUT, 221, blockIdx.x, i); break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint64_t dg = desc0 + (uint64_t)((st * STAGE) >> 4), du = dg + (A_BYTES >> 4), db = dg + ((2 * A_BYTES) >> 4);
         int nst = st + 1;
@@ -805,7 +805,7 @@ __global__ void __launch_bounds__(PAIR_THREADS) gemm_swiglu_pair_kernel(const __
           umma_commit(&empty[st]);
         }
         __syncwarp();
-        ready = mbar_test(&full[nst], nph) ? 1u : 0u;
+        ready = mbar_test_warp(&full[nst], nph) ? 1u : 0u;
         st = nst; ph = nph;
       }
       if (lane == 0) *n_consumed = i;

@@ -57,6 +57,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint32
   }
   return false;
 }
+// The same wait for a CONVERGED warp (all 32 lanes call it): every lane gets the same answer.  A phase that one lane saw
+// complete is complete, so that lane's answer counts for all; without this a lane that ran out of polls while another saw
+// the phase flip would leave the loop alone and the warp's next elect.sync would wait for it for ever.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, uint32_t limit = SPIN_LIMIT) {
+  const bool ok = mbar_wait(bar, parity, limit);
+  const bool any = __any_sync(0xffffffffu, ok);
+  if (any && !ok) mbar_test(bar, parity);      // this lane's own (acquiring) look at the completed phase
+  return any;
+}
+// non-blocking look by a converged warp: true only when every lane saw the phase complete
+__device__ __forceinline__ bool mbar_test_warp(uint64_t *bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_test(bar, parity)); }
 __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
